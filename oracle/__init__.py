@@ -1,0 +1,167 @@
+"""ctypes front end of the CPU oracle (``oracle.c``).
+
+TEST INFRASTRUCTURE ONLY.  The oracle evaluates each contraction chain as its unfused
+Einsum definition over COO input with fp64 accumulation (Table of kernels, Section 6 of
+the paper); the product code never imports this package.  ``liboracle.so`` is compiled
+from ``oracle.c`` by :func:`build` (plain ``gcc -O2 -fopenmp``).
+"""
+import ctypes
+import os
+import subprocess
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "oracle.c")
+_LIB = os.path.join(_HERE, "liboracle.so")
+_lib = None
+
+
+def build(force=False):
+    """Compile oracle.c into liboracle.so if missing or older than the source."""
+    if not force and os.path.exists(_LIB) and os.path.getmtime(_LIB) >= os.path.getmtime(_SRC):
+        return _LIB
+    tmp = _LIB + ".tmp%d" % os.getpid()
+    subprocess.check_call(["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c11", "-o", tmp, _SRC, "-lm"])
+    os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        build()
+        _lib = ctypes.CDLL(_LIB)
+        _lib.oracle_max_threads.restype = ctypes.c_int
+    return _lib
+
+
+def max_threads():
+    return int(_load().oracle_max_threads())
+
+
+_i64 = ctypes.c_int64
+_p = ctypes.c_void_p
+
+
+def _f32(a):
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    return a, a.ctypes.data_as(_p)
+
+
+def _coords(coords, order):
+    c = np.ascontiguousarray(coords, dtype=np.int32)
+    assert c.ndim == 2 and c.shape[1] == order
+    return c, c.ctypes.data_as(_p)
+
+
+def _sel(sel, I):
+    if sel is None:
+        return None, None, 0, I
+    s = np.ascontiguousarray(sel, dtype=np.int64)
+    assert len(set(s.tolist())) == s.shape[0], "selected slices must be distinct"
+    return s, s.ctypes.data_as(_p), s.shape[0], s.shape[0]
+
+
+def _check(rc):
+    if rc == -2:
+        raise ValueError("oracle: coordinate or selection out of range")
+    if rc != 0:
+        raise MemoryError("oracle: allocation failed")
+
+
+def spttm_ttm3(coords, vals, dims, C, D, sel=None, with_abs=True, threads=0):
+    """A(i,l,m) = sum_{j,k} B(i,j,k) C(j,l) D(k,m).  Returns (A, S) as float64."""
+    I, J, K = (int(d) for d in dims)
+    c, cp = _coords(coords, 3)
+    v, vp = _f32(vals)
+    C, Cp = _f32(C)
+    D, Dp = _f32(D)
+    assert C.shape[0] == J and D.shape[0] == K
+    L, M = C.shape[1], D.shape[1]
+    s, sp, n_sel, n_out = _sel(sel, I)
+    A = np.empty((n_out, L, M), dtype=np.float64)
+    S = np.empty_like(A) if with_abs else None
+    rc = _load().oracle_spttm_ttm3(_i64(v.shape[0]), cp, vp, _i64(I), _i64(J), _i64(K), _i64(L), _i64(M),
+                                   Cp, Dp, _i64(n_sel), sp, A.ctypes.data_as(_p),
+                                   S.ctypes.data_as(_p) if with_abs else None, ctypes.c_int(threads))
+    _check(rc)
+    return A, S
+
+
+def spttm_ttm4(coords, vals, dims, C, D, E, sel=None, with_abs=True, threads=0):
+    """A(i,l,m,n) = sum_{j,k,o} B(i,j,k,o) C(j,l) D(k,m) E(o,n).  Returns (A, S)."""
+    I, J, K, O = (int(d) for d in dims)
+    c, cp = _coords(coords, 4)
+    v, vp = _f32(vals)
+    C, Cp = _f32(C)
+    D, Dp = _f32(D)
+    E, Ep = _f32(E)
+    assert C.shape[0] == J and D.shape[0] == K and E.shape[0] == O
+    L, M, N = C.shape[1], D.shape[1], E.shape[1]
+    s, sp, n_sel, n_out = _sel(sel, I)
+    A = np.empty((n_out, L, M, N), dtype=np.float64)
+    S = np.empty_like(A) if with_abs else None
+    rc = _load().oracle_spttm_ttm4(_i64(v.shape[0]), cp, vp, _i64(I), _i64(J), _i64(K), _i64(O),
+                                   _i64(L), _i64(M), _i64(N), Cp, Dp, Ep, _i64(n_sel), sp,
+                                   A.ctypes.data_as(_p), S.ctypes.data_as(_p) if with_abs else None,
+                                   ctypes.c_int(threads))
+    _check(rc)
+    return A, S
+
+
+def sddmm_spmm(coords, vals, dims, C, D, E, sel=None, with_abs=True, with_sampled=False, threads=0):
+    """A(i,l) = sum_{j,k} B(i,j) C(i,k) D(j,k) E(j,l).  Returns (A, S, P).
+
+    P (if requested) holds, per stored nonzero in input order, the sampled value
+    B(i,j) * sum_k C(i,k) D(j,k); entries of rows outside ``sel`` are NaN.
+    """
+    I, J = (int(d) for d in dims)
+    c, cp = _coords(coords, 2)
+    v, vp = _f32(vals)
+    C, Cp = _f32(C)
+    D, Dp = _f32(D)
+    E, Ep = _f32(E)
+    assert C.shape[0] == I and D.shape[0] == J and E.shape[0] == J and C.shape[1] == D.shape[1]
+    K, L = C.shape[1], E.shape[1]
+    s, sp, n_sel, n_out = _sel(sel, I)
+    A = np.empty((n_out, L), dtype=np.float64)
+    S = np.empty_like(A) if with_abs else None
+    P = np.full(v.shape[0], np.nan, dtype=np.float64) if with_sampled else None
+    rc = _load().oracle_sddmm_spmm(_i64(v.shape[0]), cp, vp, _i64(I), _i64(J), _i64(K), _i64(L),
+                                   Cp, Dp, Ep, _i64(n_sel), sp, A.ctypes.data_as(_p),
+                                   S.ctypes.data_as(_p) if with_abs else None,
+                                   P.ctypes.data_as(_p) if with_sampled else None, ctypes.c_int(threads))
+    _check(rc)
+    return A, S, P
+
+
+def spmm_gemm(coords, vals, dims, C, D, sel=None, with_abs=True, threads=0):
+    """A(i,m) = sum_{j,l} B(i,j) C(j,l) D(l,m).  Returns (A, S)."""
+    I, J = (int(d) for d in dims)
+    c, cp = _coords(coords, 2)
+    v, vp = _f32(vals)
+    C, Cp = _f32(C)
+    D, Dp = _f32(D)
+    assert C.shape[0] == J and D.shape[0] == C.shape[1]
+    L, M = C.shape[1], D.shape[1]
+    s, sp, n_sel, n_out = _sel(sel, I)
+    A = np.empty((n_out, M), dtype=np.float64)
+    S = np.empty_like(A) if with_abs else None
+    rc = _load().oracle_spmm_gemm(_i64(v.shape[0]), cp, vp, _i64(I), _i64(J), _i64(L), _i64(M),
+                                  Cp, Dp, _i64(n_sel), sp, A.ctypes.data_as(_p),
+                                  S.ctypes.data_as(_p) if with_abs else None, ctypes.c_int(threads))
+    _check(rc)
+    return A, S
+
+
+def evaluate(w, sel=None, with_abs=True, threads=0):
+    """Evaluate a workload object (``workloads.configs.Workload``) -> (A, S)."""
+    if w.expr == "spttm_ttm3":
+        return spttm_ttm3(w.coords, w.vals, w.dims, *w.dense, sel=sel, with_abs=with_abs, threads=threads)
+    if w.expr == "spttm_ttm4":
+        return spttm_ttm4(w.coords, w.vals, w.dims, *w.dense, sel=sel, with_abs=with_abs, threads=threads)
+    if w.expr == "sddmm_spmm":
+        return sddmm_spmm(w.coords, w.vals, w.dims, *w.dense, sel=sel, with_abs=with_abs, threads=threads)[:2]
+    if w.expr == "spmm_gemm":
+        return spmm_gemm(w.coords, w.vals, w.dims, *w.dense, sel=sel, with_abs=with_abs, threads=threads)
+    raise ValueError(w.expr)

@@ -1,0 +1,267 @@
+"""Pins for the CPU oracle: everything here is fixed by the mathematics of the Einsum
+definitions (Table of kernels, Section 6 of the paper), not by the oracle itself.
+
+* brute force: B densified, the Einsum evaluated by explicit Python loops and by
+  numpy.einsum on tiny, non-square shapes (a transposed operand or swapped index
+  changes the result or the shape);
+* closed forms for all-ones operands;
+* special cases that reduce to densification, SpMM (scipy CSR @ dense, the loop of
+  Fig. 1b) and dense GEMM;
+* invariants: linearity in each operand, invariance under reordering of the COO list,
+  slice-subset evaluation equals the matching slices of the full evaluation;
+* the SDDMM sampled values exist exactly on B's stored coordinates.
+"""
+import itertools
+
+import numpy as np
+import pytest
+import scipy.sparse as sp
+
+import oracle
+
+
+def tiny_coo(rs, dims, nnz):
+    total = int(np.prod(dims))
+    lin = rs.choice(total, size=nnz, replace=False)
+    coords = np.stack(np.unravel_index(lin, dims), axis=1).astype(np.int32)
+    vals = rs.uniform(-1, 1, size=nnz).astype(np.float32)
+    return coords, vals
+
+
+def densify(coords, vals, dims):
+    B = np.zeros(dims, dtype=np.float64)
+    for c, v in zip(coords, vals):
+        B[tuple(c)] += float(v)
+    return B
+
+
+def dense(rs, r, c):
+    return rs.uniform(-1, 1, size=(r, c)).astype(np.float32)
+
+
+# ----------------------------------------------------------------- brute force
+
+def test_ttm3_bruteforce_loops_and_einsum():
+    rs = np.random.RandomState(1)
+    dims = (4, 5, 6)
+    coords, vals = tiny_coo(rs, dims, 37)
+    C, D = dense(rs, 5, 3), dense(rs, 6, 2)
+    A, S = oracle.spttm_ttm3(coords, vals, dims, C, D)
+    B = densify(coords, vals, dims)
+    ref = np.zeros((4, 3, 2))
+    refS = np.zeros((4, 3, 2))
+    for i, j, k, l, m in itertools.product(range(4), range(5), range(6), range(3), range(2)):
+        t = B[i, j, k] * float(C[j, l]) * float(D[k, m])
+        ref[i, l, m] += t
+        refS[i, l, m] += abs(t)
+    np.testing.assert_allclose(A, ref, rtol=0, atol=1e-13)
+    np.testing.assert_allclose(S, refS, rtol=0, atol=1e-13)
+    ein = np.einsum("ijk,jl,km->ilm", B, C.astype(np.float64), D.astype(np.float64))
+    np.testing.assert_allclose(A, ein, rtol=0, atol=1e-13)
+
+
+def test_ttm4_bruteforce_loops_and_einsum():
+    rs = np.random.RandomState(2)
+    dims = (3, 4, 5, 6)
+    coords, vals = tiny_coo(rs, dims, 61)
+    C, D, E = dense(rs, 4, 2), dense(rs, 5, 3), dense(rs, 6, 4)
+    A, S = oracle.spttm_ttm4(coords, vals, dims, C, D, E)
+    B = densify(coords, vals, dims)
+    ein = np.einsum("ijko,jl,km,on->ilmn", B, *(x.astype(np.float64) for x in (C, D, E)))
+    np.testing.assert_allclose(A, ein, rtol=0, atol=1e-13)
+    einS = np.einsum("ijko,jl,km,on->ilmn", np.abs(B), *(np.abs(x.astype(np.float64)) for x in (C, D, E)))
+    np.testing.assert_allclose(S, einS, rtol=0, atol=1e-13)
+    ref = np.zeros((3, 2, 3, 4))
+    for c, v in zip(coords, vals):
+        i, j, k, o = (int(x) for x in c)
+        for l, m, n in itertools.product(range(2), range(3), range(4)):
+            ref[i, l, m, n] += float(v) * float(C[j, l]) * float(D[k, m]) * float(E[o, n])
+    np.testing.assert_allclose(A, ref, rtol=0, atol=1e-13)
+
+
+def test_sddmm_spmm_bruteforce():
+    rs = np.random.RandomState(3)
+    dims = (5, 7)
+    coords, vals = tiny_coo(rs, dims, 17)
+    C, D, E = dense(rs, 5, 3), dense(rs, 7, 3), dense(rs, 7, 4)
+    A, S, P = oracle.sddmm_spmm(coords, vals, dims, C, D, E, with_sampled=True)
+    B = densify(coords, vals, dims)
+    ref = np.zeros((5, 4))
+    for i, j, k, l in itertools.product(range(5), range(7), range(3), range(4)):
+        ref[i, l] += B[i, j] * float(C[i, k]) * float(D[j, k]) * float(E[j, l])
+    np.testing.assert_allclose(A, ref, rtol=0, atol=1e-13)
+    C64, D64, E64 = (x.astype(np.float64) for x in (C, D, E))
+    ein = np.einsum("ij,ik,jk,jl->il", B, C64, D64, E64)
+    np.testing.assert_allclose(A, ein, rtol=0, atol=1e-13)
+    np.testing.assert_allclose(S, np.einsum("ij,ik,jk,jl->il", np.abs(B), np.abs(C64), np.abs(D64), np.abs(E64)),
+                               rtol=0, atol=1e-13)
+    # sampled matrix: (C D^T) sampled at B's coordinates and scaled by B; nothing elsewhere
+    samp = B * (C64 @ D64.T)
+    for p, c in enumerate(coords):
+        assert abs(P[p] - samp[c[0], c[1]]) < 1e-13
+    assert P.shape[0] == coords.shape[0]
+    # the SpMM of the sampled matrix gives A: fused == two separate kernels
+    np.testing.assert_allclose(A, samp @ E64, rtol=0, atol=1e-13)
+
+
+def test_spmm_gemm_bruteforce_and_both_orders():
+    rs = np.random.RandomState(4)
+    dims = (6, 5)
+    coords, vals = tiny_coo(rs, dims, 13)
+    C, D = dense(rs, 5, 4), dense(rs, 4, 3)
+    A, S = oracle.spmm_gemm(coords, vals, dims, C, D)
+    B = densify(coords, vals, dims)
+    ref = np.zeros((6, 3))
+    for i, j, l, m in itertools.product(range(6), range(5), range(4), range(3)):
+        ref[i, m] += B[i, j] * float(C[j, l]) * float(D[l, m])
+    np.testing.assert_allclose(A, ref, rtol=0, atol=1e-13)
+    C64, D64 = C.astype(np.float64), D.astype(np.float64)
+    np.testing.assert_allclose(A, (B @ C64) @ D64, rtol=0, atol=1e-13)   # (B.C).D
+    np.testing.assert_allclose(A, B @ (C64 @ D64), rtol=0, atol=1e-13)   # B.(C.D)
+    np.testing.assert_allclose(S, np.abs(B) @ np.abs(C64) @ np.abs(D64), rtol=0, atol=1e-13)
+
+
+# ----------------------------------------------------------------- closed forms
+
+def test_all_ones_closed_forms():
+    rs = np.random.RandomState(5)
+    dims = (7, 6, 5)
+    coords, _ = tiny_coo(rs, dims, 50)
+    ones = np.ones(50, dtype=np.float32)
+    A, S = oracle.spttm_ttm3(coords, ones, dims, np.ones((6, 3), np.float32), np.ones((5, 4), np.float32))
+    cnt = np.bincount(coords[:, 0], minlength=7)
+    assert np.array_equal(A, np.broadcast_to(cnt[:, None, None], (7, 3, 4)).astype(np.float64))
+    assert np.array_equal(A, S)
+
+    dims4 = (4, 3, 5, 2)
+    coords4, _ = tiny_coo(rs, dims4, 40)
+    A4, _ = oracle.spttm_ttm4(coords4, np.ones(40, np.float32), dims4, np.ones((3, 2), np.float32),
+                              np.ones((5, 3), np.float32), np.ones((2, 2), np.float32))
+    cnt4 = np.bincount(coords4[:, 0], minlength=4)
+    assert np.array_equal(A4, np.broadcast_to(cnt4[:, None, None, None], (4, 2, 3, 2)).astype(np.float64))
+
+    dims2 = (9, 8)
+    coords2, _ = tiny_coo(rs, dims2, 30)
+    deg = np.bincount(coords2[:, 0], minlength=9)
+    K, L = 5, 3
+    A1, _, P = oracle.sddmm_spmm(coords2, np.ones(30, np.float32), dims2, np.ones((9, K), np.float32),
+                                 np.ones((8, K), np.float32), np.ones((8, L), np.float32), with_sampled=True)
+    assert np.array_equal(A1, np.broadcast_to((K * deg)[:, None], (9, L)).astype(np.float64))
+    assert np.array_equal(P, np.full(30, float(K)))
+    Lg, Mg = 6, 2
+    Ag, _ = oracle.spmm_gemm(coords2, np.ones(30, np.float32), dims2, np.ones((8, Lg), np.float32),
+                             np.ones((Lg, Mg), np.float32))
+    assert np.array_equal(Ag, np.broadcast_to((Lg * deg)[:, None], (9, Mg)).astype(np.float64))
+
+
+# ----------------------------------------------------------------- special cases
+
+def test_identity_factors_densify():
+    rs = np.random.RandomState(6)
+    dims = (4, 5, 6)
+    coords, vals = tiny_coo(rs, dims, 41)
+    A, _ = oracle.spttm_ttm3(coords, vals, dims, np.eye(5, dtype=np.float32), np.eye(6, dtype=np.float32))
+    assert np.array_equal(A, densify(coords, vals, dims))
+    dims4 = (3, 4, 2, 5)
+    coords4, vals4 = tiny_coo(rs, dims4, 33)
+    A4, _ = oracle.spttm_ttm4(coords4, vals4, dims4, np.eye(4, dtype=np.float32), np.eye(2, dtype=np.float32),
+                              np.eye(5, dtype=np.float32))
+    assert np.array_equal(A4, densify(coords4, vals4, dims4))
+
+
+def test_spmm_gemm_reduces_to_spmm_and_gemm():
+    rs = np.random.RandomState(7)
+    I, J, L = 40, 30, 9
+    coords, vals = tiny_coo(rs, (I, J), 200)
+    C = dense(rs, J, L)
+    # D = identity: plain SpMM, the CSR loop nest of Fig. 1b
+    A, _ = oracle.spmm_gemm(coords, vals, (I, J), C, np.eye(L, dtype=np.float32))
+    Bcsr = sp.csr_matrix((vals.astype(np.float64), (coords[:, 0], coords[:, 1])), shape=(I, J))
+    np.testing.assert_allclose(A, Bcsr @ C.astype(np.float64), rtol=0, atol=1e-13)
+    # B = identity: dense GEMM C.D
+    n = 12
+    eye_coords = np.stack([np.arange(n), np.arange(n)], axis=1).astype(np.int32)
+    C2, D2 = dense(rs, n, 7), dense(rs, 7, 5)
+    A2, _ = oracle.spmm_gemm(eye_coords, np.ones(n, np.float32), (n, n), C2, D2)
+    np.testing.assert_allclose(A2, C2.astype(np.float64) @ D2.astype(np.float64), rtol=0, atol=1e-13)
+
+
+def test_sddmm_spmm_reduces_to_spmm():
+    rs = np.random.RandomState(8)
+    I, J, L = 25, 35, 6
+    coords, vals = tiny_coo(rs, (I, J), 150)
+    E = dense(rs, J, L)
+    A, _, _ = oracle.sddmm_spmm(coords, vals, (I, J), np.ones((I, 1), np.float32), np.ones((J, 1), np.float32), E)
+    Bcsr = sp.csr_matrix((vals.astype(np.float64), (coords[:, 0], coords[:, 1])), shape=(I, J))
+    np.testing.assert_allclose(A, Bcsr @ E.astype(np.float64), rtol=0, atol=1e-13)
+
+
+# ----------------------------------------------------------------- invariants
+
+def test_linearity_and_coo_order_invariance():
+    rs = np.random.RandomState(9)
+    dims = (6, 7, 8)
+    coords, vals = tiny_coo(rs, dims, 120)
+    C, D = dense(rs, 7, 4), dense(rs, 8, 5)
+    C2 = dense(rs, 7, 4)
+    A, S = oracle.spttm_ttm3(coords, vals, dims, C, D)
+    perm = rs.permutation(120)
+    Ap, Sp = oracle.spttm_ttm3(coords[perm], vals[perm], dims, C, D)
+    np.testing.assert_allclose(A, Ap, rtol=0, atol=1e-13)
+    np.testing.assert_allclose(S, Sp, rtol=0, atol=1e-13)
+    # linear in B (power-of-two scaling is exact), additive in C
+    A2, _ = oracle.spttm_ttm3(coords, (2 * vals).astype(np.float32), dims, C, D)
+    assert np.array_equal(A2, 2 * A)
+    Ac2, _ = oracle.spttm_ttm3(coords, vals, dims, C2, D)
+    Csum = C.astype(np.float64) + C2.astype(np.float64)
+    B = densify(coords, vals, dims)
+    np.testing.assert_allclose(A + Ac2, np.einsum("ijk,jl,km->ilm", B, Csum, D.astype(np.float64)),
+                               rtol=0, atol=1e-12)
+    assert np.all(S >= np.abs(A) - 1e-13)
+
+
+@pytest.mark.parametrize("threads", [1, 3])
+def test_slice_subset_matches_full(threads):
+    rs = np.random.RandomState(10)
+    dims = (9, 5, 6)
+    coords, vals = tiny_coo(rs, dims, 100)
+    C, D = dense(rs, 5, 3), dense(rs, 6, 2)
+    A, S = oracle.spttm_ttm3(coords, vals, dims, C, D, threads=threads)
+    sel = np.array([7, 0, 3])
+    As, Ss = oracle.spttm_ttm3(coords, vals, dims, C, D, sel=sel, threads=threads)
+    assert np.array_equal(As, A[sel]) and np.array_equal(Ss, S[sel])
+    c2, v2 = tiny_coo(rs, (9, 8), 40)
+    Cg, Dg = dense(rs, 8, 5), dense(rs, 5, 3)
+    Ag, _ = oracle.spmm_gemm(c2, v2, (9, 8), Cg, Dg)
+    Ags, _ = oracle.spmm_gemm(c2, v2, (9, 8), Cg, Dg, sel=sel)
+    assert np.array_equal(Ags, Ag[sel])
+    Cs, Ds, Es = dense(rs, 9, 4), dense(rs, 8, 4), dense(rs, 8, 3)
+    A1, _, _ = oracle.sddmm_spmm(c2, v2, (9, 8), Cs, Ds, Es)
+    A1s, _, P = oracle.sddmm_spmm(c2, v2, (9, 8), Cs, Ds, Es, sel=sel, with_sampled=True)
+    assert np.array_equal(A1s, A1[sel])
+    assert np.array_equal(~np.isnan(P), np.isin(c2[:, 0], sel))
+    c4, v4 = tiny_coo(rs, (9, 3, 4, 2), 50)
+    f = [dense(rs, 3, 2), dense(rs, 4, 2), dense(rs, 2, 3)]
+    A4, _ = oracle.spttm_ttm4(c4, v4, (9, 3, 4, 2), *f)
+    A4s, _ = oracle.spttm_ttm4(c4, v4, (9, 3, 4, 2), *f, sel=sel)
+    assert np.array_equal(A4s, A4[sel])
+
+
+def test_empty_and_out_of_range():
+    C, D = np.ones((3, 2), np.float32), np.ones((4, 2), np.float32)
+    A, S = oracle.spttm_ttm3(np.zeros((0, 3), np.int32), np.zeros(0, np.float32), (5, 3, 4), C, D)
+    assert A.shape == (5, 2, 2) and not A.any() and not S.any()
+    with pytest.raises(ValueError):
+        oracle.spttm_ttm3(np.array([[0, 3, 0]], np.int32), np.ones(1, np.float32), (5, 3, 4), C, D)
+
+
+def test_workload_generators_feed_oracle():
+    from workloads import configs
+    w = configs.make(1)
+    A, S = oracle.evaluate(w)
+    assert A.shape == (200, 16, 16) and np.isfinite(A).all()
+    # slice i only sees nonzeros with that i: zero B outside slice 5 and compare
+    keep = w.coords[:, 0] == 5
+    A5, _ = oracle.spttm_ttm3(w.coords[keep], w.vals[keep], w.dims, *w.dense)
+    np.testing.assert_array_equal(A5[5], A[5])
+    assert not A5[np.arange(200) != 5].any()
