@@ -265,7 +265,8 @@ def make_ttm4_zipf(name, seed, I, J, K, O, nnz, alpha, mean_fiber, L, M, N):
 def powerlaw_degrees(total, rows, alpha, cap):
     """Rank-Zipf degrees deg_r = min(cap, s * r^-alpha), s chosen so they sum to ``total``."""
     r = np.arange(1, rows + 1, dtype=np.float64) ** (-alpha)
-    lo, hi = 0.0, float(total) * 4.0 + 8.0
+    assert total <= cap * rows
+    lo, hi = 0.0, float(cap) * float(rows) ** alpha + 1.0
     for _ in range(200):
         mid = 0.5 * (lo + hi)
         if np.minimum(cap, mid * r).sum() < total:
