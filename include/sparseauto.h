@@ -1,0 +1,181 @@
+/*
+ * sparseauto.h -- C ABI of the B200 executor for fissioned / fused sparse contraction chains.
+ *
+ * The library evaluates chains O(idx_out) = sum_contract I_1(idx_1) * ... * I_n(idx_n) with
+ * one sparse operand B (first) and dense row-major operands (problem statement of Section 4.1;
+ * storage as in Section 2.1 and the pos/crd/vals arrays of Fig. 1b) under the branched loop
+ * nests that kernel fission and fusion produce (Section 4.2; chosen schedules in the Table
+ * of kernels, Section 6).  A fixed host table maps (expression, schedule) to ahead-of-time
+ * compiled CUDA kernels, the mapping the paper itself proposes in Section 6 ("maintaining a
+ * mapping from schedules chosen at compile-time to the corresponding compiled functions").
+ *
+ * Conventions
+ *   - Pointers marked HOST are ordinary host memory, DEVICE are device memory of the device the
+ *     tensor was created on.  No call takes or returns a C++ or framework type.
+ *   - All calls return an sa_status; nothing throws or aborts.  When a call fails before a
+ *     launch, nothing is enqueued and `out` is untouched.
+ *   - A tensor handle is immutable after creation; sa_run calls on different streams with
+ *     distinct `out` / `workspace` buffers may run concurrently.
+ *   - Requires a CUDA device of compute capability 10.0 (sm_100a); there is no CPU path.
+ */
+#ifndef SPARSEAUTO_H
+#define SPARSEAUTO_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct sa_tensor sa_tensor; /* opaque */
+
+typedef enum {
+    SA_OK = 0,
+    SA_E_ARG = 1,          /* null pointer, negative size, bad enum value                      */
+    SA_E_COORD_RANGE = 2,  /* a coordinate lies outside dims                                   */
+    SA_E_COORD_DUP = 3,    /* the same coordinate is stored twice                              */
+    SA_E_FORMAT = 4,       /* format / order combination not representable                     */
+    SA_E_SHAPE = 5,        /* dense operand shapes do not match the expression                 */
+    SA_E_UNSUPPORTED = 6,  /* valid request outside the compiled kernel table                  */
+    SA_E_ALLOC = 7,        /* host or device allocation failed                                 */
+    SA_E_WORKSPACE = 8,    /* workspace missing, misaligned or too small                       */
+    SA_E_CUDA = 9,         /* a CUDA runtime call or launch failed                             */
+    SA_E_BOUNDS = 10,      /* device-side index check failed (status word)                     */
+    SA_E_TIMEOUT = 11      /* a bounded device-side wait ran out (status word)                 */
+} sa_status;
+
+/* Level formats of Section 2.1.  CSR: dense row level + compressed column level (order 2).
+ * CSF: every level compressed (order 3 and 4); level 0 lists the non-empty slices. */
+typedef enum { SA_FMT_CSR = 1, SA_FMT_CSF = 2 } sa_format;
+
+/* Expressions (Table of kernels, Section 6; index letters as used in this library). */
+typedef enum {
+    /* kernel 6 <SpTTM,TTM>:  A(i,l,m) = sum_{j,k} B(i,j,k) C(j,l) D(k,m); ops = {C, D}          */
+    SA_EXPR_SPTTM_TTM3 = 1,
+    /* order-4 analogue:      A(i,l,m,n) = sum_{j,k,o} B(i,j,k,o) C(j,l) D(k,m) E(o,n);
+     * ops = {C, D, E}; scheduled with the two-level nesting of kernel 5's second schedule      */
+    SA_EXPR_SPTTM_TTM4 = 2,
+    /* kernel 1 <SDDMM,SpMM>: A(i,l) = sum_j B(i,j) (sum_k C(i,k) D(j,k)) E(j,l); ops = {C,D,E}  */
+    SA_EXPR_SDDMM_SPMM = 3,
+    /* kernel 4 <SpMM,GEMM>:  A(i,m) = sum_{j,l} B(i,j) C(j,l) D(l,m); ops = {C, D}             */
+    SA_EXPR_SPMM_GEMM = 4
+} sa_expr;
+
+typedef enum {
+    SA_SCHED_DEFAULT = 0,      /* the host table's choice for the expression                    */
+    SA_SCHED_FUSED = 1,        /* the fissioned / fused branched nest of the Table of kernels   */
+    SA_SCHED_ASSOC_LEFT = 2,   /* SA_EXPR_SPMM_GEMM only: (B.C).D, row temporary of L floats    */
+    SA_SCHED_ASSOC_RIGHT = 3,  /* SA_EXPR_SPMM_GEMM only: B.(C.D), J x M temporary in workspace */
+    SA_SCHED_DEBUG_MATERIALIZE = 9 /* SA_EXPR_SDDMM_SPMM only, for tests: additionally writes the
+                                      sampled values B(i,j) * sum_k C(i,k) D(j,k), aligned with
+                                      the exported last-level crd array, to the workspace       */
+} sa_schedule;
+
+/* Device allocator used for the tensor's device arrays.  alloc returns a DEVICE pointer aligned
+ * to at least 256 bytes or NULL; release frees it.  NULL allocator: cudaMalloc / cudaFree. */
+typedef struct {
+    void *(*alloc)(size_t bytes, void *ctx);
+    void (*release)(void *ptr, void *ctx);
+    void *ctx;
+} sa_allocator;
+
+/* Dense fp32 operand, DEVICE, row-major: element (r, c) at ptr[r * ld + c], ld >= cols
+ * (layout of the dense operands in Fig. 1b).  ptr must be 16-byte aligned and ld a multiple
+ * of 4.  Caller-owned; only read. */
+typedef struct {
+    const float *ptr;
+    int64_t rows, cols, ld;
+} sa_dense;
+
+/*
+ * Build the compressed representation of B from coordinate form (Section 2.1).
+ *   order   2 (with SA_FMT_CSR) or 3, 4 (with SA_FMT_CSF)
+ *   dims    HOST [order], each in [1, 2^31)
+ *   nnz     number of stored entries, 0 <= nnz < 2^31
+ *   coords  HOST [nnz * order], entry p at coords[p*order .. p*order+order-1], any order;
+ *           explicit zeros in vals stay part of the pattern
+ *   vals    HOST [nnz] fp32
+ *   device  CUDA device ordinal; becomes the tensor's device.  -1 builds a host-only handle
+ *           (levels and work lists, no device arrays) that serves sa_tensor_info / _export /
+ *           _worklist only; sa_run on it is SA_E_ARG.
+ *   dev_alloc  optional allocator for the device arrays (see sa_allocator)
+ *   out     receives the handle
+ * The entries are sorted lexicographically, the per-level pos / crd arrays and the
+ * load-balancing work lists (nonzero-balanced pieces of slices / rows, with their fiber and
+ * nonzero ranges) are built on the host and copied to the device.  coords / vals are copied;
+ * the caller may free them on return.  Synchronous.
+ * Errors: SA_E_ARG, SA_E_FORMAT, SA_E_COORD_RANGE, SA_E_COORD_DUP, SA_E_UNSUPPORTED (the
+ * packed coordinate needs more than 64 bits), SA_E_ALLOC, SA_E_CUDA.
+ */
+sa_status sa_tensor_create(int order, const int64_t *dims, int64_t nnz, const int32_t *coords,
+                           const float *vals, sa_format fmt, int device,
+                           const sa_allocator *dev_alloc, sa_tensor **out);
+
+/* Sizes.  level_counts HOST [order]: number of stored nodes per level (CSR level 0: rows;
+ * last level: nnz).  n_chunks: number of work items in the tensor's main work list.  Any
+ * output pointer may be NULL. */
+sa_status sa_tensor_info(const sa_tensor *t, int64_t *nnz, int64_t *level_counts, int64_t *n_chunks);
+
+/*
+ * Copy one level of the compressed structure back to HOST arrays (names as in Fig. 1b).
+ *   level 0..order-1.  pos: [count(level-1) + 1] entries (count(-1) = 1); crd: [count(level)];
+ *   vals: [nnz], only for the last level.  NULL outputs are skipped.  A CSR tensor has no
+ *   pos / crd at level 0 (dense level): asking for them is SA_E_ARG.
+ * The arrays are unique for a given input (lexicographic order), so they can be compared
+ * bit for bit with an independent construction.
+ */
+sa_status sa_tensor_export(const sa_tensor *t, int level, int64_t *pos, int32_t *crd, float *vals);
+
+/*
+ * Copy a load-balancing work list to HOST arrays (which: 0 = main list, 1 = the CSR tensor's
+ * second list used by SA_EXPR_SPMM_GEMM).  These are the slice / fiber / nonzero partition arrays:
+ *   counts [4]: number of items, number of leading 8-item groups that one thread block reduces
+ *               into a single tile, number of fix-up entries, number of partial-tile slots
+ *   items  [n_items * 8] int32 per item: out_row, row_end, f0, f1, p0, p1, dest, 0 --
+ *               fibers [f0,f1) (CSF) clipped to nonzeros [p0,p1) of slice out_row, or rows
+ *               [out_row,row_end) / nonzeros [p0,p1) of a long row (CSR); dest = partial slot or -1
+ *   fix    [n_fix * 4] int32 per entry: out_row, slot0, count, 0 -- out[out_row] = sum of `count`
+ *               partial tiles from slot0 (count 0: the slice / row is empty and is zero-filled)
+ * NULL outputs are skipped.
+ */
+sa_status sa_tensor_worklist(const sa_tensor *t, int which, int64_t *counts, int32_t *items, int32_t *fix);
+
+/* Bytes of DEVICE workspace sa_run needs for this tensor / expression / schedule / operand
+ * shapes (may be 0).  Only the shapes in ops are read. */
+sa_status sa_workspace_size(const sa_tensor *t, sa_expr expr, sa_schedule sched, const sa_dense *ops,
+                            int n_ops, size_t *bytes);
+
+/*
+ * Evaluate the chain: out = expr(B, ops...), asynchronously on cuda_stream.
+ *   ops        HOST array of n_ops descriptors of DEVICE operands, in the order listed at sa_expr
+ *   out        DEVICE fp32, dense row-major, contiguous, 16-byte aligned; FULLY OVERWRITTEN
+ *              (the statement is an assignment; empty slices / rows become +0.0)
+ *   workspace  DEVICE scratch of at least sa_workspace_size bytes, 256-byte aligned; may be
+ *              NULL when that size is 0.  Contents on entry are ignored.
+ *   cuda_stream  a cudaStream_t (NULL = default stream)
+ * Compiled dense ranks (anything else is SA_E_UNSUPPORTED): SPTTM_TTM3 L, M in {16, 32};
+ * SPTTM_TTM4 L = M = N = 16; SDDMM_SPMM K, L in {32, 64, 128}; SPMM_GEMM L in {128, 256},
+ * M in {32, 64}.
+ * Returns launch errors only; completion is observed by synchronising the stream.
+ * Errors: SA_E_ARG, SA_E_SHAPE, SA_E_UNSUPPORTED, SA_E_WORKSPACE, SA_E_CUDA.
+ */
+sa_status sa_run(const sa_tensor *B, sa_expr expr, sa_schedule sched, const sa_dense *ops, int n_ops,
+                 float *out, void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* Number of kernel launches the last successful sa_run on this handle enqueued. */
+sa_status sa_last_launch_count(const sa_tensor *t, int *launches);
+
+/* Synchronise cuda_stream and report the device-side status word of the tensor (SA_OK,
+ * SA_E_BOUNDS, SA_E_TIMEOUT), clearing it. */
+sa_status sa_last_device_status(const sa_tensor *t, void *cuda_stream);
+
+/* Release device and host memory of the handle.  NULL is accepted. */
+void sa_destroy(sa_tensor *t);
+
+const char *sa_status_string(sa_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPARSEAUTO_H */

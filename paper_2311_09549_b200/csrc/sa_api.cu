@@ -1,0 +1,333 @@
+// C-ABI entry points (declared in include/sparseauto.h): handle lifetime, argument checks and
+// the host table (expression, schedule) -> launcher that stands in for the paper's run-time
+// schedule lookup (Section 6, "mapping from schedules chosen at compile-time to the
+// corresponding compiled functions").
+#include <cstring>
+#include <new>
+
+#include "sa_internal.h"
+
+namespace {
+
+void *default_alloc(size_t bytes, void *)
+{
+    void *p = nullptr;
+    if (cudaMalloc(&p, bytes) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+    return p;
+}
+
+void default_release(void *p, void *) { cudaFree(p); }
+
+// Allocate device memory through the tensor's allocator and copy n elements of src into it.
+template <typename T>
+sa_status upload(sa_tensor *t, const T *src, size_t n, T **dst)
+{
+    *dst = nullptr;
+    const size_t bytes = sa_align256((n ? n : 1) * sizeof(T));
+    void *p = t->alloc.alloc(bytes, t->alloc.ctx);
+    if (!p) return SA_E_ALLOC;
+    t->dev_blocks.push_back(p);
+    if (n && cudaMemcpy(p, src, n * sizeof(T), cudaMemcpyHostToDevice) != cudaSuccess) return SA_E_CUDA;
+    *dst = static_cast<T *>(p);
+    return SA_OK;
+}
+
+sa_status upload_pos32(sa_tensor *t, const std::vector<int64_t> &pos, int32_t **dst)
+{
+    std::vector<int32_t> p32(pos.size());
+    for (size_t i = 0; i < pos.size(); ++i) p32[i] = int32_t(pos[i]);
+    return upload(t, p32.data(), p32.size(), dst);
+}
+
+sa_status upload_worklist(sa_tensor *t, sa_worklist &wl)
+{
+    sa_status s = upload(t, wl.items.data(), wl.items.size(), &wl.d_items);
+    if (s != SA_OK) return s;
+    return upload(t, wl.fix.data(), wl.fix.size(), &wl.d_fix);
+}
+
+struct device_guard {
+    int prev = -1;
+    bool ok = false;
+    explicit device_guard(int dev)
+    {
+        if (cudaGetDevice(&prev) != cudaSuccess) return;
+        ok = (prev == dev) || cudaSetDevice(dev) == cudaSuccess;
+    }
+    ~device_guard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+bool dense_ok(const sa_dense &d)
+{
+    return d.ptr != nullptr && d.rows > 0 && d.cols > 0 && d.ld >= d.cols && (d.ld % 4) == 0 &&
+           (reinterpret_cast<uintptr_t>(d.ptr) % 16) == 0;
+}
+
+// Shape check of the operand list; fills the number of operands the expression takes.
+sa_status check_ops(const sa_tensor *t, sa_expr expr, const sa_dense *ops, int n_ops, bool shapes_only)
+{
+    if (!ops) return SA_E_ARG;
+    int want = 0;
+    switch (expr) {
+        case SA_EXPR_SPTTM_TTM3: want = 2; break;
+        case SA_EXPR_SPTTM_TTM4: want = 3; break;
+        case SA_EXPR_SDDMM_SPMM: want = 3; break;
+        case SA_EXPR_SPMM_GEMM: want = 2; break;
+        default: return SA_E_ARG;
+    }
+    if (n_ops != want) return SA_E_ARG;
+    for (int i = 0; i < n_ops; ++i) {
+        if (ops[i].rows <= 0 || ops[i].cols <= 0) return SA_E_SHAPE;
+        if (!shapes_only && !dense_ok(ops[i])) return ops[i].ptr ? SA_E_SHAPE : SA_E_ARG;
+    }
+    switch (expr) {
+        case SA_EXPR_SPTTM_TTM3:
+            if (t->fmt != SA_FMT_CSF || t->order != 3) return SA_E_FORMAT;
+            if (ops[0].rows != t->dims[1] || ops[1].rows != t->dims[2]) return SA_E_SHAPE;
+            if (!sa_ranks_ok_ttm3(ops[0].cols, ops[1].cols)) return SA_E_UNSUPPORTED;
+            break;
+        case SA_EXPR_SPTTM_TTM4:
+            if (t->fmt != SA_FMT_CSF || t->order != 4) return SA_E_FORMAT;
+            if (ops[0].rows != t->dims[1] || ops[1].rows != t->dims[2] || ops[2].rows != t->dims[3]) return SA_E_SHAPE;
+            if (!sa_ranks_ok_ttm4(ops[0].cols, ops[1].cols, ops[2].cols)) return SA_E_UNSUPPORTED;
+            break;
+        case SA_EXPR_SDDMM_SPMM:
+            if (t->fmt != SA_FMT_CSR) return SA_E_FORMAT;
+            if (ops[0].rows != t->dims[0] || ops[1].rows != t->dims[1] || ops[2].rows != t->dims[1] ||
+                ops[0].cols != ops[1].cols)
+                return SA_E_SHAPE;
+            if (!sa_ranks_ok_sddmm(ops[0].cols, ops[2].cols)) return SA_E_UNSUPPORTED;
+            break;
+        case SA_EXPR_SPMM_GEMM:
+            if (t->fmt != SA_FMT_CSR) return SA_E_FORMAT;
+            if (ops[0].rows != t->dims[1] || ops[1].rows != ops[0].cols) return SA_E_SHAPE;
+            if (!sa_ranks_ok_spmm_gemm(ops[0].cols, ops[1].cols)) return SA_E_UNSUPPORTED;
+            break;
+    }
+    return SA_OK;
+}
+
+// Host table: which concrete schedule runs for (expr, sched).  Returns false if the pair is
+// not in the table.
+bool resolve_schedule(sa_expr expr, sa_schedule sched, sa_schedule *resolved)
+{
+    switch (expr) {
+        case SA_EXPR_SPTTM_TTM3:
+        case SA_EXPR_SPTTM_TTM4:
+            if (sched == SA_SCHED_DEFAULT || sched == SA_SCHED_FUSED) { *resolved = SA_SCHED_FUSED; return true; }
+            return false;
+        case SA_EXPR_SDDMM_SPMM:
+            if (sched == SA_SCHED_DEFAULT || sched == SA_SCHED_FUSED) { *resolved = SA_SCHED_FUSED; return true; }
+            if (sched == SA_SCHED_DEBUG_MATERIALIZE) { *resolved = sched; return true; }
+            return false;
+        case SA_EXPR_SPMM_GEMM:
+            // default: B.(C.D) -- fewer bytes gathered per nonzero when M < L
+            if (sched == SA_SCHED_DEFAULT) { *resolved = SA_SCHED_ASSOC_RIGHT; return true; }
+            if (sched == SA_SCHED_FUSED || sched == SA_SCHED_ASSOC_LEFT) { *resolved = SA_SCHED_ASSOC_LEFT; return true; }
+            if (sched == SA_SCHED_ASSOC_RIGHT) { *resolved = sched; return true; }
+            return false;
+    }
+    return false;
+}
+
+size_t workspace_bytes(const sa_tensor *t, sa_expr expr, sa_schedule sched, const sa_dense *ops)
+{
+    switch (expr) {
+        case SA_EXPR_SPTTM_TTM3: return sa_ws_ttm3(t, ops);
+        case SA_EXPR_SPTTM_TTM4: return sa_ws_ttm4(t, ops);
+        case SA_EXPR_SDDMM_SPMM: return sa_ws_sddmm_spmm(t, ops, sched == SA_SCHED_DEBUG_MATERIALIZE);
+        case SA_EXPR_SPMM_GEMM: return sa_ws_spmm_gemm(t, ops, sched == SA_SCHED_ASSOC_RIGHT);
+    }
+    return 0;
+}
+
+}  // namespace
+
+extern "C" {
+
+sa_status sa_tensor_create(int order, const int64_t *dims, int64_t nnz, const int32_t *coords, const float *vals,
+                           sa_format fmt, int device, const sa_allocator *dev_alloc, sa_tensor **out)
+{
+    if (!out) return SA_E_ARG;
+    *out = nullptr;
+    if (!dims || nnz < 0 || (nnz > 0 && (!coords || !vals)) || device < -1) return SA_E_ARG;
+    if (fmt != SA_FMT_CSR && fmt != SA_FMT_CSF) return SA_E_ARG;
+    if (order < 2 || order > SA_MAX_ORDER) return SA_E_FORMAT;
+    if ((fmt == SA_FMT_CSR) != (order == 2)) return SA_E_FORMAT;
+    if (nnz >= (int64_t(1) << 31) - 64) return SA_E_UNSUPPORTED;
+    for (int d = 0; d < order; ++d)
+        if (dims[d] < 1 || dims[d] >= (int64_t(1) << 31)) return SA_E_ARG;
+    if (dev_alloc && (!dev_alloc->alloc || !dev_alloc->release)) return SA_E_ARG;
+
+    sa_tensor *t = new (std::nothrow) sa_tensor();
+    if (!t) return SA_E_ALLOC;
+    t->order = order;
+    t->fmt = fmt;
+    t->nnz = nnz;
+    t->device = device;
+    for (int d = 0; d < order; ++d) t->dims[d] = dims[d];
+    if (dev_alloc) t->alloc = *dev_alloc;
+    else { t->alloc = sa_allocator{default_alloc, default_release, nullptr}; t->own_alloc = true; }
+
+    sa_status s = sa_build_levels(t, coords, vals);
+    if (s == SA_OK) {
+        try { sa_build_worklists(t); } catch (...) { s = SA_E_ALLOC; }
+    }
+    if (s == SA_OK && device >= 0) {
+        device_guard g(device);
+        if (!g.ok) s = SA_E_CUDA;
+        for (int l = 0; l < order && s == SA_OK; ++l) {
+            if (fmt == SA_FMT_CSR && l == 0) continue;   // dense level: nothing stored
+            s = upload_pos32(t, t->pos[l], &t->d_pos[l]);
+            if (s == SA_OK) s = upload(t, t->crd[l].data(), t->crd[l].size(), &t->d_crd[l]);
+        }
+        if (s == SA_OK) s = upload(t, t->vals.data(), t->vals.size(), &t->d_vals);
+        const int32_t zeros[4] = {0, 0, 0, 0};
+        if (s == SA_OK) s = upload(t, zeros, 4, &t->d_status);
+        if (s == SA_OK) s = upload_worklist(t, t->wl_main);
+        if (s == SA_OK) s = upload_worklist(t, t->wl_aux);
+        if (s == SA_OK && cudaDeviceSynchronize() != cudaSuccess) s = SA_E_CUDA;
+        if (s == SA_E_CUDA) cudaGetLastError();
+    }
+    if (s != SA_OK) { sa_destroy(t); return s; }
+    *out = t;
+    return SA_OK;
+}
+
+sa_status sa_tensor_info(const sa_tensor *t, int64_t *nnz, int64_t *level_counts, int64_t *n_chunks)
+{
+    if (!t) return SA_E_ARG;
+    if (nnz) *nnz = t->nnz;
+    if (level_counts)
+        for (int l = 0; l < t->order; ++l) level_counts[l] = t->count[l];
+    if (n_chunks) *n_chunks = int64_t(t->wl_main.items.size());
+    return SA_OK;
+}
+
+sa_status sa_tensor_export(const sa_tensor *t, int level, int64_t *pos, int32_t *crd, float *vals)
+{
+    if (!t || level < 0 || level >= t->order) return SA_E_ARG;
+    const bool dense_level = (t->fmt == SA_FMT_CSR && level == 0);
+    if (dense_level && (pos || crd)) return SA_E_ARG;
+    if (vals && level != t->order - 1) return SA_E_ARG;
+    if (pos) std::memcpy(pos, t->pos[level].data(), t->pos[level].size() * sizeof(int64_t));
+    if (crd) std::memcpy(crd, t->crd[level].data(), t->crd[level].size() * sizeof(int32_t));
+    if (vals) std::memcpy(vals, t->vals.data(), t->vals.size() * sizeof(float));
+    return SA_OK;
+}
+
+sa_status sa_tensor_worklist(const sa_tensor *t, int which, int64_t *counts, int32_t *items, int32_t *fix)
+{
+    if (!t || which < 0 || which > 1) return SA_E_ARG;
+    const sa_worklist &wl = which == 0 ? t->wl_main : t->wl_aux;
+    if (counts) {
+        counts[0] = int64_t(wl.items.size());
+        counts[1] = wl.n_group_ctas;
+        counts[2] = int64_t(wl.fix.size());
+        counts[3] = wl.n_slots;
+    }
+    if (items) std::memcpy(items, wl.items.data(), wl.items.size() * sizeof(sa_item));
+    if (fix) std::memcpy(fix, wl.fix.data(), wl.fix.size() * sizeof(sa_fix));
+    return SA_OK;
+}
+
+sa_status sa_workspace_size(const sa_tensor *t, sa_expr expr, sa_schedule sched, const sa_dense *ops, int n_ops,
+                            size_t *bytes)
+{
+    if (!t || !bytes) return SA_E_ARG;
+    sa_status s = check_ops(t, expr, ops, n_ops, true);
+    if (s != SA_OK) return s;
+    sa_schedule r;
+    if (!resolve_schedule(expr, sched, &r)) return SA_E_UNSUPPORTED;
+    *bytes = workspace_bytes(t, expr, r, ops);
+    return SA_OK;
+}
+
+sa_status sa_run(const sa_tensor *t, sa_expr expr, sa_schedule sched, const sa_dense *ops, int n_ops, float *out,
+                 void *workspace, size_t ws_bytes, void *cuda_stream)
+{
+    if (!t || !out || t->device < 0) return SA_E_ARG;
+    if (reinterpret_cast<uintptr_t>(out) % 16) return SA_E_ARG;
+    sa_status s = check_ops(t, expr, ops, n_ops, false);
+    if (s != SA_OK) return s;
+    sa_schedule r;
+    if (!resolve_schedule(expr, sched, &r)) return SA_E_UNSUPPORTED;
+    const size_t need = workspace_bytes(t, expr, r, ops);
+    if (need > 0 && (!workspace || ws_bytes < need || reinterpret_cast<uintptr_t>(workspace) % 256))
+        return SA_E_WORKSPACE;
+    device_guard g(t->device);
+    if (!g.ok) return SA_E_CUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    int launches = 0;
+    switch (expr) {
+        case SA_EXPR_SPTTM_TTM3: s = sa_launch_ttm3(t, ops, out, workspace, ws_bytes, stream, &launches); break;
+        case SA_EXPR_SPTTM_TTM4: s = sa_launch_ttm4(t, ops, out, workspace, ws_bytes, stream, &launches); break;
+        case SA_EXPR_SDDMM_SPMM:
+            s = sa_launch_sddmm_spmm(t, ops, out, workspace, ws_bytes, r == SA_SCHED_DEBUG_MATERIALIZE, stream, &launches);
+            break;
+        case SA_EXPR_SPMM_GEMM:
+            s = sa_launch_spmm_gemm(t, ops, out, workspace, ws_bytes, r == SA_SCHED_ASSOC_RIGHT, stream, &launches);
+            break;
+    }
+    if (s == SA_E_CUDA) cudaGetLastError();
+    if (s == SA_OK) t->last_launches = launches;
+    return s;
+}
+
+sa_status sa_last_launch_count(const sa_tensor *t, int *launches)
+{
+    if (!t || !launches) return SA_E_ARG;
+    *launches = t->last_launches;
+    return SA_OK;
+}
+
+sa_status sa_last_device_status(const sa_tensor *t, void *cuda_stream)
+{
+    if (!t || t->device < 0) return SA_E_ARG;
+    device_guard g(t->device);
+    if (!g.ok) return SA_E_CUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    int32_t word[4] = {0, 0, 0, 0};
+    if (cudaMemcpyAsync(word, t->d_status, sizeof(word), cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+        cudaStreamSynchronize(stream) != cudaSuccess) {
+        cudaGetLastError();
+        return SA_E_CUDA;
+    }
+    if (word[0] != 0) {
+        cudaMemsetAsync(t->d_status, 0, sizeof(word), stream);
+        cudaStreamSynchronize(stream);
+        return word[0] == SA_E_TIMEOUT ? SA_E_TIMEOUT : SA_E_BOUNDS;
+    }
+    return SA_OK;
+}
+
+void sa_destroy(sa_tensor *t)
+{
+    if (!t) return;
+    if (t->device >= 0) {
+        device_guard g(t->device);
+        for (void *p : t->dev_blocks) t->alloc.release(p, t->alloc.ctx);
+    }
+    delete t;
+}
+
+const char *sa_status_string(sa_status s)
+{
+    switch (s) {
+        case SA_OK: return "ok";
+        case SA_E_ARG: return "invalid argument";
+        case SA_E_COORD_RANGE: return "coordinate out of range";
+        case SA_E_COORD_DUP: return "duplicate coordinate";
+        case SA_E_FORMAT: return "format does not fit the order or the expression";
+        case SA_E_SHAPE: return "dense operand shape, leading dimension or alignment mismatch";
+        case SA_E_UNSUPPORTED: return "not in the compiled kernel table";
+        case SA_E_ALLOC: return "allocation failed";
+        case SA_E_WORKSPACE: return "workspace missing, misaligned or too small";
+        case SA_E_CUDA: return "CUDA runtime error";
+        case SA_E_BOUNDS: return "device-side index check failed";
+        case SA_E_TIMEOUT: return "device-side wait ran out";
+    }
+    return "unknown status";
+}
+
+}  // extern "C"

@@ -1,0 +1,370 @@
+// Host-side construction of the compressed levels (Section 2.1 of the paper: CSR / CSF as a
+// tree of levels, arrays named pos / crd / vals as in Fig. 1b) and of the load-balancing work
+// lists (nonzero-balanced pieces of slices, fibers and rows) the kernels consume.
+#include <algorithm>
+#include <cstring>
+#include <omp.h>
+
+#include "sa_internal.h"
+
+namespace {
+
+int bits_for(int64_t dim)
+{
+    int b = 1;
+    while ((int64_t(1) << b) < dim) ++b;
+    return b;
+}
+
+// Stable LSD radix sort of (key, idx) pairs on the low `total_bits` bits, 11 bits per pass.
+void radix_sort(std::vector<uint64_t> &keys, std::vector<uint32_t> &idx, int total_bits)
+{
+    const size_t n = keys.size();
+    if (n < 2) return;
+    constexpr int DB = 11, NB = 1 << DB;
+    const int passes = (total_bits + DB - 1) / DB;
+    std::vector<uint64_t> k2(n);
+    std::vector<uint32_t> i2(n);
+    const int nt = std::max(1, omp_get_max_threads());
+    std::vector<size_t> hist(size_t(nt) * NB);
+    uint64_t *ks = keys.data(), *kd = k2.data();
+    uint32_t *is = idx.data(), *id = i2.data();
+    for (int pass = 0; pass < passes; ++pass) {
+        const int shift = pass * DB;
+#pragma omp parallel num_threads(nt)
+        {
+            const int tid = omp_get_thread_num();
+            const size_t a = n * size_t(tid) / nt, b = n * size_t(tid + 1) / nt;
+            size_t *h = hist.data() + size_t(tid) * NB;
+            std::fill(h, h + NB, size_t(0));
+            for (size_t p = a; p < b; ++p) ++h[(ks[p] >> shift) & (NB - 1)];
+#pragma omp barrier
+#pragma omp single
+            {
+                size_t run = 0;
+                for (int d = 0; d < NB; ++d)
+                    for (int t = 0; t < nt; ++t) {
+                        size_t c = hist[size_t(t) * NB + d];
+                        hist[size_t(t) * NB + d] = run;
+                        run += c;
+                    }
+            }
+            for (size_t p = a; p < b; ++p) {
+                size_t q = h[(ks[p] >> shift) & (NB - 1)]++;
+                kd[q] = ks[p];
+                id[q] = is[p];
+            }
+        }
+        std::swap(ks, kd);
+        std::swap(is, id);
+    }
+    if (ks != keys.data()) {
+        std::memcpy(keys.data(), ks, n * sizeof(uint64_t));
+        std::memcpy(idx.data(), is, n * sizeof(uint32_t));
+    }
+}
+
+}  // namespace
+
+sa_status sa_build_levels(sa_tensor *t, const int32_t *coords, const float *vals)
+{
+    const int order = t->order;
+    const int64_t nnz = t->nnz;
+    int bits[SA_MAX_ORDER], shift[SA_MAX_ORDER];
+    int total = 0;
+    for (int d = 0; d < order; ++d) total += (bits[d] = bits_for(t->dims[d]));
+    if (total > 64) return SA_E_UNSUPPORTED;
+    for (int d = 0, s = total; d < order; ++d) { s -= bits[d]; shift[d] = s; }
+
+    std::vector<uint64_t> keys;
+    std::vector<uint32_t> idx;
+    try {
+        keys.resize(size_t(nnz));
+        idx.resize(size_t(nnz));
+    } catch (...) { return SA_E_ALLOC; }
+
+    int bad = 0;
+#pragma omp parallel for reduction(| : bad) schedule(static)
+    for (int64_t p = 0; p < nnz; ++p) {
+        uint64_t k = 0;
+        for (int d = 0; d < order; ++d) {
+            const int64_t c = coords[p * order + d];
+            if (c < 0 || c >= t->dims[d]) bad |= 1;
+            k |= uint64_t(uint32_t(c)) << shift[d];
+        }
+        keys[size_t(p)] = k;
+        idx[size_t(p)] = uint32_t(p);
+    }
+    if (bad) return SA_E_COORD_RANGE;
+
+    radix_sort(keys, idx, total);
+
+    int dup = 0;
+#pragma omp parallel for reduction(| : dup) schedule(static)
+    for (int64_t p = 1; p < nnz; ++p)
+        if (keys[size_t(p)] == keys[size_t(p - 1)]) dup |= 1;
+    if (dup) return SA_E_COORD_DUP;
+
+    try {
+        t->vals.resize(size_t(nnz));
+#pragma omp parallel for schedule(static)
+        for (int64_t p = 0; p < nnz; ++p) t->vals[size_t(p)] = vals[idx[size_t(p)]];
+        std::vector<uint32_t>().swap(idx);
+
+        const int last = order - 1;
+        auto coord_of = [&](uint64_t k, int d) { return int32_t((k >> shift[d]) & ((uint64_t(1) << bits[d]) - 1)); };
+
+        if (t->fmt == SA_FMT_CSR) {
+            const int64_t I = t->dims[0];
+            t->count[0] = I;
+            t->count[1] = nnz;
+            t->pos[1].assign(size_t(I) + 1, 0);
+            t->crd[1].resize(size_t(nnz));
+            for (int64_t p = 0; p < nnz; ++p) {
+                t->pos[1][size_t(coord_of(keys[size_t(p)], 0)) + 1]++;
+                t->crd[1][size_t(p)] = coord_of(keys[size_t(p)], 1);
+            }
+            for (int64_t i = 0; i < I; ++i) t->pos[1][size_t(i) + 1] += t->pos[1][size_t(i)];
+        } else {
+            // prefix of level l = key >> shift[l]; a new node opens at every level >= the first
+            // level whose prefix differs from the previous entry's
+            for (int l = 0; l <= last; ++l) { t->crd[l].clear(); t->pos[l].clear(); }
+            t->crd[last].resize(size_t(nnz));
+            for (int64_t p = 0; p < nnz; ++p) {
+                const uint64_t k = keys[size_t(p)];
+                int first = 0;
+                if (p > 0) {
+                    const uint64_t diff = k ^ keys[size_t(p - 1)];
+                    first = last;
+                    for (int l = 0; l < last; ++l)
+                        if ((diff >> shift[l]) != 0) { first = l; break; }
+                }
+                for (int l = first; l < last; ++l) {
+                    t->pos[l + 1].push_back(int64_t(l + 1 == last ? p : int64_t(t->crd[l + 1].size())));
+                    t->crd[l].push_back(coord_of(k, l));
+                }
+                t->crd[last][size_t(p)] = coord_of(k, last);
+            }
+            for (int l = 0; l <= last; ++l) t->count[l] = int64_t(t->crd[l].size());
+            for (int l = 0; l < last; ++l) t->pos[l + 1].push_back(t->count[l + 1]);
+            t->pos[0] = {0, t->count[0]};
+        }
+    } catch (...) { return SA_E_ALLOC; }
+    return SA_OK;
+}
+
+// ------------------------------------------------------------------------------ work lists
+
+namespace {
+
+sa_item empty_item()
+{
+    sa_item it;
+    it.out_row = 0; it.row_end = 0; it.f0 = 0; it.f1 = 0; it.p0 = 0; it.p1 = 0; it.dest = -1; it.pad = 0;
+    return it;
+}
+
+struct group_rec { int64_t len; std::vector<sa_item> items; };
+
+// Chunk of nonzeros one CTA reduces into a single tile: at least min_chunk, and large enough that
+// a slice is cut into at most max_parts partial tiles.
+int64_t chunk_for(int64_t n, int64_t min_chunk, int64_t max_parts)
+{
+    int64_t c = (n + max_parts - 1) / max_parts;
+    c = ((c + min_chunk - 1) / min_chunk) * min_chunk;
+    return std::max(c, min_chunk);
+}
+
+void append_empty_slices(sa_tensor *t, sa_worklist &wl)
+{
+    const int64_t I = t->dims[0];
+    size_t s = 0;
+    for (int64_t i = 0; i < I; ++i) {
+        if (s < t->crd[0].size() && t->crd[0][s] == i) { ++s; continue; }
+        wl.fix.push_back(sa_fix{int32_t(i), 0, 0, 0});
+    }
+}
+
+// Order-3 CSF: warp items are fiber ranges clipped to a nonzero range.
+void build_ttm3(sa_tensor *t, sa_worklist &wl)
+{
+    constexpr int64_t SMALL_MAX = 2048, MIN_CHUNK = 8192, MAX_PARTS = 192;
+    const auto &pos1 = t->pos[1];
+    const auto &pos2 = t->pos[2];
+    std::vector<sa_item> small;
+    std::vector<group_rec> groups;
+    for (int64_t s = 0; s < t->count[0]; ++s) {
+        const int64_t fa = pos1[size_t(s)], fb = pos1[size_t(s) + 1];
+        const int64_t pa = pos2[size_t(fa)], pb = pos2[size_t(fb)];
+        const int64_t n = pb - pa;
+        const int32_t row = t->crd[0][size_t(s)];
+        if (n <= SMALL_MAX) {
+            sa_item it = empty_item();
+            it.out_row = row; it.row_end = row + 1;
+            it.f0 = int32_t(fa); it.f1 = int32_t(fb); it.p0 = int32_t(pa); it.p1 = int32_t(pb);
+            small.push_back(it);
+            continue;
+        }
+        const int64_t chunk = chunk_for(n, MIN_CHUNK, MAX_PARTS);
+        const int64_t ng = (n + chunk - 1) / chunk;
+        int32_t slot0 = -1;
+        if (ng > 1) {
+            slot0 = int32_t(wl.n_slots);
+            wl.fix.push_back(sa_fix{row, slot0, int32_t(ng), 0});
+            wl.n_slots += ng;
+        }
+        for (int64_t g = 0; g < ng; ++g) {
+            const int64_t ga = pa + g * chunk, gb = std::min(pb, ga + chunk);
+            int64_t piece = (gb - ga + SA_WARPS_PER_CTA - 1) / SA_WARPS_PER_CTA;
+            piece = (piece + 31) / 32 * 32;
+            group_rec rec;
+            rec.len = gb - ga;
+            for (int w = 0; w < SA_WARPS_PER_CTA; ++w) {
+                sa_item it = empty_item();
+                it.out_row = row; it.row_end = row + 1;
+                it.dest = ng > 1 ? slot0 + int32_t(g) : -1;
+                const int64_t qa = std::min(gb, ga + w * piece), qb = std::min(gb, qa + piece);
+                if (qa < qb) {
+                    // fiber holding nonzero qa, and one past the fiber holding nonzero qb - 1
+                    const int64_t f0 = (std::upper_bound(pos2.begin() + fa, pos2.begin() + fb + 1, qa) - pos2.begin()) - 1;
+                    const int64_t f1 = (std::upper_bound(pos2.begin() + fa, pos2.begin() + fb + 1, qb - 1) - pos2.begin());
+                    it.f0 = int32_t(f0); it.f1 = int32_t(f1); it.p0 = int32_t(qa); it.p1 = int32_t(qb);
+                }
+                rec.items.push_back(it);
+            }
+            groups.push_back(std::move(rec));
+        }
+    }
+    std::stable_sort(groups.begin(), groups.end(), [](const group_rec &a, const group_rec &b) { return a.len > b.len; });
+    std::stable_sort(small.begin(), small.end(),
+                     [](const sa_item &a, const sa_item &b) { return (a.p1 - a.p0) > (b.p1 - b.p0); });
+    wl.n_group_ctas = int64_t(groups.size());
+    for (auto &g : groups) wl.items.insert(wl.items.end(), g.items.begin(), g.items.end());
+    wl.items.insert(wl.items.end(), small.begin(), small.end());
+    append_empty_slices(t, wl);
+}
+
+// Order-4 CSF: warp items are ranges of whole level-1 fibers (i,j) of one slice.
+void build_ttm4(sa_tensor *t, sa_worklist &wl)
+{
+    constexpr int64_t SMALL_MAX = 4096, MIN_CHUNK = 32768, MAX_PARTS = 160;
+    const auto &pos1 = t->pos[1];
+    const auto &pos2 = t->pos[2];
+    const auto &pos3 = t->pos[3];
+    auto nz_of_fiber = [&](int64_t f) { return pos3[size_t(pos2[size_t(f)])]; };   // first nonzero of fiber f
+    std::vector<sa_item> small;
+    std::vector<group_rec> groups;
+    for (int64_t s = 0; s < t->count[0]; ++s) {
+        const int64_t fa = pos1[size_t(s)], fb = pos1[size_t(s) + 1];
+        const int64_t pa = nz_of_fiber(fa), pb = nz_of_fiber(fb);
+        const int64_t n = pb - pa;
+        const int32_t row = t->crd[0][size_t(s)];
+        if (n <= SMALL_MAX || fb - fa == 1) {
+            sa_item it = empty_item();
+            it.out_row = row; it.row_end = row + 1;
+            it.f0 = int32_t(fa); it.f1 = int32_t(fb); it.p0 = int32_t(pa); it.p1 = int32_t(pb);
+            small.push_back(it);
+            continue;
+        }
+        const int64_t chunk = chunk_for(n, MIN_CHUNK, MAX_PARTS);
+        const int64_t piece = (chunk + SA_WARPS_PER_CTA - 1) / SA_WARPS_PER_CTA;
+        // cut the fiber list where the running nonzero count crosses multiples of `piece`
+        std::vector<sa_item> pieces;
+        int64_t f = fa;
+        while (f < fb) {
+            const int64_t start_nz = nz_of_fiber(f);
+            int64_t g = f + 1;
+            while (g < fb && nz_of_fiber(g) - start_nz < piece) ++g;
+            sa_item it = empty_item();
+            it.out_row = row; it.row_end = row + 1;
+            it.f0 = int32_t(f); it.f1 = int32_t(g);
+            it.p0 = int32_t(start_nz); it.p1 = int32_t(nz_of_fiber(g));
+            pieces.push_back(it);
+            f = g;
+        }
+        const int64_t ng = (int64_t(pieces.size()) + SA_WARPS_PER_CTA - 1) / SA_WARPS_PER_CTA;
+        int32_t slot0 = -1;
+        if (ng > 1) {
+            slot0 = int32_t(wl.n_slots);
+            wl.fix.push_back(sa_fix{row, slot0, int32_t(ng), 0});
+            wl.n_slots += ng;
+        }
+        for (int64_t g = 0; g < ng; ++g) {
+            group_rec rec;
+            rec.len = 0;
+            for (int w = 0; w < SA_WARPS_PER_CTA; ++w) {
+                const size_t q = size_t(g) * SA_WARPS_PER_CTA + size_t(w);
+                sa_item it = empty_item();
+                it.out_row = row; it.row_end = row + 1;
+                if (q < pieces.size()) it = pieces[q];
+                it.dest = ng > 1 ? slot0 + int32_t(g) : -1;
+                rec.len += it.p1 - it.p0;
+                rec.items.push_back(it);
+            }
+            groups.push_back(std::move(rec));
+        }
+    }
+    std::stable_sort(groups.begin(), groups.end(), [](const group_rec &a, const group_rec &b) { return a.len > b.len; });
+    std::stable_sort(small.begin(), small.end(),
+                     [](const sa_item &a, const sa_item &b) { return (a.p1 - a.p0) > (b.p1 - b.p0); });
+    wl.n_group_ctas = int64_t(groups.size());
+    for (auto &g : groups) wl.items.insert(wl.items.end(), g.items.begin(), g.items.end());
+    wl.items.insert(wl.items.end(), small.begin(), small.end());
+    append_empty_slices(t, wl);
+}
+
+// CSR: row ranges of about target_nnz nonzeros (at most max_rows rows); rows longer than
+// long_thresh are cut into pieces of `piece` nonzeros whose partial rows the fix-up kernel sums.
+void build_csr(sa_tensor *t, sa_worklist &wl, int64_t target_nnz, int64_t max_rows, int64_t long_thresh, int64_t piece)
+{
+    const auto &pos = t->pos[1];
+    const int64_t I = t->dims[0];
+    std::vector<sa_item> longs, ranges;
+    int64_t r0 = 0;
+    auto flush = [&](int64_t r1) {
+        if (r1 > r0) {
+            sa_item it = empty_item();
+            it.out_row = int32_t(r0); it.row_end = int32_t(r1);
+            it.p0 = int32_t(pos[size_t(r0)]); it.p1 = int32_t(pos[size_t(r1)]);
+            ranges.push_back(it);
+        }
+        r0 = r1;
+    };
+    for (int64_t r = 0; r < I; ++r) {
+        const int64_t a = pos[size_t(r)], b = pos[size_t(r) + 1];
+        if (b - a > long_thresh) {
+            flush(r);
+            const int64_t np = (b - a + piece - 1) / piece;
+            const int32_t slot0 = int32_t(wl.n_slots);
+            wl.fix.push_back(sa_fix{int32_t(r), slot0, int32_t(np), 0});
+            wl.n_slots += np;
+            for (int64_t q = 0; q < np; ++q) {
+                sa_item it = empty_item();
+                it.out_row = int32_t(r); it.row_end = int32_t(r + 1);
+                it.p0 = int32_t(a + q * piece); it.p1 = int32_t(std::min(b, a + (q + 1) * piece));
+                it.dest = slot0 + int32_t(q);
+                longs.push_back(it);
+            }
+            r0 = r + 1;
+            continue;
+        }
+        if (pos[size_t(r) + 1] - pos[size_t(r0)] > target_nnz && r > r0) flush(r);
+        if (r + 1 - r0 >= max_rows) flush(r + 1);
+    }
+    flush(I);
+    wl.n_group_ctas = 0;
+    wl.items = std::move(longs);
+    wl.items.insert(wl.items.end(), ranges.begin(), ranges.end());
+}
+
+}  // namespace
+
+void sa_build_worklists(sa_tensor *t)
+{
+    if (t->fmt == SA_FMT_CSF && t->order == 3) build_ttm3(t, t->wl_main);
+    if (t->fmt == SA_FMT_CSF && t->order == 4) build_ttm4(t, t->wl_main);
+    if (t->fmt == SA_FMT_CSR) {
+        build_csr(t, t->wl_main, 512, 64, 4096, 2048);   // fused SDDMM -> SpMM
+        build_csr(t, t->wl_aux, 256, 16, 4096, 2048);    // SpMM -> GEMM (both orders)
+    }
+}

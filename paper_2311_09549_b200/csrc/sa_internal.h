@@ -1,0 +1,98 @@
+// Internal declarations shared by the host builder, the API layer and the kernel launchers.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cstdint>
+#include <vector>
+
+#include "sparseauto.h"
+
+constexpr int SA_MAX_ORDER = 4;
+constexpr int SA_WARPS_PER_CTA = 8;
+
+// One unit of work for one warp.  32 bytes, read once per warp.
+//   CSF tensors: a contiguous range of level-1 fibers [f0, f1) inside ONE slice, clipped to the
+//   nonzero range [p0, p1) (order 3; a fiber may be cut between two items, each adds its part).
+//   CSR tensors: either whole rows [out_row, row_end) or, for a long row, the nonzeros [p0, p1)
+//   of row out_row (row_end == out_row + 1).
+//   dest < 0: the result is stored to `out`; dest >= 0: it is a partial result written to slot
+//   `dest` of the workspace and summed by the fix-up kernel.
+struct sa_item {
+    int32_t out_row;
+    int32_t row_end;
+    int32_t f0, f1;
+    int32_t p0, p1;
+    int32_t dest;
+    int32_t pad;
+};
+
+// Fix-up entry: out[out_row] = sum of `count` partial tiles starting at slot0 (count == 0: zeros).
+struct sa_fix {
+    int32_t out_row;
+    int32_t slot0;
+    int32_t count;
+    int32_t pad;
+};
+
+struct sa_worklist {
+    std::vector<sa_item> items;   // [n_group_ctas * SA_WARPS_PER_CTA group items][warp items]
+    std::vector<sa_fix> fix;
+    int64_t n_group_ctas = 0;     // leading CTAs whose 8 warps reduce into one tile
+    int64_t n_slots = 0;          // partial tiles in the workspace
+    sa_item *d_items = nullptr;
+    sa_fix *d_fix = nullptr;
+};
+
+struct sa_tensor {
+    int order = 0;
+    sa_format fmt = SA_FMT_CSF;
+    int64_t dims[SA_MAX_ORDER] = {0, 0, 0, 0};
+    int64_t nnz = 0;
+    int device = 0;
+    sa_allocator alloc{nullptr, nullptr, nullptr};
+    bool own_alloc = false;
+
+    // host copies (export + partitioning)
+    std::vector<int64_t> pos[SA_MAX_ORDER];   // pos[l]: count(l-1)+1 entries; empty for a dense level
+    std::vector<int32_t> crd[SA_MAX_ORDER];   // crd[l]: count(l) entries; empty for a dense level
+    std::vector<float> vals;
+    int64_t count[SA_MAX_ORDER] = {0, 0, 0, 0};
+
+    // device copies (pos as int32: nnz < 2^31)
+    int32_t *d_pos[SA_MAX_ORDER] = {nullptr, nullptr, nullptr, nullptr};
+    int32_t *d_crd[SA_MAX_ORDER] = {nullptr, nullptr, nullptr, nullptr};
+    float *d_vals = nullptr;
+    int32_t *d_status = nullptr;              // [4] device status word
+
+    sa_worklist wl_main;                      // TTM3 / TTM4 / SDDMM-SpMM
+    sa_worklist wl_aux;                       // CSR: SpMM-GEMM row items
+
+    mutable int last_launches = 0;
+    std::vector<void *> dev_blocks;           // everything obtained from the allocator
+};
+
+// ---- host builder (sa_build.cu)
+sa_status sa_build_levels(sa_tensor *t, const int32_t *coords, const float *vals);
+void sa_build_worklists(sa_tensor *t);
+
+// ---- launchers (one per chain); all asynchronous on `stream`, return SA_OK or SA_E_*.
+sa_status sa_launch_ttm3(const sa_tensor *t, const sa_dense *ops, float *out, void *ws, size_t ws_bytes,
+                         cudaStream_t stream, int *launches);
+size_t sa_ws_ttm3(const sa_tensor *t, const sa_dense *ops);
+sa_status sa_launch_ttm4(const sa_tensor *t, const sa_dense *ops, float *out, void *ws, size_t ws_bytes,
+                         cudaStream_t stream, int *launches);
+size_t sa_ws_ttm4(const sa_tensor *t, const sa_dense *ops);
+sa_status sa_launch_sddmm_spmm(const sa_tensor *t, const sa_dense *ops, float *out, void *ws, size_t ws_bytes,
+                               bool materialize, cudaStream_t stream, int *launches);
+size_t sa_ws_sddmm_spmm(const sa_tensor *t, const sa_dense *ops, bool materialize);
+sa_status sa_launch_spmm_gemm(const sa_tensor *t, const sa_dense *ops, float *out, void *ws, size_t ws_bytes,
+                              bool assoc_right, cudaStream_t stream, int *launches);
+size_t sa_ws_spmm_gemm(const sa_tensor *t, const sa_dense *ops, bool assoc_right);
+
+// Supported-rank predicates (shared by sa_workspace_size and sa_run).
+bool sa_ranks_ok_ttm3(int64_t L, int64_t M);
+bool sa_ranks_ok_ttm4(int64_t L, int64_t M, int64_t N);
+bool sa_ranks_ok_sddmm(int64_t K, int64_t L);
+bool sa_ranks_ok_spmm_gemm(int64_t L, int64_t M);
+
+static inline size_t sa_align256(size_t x) { return (x + 255) & ~size_t(255); }

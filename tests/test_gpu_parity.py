@@ -1,0 +1,42 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 oracle on the same
+seeded inputs, element by element."""
+import numpy as np
+import pytest
+
+import oracle
+from workloads import configs
+from util import TOL_FP32, TOL_TF32, assert_close, run_gpu
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def sa():
+    import torch
+    assert torch.cuda.is_available(), "these tests need a CUDA device"
+    import paper_2311_09549_b200 as sa
+    return sa
+
+
+@pytest.mark.parametrize("cfg", [1, 2, 5])
+def test_ttm_chains_mini(sa, cfg):
+    w = configs.make(cfg, "mini")
+    A_ref, S_ref = oracle.evaluate(w)
+    A, _ = run_gpu(sa, w)
+    assert_close(A, A_ref, S_ref, TOL_FP32, w.name)
+
+
+def test_sddmm_spmm_mini(sa):
+    w = configs.make(3, "mini")
+    A_ref, S_ref = oracle.evaluate(w)
+    A, _ = run_gpu(sa, w)
+    assert_close(A, A_ref, S_ref, TOL_FP32, w.name)
+
+
+@pytest.mark.parametrize("sched", ["left", "right", "default"])
+def test_spmm_gemm_mini_both_orders(sa, sched):
+    w = configs.make(4, "mini")
+    A_ref, S_ref = oracle.evaluate(w)
+    s = {"left": sa.SA_SCHED_ASSOC_LEFT, "right": sa.SA_SCHED_ASSOC_RIGHT, "default": sa.SA_SCHED_DEFAULT}[sched]
+    A, _ = run_gpu(sa, w, sched=s)
+    assert_close(A, A_ref, S_ref, TOL_FP32, w.name + "/" + sched)
