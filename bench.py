@@ -1,0 +1,336 @@
+#!/usr/bin/env python
+"""Throughput benchmark of the sparse contraction-chain executor.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 1..5] [--sched left|right]
+    python bench.py --impl reference ...        # the CPU oracle on a bounded sample
+
+One "step" is one pass of the whole hot path (sa_run: main kernel(s) + fix-up) over the
+synthetic workload.  Default workload: config 2, the order-3 <SpTTM,TTM> chain at scale.
+Prints ONE JSON line (rank 0).  With N > 1 (torchrun, one rank per GPU) every rank runs an
+independent replica of the same workload -- the path has no exchange step -- and `value`
+is the aggregate over ranks, timed as the max over ranks.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from workloads import configs  # noqa: E402
+
+METRIC = "GNNZ/s and achieved HBM GB/s (% of ~8 TB/s) per sparse contraction chain"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            return json.load(f), "measured"
+    return {"hbm_gbs": FALLBACK_HBM_GBS}, "fallback"
+
+
+def algorithmic_work(w, counts, sched):
+    """(bytes, flops) one step must move / compute under the schedule that runs: streams of
+    B's index and value arrays once, dense operands once (or one row per nonzero where the
+    table exceeds L2), the output once."""
+    nnz = w.nnz
+    sz = lambda a: a.size * 4  # noqa: E731
+    out_bytes = int(np.prod(w.out_shape)) * 4
+    if w.expr == "spttm_ttm3":
+        S, F2 = int(counts[0]), int(counts[1])
+        L, M = w.dense[0].shape[1], w.dense[1].shape[1]
+        return 8 * nnz + 8 * F2 + 8 * S + sz(w.dense[0]) + sz(w.dense[1]) + out_bytes, 2 * nnz * M + 2 * F2 * L * M
+    if w.expr == "spttm_ttm4":
+        S, F2, F3 = int(counts[0]), int(counts[1]), int(counts[2])
+        L, M, N = (d.shape[1] for d in w.dense)
+        b = 8 * nnz + 8 * F3 + 8 * F2 + 8 * S + sum(sz(d) for d in w.dense) + out_bytes
+        return b, 2 * (nnz * N + F3 * M * N + F2 * L * M * N)
+    if w.expr == "sddmm_spmm":
+        I = w.dims[0]
+        K, L = w.dense[0].shape[1], w.dense[2].shape[1]
+        return 8 * nnz + 4 * (I + 1) + 4 * (K + L) * nnz + sz(w.dense[0]) + out_bytes, nnz * (2 * K + 1 + 2 * L)
+    if w.expr == "spmm_gemm":
+        I, J = w.dims
+        L, M = w.dense[0].shape[1], w.dense[1].shape[1]
+        if sched == "left":
+            return 8 * nnz + 4 * (I + 1) + 4 * L * nnz + sz(w.dense[1]) + out_bytes, 2 * nnz * L + 2 * I * L * M
+        e_bytes = J * M * 4
+        return (sz(w.dense[0]) + e_bytes) + (8 * nnz + 4 * (I + 1) + 4 * M * nnz + out_bytes), 2 * J * L * M + 2 * nnz * M
+    raise ValueError(w.expr)
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.rows = []
+        self.proc = None
+        self.gpu_index = gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu_index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.thread.join(timeout=5)
+        sm, mx, reasons = [], [], set()
+        for r in self.rows:
+            if len(r) < 9:
+                continue
+            try:
+                sm.append(float(r[1]))
+                mx.append(float(r[2]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def oracle_sample(w, budget_s=20.0):
+    """Time the oracle, as it stands, on a bounded sample of output slices / rows of ``w``."""
+    import oracle
+    I = w.dims[0]
+    per_nnz = {"spttm_ttm3": lambda: w.dense[0].shape[1] * w.dense[1].shape[1],
+               "spttm_ttm4": lambda: w.dense[0].shape[1] * w.dense[1].shape[1] * w.dense[2].shape[1],
+               "sddmm_spmm": lambda: w.dense[0].shape[1] * w.dense[2].shape[1],
+               "spmm_gemm": lambda: w.dense[0].shape[1] * w.dense[1].shape[1]}[w.expr]()
+    cores = oracle.max_threads()
+    # ~0.25 G inner iterations per second per thread is a safe guess for the plain fp64 loop
+    target_nnz = int(budget_s * 0.25e9 * cores / per_nnz)
+    counts = np.bincount(w.coords[:, 0], minlength=I)
+    order = configs.rng.permutation(w.seed, 77, I)
+    # the oracle gives one slice to one thread: leave out slices that alone would take a thread
+    # longer than the whole budget, so that the sample stays bounded
+    cap = max(1, target_nnz // (2 * cores))
+    order = order[counts[order] <= cap]
+    csum = np.cumsum(counts[order])
+    n_take = int(np.searchsorted(csum, min(target_nnz, int(csum[-1])), side="left")) + 1
+    sel = np.sort(order[:n_take])
+    nnz_sel = int(counts[sel].sum())
+    t0 = time.perf_counter()
+    oracle.evaluate(w, sel=sel, with_abs=False)
+    dt = time.perf_counter() - t0
+    sample = ("%d of %d output slices/rows (seeded random among those with <= %d nonzeros), %d of %d nonzeros"
+              % (len(sel), I, cap, nnz_sel, w.nnz))
+    return {"value": nnz_sel / dt / 1e9, "unit": "GNNZ/s", "cores": cores, "kind": "oracle", "sample": sample,
+            "seconds": dt}
+
+
+def workload_label(cfg, sched):
+    names = {1: "cfg1 <SpTTM,TTM> 200^3 20k nnz L=M=16", 2: "cfg2 <SpTTM,TTM> 100000x80000x80000 50M nnz Zipf(1.2) L=M=32",
+             3: "cfg3 <SDDMM,SpMM> 1Mx1M 30M nnz K=L=64", 4: "cfg4 <SpMM,GEMM> 4Mx4M 100M nnz L=256 M=64",
+             5: "cfg5 order-4 <SpTTM,TTM> 50000x20000^3 100M nnz ranks 16"}
+    return names[cfg] + (" (%s)" % sched if cfg == 4 else "")
+
+
+def label(args):
+    return workload_label(args.workload, args.sched) + ("" if args.scale == "full" else " [mini-scale stand-in]")
+
+
+def run_reference(args, w, rank, world):
+    if rank != 0:
+        return
+    vals = []
+    last = None
+    for step in range(args.warmup + args.steps):
+        last = oracle_sample(w, budget_s=min(6.0, 150.0 / max(1, args.warmup + args.steps)))
+        if step >= args.warmup:
+            vals.append(last)
+    v = statistics.median(x["value"] for x in vals)
+    ms = statistics.median(x["seconds"] for x in vals) * 1e3
+    line = {"impl": "reference", "metric": METRIC, "value": v, "unit": "GNNZ/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": label(args)},
+            "cpu_baseline": {"value": v, "unit": "GNNZ/s", "cores": last["cores"], "kind": "oracle",
+                             "sample": last["sample"]},
+            "e2e": {"value": v, "unit": "GNNZ/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=31)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", type=int, default=2, choices=[1, 2, 3, 4, 5])
+    ap.add_argument("--scale", default="full", choices=["full", "mini"])
+    ap.add_argument("--sched", default="right", choices=["left", "right"], help="association order for workload 4")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        if rank == 0:
+            w = configs.make(args.workload, args.scale)
+            run_reference(args, w, rank, world)
+        return 0
+
+    import torch
+    import torch.distributed as dist
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the executor has no CPU path")
+    import paper_2311_09549_b200 as sa
+
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    w = configs.make(args.workload, args.scale)
+    fmt = sa.SA_FMT_CSR if w.fmt == "csr" else sa.SA_FMT_CSF
+    t0 = time.perf_counter()
+    tensor = sa.SparseTensor(w.dims, w.coords, w.vals, fmt, device=local_rank)
+    build_s = time.perf_counter() - t0
+    nnz, counts, n_chunks = tensor.info()
+    sched = sa.SA_SCHED_DEFAULT
+    if w.expr == "spmm_gemm":
+        sched = sa.SA_SCHED_ASSOC_LEFT if args.sched == "left" else sa.SA_SCHED_ASSOC_RIGHT
+
+    host_ops = [torch.from_numpy(np.ascontiguousarray(x)).pin_memory() for x in w.dense]
+    ops = [x.to(dev, non_blocking=False) for x in host_ops]
+    out = torch.empty(w.out_shape, dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream(dev)
+
+    def step():
+        tensor.run(w.expr, ops, out=out, sched=sched, stream=stream)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    for _ in range(args.warmup):
+        step()
+    launches_per_step = sa.sa_last_launch_count(tensor.handle)
+    barrier()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    barrier()
+    evs[0].record(stream)
+    for k in range(args.steps):
+        step()
+        evs[k + 1].record(stream)
+    barrier()
+    total_ms = evs[0].elapsed_time(evs[-1])
+    per_step = [evs[k].elapsed_time(evs[k + 1]) for k in range(args.steps)]
+    # keep the GPU busy a little longer so that the clock sampler sees the loaded state
+    if rank == 0:
+        t_end = time.perf_counter() + 1.0
+        while time.perf_counter() < t_end:
+            for _ in range(20):
+                step()
+            torch.cuda.synchronize(dev)
+        clocks = sampler.stop()
+    else:
+        clocks = None
+
+    # end to end: dense operands from pinned host memory, result back to pinned host memory
+    host_out = torch.empty(w.out_shape, dtype=torch.float32).pin_memory()
+    e2e_steps = max(1, min(args.e2e_steps, args.steps))
+
+    def e2e_step():
+        dops = [x.to(dev, non_blocking=True) for x in host_ops]
+        tensor.run(w.expr, dops, out=out, sched=sched, stream=stream)
+        host_out.copy_(out, non_blocking=True)
+
+    e2e_step()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record(stream)
+    barrier()
+    e2e_ms = e0.elapsed_time(e1) / e2e_steps
+
+    times = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    total_ms, e2e_ms = (float(x) for x in times.cpu())
+    ms_per_step = total_ms / args.steps
+
+    if rank == 0:
+        peaks, peak_kind = measured_peaks()
+        sched_name = args.sched if w.expr == "spmm_gemm" else "fused"
+        abytes, aflops = algorithmic_work(w, counts, sched_name)
+        gnnz = world * nnz / (ms_per_step * 1e-3) / 1e9
+        achieved = abytes / (ms_per_step * 1e-3) / 1e9
+        h2d = sum(int(x.numel()) * 4 for x in host_ops)
+        d2h = int(host_out.numel()) * 4
+        line = {
+            "metric": METRIC, "value": gnnz, "unit": "GNNZ/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": label(args), "scale": args.scale, "nnz": nnz,
+                       "level_counts": [int(c) for c in counts], "work_items": int(n_chunks),
+                       "l2": "inputs + output exceed L2 (126 MB); no flush" if abytes > 200e6 else "smaller than L2; launch-bound",
+                       "parallelism": "replicas x%d" % world, "build_s": round(build_s, 3),
+                       "step_ms_median": statistics.median(per_step), "step_ms_stdev": statistics.pstdev(per_step)},
+            "gflops": aflops / (ms_per_step * 1e-3) / 1e9,
+            "hbm_gbs_algorithmic": achieved, "hbm_frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS,
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_kind": "of " + peak_kind,
+                         "kernel": "whole step (main kernel + fix-up)", "algorithmic_bytes_per_launch": abytes},
+            "e2e": {"value": world * nnz / (e2e_ms * 1e-3) / 1e9, "unit": "GNNZ/s", "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
+            "gpu_launches": launches_per_step * args.steps,
+            "clocks": clocks,
+        }
+        if not args.no_cpu_baseline and world == 1:
+            cb = oracle_sample(w)
+            cb.pop("seconds")
+            line["cpu_baseline"] = cb
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())
