@@ -1,0 +1,225 @@
+"""Host builder of the C-ABI library, without a GPU (host-only handles, device = -1):
+compressed levels bit for bit against an independent construction, work-list (partition)
+invariants, error codes for malformed input, exported symbols."""
+import ctypes
+import re
+import os
+
+import numpy as np
+import pytest
+
+import paper_2311_09549_b200 as sa
+from workloads import configs
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def independent_levels(coords, vals, dims, fmt):
+    """pos/crd/vals per level built with plain Python containers from the sorted tuple list."""
+    order = coords.shape[1]
+    entries = sorted((tuple(int(x) for x in c), float(v)) for c, v in zip(coords, vals))
+    out_vals = np.array([v for _, v in entries], dtype=np.float32)
+    if fmt == "csr":
+        pos = np.zeros(dims[0] + 1, dtype=np.int64)
+        for (i, _), _ in entries:
+            pos[i + 1] += 1
+        return [(None, None), (np.cumsum(pos), np.array([c[1] for c, _ in entries], dtype=np.int32))], out_vals
+    levels = []
+    parents = [()]                      # distinct prefixes of the previous level, sorted
+    for l in range(order):
+        prefixes = sorted(set(c[:l + 1] for c, _ in entries))
+        crd = np.array([p[l] for p in prefixes], dtype=np.int32)
+        pos = np.zeros(len(parents) + 1, dtype=np.int64)
+        index_of = {p: n for n, p in enumerate(parents)}
+        for p in prefixes:
+            pos[index_of[p[:l]] + 1] += 1
+        levels.append((np.cumsum(pos), crd))
+        parents = prefixes
+    return levels, out_vals
+
+
+def export_all(t, fmt):
+    nnz, counts, _ = t.info()
+    levels = []
+    for l in range(t.order):
+        if fmt == "csr" and l == 0:
+            levels.append((None, None))
+            continue
+        n_pos = (1 if l == 0 else int(counts[l - 1])) + 1
+        pos, crd, _ = sa.sa_tensor_export(t.handle, l, n_pos=n_pos, n_crd=int(counts[l]))
+        levels.append((pos, crd if crd is not None else np.zeros(0, np.int32)))
+    _, _, vals = sa.sa_tensor_export(t.handle, t.order - 1, n_vals=nnz)
+    return levels, vals if vals is not None else np.zeros(0, np.float32)
+
+
+def small(cfg):
+    w = configs.make(cfg, "mini")
+    keep = configs.rng.permutation(5, 5, w.nnz)[:4000]
+    return w, w.coords[keep], w.vals[keep]
+
+
+@pytest.mark.parametrize("cfg", [1, 2, 3, 4, 5])
+def test_levels_match_independent_construction(cfg):
+    w, coords, vals = small(cfg)
+    t = sa.SparseTensor(w.dims, coords, vals, sa.SA_FMT_CSR if w.fmt == "csr" else sa.SA_FMT_CSF, device=-1)
+    got, got_vals = export_all(t, w.fmt)
+    want, want_vals = independent_levels(coords, vals, w.dims, w.fmt)
+    for l, ((gp, gc), (wp, wc)) in enumerate(zip(got, want)):
+        if wp is None:
+            assert gp is None
+            continue
+        assert np.array_equal(gp, wp), "pos of level %d" % l
+        assert np.array_equal(gc, wc), "crd of level %d" % l
+    assert np.array_equal(got_vals, want_vals)
+
+
+def _fiber_nnz_range(t, fmt, order, levels, f0, f1):
+    if order == 3:
+        return levels[2][0][f0], levels[2][0][f1]
+    pos2, pos3 = levels[2][0], levels[3][0]
+    return pos3[pos2[f0]], pos3[pos2[f1]]
+
+
+@pytest.mark.parametrize("cfg", [1, 2, 5])
+def test_csf_worklist_partitions_every_nonzero_once(cfg):
+    w = configs.make(cfg, "mini")
+    t = sa.SparseTensor(w.dims, w.coords, w.vals, sa.SA_FMT_CSF, device=-1)
+    levels, _ = export_all(t, "csf")
+    counts, items, fix = sa.sa_tensor_worklist(t.handle)
+    n_items, n_groups, n_fix, n_slots = (int(x) for x in counts)
+    crd0, pos1 = levels[0][1], levels[1][0]
+    slice_pos = {int(c): n for n, c in enumerate(crd0)}
+    covered = np.zeros(w.nnz, dtype=np.int32)
+    slot_owner = {}
+    for n, (row, row_end, f0, f1, p0, p1, dest, _) in enumerate(items):
+        if p0 == p1:
+            assert n < n_groups * 8 and f0 == f1, "only padding items of a group may be empty"
+            continue
+        s = slice_pos[int(row)]
+        assert pos1[s] <= f0 < f1 <= pos1[s + 1], "fibers stay inside the item's slice"
+        fa, fb = _fiber_nnz_range(t, "csf", t.order, levels, f0, f1)
+        assert fa <= p0 < p1 <= fb, "nonzero range lies inside the fiber range"
+        if t.order == 3:     # first and last fiber really intersect the clip range
+            pos2 = levels[2][0]
+            assert pos2[f0 + 1] > p0 and pos2[f1 - 1] < p1
+        else:
+            assert (fa, fb) == (p0, p1), "order-4 items hold whole (i,j) subtrees"
+        covered[p0:p1] += 1
+        if n < n_groups * 8:
+            lead = items[(n // 8) * 8]
+            assert dest == lead[6] and row == lead[0], "a group works on one slice and one destination"
+        if dest >= 0:
+            slot_owner.setdefault(int(dest), int(row))
+            assert slot_owner[int(dest)] == int(row)
+    assert (covered == 1).all(), "every nonzero belongs to exactly one item"
+    # fix-up entries: split slices own disjoint slot ranges, empty slices are listed with count 0
+    used = np.zeros(n_slots, dtype=np.int32)
+    empties = set()
+    for row, slot0, count, _ in fix:
+        if count == 0:
+            empties.add(int(row))
+            continue
+        used[slot0:slot0 + count] += 1
+        assert all(slot_owner[s] == int(row) for s in range(slot0, slot0 + count))
+    assert (used == 1).all() and set(slot_owner) == set(range(n_slots))
+    assert empties == set(range(w.dims[0])) - set(int(c) for c in crd0)
+    # nonzero balance: no warp item is larger than the small-slice bound / the piece size
+    sizes = items[:, 5] - items[:, 4]
+    assert sizes.max() <= max(4096, int(np.ceil(w.nnz / 8)))
+
+
+@pytest.mark.parametrize("cfg,which", [(3, 0), (4, 1), (4, 0)])
+def test_csr_worklist_partitions_rows_and_nonzeros(cfg, which):
+    w = configs.make(cfg, "mini")
+    t = sa.SparseTensor(w.dims, w.coords, w.vals, sa.SA_FMT_CSR, device=-1)
+    levels, _ = export_all(t, "csr")
+    pos = levels[1][0]
+    counts, items, fix = sa.sa_tensor_worklist(t.handle, which)
+    covered = np.zeros(w.nnz, dtype=np.int32)
+    rows = np.zeros(w.dims[0], dtype=np.int32)
+    for row, row_end, _, _, p0, p1, dest, _ in items:
+        if dest >= 0:
+            assert row_end == row + 1 and pos[row] <= p0 < p1 <= pos[row + 1]
+        else:
+            assert (p0, p1) == (pos[row], pos[row_end])
+            rows[row:row_end] += 1
+        covered[p0:p1] += 1
+    assert (covered == 1).all()
+    for row, slot0, count, _ in fix:
+        assert count >= 2
+        rows[row] += 1
+    assert (rows == 1).all(), "every row is written by exactly one range item or one fix-up entry"
+
+
+def test_empty_and_single_entry_tensors():
+    t = sa.SparseTensor((5, 4, 3), np.zeros((0, 3), np.int32), np.zeros(0, np.float32), sa.SA_FMT_CSF, device=-1)
+    nnz, counts, chunks = t.info()
+    assert nnz == 0 and not counts.any() and chunks == 0
+    c, items, fix = sa.sa_tensor_worklist(t.handle)
+    assert sorted(fix[:, 0].tolist()) == [0, 1, 2, 3, 4] and not fix[:, 2].any()
+    t1 = sa.SparseTensor((5, 4, 3), np.array([[4, 3, 2]], np.int32), np.ones(1, np.float32), sa.SA_FMT_CSF, device=-1)
+    assert t1.info()[1].tolist() == [1, 1, 1]
+    t2 = sa.SparseTensor((3, 3), np.zeros((0, 2), np.int32), np.zeros(0, np.float32), sa.SA_FMT_CSR, device=-1)
+    assert t2.info()[0] == 0
+
+
+def _create_status(order, dims, coords, vals, fmt):
+    try:
+        t = sa.SparseTensor(dims, np.asarray(coords, np.int32).reshape(-1, order), np.asarray(vals, np.float32), fmt,
+                            device=-1)
+        t.close()
+        return sa.SA_OK
+    except sa.SaError as e:
+        return e.status
+
+
+def test_malformed_input_is_rejected_with_a_status():
+    assert _create_status(3, (4, 4, 4), [[0, 0, 4]], [1.0], sa.SA_FMT_CSF) == sa.SA_E_COORD_RANGE
+    assert _create_status(3, (4, 4, 4), [[0, -1, 0]], [1.0], sa.SA_FMT_CSF) == sa.SA_E_COORD_RANGE
+    assert _create_status(3, (4, 4, 4), [[1, 2, 3], [0, 0, 0], [1, 2, 3]], [1.0, 2.0, 3.0], sa.SA_FMT_CSF) == sa.SA_E_COORD_DUP
+    assert _create_status(3, (4, 4, 4), [[1, 2, 3]], [1.0], sa.SA_FMT_CSR) == sa.SA_E_FORMAT
+    assert _create_status(2, (4, 4), [[1, 2]], [1.0], sa.SA_FMT_CSF) == sa.SA_E_FORMAT
+    assert _create_status(3, (4, 0, 4), [[1, 0, 3]], [1.0], sa.SA_FMT_CSF) == sa.SA_E_ARG
+    assert _create_status(3, (4, 4, 4), [[1, 2, 3]], [1.0], 7) == sa.SA_E_ARG
+    big = (2**30, 2**30, 2**30)     # 90 bits of packed coordinate
+    assert _create_status(3, big, [[1, 2, 3]], [1.0], sa.SA_FMT_CSF) == sa.SA_E_UNSUPPORTED
+    # order outside 2..4
+    h = ctypes.c_void_p()
+    dims = np.array([2] * 5, dtype=np.int64)
+    st = sa._lib.sa_tensor_create(5, dims.ctypes.data, 0, None, None, sa.SA_FMT_CSF, -1, None, ctypes.byref(h))
+    assert st == sa.SA_E_FORMAT and not h.value
+    assert sa._lib.sa_tensor_create(3, None, 0, None, None, sa.SA_FMT_CSF, -1, None, ctypes.byref(h)) == sa.SA_E_ARG
+
+
+def test_run_argument_checks_need_no_device():
+    w = configs.make(1)
+    t = sa.SparseTensor(w.dims, w.coords, w.vals, sa.SA_FMT_CSF, device=-1)
+    good = [(16, 200, 16, 16), (16, 200, 16, 16)]
+    assert sa.sa_workspace_size(t.handle, sa.SA_EXPR_SPTTM_TTM3, sa.SA_SCHED_DEFAULT, good) >= 0
+    for expr, sched, ops, want in [
+        (sa.SA_EXPR_SPTTM_TTM3, sa.SA_SCHED_DEFAULT, [(16, 199, 16, 16), (16, 200, 16, 16)], sa.SA_E_SHAPE),
+        (sa.SA_EXPR_SPTTM_TTM3, sa.SA_SCHED_DEFAULT, [(16, 200, 24, 24), (16, 200, 16, 16)], sa.SA_E_UNSUPPORTED),
+        (sa.SA_EXPR_SPTTM_TTM3, sa.SA_SCHED_ASSOC_LEFT, good, sa.SA_E_UNSUPPORTED),
+        (sa.SA_EXPR_SPTTM_TTM3, sa.SA_SCHED_DEFAULT, good[:1], sa.SA_E_ARG),
+        (sa.SA_EXPR_SDDMM_SPMM, sa.SA_SCHED_DEFAULT, good + good[:1], sa.SA_E_FORMAT),
+        (99, sa.SA_SCHED_DEFAULT, good, sa.SA_E_ARG),
+    ]:
+        with pytest.raises(sa.SaError) as e:
+            sa.sa_workspace_size(t.handle, expr, sched, ops)
+        assert e.value.status == want
+    # a host-only handle cannot run
+    with pytest.raises(sa.SaError) as e:
+        sa.sa_run(t.handle, sa.SA_EXPR_SPTTM_TTM3, sa.SA_SCHED_DEFAULT, good, 256, None, 0, None)
+    assert e.value.status == sa.SA_E_ARG
+    sa.sa_destroy(None)            # NULL-safe
+    assert sa.sa_status_string(sa.SA_E_COORD_DUP) == "duplicate coordinate"
+
+
+def test_library_exports_every_declared_symbol():
+    header = open(os.path.join(ROOT, "include", "sparseauto.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = sorted(set(re.findall(r"\b(sa_[a-z_0-9]+)\s*\(", header)))
+    assert declared and set(declared) == set(sa.EXPORTED_SYMBOLS)
+    lib = ctypes.CDLL(sa.LIB_PATH)
+    for name in declared:
+        assert hasattr(lib, name), name
