@@ -182,6 +182,12 @@ sa_status sa_tensor_create(int order, const int64_t *dims, int64_t nnz, const in
             if (s == SA_OK) s = upload(t, t->crd[l].data(), t->crd[l].size(), &t->d_crd[l]);
         }
         if (s == SA_OK) s = upload(t, t->vals.data(), t->vals.size(), &t->d_vals);
+        if (s == SA_OK && fmt == SA_FMT_CSF && order == 3) {
+            std::vector<int32_t> flagged(t->crd[2]);
+            for (int64_t f = 0; f < t->count[1]; ++f)
+                flagged[size_t(t->pos[2][size_t(f) + 1] - 1)] |= int32_t(0x80000000u);
+            s = upload(t, flagged.data(), flagged.size(), &t->d_crd_endflag);
+        }
         const int32_t zeros[4] = {0, 0, 0, 0};
         if (s == SA_OK) s = upload(t, zeros, 4, &t->d_status);
         if (s == SA_OK) s = upload_worklist(t, t->wl_main);

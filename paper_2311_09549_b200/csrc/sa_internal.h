@@ -62,6 +62,8 @@ struct sa_tensor {
     int32_t *d_pos[SA_MAX_ORDER] = {nullptr, nullptr, nullptr, nullptr};
     int32_t *d_crd[SA_MAX_ORDER] = {nullptr, nullptr, nullptr, nullptr};
     float *d_vals = nullptr;
+    int32_t *d_crd_endflag = nullptr;         // order-3 CSF: last-level crd with bit 31 set on the last
+                                              // nonzero of every fiber
     int32_t *d_status = nullptr;              // [4] device status word
 
     sa_worklist wl_main;                      // TTM3 / TTM4 / SDDMM-SpMM

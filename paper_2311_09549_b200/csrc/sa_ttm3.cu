@@ -1,97 +1,257 @@
 // Kernel 6 <SpTTM,TTM>:  A(i,l,m) = sum_{j,k} B(i,j,k) C(j,l) D(k,m), scheduled as the branched
 // nest  i, j' < t ; k': t += B(i,j,k) D(k,m) , l: A(i,l,m) += t C(j,l) >  of the paper's Table of
-// kernels (Section 6): per fiber (i,j) the SpTTM producer fills a temporary of M floats held in
-// registers (one lane per m), then the consumer adds the rank-1 update C(j,:)^T x temporary into
-// the slice's L x M tile, also held in registers.  The sampled order-3 intermediate
-// T(i,j,m) is never stored.
+// kernels (Section 6).  Producer (SpTTM, fp32 ALU): the nonzeros of a work item are streamed in
+// flat batches of 32; the D rows of a batch are gathered with cp.async into a per-warp ring of
+// shared-memory stages (several batches in flight per warp, no registers tied up); the fiber
+// temporary t(m) lives in one register per lane (lane = m) and is closed by an end-of-fiber flag
+// carried in the index stream.  Consumer (TTM, tensor cores): closed temporaries are staged eight
+// at a time in shared memory and the slice tile is updated as A(i,:,:) += Cg^T (L x 8) . T (8 x M)
+// with m16n8k8 TF32 MMAs, each operand split into a high and a low TF32 part (three products) so
+// the stage keeps fp32-level accuracy.  The order-3 intermediate T(i,j,m) is never stored.
 #include "sa_device.cuh"
 
 namespace {
 
-// One warp evaluates one work item: fibers [f0,f1) of a slice clipped to nonzeros [p0,p1).
-// Lane layout: G = 32/M lane groups; group h takes every G-th nonzero of a fiber and, in the
-// consumer stage, the l range [h*L/G, (h+1)*L/G).  acc[ll] = A(i, h*L/G + ll, m).
-template <int L, int M>
-__device__ __forceinline__ void ttm3_warp_item(const sa_item &it, const int32_t *__restrict__ pos2,
-                                               const int32_t *__restrict__ crd_j, const int32_t *__restrict__ crd_k,
-                                               const float *__restrict__ vals, const float *__restrict__ C, int64_t ldc,
-                                               const float *__restrict__ D, int64_t ldd, float (&acc)[L * M / 32])
+__device__ __forceinline__ uint32_t tf32_rna(float x)
 {
-    constexpr int G = 32 / M;
-    constexpr int LPG = L / G;
-    const int lane = threadIdx.x & 31;
-    const int h = lane / M, m = lane % M;
+    uint32_t r;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
+    return r;
+}
+
+__device__ __forceinline__ void split_tf32(float x, uint32_t &hi, uint32_t &lo)
+{
+    hi = tf32_rna(x);
+    lo = tf32_rna(x - __uint_as_float(hi));
+}
+
+__device__ __forceinline__ void mma_m16n8k8_tf32(float (&c)[4], const uint32_t (&a)[4], const uint32_t (&b)[2])
+{
+    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
+}
+
+__device__ __forceinline__ void cp_async16(float *dst_smem, const float *src)
+{
+    const uint32_t d = static_cast<uint32_t>(__cvta_generic_to_shared(dst_smem));
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+template <int L, int M>
+struct cfg {
+    static constexpr int MT = L / 16;       // m16 tiles over l
+    static constexpr int NT = M / 8;        // n8 tiles over m
+    static constexpr int TS = M;            // row stride of the staged temporaries (unpadded: two CTAs of
+                                            // 8 warps x (3 stages + ring) must fit one SM's shared memory)
+    static constexpr int RS = M + 8;        // row stride of a warp's tile in the CTA reduction
+    static constexpr int NS = 3;            // cp.async stages (batches of 32 factor rows) per warp
+    static constexpr int STAGE = 32 * M;    // floats per stage
+    static constexpr int WORK = NS * STAGE + 16 * TS;                      // stages + ring of staged temporaries
+    static constexpr int WARP_SMEM = (L * RS > WORK ? L * RS : WORK);      // floats per warp
+};
+
+// Gather the 32 rows D(k_s, :) of one batch into a stage: LPR lanes copy one row in 16-byte pieces.
+template <int M>
+__device__ __forceinline__ void stage_rows(float *stage, int kbatch, const float *__restrict__ D, int64_t ldd, int lane)
+{
+    constexpr int LPR = M / 4, RPI = 32 / LPR;
+    const int r = lane / LPR, c = lane % LPR;
 #pragma unroll
-    for (int q = 0; q < LPG; ++q) acc[q] = 0.f;
-    for (int f = it.f0; f < it.f1; ++f) {
-        const int a = max(pos2[f], it.p0), b = min(pos2[f + 1], it.p1);
-        float t = 0.f;
-        for (int base = a; base < b; base += 32) {
-            const int n = min(32, b - base);
-            int kk = 0;
-            float vv = 0.f;
-            if (lane < n) { kk = crd_k[base + lane]; vv = vals[base + lane]; }
-#pragma unroll 4
-            for (int s = 0; s < n; s += G) {
-                const int src = (s + h) & 31;
-                const int k = __shfl_sync(SA_FULL_MASK, kk, src);
-                const float v = __shfl_sync(SA_FULL_MASK, vv, src);
-                t = fmaf(v, __ldg(D + int64_t(k) * ldd + m), t);
-            }
-        }
-        if (G == 2) t += __shfl_xor_sync(SA_FULL_MASK, t, 16);
-        const float *crow = C + int64_t(crd_j[f]) * ldc + h * LPG;
+    for (int q = 0; q < 32 / RPI; ++q) {
+        const int row = q * RPI + r;
+        const int k = __shfl_sync(SA_FULL_MASK, kbatch, row) & 0x7fffffff;
+        cp_async16(stage + row * M + c * 4, D + int64_t(k) * ldd + c * 4);
+    }
+}
+
+// acc += Cg^T . T for eight staged fibers: rows (row0 + x) & 15, x = 0..7, of the 16-row ring;
+// crow_a / crow_b: rows of C of the fibers x = t and x = t + 4.
+template <int L, int M>
+__device__ __forceinline__ void ttm3_flush(float (&acc)[cfg<L, M>::MT][cfg<L, M>::NT][4], const float *__restrict__ Tbuf,
+                                           int row0, const float *__restrict__ crow_a, const float *__restrict__ crow_b,
+                                           int lane)
+{
+    using K = cfg<L, M>;
+    const int g = lane >> 2, t = lane & 3;
+    const float *ta = Tbuf + ((row0 + t) & 15) * K::TS + g;
+    const float *tb = Tbuf + ((row0 + t + 4) & 15) * K::TS + g;
+    uint32_t bh[K::NT][2], bl[K::NT][2];
 #pragma unroll
-        for (int q = 0; q < LPG; q += 4) {
-            const float4 c = sa_ldg4(crow + q);
-            acc[q + 0] = fmaf(c.x, t, acc[q + 0]);
-            acc[q + 1] = fmaf(c.y, t, acc[q + 1]);
-            acc[q + 2] = fmaf(c.z, t, acc[q + 2]);
-            acc[q + 3] = fmaf(c.w, t, acc[q + 3]);
+    for (int nt = 0; nt < K::NT; ++nt) {
+        split_tf32(ta[8 * nt], bh[nt][0], bl[nt][0]);
+        split_tf32(tb[8 * nt], bh[nt][1], bl[nt][1]);
+    }
+#pragma unroll
+    for (int mt = 0; mt < K::MT; ++mt) {
+        uint32_t ah[4], al[4];
+        split_tf32(__ldg(crow_a + 16 * mt + g), ah[0], al[0]);
+        split_tf32(__ldg(crow_a + 16 * mt + g + 8), ah[1], al[1]);
+        split_tf32(__ldg(crow_b + 16 * mt + g), ah[2], al[2]);
+        split_tf32(__ldg(crow_b + 16 * mt + g + 8), ah[3], al[3]);
+#pragma unroll
+        for (int nt = 0; nt < K::NT; ++nt) {
+            mma_m16n8k8_tf32(acc[mt][nt], al, bh[nt]);
+            mma_m16n8k8_tf32(acc[mt][nt], ah, bl[nt]);
+            mma_m16n8k8_tf32(acc[mt][nt], ah, bh[nt]);
         }
     }
 }
 
+// One warp evaluates one work item: nonzeros [p0,p1) starting inside fiber f0.
 template <int L, int M>
-__global__ void __launch_bounds__(256)
-ttm3_kernel(const sa_item *__restrict__ items, int64_t n_items, int n_group_ctas, const int32_t *__restrict__ pos2,
-            const int32_t *__restrict__ crd_j, const int32_t *__restrict__ crd_k, const float *__restrict__ vals,
-            const float *__restrict__ C, int64_t ldc, const float *__restrict__ D, int64_t ldd,
-            float *__restrict__ out, float *__restrict__ partial)
+__device__ __forceinline__ void ttm3_warp_item(const sa_item &it, const int32_t *__restrict__ crd_j,
+                                               const int32_t *__restrict__ kflag, const float *__restrict__ vals,
+                                               const float *__restrict__ C, int64_t ldc, const float *__restrict__ D,
+                                               int64_t ldd, float *__restrict__ wsm,
+                                               float (&acc)[cfg<L, M>::MT][cfg<L, M>::NT][4])
 {
-    constexpr int G = 32 / M;
-    constexpr int LPG = L / G;
+    using K = cfg<L, M>;
+    static_assert(K::NS == 3, "the register ring below is written for three stages");
+    const int lane = threadIdx.x & 31;
+    const int m = lane & (M - 1);
+    const int t4 = lane & 3;
+    float *Tbuf = wsm + K::NS * K::STAGE;
+#pragma unroll
+    for (int mt = 0; mt < K::MT; ++mt)
+#pragma unroll
+        for (int nt = 0; nt < K::NT; ++nt)
+#pragma unroll
+            for (int q = 0; q < 4; ++q) acc[mt][nt][q] = 0.f;
+    if (it.p0 >= it.p1) return;
+    const int p0 = it.p0, p1 = it.p1, f0 = it.f0, fmax = it.f1 - 1;
+    const int nb = (p1 - p0 + 31) >> 5;
+    auto load_kv = [&](int b, int &k, float &v) {
+        const int p = p0 + 32 * b + lane;
+        k = 0;
+        v = 0.f;
+        if (p < p1) { k = kflag[p]; v = vals[p]; }
+    };
+    // index/value registers of batches B .. B+3; row gathers of batches B+1, B+2 are in flight while B is consumed
+    int k0, k1, k2, k3;
+    float v0, v1, v2, v3;
+    load_kv(0, k0, v0);
+    load_kv(1, k1, v1);
+    load_kv(2, k2, v2);
+    load_kv(3, k3, v3);
+    stage_rows<M>(wsm, k0, D, ldd, lane);
+    cp_async_commit();
+    if (1 < nb) stage_rows<M>(wsm + K::STAGE, k1, D, ldd, lane);
+    cp_async_commit();
+    int nclosed = 0, nflushed = 0;          // fibers closed / handed to the tensor cores so far
+    int ja = crd_j[min(f0 + t4, fmax)], jb = crd_j[min(f0 + t4 + 4, fmax)];
+    float T = 0.f;
+    int s_cur = 0, s_issue = 2;
+#pragma unroll 1
+    for (int b = 0; b < nb; ++b) {
+        if (b + 2 < nb) stage_rows<M>(wsm + s_issue * K::STAGE, k2, D, ldd, lane);
+        cp_async_commit();
+        cp_async_wait<2>();
+        __syncwarp();
+        const float *st = wsm + s_cur * K::STAGE + m;
+        unsigned ends = __ballot_sync(SA_FULL_MASK, k0 < 0);
+        const int rem = p1 - p0 - 32 * b;
+        if (rem <= 32) ends |= 1u << (rem - 1);         // the item's last nonzero closes its (possibly cut) fiber
+        const int nchunks = rem >= 32 ? 4 : (rem + 7) >> 3;
+#pragma unroll 1
+        for (int c = 0; c < nchunks; ++c) {
+            const unsigned e8 = (ends >> (8 * c)) & 0xffu;
+            const float *sc = st + 8 * c * M;
+            if (e8 == 0) {
+#pragma unroll
+                for (int u = 0; u < 8; ++u) T = fmaf(__shfl_sync(SA_FULL_MASK, v0, 8 * c + u), sc[u * M], T);
+            } else {
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    T = fmaf(__shfl_sync(SA_FULL_MASK, v0, 8 * c + u), sc[u * M], T);
+                    if (e8 & (1u << u)) {
+                        Tbuf[(nclosed & 15) * K::TS + m] = T;
+                        T = 0.f;
+                        ++nclosed;
+                    }
+                }
+                if (nclosed - nflushed >= 8) {
+                    __syncwarp();
+                    ttm3_flush<L, M>(acc, Tbuf, nflushed, C + int64_t(ja) * ldc, C + int64_t(jb) * ldc, lane);
+                    __syncwarp();
+                    nflushed += 8;
+                    ja = crd_j[min(f0 + nflushed + t4, fmax)];
+                    jb = crd_j[min(f0 + nflushed + t4 + 4, fmax)];
+                }
+            }
+        }
+        __syncwarp();                                   // stage s_cur is free for the gather issued next
+        k0 = k1; k1 = k2; k2 = k3;
+        v0 = v1; v1 = v2; v2 = v3;
+        load_kv(b + 4, k3, v3);
+        s_issue = s_cur;
+        s_cur = s_cur == 2 ? 0 : s_cur + 1;
+    }
+    cp_async_wait<0>();
+    const int pending = nclosed - nflushed;             // 0..7
+    if (pending > 0) {
+        for (int x = pending; x < 8; ++x) Tbuf[((nflushed + x) & 15) * K::TS + m] = 0.f;   // unused rows
+        __syncwarp();
+        ttm3_flush<L, M>(acc, Tbuf, nflushed, C + int64_t(ja) * ldc, C + int64_t(jb) * ldc, lane);
+        __syncwarp();
+    }
+}
+
+template <int L, int M>
+__global__ void __launch_bounds__(256, 2)
+ttm3_kernel(const sa_item *__restrict__ items, int64_t n_items, int n_group_ctas, const int32_t *__restrict__ crd_j,
+            const int32_t *__restrict__ kflag, const float *__restrict__ vals, const float *__restrict__ C, int64_t ldc,
+            const float *__restrict__ D, int64_t ldd, float *__restrict__ out, float *__restrict__ partial)
+{
+    using K = cfg<L, M>;
     constexpr int TILE = L * M;
-    __shared__ float red[SA_WARPS_PER_CTA * TILE];
+    extern __shared__ __align__(16) float smem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int h = lane / M, m = lane % M;
+    const int g = lane >> 2, t = lane & 3;
+    float *wsm = smem + warp * K::WARP_SMEM;
     const int64_t idx = int64_t(blockIdx.x) * SA_WARPS_PER_CTA + warp;
     const bool group = int(blockIdx.x) < n_group_ctas;
-    float acc[LPG];
+    float acc[K::MT][K::NT][4];
     sa_item it;
-    it.f0 = it.f1 = 0;
+    it.f0 = it.f1 = it.p0 = it.p1 = 0;
     it.dest = -1;
     it.out_row = 0;
     if (idx < n_items) it = items[idx];
-    if (idx < n_items || group) ttm3_warp_item<L, M>(it, pos2, crd_j, crd_k, vals, C, ldc, D, ldd, acc);
+    if (idx < n_items || group) ttm3_warp_item<L, M>(it, crd_j, kflag, vals, C, ldc, D, ldd, wsm, acc);
     if (!group) {
         if (idx >= n_items) return;
-        float *dst = out + int64_t(it.out_row) * TILE + h * LPG * M + m;
+        float *dst = out + int64_t(it.out_row) * TILE;
 #pragma unroll
-        for (int q = 0; q < LPG; ++q) sa_st_cs(dst + q * M, acc[q]);
+        for (int mt = 0; mt < K::MT; ++mt)
+#pragma unroll
+            for (int nt = 0; nt < K::NT; ++nt) {
+                const int l = 16 * mt + g, mm = 8 * nt + 2 * t;
+                sa_st_cs2(dst + l * M + mm, make_float2(acc[mt][nt][0], acc[mt][nt][1]));
+                sa_st_cs2(dst + (l + 8) * M + mm, make_float2(acc[mt][nt][2], acc[mt][nt][3]));
+            }
         return;
     }
     // the CTA's eight warps hold partial tiles of the same slice: sum them in a fixed order
 #pragma unroll
-    for (int q = 0; q < LPG; ++q) red[warp * TILE + (h * LPG + q) * M + m] = acc[q];
+    for (int mt = 0; mt < K::MT; ++mt)
+#pragma unroll
+        for (int nt = 0; nt < K::NT; ++nt) {
+            const int l = 16 * mt + g, mm = 8 * nt + 2 * t;
+            *reinterpret_cast<float2 *>(wsm + l * K::RS + mm) = make_float2(acc[mt][nt][0], acc[mt][nt][1]);
+            *reinterpret_cast<float2 *>(wsm + (l + 8) * K::RS + mm) = make_float2(acc[mt][nt][2], acc[mt][nt][3]);
+        }
     __syncthreads();
     const sa_item lead = items[int64_t(blockIdx.x) * SA_WARPS_PER_CTA];
     float *dst = lead.dest >= 0 ? partial + int64_t(lead.dest) * TILE : out + int64_t(lead.out_row) * TILE;
     for (int x = threadIdx.x * 4; x < TILE; x += 256 * 4) {
-        float4 s = *reinterpret_cast<const float4 *>(red + x);
+        const int off = (x / M) * K::RS + (x % M);
+        float4 s = *reinterpret_cast<const float4 *>(smem + off);
 #pragma unroll
         for (int w = 1; w < SA_WARPS_PER_CTA; ++w) {
-            const float4 v = *reinterpret_cast<const float4 *>(red + w * TILE + x);
+            const float4 v = *reinterpret_cast<const float4 *>(smem + w * K::WARP_SMEM + off);
             s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
         }
         if (lead.dest >= 0) *reinterpret_cast<float4 *>(dst + x) = s;
@@ -107,9 +267,12 @@ cudaError_t launch(const sa_tensor *t, const sa_dense *ops, float *out, float *p
     const int64_t n_warp_items = n_items - wl.n_group_ctas * SA_WARPS_PER_CTA;
     const int64_t ctas = wl.n_group_ctas + (n_warp_items + SA_WARPS_PER_CTA - 1) / SA_WARPS_PER_CTA;
     if (ctas == 0) return cudaSuccess;
-    ttm3_kernel<L, M><<<(unsigned)ctas, 256, 0, stream>>>(wl.d_items, n_items, int(wl.n_group_ctas), t->d_pos[2],
-                                                         t->d_crd[1], t->d_crd[2], t->d_vals, ops[0].ptr, ops[0].ld,
-                                                         ops[1].ptr, ops[1].ld, out, partial);
+    constexpr size_t smem = size_t(SA_WARPS_PER_CTA) * cfg<L, M>::WARP_SMEM * sizeof(float);
+    auto kern = ttm3_kernel<L, M>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess)
+        return cudaGetLastError();
+    kern<<<(unsigned)ctas, 256, smem, stream>>>(wl.d_items, n_items, int(wl.n_group_ctas), t->d_crd[1], t->d_crd_endflag,
+                                               t->d_vals, ops[0].ptr, ops[0].ld, ops[1].ptr, ops[1].ld, out, partial);
     return cudaGetLastError();
 }
 
