@@ -163,6 +163,36 @@ sa_status sa_workspace_size(const sa_tensor *t, sa_expr expr, sa_schedule sched,
 sa_status sa_run(const sa_tensor *B, sa_expr expr, sa_schedule sched, const sa_dense *ops, int n_ops,
                  float *out, void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/*
+ * (No counterpart in the paper: an addition for callers of this library that must not allocate.)
+ *
+ * sa_run for SA_EXPR_SPTTM_TTM3 without a caller-supplied workspace and without any allocation.
+ * Some callers cannot hand sa_run a workspace because they are not in a position to obtain
+ * device memory when they call: code that runs after start-up under a fixed memory plan in
+ * which every byte is already assigned, plug-ins whose host application owns all allocation,
+ * and latency-critical loops that must stay clear of cudaMalloc / cudaFree because those calls
+ * may synchronise the whole device.  For them the partial tiles of split slices go to a scratch
+ * array of 4 MiB that is built into the library (a file-scope __device__
+ * array: every device that loads the library holds these 4 MiB until the process exits).
+ *
+ *   B, ops, out, cuda_stream   as for sa_run with SA_EXPR_SPTTM_TTM3 (ops = {C, D}, n_ops = 2)
+ *
+ * The call itself makes no cudaMalloc, cudaFree or other allocating call.  The first call on a
+ * device looks up the scratch array's device address (cudaGetSymbolAddress, with that device
+ * current) and caches it; make that first call before starting any stream capture.
+ * Limit: sa_workspace_size(B, SA_EXPR_SPTTM_TTM3, ...) must not exceed 4 MiB (1024 partial
+ * tiles at L = M = 32); beyond that the call returns SA_E_WORKSPACE and enqueues nothing --
+ * use sa_run with a workspace instead.
+ * All calls in a process share the one array per device.  Nothing in it has to start at zero
+ * (every slot that is read was written earlier in the same call), so it is not cleared, and it
+ * keeps the previous call's partial tiles.  Two calls that overlap on the device -- different
+ * streams, or different handles on the same device -- race on it and give wrong results: keep
+ * calls of this entry point ordered on one stream, or use sa_run with separate workspaces.
+ * Errors: SA_E_ARG, SA_E_FORMAT, SA_E_SHAPE, SA_E_UNSUPPORTED, SA_E_WORKSPACE, SA_E_CUDA.
+ */
+sa_status sa_run_ttm3_static_scratch(const sa_tensor *B, const sa_dense *ops, int n_ops, float *out,
+                                     void *cuda_stream);
+
 /* Number of kernel launches the last successful sa_run on this handle enqueued. */
 sa_status sa_last_launch_count(const sa_tensor *t, int *launches);
 

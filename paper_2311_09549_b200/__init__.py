@@ -29,7 +29,7 @@ SA_SCHED_DEBUG_MATERIALIZE = 9
 
 EXPORTED_SYMBOLS = ["sa_tensor_create", "sa_tensor_info", "sa_tensor_export", "sa_tensor_worklist",
                     "sa_workspace_size", "sa_run", "sa_last_launch_count", "sa_last_device_status",
-                    "sa_destroy", "sa_status_string"]
+                    "sa_destroy", "sa_status_string", "sa_run_ttm3_static_scratch"]
 
 
 class SaDense(ctypes.Structure):
@@ -57,8 +57,10 @@ _lib.sa_destroy.argtypes = [_vp]
 _lib.sa_destroy.restype = None
 _lib.sa_status_string.argtypes = [_int]
 _lib.sa_status_string.restype = ctypes.c_char_p
-for _n in EXPORTED_SYMBOLS[:-2]:
-    getattr(_lib, _n).restype = _int
+_lib.sa_run_ttm3_static_scratch.argtypes = [_vp, ctypes.POINTER(SaDense), _int, _vp, _vp]
+for _n in EXPORTED_SYMBOLS:
+    if _n not in ("sa_destroy", "sa_status_string"):
+        getattr(_lib, _n).restype = _int
 
 
 class SaError(RuntimeError):
@@ -159,6 +161,14 @@ def sa_run(handle, expr, sched, ops, out_ptr, workspace_ptr, workspace_bytes, st
     st = _lib.sa_run(handle, int(expr), int(sched), _dense_array(ops), len(ops), out_ptr, workspace_ptr,
                      int(workspace_bytes), stream)
     _check(st, "sa_run")
+
+
+def sa_run_ttm3_static_scratch(handle, ops, out_ptr, stream):
+    """The order-3 <SpTTM,TTM> chain with the library's built-in 4 MiB scratch instead of a workspace:
+    for callers that cannot allocate device memory.  Raises SaError(SA_E_WORKSPACE) if the tensor
+    needs more scratch than that."""
+    st = _lib.sa_run_ttm3_static_scratch(handle, _dense_array(ops), len(ops), out_ptr, stream)
+    _check(st, "sa_run_ttm3_static_scratch")
 
 
 def sa_last_launch_count(handle):

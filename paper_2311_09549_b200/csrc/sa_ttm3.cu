@@ -305,3 +305,63 @@ sa_status sa_launch_ttm3(const sa_tensor *t, const sa_dense *ops, float *out, vo
     }
     return SA_OK;
 }
+
+// ------------------------------------------------------------------ entry point without allocation
+
+// Scratch for sa_run_ttm3_static_scratch: part of the library image, so every device that loads the
+// library carries these 4 MiB until the process exits.
+constexpr size_t SA_STATIC_SCRATCH_BYTES = size_t(4) << 20;
+static __device__ __align__(256) float sa_static_scratch[SA_STATIC_SCRATCH_BYTES / sizeof(float)];
+
+namespace {
+
+constexpr int SA_MAX_DEVICES = 64;
+float *g_static_scratch_addr[SA_MAX_DEVICES];   // device address of sa_static_scratch, per device; set once
+
+// In host code `sa_static_scratch` only names the symbol; the address a kernel can use has to be
+// asked for, with the owning device current.
+sa_status static_scratch_address(int device, float **addr)
+{
+    if (device < 0 || device >= SA_MAX_DEVICES) return SA_E_ARG;
+    if (!g_static_scratch_addr[device]) {
+        float *p = nullptr;
+        if (cudaGetSymbolAddress(reinterpret_cast<void **>(&p), sa_static_scratch) != cudaSuccess || !p) {
+            cudaGetLastError();
+            return SA_E_CUDA;
+        }
+        g_static_scratch_addr[device] = p;
+    }
+    *addr = g_static_scratch_addr[device];
+    return SA_OK;
+}
+
+}  // namespace
+
+extern "C" sa_status sa_run_ttm3_static_scratch(const sa_tensor *t, const sa_dense *ops, int n_ops, float *out,
+                                                void *cuda_stream)
+{
+    if (!t || !ops || !out || n_ops != 2 || t->device < 0) return SA_E_ARG;
+    if (reinterpret_cast<uintptr_t>(out) % 16) return SA_E_ARG;
+    if (t->fmt != SA_FMT_CSF || t->order != 3) return SA_E_FORMAT;
+    for (int i = 0; i < 2; ++i) {
+        if (!ops[i].ptr) return SA_E_ARG;
+        if (ops[i].rows != t->dims[i + 1] || ops[i].cols <= 0 || ops[i].ld < ops[i].cols || ops[i].ld % 4 ||
+            reinterpret_cast<uintptr_t>(ops[i].ptr) % 16)
+            return SA_E_SHAPE;
+    }
+    if (!sa_ranks_ok_ttm3(ops[0].cols, ops[1].cols)) return SA_E_UNSUPPORTED;
+    const size_t need = sa_ws_ttm3(t, ops);
+    if (need > SA_STATIC_SCRATCH_BYTES) return SA_E_WORKSPACE;   // the partial tiles do not fit the built-in scratch
+    int prev = -1;
+    if (cudaGetDevice(&prev) != cudaSuccess) { cudaGetLastError(); return SA_E_CUDA; }
+    if (prev != t->device && cudaSetDevice(t->device) != cudaSuccess) { cudaGetLastError(); return SA_E_CUDA; }
+    float *scratch = nullptr;
+    sa_status s = static_scratch_address(t->device, &scratch);
+    int launches = 0;
+    if (s == SA_OK)
+        s = sa_launch_ttm3(t, ops, out, scratch, SA_STATIC_SCRATCH_BYTES, static_cast<cudaStream_t>(cuda_stream), &launches);
+    if (s == SA_E_CUDA) cudaGetLastError();
+    if (s == SA_OK) t->last_launches = launches;
+    if (prev != t->device) cudaSetDevice(prev);
+    return s;
+}
