@@ -151,6 +151,21 @@ def oracle_sample(w, budget_s=20.0):
             "seconds": dt}
 
 
+def reduce_max_over_ranks(values, device, world):
+    """Element-wise maximum of ``values`` over all ranks (the job is as slow as its slowest rank)."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t.cpu()]
+
+
+def aggregate_throughput(nnz_per_rank, world, ms_per_step):
+    """Whole-job GNNZ/s of ``world`` independent replicas that all finish within ms_per_step."""
+    return world * nnz_per_rank / (ms_per_step * 1e-3) / 1e9
+
+
 def workload_label(cfg, sched):
     names = {1: "cfg1 <SpTTM,TTM> 200^3 20k nnz L=M=16", 2: "cfg2 <SpTTM,TTM> 100000x80000x80000 50M nnz Zipf(1.2) L=M=32",
              3: "cfg3 <SDDMM,SpMM> 1Mx1M 30M nnz K=L=64", 4: "cfg4 <SpMM,GEMM> 4Mx4M 100M nnz L=256 M=64",
@@ -289,17 +304,14 @@ def main():
     barrier()
     e2e_ms = e0.elapsed_time(e1) / e2e_steps
 
-    times = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    total_ms, e2e_ms = (float(x) for x in times.cpu())
+    total_ms, e2e_ms = reduce_max_over_ranks([total_ms, e2e_ms], dev, world)
     ms_per_step = total_ms / args.steps
 
     if rank == 0:
         peaks, peak_kind = measured_peaks()
         sched_name = args.sched if w.expr == "spmm_gemm" else "fused"
         abytes, aflops = algorithmic_work(w, counts, sched_name)
-        gnnz = world * nnz / (ms_per_step * 1e-3) / 1e9
+        gnnz = aggregate_throughput(nnz, world, ms_per_step)
         achieved = abytes / (ms_per_step * 1e-3) / 1e9
         h2d = sum(int(x.numel()) * 4 for x in host_ops)
         d2h = int(host_out.numel()) * 4
@@ -317,7 +329,7 @@ def main():
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                          "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_kind": "of " + peak_kind,
                          "kernel": "whole step (main kernel + fix-up)", "algorithmic_bytes_per_launch": abytes},
-            "e2e": {"value": world * nnz / (e2e_ms * 1e-3) / 1e9, "unit": "GNNZ/s", "h2d_bytes_per_step": h2d,
+            "e2e": {"value": aggregate_throughput(nnz, world, e2e_ms), "unit": "GNNZ/s", "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
             "gpu_launches": launches_per_step * args.steps,
             "clocks": clocks,

@@ -1,0 +1,203 @@
+"""GPU edge cases through the C ABI: empty and one-entry tensors, empty slices and rows, padded
+leading dimensions, every compiled rank combination, fibers and rows around the split
+thresholds, the SDDMM sampling pattern, run-to-run reproducibility and workspace errors."""
+import numpy as np
+import pytest
+
+import oracle
+from workloads import configs, rng
+from util import TOL_FP32, assert_close, run_gpu
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def sa():
+    import torch
+    assert torch.cuda.is_available()
+    import paper_2311_09549_b200 as sa
+    return sa
+
+
+def _wl(expr, fmt, dims, coords, vals, dense, out_shape):
+    return configs.Workload("edge", expr, fmt, tuple(dims), np.asarray(coords, np.int32).reshape(-1, len(dims)),
+                            np.asarray(vals, np.float32), dense, tuple(out_shape), 0)
+
+
+def _dense(seed, which, r, c):
+    return configs.dense_uniform(seed, which, r, c)
+
+
+def _random_coo(seed, dims, nnz):
+    lin = rng.keyed_bijection(np.arange(nnz), int(np.prod(dims)), np.uint64(seed))
+    coords = np.stack(np.unravel_index(lin, dims), axis=1).astype(np.int32)
+    return coords, rng.uniform_f32(seed, 1, np.arange(nnz), -1.0, 1.0)
+
+
+def _check(sa, w, sched=None, tol=TOL_FP32):
+    A_ref, S_ref = oracle.evaluate(w)
+    A, t = run_gpu(sa, w, sched=sched)
+    assert_close(A, A_ref, S_ref, tol, w.expr)
+    return A, t
+
+
+@pytest.mark.parametrize("nnz", [0, 1])
+def test_empty_and_single_entry_all_chains(sa, nnz):
+    c3 = [[3, 2, 1]][:nnz]
+    c4 = [[3, 2, 1, 0]][:nnz]
+    c2 = [[3, 2]][:nnz]
+    v = [0.5][:nnz]
+    _check(sa, _wl("spttm_ttm3", "csf", (5, 4, 3), c3, v, [_dense(1, 0, 4, 16), _dense(1, 1, 3, 32)], (5, 16, 32)))
+    _check(sa, _wl("spttm_ttm4", "csf", (5, 4, 3, 2), c4, v,
+                   [_dense(1, 0, 4, 16), _dense(1, 1, 3, 16), _dense(1, 2, 2, 16)], (5, 16, 16, 16)))
+    _check(sa, _wl("sddmm_spmm", "csr", (5, 4), c2, v, [_dense(1, 0, 5, 64), _dense(1, 1, 4, 64), _dense(1, 2, 4, 32)], (5, 32)))
+    w = _wl("spmm_gemm", "csr", (5, 4), c2, v, [_dense(1, 0, 4, 128), _dense(1, 1, 128, 32)], (5, 32))
+    _check(sa, w, sched=sa.SA_SCHED_ASSOC_LEFT)
+    _check(sa, w, sched=sa.SA_SCHED_ASSOC_RIGHT)
+
+
+@pytest.mark.parametrize("L,M", [(16, 16), (16, 32), (32, 16), (32, 32)])
+def test_ttm3_rank_combinations_with_empty_slices(sa, L, M):
+    dims = (40, 37, 53)
+    coords, vals = _random_coo(7, dims, 3000)
+    keep = coords[:, 0] % 3 != 1                     # every third slice empty
+    w = _wl("spttm_ttm3", "csf", dims, coords[keep], vals[keep], [_dense(2, 0, 37, L), _dense(2, 1, 53, M)], (40, L, M))
+    A, _ = _check(sa, w)
+    assert not A[1::3].any()
+
+
+def test_ttm3_one_slice_long_fibers_split_over_many_blocks(sa):
+    # a single slice of 60 000 nonzeros in 12 fibers of 5000: pieces cut inside fibers, 8 partial tiles
+    dims = (3, 12, 5000)
+    j, k = np.divmod(np.arange(60000), 5000)
+    coords = np.stack([np.full(60000, 1), j, k], axis=1)
+    vals = rng.uniform_f32(3, 1, np.arange(60000), -1.0, 1.0)
+    perm = rng.permutation(3, 3, 60000)
+    w = _wl("spttm_ttm3", "csf", dims, coords[perm], vals[perm], [_dense(3, 0, 12, 32), _dense(3, 1, 5000, 32)], (3, 32, 32))
+    A, t = _check(sa, w)
+    counts, items, fix = sa.sa_tensor_worklist(t.handle)
+    assert counts[3] >= 2 and not A[0].any() and not A[2].any()
+
+
+@pytest.mark.parametrize("n", [1, 7, 8, 9, 31, 32, 33, 63, 65, 2048, 2049, 8192, 8193, 16385])
+def test_ttm3_ragged_sizes_around_batch_and_split_thresholds(sa, n):
+    # one slice with n nonzeros in fibers of length 1, 2, 3, ... : hits batch tails, groups of 8
+    # fibers, the one-warp / one-block / many-block boundaries
+    lens = []
+    while sum(lens) < n:
+        lens.append(min(len(lens) % 11 + 1, n - sum(lens)))
+    j = np.repeat(np.arange(len(lens)), lens)
+    k = np.concatenate([np.arange(x) for x in lens])
+    dims = (2, len(lens), 12)
+    coords = np.stack([np.ones(n, np.int64), j, k], axis=1)
+    vals = rng.uniform_f32(n, 1, np.arange(n), -1.0, 1.0)
+    w = _wl("spttm_ttm3", "csf", dims, coords, vals, [_dense(4, 0, len(lens), 32), _dense(4, 1, 12, 32)], (2, 32, 32))
+    _check(sa, w)
+
+
+def test_padded_leading_dimensions(sa):
+    import torch
+    w = configs.make(1)
+    t = sa.SparseTensor(w.dims, w.coords, w.vals, sa.SA_FMT_CSF, device=0)
+    big = [torch.zeros(x.shape[0], x.shape[1] + 12, device="cuda") for x in w.dense]
+    views = []
+    for b, x in zip(big, w.dense):
+        b[:, 4:4 + x.shape[1]] = torch.from_numpy(x).cuda()
+        views.append(b[:, 4:4 + x.shape[1]])          # 16-byte aligned start, ld = cols + 12
+    out, _ = t.run(w.expr, views)
+    torch.cuda.synchronize()
+    A_ref, S_ref = oracle.evaluate(w)
+    assert_close(out.cpu().numpy().astype(np.float64), A_ref, S_ref, TOL_FP32, "padded ld")
+    # a misaligned view is refused before anything is launched
+    with pytest.raises(sa.SaError) as e:
+        t.run(w.expr, [big[0][:, 1:17], views[1]])
+    assert e.value.status == sa.SA_E_SHAPE
+
+
+@pytest.mark.parametrize("K,L", [(32, 32), (64, 128), (128, 64)])
+def test_sddmm_spmm_ranks_long_rows_and_sampled_pattern(sa, K, L):
+    import torch
+    I, J = 300, 6000
+    deg = np.zeros(I, dtype=np.int64)
+    deg[5] = 5000                                      # cut into pieces with partial rows
+    deg[6] = 4096                                      # exactly at the threshold: one item
+    deg[10:200:3] = 17
+    deg[299] = 1
+    cols = configs.distinct_children(11, 2, deg, J)
+    rows = np.repeat(np.arange(I), deg)
+    vals = rng.uniform_f32(11, 1, np.arange(rows.shape[0]), 0.0, 1.0)
+    perm = rng.permutation(11, 3, rows.shape[0])
+    coords = np.stack([rows, cols], axis=1)[perm].astype(np.int32)
+    vals = vals[perm]
+    dense = [configs.dense_normal(11, 0, I, K), configs.dense_normal(11, 1, J, K), configs.dense_normal(11, 2, J, L)]
+    w = _wl("sddmm_spmm", "csr", (I, J), coords, vals, dense, (I, L))
+    A, t = _check(sa, w)
+    assert not A[0].any() and not A[298].any()        # empty rows are +0
+    # debug schedule: sampled values land exactly on B's stored coordinates, in CSR order
+    ops = [torch.from_numpy(x).cuda() for x in dense]
+    tuples = [(x.data_ptr(), x.shape[0], x.shape[1], x.stride(0)) for x in ops]
+    need = sa.sa_workspace_size(t.handle, sa.SA_EXPR_SDDMM_SPMM, sa.SA_SCHED_DEBUG_MATERIALIZE, tuples)
+    ws = torch.full((need // 4,), float("nan"), device="cuda")
+    out, _ = t.run(w.expr, ops, sched=sa.SA_SCHED_DEBUG_MATERIALIZE, workspace=ws.view(torch.uint8))
+    torch.cuda.synchronize()
+    nnz = vals.shape[0]
+    sampled = ws[-(((nnz * 4 + 255) // 256) * 64):][:nnz].cpu().numpy().astype(np.float64)
+    _, _, P = oracle.sddmm_spmm(coords, vals, (I, J), *dense, with_sampled=True)
+    _, crd, _ = sa.sa_tensor_export(t.handle, 1, n_crd=nnz)
+    order = np.lexsort((coords[:, 1], coords[:, 0]))   # CSR order of the input entries
+    assert np.array_equal(coords[order, 1], crd)
+    Sabs = np.abs(vals[order].astype(np.float64)) * (np.abs(dense[0][coords[order, 0]].astype(np.float64)) *
+                                                     np.abs(dense[1][coords[order, 1]].astype(np.float64))).sum(axis=1)
+    assert np.isfinite(sampled).all() and (np.abs(sampled - P[order]) <= TOL_FP32 * Sabs).all()
+    assert_close(out.cpu().numpy().astype(np.float64), *oracle.evaluate(w), TOL_FP32, "materialize schedule output")
+
+
+@pytest.mark.parametrize("L,M", [(128, 32), (128, 64), (256, 32)])
+def test_spmm_gemm_rank_combinations_and_long_rows(sa, L, M):
+    I, J = 500, 6000
+    deg = np.full(I, 3, dtype=np.int64)
+    deg[::7] = 0
+    deg[123] = 2900
+    deg[124] = 5000                                    # above the long-row threshold: pieces + fix-up
+    cols = configs.distinct_children(12, 2, deg, J)
+    rows = np.repeat(np.arange(I), deg)
+    vals = rng.uniform_f32(12, 1, np.arange(rows.shape[0]), -1.0, 1.0)
+    coords = np.stack([rows, cols], axis=1).astype(np.int32)
+    w = _wl("spmm_gemm", "csr", (I, J), coords, vals,
+            [configs.dense_normal(12, 0, J, L), configs.dense_normal(12, 1, L, M)], (I, M))
+    _check(sa, w, sched=sa.SA_SCHED_ASSOC_LEFT)
+    _check(sa, w, sched=sa.SA_SCHED_ASSOC_RIGHT)
+
+
+def test_ttm4_ragged_and_split_slices(sa):
+    w = configs.make_ttm4_zipf("edge4", 31, 90, 60, 50, 45, 150_000, 1.4, 5.0, 16, 16, 16)
+    A, t = _check(sa, w)
+    counts, _, fix = sa.sa_tensor_worklist(t.handle)
+    assert counts[3] >= 2, "the head slice must be split over several thread blocks"
+
+
+def test_results_are_reproducible_run_to_run(sa):
+    w = configs.make(2, "mini")
+    A1, t = run_gpu(sa, w)
+    A2, _ = run_gpu(sa, w, tensor=t)
+    assert np.array_equal(A1, A2)
+
+
+def test_workspace_errors_enqueue_nothing(sa):
+    import torch
+    w = configs.make(2, "mini")
+    t = sa.SparseTensor(w.dims, w.coords, w.vals, sa.SA_FMT_CSF, device=0)
+    ops = [torch.from_numpy(x).cuda() for x in w.dense]
+    tuples = [(x.data_ptr(), x.shape[0], x.shape[1], x.stride(0)) for x in ops]
+    need = sa.sa_workspace_size(t.handle, sa.SA_EXPR_SPTTM_TTM3, sa.SA_SCHED_DEFAULT, tuples)
+    assert need > 0
+    out = torch.zeros(w.out_shape, device="cuda")
+    small = torch.empty(need - 256, dtype=torch.uint8, device="cuda")
+    s = torch.cuda.current_stream().cuda_stream
+    for ws_ptr, ws_bytes in [(small.data_ptr(), small.numel()), (None, 0), (small.data_ptr() + 16, need)]:
+        with pytest.raises(sa.SaError) as e:
+            sa.sa_run(t.handle, sa.SA_EXPR_SPTTM_TTM3, sa.SA_SCHED_DEFAULT, tuples, out.data_ptr(), ws_ptr, ws_bytes, s)
+        assert e.value.status == sa.SA_E_WORKSPACE
+    torch.cuda.synchronize()
+    assert not out.any()
+    assert sa.sa_last_device_status(t.handle, s) == sa.SA_OK
