@@ -352,6 +352,9 @@ void build_csr(sa_tensor *t, sa_worklist &wl, int64_t target_nnz, int64_t max_ro
         if (r + 1 - r0 >= max_rows) flush(r + 1);
     }
     flush(I);
+    // longest first: the tail of the launch is then made of the cheapest items
+    std::stable_sort(ranges.begin(), ranges.end(),
+                     [](const sa_item &a, const sa_item &b) { return (a.p1 - a.p0) > (b.p1 - b.p0); });
     wl.n_group_ctas = 0;
     wl.items = std::move(longs);
     wl.items.insert(wl.items.end(), ranges.begin(), ranges.end());
@@ -364,7 +367,7 @@ void sa_build_worklists(sa_tensor *t)
     if (t->fmt == SA_FMT_CSF && t->order == 3) build_ttm3(t, t->wl_main);
     if (t->fmt == SA_FMT_CSF && t->order == 4) build_ttm4(t, t->wl_main);
     if (t->fmt == SA_FMT_CSR) {
-        build_csr(t, t->wl_main, 512, 64, 4096, 2048);   // fused SDDMM -> SpMM
+        build_csr(t, t->wl_main, 256, 32, 1024, 512);    // fused SDDMM -> SpMM
         build_csr(t, t->wl_aux, 256, 16, 4096, 2048);    // SpMM -> GEMM (both orders)
     }
 }

@@ -2,79 +2,183 @@
 // fused nest  i, j' < t ; k: t += B(i,j) C(i,k) D(j,k) , l: A(i,l) += t E(j,l) >  of the paper's
 // Table of kernels (Section 6): the sampled value is a scalar temporary that is consumed at once,
 // the sampled matrix is never written (auxiliary memory 1 in the paper's memory table).
+//
+// One warp per work item (a range of short rows, or a piece of a long row).  The rows D(j,:) and
+// E(j,:) of the item's nonzeros are gathered with cp.async into a per-warp ring of shared-memory
+// stages that runs ahead of the arithmetic, so that the random row reads (the HBM-bound part: D
+// and E exceed L2) stay in flight while earlier nonzeros are consumed.  K/4 lanes share one
+// nonzero (a float4 of D each, shuffle reduction of the dot product), 32/(K/4) nonzeros per step.
 #include "sa_device.cuh"
 
 namespace {
 
-// One warp per work item; a lane owns KV = K/32 consecutive k and LV = L/32 consecutive l.
-template <int KV, int LV>
-__global__ void __launch_bounds__(256)
+__device__ __forceinline__ void cp_async16(float *dst_smem, const float *src)
+{
+    const uint32_t d = static_cast<uint32_t>(__cvta_generic_to_shared(dst_smem));
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+template <int K, int L>
+struct sd_cfg {
+    static constexpr int LPN = K / 4;                 // lanes per nonzero
+    static constexpr int NPS = 32 / LPN;              // nonzeros per step
+    static constexpr int EV = L / LPN;                // floats of E(j,:) and of the output row per lane
+    static constexpr int ROWF = K + L;                // floats staged per nonzero: D(j,:) then E(j,:)
+    static constexpr int R = ROWF <= 128 ? 8 : 4;     // nonzeros per stage
+    static constexpr int NS = 3;                      // stages per warp: one being consumed, two in flight
+    static constexpr int STAGE = R * ROWF;            // floats per stage
+    static constexpr int CPL = STAGE / 4 / 32;        // 16-byte copies per lane per stage
+    static_assert(STAGE % 128 == 0 && R % NPS == 0 && 32 % R == 0, "stage shape");
+};
+
+template <int K, int L>
+__global__ void __launch_bounds__(256, 2)
 sddmm_spmm_kernel(const sa_item *__restrict__ items, int64_t n_items, const int32_t *__restrict__ pos,
                   const int32_t *__restrict__ crd, const float *__restrict__ vals, const float *__restrict__ C,
                   int64_t ldc, const float *__restrict__ D, int64_t ldd, const float *__restrict__ E, int64_t lde,
                   float *__restrict__ out, float *__restrict__ partial, float *__restrict__ sampled)
 {
-    constexpr int L = LV * 32;
+    using G = sd_cfg<K, L>;
+    extern __shared__ __align__(16) float smem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t idx = int64_t(blockIdx.x) * SA_WARPS_PER_CTA + warp;
     if (idx >= n_items) return;
+    float *ring = smem + warp * (G::NS * G::STAGE);
     const sa_item it = items[idx];
-    for (int r = it.out_row; r < it.row_end; ++r) {
-        const int a = it.dest >= 0 ? it.p0 : pos[r];
-        const int b = it.dest >= 0 ? it.p1 : pos[r + 1];
-        float c[KV], acc[LV];
+    const int P0 = it.p0, total = it.p1 - it.p0;      // the item's nonzeros are contiguous
+    const int li = lane % G::LPN, grp = lane / G::LPN;
+
+    // column indices / values of the consumer's batch of 32 nonzeros (j0, v0) and the two after it
+    int j0, j1, j2;
+    float v0, v1, v2;
+    auto load_jv = [&](int b, int &j, float &v) {
+        const int p = 32 * b + lane;
+        j = 0;
+        v = 0.f;
+        if (p < total) { j = crd[P0 + p]; v = vals[P0 + p]; }
+    };
+    int cb = 0;                                       // batch the consumer is in
+    auto issue_stage = [&](int s) {
+        if (s * G::R < total) {
+            float *dst = ring + (s % G::NS) * G::STAGE;
+            const int b = (s * G::R) >> 5;            // the stage lies inside one batch: cb or cb + 1
+            const int jsrc = b == cb ? j0 : j1;
 #pragma unroll
-        for (int q = 0; q < LV; ++q) acc[q] = 0.f;
-        if (b > a) {
-#pragma unroll
-            for (int q = 0; q < KV; ++q) c[q] = __ldg(C + int64_t(r) * ldc + lane * KV + q);
-        }
-        for (int base = a; base < b; base += 32) {
-            const int n = min(32, b - base);
-            int jj = 0;
-            float vv = 0.f;
-            if (lane < n) { jj = crd[base + lane]; vv = vals[base + lane]; }
-#pragma unroll 4
-            for (int s = 0; s < n; ++s) {
-                const int j = __shfl_sync(SA_FULL_MASK, jj, s);
-                const float v = __shfl_sync(SA_FULL_MASK, vv, s);
-                const float *drow = D + int64_t(j) * ldd + lane * KV;
-                const float *erow = E + int64_t(j) * lde + lane * LV;
-                float d[KV], e[LV];
-                if (KV == 4) { const float4 x = sa_ldg4(drow); d[0] = x.x; d[1] = x.y; d[2 % KV] = x.z; d[3 % KV] = x.w; }
-                else if (KV == 2) { const float2 x = sa_ldg2(drow); d[0] = x.x; d[1 % KV] = x.y; }
-                else d[0] = __ldg(drow);
-                if (LV == 4) { const float4 x = sa_ldg4(erow); e[0] = x.x; e[1] = x.y; e[2 % LV] = x.z; e[3 % LV] = x.w; }
-                else if (LV == 2) { const float2 x = sa_ldg2(erow); e[0] = x.x; e[1 % LV] = x.y; }
-                else e[0] = __ldg(erow);
-                float dot = 0.f;
-#pragma unroll
-                for (int q = 0; q < KV; ++q) dot = fmaf(c[q], d[q], dot);
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(SA_FULL_MASK, dot, o);
-                const float sc = v * dot;
-                if (sampled != nullptr && lane == 0) sampled[base + s] = sc;
-#pragma unroll
-                for (int q = 0; q < LV; ++q) acc[q] = fmaf(sc, e[q], acc[q]);
+            for (int q = 0; q < G::CPL; ++q) {
+                const int x = q * 32 + lane;
+                const int r = x / (G::ROWF / 4), cc = x % (G::ROWF / 4);
+                const int j = __shfl_sync(SA_FULL_MASK, jsrc, (s * G::R + r) & 31);   // 0 beyond the item: row 0
+                const float *src = cc < K / 4 ? D + int64_t(j) * ldd + cc * 4 : E + int64_t(j) * lde + (cc - K / 4) * 4;
+                cp_async16(dst + r * G::ROWF + cc * 4, src);
             }
         }
-        float *dst = it.dest >= 0 ? partial + int64_t(it.dest) * L : out + int64_t(r) * L;
+        cp_async_commit();
+    };
+    load_jv(0, j0, v0);
+    load_jv(1, j1, v1);
+    load_jv(2, j2, v2);
 #pragma unroll
-        for (int q = 0; q < LV; ++q) dst[lane * LV + q] = acc[q];
+    for (int s = 0; s < G::NS - 1; ++s) issue_stage(s);
+    int cur_stage = -1;
+    // called when the consumer first touches stage s: refill the stage it left, wait for s
+    auto enter = [&](int s) {
+        __syncwarp();
+        if (s > 0 && ((s * G::R) & 31) == 0) {
+            j0 = j1; j1 = j2;
+            v0 = v1; v1 = v2;
+            ++cb;
+            load_jv(cb + 2, j2, v2);
+        }
+        issue_stage(s + G::NS - 1);
+        cp_async_wait<G::NS - 1>();
+        __syncwarp();
+        cur_stage = s;
+    };
+
+    const bool piece = it.dest >= 0;
+    for (int r = it.out_row; r < it.row_end; ++r) {
+        const int a = piece ? 0 : pos[r] - P0;
+        const int b = piece ? total : pos[r + 1] - P0;
+        float acc[G::EV];
+#pragma unroll
+        for (int q = 0; q < G::EV; ++q) acc[q] = 0.f;
+        if (b > a) {
+            const float4 c4 = sa_ldg4(C + int64_t(r) * ldc + 4 * li);
+            for (int base = (a / G::NPS) * G::NPS; base < b; base += G::NPS) {
+                const int st = base / G::R;
+                if (st != cur_stage) enter(st);
+                const int prel = base + grp;
+                const bool active = prel >= a && prel < b;
+                const float v = __shfl_sync(SA_FULL_MASK, v0, prel & 31);
+                const float *slot = ring + (st % G::NS) * G::STAGE + (prel % G::R) * G::ROWF;
+                const float4 d4 = *reinterpret_cast<const float4 *>(slot + 4 * li);
+                float dot = fmaf(c4.x, d4.x, fmaf(c4.y, d4.y, fmaf(c4.z, d4.z, c4.w * d4.w)));
+#pragma unroll
+                for (int o = G::LPN / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(SA_FULL_MASK, dot, o);
+                if (active) {
+                    const float sc = v * dot;
+                    if (sampled != nullptr && li == 0) sampled[P0 + prel] = sc;
+                    const float *e = slot + K + li * G::EV;
+                    if (G::EV >= 4) {
+#pragma unroll
+                        for (int q = 0; q < G::EV; q += 4) {
+                            const float4 e4 = *reinterpret_cast<const float4 *>(e + q);
+                            acc[q] = fmaf(sc, e4.x, acc[q]);
+                            acc[(q + 1) % G::EV] = fmaf(sc, e4.y, acc[(q + 1) % G::EV]);
+                            acc[(q + 2) % G::EV] = fmaf(sc, e4.z, acc[(q + 2) % G::EV]);
+                            acc[(q + 3) % G::EV] = fmaf(sc, e4.w, acc[(q + 3) % G::EV]);
+                        }
+                    } else if (G::EV == 2) {
+                        const float2 e2 = *reinterpret_cast<const float2 *>(e);
+                        acc[0] = fmaf(sc, e2.x, acc[0]);
+                        acc[1 % G::EV] = fmaf(sc, e2.y, acc[1 % G::EV]);
+                    } else {
+                        acc[0] = fmaf(sc, e[0], acc[0]);
+                    }
+                }
+            }
+            // the NPS groups of lanes hold partial rows: add them up
+#pragma unroll
+            for (int o = 16; o >= G::LPN; o >>= 1)
+#pragma unroll
+                for (int q = 0; q < G::EV; ++q) acc[q] += __shfl_xor_sync(SA_FULL_MASK, acc[q], o);
+        }
+        if (grp == 0) {
+            float *dst = (piece ? partial + int64_t(it.dest) * L : out + int64_t(r) * L) + li * G::EV;
+            if (G::EV >= 4) {
+#pragma unroll
+                for (int q = 0; q < G::EV; q += 4)
+                    *reinterpret_cast<float4 *>(dst + q) =
+                        make_float4(acc[q], acc[(q + 1) % G::EV], acc[(q + 2) % G::EV], acc[(q + 3) % G::EV]);
+            } else if (G::EV == 2) {
+                *reinterpret_cast<float2 *>(dst) = make_float2(acc[0], acc[1 % G::EV]);
+            } else {
+                dst[0] = acc[0];
+            }
+        }
     }
+    cp_async_wait<0>();
 }
 
-template <int KV, int LV>
+template <int K, int L>
 cudaError_t launch(const sa_tensor *t, const sa_dense *ops, float *out, float *partial, float *sampled,
                    cudaStream_t stream)
 {
+    using G = sd_cfg<K, L>;
     const sa_worklist &wl = t->wl_main;
     const int64_t n_items = int64_t(wl.items.size());
     const int64_t ctas = (n_items + SA_WARPS_PER_CTA - 1) / SA_WARPS_PER_CTA;
     if (ctas == 0) return cudaSuccess;
-    sddmm_spmm_kernel<KV, LV><<<(unsigned)ctas, 256, 0, stream>>>(wl.d_items, n_items, t->d_pos[1], t->d_crd[1], t->d_vals,
-                                                                 ops[0].ptr, ops[0].ld, ops[1].ptr, ops[1].ld, ops[2].ptr,
-                                                                 ops[2].ld, out, partial, sampled);
+    constexpr size_t smem = size_t(SA_WARPS_PER_CTA) * G::NS * G::STAGE * sizeof(float);
+    auto kern = sddmm_spmm_kernel<K, L>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess)
+        return cudaGetLastError();
+    kern<<<(unsigned)ctas, 256, smem, stream>>>(wl.d_items, n_items, t->d_pos[1], t->d_crd[1], t->d_vals, ops[0].ptr,
+                                               ops[0].ld, ops[1].ptr, ops[1].ld, ops[2].ptr, ops[2].ld, out, partial,
+                                               sampled);
     return cudaGetLastError();
 }
 
@@ -101,9 +205,9 @@ sa_status sa_launch_sddmm_spmm(const sa_tensor *t, const sa_dense *ops, float *o
     if (materialize)
         sampled = reinterpret_cast<float *>(static_cast<char *>(ws) + sa_align256(size_t(t->wl_main.n_slots) * size_t(L) * sizeof(float)));
     cudaError_t e = cudaErrorInvalidValue;
-    const int kv = int(K / 32), lv = int(L / 32);
-#define SA_CASE(a, b) if (kv == a && lv == b) e = launch<a, b>(t, ops, out, partial, sampled, stream);
-    SA_CASE(1, 1) SA_CASE(1, 2) SA_CASE(1, 4) SA_CASE(2, 1) SA_CASE(2, 2) SA_CASE(2, 4) SA_CASE(4, 1) SA_CASE(4, 2) SA_CASE(4, 4)
+#define SA_CASE(a, b) if (K == a && L == b) e = launch<a, b>(t, ops, out, partial, sampled, stream);
+    SA_CASE(32, 32) SA_CASE(32, 64) SA_CASE(32, 128) SA_CASE(64, 32) SA_CASE(64, 64) SA_CASE(64, 128)
+    SA_CASE(128, 32) SA_CASE(128, 64) SA_CASE(128, 128)
 #undef SA_CASE
     if (e != cudaSuccess) return SA_E_CUDA;
     *launches = t->wl_main.items.empty() ? 0 : 1;

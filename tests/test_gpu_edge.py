@@ -120,7 +120,7 @@ def test_sddmm_spmm_ranks_long_rows_and_sampled_pattern(sa, K, L):
     I, J = 300, 6000
     deg = np.zeros(I, dtype=np.int64)
     deg[5] = 5000                                      # cut into pieces with partial rows
-    deg[6] = 4096                                      # exactly at the threshold: one item
+    deg[6] = 1024                                      # exactly at the threshold: one item
     deg[10:200:3] = 17
     deg[299] = 1
     cols = configs.distinct_children(11, 2, deg, J)
