@@ -11,6 +11,10 @@
 
 namespace {
 
+#ifndef SA_GEMM_NPROD
+#define SA_GEMM_NPROD 3
+#endif
+
 // Row (L floats in shared memory) times D (L x M in shared memory); lane owns m = lane + 32*q.
 template <int L, int M>
 __device__ __forceinline__ void row_times_D(const float *__restrict__ Ts, const float *__restrict__ Ds, int lane,
@@ -101,31 +105,143 @@ spmm_gemm_left_kernel(const sa_item *__restrict__ items, int64_t n_items, const 
     }
 }
 
-// E(j,:) = C(j,:) . D for all J rows; one warp per row, grid-stride.
-template <int L, int M>
-__global__ void __launch_bounds__(256)
-gemm_rows_kernel(int64_t J, const float *__restrict__ C, int64_t ldc, const float *__restrict__ D, int64_t ldd,
+// ---- E = C . D on tensor cores (dense stage of ASSOC_RIGHT) -----------------------------------
+// Thread block: 128 rows of C x all M columns, 8 warps as 4 (rows) x 2 (columns), warp tile
+// 32 x M/2.  D stays in shared memory for the whole (persistent) block, already split into its
+// TF32 high and low parts; C streams through a 3-stage cp.async ring in chunks of 32 columns.
+// NPROD = 3: hi*hi + lo*hi + hi*lo (fp32-level accuracy); NPROD = 1: a single TF32 product.
+__device__ __forceinline__ uint32_t g_tf32(float x)
+{
+    uint32_t r;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
+    return r;
+}
+__device__ __forceinline__ void g_mma(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void g_cp_async16(float *dst_smem, const float *src)
+{
+    const uint32_t d = static_cast<uint32_t>(__cvta_generic_to_shared(dst_smem));
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(src) : "memory");
+}
+
+template <int L, int M, int NPROD>
+struct gemm_cfg {
+    static constexpr int BM = 128, KC = 32, NS = 3;
+    static constexpr int CS = KC + 4;                 // row stride of a C chunk (conflict-free A fragments)
+    static constexpr int DS = M + 8;                  // row stride of D (conflict-free B fragments)
+    static constexpr int NT = M / 16;                 // n8 tiles per warp (warp covers M/2 columns)
+    static constexpr int D_FLOATS = L * DS * (NPROD == 3 ? 2 : 1);
+    static constexpr int STAGE = BM * CS;
+    static constexpr size_t SMEM = size_t(D_FLOATS + NS * STAGE) * sizeof(float);
+};
+
+template <int L, int M, int NPROD>
+__global__ void __launch_bounds__(256, 1)
+gemm_tf32_kernel(int64_t J, const float *__restrict__ C, int64_t ldc, const float *__restrict__ D, int64_t ldd,
                  float *__restrict__ Eout)
 {
-    constexpr int LV4 = L / 128, MV = M / 32;
+    using G = gemm_cfg<L, M, NPROD>;
     extern __shared__ __align__(16) float smem[];
-    float *Ds = smem;
+    uint32_t *Dh = reinterpret_cast<uint32_t *>(smem);
+    uint32_t *Dl = Dh + L * G::DS;                     // only with NPROD == 3
+    float *Cs = smem + G::D_FLOATS;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    float *Ts = smem + L * M + warp * L;
-    load_D<L, M>(Ds, D, ldd);
-    __syncthreads();
-    for (int64_t j = int64_t(blockIdx.x) * SA_WARPS_PER_CTA + warp; j < J; j += int64_t(gridDim.x) * SA_WARPS_PER_CTA) {
-        const float *crow = C + j * ldc + lane * 4;
-#pragma unroll
-        for (int q = 0; q < LV4; ++q)
-            *reinterpret_cast<float4 *>(Ts + q * 128 + lane * 4) = __ldcs(reinterpret_cast<const float4 *>(crow + q * 128));
-        __syncwarp();
-        float o[MV];
-        row_times_D<L, M>(Ts, Ds, lane, o);
-        __syncwarp();
-#pragma unroll
-        for (int q = 0; q < MV; ++q) Eout[j * M + q * 32 + lane] = o[q];
+    const int g = lane >> 2, t = lane & 3;
+    const int wr = warp >> 1, wc = warp & 1;           // warp tile: rows 32*wr.., columns (M/2)*wc..
+    for (int x = threadIdx.x; x < L * M; x += 256) {
+        const int l = x / M, m = x % M;
+        const float d = __ldg(D + int64_t(l) * ldd + m);
+        const uint32_t hi = g_tf32(d);
+        Dh[l * G::DS + m] = hi;
+        if (NPROD == 3) Dl[l * G::DS + m] = g_tf32(d - __uint_as_float(hi));
     }
+    const int64_t n_tiles = (J + G::BM - 1) / G::BM;
+    const int64_t my_tiles = blockIdx.x < n_tiles ? (n_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+    constexpr int KCH = L / G::KC;                     // chunks per row tile
+    const int64_t n_chunks = my_tiles * KCH;
+    // chunk q of this block: row tile blockIdx.x + (q / KCH) * gridDim.x, columns (q % KCH) * KC ..
+    auto issue = [&](int64_t q) {
+        if (q < n_chunks) {
+            const int64_t row0 = (int64_t(blockIdx.x) + (q / KCH) * gridDim.x) * G::BM;
+            const int k0 = int(q % KCH) * G::KC;
+            float *dst = Cs + int(q % G::NS) * G::STAGE;
+#pragma unroll
+            for (int x = threadIdx.x; x < G::BM * (G::KC / 4); x += 256) {
+                const int r = x / (G::KC / 4), c4 = x % (G::KC / 4);
+                const int64_t row = min(row0 + r, J - 1);            // rows past the end re-read the last row
+                g_cp_async16(dst + r * G::CS + c4 * 4, C + row * ldc + k0 + c4 * 4);
+            }
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    issue(0);
+    issue(1);
+    __syncthreads();                                   // D is in place
+    float acc[2][G::NT][4];
+    for (int64_t q = 0; q < n_chunks; ++q) {
+        const int kc = int(q % KCH);
+        if (kc == 0) {
+#pragma unroll
+            for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+                for (int nt = 0; nt < G::NT; ++nt)
+#pragma unroll
+                    for (int z = 0; z < 4; ++z) acc[mt][nt][z] = 0.f;
+        }
+        asm volatile("cp.async.wait_group 1;" ::: "memory");
+        __syncthreads();                               // chunk q landed for everyone; chunk q-1 fully consumed
+        issue(q + 2);
+        const float *cs = Cs + int(q % G::NS) * G::STAGE + (32 * wr) * G::CS;
+        const uint32_t *dh = Dh + (kc * G::KC) * G::DS + (M / 2) * wc;
+        const uint32_t *dl = Dl + (kc * G::KC) * G::DS + (M / 2) * wc;
+#pragma unroll
+        for (int kt = 0; kt < G::KC / 8; ++kt) {
+            uint32_t ah[2][4], al[2][4];
+#pragma unroll
+            for (int mt = 0; mt < 2; ++mt) {
+                const float *p = cs + (16 * mt + g) * G::CS + 8 * kt + t;
+                const float x0 = p[0], x1 = p[8 * G::CS], x2 = p[4], x3 = p[8 * G::CS + 4];
+                ah[mt][0] = g_tf32(x0); ah[mt][1] = g_tf32(x1); ah[mt][2] = g_tf32(x2); ah[mt][3] = g_tf32(x3);
+                if (NPROD == 3) {
+                    al[mt][0] = g_tf32(x0 - __uint_as_float(ah[mt][0]));
+                    al[mt][1] = g_tf32(x1 - __uint_as_float(ah[mt][1]));
+                    al[mt][2] = g_tf32(x2 - __uint_as_float(ah[mt][2]));
+                    al[mt][3] = g_tf32(x3 - __uint_as_float(ah[mt][3]));
+                }
+            }
+#pragma unroll
+            for (int nt = 0; nt < G::NT; ++nt) {
+                const int off = (8 * kt + t) * G::DS + 8 * nt + g;
+                const uint32_t bh0 = dh[off], bh1 = dh[off + 4 * G::DS];
+#pragma unroll
+                for (int mt = 0; mt < 2; ++mt) {
+                    if (NPROD == 3) {
+                        const uint32_t bl0 = dl[off], bl1 = dl[off + 4 * G::DS];
+                        g_mma(acc[mt][nt], al[mt], bh0, bh1);
+                        g_mma(acc[mt][nt], ah[mt], bl0, bl1);
+                    }
+                    g_mma(acc[mt][nt], ah[mt], bh0, bh1);
+                }
+            }
+        }
+        if (kc == KCH - 1) {
+            const int64_t row0 = (int64_t(blockIdx.x) + (q / KCH) * gridDim.x) * G::BM + 32 * wr;
+#pragma unroll
+            for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+                for (int nt = 0; nt < G::NT; ++nt) {
+                    const int64_t r = row0 + 16 * mt + g;
+                    const int col = (M / 2) * wc + 8 * nt + 2 * t;
+                    if (r < J) *reinterpret_cast<float2 *>(Eout + r * M + col) = make_float2(acc[mt][nt][0], acc[mt][nt][1]);
+                    if (r + 8 < J) *reinterpret_cast<float2 *>(Eout + (r + 8) * M + col) = make_float2(acc[mt][nt][2], acc[mt][nt][3]);
+                }
+        }
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
 }
 
 // A = B . E (the CSR SpMM nest of Fig. 1b); lane owns MV = M/32 consecutive columns.
@@ -208,11 +324,11 @@ sa_status run(const sa_tensor *t, const sa_dense *ops, float *out, void *ws, boo
     const int64_t J = t->dims[1];
     float *E = static_cast<float *>(ws);
     float *partial = reinterpret_cast<float *>(static_cast<char *>(ws) + sa_align256(size_t(J) * M * sizeof(float)));
-    auto gk = gemm_rows_kernel<L, M>;
-    if (cudaFuncSetAttribute(gk, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess) return SA_E_CUDA;
-    const int64_t gctas = std::min<int64_t>((J + SA_WARPS_PER_CTA - 1) / SA_WARPS_PER_CTA,
-                                            resident_ctas(reinterpret_cast<const void *>(gk), smem));
-    gk<<<(unsigned)gctas, 256, smem, stream>>>(J, ops[0].ptr, ops[0].ld, ops[1].ptr, ops[1].ld, E);
+    using GC = gemm_cfg<L, M, SA_GEMM_NPROD>;
+    auto gk = gemm_tf32_kernel<L, M, SA_GEMM_NPROD>;
+    if (cudaFuncSetAttribute(gk, cudaFuncAttributeMaxDynamicSharedMemorySize, int(GC::SMEM)) != cudaSuccess) return SA_E_CUDA;
+    const int64_t gctas = std::min<int64_t>((J + GC::BM - 1) / GC::BM, resident_ctas(reinterpret_cast<const void *>(gk), GC::SMEM));
+    gk<<<(unsigned)gctas, 256, GC::SMEM, stream>>>(J, ops[0].ptr, ops[0].ld, ops[1].ptr, ops[1].ld, E);
     if (cudaGetLastError() != cudaSuccess) return SA_E_CUDA;
     *launches += 1;
     const int64_t ctas = (n_items + SA_WARPS_PER_CTA - 1) / SA_WARPS_PER_CTA;
