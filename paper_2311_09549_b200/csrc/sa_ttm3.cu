@@ -50,21 +50,28 @@ struct cfg {
     static constexpr int RS = M + 8;        // row stride of a warp's tile in the CTA reduction
     static constexpr int NS = 3;            // cp.async stages (batches of 32 factor rows) per warp
     static constexpr int STAGE = 32 * M;    // floats per stage
-    static constexpr int WORK = NS * STAGE + 16 * TS;                      // stages + ring of staged temporaries
+    static constexpr int WORK = NS * STAGE + 16 * TS + 32;                 // stages + ring of temporaries + values of a batch
     static constexpr int WARP_SMEM = (L * RS > WORK ? L * RS : WORK);      // floats per warp
 };
 
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+__device__ __forceinline__ void cp_async16_raw(uint32_t dst_smem, const void *src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst_smem), "l"(src) : "memory");
+}
+
 // Gather the 32 rows D(k_s, :) of one batch into a stage: LPR lanes copy one row in 16-byte pieces.
+// dst_lane: shared address of the stage plus this lane's (row-in-group, piece) offset; src_lane: D plus
+// the lane's piece offset; row_bytes = 4 * ld(D) (byte offsets fit 32 bits, checked by the launcher).
 template <int M>
-__device__ __forceinline__ void stage_rows(float *stage, int kbatch, const float *__restrict__ D, int64_t ldd, int lane)
+__device__ __forceinline__ void stage_rows(uint32_t dst_lane, int kbatch, const char *__restrict__ src_lane,
+                                           uint32_t row_bytes, int r)
 {
     constexpr int LPR = M / 4, RPI = 32 / LPR;
-    const int r = lane / LPR, c = lane % LPR;
 #pragma unroll
     for (int q = 0; q < 32 / RPI; ++q) {
-        const int row = q * RPI + r;
-        const int k = __shfl_sync(SA_FULL_MASK, kbatch, row) & 0x7fffffff;
-        cp_async16(stage + row * M + c * 4, D + int64_t(k) * ldd + c * 4);
+        const uint32_t k = uint32_t(__shfl_sync(SA_FULL_MASK, kbatch, q * RPI + r)) & 0x7fffffffu;
+        cp_async16_raw(dst_lane + q * RPI * M * 4, src_lane + k * row_bytes);
     }
 }
 
@@ -105,8 +112,8 @@ __device__ __forceinline__ void ttm3_flush(float (&acc)[cfg<L, M>::MT][cfg<L, M>
 template <int L, int M>
 __device__ __forceinline__ void ttm3_warp_item(const sa_item &it, const int32_t *__restrict__ crd_j,
                                                const int32_t *__restrict__ kflag, const float *__restrict__ vals,
-                                               const float *__restrict__ C, int64_t ldc, const float *__restrict__ D,
-                                               int64_t ldd, float *__restrict__ wsm,
+                                               const float *__restrict__ C, uint32_t ldc, const float *__restrict__ D,
+                                               uint32_t ldd, float *__restrict__ wsm,
                                                float (&acc)[cfg<L, M>::MT][cfg<L, M>::NT][4])
 {
     using K = cfg<L, M>;
@@ -115,6 +122,7 @@ __device__ __forceinline__ void ttm3_warp_item(const sa_item &it, const int32_t 
     const int m = lane & (M - 1);
     const int t4 = lane & 3;
     float *Tbuf = wsm + K::NS * K::STAGE;
+    float *vs = Tbuf + 16 * K::TS;                  // values of the batch being consumed
 #pragma unroll
     for (int mt = 0; mt < K::MT; ++mt)
 #pragma unroll
@@ -124,31 +132,52 @@ __device__ __forceinline__ void ttm3_warp_item(const sa_item &it, const int32_t 
     if (it.p0 >= it.p1) return;
     const int p0 = it.p0, p1 = it.p1, f0 = it.f0, fmax = it.f1 - 1;
     const int nb = (p1 - p0 + 31) >> 5;
-    auto load_kv = [&](int b, int &k, float &v) {
-        const int p = p0 + 32 * b + lane;
+    // per-lane constants of the row gather
+    constexpr int LPR = M / 4;
+    const int gr = lane / LPR, gc = lane % LPR;
+    const uint32_t dst_lane = smem_u32(wsm) + uint32_t(gr * M + gc * 4) * 4u;
+    const char *src_lane = reinterpret_cast<const char *>(D + gc * 4);
+    const uint32_t row_bytes = ldd * 4u;
+    int pn = p0 + lane;                              // position this lane loads next
+    auto load_kv = [&](int &k, float &v) {
         k = 0;
         v = 0.f;
-        if (p < p1) { k = kflag[p]; v = vals[p]; }
+        if (pn < p1) { k = kflag[pn]; v = vals[pn]; }
+        pn += 32;
     };
-    // index/value registers of batches B .. B+3; row gathers of batches B+1, B+2 are in flight while B is consumed
-    int k0, k1, k2, k3;
-    float v0, v1, v2, v3;
-    load_kv(0, k0, v0);
-    load_kv(1, k1, v1);
-    load_kv(2, k2, v2);
-    load_kv(3, k3, v3);
-    stage_rows<M>(wsm, k0, D, ldd, lane);
+    // index/value registers of batches B .. B+6: the index of a batch is needed two rounds before its
+    // values (to request its rows), and a streaming load takes several rounds to arrive; row gathers
+    // of batches B+1, B+2 are in flight while B is consumed
+    int k0, k1, k2, k3, k4, k5, k6;
+    float v0, v1, v2, v3, v4, v5, v6;
+    load_kv(k0, v0);
+    load_kv(k1, v1);
+    load_kv(k2, v2);
+    load_kv(k3, v3);
+    load_kv(k4, v4);
+    load_kv(k5, v5);
+    load_kv(k6, v6);
+    stage_rows<M>(dst_lane, k0, src_lane, row_bytes, gr);
     cp_async_commit();
-    if (1 < nb) stage_rows<M>(wsm + K::STAGE, k1, D, ldd, lane);
+    if (1 < nb) stage_rows<M>(dst_lane + K::STAGE * 4, k1, src_lane, row_bytes, gr);
     cp_async_commit();
     int nclosed = 0, nflushed = 0;          // fibers closed / handed to the tensor cores so far
     int ja = crd_j[min(f0 + t4, fmax)], jb = crd_j[min(f0 + t4 + 4, fmax)];
     float T = 0.f;
     int s_cur = 0, s_issue = 2;
+    // T += v * d for one nonzero; `end` (warp-uniform) closes the fiber into the ring of temporaries
+#define SA_TTM3_STEP(v, d, end)                                   \
+    T = fmaf(v, d, T);                                            \
+    if (end) {                                                    \
+        Tbuf[(nclosed & 15) * K::TS + m] = T;                     \
+        T = 0.f;                                                  \
+        ++nclosed;                                                \
+    }
 #pragma unroll 1
     for (int b = 0; b < nb; ++b) {
-        if (b + 2 < nb) stage_rows<M>(wsm + s_issue * K::STAGE, k2, D, ldd, lane);
+        if (b + 2 < nb) stage_rows<M>(dst_lane + s_issue * (K::STAGE * 4), k2, src_lane, row_bytes, gr);
         cp_async_commit();
+        vs[lane] = v0;
         cp_async_wait<2>();
         __syncwarp();
         const float *st = wsm + s_cur * K::STAGE + m;
@@ -160,42 +189,53 @@ __device__ __forceinline__ void ttm3_warp_item(const sa_item &it, const int32_t 
         for (int c = 0; c < nchunks; ++c) {
             const unsigned e8 = (ends >> (8 * c)) & 0xffu;
             const float *sc = st + 8 * c * M;
-            if (e8 == 0) {
-#pragma unroll
-                for (int u = 0; u < 8; ++u) T = fmaf(__shfl_sync(SA_FULL_MASK, v0, 8 * c + u), sc[u * M], T);
+            const float4 va = *reinterpret_cast<const float4 *>(vs + 8 * c);
+            const float4 vb = *reinterpret_cast<const float4 *>(vs + 8 * c + 4);
+            if ((e8 & 0xfu) == 0) {
+                T = fmaf(va.x, sc[0], T);
+                T = fmaf(va.y, sc[M], T);
+                T = fmaf(va.z, sc[2 * M], T);
+                T = fmaf(va.w, sc[3 * M], T);
             } else {
-#pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    T = fmaf(__shfl_sync(SA_FULL_MASK, v0, 8 * c + u), sc[u * M], T);
-                    if (e8 & (1u << u)) {
-                        Tbuf[(nclosed & 15) * K::TS + m] = T;
-                        T = 0.f;
-                        ++nclosed;
-                    }
-                }
-                if (nclosed - nflushed >= 8) {
-                    __syncwarp();
-                    ttm3_flush<L, M>(acc, Tbuf, nflushed, C + int64_t(ja) * ldc, C + int64_t(jb) * ldc, lane);
-                    __syncwarp();
-                    nflushed += 8;
-                    ja = crd_j[min(f0 + nflushed + t4, fmax)];
-                    jb = crd_j[min(f0 + nflushed + t4 + 4, fmax)];
-                }
+                SA_TTM3_STEP(va.x, sc[0], e8 & 1u)
+                SA_TTM3_STEP(va.y, sc[M], e8 & 2u)
+                SA_TTM3_STEP(va.z, sc[2 * M], e8 & 4u)
+                SA_TTM3_STEP(va.w, sc[3 * M], e8 & 8u)
+            }
+            if ((e8 & 0xf0u) == 0) {
+                T = fmaf(vb.x, sc[4 * M], T);
+                T = fmaf(vb.y, sc[5 * M], T);
+                T = fmaf(vb.z, sc[6 * M], T);
+                T = fmaf(vb.w, sc[7 * M], T);
+            } else {
+                SA_TTM3_STEP(vb.x, sc[4 * M], e8 & 16u)
+                SA_TTM3_STEP(vb.y, sc[5 * M], e8 & 32u)
+                SA_TTM3_STEP(vb.z, sc[6 * M], e8 & 64u)
+                SA_TTM3_STEP(vb.w, sc[7 * M], e8 & 128u)
+            }
+            if (nclosed - nflushed >= 8) {
+                __syncwarp();
+                ttm3_flush<L, M>(acc, Tbuf, nflushed, C + ja * ldc, C + jb * ldc, lane);
+                __syncwarp();
+                nflushed += 8;
+                ja = crd_j[min(f0 + nflushed + t4, fmax)];
+                jb = crd_j[min(f0 + nflushed + t4 + 4, fmax)];
             }
         }
-        __syncwarp();                                   // stage s_cur is free for the gather issued next
-        k0 = k1; k1 = k2; k2 = k3;
-        v0 = v1; v1 = v2; v2 = v3;
-        load_kv(b + 4, k3, v3);
+        __syncwarp();                                   // stage s_cur and vs are free for the next round
+        k0 = k1; k1 = k2; k2 = k3; k3 = k4; k4 = k5; k5 = k6;
+        v0 = v1; v1 = v2; v2 = v3; v3 = v4; v4 = v5; v5 = v6;
+        load_kv(k6, v6);
         s_issue = s_cur;
         s_cur = s_cur == 2 ? 0 : s_cur + 1;
     }
+#undef SA_TTM3_STEP
     cp_async_wait<0>();
     const int pending = nclosed - nflushed;             // 0..7
     if (pending > 0) {
         for (int x = pending; x < 8; ++x) Tbuf[((nflushed + x) & 15) * K::TS + m] = 0.f;   // unused rows
         __syncwarp();
-        ttm3_flush<L, M>(acc, Tbuf, nflushed, C + int64_t(ja) * ldc, C + int64_t(jb) * ldc, lane);
+        ttm3_flush<L, M>(acc, Tbuf, nflushed, C + ja * ldc, C + jb * ldc, lane);
         __syncwarp();
     }
 }
@@ -203,8 +243,8 @@ __device__ __forceinline__ void ttm3_warp_item(const sa_item &it, const int32_t 
 template <int L, int M>
 __global__ void __launch_bounds__(256, 2)
 ttm3_kernel(const sa_item *__restrict__ items, int64_t n_items, int n_group_ctas, const int32_t *__restrict__ crd_j,
-            const int32_t *__restrict__ kflag, const float *__restrict__ vals, const float *__restrict__ C, int64_t ldc,
-            const float *__restrict__ D, int64_t ldd, float *__restrict__ out, float *__restrict__ partial)
+            const int32_t *__restrict__ kflag, const float *__restrict__ vals, const float *__restrict__ C, uint32_t ldc,
+            const float *__restrict__ D, uint32_t ldd, float *__restrict__ out, float *__restrict__ partial)
 {
     using K = cfg<L, M>;
     constexpr int TILE = L * M;
@@ -272,7 +312,7 @@ cudaError_t launch(const sa_tensor *t, const sa_dense *ops, float *out, float *p
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess)
         return cudaGetLastError();
     kern<<<(unsigned)ctas, 256, smem, stream>>>(wl.d_items, n_items, int(wl.n_group_ctas), t->d_crd[1], t->d_crd_endflag,
-                                               t->d_vals, ops[0].ptr, ops[0].ld, ops[1].ptr, ops[1].ld, out, partial);
+                                               t->d_vals, ops[0].ptr, uint32_t(ops[0].ld), ops[1].ptr, uint32_t(ops[1].ld), out, partial);
     return cudaGetLastError();
 }
 
@@ -290,6 +330,9 @@ sa_status sa_launch_ttm3(const sa_tensor *t, const sa_dense *ops, float *out, vo
 {
     const int64_t L = ops[0].cols, M = ops[1].cols;
     (void)ws_bytes;
+    // the kernel addresses factor rows with 32-bit byte offsets
+    for (int i = 0; i < 2; ++i)
+        if (ops[i].rows * ops[i].ld >= (int64_t(1) << 30)) return SA_E_UNSUPPORTED;
     float *partial = static_cast<float *>(ws);
     cudaError_t e;
     if (L == 16 && M == 16) e = launch<16, 16>(t, ops, out, partial, stream);
