@@ -132,9 +132,11 @@ sa_status sa_tensor_export(const sa_tensor *t, int level, int64_t *pos, int32_t 
  * second list used by SA_EXPR_SPMM_GEMM).  These are the slice / fiber / nonzero partition arrays:
  *   counts [4]: number of items, number of leading 8-item groups that one thread block reduces
  *               into a single tile, number of fix-up entries, number of partial-tile slots
- *   items  [n_items * 8] int32 per item: out_row, row_end, f0, f1, p0, p1, dest, 0 --
+ *   items  [n_items * 8] int32 per item: out_row, row_end, f0, f1, p0, p1, dest, half --
  *               fibers [f0,f1) (CSF) clipped to nonzeros [p0,p1) of slice out_row, or rows
- *               [out_row,row_end) / nonzeros [p0,p1) of a long row (CSR); dest = partial slot or -1
+ *               [out_row,row_end) / nonzeros [p0,p1) of a long row (CSR); dest = partial slot or -1;
+ *               half = 0 / 1 for order-4 tensors, whose items are listed once per half of the
+ *               last dense index (0 otherwise)
  *   fix    [n_fix * 4] int32 per entry: out_row, slot0, count, 0 -- out[out_row] = sum of `count`
  *               partial tiles from slot0 (count 0: the slice / row is empty and is zero-filled)
  * NULL outputs are skipped.

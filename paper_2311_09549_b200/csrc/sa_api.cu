@@ -188,6 +188,15 @@ sa_status sa_tensor_create(int order, const int64_t *dims, int64_t nnz, const in
                 flagged[size_t(t->pos[2][size_t(f) + 1] - 1)] |= int32_t(0x80000000u);
             s = upload(t, flagged.data(), flagged.size(), &t->d_crd_endflag);
         }
+        if (s == SA_OK && fmt == SA_FMT_CSF && order == 4 && t->dims[3] < (int64_t(1) << 30)) {
+            // bit 31: last nonzero of its (i,j,k) fiber; bit 30: last nonzero of its (i,j) fiber
+            std::vector<int32_t> flagged(t->crd[3]);
+            for (int64_t g = 0; g < t->count[2]; ++g)
+                flagged[size_t(t->pos[3][size_t(g) + 1] - 1)] |= int32_t(0x80000000u);
+            for (int64_t f = 0; f < t->count[1]; ++f)
+                flagged[size_t(t->pos[3][size_t(t->pos[2][size_t(f) + 1])] - 1)] |= int32_t(0x40000000);
+            s = upload(t, flagged.data(), flagged.size(), &t->d_crd_endflag);
+        }
         const int32_t zeros[4] = {0, 0, 0, 0};
         if (s == SA_OK) s = upload(t, zeros, 4, &t->d_status);
         if (s == SA_OK) s = upload_worklist(t, t->wl_main);

@@ -307,9 +307,13 @@ void build_ttm4(sa_tensor *t, sa_worklist &wl)
     std::stable_sort(groups.begin(), groups.end(), [](const group_rec &a, const group_rec &b) { return a.len > b.len; });
     std::stable_sort(small.begin(), small.end(),
                      [](const sa_item &a, const sa_item &b) { return (a.p1 - a.p0) > (b.p1 - b.p0); });
-    wl.n_group_ctas = int64_t(groups.size());
-    for (auto &g : groups) wl.items.insert(wl.items.end(), g.items.begin(), g.items.end());
-    wl.items.insert(wl.items.end(), small.begin(), small.end());
+    // every item is evaluated twice, once per half of the last dense index n (field pad = 0 / 1)
+    wl.n_group_ctas = 2 * int64_t(groups.size());
+    for (auto &g : groups)
+        for (int nh = 0; nh < 2; ++nh)
+            for (sa_item it : g.items) { it.pad = nh; wl.items.push_back(it); }
+    for (sa_item it : small)
+        for (int nh = 0; nh < 2; ++nh) { it.pad = nh; wl.items.push_back(it); }
     append_empty_slices(t, wl);
 }
 

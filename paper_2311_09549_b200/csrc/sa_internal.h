@@ -23,7 +23,7 @@ struct sa_item {
     int32_t f0, f1;
     int32_t p0, p1;
     int32_t dest;
-    int32_t pad;
+    int32_t pad;      // order-4 CSF: which half of the last dense index n this item covers (0 / 1)
 };
 
 // Fix-up entry: out[out_row] = sum of `count` partial tiles starting at slot0 (count == 0: zeros).
@@ -62,8 +62,9 @@ struct sa_tensor {
     int32_t *d_pos[SA_MAX_ORDER] = {nullptr, nullptr, nullptr, nullptr};
     int32_t *d_crd[SA_MAX_ORDER] = {nullptr, nullptr, nullptr, nullptr};
     float *d_vals = nullptr;
-    int32_t *d_crd_endflag = nullptr;         // order-3 CSF: last-level crd with bit 31 set on the last
-                                              // nonzero of every fiber
+    int32_t *d_crd_endflag = nullptr;         // CSF: last-level crd with bit 31 set on the last nonzero of
+                                              // every last-level fiber (order 4: bit 30 on the last nonzero
+                                              // of every (i,j) fiber as well)
     int32_t *d_status = nullptr;              // [4] device status word
 
     sa_worklist wl_main;                      // TTM3 / TTM4 / SDDMM-SpMM
