@@ -121,21 +121,11 @@ class ClockSampler:
         return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons), "samples": len(sm)}
 
 
-def oracle_sample(w, budget_s=20.0):
-    """Time the oracle, as it stands, on a bounded sample of output slices / rows of ``w``."""
+def _oracle_run(w, counts, order, target_nnz, cores):
+    """Evaluate the oracle on seeded random slices / rows holding about target_nnz nonzeros."""
     import oracle
-    I = w.dims[0]
-    per_nnz = {"spttm_ttm3": lambda: w.dense[0].shape[1] * w.dense[1].shape[1],
-               "spttm_ttm4": lambda: w.dense[0].shape[1] * w.dense[1].shape[1] * w.dense[2].shape[1],
-               "sddmm_spmm": lambda: w.dense[0].shape[1] * w.dense[2].shape[1],
-               "spmm_gemm": lambda: w.dense[0].shape[1] * w.dense[1].shape[1]}[w.expr]()
-    cores = oracle.max_threads()
-    # ~0.25 G inner iterations per second per thread is a safe guess for the plain fp64 loop
-    target_nnz = int(budget_s * 0.25e9 * cores / per_nnz)
-    counts = np.bincount(w.coords[:, 0], minlength=I)
-    order = configs.rng.permutation(w.seed, 77, I)
-    # the oracle gives one slice to one thread: leave out slices that alone would take a thread
-    # longer than the whole budget, so that the sample stays bounded
+    # the oracle gives one slice to one thread: leave out slices that alone would occupy a thread for
+    # a large part of the run, so that the sample stays bounded
     cap = max(1, target_nnz // (2 * cores))
     order = order[counts[order] <= cap]
     csum = np.cumsum(counts[order])
@@ -144,9 +134,27 @@ def oracle_sample(w, budget_s=20.0):
     nnz_sel = int(counts[sel].sum())
     t0 = time.perf_counter()
     oracle.evaluate(w, sel=sel, with_abs=False)
-    dt = time.perf_counter() - t0
+    return nnz_sel, time.perf_counter() - t0, len(sel), cap
+
+
+def oracle_sample(w, budget_s=15.0):
+    """Time the oracle, as it stands, on a bounded sample of output slices / rows of ``w``: a short
+    pilot run measures its speed on this host, the timed run is sized to take about budget_s."""
+    import oracle
+    I = w.dims[0]
+    per_nnz = {"spttm_ttm3": lambda: w.dense[0].shape[1] * w.dense[1].shape[1],
+               "spttm_ttm4": lambda: w.dense[0].shape[1] * w.dense[1].shape[1] * w.dense[2].shape[1],
+               "sddmm_spmm": lambda: w.dense[0].shape[1] * w.dense[2].shape[1],
+               "spmm_gemm": lambda: w.dense[0].shape[1] * w.dense[1].shape[1]}[w.expr]()
+    cores = oracle.max_threads()
+    counts = np.bincount(w.coords[:, 0], minlength=I)
+    order = configs.rng.permutation(w.seed, 77, I)
+    pilot_nnz = max(1000, int(0.5 * 0.25e9 * cores / per_nnz))          # ~0.5 s at a guessed rate
+    n0, t0, _, _ = _oracle_run(w, counts, order, pilot_nnz, cores)
+    rate = n0 / max(t0, 1e-3)
+    nnz_sel, dt, n_sel, cap = _oracle_run(w, counts, order, max(pilot_nnz, int(rate * budget_s)), cores)
     sample = ("%d of %d output slices/rows (seeded random among those with <= %d nonzeros), %d of %d nonzeros"
-              % (len(sel), I, cap, nnz_sel, w.nnz))
+              % (n_sel, I, cap, nnz_sel, w.nnz))
     return {"value": nnz_sel / dt / 1e9, "unit": "GNNZ/s", "cores": cores, "kind": "oracle", "sample": sample,
             "seconds": dt}
 
@@ -174,7 +182,7 @@ def workload_label(cfg, sched):
 
 
 def label(args):
-    return workload_label(args.workload, args.sched) + ("" if args.scale == "full" else " [mini-scale stand-in]")
+    return workload_label(args.workload, args.sched) + ("" if args.scale == "full" else " [%s-scale stand-in]" % args.scale)
 
 
 def run_reference(args, w, rank, world):
@@ -206,7 +214,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", type=int, default=2, choices=[1, 2, 3, 4, 5])
-    ap.add_argument("--scale", default="full", choices=["full", "mini"])
+    ap.add_argument("--scale", default="full", choices=["full", "mid", "mini"])
     ap.add_argument("--sched", default="right", choices=["left", "right"], help="association order for workload 4")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=5)

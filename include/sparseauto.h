@@ -63,7 +63,8 @@ typedef enum {
 } sa_expr;
 
 typedef enum {
-    SA_SCHED_DEFAULT = 0,      /* the host table's choice for the expression                    */
+    SA_SCHED_DEFAULT = 0,      /* the host table's choice for the expression; for SPMM_GEMM the
+                                  association order that moves fewer bytes for this tensor      */
     SA_SCHED_FUSED = 1,        /* the fissioned / fused branched nest of the Table of kernels   */
     SA_SCHED_ASSOC_LEFT = 2,   /* SA_EXPR_SPMM_GEMM only: (B.C).D, row temporary of L floats    */
     SA_SCHED_ASSOC_RIGHT = 3,  /* SA_EXPR_SPMM_GEMM only: B.(C.D), J x M temporary in workspace */

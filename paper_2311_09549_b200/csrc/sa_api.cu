@@ -108,8 +108,14 @@ sa_status check_ops(const sa_tensor *t, sa_expr expr, const sa_dense *ops, int n
 }
 
 // Host table: which concrete schedule runs for (expr, sched).  Returns false if the pair is
-// not in the table.
-bool resolve_schedule(sa_expr expr, sa_schedule sched, sa_schedule *resolved)
+// not in the table.  For SA_EXPR_SPMM_GEMM the default is chosen per tensor, in the spirit of the
+// paper's run-time Stage 4 (Section 5: the schedules that survive compile-time pruning are
+// compared with the concrete sizes plugged into their cost expressions): both association orders
+// are bound by memory traffic here, so the cost is the bytes each one must move,
+//   (B.C).D : nnz * (8 + 4 L)                     one row of C per nonzero
+//   B.(C.D) : 4 J (L + M) + nnz * (8 + 4 M)       C read and E = C.D written once, one row of E per nonzero
+// and the cheaper one runs (its J x M temporary comes out of the caller's workspace).
+bool resolve_schedule(const sa_tensor *t, sa_expr expr, sa_schedule sched, const sa_dense *ops, sa_schedule *resolved)
 {
     switch (expr) {
         case SA_EXPR_SPTTM_TTM3:
@@ -121,8 +127,13 @@ bool resolve_schedule(sa_expr expr, sa_schedule sched, sa_schedule *resolved)
             if (sched == SA_SCHED_DEBUG_MATERIALIZE) { *resolved = sched; return true; }
             return false;
         case SA_EXPR_SPMM_GEMM:
-            // default: B.(C.D) -- fewer bytes gathered per nonzero when M < L
-            if (sched == SA_SCHED_DEFAULT) { *resolved = SA_SCHED_ASSOC_RIGHT; return true; }
+            if (sched == SA_SCHED_DEFAULT) {
+                const double nnz = double(t->nnz), J = double(t->dims[1]), L = double(ops[0].cols), M = double(ops[1].cols);
+                const double left = nnz * (8.0 + 4.0 * L);
+                const double right = 4.0 * J * (L + M) + nnz * (8.0 + 4.0 * M);
+                *resolved = left <= right ? SA_SCHED_ASSOC_LEFT : SA_SCHED_ASSOC_RIGHT;
+                return true;
+            }
             if (sched == SA_SCHED_FUSED || sched == SA_SCHED_ASSOC_LEFT) { *resolved = SA_SCHED_ASSOC_LEFT; return true; }
             if (sched == SA_SCHED_ASSOC_RIGHT) { *resolved = sched; return true; }
             return false;
@@ -253,7 +264,7 @@ sa_status sa_workspace_size(const sa_tensor *t, sa_expr expr, sa_schedule sched,
     sa_status s = check_ops(t, expr, ops, n_ops, true);
     if (s != SA_OK) return s;
     sa_schedule r;
-    if (!resolve_schedule(expr, sched, &r)) return SA_E_UNSUPPORTED;
+    if (!resolve_schedule(t, expr, sched, ops, &r)) return SA_E_UNSUPPORTED;
     *bytes = workspace_bytes(t, expr, r, ops);
     return SA_OK;
 }
@@ -266,7 +277,7 @@ sa_status sa_run(const sa_tensor *t, sa_expr expr, sa_schedule sched, const sa_d
     sa_status s = check_ops(t, expr, ops, n_ops, false);
     if (s != SA_OK) return s;
     sa_schedule r;
-    if (!resolve_schedule(expr, sched, &r)) return SA_E_UNSUPPORTED;
+    if (!resolve_schedule(t, expr, sched, ops, &r)) return SA_E_UNSUPPORTED;
     const size_t need = workspace_bytes(t, expr, r, ops);
     if (need > 0 && (!workspace || ws_bytes < need || reinterpret_cast<uintptr_t>(workspace) % 256))
         return SA_E_WORKSPACE;

@@ -343,7 +343,7 @@ def make_spmm_gemm(name, seed, I, J, nnz, L, M):
 # --------------------------------------------------------------------------- presets
 
 def make(config, scale="full", seed=None):
-    """Build workload ``config`` (1..5) at ``scale`` 'full' or 'mini'."""
+    """Build workload ``config`` (1..5) at ``scale`` 'full' or 'mini' ('mid' exists for config 4 only)."""
     config = int(config)
     s = BASE_SEED + config if seed is None else int(seed)
     full = scale == "full"
@@ -360,6 +360,8 @@ def make(config, scale="full", seed=None):
     if config == 4:
         if full:
             return make_spmm_gemm("cfg4-spmm-gemm", s, 4_000_000, 4_000_000, 100_000_000, 256, 64)
+        if scale == "mid":      # a quarter of the full size: same row law, C still 8x larger than L2 (profiling case)
+            return make_spmm_gemm("cfg4-spmm-gemm-mid", s, 1_000_000, 1_000_000, 25_000_000, 256, 64)
         return make_spmm_gemm("cfg4-spmm-gemm-mini", s, 12_000, 12_000, 300_000, 256, 64)
     if config == 5:
         if full:
