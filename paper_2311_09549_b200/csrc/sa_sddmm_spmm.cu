@@ -12,10 +12,10 @@
 
 namespace {
 
-__device__ __forceinline__ void cp_async16(float *dst_smem, const float *src)
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+__device__ __forceinline__ void cp_async16_raw(uint32_t dst_smem, const void *src)
 {
-    const uint32_t d = static_cast<uint32_t>(__cvta_generic_to_shared(dst_smem));
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(src) : "memory");
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst_smem), "l"(src) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
@@ -38,7 +38,7 @@ template <int K, int L>
 __global__ void __launch_bounds__(256, 2)
 sddmm_spmm_kernel(const sa_item *__restrict__ items, int64_t n_items, const int32_t *__restrict__ pos,
                   const int32_t *__restrict__ crd, const float *__restrict__ vals, const float *__restrict__ C,
-                  int64_t ldc, const float *__restrict__ D, int64_t ldd, const float *__restrict__ E, int64_t lde,
+                  uint32_t ldc, const float *__restrict__ D, uint32_t ldd, const float *__restrict__ E, uint32_t lde,
                   float *__restrict__ out, float *__restrict__ partial, float *__restrict__ sampled)
 {
     using G = sd_cfg<K, L>;
@@ -61,20 +61,34 @@ sddmm_spmm_kernel(const sa_item *__restrict__ items, int64_t n_items, const int3
         if (p < total) { j = crd[P0 + p]; v = vals[P0 + p]; }
     };
     int cb = 0;                                       // batch the consumer is in
+    // per-lane constants of the gather: copy q of a stage moves 16-byte piece x = 32 q + lane, i.e. piece
+    // cc = x % (ROWF/4) of nonzero r = x / (ROWF/4); pieces lie in the stage in the same order (byte 16 x)
+    const char *src_q[G::CPL];                        // D or E plus the piece offset
+    uint32_t rowb_q[G::CPL];                          // bytes between rows of that operand
+    int r_q[G::CPL];
+#pragma unroll
+    for (int q = 0; q < G::CPL; ++q) {
+        const int x = q * 32 + lane;
+        const int cc = x % (G::ROWF / 4);
+        r_q[q] = x / (G::ROWF / 4);
+        src_q[q] = reinterpret_cast<const char *>(cc < K / 4 ? D + cc * 4 : E + (cc - K / 4) * 4);
+        rowb_q[q] = (cc < K / 4 ? ldd : lde) * 4u;
+    }
+    const uint32_t ring_lane = smem_u32(ring) + uint32_t(lane) * 16u;
+    int issue_slot = 0;                               // ring slot the next issued stage goes to
     auto issue_stage = [&](int s) {
         if (s * G::R < total) {
-            float *dst = ring + (s % G::NS) * G::STAGE;
+            const uint32_t dst = ring_lane + uint32_t(issue_slot * G::STAGE) * 4u;
             const int b = (s * G::R) >> 5;            // the stage lies inside one batch: cb or cb + 1
             const int jsrc = b == cb ? j0 : j1;
+            const int lane0 = (s * G::R) & 31;
 #pragma unroll
             for (int q = 0; q < G::CPL; ++q) {
-                const int x = q * 32 + lane;
-                const int r = x / (G::ROWF / 4), cc = x % (G::ROWF / 4);
-                const int j = __shfl_sync(SA_FULL_MASK, jsrc, (s * G::R + r) & 31);   // 0 beyond the item: row 0
-                const float *src = cc < K / 4 ? D + int64_t(j) * ldd + cc * 4 : E + int64_t(j) * lde + (cc - K / 4) * 4;
-                cp_async16(dst + r * G::ROWF + cc * 4, src);
+                const uint32_t j = uint32_t(__shfl_sync(SA_FULL_MASK, jsrc, lane0 + r_q[q]));   // 0 beyond the item: row 0
+                cp_async16_raw(dst + q * 512u, src_q[q] + j * rowb_q[q]);
             }
         }
+        issue_slot = issue_slot == G::NS - 1 ? 0 : issue_slot + 1;
         cp_async_commit();
     };
     load_jv(0, j0, v0);
@@ -83,9 +97,11 @@ sddmm_spmm_kernel(const sa_item *__restrict__ items, int64_t n_items, const int3
 #pragma unroll
     for (int s = 0; s < G::NS - 1; ++s) issue_stage(s);
     int cur_stage = -1;
+    int cur_off = -G::STAGE;                          // float offset of the consumer's stage in the ring
     // called when the consumer first touches stage s: refill the stage it left, wait for s
     auto enter = [&](int s) {
         __syncwarp();
+        cur_off = cur_off == (G::NS - 1) * G::STAGE ? 0 : cur_off + G::STAGE;
         if (s > 0 && ((s * G::R) & 31) == 0) {
             j0 = j1; j1 = j2;
             v0 = v1; v1 = v2;
@@ -106,14 +122,14 @@ sddmm_spmm_kernel(const sa_item *__restrict__ items, int64_t n_items, const int3
 #pragma unroll
         for (int q = 0; q < G::EV; ++q) acc[q] = 0.f;
         if (b > a) {
-            const float4 c4 = sa_ldg4(C + int64_t(r) * ldc + 4 * li);
+            const float4 c4 = sa_ldg4(C + uint32_t(r) * ldc + 4 * li);
             for (int base = (a / G::NPS) * G::NPS; base < b; base += G::NPS) {
                 const int st = base / G::R;
                 if (st != cur_stage) enter(st);
                 const int prel = base + grp;
                 const bool active = prel >= a && prel < b;
                 const float v = __shfl_sync(SA_FULL_MASK, v0, prel & 31);
-                const float *slot = ring + (st % G::NS) * G::STAGE + (prel % G::R) * G::ROWF;
+                const float *slot = ring + cur_off + (prel & (G::R - 1)) * G::ROWF;
                 const float4 d4 = *reinterpret_cast<const float4 *>(slot + 4 * li);
                 float dot = fmaf(c4.x, d4.x, fmaf(c4.y, d4.y, fmaf(c4.z, d4.z, c4.w * d4.w)));
 #pragma unroll
@@ -177,8 +193,8 @@ cudaError_t launch(const sa_tensor *t, const sa_dense *ops, float *out, float *p
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess)
         return cudaGetLastError();
     kern<<<(unsigned)ctas, 256, smem, stream>>>(wl.d_items, n_items, t->d_pos[1], t->d_crd[1], t->d_vals, ops[0].ptr,
-                                               ops[0].ld, ops[1].ptr, ops[1].ld, ops[2].ptr, ops[2].ld, out, partial,
-                                               sampled);
+                                               uint32_t(ops[0].ld), ops[1].ptr, uint32_t(ops[1].ld), ops[2].ptr,
+                                               uint32_t(ops[2].ld), out, partial, sampled);
     return cudaGetLastError();
 }
 
@@ -202,6 +218,8 @@ sa_status sa_launch_sddmm_spmm(const sa_tensor *t, const sa_dense *ops, float *o
     const int64_t K = ops[0].cols, L = ops[2].cols;
     float *partial = static_cast<float *>(ws);
     float *sampled = nullptr;
+    for (int i = 0; i < 3; ++i)                       // the kernel addresses dense rows with 32-bit byte offsets
+        if (ops[i].rows * ops[i].ld >= (int64_t(1) << 30)) return SA_E_UNSUPPORTED;
     if (materialize)
         sampled = reinterpret_cast<float *>(static_cast<char *>(ws) + sa_align256(size_t(t->wl_main.n_slots) * size_t(L) * sizeof(float)));
     cudaError_t e = cudaErrorInvalidValue;
