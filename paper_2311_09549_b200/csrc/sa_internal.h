@@ -2,6 +2,7 @@
 #pragma once
 
 #include <cuda_runtime.h>
+#include <atomic>
 #include <cstdint>
 #include <vector>
 
@@ -70,7 +71,7 @@ struct sa_tensor {
     sa_worklist wl_main;                      // TTM3 / TTM4 / SDDMM-SpMM
     sa_worklist wl_aux;                       // CSR: SpMM-GEMM row items
 
-    mutable int last_launches = 0;
+    mutable std::atomic<int> last_launches{0};   // the only mutable field: concurrent sa_run calls may write it
     std::vector<void *> dev_blocks;           // everything obtained from the allocator
 };
 

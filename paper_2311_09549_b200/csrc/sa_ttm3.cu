@@ -75,12 +75,27 @@ __device__ __forceinline__ void stage_rows(uint32_t dst_lane, int kbatch, const 
     }
 }
 
-// acc += Cg^T . T for eight staged fibers: rows (row0 + x) & 15, x = 0..7, of the 16-row ring;
-// crow_a / crow_b: rows of C of the fibers x = t and x = t + 4.
+// The values of C one flush needs: rows of the fibers x = t and x = t + 4 of the next group of eight,
+// columns 16 mt + g and 16 mt + g + 8.  Loaded right after the previous flush so that the L2 latency
+// is covered by the producer work in between.
+template <int L, int M>
+__device__ __forceinline__ void load_cfrag(float (&cf)[cfg<L, M>::MT][4], const float *__restrict__ crow_a,
+                                           const float *__restrict__ crow_b, int lane)
+{
+    const int g = lane >> 2;
+#pragma unroll
+    for (int mt = 0; mt < cfg<L, M>::MT; ++mt) {
+        cf[mt][0] = __ldg(crow_a + 16 * mt + g);
+        cf[mt][1] = __ldg(crow_a + 16 * mt + g + 8);
+        cf[mt][2] = __ldg(crow_b + 16 * mt + g);
+        cf[mt][3] = __ldg(crow_b + 16 * mt + g + 8);
+    }
+}
+
+// acc += Cg^T . T for eight staged fibers: rows (row0 + x) & 15, x = 0..7, of the 16-row ring.
 template <int L, int M>
 __device__ __forceinline__ void ttm3_flush(float (&acc)[cfg<L, M>::MT][cfg<L, M>::NT][4], const float *__restrict__ Tbuf,
-                                           int row0, const float *__restrict__ crow_a, const float *__restrict__ crow_b,
-                                           int lane)
+                                           int row0, const float (&cf)[cfg<L, M>::MT][4], int lane)
 {
     using K = cfg<L, M>;
     const int g = lane >> 2, t = lane & 3;
@@ -95,10 +110,8 @@ __device__ __forceinline__ void ttm3_flush(float (&acc)[cfg<L, M>::MT][cfg<L, M>
 #pragma unroll
     for (int mt = 0; mt < K::MT; ++mt) {
         uint32_t ah[4], al[4];
-        split_tf32(__ldg(crow_a + 16 * mt + g), ah[0], al[0]);
-        split_tf32(__ldg(crow_a + 16 * mt + g + 8), ah[1], al[1]);
-        split_tf32(__ldg(crow_b + 16 * mt + g), ah[2], al[2]);
-        split_tf32(__ldg(crow_b + 16 * mt + g + 8), ah[3], al[3]);
+#pragma unroll
+        for (int x = 0; x < 4; ++x) split_tf32(cf[mt][x], ah[x], al[x]);
 #pragma unroll
         for (int nt = 0; nt < K::NT; ++nt) {
             mma_m16n8k8_tf32(acc[mt][nt], al, bh[nt]);
@@ -162,15 +175,17 @@ __device__ __forceinline__ void ttm3_warp_item(const sa_item &it, const int32_t 
     if (1 < nb) stage_rows<M>(dst_lane + K::STAGE * 4, k1, src_lane, row_bytes, gr);
     cp_async_commit();
     int nclosed = 0, nflushed = 0;          // fibers closed / handed to the tensor cores so far
-    int ja = crd_j[min(f0 + t4, fmax)], jb = crd_j[min(f0 + t4 + 4, fmax)];
-    float T = 0.f;
+    float cf[K::MT][4];                     // C values of the next flush
+    load_cfrag<L, M>(cf, C + uint32_t(crd_j[min(f0 + t4, fmax)]) * ldc, C + uint32_t(crd_j[min(f0 + t4 + 4, fmax)]) * ldc, lane);
+    float T = 0.f, U = 0.f;                 // two partial sums of the open fiber (shorter dependency chains)
     int s_cur = 0, s_issue = 2;
     // T += v * d for one nonzero; `end` (warp-uniform) closes the fiber into the ring of temporaries
 #define SA_TTM3_STEP(v, d, end)                                   \
     T = fmaf(v, d, T);                                            \
     if (end) {                                                    \
-        Tbuf[(nclosed & 15) * K::TS + m] = T;                     \
+        Tbuf[(nclosed & 15) * K::TS + m] = T + U;                 \
         T = 0.f;                                                  \
+        U = 0.f;                                                  \
         ++nclosed;                                                \
     }
 #pragma unroll 1
@@ -193,9 +208,9 @@ __device__ __forceinline__ void ttm3_warp_item(const sa_item &it, const int32_t 
             const float4 vb = *reinterpret_cast<const float4 *>(vs + 8 * c + 4);
             if ((e8 & 0xfu) == 0) {
                 T = fmaf(va.x, sc[0], T);
-                T = fmaf(va.y, sc[M], T);
+                U = fmaf(va.y, sc[M], U);
                 T = fmaf(va.z, sc[2 * M], T);
-                T = fmaf(va.w, sc[3 * M], T);
+                U = fmaf(va.w, sc[3 * M], U);
             } else {
                 SA_TTM3_STEP(va.x, sc[0], e8 & 1u)
                 SA_TTM3_STEP(va.y, sc[M], e8 & 2u)
@@ -204,9 +219,9 @@ __device__ __forceinline__ void ttm3_warp_item(const sa_item &it, const int32_t 
             }
             if ((e8 & 0xf0u) == 0) {
                 T = fmaf(vb.x, sc[4 * M], T);
-                T = fmaf(vb.y, sc[5 * M], T);
+                U = fmaf(vb.y, sc[5 * M], U);
                 T = fmaf(vb.z, sc[6 * M], T);
-                T = fmaf(vb.w, sc[7 * M], T);
+                U = fmaf(vb.w, sc[7 * M], U);
             } else {
                 SA_TTM3_STEP(vb.x, sc[4 * M], e8 & 16u)
                 SA_TTM3_STEP(vb.y, sc[5 * M], e8 & 32u)
@@ -215,11 +230,11 @@ __device__ __forceinline__ void ttm3_warp_item(const sa_item &it, const int32_t 
             }
             if (nclosed - nflushed >= 8) {
                 __syncwarp();
-                ttm3_flush<L, M>(acc, Tbuf, nflushed, C + ja * ldc, C + jb * ldc, lane);
+                ttm3_flush<L, M>(acc, Tbuf, nflushed, cf, lane);
                 __syncwarp();
                 nflushed += 8;
-                ja = crd_j[min(f0 + nflushed + t4, fmax)];
-                jb = crd_j[min(f0 + nflushed + t4 + 4, fmax)];
+                load_cfrag<L, M>(cf, C + uint32_t(crd_j[min(f0 + nflushed + t4, fmax)]) * ldc,
+                                 C + uint32_t(crd_j[min(f0 + nflushed + t4 + 4, fmax)]) * ldc, lane);
             }
         }
         __syncwarp();                                   // stage s_cur and vs are free for the next round
@@ -235,7 +250,7 @@ __device__ __forceinline__ void ttm3_warp_item(const sa_item &it, const int32_t 
     if (pending > 0) {
         for (int x = pending; x < 8; ++x) Tbuf[((nflushed + x) & 15) * K::TS + m] = 0.f;   // unused rows
         __syncwarp();
-        ttm3_flush<L, M>(acc, Tbuf, nflushed, C + ja * ldc, C + jb * ldc, lane);
+        ttm3_flush<L, M>(acc, Tbuf, nflushed, cf, lane);
         __syncwarp();
     }
 }
