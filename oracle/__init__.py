@@ -154,12 +154,39 @@ def spmm_gemm(coords, vals, dims, C, D, sel=None, with_abs=True, threads=0):
     return A, S
 
 
+def ttmc3(coords, vals, dims, C, D, E, sel=None, with_abs=True, threads=0):
+    """A(l,m,n) = sum_{i,j,k} B(i,j,k) C(i,l) D(j,m) E(k,n).  Returns (A, S) of shape (L, M, N), or of
+    shape (len(sel),) when ``sel`` lists flat output indices (l*M + m)*N + n."""
+    I, J, K = (int(d) for d in dims)
+    c, cp = _coords(coords, 3)
+    v, vp = _f32(vals)
+    C, Cp = _f32(C)
+    D, Dp = _f32(D)
+    E, Ep = _f32(E)
+    assert C.shape[0] == I and D.shape[0] == J and E.shape[0] == K
+    L, M, N = C.shape[1], D.shape[1], E.shape[1]
+    if sel is None:
+        s, sp, n_sel, shape = None, None, 0, (L, M, N)
+    else:
+        s = np.ascontiguousarray(sel, dtype=np.int64)
+        sp, n_sel, shape = s.ctypes.data_as(_p), s.shape[0], (s.shape[0],)
+    A = np.empty(shape, dtype=np.float64)
+    S = np.empty_like(A) if with_abs else None
+    rc = _load().oracle_ttmc3(_i64(v.shape[0]), cp, vp, _i64(I), _i64(J), _i64(K), _i64(L), _i64(M), _i64(N),
+                              Cp, Dp, Ep, _i64(n_sel), sp, A.ctypes.data_as(_p),
+                              S.ctypes.data_as(_p) if with_abs else None, ctypes.c_int(threads))
+    _check(rc)
+    return A, S
+
+
 def evaluate(w, sel=None, with_abs=True, threads=0):
     """Evaluate a workload object (``workloads.configs.Workload``) -> (A, S)."""
     if w.expr == "spttm_ttm3":
         return spttm_ttm3(w.coords, w.vals, w.dims, *w.dense, sel=sel, with_abs=with_abs, threads=threads)
     if w.expr == "spttm_ttm4":
         return spttm_ttm4(w.coords, w.vals, w.dims, *w.dense, sel=sel, with_abs=with_abs, threads=threads)
+    if w.expr == "ttmc3":
+        return ttmc3(w.coords, w.vals, w.dims, *w.dense, sel=sel, with_abs=with_abs, threads=threads)
     if w.expr == "sddmm_spmm":
         return sddmm_spmm(w.coords, w.vals, w.dims, *w.dense, sel=sel, with_abs=with_abs, threads=threads)[:2]
     if w.expr == "spmm_gemm":

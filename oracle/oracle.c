@@ -249,3 +249,40 @@ int oracle_spmm_gemm(int64_t nnz, const int32_t *coords, const float *vals,
     free_buckets(&b);
     return 0;
 }
+
+/* Kernel 5 <3D TTMC>:  A(l,m,n) = sum_{i,j,k} B(i,j,k) * C(i,l) * D(j,m) * E(k,n)  (all three
+ * modes contracted; the running example of Sections 1, 3 and 4).  Every nonzero contributes to
+ * every output element, so the loop nest is the linear one of the paper's first schedule with the
+ * nonzero loop innermost per output element; threads split the output elements, the order of the
+ * terms of one element is the input order.
+ * n_sel > 0: only the output elements listed in sel (flat indices (l*M + m)*N + n) are computed,
+ * A and S then hold n_sel values. */
+int oracle_ttmc3(int64_t nnz, const int32_t *coords, const float *vals,
+                 int64_t I, int64_t J, int64_t K, int64_t L, int64_t M, int64_t N,
+                 const float *C, const float *D, const float *E,
+                 int64_t n_sel, const int64_t *sel, double *A, double *S, int threads)
+{
+    for (int64_t p = 0; p < nnz; ++p)
+        if (coords[3 * p] < 0 || coords[3 * p] >= I || coords[3 * p + 1] < 0 || coords[3 * p + 1] >= J ||
+            coords[3 * p + 2] < 0 || coords[3 * p + 2] >= K)
+            return -2;
+    const int64_t n_out = sel ? n_sel : L * M * N;
+    for (int64_t x = 0; x < n_out; ++x)
+        if (sel && (sel[x] < 0 || sel[x] >= L * M * N)) return -2;
+    set_threads(threads);
+    #pragma omp parallel for schedule(static)
+    for (int64_t x = 0; x < n_out; ++x) {
+        const int64_t e = sel ? sel[x] : x;
+        const int64_t l = e / (M * N), m = (e / N) % M, n = e % N;
+        double a = 0.0, s = 0.0;
+        for (int64_t p = 0; p < nnz; ++p) {
+            const int64_t i = coords[3 * p], j = coords[3 * p + 1], k = coords[3 * p + 2];
+            const double term = (double)vals[p] * (double)C[i * L + l] * (double)D[j * M + m] * (double)E[k * N + n];
+            a += term;
+            s += fabs(term);
+        }
+        A[x] = a;
+        if (S) S[x] = s;
+    }
+    return 0;
+}

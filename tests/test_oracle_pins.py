@@ -265,3 +265,35 @@ def test_workload_generators_feed_oracle():
     A5, _ = oracle.spttm_ttm3(w.coords[keep], w.vals[keep], w.dims, *w.dense)
     np.testing.assert_array_equal(A5[5], A[5])
     assert not A5[np.arange(200) != 5].any()
+
+
+# ----------------------------------------------------------------- kernel 5, all-mode TTMC
+
+def test_ttmc3_bruteforce_closed_form_and_relation_to_the_partial_chain():
+    rs = np.random.RandomState(11)
+    dims = (5, 4, 6)
+    coords, vals = tiny_coo(rs, dims, 43)
+    C, D, E = dense(rs, 5, 2), dense(rs, 4, 3), dense(rs, 6, 4)
+    A, S = oracle.ttmc3(coords, vals, dims, C, D, E)
+    B = densify(coords, vals, dims)
+    C64, D64, E64 = (x.astype(np.float64) for x in (C, D, E))
+    ref = np.zeros((2, 3, 4))
+    for i, j, k, l, m, n in itertools.product(range(5), range(4), range(6), range(2), range(3), range(4)):
+        ref[l, m, n] += B[i, j, k] * C64[i, l] * D64[j, m] * E64[k, n]
+    np.testing.assert_allclose(A, ref, rtol=0, atol=1e-13)
+    np.testing.assert_allclose(A, np.einsum("ijk,il,jm,kn->lmn", B, C64, D64, E64), rtol=0, atol=1e-13)
+    np.testing.assert_allclose(S, np.einsum("ijk,il,jm,kn->lmn", np.abs(B), np.abs(C64), np.abs(D64), np.abs(E64)),
+                               rtol=0, atol=1e-13)
+    # fissioned form: the per-slice chain over (j,k) first, then the contraction over i
+    T, _ = oracle.spttm_ttm3(coords, vals, dims, D, E)
+    np.testing.assert_allclose(A, np.einsum("il,imn->lmn", C64, T), rtol=0, atol=1e-12)
+    # element list = the same elements of the full result; all ones: every element counts the nonzeros
+    sel = np.array([23, 0, 7, 12])
+    As, Ss = oracle.ttmc3(coords, vals, dims, C, D, E, sel=sel)
+    assert np.array_equal(As, A.reshape(-1)[sel]) and np.array_equal(Ss, S.reshape(-1)[sel])
+    ones = [np.ones((d, r), np.float32) for d, r in zip(dims, (2, 3, 4))]
+    A1, _ = oracle.ttmc3(coords, np.ones(43, np.float32), dims, *ones)
+    assert np.array_equal(A1, np.full((2, 3, 4), 43.0))
+    # identity factors return the densified tensor
+    Ai, _ = oracle.ttmc3(coords, vals, dims, *(np.eye(d, dtype=np.float32) for d in dims))
+    assert np.array_equal(Ai, B)
