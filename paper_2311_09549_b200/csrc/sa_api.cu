@@ -73,6 +73,7 @@ sa_status check_ops(const sa_tensor *t, sa_expr expr, const sa_dense *ops, int n
         case SA_EXPR_SPTTM_TTM4: want = 3; break;
         case SA_EXPR_SDDMM_SPMM: want = 3; break;
         case SA_EXPR_SPMM_GEMM: want = 2; break;
+        case SA_EXPR_TTMC3: want = 3; break;
         default: return SA_E_ARG;
     }
     if (n_ops != want) return SA_E_ARG;
@@ -103,6 +104,11 @@ sa_status check_ops(const sa_tensor *t, sa_expr expr, const sa_dense *ops, int n
             if (ops[0].rows != t->dims[1] || ops[1].rows != ops[0].cols) return SA_E_SHAPE;
             if (!sa_ranks_ok_spmm_gemm(ops[0].cols, ops[1].cols)) return SA_E_UNSUPPORTED;
             break;
+        case SA_EXPR_TTMC3:
+            if (t->fmt != SA_FMT_CSF || t->order != 3) return SA_E_FORMAT;
+            if (ops[0].rows != t->dims[0] || ops[1].rows != t->dims[1] || ops[2].rows != t->dims[2]) return SA_E_SHAPE;
+            if (!sa_ranks_ok_ttmc3(ops[0].cols, ops[1].cols, ops[2].cols)) return SA_E_UNSUPPORTED;
+            break;
     }
     return SA_OK;
 }
@@ -120,6 +126,7 @@ bool resolve_schedule(const sa_tensor *t, sa_expr expr, sa_schedule sched, const
     switch (expr) {
         case SA_EXPR_SPTTM_TTM3:
         case SA_EXPR_SPTTM_TTM4:
+        case SA_EXPR_TTMC3:
             if (sched == SA_SCHED_DEFAULT || sched == SA_SCHED_FUSED) { *resolved = SA_SCHED_FUSED; return true; }
             return false;
         case SA_EXPR_SDDMM_SPMM:
@@ -148,6 +155,7 @@ size_t workspace_bytes(const sa_tensor *t, sa_expr expr, sa_schedule sched, cons
         case SA_EXPR_SPTTM_TTM4: return sa_ws_ttm4(t, ops);
         case SA_EXPR_SDDMM_SPMM: return sa_ws_sddmm_spmm(t, ops, sched == SA_SCHED_DEBUG_MATERIALIZE);
         case SA_EXPR_SPMM_GEMM: return sa_ws_spmm_gemm(t, ops, sched == SA_SCHED_ASSOC_RIGHT);
+        case SA_EXPR_TTMC3: return sa_ws_ttmc3(t, ops);
     }
     return 0;
 }
@@ -294,6 +302,7 @@ sa_status sa_run(const sa_tensor *t, sa_expr expr, sa_schedule sched, const sa_d
         case SA_EXPR_SPMM_GEMM:
             s = sa_launch_spmm_gemm(t, ops, out, workspace, ws_bytes, r == SA_SCHED_ASSOC_RIGHT, stream, &launches);
             break;
+        case SA_EXPR_TTMC3: s = sa_launch_ttmc3(t, ops, out, workspace, ws_bytes, stream, &launches); break;
     }
     if (s == SA_E_CUDA) cudaGetLastError();
     if (s == SA_OK) t->last_launches = launches;

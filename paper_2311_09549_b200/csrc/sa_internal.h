@@ -93,9 +93,14 @@ sa_status sa_launch_spmm_gemm(const sa_tensor *t, const sa_dense *ops, float *ou
                               bool assoc_right, cudaStream_t stream, int *launches);
 size_t sa_ws_spmm_gemm(const sa_tensor *t, const sa_dense *ops, bool assoc_right);
 
+sa_status sa_launch_ttmc3(const sa_tensor *t, const sa_dense *ops, float *out, void *ws, size_t ws_bytes,
+                          cudaStream_t stream, int *launches);
+size_t sa_ws_ttmc3(const sa_tensor *t, const sa_dense *ops);
+
 // Supported-rank predicates (shared by sa_workspace_size and sa_run).
 bool sa_ranks_ok_ttm3(int64_t L, int64_t M);
 bool sa_ranks_ok_ttm4(int64_t L, int64_t M, int64_t N);
+bool sa_ranks_ok_ttmc3(int64_t L, int64_t M, int64_t N);
 bool sa_ranks_ok_sddmm(int64_t K, int64_t L);
 bool sa_ranks_ok_spmm_gemm(int64_t L, int64_t M);
 

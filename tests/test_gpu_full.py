@@ -103,3 +103,19 @@ def test_cfg5_full_sampled(sa):
     _compare(out, w, sel, w.name)
     del out, t
     torch.cuda.empty_cache()
+
+
+def test_cfg6_ttmc_full_sampled(sa):
+    """Kernel 5 on the nell-2-shaped tensor: every output element sums over all nonzeros, so the
+    oracle evaluates a seeded sample of output elements one by one."""
+    import torch
+    w = configs.make(6, "full")
+    out, t = _run_full(sa, w)
+    n_out = int(np.prod(w.out_shape))
+    sel = np.sort(configs.rng.permutation(w.seed, 56, n_out)[:48])
+    A_ref, S_ref = oracle.evaluate(w, sel=sel)
+    got = out.reshape(-1)[torch.from_numpy(sel).cuda()].cpu().numpy().astype(np.float64)
+    assert_close(got, A_ref, S_ref, TOL_FP32, w.name)
+    assert bool(torch.isfinite(out).all())
+    del out, t
+    torch.cuda.empty_cache()

@@ -18,7 +18,7 @@ def sa():
     return sa
 
 
-@pytest.mark.parametrize("cfg", [1, 2, 5])
+@pytest.mark.parametrize("cfg", [1, 2, 5, 6])
 def test_ttm_chains_mini(sa, cfg):
     w = configs.make(cfg, "mini")
     A_ref, S_ref = oracle.evaluate(w)

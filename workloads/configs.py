@@ -35,7 +35,7 @@ S_STRUCT, S_VALS, S_DENSE, S_SHUFFLE = 0, 1, 2, 3
 @dataclass
 class Workload:
     name: str
-    expr: str                  # 'spttm_ttm3' | 'spttm_ttm4' | 'sddmm_spmm' | 'spmm_gemm'
+    expr: str                  # 'spttm_ttm3' | 'spttm_ttm4' | 'sddmm_spmm' | 'spmm_gemm' | 'ttmc3'
     fmt: str                   # 'csf' | 'csr'
     dims: tuple                # dimensions of B
     coords: np.ndarray         # int32 [nnz, order], shuffled
@@ -235,6 +235,13 @@ def make_ttm3_zipf(name, seed, I, J, K, nnz, alpha, mean_fiber, L, M):
     return Workload(name, "spttm_ttm3", "csf", (I, J, K), coords, vals, [C, D], (I, L, M), seed, notes)
 
 
+def make_ttmc3_zipf(name, seed, I, J, K, nnz, alpha, mean_fiber, L, M, N):
+    """Kernel 5 workload: the order-3 Zipf tensor of make_ttm3_zipf with a factor matrix per mode."""
+    w = make_ttm3_zipf(name, seed, I, J, K, nnz, alpha, mean_fiber, M, N)      # D (J x M), E (K x N)
+    C = dense_uniform(seed, 2, I, L)
+    return Workload(name, "ttmc3", "csf", (I, J, K), w.coords, w.vals, [C] + w.dense, (L, M, N), seed, w.notes)
+
+
 def make_ttm4_zipf(name, seed, I, J, K, O, nnz, alpha, mean_fiber, L, M, N):
     """Order-4 CSF workload: Zipf slices, geometric-like fan-out (mean ``mean_fiber``) per level."""
     n_i = _zipf_slices(seed, I, nnz, alpha)
@@ -368,4 +375,9 @@ def make(config, scale="full", seed=None):
             return make_ttm4_zipf("cfg5-ttm4-zipf", s, 50_000, 20_000, 20_000, 20_000, 100_000_000,
                                   1.2, 6.0, 16, 16, 16)
         return make_ttm4_zipf("cfg5-ttm4-zipf-mini", s, 600, 150, 120, 130, 200_000, 1.2, 6.0, 16, 16, 16)
-    raise ValueError("config must be 1..5")
+    if config == 6:
+        # kernel 5 (all-mode TTMC) on a tensor with the shape and size the paper quotes for nell-2
+        if full:
+            return make_ttmc3_zipf("cfg6-ttmc3-nell2-shaped", s, 12_000, 9_000, 288_000, 76_880_000, 1.2, 8.0, 16, 16, 16)
+        return make_ttmc3_zipf("cfg6-ttmc3-mini", s, 300, 200, 250, 60_000, 1.2, 8.0, 16, 16, 16)
+    raise ValueError("config must be 1..6")
