@@ -135,6 +135,27 @@ def sddmm_spmm(coords, vals, dims, C, D, E, sel=None, with_abs=True, with_sample
     return A, S, P
 
 
+def sddmm_spmm_gemm(coords, vals, dims, C, D, E, F, sel=None, with_abs=True, threads=0):
+    """A(i,m) = sum_{j,k,l} B(i,j) C(i,k) D(j,k) E(j,l) F(l,m).  Returns (A, S)."""
+    I, J = (int(d) for d in dims)
+    c, cp = _coords(coords, 2)
+    v, vp = _f32(vals)
+    C, Cp = _f32(C)
+    D, Dp = _f32(D)
+    E, Ep = _f32(E)
+    F, Fp = _f32(F)
+    assert C.shape[0] == I and D.shape[0] == J and E.shape[0] == J and C.shape[1] == D.shape[1] and F.shape[0] == E.shape[1]
+    K, L, M = C.shape[1], E.shape[1], F.shape[1]
+    s, sp, n_sel, n_out = _sel(sel, I)
+    A = np.empty((n_out, M), dtype=np.float64)
+    S = np.empty_like(A) if with_abs else None
+    rc = _load().oracle_sddmm_spmm_gemm(_i64(v.shape[0]), cp, vp, _i64(I), _i64(J), _i64(K), _i64(L), _i64(M),
+                                        Cp, Dp, Ep, Fp, _i64(n_sel), sp, A.ctypes.data_as(_p),
+                                        S.ctypes.data_as(_p) if with_abs else None, ctypes.c_int(threads))
+    _check(rc)
+    return A, S
+
+
 def spmm_gemm(coords, vals, dims, C, D, sel=None, with_abs=True, threads=0):
     """A(i,m) = sum_{j,l} B(i,j) C(j,l) D(l,m).  Returns (A, S)."""
     I, J = (int(d) for d in dims)
@@ -187,6 +208,8 @@ def evaluate(w, sel=None, with_abs=True, threads=0):
         return spttm_ttm4(w.coords, w.vals, w.dims, *w.dense, sel=sel, with_abs=with_abs, threads=threads)
     if w.expr == "ttmc3":
         return ttmc3(w.coords, w.vals, w.dims, *w.dense, sel=sel, with_abs=with_abs, threads=threads)
+    if w.expr == "sddmm_spmm_gemm":
+        return sddmm_spmm_gemm(w.coords, w.vals, w.dims, *w.dense, sel=sel, with_abs=with_abs, threads=threads)
     if w.expr == "sddmm_spmm":
         return sddmm_spmm(w.coords, w.vals, w.dims, *w.dense, sel=sel, with_abs=with_abs, threads=threads)[:2]
     if w.expr == "spmm_gemm":

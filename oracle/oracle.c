@@ -286,3 +286,38 @@ int oracle_ttmc3(int64_t nnz, const int32_t *coords, const float *vals,
     }
     return 0;
 }
+
+/* Kernel 2 <SDDMM,SpMM,GEMM>:  A(i,m) = sum_{j,k,l} B(i,j) * C(i,k) * D(j,k) * E(j,l) * F(l,m). */
+int oracle_sddmm_spmm_gemm(int64_t nnz, const int32_t *coords, const float *vals,
+                           int64_t I, int64_t J, int64_t K, int64_t L, int64_t M,
+                           const float *C, const float *D, const float *E, const float *F,
+                           int64_t n_sel, const int64_t *sel, double *A, double *S, int threads)
+{
+    buckets_t b;
+    int rc = make_buckets(&b, nnz, coords, 2, I, n_sel, sel);
+    if (rc) { free_buckets(&b); return rc; }
+    for (int64_t p = 0; p < nnz; ++p)
+        if (coords[2 * p + 1] < 0 || coords[2 * p + 1] >= J) { free_buckets(&b); return -2; }
+    set_threads(threads);
+    #pragma omp parallel for schedule(dynamic, 4)
+    for (int64_t o = 0; o < b.n_out; ++o) {
+        double *Ao = A + o * M;
+        double *So = S ? S + o * M : NULL;
+        for (int64_t x = 0; x < M; ++x) Ao[x] = 0.0;
+        if (So) for (int64_t x = 0; x < M; ++x) So[x] = 0.0;
+        for (int64_t q = b.start[o]; q < b.start[o + 1]; ++q) {
+            int64_t p = b.order[q];
+            int64_t i = coords[2 * p], j = coords[2 * p + 1];
+            double v = (double)vals[p];
+            for (int64_t k = 0; k < K; ++k)
+                for (int64_t l = 0; l < L; ++l)
+                    for (int64_t m = 0; m < M; ++m) {
+                        double term = v * (double)C[i * K + k] * (double)D[j * K + k] * (double)E[j * L + l] * (double)F[l * M + m];
+                        Ao[m] += term;
+                        if (So) So[m] += fabs(term);
+                    }
+        }
+    }
+    free_buckets(&b);
+    return 0;
+}

@@ -297,3 +297,30 @@ def test_ttmc3_bruteforce_closed_form_and_relation_to_the_partial_chain():
     # identity factors return the densified tensor
     Ai, _ = oracle.ttmc3(coords, vals, dims, *(np.eye(d, dtype=np.float32) for d in dims))
     assert np.array_equal(Ai, B)
+
+
+# ----------------------------------------------------------------- kernel 2, SDDMM -> SpMM -> GEMM
+
+def test_sddmm_spmm_gemm_bruteforce_and_relation_to_kernel_1():
+    rs = np.random.RandomState(12)
+    dims = (6, 5)
+    coords, vals = tiny_coo(rs, dims, 14)
+    C, D, E, F = dense(rs, 6, 3), dense(rs, 5, 3), dense(rs, 5, 4), dense(rs, 4, 2)
+    A, S = oracle.sddmm_spmm_gemm(coords, vals, dims, C, D, E, F)
+    B = densify(coords, vals, dims)
+    f64 = [x.astype(np.float64) for x in (C, D, E, F)]
+    ref = np.zeros((6, 2))
+    for i, j, k, l, m in itertools.product(range(6), range(5), range(3), range(4), range(2)):
+        ref[i, m] += B[i, j] * f64[0][i, k] * f64[1][j, k] * f64[2][j, l] * f64[3][l, m]
+    np.testing.assert_allclose(A, ref, rtol=0, atol=1e-13)
+    np.testing.assert_allclose(A, np.einsum("ij,ik,jk,jl,lm->im", B, *f64), rtol=0, atol=1e-13)
+    np.testing.assert_allclose(S, np.einsum("ij,ik,jk,jl,lm->im", np.abs(B), *(np.abs(x) for x in f64)), rtol=0, atol=1e-13)
+    # two-level schedule: the row temporary T_l of kernel 1, then the product with F
+    A1, _, _ = oracle.sddmm_spmm(coords, vals, dims, C, D, E)
+    np.testing.assert_allclose(A, A1 @ f64[3], rtol=0, atol=1e-13)
+    # F = identity reduces to kernel 1; subset mode
+    Ai, _ = oracle.sddmm_spmm_gemm(coords, vals, dims, C, D, E, np.eye(4, dtype=np.float32))
+    np.testing.assert_allclose(Ai, A1, rtol=0, atol=1e-14)
+    sel = np.array([4, 1])
+    As, Ss = oracle.sddmm_spmm_gemm(coords, vals, dims, C, D, E, F, sel=sel)
+    assert np.array_equal(As, A[sel]) and np.array_equal(Ss, S[sel])
