@@ -97,6 +97,14 @@ sa_status sa_launch_ttmc3(const sa_tensor *t, const sa_dense *ops, float *out, v
                           cudaStream_t stream, int *launches);
 size_t sa_ws_ttmc3(const sa_tensor *t, const sa_dense *ops);
 
+// Kernel 2 <SDDMM,SpMM,GEMM>: the fused SDDMM->SpMM kernel into a row temporary, then the dense stage.
+sa_status sa_launch_sddmm_spmm_gemm(const sa_tensor *t, const sa_dense *ops, float *out, void *ws, size_t ws_bytes,
+                                    cudaStream_t stream, int *launches);
+size_t sa_ws_sddmm_spmm_gemm(const sa_tensor *t, const sa_dense *ops);
+bool sa_dense_gemm_ok(int64_t L, int64_t M);
+sa_status sa_launch_dense_gemm(int64_t rows, const float *A, int64_t lda, const float *B, int64_t ldb, int64_t L,
+                               int64_t M, float *out, cudaStream_t stream);
+
 // Supported-rank predicates (shared by sa_workspace_size and sa_run).
 bool sa_ranks_ok_ttm3(int64_t L, int64_t M);
 bool sa_ranks_ok_ttm4(int64_t L, int64_t M, int64_t N);

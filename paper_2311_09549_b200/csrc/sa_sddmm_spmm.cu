@@ -235,3 +235,28 @@ sa_status sa_launch_sddmm_spmm(const sa_tensor *t, const sa_dense *ops, float *o
     }
     return SA_OK;
 }
+
+// ---- kernel 2 <SDDMM,SpMM,GEMM>:  A(i,m) = sum_{j,k,l} B(i,j) C(i,k) D(j,k) E(j,l) F(l,m), the two-level
+// schedule  i < T(l) ; j' < t ; k: ... , l: T(l) += t E(j,l) > , m,l: A(i,m) += T(l) F(l,m) >  of the paper's
+// Table of kernels: the row temporary T is what the fused kernel above produces per row; here it goes
+// through the workspace (I x L floats) to a tensor-core product with F instead of staying in registers.
+// workspace: [T: I x L][partial rows of long-row pieces]
+size_t sa_ws_sddmm_spmm_gemm(const sa_tensor *t, const sa_dense *ops)
+{
+    return sa_align256(size_t(t->dims[0]) * size_t(ops[2].cols) * sizeof(float)) + sa_ws_sddmm_spmm(t, ops, false);
+}
+
+sa_status sa_launch_sddmm_spmm_gemm(const sa_tensor *t, const sa_dense *ops, float *out, void *ws, size_t ws_bytes,
+                                    cudaStream_t stream, int *launches)
+{
+    const int64_t I = t->dims[0], L = ops[2].cols, M = ops[3].cols;
+    const size_t t_bytes = sa_align256(size_t(I) * size_t(L) * sizeof(float));
+    float *T = static_cast<float *>(ws);
+    int n1 = 0;
+    const sa_status s = sa_launch_sddmm_spmm(t, ops, T, static_cast<char *>(ws) + t_bytes, ws_bytes - t_bytes, false, stream, &n1);
+    if (s != SA_OK) return s;
+    const sa_status g = sa_launch_dense_gemm(I, T, L, ops[3].ptr, ops[3].ld, L, M, out, stream);
+    if (g != SA_OK) return g;
+    *launches = n1 + 1;
+    return SA_OK;
+}

@@ -347,6 +347,31 @@ sa_status run(const sa_tensor *t, const sa_dense *ops, float *out, void *ws, boo
 
 }  // namespace
 
+// out (rows x M) = A (rows x L, leading dimension lda) . B (L x M), TF32x3 on tensor cores; used as the
+// dense stage of other chains.  L in {32, 64, 128, 256}, M in {32, 64}.
+template <int L, int M>
+static sa_status dense_gemm(int64_t rows, const float *A, int64_t lda, const float *B, int64_t ldb, float *out,
+                            cudaStream_t stream)
+{
+    using GC = gemm_cfg<L, M, SA_GEMM_NPROD>;
+    auto gk = gemm_tf32_kernel<L, M, SA_GEMM_NPROD>;
+    if (cudaFuncSetAttribute(gk, cudaFuncAttributeMaxDynamicSharedMemorySize, int(GC::SMEM)) != cudaSuccess) return SA_E_CUDA;
+    const int64_t ctas = std::min<int64_t>((rows + GC::BM - 1) / GC::BM, resident_ctas(reinterpret_cast<const void *>(gk), GC::SMEM));
+    if (ctas > 0) gk<<<(unsigned)ctas, 256, GC::SMEM, stream>>>(rows, A, lda, B, ldb, out);
+    return cudaGetLastError() == cudaSuccess ? SA_OK : SA_E_CUDA;
+}
+
+bool sa_dense_gemm_ok(int64_t L, int64_t M) { return (L == 32 || L == 64 || L == 128 || L == 256) && (M == 32 || M == 64); }
+
+sa_status sa_launch_dense_gemm(int64_t rows, const float *A, int64_t lda, const float *B, int64_t ldb, int64_t L,
+                               int64_t M, float *out, cudaStream_t stream)
+{
+#define SA_CASE(l, m) if (L == l && M == m) return dense_gemm<l, m>(rows, A, lda, B, ldb, out, stream);
+    SA_CASE(32, 32) SA_CASE(32, 64) SA_CASE(64, 32) SA_CASE(64, 64) SA_CASE(128, 32) SA_CASE(128, 64) SA_CASE(256, 32) SA_CASE(256, 64)
+#undef SA_CASE
+    return SA_E_UNSUPPORTED;
+}
+
 bool sa_ranks_ok_spmm_gemm(int64_t L, int64_t M) { return (L == 128 || L == 256) && (M == 32 || M == 64); }
 
 // workspace: ASSOC_RIGHT [E = C.D, J x M][partial rows]; ASSOC_LEFT [partial rows]

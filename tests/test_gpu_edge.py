@@ -52,6 +52,8 @@ def test_empty_and_single_entry_all_chains(sa, nnz):
                    [_dense(1, 0, 4, 16), _dense(1, 1, 3, 16), _dense(1, 2, 2, 16)], (5, 16, 16, 16)))
     _check(sa, _wl("sddmm_spmm", "csr", (5, 4), c2, v, [_dense(1, 0, 5, 64), _dense(1, 1, 4, 64), _dense(1, 2, 4, 32)], (5, 32)))
     _check(sa, _wl("ttmc3", "csf", (5, 4, 3), c3, v, [_dense(1, 0, 5, 32), _dense(1, 1, 4, 16), _dense(1, 2, 3, 32)], (32, 16, 32)))
+    _check(sa, _wl("sddmm_spmm_gemm", "csr", (5, 4), c2, v,
+                   [_dense(1, 0, 5, 64), _dense(1, 1, 4, 64), _dense(1, 2, 4, 128), _dense(1, 3, 128, 32)], (5, 32)))
     w = _wl("spmm_gemm", "csr", (5, 4), c2, v, [_dense(1, 0, 4, 128), _dense(1, 1, 128, 32)], (5, 32))
     _check(sa, w, sched=sa.SA_SCHED_ASSOC_LEFT)
     _check(sa, w, sched=sa.SA_SCHED_ASSOC_RIGHT)

@@ -119,3 +119,13 @@ def test_cfg6_ttmc_full_sampled(sa):
     assert bool(torch.isfinite(out).all())
     del out, t
     torch.cuda.empty_cache()
+
+
+def test_cfg7_sddmm_spmm_gemm_full_sampled(sa):
+    import torch
+    w = configs.make(7, "full")
+    out, t = _run_full(sa, w)
+    sel = _sample(w, 5_000, 1200)
+    _compare(out, w, sel, w.name)
+    del out, t
+    torch.cuda.empty_cache()

@@ -26,8 +26,9 @@ def test_ttm_chains_mini(sa, cfg):
     assert_close(A, A_ref, S_ref, TOL_FP32, w.name)
 
 
-def test_sddmm_spmm_mini(sa):
-    w = configs.make(3, "mini")
+@pytest.mark.parametrize("cfg", [3, 7])
+def test_sddmm_spmm_mini(sa, cfg):
+    w = configs.make(cfg, "mini")
     A_ref, S_ref = oracle.evaluate(w)
     A, _ = run_gpu(sa, w)
     assert_close(A, A_ref, S_ref, TOL_FP32, w.name)

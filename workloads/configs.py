@@ -380,4 +380,15 @@ def make(config, scale="full", seed=None):
         if full:
             return make_ttmc3_zipf("cfg6-ttmc3-nell2-shaped", s, 12_000, 9_000, 288_000, 76_880_000, 1.2, 8.0, 16, 16, 16)
         return make_ttmc3_zipf("cfg6-ttmc3-mini", s, 300, 200, 250, 60_000, 1.2, 8.0, 16, 16, 16)
-    raise ValueError("config must be 1..6")
+    if config == 7:
+        # kernel 2 (SDDMM, SpMM, GEMM) on the tensor of config 3 with a 64 x 64 weight matrix F
+        if full:
+            w = make(3, "full", seed=s)
+            F = dense_normal(s, 3, 64, 64)
+            return Workload("cfg7-sddmm-spmm-gemm", "sddmm_spmm_gemm", "csr", w.dims, w.coords, w.vals, w.dense + [F],
+                            (w.dims[0], 64), s, w.notes)
+        w = make_sddmm_spmm("tmp", s, 6_000, 6_000, 60_000, 1.5, 1_500, 32, 32)
+        F = dense_normal(s, 3, 32, 32)
+        return Workload("cfg7-sddmm-spmm-gemm-mini", "sddmm_spmm_gemm", "csr", w.dims, w.coords, w.vals, w.dense + [F],
+                        (w.dims[0], 32), s, w.notes)
+    raise ValueError("config must be 1..7")
