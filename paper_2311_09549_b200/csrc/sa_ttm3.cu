@@ -158,18 +158,16 @@ __device__ __forceinline__ void ttm3_warp_item(const sa_item &it, const int32_t 
         if (pn < p1) { k = kflag[pn]; v = vals[pn]; }
         pn += 32;
     };
-    // index/value registers of batches B .. B+6: the index of a batch is needed two rounds before its
-    // values (to request its rows), and a streaming load takes several rounds to arrive; row gathers
-    // of batches B+1, B+2 are in flight while B is consumed
-    int k0, k1, k2, k3, k4, k5, k6;
-    float v0, v1, v2, v3, v4, v5, v6;
+    // index/value registers of four batches with FIXED roles: register r holds the batches b with
+    // b % 4 == r and is reloaded (for batch b + 4) right after batch b is consumed.  The batch loop is
+    // unrolled by four so that no register is ever copied while its load is still in flight; the
+    // index of a batch is first needed two rounds after its load (to request its rows).
+    int k0, k1, k2, k3;
+    float v0, v1, v2, v3;
     load_kv(k0, v0);
     load_kv(k1, v1);
     load_kv(k2, v2);
     load_kv(k3, v3);
-    load_kv(k4, v4);
-    load_kv(k5, v5);
-    load_kv(k6, v6);
     stage_rows<M>(dst_lane, k0, src_lane, row_bytes, gr);
     cp_async_commit();
     if (1 < nb) stage_rows<M>(dst_lane + K::STAGE * 4, k1, src_lane, row_bytes, gr);
@@ -188,15 +186,15 @@ __device__ __forceinline__ void ttm3_warp_item(const sa_item &it, const int32_t 
         U = 0.f;                                                  \
         ++nclosed;                                                \
     }
-#pragma unroll 1
-    for (int b = 0; b < nb; ++b) {
-        if (b + 2 < nb) stage_rows<M>(dst_lane + s_issue * (K::STAGE * 4), k2, src_lane, row_bytes, gr);
+    // one round: request the rows of batch b + 2 (indices kis), consume batch b (indices/flags kc, values vc)
+    auto do_round = [&](int b, int &kc, float &vc, int kis) {
+        if (b + 2 < nb) stage_rows<M>(dst_lane + s_issue * (K::STAGE * 4), kis, src_lane, row_bytes, gr);
         cp_async_commit();
-        vs[lane] = v0;
+        vs[lane] = vc;
         cp_async_wait<2>();
         __syncwarp();
         const float *st = wsm + s_cur * K::STAGE + m;
-        unsigned ends = __ballot_sync(SA_FULL_MASK, k0 < 0);
+        unsigned ends = __ballot_sync(SA_FULL_MASK, kc < 0);
         const int rem = p1 - p0 - 32 * b;
         if (rem <= 32) ends |= 1u << (rem - 1);         // the item's last nonzero closes its (possibly cut) fiber
         const int nchunks = rem >= 32 ? 4 : (rem + 7) >> 3;
@@ -238,11 +236,16 @@ __device__ __forceinline__ void ttm3_warp_item(const sa_item &it, const int32_t 
             }
         }
         __syncwarp();                                   // stage s_cur and vs are free for the next round
-        k0 = k1; k1 = k2; k2 = k3; k3 = k4; k4 = k5; k5 = k6;
-        v0 = v1; v1 = v2; v2 = v3; v3 = v4; v4 = v5; v5 = v6;
-        load_kv(k6, v6);
+        load_kv(kc, vc);                                // batch b + 4
         s_issue = s_cur;
         s_cur = s_cur == 2 ? 0 : s_cur + 1;
+    };
+#pragma unroll 1
+    for (int b = 0; b < nb; b += 4) {
+        do_round(b, k0, v0, k2);
+        if (b + 1 < nb) do_round(b + 1, k1, v1, k3);
+        if (b + 2 < nb) do_round(b + 2, k2, v2, k0);
+        if (b + 3 < nb) do_round(b + 3, k3, v3, k1);
     }
 #undef SA_TTM3_STEP
     cp_async_wait<0>();
