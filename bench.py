@@ -37,8 +37,8 @@ FALLBACK_HBM_GBS = 6650.0
 # counters were taken; otherwise `traffic` is null.
 NCU_TRAFFIC = {
     2: {"kernel": "ttm3_kernel<32,32>", "source": "paper_2311_09549_b200/csrc/sa_ttm3.cu",
-        "sha256": "089a11f8ca15e5422ed78e1637a0992abd64800a3b31d1daa363b74de54b7d56",
-        "dram_bytes": 838193152, "profile": "profiles/ttm3_kernel_cfg2.md"},
+        "sha256": "58c94ba4a8390c8f9dc91e7221b73ed58684f9066821dc0ec4c4946d5da04339",
+        "dram_bytes": 839057408, "profile": "profiles/ttm3_kernel_cfg2.md"},
     5: {"kernel": "ttm4_kernel", "source": "paper_2311_09549_b200/csrc/sa_ttm4.cu",
         "sha256": "9cba007669e3a8a4dd06731b80f4aa5b19c9c867827b3993f784ee88816ec80b",
         "dram_bytes": 1692932352, "profile": "profiles/ttm4_kernel_cfg5.md"},
