@@ -143,7 +143,10 @@ sa_status sa_tensor_export(const sa_tensor *t, int level, int64_t *pos, int32_t 
  *               fibers [f0,f1) (CSF) clipped to nonzeros [p0,p1) of slice out_row, or rows
  *               [out_row,row_end) / nonzeros [p0,p1) of a long row (CSR); dest = partial slot or -1;
  *               half = 0 / 1 for order-4 tensors, whose items are listed once per half of the
- *               last dense index (0 otherwise)
+ *               last dense index.  Order-3 tensors use the last field for the position of the
+ *               item's (first) slice in the level-0 crd array; items after the leading groups are
+ *               runs of whole small slices at positions [that field, row_end), out_row being the
+ *               coordinate of the first of them
  *   fix    [n_fix * 4] int32 per entry: out_row, slot0, count, 0 -- out[out_row] = sum of `count`
  *               partial tiles from slot0 (count 0: the slice / row is empty and is zero-filled)
  * NULL outputs are skipped.

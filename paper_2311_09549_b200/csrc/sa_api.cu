@@ -211,10 +211,13 @@ sa_status sa_tensor_create(int order, const int64_t *dims, int64_t nnz, const in
             if (s == SA_OK) s = upload(t, t->crd[l].data(), t->crd[l].size(), &t->d_crd[l]);
         }
         if (s == SA_OK) s = upload(t, t->vals.data(), t->vals.size(), &t->d_vals);
-        if (s == SA_OK && fmt == SA_FMT_CSF && order == 3) {
+        if (s == SA_OK && fmt == SA_FMT_CSF && order == 3 && t->dims[2] < (int64_t(1) << 30)) {
+            // bit 31: last nonzero of its (i,j) fiber; bit 30: last nonzero of its slice
             std::vector<int32_t> flagged(t->crd[2]);
             for (int64_t f = 0; f < t->count[1]; ++f)
                 flagged[size_t(t->pos[2][size_t(f) + 1] - 1)] |= int32_t(0x80000000u);
+            for (int64_t sl = 0; sl < t->count[0]; ++sl)
+                flagged[size_t(t->pos[2][size_t(t->pos[1][size_t(sl) + 1])] - 1)] |= int32_t(0x40000000);
             s = upload(t, flagged.data(), flagged.size(), &t->d_crd_endflag);
         }
         if (s == SA_OK && fmt == SA_FMT_CSF && order == 4 && t->dims[3] < (int64_t(1) << 30)) {

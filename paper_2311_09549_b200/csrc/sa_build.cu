@@ -193,18 +193,32 @@ void build_ttm3(sa_tensor *t, sa_worklist &wl)
     const auto &pos2 = t->pos[2];
     std::vector<sa_item> small;
     std::vector<group_rec> groups;
+    // Runs of consecutive small slices are merged into one warp item of at most SMALL_MAX nonzeros: the
+    // warp streams through them without restarting its pipelines and stores one tile per slice.  Such an
+    // item names its slices by position: pad = first slice position, row_end = one past the last.
+    sa_item run = empty_item();
+    bool open = false;
+    auto close_run = [&]() {
+        if (open) small.push_back(run);
+        open = false;
+    };
     for (int64_t s = 0; s < t->count[0]; ++s) {
         const int64_t fa = pos1[size_t(s)], fb = pos1[size_t(s) + 1];
         const int64_t pa = pos2[size_t(fa)], pb = pos2[size_t(fb)];
         const int64_t n = pb - pa;
         const int32_t row = t->crd[0][size_t(s)];
         if (n <= SMALL_MAX) {
-            sa_item it = empty_item();
-            it.out_row = row; it.row_end = row + 1;
-            it.f0 = int32_t(fa); it.f1 = int32_t(fb); it.p0 = int32_t(pa); it.p1 = int32_t(pb);
-            small.push_back(it);
+            if (open && (pb - run.p0) > SMALL_MAX) close_run();
+            if (!open) {
+                run = empty_item();
+                run.out_row = row; run.pad = int32_t(s);
+                run.f0 = int32_t(fa); run.p0 = int32_t(pa);
+                open = true;
+            }
+            run.row_end = int32_t(s + 1); run.f1 = int32_t(fb); run.p1 = int32_t(pb);
             continue;
         }
+        close_run();
         const int64_t chunk = chunk_for(n, MIN_CHUNK, MAX_PARTS);
         const int64_t ng = (n + chunk - 1) / chunk;
         int32_t slot0 = -1;
@@ -221,7 +235,7 @@ void build_ttm3(sa_tensor *t, sa_worklist &wl)
             rec.len = gb - ga;
             for (int w = 0; w < SA_WARPS_PER_CTA; ++w) {
                 sa_item it = empty_item();
-                it.out_row = row; it.row_end = row + 1;
+                it.out_row = row; it.pad = int32_t(s); it.row_end = int32_t(s + 1);
                 it.dest = ng > 1 ? slot0 + int32_t(g) : -1;
                 const int64_t qa = std::min(gb, ga + w * piece), qb = std::min(gb, qa + piece);
                 if (qa < qb) {
@@ -235,6 +249,7 @@ void build_ttm3(sa_tensor *t, sa_worklist &wl)
             groups.push_back(std::move(rec));
         }
     }
+    close_run();
     std::stable_sort(groups.begin(), groups.end(), [](const group_rec &a, const group_rec &b) { return a.len > b.len; });
     std::stable_sort(small.begin(), small.end(),
                      [](const sa_item &a, const sa_item &b) { return (a.p1 - a.p0) > (b.p1 - b.p0); });

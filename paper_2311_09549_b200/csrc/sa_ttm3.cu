@@ -70,7 +70,7 @@ __device__ __forceinline__ void stage_rows(uint32_t dst_lane, int kbatch, const 
     constexpr int LPR = M / 4, RPI = 32 / LPR;
 #pragma unroll
     for (int q = 0; q < 32 / RPI; ++q) {
-        const uint32_t k = uint32_t(__shfl_sync(SA_FULL_MASK, kbatch, q * RPI + r)) & 0x7fffffffu;
+        const uint32_t k = uint32_t(__shfl_sync(SA_FULL_MASK, kbatch, q * RPI + r)) & 0x3fffffffu;
         cp_async16_raw(dst_lane + q * RPI * M * 4, src_lane + k * row_bytes);
     }
 }
@@ -121,13 +121,33 @@ __device__ __forceinline__ void ttm3_flush(float (&acc)[cfg<L, M>::MT][cfg<L, M>
     }
 }
 
-// One warp evaluates one work item: nonzeros [p0,p1) starting inside fiber f0.
+// Store a slice tile held as MMA accumulator fragments (streaming stores: the output is written once).
+template <int L, int M>
+__device__ __forceinline__ void store_tile(const float (&acc)[cfg<L, M>::MT][cfg<L, M>::NT][4], float *__restrict__ dst, int lane)
+{
+    using K = cfg<L, M>;
+    const int g = lane >> 2, t = lane & 3;
+#pragma unroll
+    for (int mt = 0; mt < K::MT; ++mt)
+#pragma unroll
+        for (int nt = 0; nt < K::NT; ++nt) {
+            const int l = 16 * mt + g, mm = 8 * nt + 2 * t;
+            sa_st_cs2(dst + l * M + mm, make_float2(acc[mt][nt][0], acc[mt][nt][1]));
+            sa_st_cs2(dst + (l + 8) * M + mm, make_float2(acc[mt][nt][2], acc[mt][nt][3]));
+        }
+}
+
+// One warp evaluates one work item: nonzeros [p0,p1) starting inside fiber f0.  MULTI: the item is a run
+// of whole small slices (positions it.pad .. it.row_end - 1 in crd_i); the warp streams through all of
+// them and stores each slice's tile to `out` when the slice-end flag (bit 30 of the index stream) comes
+// by.  Otherwise the item is a piece of one slice and the tile is left in acc for the caller.
 template <int L, int M>
 __device__ __forceinline__ void ttm3_warp_item(const sa_item &it, const int32_t *__restrict__ crd_j,
                                                const int32_t *__restrict__ kflag, const float *__restrict__ vals,
                                                const float *__restrict__ C, uint32_t ldc, const float *__restrict__ D,
                                                uint32_t ldd, float *__restrict__ wsm,
-                                               float (&acc)[cfg<L, M>::MT][cfg<L, M>::NT][4])
+                                               float (&acc)[cfg<L, M>::MT][cfg<L, M>::NT][4], const bool multi,
+                                               const int32_t *__restrict__ crd_i, float *__restrict__ out)
 {
     using K = cfg<L, M>;
     static_assert(K::NS == 3, "the register ring below is written for three stages");
@@ -158,16 +178,18 @@ __device__ __forceinline__ void ttm3_warp_item(const sa_item &it, const int32_t 
         if (pn < p1) { k = kflag[pn]; v = vals[pn]; }
         pn += 32;
     };
-    // index/value registers of four batches with FIXED roles: register r holds the batches b with
-    // b % 4 == r and is reloaded (for batch b + 4) right after batch b is consumed.  The batch loop is
-    // unrolled by four so that no register is ever copied while its load is still in flight; the
-    // index of a batch is first needed two rounds after its load (to request its rows).
-    int k0, k1, k2, k3;
-    float v0, v1, v2, v3;
+    // index/value registers of batches B .. B+6: the index of a batch is needed two rounds before its
+    // values (to request its rows), and a streaming load takes several rounds to arrive; row gathers
+    // of batches B+1, B+2 are in flight while B is consumed
+    int k0, k1, k2, k3, k4, k5, k6;
+    float v0, v1, v2, v3, v4, v5, v6;
     load_kv(k0, v0);
     load_kv(k1, v1);
     load_kv(k2, v2);
     load_kv(k3, v3);
+    load_kv(k4, v4);
+    load_kv(k5, v5);
+    load_kv(k6, v6);
     stage_rows<M>(dst_lane, k0, src_lane, row_bytes, gr);
     cp_async_commit();
     if (1 < nb) stage_rows<M>(dst_lane + K::STAGE * 4, k1, src_lane, row_bytes, gr);
@@ -177,6 +199,17 @@ __device__ __forceinline__ void ttm3_warp_item(const sa_item &it, const int32_t 
     load_cfrag<L, M>(cf, C + uint32_t(crd_j[min(f0 + t4, fmax)]) * ldc, C + uint32_t(crd_j[min(f0 + t4 + 4, fmax)]) * ldc, lane);
     float T = 0.f, U = 0.f;                 // two partial sums of the open fiber (shorter dependency chains)
     int s_cur = 0, s_issue = 2;
+    int slice = it.pad;                     // MULTI: position of the slice being accumulated
+    // hand the n (<= 8) oldest closed fibers to the tensor cores and fetch the C values of the next group
+    auto flush_group = [&](int n) {
+        for (int x = n; x < 8; ++x) Tbuf[((nflushed + x) & 15) * K::TS + m] = 0.f;   // unused rows
+        __syncwarp();
+        ttm3_flush<L, M>(acc, Tbuf, nflushed, cf, lane);
+        __syncwarp();
+        nflushed += n;
+        load_cfrag<L, M>(cf, C + uint32_t(crd_j[min(f0 + nflushed + t4, fmax)]) * ldc,
+                         C + uint32_t(crd_j[min(f0 + nflushed + t4 + 4, fmax)]) * ldc, lane);
+    };
     // T += v * d for one nonzero; `end` (warp-uniform) closes the fiber into the ring of temporaries
 #define SA_TTM3_STEP(v, d, end)                                   \
     T = fmaf(v, d, T);                                            \
@@ -186,15 +219,16 @@ __device__ __forceinline__ void ttm3_warp_item(const sa_item &it, const int32_t 
         U = 0.f;                                                  \
         ++nclosed;                                                \
     }
-    // one round: request the rows of batch b + 2 (indices kis), consume batch b (indices/flags kc, values vc)
-    auto do_round = [&](int b, int &kc, float &vc, int kis) {
-        if (b + 2 < nb) stage_rows<M>(dst_lane + s_issue * (K::STAGE * 4), kis, src_lane, row_bytes, gr);
+#pragma unroll 1
+    for (int b = 0; b < nb; ++b) {
+        if (b + 2 < nb) stage_rows<M>(dst_lane + s_issue * (K::STAGE * 4), k2, src_lane, row_bytes, gr);
         cp_async_commit();
-        vs[lane] = vc;
+        vs[lane] = v0;
         cp_async_wait<2>();
         __syncwarp();
         const float *st = wsm + s_cur * K::STAGE + m;
-        unsigned ends = __ballot_sync(SA_FULL_MASK, kc < 0);
+        unsigned ends = __ballot_sync(SA_FULL_MASK, k0 < 0);
+        const unsigned sends = multi ? __ballot_sync(SA_FULL_MASK, (k0 & 0x40000000) != 0) : 0u;
         const int rem = p1 - p0 - 32 * b;
         if (rem <= 32) ends |= 1u << (rem - 1);         // the item's last nonzero closes its (possibly cut) fiber
         const int nchunks = rem >= 32 ? 4 : (rem + 7) >> 3;
@@ -204,6 +238,34 @@ __device__ __forceinline__ void ttm3_warp_item(const sa_item &it, const int32_t 
             const float *sc = st + 8 * c * M;
             const float4 va = *reinterpret_cast<const float4 *>(vs + 8 * c);
             const float4 vb = *reinterpret_cast<const float4 *>(vs + 8 * c + 4);
+            if (((sends >> (8 * c)) & 0xffu) != 0) {
+                // a slice ends inside this chunk: one nonzero at a time, the tile leaves at the slice end
+                const unsigned s8 = (sends >> (8 * c)) & 0xffu;
+                T += U;
+                U = 0.f;
+#pragma unroll 1
+                for (int u = 0; u < 8; ++u) {
+                    T = fmaf(vs[8 * c + u], sc[u * M], T);
+                    if (e8 & (1u << u)) {
+                        Tbuf[(nclosed & 15) * K::TS + m] = T;
+                        T = 0.f;
+                        ++nclosed;
+                        const bool slice_end = (s8 & (1u << u)) != 0;
+                        if (slice_end || nclosed - nflushed >= 8) flush_group(min(8, nclosed - nflushed));
+                        if (slice_end) {
+                            store_tile<L, M>(acc, out + int64_t(crd_i[slice]) * (L * M), lane);
+                            ++slice;
+#pragma unroll
+                            for (int mt = 0; mt < K::MT; ++mt)
+#pragma unroll
+                                for (int nt = 0; nt < K::NT; ++nt)
+#pragma unroll
+                                    for (int q = 0; q < 4; ++q) acc[mt][nt][q] = 0.f;
+                        }
+                    }
+                }
+                continue;
+            }
             if ((e8 & 0xfu) == 0) {
                 T = fmaf(va.x, sc[0], T);
                 U = fmaf(va.y, sc[M], U);
@@ -226,42 +288,24 @@ __device__ __forceinline__ void ttm3_warp_item(const sa_item &it, const int32_t 
                 SA_TTM3_STEP(vb.z, sc[6 * M], e8 & 64u)
                 SA_TTM3_STEP(vb.w, sc[7 * M], e8 & 128u)
             }
-            if (nclosed - nflushed >= 8) {
-                __syncwarp();
-                ttm3_flush<L, M>(acc, Tbuf, nflushed, cf, lane);
-                __syncwarp();
-                nflushed += 8;
-                load_cfrag<L, M>(cf, C + uint32_t(crd_j[min(f0 + nflushed + t4, fmax)]) * ldc,
-                                 C + uint32_t(crd_j[min(f0 + nflushed + t4 + 4, fmax)]) * ldc, lane);
-            }
+            if (nclosed - nflushed >= 8) flush_group(8);
         }
         __syncwarp();                                   // stage s_cur and vs are free for the next round
-        load_kv(kc, vc);                                // batch b + 4
+        k0 = k1; k1 = k2; k2 = k3; k3 = k4; k4 = k5; k5 = k6;
+        v0 = v1; v1 = v2; v2 = v3; v3 = v4; v4 = v5; v5 = v6;
+        load_kv(k6, v6);
         s_issue = s_cur;
         s_cur = s_cur == 2 ? 0 : s_cur + 1;
-    };
-#pragma unroll 1
-    for (int b = 0; b < nb; b += 4) {
-        do_round(b, k0, v0, k2);
-        if (b + 1 < nb) do_round(b + 1, k1, v1, k3);
-        if (b + 2 < nb) do_round(b + 2, k2, v2, k0);
-        if (b + 3 < nb) do_round(b + 3, k3, v3, k1);
     }
 #undef SA_TTM3_STEP
     cp_async_wait<0>();
-    const int pending = nclosed - nflushed;             // 0..7
-    if (pending > 0) {
-        for (int x = pending; x < 8; ++x) Tbuf[((nflushed + x) & 15) * K::TS + m] = 0.f;   // unused rows
-        __syncwarp();
-        ttm3_flush<L, M>(acc, Tbuf, nflushed, cf, lane);
-        __syncwarp();
-    }
+    if (nclosed - nflushed > 0) flush_group(nclosed - nflushed);      // pieces of one slice: the open group
 }
 
 template <int L, int M>
 __global__ void __launch_bounds__(256, 2)
-ttm3_kernel(const sa_item *__restrict__ items, int64_t n_items, int n_group_ctas, const int32_t *__restrict__ crd_j,
-            const int32_t *__restrict__ kflag, const float *__restrict__ vals, const float *__restrict__ C, uint32_t ldc,
+ttm3_kernel(const sa_item *__restrict__ items, int64_t n_items, int n_group_ctas, const int32_t *__restrict__ crd_i,
+            const int32_t *__restrict__ crd_j, const int32_t *__restrict__ kflag, const float *__restrict__ vals, const float *__restrict__ C, uint32_t ldc,
             const float *__restrict__ D, uint32_t ldd, float *__restrict__ out, float *__restrict__ partial)
 {
     using K = cfg<L, M>;
@@ -277,21 +321,11 @@ ttm3_kernel(const sa_item *__restrict__ items, int64_t n_items, int n_group_ctas
     it.f0 = it.f1 = it.p0 = it.p1 = 0;
     it.dest = -1;
     it.out_row = 0;
+    it.pad = it.row_end = 0;
     if (idx < n_items) it = items[idx];
-    if (idx < n_items || group) ttm3_warp_item<L, M>(it, crd_j, kflag, vals, C, ldc, D, ldd, wsm, acc);
-    if (!group) {
-        if (idx >= n_items) return;
-        float *dst = out + int64_t(it.out_row) * TILE;
-#pragma unroll
-        for (int mt = 0; mt < K::MT; ++mt)
-#pragma unroll
-            for (int nt = 0; nt < K::NT; ++nt) {
-                const int l = 16 * mt + g, mm = 8 * nt + 2 * t;
-                sa_st_cs2(dst + l * M + mm, make_float2(acc[mt][nt][0], acc[mt][nt][1]));
-                sa_st_cs2(dst + (l + 8) * M + mm, make_float2(acc[mt][nt][2], acc[mt][nt][3]));
-            }
-        return;
-    }
+    if (idx < n_items || group)
+        ttm3_warp_item<L, M>(it, crd_j, kflag, vals, C, ldc, D, ldd, wsm, acc, !group, crd_i, out);
+    if (!group) return;                 // runs of small slices: every tile was stored at its slice end
     // the CTA's eight warps hold partial tiles of the same slice: sum them in a fixed order
 #pragma unroll
     for (int mt = 0; mt < K::MT; ++mt)
@@ -329,7 +363,7 @@ cudaError_t launch(const sa_tensor *t, const sa_dense *ops, float *out, float *p
     auto kern = ttm3_kernel<L, M>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess)
         return cudaGetLastError();
-    kern<<<(unsigned)ctas, 256, smem, stream>>>(wl.d_items, n_items, int(wl.n_group_ctas), t->d_crd[1], t->d_crd_endflag,
+    kern<<<(unsigned)ctas, 256, smem, stream>>>(wl.d_items, n_items, int(wl.n_group_ctas), t->d_crd[0], t->d_crd[1], t->d_crd_endflag,
                                                t->d_vals, ops[0].ptr, uint32_t(ops[0].ld), ops[1].ptr, uint32_t(ops[1].ld), out, partial);
     return cudaGetLastError();
 }
@@ -351,6 +385,7 @@ sa_status sa_launch_ttm3(const sa_tensor *t, const sa_dense *ops, float *out, vo
     // the kernel addresses factor rows with 32-bit byte offsets
     for (int i = 0; i < 2; ++i)
         if (ops[i].rows * ops[i].ld >= (int64_t(1) << 30)) return SA_E_UNSUPPORTED;
+    if (!t->d_crd_endflag) return SA_E_UNSUPPORTED;      // last dimension >= 2^30: no room for the flag bits
     float *partial = static_cast<float *>(ws);
     cudaError_t e;
     if (L == 16 && M == 16) e = launch<16, 16>(t, ops, out, partial, stream);

@@ -96,14 +96,20 @@ def test_csf_worklist_partitions_every_nonzero_once(cfg):
             assert n < n_groups * 8 and f0 == f1, "only padding items of a group may be empty"
             continue
         s = slice_pos[int(row)]
-        assert pos1[s] <= f0 < f1 <= pos1[s + 1], "fibers stay inside the item's slice"
         fa, fb = _fiber_nnz_range(t, "csf", t.order, levels, f0, f1)
-        assert fa <= p0 < p1 <= fb, "nonzero range lies inside the fiber range"
-        if t.order == 3:     # first and last fiber really intersect the clip range
-            pos2 = levels[2][0]
-            assert pos2[f0 + 1] > p0 and pos2[f1 - 1] < p1
+        if t.order == 3 and n >= n_groups * 8:
+            # a run of whole small slices, named by position: [pad, row_end)
+            s0, s1 = int(items[n][7]), int(row_end)
+            assert s0 == s and s1 > s0 and (f0, f1) == (pos1[s0], pos1[s1]) and (fa, fb) == (p0, p1)
+            assert p1 - p0 <= 2048 or s1 == s0 + 1
         else:
-            assert (fa, fb) == (p0, p1), "order-4 items hold whole (i,j) subtrees"
+            assert pos1[s] <= f0 < f1 <= pos1[s + 1], "fibers stay inside the item's slice"
+            assert fa <= p0 < p1 <= fb, "nonzero range lies inside the fiber range"
+            if t.order == 3:     # first and last fiber really intersect the clip range
+                pos2 = levels[2][0]
+                assert pos2[f0 + 1] > p0 and pos2[f1 - 1] < p1 and int(items[n][7]) == s
+            else:
+                assert (fa, fb) == (p0, p1), "order-4 items hold whole (i,j) subtrees"
         covered[p0:p1] += 1
         if n < n_groups * 8:
             lead = items[(n // 8) * 8]
