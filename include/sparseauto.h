@@ -137,21 +137,38 @@ sa_status sa_tensor_export(const sa_tensor *t, int level, int64_t *pos, int32_t 
 /*
  * Copy a load-balancing work list to HOST arrays (which: 0 = main list, 1 = the CSR tensor's
  * second list used by SA_EXPR_SPMM_GEMM).  These are the slice / fiber / nonzero partition arrays:
- *   counts [4]: number of items, number of leading 8-item groups that one thread block reduces
- *               into a single tile, number of fix-up entries, number of partial-tile slots
+ *   counts [4]: number of items, number of leading groups that one thread block reduces into a
+ *               single tile (8 items each; order-3 tensors: 4 tasks each, see sa_tensor_tasks),
+ *               number of fix-up entries, number of partial-tile slots
  *   items  [n_items * 8] int32 per item: out_row, row_end, f0, f1, p0, p1, dest, half --
  *               fibers [f0,f1) (CSF) clipped to nonzeros [p0,p1) of slice out_row, or rows
  *               [out_row,row_end) / nonzeros [p0,p1) of a long row (CSR); dest = partial slot or -1;
  *               half = 0 / 1 for order-4 tensors, whose items are listed once per half of the
  *               last dense index.  Order-3 tensors use the last field for the position of the
- *               item's (first) slice in the level-0 crd array; items after the leading groups are
- *               runs of whole small slices at positions [that field, row_end), out_row being the
- *               coordinate of the first of them
+ *               item's slice in the level-0 crd array; their items are grouped into tasks, see
+ *               sa_tensor_tasks
  *   fix    [n_fix * 4] int32 per entry: out_row, slot0, count, 0 -- out[out_row] = sum of `count`
  *               partial tiles from slot0 (count 0: the slice / row is empty and is zero-filled)
  * NULL outputs are skipped.
  */
 sa_status sa_tensor_worklist(const sa_tensor *t, int which, int64_t *counts, int32_t *items, int32_t *fix);
+
+/*
+ * Order-3 CSF tensors: how the items of the main work list are handed to warps (the warp-level
+ * partition arrays of the fiber stage).
+ *   n_tasks     number of tasks; warp w of the launch evaluates task w
+ *   task_start  HOST [n_tasks + 1]: task w holds the items [task_start[w], task_start[w + 1]).  The first
+ *               4 * counts[1] tasks (counts of sa_tensor_worklist) hold one item or none: four
+ *               consecutive ones are the pieces of one chunk of a large slice, summed by one thread
+ *               block.  Every later task holds up to 16 whole small slices.
+ *   stream_f0   HOST [n_items * 4]: inside an item the warp's four groups of eight lanes each stream a
+ *               contiguous part of the nonzeros [p0, p1).  With b = p0 rounded down to a multiple of 8
+ *               and s = ceil((p1 - b) / 4) rounded up to a multiple of 8, part q is
+ *               [b + q s, b + (q + 1) s) clipped to [p0, p1); stream_f0[4 n + q] is the level-1 fiber
+ *               that holds the first nonzero of part q of item n (f0 of the item if the part is empty).
+ * NULL outputs are skipped.  Errors: SA_E_ARG, SA_E_FORMAT (not an order-3 CSF tensor).
+ */
+sa_status sa_tensor_tasks(const sa_tensor *t, int64_t *n_tasks, int32_t *task_start, int32_t *stream_f0);
 
 /* Bytes of DEVICE workspace sa_run needs for this tensor / expression / schedule / operand
  * shapes (may be 0).  Only the shapes in ops are read. */
@@ -211,6 +228,11 @@ sa_status sa_last_launch_count(const sa_tensor *t, int *launches);
 /* Synchronise cuda_stream and report the device-side status word of the tensor (SA_OK,
  * SA_E_BOUNDS, SA_E_TIMEOUT), clearing it. */
 sa_status sa_last_device_status(const sa_tensor *t, void *cuda_stream);
+
+/* Synchronise cuda_stream and copy the raw status word to HOST words[4] without clearing it: words[0] is
+ * 0 or the status above; for SA_E_BOUNDS (set only by a library built with -DSA_DEBUG_BOUNDS) words[1] is
+ * the number of the check that failed, words[2] the offending index, words[3] the global thread. */
+sa_status sa_device_status_words(const sa_tensor *t, void *cuda_stream, int32_t *words);
 
 /* Release device and host memory of the handle.  NULL is accepted. */
 void sa_destroy(sa_tensor *t);

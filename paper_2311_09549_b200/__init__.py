@@ -28,7 +28,7 @@ SA_SCHED_DEFAULT, SA_SCHED_FUSED, SA_SCHED_ASSOC_LEFT, SA_SCHED_ASSOC_RIGHT = 0,
 SA_SCHED_DEBUG_MATERIALIZE = 9
 
 EXPORTED_SYMBOLS = ["sa_tensor_create", "sa_tensor_info", "sa_tensor_export", "sa_tensor_worklist",
-                    "sa_workspace_size", "sa_run", "sa_last_launch_count", "sa_last_device_status",
+                    "sa_tensor_tasks", "sa_workspace_size", "sa_run", "sa_last_launch_count", "sa_last_device_status", "sa_device_status_words",
                     "sa_destroy", "sa_status_string", "sa_run_ttm3_static_scratch"]
 
 
@@ -49,10 +49,12 @@ _lib.sa_tensor_create.argtypes = [_int, _vp, _i64, _vp, _vp, _int, _int, ctypes.
 _lib.sa_tensor_info.argtypes = [_vp, ctypes.POINTER(_i64), _vp, ctypes.POINTER(_i64)]
 _lib.sa_tensor_export.argtypes = [_vp, _int, _vp, _vp, _vp]
 _lib.sa_tensor_worklist.argtypes = [_vp, _int, _vp, _vp, _vp]
+_lib.sa_tensor_tasks.argtypes = [_vp, ctypes.POINTER(_i64), _vp, _vp]
 _lib.sa_workspace_size.argtypes = [_vp, _int, _int, ctypes.POINTER(SaDense), _int, ctypes.POINTER(ctypes.c_size_t)]
 _lib.sa_run.argtypes = [_vp, _int, _int, ctypes.POINTER(SaDense), _int, _vp, _vp, ctypes.c_size_t, _vp]
 _lib.sa_last_launch_count.argtypes = [_vp, ctypes.POINTER(_int)]
 _lib.sa_last_device_status.argtypes = [_vp, _vp]
+_lib.sa_device_status_words.argtypes = [_vp, _vp, _vp]
 _lib.sa_destroy.argtypes = [_vp]
 _lib.sa_destroy.restype = None
 _lib.sa_status_string.argtypes = [_int]
@@ -142,6 +144,18 @@ def sa_tensor_worklist(handle, which=0):
     return counts, items, fix
 
 
+def sa_tensor_tasks(handle):
+    """Order-3 CSF: (task_start int32 [n_tasks + 1], stream_f0 int32 [n_items, 4])."""
+    n = _i64()
+    _check(_lib.sa_tensor_tasks(handle, ctypes.byref(n), None, None), "sa_tensor_tasks")
+    counts = np.zeros(4, dtype=np.int64)
+    _check(_lib.sa_tensor_worklist(handle, 0, counts.ctypes.data, None, None), "sa_tensor_worklist")
+    task_start = np.zeros(n.value + 1, dtype=np.int32)
+    stream_f0 = np.zeros((int(counts[0]), 4), dtype=np.int32)
+    _check(_lib.sa_tensor_tasks(handle, None, task_start.ctypes.data, stream_f0.ctypes.data), "sa_tensor_tasks")
+    return task_start, stream_f0
+
+
 def _dense_array(ops):
     arr = (SaDense * len(ops))()
     for i, (ptr, rows, cols, ld) in enumerate(ops):
@@ -179,6 +193,12 @@ def sa_last_launch_count(handle):
 
 def sa_last_device_status(handle, stream):
     return int(_lib.sa_last_device_status(handle, stream))
+
+
+def sa_device_status_words(handle, stream):
+    words = np.zeros(4, dtype=np.int32)
+    _check(_lib.sa_device_status_words(handle, stream, words.ctypes.data), "sa_device_status_words")
+    return words
 
 
 def sa_destroy(handle):

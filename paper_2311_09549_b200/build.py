@@ -21,7 +21,9 @@ def _stale():
 
 
 def build(force=False, verbose=False):
-    if not force and not _stale():
+    """SA_NVCC_EXTRA (environment) adds flags, e.g. -DSA_DEBUG_BOUNDS for the self-checking kernels."""
+    extra = os.environ.get("SA_NVCC_EXTRA", "").split()
+    if not force and not extra and not _stale():
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     objs = []
@@ -29,7 +31,7 @@ def build(force=False, verbose=False):
     os.makedirs(os.path.join(HERE, "_build"), exist_ok=True)
     for src in SOURCES:
         obj = os.path.join(HERE, "_build", src.replace(".cu", ".o"))
-        cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-c", os.path.join(CSRC, src), "-o", obj]
+        cmd = [nvcc] + NVCC_FLAGS + extra + (["-Xptxas", "-v"] if verbose else []) + ["-c", os.path.join(CSRC, src), "-o", obj]
         procs.append((src, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
         objs.append(obj)
     failed = False

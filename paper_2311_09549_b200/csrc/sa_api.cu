@@ -18,16 +18,20 @@ void *default_alloc(size_t bytes, void *)
 
 void default_release(void *p, void *) { cudaFree(p); }
 
-// Allocate device memory through the tensor's allocator and copy n elements of src into it.
+// Allocate device memory through the tensor's allocator and copy n elements of src into it.  The block
+// ends with at least 64 zero bytes: kernels that read index and value arrays in aligned groups of eight
+// elements may run past the last element and must find valid (zero) indices there.
 template <typename T>
 sa_status upload(sa_tensor *t, const T *src, size_t n, T **dst)
 {
     *dst = nullptr;
-    const size_t bytes = sa_align256((n ? n : 1) * sizeof(T));
+    const size_t used = n * sizeof(T);
+    const size_t bytes = sa_align256(used + 64);
     void *p = t->alloc.alloc(bytes, t->alloc.ctx);
     if (!p) return SA_E_ALLOC;
     t->dev_blocks.push_back(p);
-    if (n && cudaMemcpy(p, src, n * sizeof(T), cudaMemcpyHostToDevice) != cudaSuccess) return SA_E_CUDA;
+    if (n && cudaMemcpy(p, src, used, cudaMemcpyHostToDevice) != cudaSuccess) return SA_E_CUDA;
+    if (cudaMemset(static_cast<char *>(p) + used, 0, bytes - used) != cudaSuccess) return SA_E_CUDA;
     *dst = static_cast<T *>(p);
     return SA_OK;
 }
@@ -41,9 +45,19 @@ sa_status upload_pos32(sa_tensor *t, const std::vector<int64_t> &pos, int32_t **
 
 sa_status upload_worklist(sa_tensor *t, sa_worklist &wl)
 {
-    sa_status s = upload(t, wl.items.data(), wl.items.size(), &wl.d_items);
+    sa_status s = upload(t, wl.fix.data(), wl.fix.size(), &wl.d_fix);
     if (s != SA_OK) return s;
-    return upload(t, wl.fix.data(), wl.fix.size(), &wl.d_fix);
+    if (wl.task_start.empty()) return upload(t, wl.items.data(), wl.items.size(), &wl.d_items);
+    // order-3 CSF: the kernel reads the compact per-unit records and the task list
+    std::vector<sa_unit3> units(wl.items.size());
+    for (size_t u = 0; u < units.size(); ++u) {
+        const sa_item &it = wl.items[u];
+        units[u].out_row = it.out_row; units[u].dest = it.dest; units[u].p0 = it.p0; units[u].p1 = it.p1;
+        for (int q = 0; q < SA_STREAMS; ++q) units[u].sf[q] = wl.stream_f0[u * SA_STREAMS + size_t(q)];
+    }
+    s = upload(t, units.data(), units.size(), &wl.d_units3);
+    if (s != SA_OK) return s;
+    return upload(t, wl.task_start.data(), wl.task_start.size(), &wl.d_task_start);
 }
 
 struct device_guard {
@@ -211,14 +225,14 @@ sa_status sa_tensor_create(int order, const int64_t *dims, int64_t nnz, const in
             if (s == SA_OK) s = upload(t, t->crd[l].data(), t->crd[l].size(), &t->d_crd[l]);
         }
         if (s == SA_OK) s = upload(t, t->vals.data(), t->vals.size(), &t->d_vals);
-        if (s == SA_OK && fmt == SA_FMT_CSF && order == 3 && t->dims[2] < (int64_t(1) << 30)) {
-            // bit 31: last nonzero of its (i,j) fiber; bit 30: last nonzero of its slice
-            std::vector<int32_t> flagged(t->crd[2]);
-            for (int64_t f = 0; f < t->count[1]; ++f)
-                flagged[size_t(t->pos[2][size_t(f) + 1] - 1)] |= int32_t(0x80000000u);
-            for (int64_t sl = 0; sl < t->count[0]; ++sl)
-                flagged[size_t(t->pos[2][size_t(t->pos[1][size_t(sl) + 1])] - 1)] |= int32_t(0x40000000);
-            s = upload(t, flagged.data(), flagged.size(), &t->d_crd_endflag);
+        if (s == SA_OK && fmt == SA_FMT_CSF && order == 3) {
+            // one bit per nonzero: set on the last nonzero of every (i,j) fiber
+            std::vector<uint32_t> bits(size_t(nnz / 32 + 1), 0u);
+            for (int64_t f = 0; f < t->count[1]; ++f) {
+                const int64_t p = t->pos[2][size_t(f) + 1] - 1;
+                bits[size_t(p >> 5)] |= 1u << (p & 31);
+            }
+            s = upload(t, bits.data(), bits.size(), &t->d_endbits);
         }
         if (s == SA_OK && fmt == SA_FMT_CSF && order == 4 && t->dims[3] < (int64_t(1) << 30)) {
             // bit 31: last nonzero of its (i,j,k) fiber; bit 30: last nonzero of its (i,j) fiber
@@ -278,6 +292,17 @@ sa_status sa_tensor_worklist(const sa_tensor *t, int which, int64_t *counts, int
     return SA_OK;
 }
 
+sa_status sa_tensor_tasks(const sa_tensor *t, int64_t *n_tasks, int32_t *task_start, int32_t *stream_f0)
+{
+    if (!t) return SA_E_ARG;
+    if (t->fmt != SA_FMT_CSF || t->order != 3) return SA_E_FORMAT;
+    const sa_worklist &wl = t->wl_main;
+    if (n_tasks) *n_tasks = int64_t(wl.task_start.size()) - 1;
+    if (task_start) std::memcpy(task_start, wl.task_start.data(), wl.task_start.size() * sizeof(int32_t));
+    if (stream_f0) std::memcpy(stream_f0, wl.stream_f0.data(), wl.stream_f0.size() * sizeof(int32_t));
+    return SA_OK;
+}
+
 sa_status sa_workspace_size(const sa_tensor *t, sa_expr expr, sa_schedule sched, const sa_dense *ops, int n_ops,
                             size_t *bytes)
 {
@@ -327,6 +352,20 @@ sa_status sa_last_launch_count(const sa_tensor *t, int *launches)
 {
     if (!t || !launches) return SA_E_ARG;
     *launches = t->last_launches;
+    return SA_OK;
+}
+
+sa_status sa_device_status_words(const sa_tensor *t, void *cuda_stream, int32_t *words)
+{
+    if (!t || t->device < 0 || !words) return SA_E_ARG;
+    device_guard g(t->device);
+    if (!g.ok) return SA_E_CUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaMemcpyAsync(words, t->d_status, 4 * sizeof(int32_t), cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+        cudaStreamSynchronize(stream) != cudaSuccess) {
+        cudaGetLastError();
+        return SA_E_CUDA;
+    }
     return SA_OK;
 }
 

@@ -185,40 +185,31 @@ void append_empty_slices(sa_tensor *t, sa_worklist &wl)
     }
 }
 
-// Order-3 CSF: warp items are fiber ranges clipped to a nonzero range.
+// Order-3 CSF.  An item ("unit") is a piece [p0, p1) of one slice with the fibers [f0, f1) it touches (a
+// fiber may be cut between two units, each adds its part).  Slices above SMALL_MAX nonzeros are cut into
+// chunks; the SA_TTM3_WARPS warps of a thread block take equal pieces of a chunk and reduce their tiles on chip.
+// Smaller slices are one unit each; a warp evaluates a task of up to MAX_UNITS such units, about
+// SMALL_MAX nonzeros in total.  Inside a unit the warp's SA_STREAMS lane groups stream the parts given by
+// sa_unit3_streams; stream_f0 holds the fiber in which each part starts.
 void build_ttm3(sa_tensor *t, sa_worklist &wl)
 {
-    constexpr int64_t SMALL_MAX = 2048, MIN_CHUNK = 8192, MAX_PARTS = 192;
+    constexpr int64_t SMALL_MAX = 2048, MIN_CHUNK = 8192, MAX_PARTS = 192, MAX_UNITS = 16;
     const auto &pos1 = t->pos[1];
     const auto &pos2 = t->pos[2];
     std::vector<sa_item> small;
     std::vector<group_rec> groups;
-    // Runs of consecutive small slices are merged into one warp item of at most SMALL_MAX nonzeros: the
-    // warp streams through them without restarting its pipelines and stores one tile per slice.  Such an
-    // item names its slices by position: pad = first slice position, row_end = one past the last.
-    sa_item run = empty_item();
-    bool open = false;
-    auto close_run = [&]() {
-        if (open) small.push_back(run);
-        open = false;
-    };
     for (int64_t s = 0; s < t->count[0]; ++s) {
         const int64_t fa = pos1[size_t(s)], fb = pos1[size_t(s) + 1];
         const int64_t pa = pos2[size_t(fa)], pb = pos2[size_t(fb)];
         const int64_t n = pb - pa;
         const int32_t row = t->crd[0][size_t(s)];
         if (n <= SMALL_MAX) {
-            if (open && (pb - run.p0) > SMALL_MAX) close_run();
-            if (!open) {
-                run = empty_item();
-                run.out_row = row; run.pad = int32_t(s);
-                run.f0 = int32_t(fa); run.p0 = int32_t(pa);
-                open = true;
-            }
-            run.row_end = int32_t(s + 1); run.f1 = int32_t(fb); run.p1 = int32_t(pb);
+            sa_item it = empty_item();
+            it.out_row = row; it.row_end = row + 1; it.pad = int32_t(s);
+            it.f0 = int32_t(fa); it.f1 = int32_t(fb); it.p0 = int32_t(pa); it.p1 = int32_t(pb);
+            small.push_back(it);
             continue;
         }
-        close_run();
         const int64_t chunk = chunk_for(n, MIN_CHUNK, MAX_PARTS);
         const int64_t ng = (n + chunk - 1) / chunk;
         int32_t slot0 = -1;
@@ -229,33 +220,57 @@ void build_ttm3(sa_tensor *t, sa_worklist &wl)
         }
         for (int64_t g = 0; g < ng; ++g) {
             const int64_t ga = pa + g * chunk, gb = std::min(pb, ga + chunk);
-            int64_t piece = (gb - ga + SA_WARPS_PER_CTA - 1) / SA_WARPS_PER_CTA;
+            int64_t piece = (gb - ga + SA_TTM3_WARPS - 1) / SA_TTM3_WARPS;
             piece = (piece + 31) / 32 * 32;
             group_rec rec;
             rec.len = gb - ga;
-            for (int w = 0; w < SA_WARPS_PER_CTA; ++w) {
-                sa_item it = empty_item();
-                it.out_row = row; it.pad = int32_t(s); it.row_end = int32_t(s + 1);
-                it.dest = ng > 1 ? slot0 + int32_t(g) : -1;
+            for (int w = 0; w < SA_TTM3_WARPS; ++w) {
                 const int64_t qa = std::min(gb, ga + w * piece), qb = std::min(gb, qa + piece);
-                if (qa < qb) {
-                    // fiber holding nonzero qa, and one past the fiber holding nonzero qb - 1
-                    const int64_t f0 = (std::upper_bound(pos2.begin() + fa, pos2.begin() + fb + 1, qa) - pos2.begin()) - 1;
-                    const int64_t f1 = (std::upper_bound(pos2.begin() + fa, pos2.begin() + fb + 1, qb - 1) - pos2.begin());
-                    it.f0 = int32_t(f0); it.f1 = int32_t(f1); it.p0 = int32_t(qa); it.p1 = int32_t(qb);
-                }
+                if (qa >= qb) break;              // the remaining warps of this block have nothing to do
+                sa_item it = empty_item();
+                it.out_row = row; it.row_end = row + 1; it.pad = int32_t(s);
+                it.dest = ng > 1 ? slot0 + int32_t(g) : -1;
+                // fiber holding nonzero qa, and one past the fiber holding nonzero qb - 1
+                const int64_t f0 = (std::upper_bound(pos2.begin() + fa, pos2.begin() + fb + 1, qa) - pos2.begin()) - 1;
+                const int64_t f1 = (std::upper_bound(pos2.begin() + fa, pos2.begin() + fb + 1, qb - 1) - pos2.begin());
+                it.f0 = int32_t(f0); it.f1 = int32_t(f1); it.p0 = int32_t(qa); it.p1 = int32_t(qb);
                 rec.items.push_back(it);
             }
             groups.push_back(std::move(rec));
         }
     }
-    close_run();
     std::stable_sort(groups.begin(), groups.end(), [](const group_rec &a, const group_rec &b) { return a.len > b.len; });
     std::stable_sort(small.begin(), small.end(),
                      [](const sa_item &a, const sa_item &b) { return (a.p1 - a.p0) > (b.p1 - b.p0); });
     wl.n_group_ctas = int64_t(groups.size());
-    for (auto &g : groups) wl.items.insert(wl.items.end(), g.items.begin(), g.items.end());
-    wl.items.insert(wl.items.end(), small.begin(), small.end());
+    wl.task_start.clear();
+    for (auto &g : groups)
+        for (int w = 0; w < SA_TTM3_WARPS; ++w) {
+            wl.task_start.push_back(int32_t(wl.items.size()));
+            if (size_t(w) < g.items.size()) wl.items.push_back(g.items[size_t(w)]);
+        }
+    for (size_t x = 0; x < small.size();) {
+        wl.task_start.push_back(int32_t(wl.items.size()));
+        int64_t total = 0, cnt = 0;
+        while (x < small.size() && cnt < MAX_UNITS && (cnt == 0 || total + (small[x].p1 - small[x].p0) <= SMALL_MAX)) {
+            total += small[x].p1 - small[x].p0;
+            wl.items.push_back(small[x]);
+            ++x; ++cnt;
+        }
+    }
+    wl.task_start.push_back(int32_t(wl.items.size()));
+    wl.stream_f0.resize(wl.items.size() * SA_STREAMS);
+    for (size_t u = 0; u < wl.items.size(); ++u) {
+        const sa_item &it = wl.items[u];
+        int64_t lo[SA_STREAMS], hi[SA_STREAMS];
+        sa_unit3_streams(it.p0, it.p1, lo, hi);
+        for (int q = 0; q < SA_STREAMS; ++q) {
+            int64_t f = it.f0;
+            if (lo[q] < hi[q])
+                f = (std::upper_bound(pos2.begin() + it.f0, pos2.begin() + it.f1 + 1, lo[q]) - pos2.begin()) - 1;
+            wl.stream_f0[u * SA_STREAMS + size_t(q)] = int32_t(f);
+        }
+    }
     append_empty_slices(t, wl);
 }
 

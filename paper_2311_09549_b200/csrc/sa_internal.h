@@ -10,6 +10,7 @@
 
 constexpr int SA_MAX_ORDER = 4;
 constexpr int SA_WARPS_PER_CTA = 8;
+constexpr int SA_TTM3_WARPS = 4;     // warps per thread block of the order-3 kernel (they share one chunk of a large slice)
 
 // One unit of work for one warp.  32 bytes, read once per warp.
 //   CSF tensors: a contiguous range of level-1 fibers [f0, f1) inside ONE slice, clipped to the
@@ -35,6 +36,33 @@ struct sa_fix {
     int32_t pad;
 };
 
+// Order-3 CSF only: what the kernel reads per item (a piece of one slice, "unit").  The warp's 32 lanes
+// form SA_STREAMS groups of 8 lanes; each group streams one contiguous part of [p0, p1) whose start is a
+// multiple of 8 nonzeros (see sa_unit3_streams); sf[q] is the level-1 fiber that holds the first
+// nonzero of part q.
+constexpr int SA_STREAMS = 4;
+struct sa_unit3 {
+    int32_t out_row;
+    int32_t dest;
+    int32_t p0, p1;
+    int32_t sf[SA_STREAMS];
+};
+static_assert(sizeof(sa_unit3) == 32, "sa_unit3 is read as two 16-byte pieces");
+
+// Nonzero ranges of the SA_STREAMS parts of a unit [p0, p1): part q = [lo[q], hi[q]) (empty if lo >= hi);
+// every part starts at base8 + q * slen with base8 = p0 rounded down to a multiple of 8 and slen a
+// multiple of 8, clipped to [p0, p1).  The same arithmetic runs in the kernel.
+static inline void sa_unit3_streams(int64_t p0, int64_t p1, int64_t *lo, int64_t *hi)
+{
+    const int64_t base8 = p0 & ~int64_t(7), span = p1 - base8;
+    const int64_t slen = ((span + SA_STREAMS - 1) / SA_STREAMS + 7) & ~int64_t(7);
+    for (int q = 0; q < SA_STREAMS; ++q) {
+        const int64_t a = base8 + q * slen;
+        lo[q] = a > p0 ? a : p0;
+        hi[q] = a + slen < p1 ? a + slen : p1;
+    }
+}
+
 struct sa_worklist {
     std::vector<sa_item> items;   // [n_group_ctas * SA_WARPS_PER_CTA group items][warp items]
     std::vector<sa_fix> fix;
@@ -42,6 +70,12 @@ struct sa_worklist {
     int64_t n_slots = 0;          // partial tiles in the workspace
     sa_item *d_items = nullptr;
     sa_fix *d_fix = nullptr;
+    // order-3 CSF: warp w evaluates items [task_start[w], task_start[w + 1]); the first
+    // n_group_ctas * SA_TTM3_WARPS tasks hold at most one item each
+    std::vector<int32_t> task_start;
+    std::vector<int32_t> stream_f0;   // [items * SA_STREAMS]
+    int32_t *d_task_start = nullptr;
+    sa_unit3 *d_units3 = nullptr;
 };
 
 struct sa_tensor {
@@ -63,9 +97,10 @@ struct sa_tensor {
     int32_t *d_pos[SA_MAX_ORDER] = {nullptr, nullptr, nullptr, nullptr};
     int32_t *d_crd[SA_MAX_ORDER] = {nullptr, nullptr, nullptr, nullptr};
     float *d_vals = nullptr;
-    int32_t *d_crd_endflag = nullptr;         // CSF: last-level crd with bit 31 set on the last nonzero of
-                                              // every last-level fiber (order 4: bit 30 on the last nonzero
-                                              // of every (i,j) fiber as well)
+    int32_t *d_crd_endflag = nullptr;         // order-4 CSF: last-level crd with bit 31 set on the last nonzero of
+                                              // every (i,j,k) fiber and bit 30 on the last nonzero of every (i,j) fiber
+    uint32_t *d_endbits = nullptr;            // order-3 CSF: bit (p & 31) of word p / 32 is set when nonzero p is the
+                                              // last of its (i,j) fiber
     int32_t *d_status = nullptr;              // [4] device status word
 
     sa_worklist wl_main;                      // TTM3 / TTM4 / SDDMM-SpMM

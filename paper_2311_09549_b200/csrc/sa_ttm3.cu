@@ -1,13 +1,21 @@
 // Kernel 6 <SpTTM,TTM>:  A(i,l,m) = sum_{j,k} B(i,j,k) C(j,l) D(k,m), scheduled as the branched
 // nest  i, j' < t ; k': t += B(i,j,k) D(k,m) , l: A(i,l,m) += t C(j,l) >  of the paper's Table of
-// kernels (Section 6).  Producer (SpTTM, fp32 ALU): the nonzeros of a work item are streamed in
-// flat batches of 32; the D rows of a batch are gathered with cp.async into a per-warp ring of
-// shared-memory stages (several batches in flight per warp, no registers tied up); the fiber
-// temporary t(m) lives in one register per lane (lane = m) and is closed by an end-of-fiber flag
-// carried in the index stream.  Consumer (TTM, tensor cores): closed temporaries are staged eight
-// at a time in shared memory and the slice tile is updated as A(i,:,:) += Cg^T (L x 8) . T (8 x M)
-// with m16n8k8 TF32 MMAs, each operand split into a high and a low TF32 part (three products) so
-// the stage keeps fp32-level accuracy.  The order-3 intermediate T(i,j,m) is never stored.
+// kernels (Section 6).
+//
+// Producer (SpTTM, fp32 ALU).  A warp is four independent lane groups ("streams") of eight lanes.  Every
+// stream walks its own contiguous part of the unit's nonzeros, eight per round; a lane holds M/8
+// consecutive entries of the fiber temporary t(:), so the eight lanes of a stream fetch one row D(k,:)
+// with a single vector load and the row is consumed from registers one round after it was requested
+// (eight rows in flight per lane).  The index, value and end-of-fiber-bit arrays reach the streams
+// through a per-warp cp.async ring in shared memory that runs seven rounds ahead and continues across
+// the units of a task, so a warp that evaluates many small slices never drains its pipelines.
+// Consumer (TTM, tensor cores).  A stream that meets an end-of-fiber bit parks t(:) and the fiber's C row
+// offset in a ring of rows in shared memory; eight parked rows at a time update the slice tile as
+// A(i,:,:) += Cg^T (L x 8) . T (8 x M) with m16n8k8 TF32 MMAs, each operand split into a high and a low
+// TF32 part (three products), which keeps fp32-level accuracy.  The order-3 intermediate T(i,j,m) is
+// never stored.
+#include <type_traits>
+
 #include "sa_device.cuh"
 
 namespace {
@@ -32,26 +40,49 @@ __device__ __forceinline__ void mma_m16n8k8_tf32(float (&c)[4], const uint32_t (
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
 }
 
-__device__ __forceinline__ void cp_async16(float *dst_smem, const float *src)
-{
-    const uint32_t d = static_cast<uint32_t>(__cvta_generic_to_shared(dst_smem));
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(src) : "memory");
-}
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
+
+// Debug build (-DSA_DEBUG_BOUNDS): every index that comes out of the tensor's arrays is checked before it
+// is turned into an address; the first violation is recorded in the tensor's status word (read back by
+// sa_last_device_status) and the access is redirected to element 0.  Nothing traps.
+struct dbg_limits {
+    int32_t *status;
+    uint32_t c_rows, d_rows, n_fibers, n_slices_dim;
+    int64_t nnz;
+};
+#ifdef SA_DEBUG_BOUNDS
+__device__ __forceinline__ bool dbg_ok(const dbg_limits &lim, bool ok, int code, int64_t value)
+{
+    if (!ok && atomicCAS(lim.status, 0, int(SA_E_BOUNDS)) == 0) {
+        lim.status[1] = code;
+        lim.status[2] = int32_t(value);
+        lim.status[3] = int32_t(blockIdx.x * blockDim.x + threadIdx.x);
+    }
+    return ok;
+}
+#define SA_CHK(lim, cond, code, value) dbg_ok(lim, cond, code, int64_t(value))
+#else
+#define SA_CHK(lim, cond, code, value) true
+#endif
+
 template <int L, int M>
 struct cfg {
-    static constexpr int MT = L / 16;       // m16 tiles over l
-    static constexpr int NT = M / 8;        // n8 tiles over m
-    static constexpr int TS = M;            // row stride of the staged temporaries (unpadded: two CTAs of
-                                            // 8 warps x (3 stages + ring) must fit one SM's shared memory)
-    static constexpr int RS = M + 8;        // row stride of a warp's tile in the CTA reduction
-    static constexpr int NS = 3;            // cp.async stages (batches of 32 factor rows) per warp
-    static constexpr int STAGE = 32 * M;    // floats per stage
-    static constexpr int WORK = NS * STAGE + 16 * TS + 32;                 // stages + ring of temporaries + values of a batch
-    static constexpr int WARP_SMEM = (L * RS > WORK ? L * RS : WORK);      // floats per warp
+    static constexpr int MT = L / 16;            // m16 tiles over l
+    static constexpr int NT = M / 8;             // n8 tiles over m
+    static constexpr int NS = SA_STREAMS;        // streams per warp
+    static constexpr int VEC = M / 8;            // floats of a factor row per lane (eight lanes per row)
+    static constexpr int RS = M + 8;             // row stride of the ring of parked temporaries and of a warp's
+                                                 // tile in the CTA reduction; word M of a ring row = C row offset
+    static constexpr int RING = 64;              // ring rows: at most 7 left over + 32 parked in one round
+    static constexpr int DEPTH = 8;              // rounds of index / value data in flight (cp.async ring)
+    static constexpr int SLOT = 80;              // bytes per (round, stream): 8 indices | 8 values | end bits | pad
+    static constexpr int OFF_KV = 0;
+    static constexpr int OFF_RING = OFF_KV + DEPTH * NS * SLOT;
+    static constexpr int WARP_BYTES = OFF_RING + RING * RS * 4;
+    static_assert(L * RS * 4 <= WARP_BYTES, "the CTA reduction reuses a warp's region for its tile");
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
@@ -59,53 +90,85 @@ __device__ __forceinline__ void cp_async16_raw(uint32_t dst_smem, const void *sr
 {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst_smem), "l"(src) : "memory");
 }
-
-// Gather the 32 rows D(k_s, :) of one batch into a stage: LPR lanes copy one row in 16-byte pieces.
-// dst_lane: shared address of the stage plus this lane's (row-in-group, piece) offset; src_lane: D plus
-// the lane's piece offset; row_bytes = 4 * ld(D) (byte offsets fit 32 bits, checked by the launcher).
-template <int M>
-__device__ __forceinline__ void stage_rows(uint32_t dst_lane, int kbatch, const char *__restrict__ src_lane,
-                                           uint32_t row_bytes, int r)
+__device__ __forceinline__ void cp_async4_raw(uint32_t dst_smem, const void *src)
 {
-    constexpr int LPR = M / 4, RPI = 32 / LPR;
-#pragma unroll
-    for (int q = 0; q < 32 / RPI; ++q) {
-        const uint32_t k = uint32_t(__shfl_sync(SA_FULL_MASK, kbatch, q * RPI + r)) & 0x3fffffffu;
-        cp_async16_raw(dst_lane + q * RPI * M * 4, src_lane + k * row_bytes);
-    }
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst_smem), "l"(src) : "memory");
 }
-
-// The values of C one flush needs: rows of the fibers x = t and x = t + 4 of the next group of eight,
-// columns 16 mt + g and 16 mt + g + 8.  Loaded right after the previous flush so that the L2 latency
-// is covered by the producer work in between.
-template <int L, int M>
-__device__ __forceinline__ void load_cfrag(float (&cf)[cfg<L, M>::MT][4], const float *__restrict__ crow_a,
-                                           const float *__restrict__ crow_b, int lane)
+__device__ __forceinline__ uint32_t lds32(uint32_t a)
 {
-    const int g = lane >> 2;
-#pragma unroll
-    for (int mt = 0; mt < cfg<L, M>::MT; ++mt) {
-        cf[mt][0] = __ldg(crow_a + 16 * mt + g);
-        cf[mt][1] = __ldg(crow_a + 16 * mt + g + 8);
-        cf[mt][2] = __ldg(crow_b + 16 * mt + g);
-        cf[mt][3] = __ldg(crow_b + 16 * mt + g + 8);
-    }
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a));
+    return v;
 }
+__device__ __forceinline__ uint4 lds128(uint32_t a)
+{
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ void sts32(uint32_t a, uint32_t v) { asm volatile("st.shared.u32 [%0], %1;" ::"r"(a), "r"(v) : "memory"); }
+__device__ __forceinline__ void prefetch_l1(const void *p) { asm volatile("prefetch.global.L1 [%0];" ::"l"(p)); }
 
-// acc += Cg^T . T for eight staged fibers: rows (row0 + x) & 15, x = 0..7, of the 16-row ring.
+// A lane's piece of a factor row: VEC = 4 or 2 consecutive floats, read once and not kept in L1.
+template <int VEC>
+struct rowvec;
+template <>
+struct rowvec<4> {
+    float x[4];
+    __device__ __forceinline__ void load(const char *p)
+    {
+        asm volatile("ld.global.nc.L1::no_allocate.v4.f32 {%0,%1,%2,%3}, [%4];"
+                     : "=f"(x[0]), "=f"(x[1]), "=f"(x[2]), "=f"(x[3]) : "l"(p));
+    }
+    __device__ __forceinline__ void store_shared(uint32_t a) const
+    {
+        asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};" ::"r"(a), "f"(x[0]), "f"(x[1]), "f"(x[2]), "f"(x[3]) : "memory");
+    }
+};
+template <>
+struct rowvec<2> {
+    float x[2];
+    __device__ __forceinline__ void load(const char *p)
+    {
+        asm volatile("ld.global.nc.L1::no_allocate.v2.f32 {%0,%1}, [%2];" : "=f"(x[0]), "=f"(x[1]) : "l"(p));
+    }
+    __device__ __forceinline__ void store_shared(uint32_t a) const
+    {
+        asm volatile("st.shared.v2.f32 [%0], {%1,%2};" ::"r"(a), "f"(x[0]), "f"(x[1]) : "memory");
+    }
+};
+
+// acc += Cg^T . T for the ring rows (row0 + x) & (RING - 1), x = 0 .. 7, of which the first n are in use.
 template <int L, int M>
-__device__ __forceinline__ void ttm3_flush(float (&acc)[cfg<L, M>::MT][cfg<L, M>::NT][4], const float *__restrict__ Tbuf,
-                                           int row0, const float (&cf)[cfg<L, M>::MT][4], int lane)
+__device__ __forceinline__ void ttm3_flush(float (&acc)[cfg<L, M>::MT][cfg<L, M>::NT][4], const float *__restrict__ ring,
+                                           int row0, int n, const float *__restrict__ C, int lane, const dbg_limits &lim, uint32_t ldc)
 {
     using K = cfg<L, M>;
     const int g = lane >> 2, t = lane & 3;
-    const float *ta = Tbuf + ((row0 + t) & 15) * K::TS + g;
-    const float *tb = Tbuf + ((row0 + t + 4) & 15) * K::TS + g;
+    const float *ra = ring + ((row0 + t) & (K::RING - 1)) * K::RS;
+    const float *rb = ring + ((row0 + t + 4) & (K::RING - 1)) * K::RS;
+    // the values of C this flush needs: rows of the fibers x = t and x = t + 4, columns 16 mt + g (+ 8)
+    float cf[K::MT][4];
+    {
+        const bool va = t < n, vb = t + 4 < n;
+        uint32_t oa = va ? __float_as_uint(ra[M]) : 0u, ob = vb ? __float_as_uint(rb[M]) : 0u;
+        if (!SA_CHK(lim, oa < lim.c_rows * ldc, 1, oa)) oa = 0u;
+        if (!SA_CHK(lim, ob < lim.c_rows * ldc, 2, ob)) ob = 0u;
+        const float *ca = C + oa + g;
+        const float *cb = C + ob + g;
+#pragma unroll
+        for (int mt = 0; mt < K::MT; ++mt) {
+            cf[mt][0] = va ? __ldg(ca + 16 * mt) : 0.f;
+            cf[mt][1] = va ? __ldg(ca + 16 * mt + 8) : 0.f;
+            cf[mt][2] = vb ? __ldg(cb + 16 * mt) : 0.f;
+            cf[mt][3] = vb ? __ldg(cb + 16 * mt + 8) : 0.f;
+        }
+    }
     uint32_t bh[K::NT][2], bl[K::NT][2];
 #pragma unroll
     for (int nt = 0; nt < K::NT; ++nt) {
-        split_tf32(ta[8 * nt], bh[nt][0], bl[nt][0]);
-        split_tf32(tb[8 * nt], bh[nt][1], bl[nt][1]);
+        split_tf32(ra[8 * nt + g], bh[nt][0], bl[nt][0]);
+        split_tf32(rb[8 * nt + g], bh[nt][1], bl[nt][1]);
     }
 #pragma unroll
     for (int mt = 0; mt < K::MT; ++mt) {
@@ -137,213 +200,269 @@ __device__ __forceinline__ void store_tile(const float (&acc)[cfg<L, M>::MT][cfg
         }
 }
 
-// One warp evaluates one work item: nonzeros [p0,p1) starting inside fiber f0.  MULTI: the item is a run
-// of whole small slices (positions it.pad .. it.row_end - 1 in crd_i); the warp streams through all of
-// them and stores each slice's tile to `out` when the slice-end flag (bit 30 of the index stream) comes
-// by.  Otherwise the item is a piece of one slice and the tile is left in acc for the caller.
 template <int L, int M>
-__device__ __forceinline__ void ttm3_warp_item(const sa_item &it, const int32_t *__restrict__ crd_j,
-                                               const int32_t *__restrict__ kflag, const float *__restrict__ vals,
+__device__ __forceinline__ void zero_tile(float (&acc)[cfg<L, M>::MT][cfg<L, M>::NT][4])
+{
+#pragma unroll
+    for (int mt = 0; mt < cfg<L, M>::MT; ++mt)
+#pragma unroll
+        for (int nt = 0; nt < cfg<L, M>::NT; ++nt)
+#pragma unroll
+            for (int x = 0; x < 4; ++x) acc[mt][nt][x] = 0.f;
+}
+
+// Where stream q of a unit runs: rounds, aligned start, and the clipped range [lo, hi) (see sa_unit3_streams).
+struct stream_range {
+    int rounds, base, lo, hi;
+};
+__device__ __forceinline__ stream_range stream_of(int p0, int p1, int q)
+{
+    const int base8 = p0 & ~7, span = p1 - base8;
+    const int slen = ((span + SA_STREAMS - 1) / SA_STREAMS + 7) & ~7;
+    stream_range r;
+    r.rounds = slen >> 3;
+    r.base = base8 + q * slen;
+    r.lo = max(p0, r.base);
+    r.hi = min(p1, r.base + slen);
+    return r;
+}
+
+// One warp evaluates the units [u0, u0 + nu) of its task.  `keep`: the (single) unit is a piece of a slice
+// whose tile the caller reduces over the CTA, so it is left in acc; otherwise every unit is a whole slice
+// and its tile is stored to `out` when the unit ends.
+template <int L, int M>
+__device__ __forceinline__ void ttm3_warp_task(const sa_unit3 *__restrict__ units, int u0, int nu,
+                                               const int32_t *__restrict__ crd_j, const int32_t *__restrict__ crd_k,
+                                               const float *__restrict__ vals, const uint32_t *__restrict__ endbits,
                                                const float *__restrict__ C, uint32_t ldc, const float *__restrict__ D,
-                                               uint32_t ldd, float *__restrict__ wsm,
-                                               float (&acc)[cfg<L, M>::MT][cfg<L, M>::NT][4], const bool multi,
-                                               const int32_t *__restrict__ crd_i, float *__restrict__ out)
+                                               uint32_t ldd, unsigned char *__restrict__ wsm,
+                                               float (&acc)[cfg<L, M>::MT][cfg<L, M>::NT][4], const bool keep,
+                                               float *__restrict__ out, const dbg_limits &lim)
 {
     using K = cfg<L, M>;
-    static_assert(K::NS == 3, "the register ring below is written for three stages");
+    constexpr int VEC = K::VEC, DEPTH = K::DEPTH;
     const int lane = threadIdx.x & 31;
-    const int m = lane & (M - 1);
-    const int t4 = lane & 3;
-    float *Tbuf = wsm + K::NS * K::STAGE;
-    float *vs = Tbuf + 16 * K::TS;                  // values of the batch being consumed
-#pragma unroll
-    for (int mt = 0; mt < K::MT; ++mt)
-#pragma unroll
-        for (int nt = 0; nt < K::NT; ++nt)
-#pragma unroll
-            for (int q = 0; q < 4; ++q) acc[mt][nt][q] = 0.f;
-    if (it.p0 >= it.p1) return;
-    const int p0 = it.p0, p1 = it.p1, f0 = it.f0, fmax = it.f1 - 1;
-    const int nb = (p1 - p0 + 31) >> 5;
-    // per-lane constants of the row gather
-    constexpr int LPR = M / 4;
-    const int gr = lane / LPR, gc = lane % LPR;
-    const uint32_t dst_lane = smem_u32(wsm) + uint32_t(gr * M + gc * 4) * 4u;
-    const char *src_lane = reinterpret_cast<const char *>(D + gc * 4);
-    const uint32_t row_bytes = ldd * 4u;
-    int pn = p0 + lane;                              // position this lane loads next
-    auto load_kv = [&](int &k, float &v) {
-        k = 0;
-        v = 0.f;
-        if (pn < p1) { k = kflag[pn]; v = vals[pn]; }
-        pn += 32;
+    const int q = lane >> 3, c = lane & 7;
+    const uint32_t s_base = smem_u32(wsm), s_kv = s_base + K::OFF_KV + q * K::SLOT, s_ring = s_base + K::OFF_RING;
+    float *ring = reinterpret_cast<float *>(wsm + K::OFF_RING);
+    // the index / value ring starts as zeros: a stream that has nothing to fetch in some round still
+    // turns the indices it finds there into (unused) row loads, which must stay inside D
+    for (int x = lane; x < DEPTH * K::NS * K::SLOT / 16; x += 32)
+        *reinterpret_cast<uint4 *>(wsm + K::OFF_KV + 16 * x) = make_uint4(0u, 0u, 0u, 0u);
+    __syncwarp();
+    // unit records are read straight from global memory, one unit ahead of their use
+    struct unit_head { int row, p0, p1; };
+    auto load_head = [&](int u) {
+        const int4 w = __ldg(reinterpret_cast<const int4 *>(units + u0 + u));   // out_row, dest, p0, p1
+        unit_head h;
+        h.row = w.x; h.p0 = w.z; h.p1 = w.w;
+        return h;
     };
-    // index/value registers of batches B .. B+6: the index of a batch is needed two rounds before its
-    // values (to request its rows), and a streaming load takes several rounds to arrive; row gathers
-    // of batches B+1, B+2 are in flight while B is consumed
-    int k0, k1, k2, k3, k4, k5, k6;
-    float v0, v1, v2, v3, v4, v5, v6;
-    load_kv(k0, v0);
-    load_kv(k1, v1);
-    load_kv(k2, v2);
-    load_kv(k3, v3);
-    load_kv(k4, v4);
-    load_kv(k5, v5);
-    load_kv(k6, v6);
-    stage_rows<M>(dst_lane, k0, src_lane, row_bytes, gr);
-    cp_async_commit();
-    if (1 < nb) stage_rows<M>(dst_lane + K::STAGE * 4, k1, src_lane, row_bytes, gr);
-    cp_async_commit();
-    int nclosed = 0, nflushed = 0;          // fibers closed / handed to the tensor cores so far
-    float cf[K::MT][4];                     // C values of the next flush
-    load_cfrag<L, M>(cf, C + uint32_t(crd_j[min(f0 + t4, fmax)]) * ldc, C + uint32_t(crd_j[min(f0 + t4 + 4, fmax)]) * ldc, lane);
-    float T = 0.f, U = 0.f;                 // two partial sums of the open fiber (shorter dependency chains)
-    int s_cur = 0, s_issue = 2;
-    int slice = it.pad;                     // MULTI: position of the slice being accumulated
-    // hand the n (<= 8) oldest closed fibers to the tensor cores and fetch the C values of the next group
-    auto flush_group = [&](int n) {
-        for (int x = n; x < 8; ++x) Tbuf[((nflushed + x) & 15) * K::TS + m] = 0.f;   // unused rows
-        __syncwarp();
-        ttm3_flush<L, M>(acc, Tbuf, nflushed, cf, lane);
-        __syncwarp();
-        nflushed += n;
-        load_cfrag<L, M>(cf, C + uint32_t(crd_j[min(f0 + nflushed + t4, fmax)]) * ldc,
-                         C + uint32_t(crd_j[min(f0 + nflushed + t4 + 4, fmax)]) * ldc, lane);
-    };
-    // T += v * d for one nonzero; `end` (warp-uniform) closes the fiber into the ring of temporaries
-#define SA_TTM3_STEP(v, d, end)                                   \
-    T = fmaf(v, d, T);                                            \
-    if (end) {                                                    \
-        Tbuf[(nclosed & 15) * K::TS + m] = T + U;                 \
-        T = 0.f;                                                  \
-        U = 0.f;                                                  \
-        ++nclosed;                                                \
-    }
-#pragma unroll 1
-    for (int b = 0; b < nb; ++b) {
-        if (b + 2 < nb) stage_rows<M>(dst_lane + s_issue * (K::STAGE * 4), k2, src_lane, row_bytes, gr);
+    auto load_sf = [&](int u) { return __ldg(&units[u0 + u].sf[q]); };
+
+    // ---- fetcher: copies the data of one round (of this or a later unit) into ring slot `slot`
+    int fu = 0, fr = 0;
+    const unit_head h0 = load_head(0);
+    unit_head fnext = load_head(nu > 1 ? 1 : 0);             // the unit the fetcher turns to next
+    stream_range fs = stream_of(h0.p0, h0.p1, q);
+    auto fetch_round = [&](int slot) {
+        if (fu < nu) {
+            const int pg = fs.base + 8 * fr;
+            if (pg < fs.hi && pg + 8 > fs.lo && SA_CHK(lim, pg >= 0 && pg + 8 <= lim.nnz + 8, 3, pg)) {
+                const uint32_t dst = s_kv + slot * (K::NS * K::SLOT);
+                if (c < 4) cp_async16_raw(dst + 16 * c, (c < 2 ? reinterpret_cast<const char *>(crd_k) : reinterpret_cast<const char *>(vals)) + 4 * int64_t(pg) + 16 * (c & 1));
+                else if (c == 4) cp_async4_raw(dst + 64, endbits + (pg >> 5));
+            }
+            if (++fr == fs.rounds) {
+                fr = 0;
+                if (++fu < nu) {
+                    fs = stream_of(fnext.p0, fnext.p1, q);
+                    if (fu + 1 < nu) fnext = load_head(fu + 1);
+                }
+            }
+        }
         cp_async_commit();
-        vs[lane] = v0;
-        cp_async_wait<2>();
+    };
+#pragma unroll
+    for (int r = 0; r < DEPTH - 1; ++r) fetch_round(r);
+
+    // ---- consumer state
+    int cu = 0, cr = 0;
+    stream_range cs = stream_of(h0.p0, h0.p1, q);
+    int crow = h0.row;                                  // output row of the unit being consumed
+    unit_head cnext = load_head(nu > 1 ? 1 : 0);        // the unit the consumer turns to next
+    int fnext_q = load_sf(nu > 1 ? 1 : 0);              // and the fiber its stream q starts in
+    int fq = load_sf(0);                                // next fiber this stream parks
+    if (!SA_CHK(lim, uint32_t(fq) <= lim.n_fibers, 4, fq)) fq = 0;
+    int jreg = __ldg(crd_j + fq + c);                   // C rows of the next eight fibers of the stream, one per lane
+    const char *dlane = reinterpret_cast<const char *>(D + c * VEC);
+    const uint32_t row_bytes = ldd * 4u;
+    cp_async_wait<DEPTH - 2>();
+    __syncwarp();
+    rowvec<VEC> buf[8];                                  // rows of the round about to be consumed
+    {
+        const uint4 ka = lds128(s_kv), kb = lds128(s_kv + 16);
+        const uint32_t k8[8] = {ka.x, ka.y, ka.z, ka.w, kb.x, kb.y, kb.z, kb.w};
+#pragma unroll
+        for (int s = 0; s < 8; ++s) buf[s].load(dlane + uint64_t(SA_CHK(lim, k8[s] < lim.d_rows, 5, k8[s]) ? k8[s] : 0u) * row_bytes);
+    }
+    float T[VEC];
+#pragma unroll
+    for (int x = 0; x < VEC; ++x) T[x] = 0.f;
+    int nclosed = 0, nflushed = 0, sc = 0;
+#ifdef SA_DEBUG_BOUNDS
+    int dbg_rounds = 0;
+#endif
+    while (cu < nu) {
+#ifdef SA_DEBUG_BOUNDS
+        if (!SA_CHK(lim, ++dbg_rounds <= (1 << 16), 9, cs.rounds)) break;    // a task has at most ~300 rounds
+#endif
+        fetch_round(sc == 0 ? DEPTH - 1 : sc - 1);
+        cp_async_wait<DEPTH - 2>();
         __syncwarp();
-        const float *st = wsm + s_cur * K::STAGE + m;
-        unsigned ends = __ballot_sync(SA_FULL_MASK, k0 < 0);
-        const unsigned sends = multi ? __ballot_sync(SA_FULL_MASK, (k0 & 0x40000000) != 0) : 0u;
-        const int rem = p1 - p0 - 32 * b;
-        if (rem <= 32) ends |= 1u << (rem - 1);         // the item's last nonzero closes its (possibly cut) fiber
-        const int nchunks = rem >= 32 ? 4 : (rem + 7) >> 3;
-#pragma unroll 1
-        for (int c = 0; c < nchunks; ++c) {
-            const unsigned e8 = (ends >> (8 * c)) & 0xffu;
-            const float *sc = st + 8 * c * M;
-            const float4 va = *reinterpret_cast<const float4 *>(vs + 8 * c);
-            const float4 vb = *reinterpret_cast<const float4 *>(vs + 8 * c + 4);
-            if (((sends >> (8 * c)) & 0xffu) != 0) {
-                // a slice ends inside this chunk: one nonzero at a time, the tile leaves at the slice end
-                const unsigned s8 = (sends >> (8 * c)) & 0xffu;
-                T += U;
-                U = 0.f;
-#pragma unroll 1
-                for (int u = 0; u < 8; ++u) {
-                    T = fmaf(vs[8 * c + u], sc[u * M], T);
-                    if (e8 & (1u << u)) {
-                        Tbuf[(nclosed & 15) * K::TS + m] = T;
-                        T = 0.f;
-                        ++nclosed;
-                        const bool slice_end = (s8 & (1u << u)) != 0;
-                        if (slice_end || nclosed - nflushed >= 8) flush_group(min(8, nclosed - nflushed));
-                        if (slice_end) {
-                            store_tile<L, M>(acc, out + int64_t(crd_i[slice]) * (L * M), lane);
-                            ++slice;
+        const int sn = sc == DEPTH - 1 ? 0 : sc + 1;
+        const uint32_t slot_c = s_kv + sc * (K::NS * K::SLOT), slot_n = s_kv + sn * (K::NS * K::SLOT);
+        const uint32_t fw = lds32(slot_c + 64);
+        // which of the eight positions pg .. pg + 7 belong to the stream, and which of them end a fiber
+        const int pg = cs.base + 8 * cr;
+        const int a = min(max(cs.lo - pg, 0), 8), b = min(max(cs.hi - pg, 0), 8);
+        const uint32_t vm = ((1u << b) - 1u) & ~((1u << a) - 1u);
+        uint32_t e8 = (fw >> (pg & 24)) & vm;
+        if (cs.hi > cs.lo && uint32_t(cs.hi - pg - 1) < 8u) e8 |= 1u << (cs.hi - pg - 1);   // the part's last nonzero closes its (possibly cut) fiber
+        // ring rows for the fibers this round parks: stream-major
+        const int cnt = __popc(e8);
+        int incl = cnt;
+        {
+            int o = __shfl_up_sync(SA_FULL_MASK, incl, 8);
+            if (lane >= 8) incl += o;
+            o = __shfl_up_sync(SA_FULL_MASK, incl, 16);
+            if (lane >= 16) incl += o;
+        }
+        const int total = __shfl_sync(SA_FULL_MASK, incl, 31);
+        int slot = nclosed + incl - cnt;
+        nclosed += total;
+        if (c < cnt) {
+            const uint32_t off = uint32_t(jreg) * ldc;
+            sts32(s_ring + (((slot + c) & (K::RING - 1)) * K::RS + M) * 4, off);
+            prefetch_l1(C + off);
+        }
+        fq += cnt;
+        const bool last = cr + 1 == cs.rounds;
+        if (last && cu + 1 < nu) fq = fnext_q;
+        if (!SA_CHK(lim, uint32_t(fq) <= lim.n_fibers, 6, fq)) fq = 0;
+        const int jnext = __ldg(crd_j + fq + c);
+        // Eight steps: consume the row requested one round ago, then request the row of the same step of
+        // the next round into the same registers.  MASKED: some stream of the warp is at a ragged end of
+        // its part; positions outside the part contribute nothing (their rows are not even read as numbers).
+        auto steps = [&](auto masked) {
+            constexpr bool MASKED = decltype(masked)::value;
 #pragma unroll
-                            for (int mt = 0; mt < K::MT; ++mt)
+            for (int h = 0; h < 2; ++h) {
+                const uint4 vv = lds128(slot_c + 32 + 16 * h);
+                const uint4 kk = lds128(slot_n + 16 * h);
+                const float v4[4] = {__uint_as_float(vv.x), __uint_as_float(vv.y), __uint_as_float(vv.z), __uint_as_float(vv.w)};
+                const uint32_t k4[4] = {kk.x, kk.y, kk.z, kk.w};
 #pragma unroll
-                                for (int nt = 0; nt < K::NT; ++nt)
+                for (int s4 = 0; s4 < 4; ++s4) {
+                    const int s = 4 * h + s4;
+                    if (!MASKED || ((vm >> s) & 1u)) {
 #pragma unroll
-                                    for (int q = 0; q < 4; ++q) acc[mt][nt][q] = 0.f;
-                        }
+                        for (int x = 0; x < VEC; ++x) T[x] = fmaf(v4[s4], buf[s].x[x], T[x]);
+                    }
+                    buf[s].load(dlane + uint64_t(SA_CHK(lim, k4[s4] < lim.d_rows, 7, k4[s4]) ? k4[s4] : 0u) * row_bytes);
+                    if (e8 & (1u << s)) {
+                        rowvec<VEC> tv;
+#pragma unroll
+                        for (int x = 0; x < VEC; ++x) { tv.x[x] = T[x]; T[x] = 0.f; }
+                        tv.store_shared(s_ring + ((slot & (K::RING - 1)) * K::RS + c * VEC) * 4);
+                        ++slot;
                     }
                 }
-                continue;
             }
-            if ((e8 & 0xfu) == 0) {
-                T = fmaf(va.x, sc[0], T);
-                U = fmaf(va.y, sc[M], U);
-                T = fmaf(va.z, sc[2 * M], T);
-                U = fmaf(va.w, sc[3 * M], U);
-            } else {
-                SA_TTM3_STEP(va.x, sc[0], e8 & 1u)
-                SA_TTM3_STEP(va.y, sc[M], e8 & 2u)
-                SA_TTM3_STEP(va.z, sc[2 * M], e8 & 4u)
-                SA_TTM3_STEP(va.w, sc[3 * M], e8 & 8u)
-            }
-            if ((e8 & 0xf0u) == 0) {
-                T = fmaf(vb.x, sc[4 * M], T);
-                U = fmaf(vb.y, sc[5 * M], U);
-                T = fmaf(vb.z, sc[6 * M], T);
-                U = fmaf(vb.w, sc[7 * M], U);
-            } else {
-                SA_TTM3_STEP(vb.x, sc[4 * M], e8 & 16u)
-                SA_TTM3_STEP(vb.y, sc[5 * M], e8 & 32u)
-                SA_TTM3_STEP(vb.z, sc[6 * M], e8 & 64u)
-                SA_TTM3_STEP(vb.w, sc[7 * M], e8 & 128u)
-            }
-            if (nclosed - nflushed >= 8) flush_group(8);
+        };
+        if (__any_sync(SA_FULL_MASK, vm != 0xffu)) steps(std::true_type{});
+        else steps(std::false_type{});
+        __syncwarp();
+        while (nclosed - nflushed >= 8) {
+            ttm3_flush<L, M>(acc, ring, nflushed, 8, C, lane, lim, ldc);
+            nflushed += 8;
         }
-        __syncwarp();                                   // stage s_cur and vs are free for the next round
-        k0 = k1; k1 = k2; k2 = k3; k3 = k4; k4 = k5; k5 = k6;
-        v0 = v1; v1 = v2; v2 = v3; v3 = v4; v4 = v5; v5 = v6;
-        load_kv(k6, v6);
-        s_issue = s_cur;
-        s_cur = s_cur == 2 ? 0 : s_cur + 1;
+        if (last) {
+            const int n = nclosed - nflushed;
+            if (n > 0) {
+                for (int x = n; x < 8; ++x) ring[((nflushed + x) & (K::RING - 1)) * K::RS + lane % M] = 0.f;
+                __syncwarp();
+                ttm3_flush<L, M>(acc, ring, nflushed, n, C, lane, lim, ldc);
+            }
+            nclosed = nflushed = 0;
+            if (!keep) {
+                if (SA_CHK(lim, uint32_t(crow) < lim.n_slices_dim, 8, crow)) store_tile<L, M>(acc, out + int64_t(crow) * (L * M), lane);
+                zero_tile<L, M>(acc);
+            }
+            ++cu;
+            cr = 0;
+            if (cu < nu) {
+                cs = stream_of(cnext.p0, cnext.p1, q);
+                crow = cnext.row;
+                SA_CHK(lim, cs.rounds >= 1, 10, cu);
+                if (cu + 1 < nu) {
+                    cnext = load_head(cu + 1);
+                    fnext_q = load_sf(cu + 1);
+                }
+            }
+        } else {
+            ++cr;
+        }
+        __syncwarp();
+        jreg = jnext;
+        sc = sn;
     }
-#undef SA_TTM3_STEP
     cp_async_wait<0>();
-    if (nclosed - nflushed > 0) flush_group(nclosed - nflushed);      // pieces of one slice: the open group
+    __syncwarp();
 }
 
 template <int L, int M>
-__global__ void __launch_bounds__(256, 2)
-ttm3_kernel(const sa_item *__restrict__ items, int64_t n_items, int n_group_ctas, const int32_t *__restrict__ crd_i,
-            const int32_t *__restrict__ crd_j, const int32_t *__restrict__ kflag, const float *__restrict__ vals, const float *__restrict__ C, uint32_t ldc,
-            const float *__restrict__ D, uint32_t ldd, float *__restrict__ out, float *__restrict__ partial)
+__global__ void __launch_bounds__(32 * SA_TTM3_WARPS, 3)
+ttm3_kernel(const sa_unit3 *__restrict__ units, const int32_t *__restrict__ task_start, int64_t n_tasks, int n_group_ctas,
+            const int32_t *__restrict__ crd_j, const int32_t *__restrict__ crd_k, const float *__restrict__ vals,
+            const uint32_t *__restrict__ endbits, const float *__restrict__ C, uint32_t ldc,
+            const float *__restrict__ D, uint32_t ldd, float *__restrict__ out, float *__restrict__ partial,
+            const dbg_limits lim)
 {
     using K = cfg<L, M>;
     constexpr int TILE = L * M;
-    extern __shared__ __align__(16) float smem[];
+    extern __shared__ __align__(16) unsigned char smem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int g = lane >> 2, t = lane & 3;
-    float *wsm = smem + warp * K::WARP_SMEM;
-    const int64_t idx = int64_t(blockIdx.x) * SA_WARPS_PER_CTA + warp;
+    unsigned char *wsm = smem + warp * K::WARP_BYTES;
+    const int64_t task = int64_t(blockIdx.x) * SA_TTM3_WARPS + warp;
     const bool group = int(blockIdx.x) < n_group_ctas;
     float acc[K::MT][K::NT][4];
-    sa_item it;
-    it.f0 = it.f1 = it.p0 = it.p1 = 0;
-    it.dest = -1;
-    it.out_row = 0;
-    it.pad = it.row_end = 0;
-    if (idx < n_items) it = items[idx];
-    if (idx < n_items || group)
-        ttm3_warp_item<L, M>(it, crd_j, kflag, vals, C, ldc, D, ldd, wsm, acc, !group, crd_i, out);
-    if (!group) return;                 // runs of small slices: every tile was stored at its slice end
-    // the CTA's eight warps hold partial tiles of the same slice: sum them in a fixed order
+    zero_tile<L, M>(acc);
+    int u0 = 0, u1 = 0;
+    if (task < n_tasks) { u0 = task_start[task]; u1 = task_start[task + 1]; }
+    if (u1 > u0) ttm3_warp_task<L, M>(units, u0, u1 - u0, crd_j, crd_k, vals, endbits, C, ldc, D, ldd, wsm, acc, group, out, lim);
+    if (!group) return;                 // whole small slices: every tile was stored when its unit ended
+    // the CTA's warps hold partial tiles of the same slice: sum them in a fixed order
+    float *wt = reinterpret_cast<float *>(wsm);
 #pragma unroll
     for (int mt = 0; mt < K::MT; ++mt)
 #pragma unroll
         for (int nt = 0; nt < K::NT; ++nt) {
             const int l = 16 * mt + g, mm = 8 * nt + 2 * t;
-            *reinterpret_cast<float2 *>(wsm + l * K::RS + mm) = make_float2(acc[mt][nt][0], acc[mt][nt][1]);
-            *reinterpret_cast<float2 *>(wsm + (l + 8) * K::RS + mm) = make_float2(acc[mt][nt][2], acc[mt][nt][3]);
+            *reinterpret_cast<float2 *>(wt + l * K::RS + mm) = make_float2(acc[mt][nt][0], acc[mt][nt][1]);
+            *reinterpret_cast<float2 *>(wt + (l + 8) * K::RS + mm) = make_float2(acc[mt][nt][2], acc[mt][nt][3]);
         }
     __syncthreads();
-    const sa_item lead = items[int64_t(blockIdx.x) * SA_WARPS_PER_CTA];
+    const sa_unit3 lead = units[task_start[int64_t(blockIdx.x) * SA_TTM3_WARPS]];   // warp 0 always has a unit
     float *dst = lead.dest >= 0 ? partial + int64_t(lead.dest) * TILE : out + int64_t(lead.out_row) * TILE;
-    for (int x = threadIdx.x * 4; x < TILE; x += 256 * 4) {
+    const float *all = reinterpret_cast<const float *>(smem);
+    for (int x = threadIdx.x * 4; x < TILE; x += 32 * SA_TTM3_WARPS * 4) {
         const int off = (x / M) * K::RS + (x % M);
-        float4 s = *reinterpret_cast<const float4 *>(smem + off);
+        float4 s = *reinterpret_cast<const float4 *>(all + off);
 #pragma unroll
-        for (int w = 1; w < SA_WARPS_PER_CTA; ++w) {
-            const float4 v = *reinterpret_cast<const float4 *>(smem + w * K::WARP_SMEM + off);
+        for (int w = 1; w < SA_TTM3_WARPS; ++w) {
+            const float4 v = *reinterpret_cast<const float4 *>(all + w * (K::WARP_BYTES / 4) + off);
             s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
         }
         if (lead.dest >= 0) *reinterpret_cast<float4 *>(dst + x) = s;
@@ -355,16 +474,21 @@ template <int L, int M>
 cudaError_t launch(const sa_tensor *t, const sa_dense *ops, float *out, float *partial, cudaStream_t stream)
 {
     const sa_worklist &wl = t->wl_main;
-    const int64_t n_items = int64_t(wl.items.size());
-    const int64_t n_warp_items = n_items - wl.n_group_ctas * SA_WARPS_PER_CTA;
-    const int64_t ctas = wl.n_group_ctas + (n_warp_items + SA_WARPS_PER_CTA - 1) / SA_WARPS_PER_CTA;
-    if (ctas == 0) return cudaSuccess;
-    constexpr size_t smem = size_t(SA_WARPS_PER_CTA) * cfg<L, M>::WARP_SMEM * sizeof(float);
+    const int64_t n_tasks = int64_t(wl.task_start.size()) - 1;
+    const int64_t ctas = (n_tasks + SA_TTM3_WARPS - 1) / SA_TTM3_WARPS;
+    if (ctas <= 0) return cudaSuccess;
+    constexpr size_t smem = size_t(SA_TTM3_WARPS) * cfg<L, M>::WARP_BYTES;
     auto kern = ttm3_kernel<L, M>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess)
         return cudaGetLastError();
-    kern<<<(unsigned)ctas, 256, smem, stream>>>(wl.d_items, n_items, int(wl.n_group_ctas), t->d_crd[0], t->d_crd[1], t->d_crd_endflag,
-                                               t->d_vals, ops[0].ptr, uint32_t(ops[0].ld), ops[1].ptr, uint32_t(ops[1].ld), out, partial);
+    dbg_limits lim;
+    lim.status = t->d_status;
+    lim.c_rows = uint32_t(ops[0].rows); lim.d_rows = uint32_t(ops[1].rows);
+    lim.n_fibers = uint32_t(t->count[1]); lim.n_slices_dim = uint32_t(t->dims[0]);
+    lim.nnz = t->nnz;
+    kern<<<(unsigned)ctas, 32 * SA_TTM3_WARPS, smem, stream>>>(wl.d_units3, wl.d_task_start, n_tasks, int(wl.n_group_ctas), t->d_crd[1], t->d_crd[2],
+                                               t->d_vals, t->d_endbits, ops[0].ptr, uint32_t(ops[0].ld), ops[1].ptr,
+                                               uint32_t(ops[1].ld), out, partial, lim);
     return cudaGetLastError();
 }
 
@@ -385,7 +509,7 @@ sa_status sa_launch_ttm3(const sa_tensor *t, const sa_dense *ops, float *out, vo
     // the kernel addresses factor rows with 32-bit byte offsets
     for (int i = 0; i < 2; ++i)
         if (ops[i].rows * ops[i].ld >= (int64_t(1) << 30)) return SA_E_UNSUPPORTED;
-    if (!t->d_crd_endflag) return SA_E_UNSUPPORTED;      // last dimension >= 2^30: no room for the flag bits
+    if (!t->d_endbits) return SA_E_UNSUPPORTED;
     float *partial = static_cast<float *>(ws);
     cudaError_t e;
     if (L == 16 && M == 16) e = launch<16, 16>(t, ops, out, partial, stream);

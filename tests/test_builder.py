@@ -91,17 +91,22 @@ def test_csf_worklist_partitions_every_nonzero_once(cfg):
     slice_pos = {int(c): n for n, c in enumerate(crd0)}
     covered = np.zeros(w.nnz, dtype=np.int32)
     slot_owner = {}
+    group_items = n_groups * 8
+    G = 4                                   # warps (tasks) per thread block of the order-3 kernel
+    if t.order == 3:
+        task_start, stream_f0 = sa.sa_tensor_tasks(t.handle)
+        group_items = int(task_start[n_groups * G])
+        item_group = np.searchsorted(task_start, np.arange(n_items), side="right") - 1
     for n, (row, row_end, f0, f1, p0, p1, dest, _) in enumerate(items):
         if p0 == p1:
-            assert n < n_groups * 8 and f0 == f1, "only padding items of a group may be empty"
+            assert t.order == 4 and n < n_groups * 8 and f0 == f1, "only padding items of an order-4 group may be empty"
             continue
         s = slice_pos[int(row)]
         fa, fb = _fiber_nnz_range(t, "csf", t.order, levels, f0, f1)
-        if t.order == 3 and n >= n_groups * 8:
-            # a run of whole small slices, named by position: [pad, row_end)
-            s0, s1 = int(items[n][7]), int(row_end)
-            assert s0 == s and s1 > s0 and (f0, f1) == (pos1[s0], pos1[s1]) and (fa, fb) == (p0, p1)
-            assert p1 - p0 <= 2048 or s1 == s0 + 1
+        if t.order == 3 and n >= group_items:
+            # a whole small slice
+            assert int(items[n][7]) == s and (f0, f1) == (pos1[s], pos1[s + 1]) and (fa, fb) == (p0, p1)
+            assert p1 - p0 <= 2048 and dest == -1
         else:
             assert pos1[s] <= f0 < f1 <= pos1[s + 1], "fibers stay inside the item's slice"
             assert fa <= p0 < p1 <= fb, "nonzero range lies inside the fiber range"
@@ -111,7 +116,10 @@ def test_csf_worklist_partitions_every_nonzero_once(cfg):
             else:
                 assert (fa, fb) == (p0, p1), "order-4 items hold whole (i,j) subtrees"
         covered[p0:p1] += 1
-        if n < n_groups * 8:
+        if t.order == 3 and n < group_items:
+            lead = items[task_start[(item_group[n] // G) * G]]
+            assert dest == lead[6] and row == lead[0], "a group works on one slice and one destination"
+        if t.order == 4 and n < n_groups * 8:
             lead = items[(n // 8) * 8]
             assert dest == lead[6] and row == lead[0], "a group works on one slice and one destination"
         if dest >= 0:
@@ -137,6 +145,27 @@ def test_csf_worklist_partitions_every_nonzero_once(cfg):
     # nonzero balance: no warp item is larger than the small-slice bound / the piece size
     sizes = items[:, 5] - items[:, 4]
     assert sizes.max() <= max(4096, int(np.ceil(w.nnz / 8)))
+    if t.order == 3:
+        # tasks: a partition of the item list; group tasks hold at most one item and warp 0 of a group has one;
+        # small-slice tasks hold at most 16 items and about 2048 nonzeros
+        assert task_start[0] == 0 and task_start[-1] == n_items and (np.diff(task_start) >= 0).all()
+        per_task = np.diff(task_start)
+        assert (per_task[:n_groups * G] <= 1).all() and (per_task[:n_groups * G:G] == 1).all()
+        assert (per_task[n_groups * G:] >= 1).all() and (per_task[n_groups * G:] <= 16).all()
+        for a, b in zip(task_start[n_groups * G:-1], task_start[n_groups * G + 1:]):
+            assert b - a == 1 or sizes[a:b].sum() <= 2048
+        # stream starts: part q of an item begins in fiber stream_f0[n, q]
+        pos2 = levels[2][0]
+        for n, (row, row_end, f0, f1, p0, p1, dest, _) in enumerate(items):
+            b8 = (p0 // 8) * 8
+            slen = -(-(-(-(p1 - b8) // 4)) // 8) * 8
+            for q in range(4):
+                lo, hi = max(p0, b8 + q * slen), min(p1, b8 + (q + 1) * slen)
+                f = int(stream_f0[n, q])
+                if lo < hi:
+                    assert f0 <= f < f1 and pos2[f] <= lo < pos2[f + 1]
+                else:
+                    assert f == f0
 
 
 @pytest.mark.parametrize("cfg,which", [(3, 0), (4, 1), (4, 0)])
