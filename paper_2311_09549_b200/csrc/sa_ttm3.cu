@@ -20,17 +20,13 @@
 
 namespace {
 
-__device__ __forceinline__ uint32_t tf32_rna(float x)
-{
-    uint32_t r;
-    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
-    return r;
-}
-
+// x = hi + lo with hi the upper 19 bits of x (a TF32 number) and lo = x - hi (exact in fp32), itself cut to
+// TF32.  hi.hi + hi.lo + lo.hi then misses the true product by about 2^-20 relative.  (cvt.rna.tf32 costs
+// several instructions per value on this target; plain masking is one.)
 __device__ __forceinline__ void split_tf32(float x, uint32_t &hi, uint32_t &lo)
 {
-    hi = tf32_rna(x);
-    lo = tf32_rna(x - __uint_as_float(hi));
+    hi = __float_as_uint(x) & 0xffffe000u;
+    lo = __float_as_uint(x - __uint_as_float(hi)) & 0xffffe000u;
 }
 
 __device__ __forceinline__ void mma_m16n8k8_tf32(float (&c)[4], const uint32_t (&a)[4], const uint32_t (&b)[2])
@@ -86,9 +82,29 @@ struct cfg {
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
-__device__ __forceinline__ void cp_async16_raw(uint32_t dst_smem, const void *src)
+// L2 policies: the factor matrices are re-read by every block and should stay in L2; the index / value
+// streams and the output pass through once.
+__device__ __forceinline__ uint64_t l2_policy_keep()
 {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst_smem), "l"(src) : "memory");
+    uint64_t p;
+    asm("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_stream()
+{
+    uint64_t p;
+    asm("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ void cp_async16_raw(uint32_t dst_smem, const void *src, uint64_t policy)
+{
+    asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;" ::"r"(dst_smem), "l"(src), "l"(policy) : "memory");
+}
+__device__ __forceinline__ float ldg_keep(const float *p, uint64_t policy)
+{
+    float v;
+    asm volatile("ld.global.nc.L2::cache_hint.f32 %0, [%1], %2;" : "=f"(v) : "l"(p), "l"(policy));
+    return v;
 }
 __device__ __forceinline__ void cp_async4_raw(uint32_t dst_smem, const void *src)
 {
@@ -115,10 +131,10 @@ struct rowvec;
 template <>
 struct rowvec<4> {
     float x[4];
-    __device__ __forceinline__ void load(const char *p)
+    __device__ __forceinline__ void load(const char *p, uint64_t policy)
     {
-        asm volatile("ld.global.nc.L1::no_allocate.v4.f32 {%0,%1,%2,%3}, [%4];"
-                     : "=f"(x[0]), "=f"(x[1]), "=f"(x[2]), "=f"(x[3]) : "l"(p));
+        asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.v4.f32 {%0,%1,%2,%3}, [%4], %5;"
+                     : "=f"(x[0]), "=f"(x[1]), "=f"(x[2]), "=f"(x[3]) : "l"(p), "l"(policy));
     }
     __device__ __forceinline__ void store_shared(uint32_t a) const
     {
@@ -128,9 +144,10 @@ struct rowvec<4> {
 template <>
 struct rowvec<2> {
     float x[2];
-    __device__ __forceinline__ void load(const char *p)
+    __device__ __forceinline__ void load(const char *p, uint64_t policy)
     {
-        asm volatile("ld.global.nc.L1::no_allocate.v2.f32 {%0,%1}, [%2];" : "=f"(x[0]), "=f"(x[1]) : "l"(p));
+        asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.v2.f32 {%0,%1}, [%2], %3;"
+                     : "=f"(x[0]), "=f"(x[1]) : "l"(p), "l"(policy));
     }
     __device__ __forceinline__ void store_shared(uint32_t a) const
     {
@@ -141,7 +158,8 @@ struct rowvec<2> {
 // acc += Cg^T . T for the ring rows (row0 + x) & (RING - 1), x = 0 .. 7, of which the first n are in use.
 template <int L, int M>
 __device__ __forceinline__ void ttm3_flush(float (&acc)[cfg<L, M>::MT][cfg<L, M>::NT][4], const float *__restrict__ ring,
-                                           int row0, int n, const float *__restrict__ C, int lane, const dbg_limits &lim, uint32_t ldc)
+                                           int row0, int n, const float *__restrict__ C, int lane, const dbg_limits &lim, uint32_t ldc,
+                                           uint64_t keep_policy)
 {
     using K = cfg<L, M>;
     const int g = lane >> 2, t = lane & 3;
@@ -158,10 +176,10 @@ __device__ __forceinline__ void ttm3_flush(float (&acc)[cfg<L, M>::MT][cfg<L, M>
         const float *cb = C + ob + g;
 #pragma unroll
         for (int mt = 0; mt < K::MT; ++mt) {
-            cf[mt][0] = va ? __ldg(ca + 16 * mt) : 0.f;
-            cf[mt][1] = va ? __ldg(ca + 16 * mt + 8) : 0.f;
-            cf[mt][2] = vb ? __ldg(cb + 16 * mt) : 0.f;
-            cf[mt][3] = vb ? __ldg(cb + 16 * mt + 8) : 0.f;
+            cf[mt][0] = va ? ldg_keep(ca + 16 * mt, keep_policy) : 0.f;
+            cf[mt][1] = va ? ldg_keep(ca + 16 * mt + 8, keep_policy) : 0.f;
+            cf[mt][2] = vb ? ldg_keep(cb + 16 * mt, keep_policy) : 0.f;
+            cf[mt][3] = vb ? ldg_keep(cb + 16 * mt + 8, keep_policy) : 0.f;
         }
     }
     uint32_t bh[K::NT][2], bl[K::NT][2];
@@ -243,6 +261,7 @@ __device__ __forceinline__ void ttm3_warp_task(const sa_unit3 *__restrict__ unit
     constexpr int VEC = K::VEC, DEPTH = K::DEPTH;
     const int lane = threadIdx.x & 31;
     const int q = lane >> 3, c = lane & 7;
+    const uint64_t pol_keep = l2_policy_keep(), pol_stream = l2_policy_stream();
     const uint32_t s_base = smem_u32(wsm), s_kv = s_base + K::OFF_KV + q * K::SLOT, s_ring = s_base + K::OFF_RING;
     float *ring = reinterpret_cast<float *>(wsm + K::OFF_RING);
     // the index / value ring starts as zeros: a stream that has nothing to fetch in some round still
@@ -270,7 +289,7 @@ __device__ __forceinline__ void ttm3_warp_task(const sa_unit3 *__restrict__ unit
             const int pg = fs.base + 8 * fr;
             if (pg < fs.hi && pg + 8 > fs.lo && SA_CHK(lim, pg >= 0 && pg + 8 <= lim.nnz + 8, 3, pg)) {
                 const uint32_t dst = s_kv + slot * (K::NS * K::SLOT);
-                if (c < 4) cp_async16_raw(dst + 16 * c, (c < 2 ? reinterpret_cast<const char *>(crd_k) : reinterpret_cast<const char *>(vals)) + 4 * int64_t(pg) + 16 * (c & 1));
+                if (c < 4) cp_async16_raw(dst + 16 * c, (c < 2 ? reinterpret_cast<const char *>(crd_k) : reinterpret_cast<const char *>(vals)) + 4 * int64_t(pg) + 16 * (c & 1), pol_stream);
                 else if (c == 4) cp_async4_raw(dst + 64, endbits + (pg >> 5));
             }
             if (++fr == fs.rounds) {
@@ -304,7 +323,7 @@ __device__ __forceinline__ void ttm3_warp_task(const sa_unit3 *__restrict__ unit
         const uint4 ka = lds128(s_kv), kb = lds128(s_kv + 16);
         const uint32_t k8[8] = {ka.x, ka.y, ka.z, ka.w, kb.x, kb.y, kb.z, kb.w};
 #pragma unroll
-        for (int s = 0; s < 8; ++s) buf[s].load(dlane + uint64_t(SA_CHK(lim, k8[s] < lim.d_rows, 5, k8[s]) ? k8[s] : 0u) * row_bytes);
+        for (int s = 0; s < 8; ++s) buf[s].load(dlane + uint64_t(SA_CHK(lim, k8[s] < lim.d_rows, 5, k8[s]) ? k8[s] : 0u) * row_bytes, pol_keep);
     }
     float T[VEC];
 #pragma unroll
@@ -314,8 +333,11 @@ __device__ __forceinline__ void ttm3_warp_task(const sa_unit3 *__restrict__ unit
     int dbg_rounds = 0;
 #endif
     while (cu < nu) {
+      const int rounds = cs.rounds;
+#pragma unroll 1
+      for (cr = 0; cr < rounds; ++cr) {
 #ifdef SA_DEBUG_BOUNDS
-        if (!SA_CHK(lim, ++dbg_rounds <= (1 << 16), 9, cs.rounds)) break;    // a task has at most ~300 rounds
+        if (!SA_CHK(lim, ++dbg_rounds <= (1 << 16), 9, cs.rounds)) return;    // a task has at most ~300 rounds
 #endif
         fetch_round(sc == 0 ? DEPTH - 1 : sc - 1);
         cp_async_wait<DEPTH - 2>();
@@ -347,7 +369,7 @@ __device__ __forceinline__ void ttm3_warp_task(const sa_unit3 *__restrict__ unit
             prefetch_l1(C + off);
         }
         fq += cnt;
-        const bool last = cr + 1 == cs.rounds;
+        const bool last = cr + 1 == rounds;
         if (last && cu + 1 < nu) fq = fnext_q;
         if (!SA_CHK(lim, uint32_t(fq) <= lim.n_fibers, 6, fq)) fq = 0;
         const int jnext = __ldg(crd_j + fq + c);
@@ -369,7 +391,7 @@ __device__ __forceinline__ void ttm3_warp_task(const sa_unit3 *__restrict__ unit
 #pragma unroll
                         for (int x = 0; x < VEC; ++x) T[x] = fmaf(v4[s4], buf[s].x[x], T[x]);
                     }
-                    buf[s].load(dlane + uint64_t(SA_CHK(lim, k4[s4] < lim.d_rows, 7, k4[s4]) ? k4[s4] : 0u) * row_bytes);
+                    buf[s].load(dlane + uint64_t(SA_CHK(lim, k4[s4] < lim.d_rows, 7, k4[s4]) ? k4[s4] : 0u) * row_bytes, pol_keep);
                     if (e8 & (1u << s)) {
                         rowvec<VEC> tv;
 #pragma unroll
@@ -384,38 +406,38 @@ __device__ __forceinline__ void ttm3_warp_task(const sa_unit3 *__restrict__ unit
         else steps(std::false_type{});
         __syncwarp();
         while (nclosed - nflushed >= 8) {
-            ttm3_flush<L, M>(acc, ring, nflushed, 8, C, lane, lim, ldc);
+            ttm3_flush<L, M>(acc, ring, nflushed, 8, C, lane, lim, ldc, pol_keep);
             nflushed += 8;
-        }
-        if (last) {
-            const int n = nclosed - nflushed;
-            if (n > 0) {
-                for (int x = n; x < 8; ++x) ring[((nflushed + x) & (K::RING - 1)) * K::RS + lane % M] = 0.f;
-                __syncwarp();
-                ttm3_flush<L, M>(acc, ring, nflushed, n, C, lane, lim, ldc);
-            }
-            nclosed = nflushed = 0;
-            if (!keep) {
-                if (SA_CHK(lim, uint32_t(crow) < lim.n_slices_dim, 8, crow)) store_tile<L, M>(acc, out + int64_t(crow) * (L * M), lane);
-                zero_tile<L, M>(acc);
-            }
-            ++cu;
-            cr = 0;
-            if (cu < nu) {
-                cs = stream_of(cnext.p0, cnext.p1, q);
-                crow = cnext.row;
-                SA_CHK(lim, cs.rounds >= 1, 10, cu);
-                if (cu + 1 < nu) {
-                    cnext = load_head(cu + 1);
-                    fnext_q = load_sf(cu + 1);
-                }
-            }
-        } else {
-            ++cr;
         }
         __syncwarp();
         jreg = jnext;
         sc = sn;
+      }
+      // the unit ends: the open group of parked rows, the tile, the next unit
+      {
+        const int n = nclosed - nflushed;
+        if (n > 0) {
+            for (int x = n; x < 8; ++x) ring[((nflushed + x) & (K::RING - 1)) * K::RS + lane % M] = 0.f;
+            __syncwarp();
+            ttm3_flush<L, M>(acc, ring, nflushed, n, C, lane, lim, ldc, pol_keep);
+            __syncwarp();
+        }
+        nclosed = nflushed = 0;
+        if (!keep) {
+            if (SA_CHK(lim, uint32_t(crow) < lim.n_slices_dim, 8, crow)) store_tile<L, M>(acc, out + int64_t(crow) * (L * M), lane);
+            zero_tile<L, M>(acc);
+        }
+        ++cu;
+        if (cu < nu) {
+            cs = stream_of(cnext.p0, cnext.p1, q);
+            crow = cnext.row;
+            SA_CHK(lim, cs.rounds >= 1, 10, cu);
+            if (cu + 1 < nu) {
+                cnext = load_head(cu + 1);
+                fnext_q = load_sf(cu + 1);
+            }
+        }
+      }
     }
     cp_async_wait<0>();
     __syncwarp();
