@@ -64,6 +64,8 @@ __device__ __forceinline__ bool dbg_ok(const dbg_limits &lim, bool ok, int code,
 #define SA_CHK(lim, cond, code, value) true
 #endif
 
+constexpr int SA_TTM3_MINCTAS = 4;   // thread blocks per SM the register budget is set for (16 warps)
+
 template <int L, int M>
 struct cfg {
     static constexpr int MT = L / 16;            // m16 tiles over l
@@ -82,29 +84,9 @@ struct cfg {
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
-// L2 policies: the factor matrices are re-read by every block and should stay in L2; the index / value
-// streams and the output pass through once.
-__device__ __forceinline__ uint64_t l2_policy_keep()
+__device__ __forceinline__ void cp_async16_raw(uint32_t dst_smem, const void *src)
 {
-    uint64_t p;
-    asm("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
-    return p;
-}
-__device__ __forceinline__ uint64_t l2_policy_stream()
-{
-    uint64_t p;
-    asm("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
-    return p;
-}
-__device__ __forceinline__ void cp_async16_raw(uint32_t dst_smem, const void *src, uint64_t policy)
-{
-    asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;" ::"r"(dst_smem), "l"(src), "l"(policy) : "memory");
-}
-__device__ __forceinline__ float ldg_keep(const float *p, uint64_t policy)
-{
-    float v;
-    asm volatile("ld.global.nc.L2::cache_hint.f32 %0, [%1], %2;" : "=f"(v) : "l"(p), "l"(policy));
-    return v;
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst_smem), "l"(src) : "memory");
 }
 __device__ __forceinline__ void cp_async4_raw(uint32_t dst_smem, const void *src)
 {
@@ -125,16 +107,16 @@ __device__ __forceinline__ uint4 lds128(uint32_t a)
 __device__ __forceinline__ void sts32(uint32_t a, uint32_t v) { asm volatile("st.shared.u32 [%0], %1;" ::"r"(a), "r"(v) : "memory"); }
 __device__ __forceinline__ void prefetch_l1(const void *p) { asm volatile("prefetch.global.L1 [%0];" ::"l"(p)); }
 
-// A lane's piece of a factor row: VEC = 4 or 2 consecutive floats, read once and not kept in L1.
+// A lane's piece of a factor row: VEC = 4 or 2 consecutive floats.  Plain read-only loads: with the
+// L1::no_allocate qualifier the rows also lost their place in L2 (hit rate 57 % instead of 87 %).
 template <int VEC>
 struct rowvec;
 template <>
 struct rowvec<4> {
     float x[4];
-    __device__ __forceinline__ void load(const char *p, uint64_t policy)
+    __device__ __forceinline__ void load(const char *p)
     {
-        asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.v4.f32 {%0,%1,%2,%3}, [%4], %5;"
-                     : "=f"(x[0]), "=f"(x[1]), "=f"(x[2]), "=f"(x[3]) : "l"(p), "l"(policy));
+        asm volatile("ld.global.nc.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(x[0]), "=f"(x[1]), "=f"(x[2]), "=f"(x[3]) : "l"(p));
     }
     __device__ __forceinline__ void store_shared(uint32_t a) const
     {
@@ -144,10 +126,9 @@ struct rowvec<4> {
 template <>
 struct rowvec<2> {
     float x[2];
-    __device__ __forceinline__ void load(const char *p, uint64_t policy)
+    __device__ __forceinline__ void load(const char *p)
     {
-        asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.v2.f32 {%0,%1}, [%2], %3;"
-                     : "=f"(x[0]), "=f"(x[1]) : "l"(p), "l"(policy));
+        asm volatile("ld.global.nc.v2.f32 {%0,%1}, [%2];" : "=f"(x[0]), "=f"(x[1]) : "l"(p));
     }
     __device__ __forceinline__ void store_shared(uint32_t a) const
     {
@@ -158,8 +139,7 @@ struct rowvec<2> {
 // acc += Cg^T . T for the ring rows (row0 + x) & (RING - 1), x = 0 .. 7, of which the first n are in use.
 template <int L, int M>
 __device__ __forceinline__ void ttm3_flush(float (&acc)[cfg<L, M>::MT][cfg<L, M>::NT][4], const float *__restrict__ ring,
-                                           int row0, int n, const float *__restrict__ C, int lane, const dbg_limits &lim, uint32_t ldc,
-                                           uint64_t keep_policy)
+                                           int row0, int n, const float *__restrict__ C, int lane, const dbg_limits &lim, uint32_t ldc)
 {
     using K = cfg<L, M>;
     const int g = lane >> 2, t = lane & 3;
@@ -176,10 +156,10 @@ __device__ __forceinline__ void ttm3_flush(float (&acc)[cfg<L, M>::MT][cfg<L, M>
         const float *cb = C + ob + g;
 #pragma unroll
         for (int mt = 0; mt < K::MT; ++mt) {
-            cf[mt][0] = va ? ldg_keep(ca + 16 * mt, keep_policy) : 0.f;
-            cf[mt][1] = va ? ldg_keep(ca + 16 * mt + 8, keep_policy) : 0.f;
-            cf[mt][2] = vb ? ldg_keep(cb + 16 * mt, keep_policy) : 0.f;
-            cf[mt][3] = vb ? ldg_keep(cb + 16 * mt + 8, keep_policy) : 0.f;
+            cf[mt][0] = va ? __ldg(ca + 16 * mt) : 0.f;
+            cf[mt][1] = va ? __ldg(ca + 16 * mt + 8) : 0.f;
+            cf[mt][2] = vb ? __ldg(cb + 16 * mt) : 0.f;
+            cf[mt][3] = vb ? __ldg(cb + 16 * mt + 8) : 0.f;
         }
     }
     uint32_t bh[K::NT][2], bl[K::NT][2];
@@ -261,7 +241,6 @@ __device__ __forceinline__ void ttm3_warp_task(const sa_unit3 *__restrict__ unit
     constexpr int VEC = K::VEC, DEPTH = K::DEPTH;
     const int lane = threadIdx.x & 31;
     const int q = lane >> 3, c = lane & 7;
-    const uint64_t pol_keep = l2_policy_keep(), pol_stream = l2_policy_stream();
     const uint32_t s_base = smem_u32(wsm), s_kv = s_base + K::OFF_KV + q * K::SLOT, s_ring = s_base + K::OFF_RING;
     float *ring = reinterpret_cast<float *>(wsm + K::OFF_RING);
     // the index / value ring starts as zeros: a stream that has nothing to fetch in some round still
@@ -289,7 +268,7 @@ __device__ __forceinline__ void ttm3_warp_task(const sa_unit3 *__restrict__ unit
             const int pg = fs.base + 8 * fr;
             if (pg < fs.hi && pg + 8 > fs.lo && SA_CHK(lim, pg >= 0 && pg + 8 <= lim.nnz + 8, 3, pg)) {
                 const uint32_t dst = s_kv + slot * (K::NS * K::SLOT);
-                if (c < 4) cp_async16_raw(dst + 16 * c, (c < 2 ? reinterpret_cast<const char *>(crd_k) : reinterpret_cast<const char *>(vals)) + 4 * int64_t(pg) + 16 * (c & 1), pol_stream);
+                if (c < 4) cp_async16_raw(dst + 16 * c, (c < 2 ? reinterpret_cast<const char *>(crd_k) : reinterpret_cast<const char *>(vals)) + 4 * int64_t(pg) + 16 * (c & 1));
                 else if (c == 4) cp_async4_raw(dst + 64, endbits + (pg >> 5));
             }
             if (++fr == fs.rounds) {
@@ -323,7 +302,7 @@ __device__ __forceinline__ void ttm3_warp_task(const sa_unit3 *__restrict__ unit
         const uint4 ka = lds128(s_kv), kb = lds128(s_kv + 16);
         const uint32_t k8[8] = {ka.x, ka.y, ka.z, ka.w, kb.x, kb.y, kb.z, kb.w};
 #pragma unroll
-        for (int s = 0; s < 8; ++s) buf[s].load(dlane + uint64_t(SA_CHK(lim, k8[s] < lim.d_rows, 5, k8[s]) ? k8[s] : 0u) * row_bytes, pol_keep);
+        for (int s = 0; s < 8; ++s) buf[s].load(dlane + uint64_t(SA_CHK(lim, k8[s] < lim.d_rows, 5, k8[s]) ? k8[s] : 0u) * row_bytes);
     }
     float T[VEC];
 #pragma unroll
@@ -391,7 +370,7 @@ __device__ __forceinline__ void ttm3_warp_task(const sa_unit3 *__restrict__ unit
 #pragma unroll
                         for (int x = 0; x < VEC; ++x) T[x] = fmaf(v4[s4], buf[s].x[x], T[x]);
                     }
-                    buf[s].load(dlane + uint64_t(SA_CHK(lim, k4[s4] < lim.d_rows, 7, k4[s4]) ? k4[s4] : 0u) * row_bytes, pol_keep);
+                    buf[s].load(dlane + uint64_t(SA_CHK(lim, k4[s4] < lim.d_rows, 7, k4[s4]) ? k4[s4] : 0u) * row_bytes);
                     if (e8 & (1u << s)) {
                         rowvec<VEC> tv;
 #pragma unroll
@@ -406,7 +385,7 @@ __device__ __forceinline__ void ttm3_warp_task(const sa_unit3 *__restrict__ unit
         else steps(std::false_type{});
         __syncwarp();
         while (nclosed - nflushed >= 8) {
-            ttm3_flush<L, M>(acc, ring, nflushed, 8, C, lane, lim, ldc, pol_keep);
+            ttm3_flush<L, M>(acc, ring, nflushed, 8, C, lane, lim, ldc);
             nflushed += 8;
         }
         __syncwarp();
@@ -419,7 +398,7 @@ __device__ __forceinline__ void ttm3_warp_task(const sa_unit3 *__restrict__ unit
         if (n > 0) {
             for (int x = n; x < 8; ++x) ring[((nflushed + x) & (K::RING - 1)) * K::RS + lane % M] = 0.f;
             __syncwarp();
-            ttm3_flush<L, M>(acc, ring, nflushed, n, C, lane, lim, ldc, pol_keep);
+            ttm3_flush<L, M>(acc, ring, nflushed, n, C, lane, lim, ldc);
             __syncwarp();
         }
         nclosed = nflushed = 0;
@@ -444,7 +423,7 @@ __device__ __forceinline__ void ttm3_warp_task(const sa_unit3 *__restrict__ unit
 }
 
 template <int L, int M>
-__global__ void __launch_bounds__(32 * SA_TTM3_WARPS, 3)
+__global__ void __launch_bounds__(32 * SA_TTM3_WARPS, SA_TTM3_MINCTAS)
 ttm3_kernel(const sa_unit3 *__restrict__ units, const int32_t *__restrict__ task_start, int64_t n_tasks, int n_group_ctas,
             const int32_t *__restrict__ crd_j, const int32_t *__restrict__ crd_k, const float *__restrict__ vals,
             const uint32_t *__restrict__ endbits, const float *__restrict__ C, uint32_t ldc,
