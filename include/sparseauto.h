@@ -54,7 +54,8 @@ typedef enum {
     /* kernel 6 <SpTTM,TTM>:  A(i,l,m) = sum_{j,k} B(i,j,k) C(j,l) D(k,m); ops = {C, D}          */
     SA_EXPR_SPTTM_TTM3 = 1,
     /* order-4 analogue:      A(i,l,m,n) = sum_{j,k,o} B(i,j,k,o) C(j,l) D(k,m) E(o,n);
-     * ops = {C, D, E}; scheduled with the two-level nesting of kernel 5's second schedule      */
+     * ops = {C, D, E}; the two-level nesting of kernel 5's second schedule, evaluated in two
+     * passes with the 16 x 16 temporaries T2(m,n) of the (i,j) subtrees in the workspace       */
     SA_EXPR_SPTTM_TTM4 = 2,
     /* kernel 1 <SDDMM,SpMM>: A(i,l) = sum_j B(i,j) (sum_k C(i,k) D(j,k)) E(j,l); ops = {C,D,E}  */
     SA_EXPR_SDDMM_SPMM = 3,
@@ -135,18 +136,21 @@ sa_status sa_tensor_info(const sa_tensor *t, int64_t *nnz, int64_t *level_counts
 sa_status sa_tensor_export(const sa_tensor *t, int level, int64_t *pos, int32_t *crd, float *vals);
 
 /*
- * Copy a load-balancing work list to HOST arrays (which: 0 = main list, 1 = the CSR tensor's
- * second list used by SA_EXPR_SPMM_GEMM).  These are the slice / fiber / nonzero partition arrays:
+ * Copy a load-balancing work list to HOST arrays (which: 0 = main list, 1 = second list: a CSR
+ * tensor's list for SA_EXPR_SPMM_GEMM, an order-4 tensor's list for the second pass of
+ * SA_EXPR_SPTTM_TTM4).  These are the slice / fiber / nonzero partition arrays:
  *   counts [4]: number of items, number of leading groups that one thread block reduces into a
  *               single tile (8 items each; order-3 tensors: 4 tasks each, see sa_tensor_tasks),
  *               number of fix-up entries, number of partial-tile slots
  *   items  [n_items * 8] int32 per item: out_row, row_end, f0, f1, p0, p1, dest, half --
  *               fibers [f0,f1) (CSF) clipped to nonzeros [p0,p1) of slice out_row, or rows
  *               [out_row,row_end) / nonzeros [p0,p1) of a long row (CSR); dest = partial slot or -1;
- *               half = 0 / 1 for order-4 tensors, whose items are listed once per half of the
- *               last dense index.  Order-3 tensors use the last field for the position of the
- *               item's slice in the level-0 crd array; their items are grouped into tasks, see
- *               sa_tensor_tasks
+ *               the last field is the position of the item's slice in the level-0 crd array.  The
+ *               main list of a CSF tensor is grouped into tasks, see sa_tensor_tasks.  For an
+ *               order-4 tensor the "slices" of the main list are the (i,j) subtrees: out_row is the
+ *               index of the level-1 fiber, [f0,f1) are level-2 nodes; its second list has one item
+ *               per (piece of a slice, quarter of the 256 columns (m,n)): level-1 fibers [f0,f1) of
+ *               slice out_row, last field = quarter 0..3
  *   fix    [n_fix * 4] int32 per entry: out_row, slot0, count, 0 -- out[out_row] = sum of `count`
  *               partial tiles from slot0 (count 0: the slice / row is empty and is zero-filled)
  * NULL outputs are skipped.
@@ -154,7 +158,7 @@ sa_status sa_tensor_export(const sa_tensor *t, int level, int64_t *pos, int32_t 
 sa_status sa_tensor_worklist(const sa_tensor *t, int which, int64_t *counts, int32_t *items, int32_t *fix);
 
 /*
- * Order-3 CSF tensors: how the items of the main work list are handed to warps (the warp-level
+ * CSF tensors: how the items of the main work list are handed to warps (the warp-level
  * partition arrays of the fiber stage).
  *   n_tasks     number of tasks; warp w of the launch evaluates task w
  *   task_start  HOST [n_tasks + 1]: task w holds the items [task_start[w], task_start[w + 1]).  The first
@@ -166,7 +170,7 @@ sa_status sa_tensor_worklist(const sa_tensor *t, int which, int64_t *counts, int
  *               and s = ceil((p1 - b) / 4) rounded up to a multiple of 8, part q is
  *               [b + q s, b + (q + 1) s) clipped to [p0, p1); stream_f0[4 n + q] is the level-1 fiber
  *               that holds the first nonzero of part q of item n (f0 of the item if the part is empty).
- * NULL outputs are skipped.  Errors: SA_E_ARG, SA_E_FORMAT (not an order-3 CSF tensor).
+ * NULL outputs are skipped.  Errors: SA_E_ARG, SA_E_FORMAT (not a CSF tensor).
  */
 sa_status sa_tensor_tasks(const sa_tensor *t, int64_t *n_tasks, int32_t *task_start, int32_t *stream_f0);
 

@@ -225,23 +225,15 @@ sa_status sa_tensor_create(int order, const int64_t *dims, int64_t nnz, const in
             if (s == SA_OK) s = upload(t, t->crd[l].data(), t->crd[l].size(), &t->d_crd[l]);
         }
         if (s == SA_OK) s = upload(t, t->vals.data(), t->vals.size(), &t->d_vals);
-        if (s == SA_OK && fmt == SA_FMT_CSF && order == 3) {
-            // one bit per nonzero: set on the last nonzero of every (i,j) fiber
+        if (s == SA_OK && fmt == SA_FMT_CSF) {
+            // one bit per nonzero: set on the last nonzero of every last-level fiber
+            const int last = order - 1;
             std::vector<uint32_t> bits(size_t(nnz / 32 + 1), 0u);
-            for (int64_t f = 0; f < t->count[1]; ++f) {
-                const int64_t p = t->pos[2][size_t(f) + 1] - 1;
+            for (int64_t f = 0; f < t->count[last - 1]; ++f) {
+                const int64_t p = t->pos[last][size_t(f) + 1] - 1;
                 bits[size_t(p >> 5)] |= 1u << (p & 31);
             }
             s = upload(t, bits.data(), bits.size(), &t->d_endbits);
-        }
-        if (s == SA_OK && fmt == SA_FMT_CSF && order == 4 && t->dims[3] < (int64_t(1) << 30)) {
-            // bit 31: last nonzero of its (i,j,k) fiber; bit 30: last nonzero of its (i,j) fiber
-            std::vector<int32_t> flagged(t->crd[3]);
-            for (int64_t g = 0; g < t->count[2]; ++g)
-                flagged[size_t(t->pos[3][size_t(g) + 1] - 1)] |= int32_t(0x80000000u);
-            for (int64_t f = 0; f < t->count[1]; ++f)
-                flagged[size_t(t->pos[3][size_t(t->pos[2][size_t(f) + 1])] - 1)] |= int32_t(0x40000000);
-            s = upload(t, flagged.data(), flagged.size(), &t->d_crd_endflag);
         }
         const int32_t zeros[4] = {0, 0, 0, 0};
         if (s == SA_OK) s = upload(t, zeros, 4, &t->d_status);
@@ -295,7 +287,7 @@ sa_status sa_tensor_worklist(const sa_tensor *t, int which, int64_t *counts, int
 sa_status sa_tensor_tasks(const sa_tensor *t, int64_t *n_tasks, int32_t *task_start, int32_t *stream_f0)
 {
     if (!t) return SA_E_ARG;
-    if (t->fmt != SA_FMT_CSF || t->order != 3) return SA_E_FORMAT;
+    if (t->fmt != SA_FMT_CSF) return SA_E_FORMAT;
     const sa_worklist &wl = t->wl_main;
     if (n_tasks) *n_tasks = int64_t(wl.task_start.size()) - 1;
     if (task_start) std::memcpy(task_start, wl.task_start.data(), wl.task_start.size() * sizeof(int32_t));

@@ -191,18 +191,21 @@ void append_empty_slices(sa_tensor *t, sa_worklist &wl)
 // Smaller slices are one unit each; a warp evaluates a task of up to MAX_UNITS such units, about
 // SMALL_MAX nonzeros in total.  Inside a unit the warp's SA_STREAMS lane groups stream the parts given by
 // sa_unit3_streams; stream_f0 holds the fiber in which each part starts.
-void build_ttm3(sa_tensor *t, sa_worklist &wl)
+// `n_slices` slices; slice s is output row row_of(s), owns the fibers [pos1[s], pos1[s + 1]) whose nonzeros are
+// [pos2[f], pos2[f + 1]).  (Order 3: the slices of the tensor.  Order 4: the (i,j) subtrees, whose "fibers" are
+// the (i,j,k) fibers; output row = index of the (i,j) fiber.)
+template <typename RowOf>
+void build_ttm3_lists(sa_worklist &wl, int64_t n_slices, RowOf row_of, const std::vector<int64_t> &pos1,
+                      const std::vector<int64_t> &pos2)
 {
     constexpr int64_t SMALL_MAX = 2048, MIN_CHUNK = 8192, MAX_PARTS = 192, MAX_UNITS = 16;
-    const auto &pos1 = t->pos[1];
-    const auto &pos2 = t->pos[2];
     std::vector<sa_item> small;
     std::vector<group_rec> groups;
-    for (int64_t s = 0; s < t->count[0]; ++s) {
+    for (int64_t s = 0; s < n_slices; ++s) {
         const int64_t fa = pos1[size_t(s)], fb = pos1[size_t(s) + 1];
         const int64_t pa = pos2[size_t(fa)], pb = pos2[size_t(fb)];
         const int64_t n = pb - pa;
-        const int32_t row = t->crd[0][size_t(s)];
+        const int32_t row = row_of(s);
         if (n <= SMALL_MAX) {
             sa_item it = empty_item();
             it.out_row = row; it.row_end = row + 1; it.pad = int32_t(s);
@@ -271,80 +274,52 @@ void build_ttm3(sa_tensor *t, sa_worklist &wl)
             wl.stream_f0[u * SA_STREAMS + size_t(q)] = int32_t(f);
         }
     }
+}
+
+void build_ttm3(sa_tensor *t, sa_worklist &wl)
+{
+    build_ttm3_lists(wl, t->count[0], [&](int64_t s) { return t->crd[0][size_t(s)]; }, t->pos[1], t->pos[2]);
     append_empty_slices(t, wl);
 }
 
-// Order-4 CSF: warp items are ranges of whole level-1 fibers (i,j) of one slice.
-void build_ttm4(sa_tensor *t, sa_worklist &wl)
+
+// Order-4 CSF.  The chain is evaluated in two passes (see sa_ttm4.cu).  Pass 1 runs the order-3 kernel with
+// the (i,j) subtrees as slices: `wl` gets the same lists as an order-3 tensor whose slices are the level-1
+// fibers (output row = fiber index).  Pass 2 contracts the per-fiber temporaries of each slice with rows of
+// C: `wl2` holds one item per (piece of a slice, quarter of the 256 temporaries' columns); a slice with more
+// than CHUNK_F fibers is cut into pieces whose partial tiles the fix-up kernel sums.
+void build_ttm4(sa_tensor *t, sa_worklist &wl, sa_worklist &wl2)
 {
-    constexpr int64_t SMALL_MAX = 4096, MIN_CHUNK = 32768, MAX_PARTS = 160;
+    build_ttm3_lists(wl, t->count[1], [](int64_t f) { return int32_t(f); }, t->pos[2], t->pos[3]);
+    constexpr int64_t CHUNK_F = 512;
     const auto &pos1 = t->pos[1];
-    const auto &pos2 = t->pos[2];
-    const auto &pos3 = t->pos[3];
-    auto nz_of_fiber = [&](int64_t f) { return pos3[size_t(pos2[size_t(f)])]; };   // first nonzero of fiber f
-    std::vector<sa_item> small;
-    std::vector<group_rec> groups;
+    std::vector<sa_item> items;
     for (int64_t s = 0; s < t->count[0]; ++s) {
         const int64_t fa = pos1[size_t(s)], fb = pos1[size_t(s) + 1];
-        const int64_t pa = nz_of_fiber(fa), pb = nz_of_fiber(fb);
-        const int64_t n = pb - pa;
         const int32_t row = t->crd[0][size_t(s)];
-        if (n <= SMALL_MAX || fb - fa == 1) {
-            sa_item it = empty_item();
-            it.out_row = row; it.row_end = row + 1;
-            it.f0 = int32_t(fa); it.f1 = int32_t(fb); it.p0 = int32_t(pa); it.p1 = int32_t(pb);
-            small.push_back(it);
-            continue;
-        }
-        const int64_t chunk = chunk_for(n, MIN_CHUNK, MAX_PARTS);
-        const int64_t piece = (chunk + SA_WARPS_PER_CTA - 1) / SA_WARPS_PER_CTA;
-        // cut the fiber list where the running nonzero count crosses multiples of `piece`
-        std::vector<sa_item> pieces;
-        int64_t f = fa;
-        while (f < fb) {
-            const int64_t start_nz = nz_of_fiber(f);
-            int64_t g = f + 1;
-            while (g < fb && nz_of_fiber(g) - start_nz < piece) ++g;
-            sa_item it = empty_item();
-            it.out_row = row; it.row_end = row + 1;
-            it.f0 = int32_t(f); it.f1 = int32_t(g);
-            it.p0 = int32_t(start_nz); it.p1 = int32_t(nz_of_fiber(g));
-            pieces.push_back(it);
-            f = g;
-        }
-        const int64_t ng = (int64_t(pieces.size()) + SA_WARPS_PER_CTA - 1) / SA_WARPS_PER_CTA;
+        const int64_t nc = (fb - fa + CHUNK_F - 1) / CHUNK_F;
         int32_t slot0 = -1;
-        if (ng > 1) {
-            slot0 = int32_t(wl.n_slots);
-            wl.fix.push_back(sa_fix{row, slot0, int32_t(ng), 0});
-            wl.n_slots += ng;
+        if (nc > 1) {
+            slot0 = int32_t(wl2.n_slots);
+            wl2.fix.push_back(sa_fix{row, slot0, int32_t(nc), 0});
+            wl2.n_slots += nc;
         }
-        for (int64_t g = 0; g < ng; ++g) {
-            group_rec rec;
-            rec.len = 0;
-            for (int w = 0; w < SA_WARPS_PER_CTA; ++w) {
-                const size_t q = size_t(g) * SA_WARPS_PER_CTA + size_t(w);
+        for (int64_t c = 0; c < nc; ++c)
+            for (int qc = 0; qc < 4; ++qc) {
                 sa_item it = empty_item();
                 it.out_row = row; it.row_end = row + 1;
-                if (q < pieces.size()) it = pieces[q];
-                it.dest = ng > 1 ? slot0 + int32_t(g) : -1;
-                rec.len += it.p1 - it.p0;
-                rec.items.push_back(it);
+                it.f0 = int32_t(fa + c * CHUNK_F); it.f1 = int32_t(std::min(fb, fa + (c + 1) * CHUNK_F));
+                it.p0 = it.f0; it.p1 = it.f1;          // size key: fibers
+                it.dest = nc > 1 ? slot0 + int32_t(c) : -1;
+                it.pad = qc;
+                items.push_back(it);
             }
-            groups.push_back(std::move(rec));
-        }
     }
-    std::stable_sort(groups.begin(), groups.end(), [](const group_rec &a, const group_rec &b) { return a.len > b.len; });
-    std::stable_sort(small.begin(), small.end(),
-                     [](const sa_item &a, const sa_item &b) { return (a.p1 - a.p0) > (b.p1 - b.p0); });
-    // every item is evaluated twice, once per half of the last dense index n (field pad = 0 / 1)
-    wl.n_group_ctas = 2 * int64_t(groups.size());
-    for (auto &g : groups)
-        for (int nh = 0; nh < 2; ++nh)
-            for (sa_item it : g.items) { it.pad = nh; wl.items.push_back(it); }
-    for (sa_item it : small)
-        for (int nh = 0; nh < 2; ++nh) { it.pad = nh; wl.items.push_back(it); }
-    append_empty_slices(t, wl);
+    // largest first: the tail of the launch is then made of the cheapest items
+    std::stable_sort(items.begin(), items.end(), [](const sa_item &a, const sa_item &b) { return (a.f1 - a.f0) > (b.f1 - b.f0); });
+    wl2.items = std::move(items);
+    wl2.n_group_ctas = 0;
+    append_empty_slices(t, wl2);
 }
 
 // CSR: row ranges of about target_nnz nonzeros (at most max_rows rows); rows longer than
@@ -399,7 +374,7 @@ void build_csr(sa_tensor *t, sa_worklist &wl, int64_t target_nnz, int64_t max_ro
 void sa_build_worklists(sa_tensor *t)
 {
     if (t->fmt == SA_FMT_CSF && t->order == 3) build_ttm3(t, t->wl_main);
-    if (t->fmt == SA_FMT_CSF && t->order == 4) build_ttm4(t, t->wl_main);
+    if (t->fmt == SA_FMT_CSF && t->order == 4) build_ttm4(t, t->wl_main, t->wl_aux);
     if (t->fmt == SA_FMT_CSR) {
         build_csr(t, t->wl_main, 256, 32, 1024, 512);    // fused SDDMM -> SpMM
         build_csr(t, t->wl_aux, 256, 16, 4096, 2048);    // SpMM -> GEMM (both orders)

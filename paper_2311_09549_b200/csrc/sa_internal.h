@@ -97,14 +97,12 @@ struct sa_tensor {
     int32_t *d_pos[SA_MAX_ORDER] = {nullptr, nullptr, nullptr, nullptr};
     int32_t *d_crd[SA_MAX_ORDER] = {nullptr, nullptr, nullptr, nullptr};
     float *d_vals = nullptr;
-    int32_t *d_crd_endflag = nullptr;         // order-4 CSF: last-level crd with bit 31 set on the last nonzero of
-                                              // every (i,j,k) fiber and bit 30 on the last nonzero of every (i,j) fiber
-    uint32_t *d_endbits = nullptr;            // order-3 CSF: bit (p & 31) of word p / 32 is set when nonzero p is the
-                                              // last of its (i,j) fiber
+    uint32_t *d_endbits = nullptr;            // CSF: bit (p & 31) of word p / 32 is set when nonzero p is the last of
+                                              // its last-level fiber ((i,j) for order 3, (i,j,k) for order 4)
     int32_t *d_status = nullptr;              // [4] device status word
 
-    sa_worklist wl_main;                      // TTM3 / TTM4 / SDDMM-SpMM
-    sa_worklist wl_aux;                       // CSR: SpMM-GEMM row items
+    sa_worklist wl_main;                      // TTM3 / pass 1 of TTM4 / SDDMM-SpMM
+    sa_worklist wl_aux;                       // CSR: SpMM-GEMM row items; order-4 CSF: pass 2 of TTM4
 
     mutable std::atomic<int> last_launches{0};   // the only mutable field: concurrent sa_run calls may write it
     std::vector<void *> dev_blocks;           // everything obtained from the allocator
@@ -113,6 +111,20 @@ struct sa_tensor {
 // ---- host builder (sa_build.cu)
 sa_status sa_build_levels(sa_tensor *t, const int32_t *coords, const float *vals);
 void sa_build_worklists(sa_tensor *t);
+
+// What the order-3 kernel needs to know about the tensor it walks: an order-3 CSF tensor, or an order-4 one
+// seen as a collection of (i,j) subtrees (slices = level-1 fibers, fibers = level-2 nodes).
+struct sa_ttm3_view {
+    const sa_worklist *wl;        // units, tasks, fix-up entries
+    const int32_t *crd_fiber;     // per fiber: row of the first factor
+    const int32_t *crd_nz;        // per nonzero: row of the second factor
+    const float *vals;
+    const uint32_t *endbits;      // bit p set: nonzero p is the last of its fiber
+    int64_t n_fibers, n_out_rows, nnz;
+    int32_t *status;              // the tensor's device status word
+};
+sa_status sa_launch_ttm3_view(const sa_ttm3_view &v, const sa_dense &first, const sa_dense &second, float *out,
+                              float *partial, cudaStream_t stream, int *launches);
 
 // ---- launchers (one per chain); all asynchronous on `stream`, return SA_OK or SA_E_*.
 sa_status sa_launch_ttm3(const sa_tensor *t, const sa_dense *ops, float *out, void *ws, size_t ws_bytes,

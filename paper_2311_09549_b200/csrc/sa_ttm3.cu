@@ -472,9 +472,10 @@ ttm3_kernel(const sa_unit3 *__restrict__ units, const int32_t *__restrict__ task
 }
 
 template <int L, int M>
-cudaError_t launch(const sa_tensor *t, const sa_dense *ops, float *out, float *partial, cudaStream_t stream)
+cudaError_t launch(const sa_ttm3_view &v, const sa_dense &first, const sa_dense &second, float *out, float *partial,
+                   cudaStream_t stream)
 {
-    const sa_worklist &wl = t->wl_main;
+    const sa_worklist &wl = *v.wl;
     const int64_t n_tasks = int64_t(wl.task_start.size()) - 1;
     const int64_t ctas = (n_tasks + SA_TTM3_WARPS - 1) / SA_TTM3_WARPS;
     if (ctas <= 0) return cudaSuccess;
@@ -483,13 +484,13 @@ cudaError_t launch(const sa_tensor *t, const sa_dense *ops, float *out, float *p
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess)
         return cudaGetLastError();
     dbg_limits lim;
-    lim.status = t->d_status;
-    lim.c_rows = uint32_t(ops[0].rows); lim.d_rows = uint32_t(ops[1].rows);
-    lim.n_fibers = uint32_t(t->count[1]); lim.n_slices_dim = uint32_t(t->dims[0]);
-    lim.nnz = t->nnz;
-    kern<<<(unsigned)ctas, 32 * SA_TTM3_WARPS, smem, stream>>>(wl.d_units3, wl.d_task_start, n_tasks, int(wl.n_group_ctas), t->d_crd[1], t->d_crd[2],
-                                               t->d_vals, t->d_endbits, ops[0].ptr, uint32_t(ops[0].ld), ops[1].ptr,
-                                               uint32_t(ops[1].ld), out, partial, lim);
+    lim.status = v.status;
+    lim.c_rows = uint32_t(first.rows); lim.d_rows = uint32_t(second.rows);
+    lim.n_fibers = uint32_t(v.n_fibers); lim.n_slices_dim = uint32_t(v.n_out_rows);
+    lim.nnz = v.nnz;
+    kern<<<(unsigned)ctas, 32 * SA_TTM3_WARPS, smem, stream>>>(wl.d_units3, wl.d_task_start, n_tasks, int(wl.n_group_ctas), v.crd_fiber,
+                                                              v.crd_nz, v.vals, v.endbits, first.ptr, uint32_t(first.ld), second.ptr,
+                                                              uint32_t(second.ld), out, partial, lim);
     return cudaGetLastError();
 }
 
@@ -502,29 +503,43 @@ size_t sa_ws_ttm3(const sa_tensor *t, const sa_dense *ops)
     return sa_align256(size_t(t->wl_main.n_slots) * size_t(ops[0].cols * ops[1].cols) * sizeof(float));
 }
 
-sa_status sa_launch_ttm3(const sa_tensor *t, const sa_dense *ops, float *out, void *ws, size_t ws_bytes,
-                         cudaStream_t stream, int *launches)
+sa_status sa_launch_ttm3_view(const sa_ttm3_view &v, const sa_dense &first, const sa_dense &second, float *out,
+                              float *partial, cudaStream_t stream, int *launches)
 {
-    const int64_t L = ops[0].cols, M = ops[1].cols;
-    (void)ws_bytes;
-    // the kernel addresses factor rows with 32-bit byte offsets
-    for (int i = 0; i < 2; ++i)
-        if (ops[i].rows * ops[i].ld >= (int64_t(1) << 30)) return SA_E_UNSUPPORTED;
-    if (!t->d_endbits) return SA_E_UNSUPPORTED;
-    float *partial = static_cast<float *>(ws);
+    const int64_t L = first.cols, M = second.cols;
+    // the kernel addresses factor rows with 32-bit offsets
+    if (first.rows * first.ld >= (int64_t(1) << 30) || second.rows * second.ld >= (int64_t(1) << 30)) return SA_E_UNSUPPORTED;
+    if (!v.endbits) return SA_E_UNSUPPORTED;
     cudaError_t e;
-    if (L == 16 && M == 16) e = launch<16, 16>(t, ops, out, partial, stream);
-    else if (L == 32 && M == 16) e = launch<32, 16>(t, ops, out, partial, stream);
-    else if (L == 16 && M == 32) e = launch<16, 32>(t, ops, out, partial, stream);
-    else if (L == 32 && M == 32) e = launch<32, 32>(t, ops, out, partial, stream);
+    if (L == 16 && M == 16) e = launch<16, 16>(v, first, second, out, partial, stream);
+    else if (L == 32 && M == 16) e = launch<32, 16>(v, first, second, out, partial, stream);
+    else if (L == 16 && M == 32) e = launch<16, 32>(v, first, second, out, partial, stream);
+    else if (L == 32 && M == 32) e = launch<32, 32>(v, first, second, out, partial, stream);
     else return SA_E_UNSUPPORTED;
     if (e != cudaSuccess) return SA_E_CUDA;
-    *launches = t->wl_main.items.empty() ? 0 : 1;
-    if (!t->wl_main.fix.empty()) {
-        if (sa_launch_fixup(t->wl_main, partial, out, int(L * M), stream) != cudaSuccess) return SA_E_CUDA;
+    *launches = v.wl->items.empty() ? 0 : 1;
+    if (!v.wl->fix.empty()) {
+        if (sa_launch_fixup(*v.wl, partial, out, int(L * M), stream) != cudaSuccess) return SA_E_CUDA;
         *launches += 1;
     }
     return SA_OK;
+}
+
+sa_status sa_launch_ttm3(const sa_tensor *t, const sa_dense *ops, float *out, void *ws, size_t ws_bytes,
+                         cudaStream_t stream, int *launches)
+{
+    (void)ws_bytes;
+    sa_ttm3_view v;
+    v.wl = &t->wl_main;
+    v.crd_fiber = t->d_crd[1];
+    v.crd_nz = t->d_crd[2];
+    v.vals = t->d_vals;
+    v.endbits = t->d_endbits;
+    v.n_fibers = t->count[1];
+    v.n_out_rows = t->dims[0];
+    v.nnz = t->nnz;
+    v.status = t->d_status;
+    return sa_launch_ttm3_view(v, ops[0], ops[1], out, static_cast<float *>(ws), stream, launches);
 }
 
 // ------------------------------------------------------------------ entry point without allocation

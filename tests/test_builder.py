@@ -73,64 +73,47 @@ def test_levels_match_independent_construction(cfg):
     assert np.array_equal(got_vals, want_vals)
 
 
-def _fiber_nnz_range(t, fmt, order, levels, f0, f1):
-    if order == 3:
-        return levels[2][0][f0], levels[2][0][f1]
-    pos2, pos3 = levels[2][0], levels[3][0]
-    return pos3[pos2[f0]], pos3[pos2[f1]]
-
-
 @pytest.mark.parametrize("cfg", [1, 2, 5])
 def test_csf_worklist_partitions_every_nonzero_once(cfg):
+    """Main list of a CSF tensor: the units of the order-3 kernel.  For an order-4 tensor its "slices" are the
+    (i,j) subtrees (output row = index of the level-1 fiber) and its fibers the (i,j,k) fibers."""
     w = configs.make(cfg, "mini")
     t = sa.SparseTensor(w.dims, w.coords, w.vals, sa.SA_FMT_CSF, device=-1)
     levels, _ = export_all(t, "csf")
     counts, items, fix = sa.sa_tensor_worklist(t.handle)
     n_items, n_groups, n_fix, n_slots = (int(x) for x in counts)
-    crd0, pos1 = levels[0][1], levels[1][0]
-    slice_pos = {int(c): n for n, c in enumerate(crd0)}
+    if t.order == 3:
+        slice_rows, pos1, pos2 = levels[0][1], levels[1][0], levels[2][0]
+    else:
+        pos1, pos2 = levels[2][0], levels[3][0]
+        slice_rows = np.arange(len(pos1) - 1)
+    slice_pos = {int(c): n for n, c in enumerate(slice_rows)}
     covered = np.zeros(w.nnz, dtype=np.int32)
     slot_owner = {}
-    group_items = n_groups * 8
     G = 4                                   # warps (tasks) per thread block of the order-3 kernel
-    if t.order == 3:
-        task_start, stream_f0 = sa.sa_tensor_tasks(t.handle)
-        group_items = int(task_start[n_groups * G])
-        item_group = np.searchsorted(task_start, np.arange(n_items), side="right") - 1
-    for n, (row, row_end, f0, f1, p0, p1, dest, _) in enumerate(items):
-        if p0 == p1:
-            assert t.order == 4 and n < n_groups * 8 and f0 == f1, "only padding items of an order-4 group may be empty"
-            continue
+    task_start, stream_f0 = sa.sa_tensor_tasks(t.handle)
+    group_items = int(task_start[n_groups * G])
+    item_group = np.searchsorted(task_start, np.arange(n_items), side="right") - 1
+    for n, (row, row_end, f0, f1, p0, p1, dest, spos) in enumerate(items):
+        assert p0 < p1, "no empty units"
         s = slice_pos[int(row)]
-        fa, fb = _fiber_nnz_range(t, "csf", t.order, levels, f0, f1)
-        if t.order == 3 and n >= group_items:
+        fa, fb = pos2[f0], pos2[f1]
+        if n >= group_items:
             # a whole small slice
-            assert int(items[n][7]) == s and (f0, f1) == (pos1[s], pos1[s + 1]) and (fa, fb) == (p0, p1)
+            assert int(spos) == s and (f0, f1) == (pos1[s], pos1[s + 1]) and (fa, fb) == (p0, p1)
             assert p1 - p0 <= 2048 and dest == -1
         else:
             assert pos1[s] <= f0 < f1 <= pos1[s + 1], "fibers stay inside the item's slice"
             assert fa <= p0 < p1 <= fb, "nonzero range lies inside the fiber range"
-            if t.order == 3:     # first and last fiber really intersect the clip range
-                pos2 = levels[2][0]
-                assert pos2[f0 + 1] > p0 and pos2[f1 - 1] < p1 and int(items[n][7]) == s
-            else:
-                assert (fa, fb) == (p0, p1), "order-4 items hold whole (i,j) subtrees"
-        covered[p0:p1] += 1
-        if t.order == 3 and n < group_items:
+            # first and last fiber really intersect the clip range
+            assert pos2[f0 + 1] > p0 and pos2[f1 - 1] < p1 and int(spos) == s
             lead = items[task_start[(item_group[n] // G) * G]]
             assert dest == lead[6] and row == lead[0], "a group works on one slice and one destination"
-        if t.order == 4 and n < n_groups * 8:
-            lead = items[(n // 8) * 8]
-            assert dest == lead[6] and row == lead[0], "a group works on one slice and one destination"
+        covered[p0:p1] += 1
         if dest >= 0:
             slot_owner.setdefault(int(dest), int(row))
             assert slot_owner[int(dest)] == int(row)
-    # order 4: every item appears once per half of the last dense index (field 7 = 0 / 1)
-    want = 2 if t.order == 4 else 1
-    assert (covered == want).all(), "every nonzero belongs to exactly one item (per half)"
-    if t.order == 4:
-        assert np.array_equal(np.sort(items[items[:, 5] > items[:, 4]][:, 7].astype(np.int64)).reshape(2, -1).sum(axis=1),
-                              [0, (items[:, 5] > items[:, 4]).sum() // 2])
+    assert (covered == 1).all(), "every nonzero belongs to exactly one unit"
     # fix-up entries: split slices own disjoint slot ranges, empty slices are listed with count 0
     used = np.zeros(n_slots, dtype=np.int32)
     empties = set()
@@ -141,31 +124,64 @@ def test_csf_worklist_partitions_every_nonzero_once(cfg):
         used[slot0:slot0 + count] += 1
         assert all(slot_owner[s] == int(row) for s in range(slot0, slot0 + count))
     assert (used == 1).all() and set(slot_owner) == set(range(n_slots))
-    assert empties == set(range(w.dims[0])) - set(int(c) for c in crd0)
-    # nonzero balance: no warp item is larger than the small-slice bound / the piece size
+    if t.order == 3:
+        assert empties == set(range(w.dims[0])) - set(int(c) for c in slice_rows)
+    else:
+        assert not empties, "every level-1 fiber has nonzeros"
+    # nonzero balance: no unit is larger than the small-slice bound / the piece size
     sizes = items[:, 5] - items[:, 4]
     assert sizes.max() <= max(4096, int(np.ceil(w.nnz / 8)))
-    if t.order == 3:
-        # tasks: a partition of the item list; group tasks hold at most one item and warp 0 of a group has one;
-        # small-slice tasks hold at most 16 items and about 2048 nonzeros
-        assert task_start[0] == 0 and task_start[-1] == n_items and (np.diff(task_start) >= 0).all()
-        per_task = np.diff(task_start)
-        assert (per_task[:n_groups * G] <= 1).all() and (per_task[:n_groups * G:G] == 1).all()
-        assert (per_task[n_groups * G:] >= 1).all() and (per_task[n_groups * G:] <= 16).all()
-        for a, b in zip(task_start[n_groups * G:-1], task_start[n_groups * G + 1:]):
-            assert b - a == 1 or sizes[a:b].sum() <= 2048
-        # stream starts: part q of an item begins in fiber stream_f0[n, q]
-        pos2 = levels[2][0]
-        for n, (row, row_end, f0, f1, p0, p1, dest, _) in enumerate(items):
-            b8 = (p0 // 8) * 8
-            slen = -(-(-(-(p1 - b8) // 4)) // 8) * 8
-            for q in range(4):
-                lo, hi = max(p0, b8 + q * slen), min(p1, b8 + (q + 1) * slen)
-                f = int(stream_f0[n, q])
-                if lo < hi:
-                    assert f0 <= f < f1 and pos2[f] <= lo < pos2[f + 1]
-                else:
-                    assert f == f0
+    # tasks: a partition of the item list; group tasks hold at most one item and warp 0 of a group has one;
+    # small-slice tasks hold at most 16 items and about 2048 nonzeros
+    assert task_start[0] == 0 and task_start[-1] == n_items and (np.diff(task_start) >= 0).all()
+    per_task = np.diff(task_start)
+    assert (per_task[:n_groups * G] <= 1).all() and (per_task[:n_groups * G:G] == 1).all()
+    assert (per_task[n_groups * G:] >= 1).all() and (per_task[n_groups * G:] <= 16).all()
+    for a, b in zip(task_start[n_groups * G:-1], task_start[n_groups * G + 1:]):
+        assert b - a == 1 or sizes[a:b].sum() <= 2048
+    # stream starts: part q of an item begins in fiber stream_f0[n, q]
+    for n, (row, row_end, f0, f1, p0, p1, dest, _) in enumerate(items):
+        b8 = (p0 // 8) * 8
+        slen = -(-(-(-(p1 - b8) // 4)) // 8) * 8
+        for q in range(4):
+            lo, hi = max(p0, b8 + q * slen), min(p1, b8 + (q + 1) * slen)
+            f = int(stream_f0[n, q])
+            if lo < hi:
+                assert f0 <= f < f1 and pos2[f] <= lo < pos2[f + 1]
+            else:
+                assert f == f0
+
+
+def test_order4_second_pass_worklist_covers_every_fiber_quarter_once():
+    """Second list of an order-4 tensor: (piece of a slice) x (quarter of the temporaries' columns)."""
+    w = configs.make(5, "mini")
+    t = sa.SparseTensor(w.dims, w.coords, w.vals, sa.SA_FMT_CSF, device=-1)
+    levels, _ = export_all(t, "csf")
+    crd0, pos1 = levels[0][1], levels[1][0]
+    counts, items, fix = sa.sa_tensor_worklist(t.handle, 1)
+    slice_pos = {int(c): n for n, c in enumerate(crd0)}
+    covered = np.zeros((len(levels[1][1]), 4), dtype=np.int32)
+    pieces = {}
+    for row, row_end, f0, f1, _, _, dest, quarter in items:
+        s = slice_pos[int(row)]
+        assert pos1[s] <= f0 < f1 <= pos1[s + 1] and f1 - f0 <= 512 and 0 <= quarter < 4
+        covered[f0:f1, quarter] += 1
+        if dest >= 0:
+            pieces.setdefault(int(row), set()).add(int(dest))
+        else:
+            assert (f0, f1) == (pos1[s], pos1[s + 1])
+    assert (covered == 1).all()
+    assert (np.diff(items[:, 3] - items[:, 2]) <= 0).all(), "largest items first"
+    empties = set()
+    used = np.zeros(int(counts[3]), dtype=np.int32)
+    for row, slot0, count, _ in fix:
+        if count == 0:
+            empties.add(int(row))
+            continue
+        assert pieces[int(row)] == set(range(slot0, slot0 + count))
+        used[slot0:slot0 + count] += 1
+    assert (used == 1).all()
+    assert empties == set(range(w.dims[0])) - set(int(c) for c in crd0)
 
 
 @pytest.mark.parametrize("cfg,which", [(3, 0), (4, 1), (4, 0)])

@@ -173,10 +173,15 @@ def test_spmm_gemm_rank_combinations_and_long_rows(sa, L, M):
 
 
 def test_ttm4_ragged_and_split_slices(sa):
-    w = configs.make_ttm4_zipf("edge4", 31, 90, 60, 50, 45, 150_000, 1.4, 5.0, 16, 16, 16)
+    # few level-1 fibers per slice: the head slice's (i,j) subtrees exceed one thread block's chunk, so the
+    # first pass writes partial temporaries that the fix-up kernel sums
+    w = configs.make_ttm4_zipf("edge4", 31, 90, 6, 130, 110, 150_000, 1.4, 5.0, 16, 16, 16)
     A, t = _check(sa, w)
-    counts, _, fix = sa.sa_tensor_worklist(t.handle)
-    assert counts[3] >= 2, "the head slice must be split over several thread blocks"
+    assert sa.sa_tensor_worklist(t.handle, 0)[0][3] >= 2, "a large (i,j) subtree must be split over several thread blocks"
+    # many level-1 fibers per slice: the second pass cuts the head slices into pieces of 512 fibers
+    w = configs.make_ttm4_zipf("edge4b", 32, 90, 700, 50, 45, 150_000, 1.4, 5.0, 16, 16, 16)
+    A, t = _check(sa, w)
+    assert sa.sa_tensor_worklist(t.handle, 1)[0][3] >= 2, "the head slice must be split into several pieces"
 
 
 def test_results_are_reproducible_run_to_run(sa):
