@@ -252,10 +252,13 @@ void build_ttm3_lists(sa_worklist &wl, int64_t n_slices, RowOf row_of, const std
             wl.task_start.push_back(int32_t(wl.items.size()));
             if (size_t(w) < g.items.size()) wl.items.push_back(g.items[size_t(w)]);
         }
+    // a task strings several small slices together only when there are enough of them to fill the machine
+    // (a few thousand warps) anyway
+    const int64_t max_units = std::min<int64_t>(MAX_UNITS, std::max<int64_t>(1, int64_t(small.size()) / 4096));
     for (size_t x = 0; x < small.size();) {
         wl.task_start.push_back(int32_t(wl.items.size()));
         int64_t total = 0, cnt = 0;
-        while (x < small.size() && cnt < MAX_UNITS && (cnt == 0 || total + (small[x].p1 - small[x].p0) <= SMALL_MAX)) {
+        while (x < small.size() && cnt < max_units && (cnt == 0 || total + (small[x].p1 - small[x].p0) <= SMALL_MAX)) {
             total += small[x].p1 - small[x].p0;
             wl.items.push_back(small[x]);
             ++x; ++cnt;

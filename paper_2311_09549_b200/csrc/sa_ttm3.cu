@@ -74,7 +74,8 @@ struct cfg {
     static constexpr int VEC = M / 8;            // floats of a factor row per lane (eight lanes per row)
     static constexpr int RS = M + 8;             // row stride of the ring of parked temporaries and of a warp's
                                                  // tile in the CTA reduction; word M of a ring row = C row offset
-    static constexpr int RING = 64;              // ring rows: at most 7 left over + 32 parked in one round
+    static constexpr int RING = 64;              // rows parked fibers wait in: a round starts at row <= 31 with at most
+                                                 // 7 rows left over and parks at most 32 more
     static constexpr int DEPTH = 8;              // rounds of index / value data in flight (cp.async ring)
     static constexpr int SLOT = 80;              // bytes per (round, stream): 8 indices | 8 values | end bits | pad
     static constexpr int OFF_KV = 0;
@@ -136,15 +137,15 @@ struct rowvec<2> {
     }
 };
 
-// acc += Cg^T . T for the ring rows (row0 + x) & (RING - 1), x = 0 .. 7, of which the first n are in use.
+// acc += Cg^T . T for the parked rows row0 + x, x = 0 .. 7, of which the first n are in use.
 template <int L, int M>
 __device__ __forceinline__ void ttm3_flush(float (&acc)[cfg<L, M>::MT][cfg<L, M>::NT][4], const float *__restrict__ ring,
                                            int row0, int n, const float *__restrict__ C, int lane, const dbg_limits &lim, uint32_t ldc)
 {
     using K = cfg<L, M>;
     const int g = lane >> 2, t = lane & 3;
-    const float *ra = ring + ((row0 + t) & (K::RING - 1)) * K::RS;
-    const float *rb = ring + ((row0 + t + 4) & (K::RING - 1)) * K::RS;
+    const float *ra = ring + (row0 + t) * K::RS;
+    const float *rb = ring + (row0 + t + 4) * K::RS;
     // the values of C this flush needs: rows of the fibers x = t and x = t + 4, columns 16 mt + g (+ 8)
     float cf[K::MT][4];
     {
@@ -212,6 +213,7 @@ __device__ __forceinline__ void zero_tile(float (&acc)[cfg<L, M>::MT][cfg<L, M>:
 // Where stream q of a unit runs: rounds, aligned start, and the clipped range [lo, hi) (see sa_unit3_streams).
 struct stream_range {
     int rounds, base, lo, hi;
+    int full;       // rounds 1 .. full - 2 lie inside every stream's part: nothing to mask, no cut fiber to close
 };
 __device__ __forceinline__ stream_range stream_of(int p0, int p1, int q)
 {
@@ -222,6 +224,7 @@ __device__ __forceinline__ stream_range stream_of(int p0, int p1, int q)
     r.base = base8 + q * slen;
     r.lo = max(p0, r.base);
     r.hi = min(p1, r.base + slen);
+    r.full = (span - (SA_STREAMS - 1) * slen) >> 3;
     return r;
 }
 
@@ -307,7 +310,7 @@ __device__ __forceinline__ void ttm3_warp_task(const sa_unit3 *__restrict__ unit
     float T[VEC];
 #pragma unroll
     for (int x = 0; x < VEC; ++x) T[x] = 0.f;
-    int nclosed = 0, nflushed = 0, sc = 0;
+    int rbase = 0, npend = 0, sc = 0;               // parked rows waiting for the tensor cores: rbase .. rbase + npend - 1
 #ifdef SA_DEBUG_BOUNDS
     int dbg_rounds = 0;
 #endif
@@ -326,10 +329,14 @@ __device__ __forceinline__ void ttm3_warp_task(const sa_unit3 *__restrict__ unit
         const uint32_t fw = lds32(slot_c + 64);
         // which of the eight positions pg .. pg + 7 belong to the stream, and which of them end a fiber
         const int pg = cs.base + 8 * cr;
-        const int a = min(max(cs.lo - pg, 0), 8), b = min(max(cs.hi - pg, 0), 8);
-        const uint32_t vm = ((1u << b) - 1u) & ~((1u << a) - 1u);
-        uint32_t e8 = (fw >> (pg & 24)) & vm;
-        if (cs.hi > cs.lo && uint32_t(cs.hi - pg - 1) < 8u) e8 |= 1u << (cs.hi - pg - 1);   // the part's last nonzero closes its (possibly cut) fiber
+        const bool interior = cr >= 1 && cr < cs.full - 1;      // warp-uniform
+        uint32_t vm = 0xffu, e8 = (fw >> (pg & 24)) & 0xffu;
+        if (!interior) {
+            const int a = min(max(cs.lo - pg, 0), 8), b = min(max(cs.hi - pg, 0), 8);
+            vm = ((1u << b) - 1u) & ~((1u << a) - 1u);
+            e8 &= vm;
+            if (cs.hi > cs.lo && uint32_t(cs.hi - pg - 1) < 8u) e8 |= 1u << (cs.hi - pg - 1);   // the part's last nonzero closes its (possibly cut) fiber
+        }
         // ring rows for the fibers this round parks: stream-major
         const int cnt = __popc(e8);
         int incl = cnt;
@@ -340,11 +347,12 @@ __device__ __forceinline__ void ttm3_warp_task(const sa_unit3 *__restrict__ unit
             if (lane >= 16) incl += o;
         }
         const int total = __shfl_sync(SA_FULL_MASK, incl, 31);
-        int slot = nclosed + incl - cnt;
-        nclosed += total;
+        const int slot = rbase + npend + incl - cnt;          // first row of this stream's fibers in this round
+        npend += total;
+        uint32_t waddr = s_ring + (slot * K::RS + c * VEC) * 4;
         if (c < cnt) {
             const uint32_t off = uint32_t(jreg) * ldc;
-            sts32(s_ring + (((slot + c) & (K::RING - 1)) * K::RS + M) * 4, off);
+            sts32(s_ring + ((slot + c) * K::RS + M) * 4, off);
             prefetch_l1(C + off);
         }
         fq += cnt;
@@ -375,33 +383,45 @@ __device__ __forceinline__ void ttm3_warp_task(const sa_unit3 *__restrict__ unit
                         rowvec<VEC> tv;
 #pragma unroll
                         for (int x = 0; x < VEC; ++x) { tv.x[x] = T[x]; T[x] = 0.f; }
-                        tv.store_shared(s_ring + ((slot & (K::RING - 1)) * K::RS + c * VEC) * 4);
-                        ++slot;
+                        tv.store_shared(waddr);
+                        waddr += K::RS * 4;
                     }
                 }
             }
         };
-        if (__any_sync(SA_FULL_MASK, vm != 0xffu)) steps(std::true_type{});
+        if (!interior && __any_sync(SA_FULL_MASK, vm != 0xffu)) steps(std::true_type{});
         else steps(std::false_type{});
         __syncwarp();
-        while (nclosed - nflushed >= 8) {
-            ttm3_flush<L, M>(acc, ring, nflushed, 8, C, lane, lim, ldc);
-            nflushed += 8;
+        while (npend >= 8) {
+            ttm3_flush<L, M>(acc, ring, rbase, 8, C, lane, lim, ldc);
+            rbase += 8;
+            npend -= 8;
         }
         __syncwarp();
+        if (rbase >= 32) {
+            // move the (at most seven) rows left over to the front so that the next round's rows fit behind them
+            constexpr int CH = K::RS / 4;                          // 16-byte pieces per row
+            for (int x = lane; x < npend * CH; x += 32) {
+                const int r = x / CH, ch = x - r * CH;
+                const uint4 w = lds128(s_ring + ((rbase + r) * K::RS) * 4 + 16 * ch);
+                asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(s_ring + (r * K::RS) * 4 + 16 * ch), "r"(w.x), "r"(w.y), "r"(w.z), "r"(w.w) : "memory");
+            }
+            rbase = 0;
+            __syncwarp();
+        }
         jreg = jnext;
         sc = sn;
       }
       // the unit ends: the open group of parked rows, the tile, the next unit
       {
-        const int n = nclosed - nflushed;
+        const int n = npend;
         if (n > 0) {
-            for (int x = n; x < 8; ++x) ring[((nflushed + x) & (K::RING - 1)) * K::RS + lane % M] = 0.f;
+            for (int x = n; x < 8; ++x) ring[(rbase + x) * K::RS + lane % M] = 0.f;
             __syncwarp();
-            ttm3_flush<L, M>(acc, ring, nflushed, n, C, lane, lim, ldc);
+            ttm3_flush<L, M>(acc, ring, rbase, n, C, lane, lim, ldc);
             __syncwarp();
         }
-        nclosed = nflushed = 0;
+        rbase = npend = 0;
         if (!keep) {
             if (SA_CHK(lim, uint32_t(crow) < lim.n_slices_dim, 8, crow)) store_tile<L, M>(acc, out + int64_t(crow) * (L * M), lane);
             zero_tile<L, M>(acc);
