@@ -99,6 +99,11 @@ def algorithmic_work(w, counts, sched):
         I = w.dims[0]
         K, L = w.dense[0].shape[1], w.dense[2].shape[1]
         return 8 * nnz + 4 * (I + 1) + 4 * (K + L) * nnz + sz(w.dense[0]) + out_bytes, nnz * (2 * K + 1 + 2 * L)
+    if w.expr == "spmmh_gemm":
+        # two gathered rows of L floats per nonzero (C and its Hadamard partner), E once, the output once
+        I, J = w.dims
+        L, M = w.dense[0].shape[1], w.dense[2].shape[1]
+        return 8 * nnz + 4 * (I + 1) + 8 * L * nnz + sz(w.dense[2]) + out_bytes, 3 * nnz * L + 2 * I * L * M
     if w.expr == "spmm_gemm":
         I, J = w.dims
         L, M = w.dense[0].shape[1], w.dense[1].shape[1]
@@ -185,6 +190,7 @@ def oracle_sample(w, budget_s=15.0):
                "spttm_ttm4": lambda: w.dense[0].shape[1] * w.dense[1].shape[1] * w.dense[2].shape[1],
                "sddmm_spmm": lambda: w.dense[0].shape[1] * w.dense[2].shape[1],
                "spmm_gemm": lambda: w.dense[0].shape[1] * w.dense[1].shape[1],
+               "spmmh_gemm": lambda: w.dense[0].shape[1] * w.dense[2].shape[1],
                "sddmm_spmm_gemm": lambda: w.dense[0].shape[1] * w.dense[2].shape[1] * w.dense[3].shape[1],
                "ttmc3": lambda: w.dense[0].shape[1] * w.dense[1].shape[1] * w.dense[2].shape[1]}[w.expr]()
     cores = oracle.max_threads()
@@ -235,7 +241,8 @@ def workload_label(cfg, sched):
              3: "cfg3 <SDDMM,SpMM> 1Mx1M 30M nnz K=L=64", 4: "cfg4 <SpMM,GEMM> 4Mx4M 100M nnz L=256 M=64",
              5: "cfg5 order-4 <SpTTM,TTM> 50000x20000^3 100M nnz ranks 16",
              7: "kernel 2 <SDDMM,SpMM,GEMM> on the config-3 tensor, K=L=M=64",
-             6: "kernel 5 <3D TTMC> on a nell-2-shaped tensor 12000x9000x288000 76.88M nnz L=M=N=16"}
+             6: "kernel 5 <3D TTMC> on a nell-2-shaped tensor 12000x9000x288000 76.88M nnz L=M=N=16",
+             8: "kernel 3 <SpMMH,GEMM> on the config-4 tensor recipe 4Mx4M 100M nnz L=256 M=64"}
     return names[cfg] + (" (%s)" % sched if cfg == 4 else "")
 
 
@@ -271,7 +278,7 @@ def main():
     ap.add_argument("--steps", type=int, default=31)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", type=int, default=2, choices=[1, 2, 3, 4, 5, 6, 7])
+    ap.add_argument("--workload", type=int, default=2, choices=[1, 2, 3, 4, 5, 6, 7, 8])
     ap.add_argument("--scale", default="full", choices=["full", "mid", "mini"])
     ap.add_argument("--sched", default="right", choices=["left", "right"], help="association order for workload 4")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -66,7 +66,11 @@ typedef enum {
     SA_EXPR_TTMC3 = 5,
     /* kernel 2 <SDDMM,SpMM,GEMM>: A(i,m) = sum_{j,k,l} B(i,j) C(i,k) D(j,k) E(j,l) F(l,m);
      * ops = {C, D, E, F}; B CSR; two-level schedule with the row temporary T(l) in the workspace */
-    SA_EXPR_SDDMM_SPMM_GEMM = 6
+    SA_EXPR_SDDMM_SPMM_GEMM = 6,
+    /* kernel 3 <SpMMH,GEMM>: A(i,m) = sum_{j,l} B(i,j) C(j,l) D(j,l) E(l,m); ops = {C, D, E}; B CSR;
+     * the Description column of the Table of kernels (SpMM with a Hadamard product, then GEMM),
+     * evaluated per row as T(l) = sum_j B(i,j) C(j,l) D(j,l) followed by T . E                   */
+    SA_EXPR_SPMMH_GEMM = 7
 } sa_expr;
 
 typedef enum {
@@ -189,7 +193,8 @@ sa_status sa_workspace_size(const sa_tensor *t, sa_expr expr, sa_schedule sched,
  *   cuda_stream  a cudaStream_t (NULL = default stream)
  * Compiled dense ranks (anything else is SA_E_UNSUPPORTED): SPTTM_TTM3 L, M in {16, 32};
  * SPTTM_TTM4 L = M = N = 16; SDDMM_SPMM K, L in {32, 64, 128}; SPMM_GEMM L in {128, 256},
- * M in {32, 64}; TTMC3 L, M, N in {16, 32}; SDDMM_SPMM_GEMM K, L in {32, 64, 128}, M in {32, 64}.
+ * M in {32, 64}; TTMC3 L, M, N in {16, 32}; SDDMM_SPMM_GEMM K, L in {32, 64, 128}, M in {32, 64};
+ * SPMMH_GEMM L in {128, 256}, M in {32, 64}.
  * Returns launch errors only; completion is observed by synchronising the stream.
  * Errors: SA_E_ARG, SA_E_SHAPE, SA_E_UNSUPPORTED, SA_E_WORKSPACE, SA_E_CUDA.
  */

@@ -139,6 +139,10 @@ size_t sa_ws_sddmm_spmm(const sa_tensor *t, const sa_dense *ops, bool materializ
 sa_status sa_launch_spmm_gemm(const sa_tensor *t, const sa_dense *ops, float *out, void *ws, size_t ws_bytes,
                               bool assoc_right, cudaStream_t stream, int *launches);
 size_t sa_ws_spmm_gemm(const sa_tensor *t, const sa_dense *ops, bool assoc_right);
+// Kernel 3 <SpMMH,GEMM>: the row kernel of (B.C).D with the Hadamard product C(j,:) * D(j,:) as the gathered row.
+sa_status sa_launch_spmmh_gemm(const sa_tensor *t, const sa_dense *ops, float *out, void *ws, size_t ws_bytes,
+                               cudaStream_t stream, int *launches);
+size_t sa_ws_spmmh_gemm(const sa_tensor *t, const sa_dense *ops);
 
 sa_status sa_launch_ttmc3(const sa_tensor *t, const sa_dense *ops, float *out, void *ws, size_t ws_bytes,
                           cudaStream_t stream, int *launches);

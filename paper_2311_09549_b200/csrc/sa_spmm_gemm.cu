@@ -46,12 +46,12 @@ __device__ __forceinline__ void load_D(float *Ds, const float *__restrict__ D, i
     }
 }
 
-template <int L, int M>
+template <int L, int M, bool HAD>
 __global__ void __launch_bounds__(256)
 spmm_gemm_left_kernel(const sa_item *__restrict__ items, int64_t n_items, const int32_t *__restrict__ pos,
                       const int32_t *__restrict__ crd, const float *__restrict__ vals, const float *__restrict__ C,
-                      int64_t ldc, const float *__restrict__ D, int64_t ldd, float *__restrict__ out,
-                      float *__restrict__ partial)
+                      int64_t ldc, const float *__restrict__ H, int64_t ldh, const float *__restrict__ D, int64_t ldd,
+                      float *__restrict__ out, float *__restrict__ partial)
 {
     constexpr int LV4 = L / 128, MV = M / 32;
     extern __shared__ __align__(16) float smem[];
@@ -79,9 +79,14 @@ spmm_gemm_left_kernel(const sa_item *__restrict__ items, int64_t n_items, const 
                     const int j = __shfl_sync(SA_FULL_MASK, jj, s);
                     const float v = __shfl_sync(SA_FULL_MASK, vv, s);
                     const float *crow = C + int64_t(j) * ldc + lane * 4;
+                    const float *hrow = H + int64_t(j) * ldh + lane * 4;     // HAD: the row of the Hadamard partner
 #pragma unroll
                     for (int q = 0; q < LV4; ++q) {
-                        const float4 c = sa_ldg4(crow + q * 128);
+                        float4 c = sa_ldg4(crow + q * 128);
+                        if (HAD) {
+                            const float4 h = sa_ldg4(hrow + q * 128);
+                            c.x *= h.x; c.y *= h.y; c.z *= h.z; c.w *= h.w;
+                        }
                         t[q].x = fmaf(v, c.x, t[q].x); t[q].y = fmaf(v, c.y, t[q].y);
                         t[q].z = fmaf(v, c.z, t[q].z); t[q].w = fmaf(v, c.w, t[q].w);
                     }
@@ -305,13 +310,13 @@ sa_status run(const sa_tensor *t, const sa_dense *ops, float *out, void *ws, boo
     *launches = 0;
     if (!right) {
         float *partial = static_cast<float *>(ws);
-        auto kern = spmm_gemm_left_kernel<L, M>;
+        auto kern = spmm_gemm_left_kernel<L, M, false>;
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess) return SA_E_CUDA;
         const int64_t want = (n_items + SA_WARPS_PER_CTA - 1) / SA_WARPS_PER_CTA;
         const int64_t ctas = std::min<int64_t>(want, resident_ctas(reinterpret_cast<const void *>(kern), smem));
         if (ctas > 0) {
             kern<<<(unsigned)ctas, 256, smem, stream>>>(wl.d_items, n_items, t->d_pos[1], t->d_crd[1], t->d_vals, ops[0].ptr,
-                                                       ops[0].ld, ops[1].ptr, ops[1].ld, out, partial);
+                                                       ops[0].ld, ops[0].ptr, ops[0].ld, ops[1].ptr, ops[1].ld, out, partial);
             if (cudaGetLastError() != cudaSuccess) return SA_E_CUDA;
             *launches += 1;
         }
@@ -335,6 +340,32 @@ sa_status run(const sa_tensor *t, const sa_dense *ops, float *out, void *ws, boo
     if (ctas > 0) {
         spmm_kernel<M / 32><<<(unsigned)ctas, 256, 0, stream>>>(wl.d_items, n_items, t->d_pos[1], t->d_crd[1], t->d_vals, E,
                                                                out, partial);
+        if (cudaGetLastError() != cudaSuccess) return SA_E_CUDA;
+        *launches += 1;
+    }
+    if (!wl.fix.empty()) {
+        if (sa_launch_fixup(wl, partial, out, M, stream) != cudaSuccess) return SA_E_CUDA;
+        *launches += 1;
+    }
+    return SA_OK;
+}
+
+// Kernel 3 <SpMMH,GEMM>: ops = {C, D, E}; the gathered row is C(j,:) * D(j,:), the resident matrix is E.
+template <int L, int M>
+sa_status run_hadamard(const sa_tensor *t, const sa_dense *ops, float *out, void *ws, cudaStream_t stream, int *launches)
+{
+    const sa_worklist &wl = t->wl_aux;
+    const int64_t n_items = int64_t(wl.items.size());
+    const size_t smem = size_t(L * M + SA_WARPS_PER_CTA * L) * sizeof(float);
+    *launches = 0;
+    float *partial = static_cast<float *>(ws);
+    auto kern = spmm_gemm_left_kernel<L, M, true>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess) return SA_E_CUDA;
+    const int64_t want = (n_items + SA_WARPS_PER_CTA - 1) / SA_WARPS_PER_CTA;
+    const int64_t ctas = std::min<int64_t>(want, resident_ctas(reinterpret_cast<const void *>(kern), smem));
+    if (ctas > 0) {
+        kern<<<(unsigned)ctas, 256, smem, stream>>>(wl.d_items, n_items, t->d_pos[1], t->d_crd[1], t->d_vals, ops[0].ptr,
+                                                   ops[0].ld, ops[1].ptr, ops[1].ld, ops[2].ptr, ops[2].ld, out, partial);
         if (cudaGetLastError() != cudaSuccess) return SA_E_CUDA;
         *launches += 1;
     }
@@ -391,5 +422,21 @@ sa_status sa_launch_spmm_gemm(const sa_tensor *t, const sa_dense *ops, float *ou
     if (L == 128 && M == 64) return run<128, 64>(t, ops, out, ws, right, stream, launches);
     if (L == 256 && M == 32) return run<256, 32>(t, ops, out, ws, right, stream, launches);
     if (L == 256 && M == 64) return run<256, 64>(t, ops, out, ws, right, stream, launches);
+    return SA_E_UNSUPPORTED;
+}
+
+size_t sa_ws_spmmh_gemm(const sa_tensor *t, const sa_dense *ops)
+{
+    return sa_align256(size_t(t->wl_aux.n_slots) * size_t(ops[2].cols) * sizeof(float));
+}
+
+sa_status sa_launch_spmmh_gemm(const sa_tensor *t, const sa_dense *ops, float *out, void *ws, size_t, cudaStream_t stream,
+                               int *launches)
+{
+    const int64_t L = ops[0].cols, M = ops[2].cols;
+    if (L == 128 && M == 32) return run_hadamard<128, 32>(t, ops, out, ws, stream, launches);
+    if (L == 128 && M == 64) return run_hadamard<128, 64>(t, ops, out, ws, stream, launches);
+    if (L == 256 && M == 32) return run_hadamard<256, 32>(t, ops, out, ws, stream, launches);
+    if (L == 256 && M == 64) return run_hadamard<256, 64>(t, ops, out, ws, stream, launches);
     return SA_E_UNSUPPORTED;
 }

@@ -57,6 +57,7 @@ def test_empty_and_single_entry_all_chains(sa, nnz):
     w = _wl("spmm_gemm", "csr", (5, 4), c2, v, [_dense(1, 0, 4, 128), _dense(1, 1, 128, 32)], (5, 32))
     _check(sa, w, sched=sa.SA_SCHED_ASSOC_LEFT)
     _check(sa, w, sched=sa.SA_SCHED_ASSOC_RIGHT)
+    _check(sa, _wl("spmmh_gemm", "csr", (5, 4), c2, v, [_dense(1, 0, 4, 128), _dense(1, 3, 4, 128), _dense(1, 1, 128, 32)], (5, 32)))
 
 
 @pytest.mark.parametrize("L,M", [(16, 16), (16, 32), (32, 16), (32, 32)])
@@ -170,6 +171,10 @@ def test_spmm_gemm_rank_combinations_and_long_rows(sa, L, M):
             [configs.dense_normal(12, 0, J, L), configs.dense_normal(12, 1, L, M)], (I, M))
     _check(sa, w, sched=sa.SA_SCHED_ASSOC_LEFT)
     _check(sa, w, sched=sa.SA_SCHED_ASSOC_RIGHT)
+    # kernel 3 on the same tensor: empty rows, long rows cut into pieces, every rank combination
+    wh = _wl("spmmh_gemm", "csr", (I, J), coords, vals,
+             [w.dense[0], configs.dense_normal(12, 2, J, L), w.dense[1]], (I, M))
+    _check(sa, wh)
 
 
 def test_ttm4_ragged_and_split_slices(sa):

@@ -41,3 +41,10 @@ def test_spmm_gemm_mini_both_orders(sa, sched):
     s = {"left": sa.SA_SCHED_ASSOC_LEFT, "right": sa.SA_SCHED_ASSOC_RIGHT, "default": sa.SA_SCHED_DEFAULT}[sched]
     A, _ = run_gpu(sa, w, sched=s)
     assert_close(A, A_ref, S_ref, TOL_FP32, w.name + "/" + sched)
+
+
+def test_spmmh_gemm_mini(sa):
+    w = configs.make(8, "mini")
+    A_ref, S_ref = oracle.evaluate(w)
+    A, _ = run_gpu(sa, w)
+    assert_close(A, A_ref, S_ref, TOL_FP32, w.name)

@@ -324,3 +324,48 @@ def test_sddmm_spmm_gemm_bruteforce_and_relation_to_kernel_1():
     sel = np.array([4, 1])
     As, Ss = oracle.sddmm_spmm_gemm(coords, vals, dims, C, D, E, F, sel=sel)
     assert np.array_equal(As, A[sel]) and np.array_equal(Ss, S[sel])
+
+
+# ----------------------------------------------------------------- kernel 3 <SpMMH,GEMM>
+
+def test_spmmh_gemm_bruteforce_special_cases_and_invariants():
+    """A(i,m) = sum_{j,l} B(i,j) C(j,l) D(j,l) E(l,m) (Table of kernels, row 3, Description column)."""
+    rs = np.random.RandomState(21)
+    dims = (6, 5)
+    coords, vals = tiny_coo(rs, dims, 14)
+    C, D, E = dense(rs, 5, 4), dense(rs, 5, 4), dense(rs, 4, 3)
+    A, S = oracle.spmmh_gemm(coords, vals, dims, C, D, E)
+    B = densify(coords, vals, dims)
+    ref = np.zeros((6, 3))
+    for i, j, l, m in itertools.product(range(6), range(5), range(4), range(3)):
+        ref[i, m] += B[i, j] * float(C[j, l]) * float(D[j, l]) * float(E[l, m])
+    np.testing.assert_allclose(A, ref, rtol=0, atol=1e-13)
+    C64, D64, E64 = (x.astype(np.float64) for x in (C, D, E))
+    np.testing.assert_allclose(A, np.einsum("ij,jl,jl,lm->im", B, C64, D64, E64), rtol=0, atol=1e-13)
+    np.testing.assert_allclose(A, (B @ (C64 * D64)) @ E64, rtol=0, atol=1e-13)       # the two stages the name spells
+    np.testing.assert_allclose(S, np.abs(B) @ (np.abs(C64) * np.abs(D64)) @ np.abs(E64), rtol=0, atol=1e-13)
+    # D = all ones: kernel 4 with the same C and E
+    A4, S4 = oracle.spmm_gemm(coords, vals, dims, C, E)
+    A1, S1 = oracle.spmmh_gemm(coords, vals, dims, C, np.ones_like(C), E)
+    assert np.array_equal(A1, A4) and np.array_equal(S1, S4)
+    # E = identity: SpMM of B with the Hadamard product (library CSR product)
+    Ai, _ = oracle.spmmh_gemm(coords, vals, dims, C, D, np.eye(4, dtype=np.float32))
+    Bcsr = sp.csr_matrix((vals.astype(np.float64), (coords[:, 0], coords[:, 1])), shape=dims)
+    np.testing.assert_allclose(Ai, Bcsr @ (C64 * D64), rtol=0, atol=1e-13)
+    # the Hadamard factors commute; a transposed (wrongly indexed) D does not give the same result
+    A2, _ = oracle.spmmh_gemm(coords, vals, dims, D, C, E)
+    np.testing.assert_allclose(A2, A, rtol=0, atol=1e-13)
+    # all ones: A(i,m) = L * deg(i)
+    Ao, So = oracle.spmmh_gemm(coords, np.ones(14, np.float32), dims, np.ones((5, 4), np.float32), np.ones((5, 4), np.float32),
+                               np.ones((4, 3), np.float32))
+    deg = np.bincount(coords[:, 0], minlength=6)
+    assert np.array_equal(Ao, np.broadcast_to(4.0 * deg[:, None], (6, 3))) and np.array_equal(Ao, So)
+    # linearity in B, invariance under the COO order, subset mode
+    A3, _ = oracle.spmmh_gemm(coords, 4.0 * vals, dims, C, D, E)        # a power of two: exact in fp32
+    np.testing.assert_allclose(A3, 4.0 * A, rtol=0, atol=1e-12)
+    perm = rs.permutation(14)
+    Ap, _ = oracle.spmmh_gemm(coords[perm], vals[perm], dims, C, D, E)
+    np.testing.assert_allclose(Ap, A, rtol=0, atol=1e-13)
+    sel = np.array([4, 0, 5], dtype=np.int64)
+    As, Ss = oracle.spmmh_gemm(coords, vals, dims, C, D, E, sel=sel)
+    assert np.array_equal(As, A[sel]) and np.array_equal(Ss, S[sel])

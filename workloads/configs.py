@@ -35,7 +35,7 @@ S_STRUCT, S_VALS, S_DENSE, S_SHUFFLE = 0, 1, 2, 3
 @dataclass
 class Workload:
     name: str
-    expr: str                  # 'spttm_ttm3' | 'spttm_ttm4' | 'sddmm_spmm' | 'spmm_gemm' | 'ttmc3'
+    expr: str                  # 'spttm_ttm3' | 'spttm_ttm4' | 'sddmm_spmm' | 'spmm_gemm' | 'ttmc3' | 'sddmm_spmm_gemm' | 'spmmh_gemm'
     fmt: str                   # 'csf' | 'csr'
     dims: tuple                # dimensions of B
     coords: np.ndarray         # int32 [nnz, order], shuffled
@@ -391,4 +391,16 @@ def make(config, scale="full", seed=None):
         F = dense_normal(s, 3, 32, 32)
         return Workload("cfg7-sddmm-spmm-gemm-mini", "sddmm_spmm_gemm", "csr", w.dims, w.coords, w.vals, w.dense + [F],
                         (w.dims[0], 32), s, w.notes)
-    raise ValueError("config must be 1..7")
+    if config == 8:
+        # kernel 3 (SpMMH, GEMM): the tensor recipe of config 4 with a second J x L matrix for the Hadamard product
+        if full:
+            w = make_spmm_gemm("tmp", s, 4_000_000, 4_000_000, 100_000_000, 256, 64)
+        elif scale == "mid":
+            w = make_spmm_gemm("tmp", s, 1_000_000, 1_000_000, 25_000_000, 256, 64)
+        else:
+            w = make_spmm_gemm("tmp", s, 9_000, 9_000, 200_000, 128, 32)
+        C, E = w.dense
+        D = dense_normal(s, 2, C.shape[0], C.shape[1])
+        return Workload("cfg8-spmmh-gemm" + ("" if full else "-" + scale), "spmmh_gemm", "csr", w.dims, w.coords, w.vals,
+                        [C, D, E], w.out_shape, s, w.notes)
+    raise ValueError("config must be 1..8")
