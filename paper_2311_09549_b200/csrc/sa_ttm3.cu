@@ -64,10 +64,14 @@ __device__ __forceinline__ bool dbg_ok(const dbg_limits &lim, bool ok, int code,
 #define SA_CHK(lim, cond, code, value) true
 #endif
 
-constexpr int SA_TTM3_MINCTAS = 4;   // thread blocks per SM the register budget is set for (16 warps)
 
 template <int L, int M>
 struct cfg {
+    // Thread blocks per SM the register budget is set for: 4 (16 warps, 128 registers).  The 16 x 16 kernel also
+    // compiles without spills for 6 blocks (24 warps, 80 registers); that variant is slower on long units but
+    // faster when the units are short (many unit switches, whose latencies more warps hide): the launcher picks.
+    static constexpr int MINCTAS = 4;
+    static constexpr int MINCTAS_SHORT = (L == 16 && M == 16) ? 6 : 4;
     static constexpr int MT = L / 16;            // m16 tiles over l
     static constexpr int NT = M / 8;             // n8 tiles over m
     static constexpr int NS = SA_STREAMS;        // streams per warp
@@ -442,8 +446,8 @@ __device__ __forceinline__ void ttm3_warp_task(const sa_unit3 *__restrict__ unit
     __syncwarp();
 }
 
-template <int L, int M>
-__global__ void __launch_bounds__(32 * SA_TTM3_WARPS, SA_TTM3_MINCTAS)
+template <int L, int M, int NCTA>
+__global__ void __launch_bounds__(32 * SA_TTM3_WARPS, NCTA)
 ttm3_kernel(const sa_unit3 *__restrict__ units, const int32_t *__restrict__ task_start, int64_t n_tasks, int n_group_ctas,
             const int32_t *__restrict__ crd_j, const int32_t *__restrict__ crd_k, const float *__restrict__ vals,
             const uint32_t *__restrict__ endbits, const float *__restrict__ C, uint32_t ldc,
@@ -500,7 +504,8 @@ cudaError_t launch(const sa_ttm3_view &v, const sa_dense &first, const sa_dense 
     const int64_t ctas = (n_tasks + SA_TTM3_WARPS - 1) / SA_TTM3_WARPS;
     if (ctas <= 0) return cudaSuccess;
     constexpr size_t smem = size_t(SA_TTM3_WARPS) * cfg<L, M>::WARP_BYTES;
-    auto kern = ttm3_kernel<L, M>;
+    const bool short_units = v.nnz < int64_t(512) * int64_t(wl.items.size());          // mean unit below 512 nonzeros
+    auto kern = short_units ? ttm3_kernel<L, M, cfg<L, M>::MINCTAS_SHORT> : ttm3_kernel<L, M, cfg<L, M>::MINCTAS>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess)
         return cudaGetLastError();
     dbg_limits lim;
