@@ -231,6 +231,40 @@ def reduce_max_over_ranks(values, device, world):
     return [float(x) for x in t.cpu()]
 
 
+def l2_gather_ceiling(sa, torch, w, ops, dev, stream):
+    """For the TTM chains: time a bare gather of one factor row per nonzero (the rows the fiber stage reads, from
+    the same table, uniformly random row indices) with the library's probe kernel.  Returns a dict or None."""
+    which = {"spttm_ttm3": 1, "spttm_ttm4": 2, "ttmc3": 2}.get(w.expr)
+    if which is None:
+        return None
+    table = ops[which]
+    rows, cols = int(table.shape[0]), int(table.shape[1])
+    if cols not in (16, 32):
+        return None
+    n = int(w.nnz)
+    g = torch.Generator(device=dev)
+    g.manual_seed(12345)
+    idx = torch.randint(0, rows, (n,), dtype=torch.int32, device=dev, generator=g)
+    sink = torch.zeros(1, dtype=torch.float32, device=dev)
+    run = lambda: sa.sa_probe_row_gather(table.data_ptr(), rows, table.stride(0), cols, idx.data_ptr(), n, sink.data_ptr(),
+                                         stream.cuda_stream)
+    for _ in range(3):
+        run()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize(dev)
+    e0.record(stream)
+    reps = 10
+    for _ in range(reps):
+        run()
+    e1.record(stream)
+    torch.cuda.synchronize(dev)
+    ms = e0.elapsed_time(e1) / reps
+    nbytes = n * cols * 4
+    return {"what": "bare gather of one %d-byte factor row per nonzero from the L2-resident %d x %d table "
+                    "(uniform random rows; plus 4 index bytes per row from HBM)" % (cols * 4, rows, cols),
+            "ms": ms, "gbs": nbytes / (ms * 1e-3) / 1e9}
+
+
 def aggregate_throughput(nnz_per_rank, world, ms_per_step):
     """Whole-job GNNZ/s of ``world`` independent replicas that all finish within ms_per_step."""
     return world * nnz_per_rank / (ms_per_step * 1e-3) / 1e9
@@ -409,6 +443,9 @@ def main():
             "gpu_launches": launches_per_step * args.steps,
             "clocks": clocks,
         }
+        gather = l2_gather_ceiling(sa, torch, w, ops, dev, stream) if args.scale == "full" else None
+        if gather is not None:
+            line["l2_gather_ceiling"] = gather
         if not args.no_cpu_baseline and world == 1:
             cb = oracle_sample(w)
             cb.pop("seconds")

@@ -231,6 +231,20 @@ sa_status sa_run(const sa_tensor *B, sa_expr expr, sa_schedule sched, const sa_d
 sa_status sa_run_ttm3_static_scratch(const sa_tensor *B, const sa_dense *ops, int n_ops, float *out,
                                      void *cuda_stream);
 
+/*
+ * (Measurement aid; no counterpart in the paper.)  Gather n rows of a small dense table through L2 the way the
+ * fiber stage of the TTM chains does -- eight lanes per row, one vector load per lane, eight rows in flight per
+ * lane -- and do nothing else, asynchronously on cuda_stream.  Timing it gives the ceiling of that access
+ * pattern on the device: bytes gathered = (n rounded down to a multiple of 8 per lane group) * row_floats * 4.
+ *   table      DEVICE fp32 [rows x ld], row-major, 16-byte aligned, rows * ld < 2^30
+ *   row_floats 32 or 16 (floats read per row)
+ *   idx        DEVICE int32 [n], every entry in [0, rows); 16-byte aligned
+ *   sink       DEVICE fp32 [1]; keeps the loads from being optimised away, practically never written
+ * Errors: SA_E_ARG, SA_E_UNSUPPORTED, SA_E_CUDA.
+ */
+sa_status sa_probe_row_gather(const float *table, int64_t rows, int64_t ld, int row_floats, const int32_t *idx,
+                              int64_t n, float *sink, void *cuda_stream);
+
 /* Number of kernel launches the last successful sa_run on this handle enqueued. */
 sa_status sa_last_launch_count(const sa_tensor *t, int *launches);
 
