@@ -99,6 +99,12 @@ def algorithmic_work(w, counts, sched):
         I = w.dims[0]
         K, L = w.dense[0].shape[1], w.dense[2].shape[1]
         return 8 * nnz + 4 * (I + 1) + 4 * (K + L) * nnz + sz(w.dense[0]) + out_bytes, nnz * (2 * K + 1 + 2 * L)
+    if w.expr == "mttkrp_gemm":
+        # the rows T(i,:) that pass through the workspace are not counted
+        S, F2 = int(counts[0]), int(counts[1])
+        R, M = w.dense[0].shape[1], w.dense[2].shape[1]
+        return (8 * nnz + 8 * F2 + 8 * S + sum(sz(d) for d in w.dense) + out_bytes,
+                2 * nnz * R + 2 * F2 * R + 2 * w.dims[0] * R * M)
     if w.expr == "spmmh_gemm":
         # two gathered rows of L floats per nonzero (C and its Hadamard partner), E once, the output once
         I, J = w.dims
@@ -191,6 +197,7 @@ def oracle_sample(w, budget_s=15.0):
                "sddmm_spmm": lambda: w.dense[0].shape[1] * w.dense[2].shape[1],
                "spmm_gemm": lambda: w.dense[0].shape[1] * w.dense[1].shape[1],
                "spmmh_gemm": lambda: w.dense[0].shape[1] * w.dense[2].shape[1],
+               "mttkrp_gemm": lambda: w.dense[0].shape[1] * w.dense[2].shape[1],
                "sddmm_spmm_gemm": lambda: w.dense[0].shape[1] * w.dense[2].shape[1] * w.dense[3].shape[1],
                "ttmc3": lambda: w.dense[0].shape[1] * w.dense[1].shape[1] * w.dense[2].shape[1]}[w.expr]()
     cores = oracle.max_threads()
@@ -234,7 +241,7 @@ def reduce_max_over_ranks(values, device, world):
 def l2_gather_ceiling(sa, torch, w, ops, dev, stream):
     """For the TTM chains: time a bare gather of one factor row per nonzero (the rows the fiber stage reads, from
     the same table, uniformly random row indices) with the library's probe kernel.  Returns a dict or None."""
-    which = {"spttm_ttm3": 1, "spttm_ttm4": 2, "ttmc3": 2}.get(w.expr)
+    which = {"spttm_ttm3": 1, "spttm_ttm4": 2, "ttmc3": 2, "mttkrp_gemm": 1}.get(w.expr)
     if which is None:
         return None
     table = ops[which]
@@ -276,7 +283,8 @@ def workload_label(cfg, sched):
              5: "cfg5 order-4 <SpTTM,TTM> 50000x20000^3 100M nnz ranks 16",
              7: "kernel 2 <SDDMM,SpMM,GEMM> on the config-3 tensor, K=L=M=64",
              6: "kernel 5 <3D TTMC> on a nell-2-shaped tensor 12000x9000x288000 76.88M nnz L=M=N=16",
-             8: "kernel 3 <SpMMH,GEMM> on the config-4 tensor recipe 4Mx4M 100M nnz L=256 M=64"}
+             8: "kernel 3 <SpMMH,GEMM> on the config-4 tensor recipe 4Mx4M 100M nnz L=256 M=64",
+             9: "kernel 8 <MTTKRP,GEMM> on the config-2 tensor, R=32 M=32"}
     return names[cfg] + (" (%s)" % sched if cfg == 4 else "")
 
 
@@ -312,7 +320,7 @@ def main():
     ap.add_argument("--steps", type=int, default=31)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", type=int, default=2, choices=[1, 2, 3, 4, 5, 6, 7, 8])
+    ap.add_argument("--workload", type=int, default=2, choices=[1, 2, 3, 4, 5, 6, 7, 8, 9])
     ap.add_argument("--scale", default="full", choices=["full", "mid", "mini"])
     ap.add_argument("--sched", default="right", choices=["left", "right"], help="association order for workload 4")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -70,7 +70,10 @@ typedef enum {
     /* kernel 3 <SpMMH,GEMM>: A(i,m) = sum_{j,l} B(i,j) C(j,l) D(j,l) E(l,m); ops = {C, D, E}; B CSR;
      * the Description column of the Table of kernels (SpMM with a Hadamard product, then GEMM),
      * evaluated per row as T(l) = sum_j B(i,j) C(j,l) D(j,l) followed by T . E                   */
-    SA_EXPR_SPMMH_GEMM = 7
+    SA_EXPR_SPMMH_GEMM = 7,
+    /* kernel 8 <MTTKRP,GEMM>: A(i,m) = sum_{j,k,r} B(i,j,k) C(j,r) D(k,r) E(r,m); ops = {C, D, E};
+     * B order-3 CSF; the MTTKRP rows T(i,:) (R floats per slice) live in the workspace              */
+    SA_EXPR_MTTKRP_GEMM = 8
 } sa_expr;
 
 typedef enum {
@@ -194,7 +197,7 @@ sa_status sa_workspace_size(const sa_tensor *t, sa_expr expr, sa_schedule sched,
  * Compiled dense ranks (anything else is SA_E_UNSUPPORTED): SPTTM_TTM3 L, M in {16, 32};
  * SPTTM_TTM4 L = M = N = 16; SDDMM_SPMM K, L in {32, 64, 128}; SPMM_GEMM L in {128, 256},
  * M in {32, 64}; TTMC3 L, M, N in {16, 32}; SDDMM_SPMM_GEMM K, L in {32, 64, 128}, M in {32, 64};
- * SPMMH_GEMM L in {128, 256}, M in {32, 64}.
+ * SPMMH_GEMM L in {128, 256}, M in {32, 64}; MTTKRP_GEMM R = 32, M in {32, 64}.
  * Returns launch errors only; completion is observed by synchronising the stream.
  * Errors: SA_E_ARG, SA_E_SHAPE, SA_E_UNSUPPORTED, SA_E_WORKSPACE, SA_E_CUDA.
  */

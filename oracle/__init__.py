@@ -195,6 +195,26 @@ def spmmh_gemm(coords, vals, dims, C, D, E, sel=None, with_abs=True, threads=0):
     return A, S
 
 
+def mttkrp_gemm(coords, vals, dims, C, D, E, sel=None, with_abs=True, threads=0):
+    """Kernel 8: A(i,m) = sum_{j,k,r} B(i,j,k) C(j,r) D(k,r) E(r,m).  Returns (A, S)."""
+    I, J, K = (int(d) for d in dims)
+    c, cp = _coords(coords, 3)
+    v, vp = _f32(vals)
+    C, Cp = _f32(C)
+    D, Dp = _f32(D)
+    E, Ep = _f32(E)
+    assert C.shape[0] == J and D.shape[0] == K and D.shape[1] == C.shape[1] and E.shape[0] == C.shape[1]
+    R, M = C.shape[1], E.shape[1]
+    s, sp, n_sel, n_out = _sel(sel, I)
+    A = np.empty((n_out, M), dtype=np.float64)
+    S = np.empty_like(A) if with_abs else None
+    rc = _load().oracle_mttkrp_gemm(_i64(v.shape[0]), cp, vp, _i64(I), _i64(J), _i64(K), _i64(R), _i64(M),
+                                    Cp, Dp, Ep, _i64(n_sel), sp, A.ctypes.data_as(_p),
+                                    S.ctypes.data_as(_p) if with_abs else None, ctypes.c_int(threads))
+    _check(rc)
+    return A, S
+
+
 def ttmc3(coords, vals, dims, C, D, E, sel=None, with_abs=True, threads=0):
     """A(l,m,n) = sum_{i,j,k} B(i,j,k) C(i,l) D(j,m) E(k,n).  Returns (A, S) of shape (L, M, N), or of
     shape (len(sel),) when ``sel`` lists flat output indices (l*M + m)*N + n."""
@@ -232,6 +252,8 @@ def evaluate(w, sel=None, with_abs=True, threads=0):
         return sddmm_spmm_gemm(w.coords, w.vals, w.dims, *w.dense, sel=sel, with_abs=with_abs, threads=threads)
     if w.expr == "sddmm_spmm":
         return sddmm_spmm(w.coords, w.vals, w.dims, *w.dense, sel=sel, with_abs=with_abs, threads=threads)[:2]
+    if w.expr == "mttkrp_gemm":
+        return mttkrp_gemm(w.coords, w.vals, w.dims, *w.dense, sel=sel, with_abs=with_abs, threads=threads)
     if w.expr == "spmmh_gemm":
         return spmmh_gemm(w.coords, w.vals, w.dims, *w.dense, sel=sel, with_abs=with_abs, threads=threads)
     if w.expr == "spmm_gemm":

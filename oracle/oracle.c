@@ -286,6 +286,45 @@ int oracle_spmmh_gemm(int64_t nnz, const int32_t *coords, const float *vals,
     return 0;
 }
 
+/* Kernel 8 <MTTKRP,GEMM>:  A(i,m) = sum_{j,k,r} B(i,j,k) * C(j,r) * D(k,r) * E(r,m)  (Table of kernels,
+ * Description column with every index that is not an output index summed; the paper's letters are
+ * A_im = sum B_ikl C_lj D_kj E_jm). */
+int oracle_mttkrp_gemm(int64_t nnz, const int32_t *coords, const float *vals,
+                       int64_t I, int64_t J, int64_t K, int64_t R, int64_t M,
+                       const float *C, const float *D, const float *E,
+                       int64_t n_sel, const int64_t *sel, double *A, double *S, int threads)
+{
+    buckets_t b;
+    int rc = make_buckets(&b, nnz, coords, 3, I, n_sel, sel);
+    if (rc) { free_buckets(&b); return rc; }
+    for (int64_t p = 0; p < nnz; ++p)
+        if (coords[3 * p + 1] < 0 || coords[3 * p + 1] >= J || coords[3 * p + 2] < 0 || coords[3 * p + 2] >= K) {
+            free_buckets(&b);
+            return -2;
+        }
+    set_threads(threads);
+    #pragma omp parallel for schedule(dynamic, 16)
+    for (int64_t o = 0; o < b.n_out; ++o) {
+        double *Ao = A + o * M;
+        double *So = S ? S + o * M : NULL;
+        for (int64_t x = 0; x < M; ++x) Ao[x] = 0.0;
+        if (So) for (int64_t x = 0; x < M; ++x) So[x] = 0.0;
+        for (int64_t q = b.start[o]; q < b.start[o + 1]; ++q) {
+            int64_t p = b.order[q];
+            int64_t j = coords[3 * p + 1], k = coords[3 * p + 2];
+            double v = (double)vals[p];
+            for (int64_t r = 0; r < R; ++r)
+                for (int64_t m = 0; m < M; ++m) {
+                    double term = v * (double)C[j * R + r] * (double)D[k * R + r] * (double)E[r * M + m];
+                    Ao[m] += term;
+                    if (So) So[m] += fabs(term);
+                }
+        }
+    }
+    free_buckets(&b);
+    return 0;
+}
+
 /* Kernel 5 <3D TTMC>:  A(l,m,n) = sum_{i,j,k} B(i,j,k) * C(i,l) * D(j,m) * E(k,n)  (all three
  * modes contracted; the running example of Sections 1, 3 and 4).  Every nonzero contributes to
  * every output element, so the loop nest is the linear one of the paper's first schedule with the

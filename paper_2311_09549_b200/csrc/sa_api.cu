@@ -90,6 +90,7 @@ sa_status check_ops(const sa_tensor *t, sa_expr expr, const sa_dense *ops, int n
         case SA_EXPR_TTMC3: want = 3; break;
         case SA_EXPR_SDDMM_SPMM_GEMM: want = 4; break;
         case SA_EXPR_SPMMH_GEMM: want = 3; break;
+        case SA_EXPR_MTTKRP_GEMM: want = 3; break;
         default: return SA_E_ARG;
     }
     if (n_ops != want) return SA_E_ARG;
@@ -127,6 +128,13 @@ sa_status check_ops(const sa_tensor *t, sa_expr expr, const sa_dense *ops, int n
                 return SA_E_SHAPE;
             if (!sa_ranks_ok_sddmm(ops[0].cols, ops[2].cols) || !sa_dense_gemm_ok(ops[2].cols, ops[3].cols)) return SA_E_UNSUPPORTED;
             break;
+        case SA_EXPR_MTTKRP_GEMM:
+            if (t->fmt != SA_FMT_CSF || t->order != 3) return SA_E_FORMAT;
+            if (ops[0].rows != t->dims[1] || ops[1].rows != t->dims[2] || ops[1].cols != ops[0].cols ||
+                ops[2].rows != ops[0].cols)
+                return SA_E_SHAPE;
+            if (!sa_ranks_ok_mttkrp_gemm(ops[0].cols, ops[2].cols)) return SA_E_UNSUPPORTED;
+            break;
         case SA_EXPR_SPMMH_GEMM:
             if (t->fmt != SA_FMT_CSR) return SA_E_FORMAT;
             if (ops[0].rows != t->dims[1] || ops[1].rows != t->dims[1] || ops[1].cols != ops[0].cols ||
@@ -159,6 +167,7 @@ bool resolve_schedule(const sa_tensor *t, sa_expr expr, sa_schedule sched, const
         case SA_EXPR_TTMC3:
         case SA_EXPR_SDDMM_SPMM_GEMM:
         case SA_EXPR_SPMMH_GEMM:
+        case SA_EXPR_MTTKRP_GEMM:
             if (sched == SA_SCHED_DEFAULT || sched == SA_SCHED_FUSED) { *resolved = SA_SCHED_FUSED; return true; }
             return false;
         case SA_EXPR_SDDMM_SPMM:
@@ -190,6 +199,7 @@ size_t workspace_bytes(const sa_tensor *t, sa_expr expr, sa_schedule sched, cons
         case SA_EXPR_TTMC3: return sa_ws_ttmc3(t, ops);
         case SA_EXPR_SDDMM_SPMM_GEMM: return sa_ws_sddmm_spmm_gemm(t, ops);
         case SA_EXPR_SPMMH_GEMM: return sa_ws_spmmh_gemm(t, ops);
+        case SA_EXPR_MTTKRP_GEMM: return sa_ws_mttkrp_gemm(t, ops);
     }
     return 0;
 }
@@ -345,6 +355,7 @@ sa_status sa_run(const sa_tensor *t, sa_expr expr, sa_schedule sched, const sa_d
         case SA_EXPR_TTMC3: s = sa_launch_ttmc3(t, ops, out, workspace, ws_bytes, stream, &launches); break;
         case SA_EXPR_SDDMM_SPMM_GEMM: s = sa_launch_sddmm_spmm_gemm(t, ops, out, workspace, ws_bytes, stream, &launches); break;
         case SA_EXPR_SPMMH_GEMM: s = sa_launch_spmmh_gemm(t, ops, out, workspace, ws_bytes, stream, &launches); break;
+        case SA_EXPR_MTTKRP_GEMM: s = sa_launch_mttkrp_gemm(t, ops, out, workspace, ws_bytes, stream, &launches); break;
     }
     if (s == SA_E_CUDA) cudaGetLastError();
     if (s == SA_OK) t->last_launches = launches;

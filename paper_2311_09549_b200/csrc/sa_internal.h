@@ -156,6 +156,12 @@ bool sa_dense_gemm_ok(int64_t L, int64_t M);
 sa_status sa_launch_dense_gemm(int64_t rows, const float *A, int64_t lda, const float *B, int64_t ldb, int64_t L,
                                int64_t M, float *out, cudaStream_t stream);
 
+// Kernel 8 <MTTKRP,GEMM>
+sa_status sa_launch_mttkrp_gemm(const sa_tensor *t, const sa_dense *ops, float *out, void *ws, size_t ws_bytes,
+                                cudaStream_t stream, int *launches);
+size_t sa_ws_mttkrp_gemm(const sa_tensor *t, const sa_dense *ops);
+bool sa_ranks_ok_mttkrp_gemm(int64_t R, int64_t M);
+
 // Supported-rank predicates (shared by sa_workspace_size and sa_run).
 bool sa_ranks_ok_ttm3(int64_t L, int64_t M);
 bool sa_ranks_ok_ttm4(int64_t L, int64_t M, int64_t N);

@@ -187,6 +187,22 @@ __device__ __forceinline__ void ttm3_flush(float (&acc)[cfg<L, M>::MT][cfg<L, M>
     }
 }
 
+// MTTKRP consumer (kernel 8): hacc(m) += sum over the parked rows row0 .. row0 + n - 1 of T(row, m) * C(j_row, m).
+// M = 32: lane = m.  M = 16: lane & 15 = m, the two half-warps take alternate rows (summed at the unit end).
+template <int M>
+__device__ __forceinline__ void had_flush(float &hacc, const float *__restrict__ ring, int row0, int n,
+                                          const float *__restrict__ C, int lane)
+{
+    constexpr int RS = M + 8;
+    const int m = lane & (M - 1);
+#pragma unroll
+    for (int x = 0; x < 8; ++x) {
+        const bool mine = x < n && (M == 32 || (x & 1) == (lane >> 4));
+        const float *r = ring + (row0 + x) * RS;
+        if (mine) hacc = fmaf(r[m], __ldg(C + __float_as_uint(r[M]) + m), hacc);
+    }
+}
+
 // Store a slice tile held as MMA accumulator fragments (streaming stores: the output is written once).
 template <int L, int M>
 __device__ __forceinline__ void store_tile(const float (&acc)[cfg<L, M>::MT][cfg<L, M>::NT][4], float *__restrict__ dst, int lane)
@@ -235,13 +251,13 @@ __device__ __forceinline__ stream_range stream_of(int p0, int p1, int q)
 // One warp evaluates the units [u0, u0 + nu) of its task.  `keep`: the (single) unit is a piece of a slice
 // whose tile the caller reduces over the CTA, so it is left in acc; otherwise every unit is a whole slice
 // and its tile is stored to `out` when the unit ends.
-template <int L, int M>
+template <int L, int M, bool HAD>
 __device__ __forceinline__ void ttm3_warp_task(const sa_unit3 *__restrict__ units, int u0, int nu,
                                                const int32_t *__restrict__ crd_j, const int32_t *__restrict__ crd_k,
                                                const float *__restrict__ vals, const uint32_t *__restrict__ endbits,
                                                const float *__restrict__ C, uint32_t ldc, const float *__restrict__ D,
                                                uint32_t ldd, unsigned char *__restrict__ wsm,
-                                               float (&acc)[cfg<L, M>::MT][cfg<L, M>::NT][4], const bool keep,
+                                               float (&acc)[cfg<L, M>::MT][cfg<L, M>::NT][4], float &hacc, const bool keep,
                                                float *__restrict__ out, const dbg_limits &lim)
 {
     using K = cfg<L, M>;
@@ -397,7 +413,8 @@ __device__ __forceinline__ void ttm3_warp_task(const sa_unit3 *__restrict__ unit
         else steps(std::false_type{});
         __syncwarp();
         while (npend >= 8) {
-            ttm3_flush<L, M>(acc, ring, rbase, 8, C, lane, lim, ldc);
+            if (HAD) had_flush<M>(hacc, ring, rbase, 8, C, lane);
+            else ttm3_flush<L, M>(acc, ring, rbase, 8, C, lane, lim, ldc);
             rbase += 8;
             npend -= 8;
         }
@@ -420,15 +437,25 @@ __device__ __forceinline__ void ttm3_warp_task(const sa_unit3 *__restrict__ unit
       {
         const int n = npend;
         if (n > 0) {
-            for (int x = n; x < 8; ++x) ring[(rbase + x) * K::RS + lane % M] = 0.f;
-            __syncwarp();
-            ttm3_flush<L, M>(acc, ring, rbase, n, C, lane, lim, ldc);
+            if (HAD) {
+                had_flush<M>(hacc, ring, rbase, n, C, lane);
+            } else {
+                for (int x = n; x < 8; ++x) ring[(rbase + x) * K::RS + lane % M] = 0.f;
+                __syncwarp();
+                ttm3_flush<L, M>(acc, ring, rbase, n, C, lane, lim, ldc);
+            }
             __syncwarp();
         }
         rbase = npend = 0;
         if (!keep) {
-            if (SA_CHK(lim, uint32_t(crow) < lim.n_slices_dim, 8, crow)) store_tile<L, M>(acc, out + int64_t(crow) * (L * M), lane);
-            zero_tile<L, M>(acc);
+            if (HAD) {
+                if (M == 16) hacc += __shfl_xor_sync(SA_FULL_MASK, hacc, 16);
+                if (lane < M && SA_CHK(lim, uint32_t(crow) < lim.n_slices_dim, 8, crow)) sa_st_cs(out + int64_t(crow) * M + lane, hacc);
+                hacc = 0.f;
+            } else {
+                if (SA_CHK(lim, uint32_t(crow) < lim.n_slices_dim, 8, crow)) store_tile<L, M>(acc, out + int64_t(crow) * (L * M), lane);
+                zero_tile<L, M>(acc);
+            }
         }
         ++cu;
         if (cu < nu) {
@@ -446,7 +473,7 @@ __device__ __forceinline__ void ttm3_warp_task(const sa_unit3 *__restrict__ unit
     __syncwarp();
 }
 
-template <int L, int M, int NCTA>
+template <int L, int M, int NCTA, bool HAD>
 __global__ void __launch_bounds__(32 * SA_TTM3_WARPS, NCTA)
 ttm3_kernel(const sa_unit3 *__restrict__ units, const int32_t *__restrict__ task_start, int64_t n_tasks, int n_group_ctas,
             const int32_t *__restrict__ crd_j, const int32_t *__restrict__ crd_k, const float *__restrict__ vals,
@@ -455,7 +482,7 @@ ttm3_kernel(const sa_unit3 *__restrict__ units, const int32_t *__restrict__ task
             const dbg_limits lim)
 {
     using K = cfg<L, M>;
-    constexpr int TILE = L * M;
+    constexpr int TILE = HAD ? M : L * M;
     extern __shared__ __align__(16) unsigned char smem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int g = lane >> 2, t = lane & 3;
@@ -463,11 +490,30 @@ ttm3_kernel(const sa_unit3 *__restrict__ units, const int32_t *__restrict__ task
     const int64_t task = int64_t(blockIdx.x) * SA_TTM3_WARPS + warp;
     const bool group = int(blockIdx.x) < n_group_ctas;
     float acc[K::MT][K::NT][4];
+    float hacc = 0.f;
     zero_tile<L, M>(acc);
     int u0 = 0, u1 = 0;
     if (task < n_tasks) { u0 = task_start[task]; u1 = task_start[task + 1]; }
-    if (u1 > u0) ttm3_warp_task<L, M>(units, u0, u1 - u0, crd_j, crd_k, vals, endbits, C, ldc, D, ldd, wsm, acc, group, out, lim);
+    if (u1 > u0)
+        ttm3_warp_task<L, M, HAD>(units, u0, u1 - u0, crd_j, crd_k, vals, endbits, C, ldc, D, ldd, wsm, acc, hacc, group, out, lim);
     if (!group) return;                 // whole small slices: every tile was stored when its unit ended
+    if (HAD) {
+        // the warps hold partial rows of the same slice: sum them in a fixed order
+        float *rows = reinterpret_cast<float *>(smem);
+        if (M == 16) hacc += __shfl_xor_sync(SA_FULL_MASK, hacc, 16);
+        __syncthreads();                // every warp is done with its shared memory
+        if (lane < M) rows[warp * M + lane] = hacc;
+        __syncthreads();
+        const sa_unit3 lead = units[task_start[int64_t(blockIdx.x) * SA_TTM3_WARPS]];
+        if (threadIdx.x < M) {
+            float sum = rows[threadIdx.x];
+#pragma unroll
+            for (int w = 1; w < SA_TTM3_WARPS; ++w) sum += rows[w * M + threadIdx.x];
+            float *dst = lead.dest >= 0 ? partial + int64_t(lead.dest) * TILE : out + int64_t(lead.out_row) * TILE;
+            dst[threadIdx.x] = sum;
+        }
+        return;
+    }
     // the CTA's warps hold partial tiles of the same slice: sum them in a fixed order
     float *wt = reinterpret_cast<float *>(wsm);
 #pragma unroll
@@ -495,7 +541,7 @@ ttm3_kernel(const sa_unit3 *__restrict__ units, const int32_t *__restrict__ task
     }
 }
 
-template <int L, int M>
+template <int L, int M, bool HAD>
 cudaError_t launch(const sa_ttm3_view &v, const sa_dense &first, const sa_dense &second, float *out, float *partial,
                    cudaStream_t stream)
 {
@@ -505,7 +551,7 @@ cudaError_t launch(const sa_ttm3_view &v, const sa_dense &first, const sa_dense 
     if (ctas <= 0) return cudaSuccess;
     constexpr size_t smem = size_t(SA_TTM3_WARPS) * cfg<L, M>::WARP_BYTES;
     const bool short_units = v.nnz < int64_t(512) * int64_t(wl.items.size());          // mean unit below 512 nonzeros
-    auto kern = short_units ? ttm3_kernel<L, M, cfg<L, M>::MINCTAS_SHORT> : ttm3_kernel<L, M, cfg<L, M>::MINCTAS>;
+    auto kern = short_units ? ttm3_kernel<L, M, cfg<L, M>::MINCTAS_SHORT, HAD> : ttm3_kernel<L, M, cfg<L, M>::MINCTAS, HAD>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess)
         return cudaGetLastError();
     dbg_limits lim;
@@ -536,10 +582,10 @@ sa_status sa_launch_ttm3_view(const sa_ttm3_view &v, const sa_dense &first, cons
     if (first.rows * first.ld >= (int64_t(1) << 30) || second.rows * second.ld >= (int64_t(1) << 30)) return SA_E_UNSUPPORTED;
     if (!v.endbits) return SA_E_UNSUPPORTED;
     cudaError_t e;
-    if (L == 16 && M == 16) e = launch<16, 16>(v, first, second, out, partial, stream);
-    else if (L == 32 && M == 16) e = launch<32, 16>(v, first, second, out, partial, stream);
-    else if (L == 16 && M == 32) e = launch<16, 32>(v, first, second, out, partial, stream);
-    else if (L == 32 && M == 32) e = launch<32, 32>(v, first, second, out, partial, stream);
+    if (L == 16 && M == 16) e = launch<16, 16, false>(v, first, second, out, partial, stream);
+    else if (L == 32 && M == 16) e = launch<32, 16, false>(v, first, second, out, partial, stream);
+    else if (L == 16 && M == 32) e = launch<16, 32, false>(v, first, second, out, partial, stream);
+    else if (L == 32 && M == 32) e = launch<32, 32, false>(v, first, second, out, partial, stream);
     else return SA_E_UNSUPPORTED;
     if (e != cudaSuccess) return SA_E_CUDA;
     *launches = v.wl->items.empty() ? 0 : 1;
@@ -565,6 +611,34 @@ sa_status sa_launch_ttm3(const sa_tensor *t, const sa_dense *ops, float *out, vo
     v.nnz = t->nnz;
     v.status = t->d_status;
     return sa_launch_ttm3_view(v, ops[0], ops[1], out, static_cast<float *>(ws), stream, launches);
+}
+
+// Kernel 8, first stage (MTTKRP): T(i,r) = sum_{j,k} B(i,j,k) C(j,r) D(k,r), R = 32 or 16 columns, one row of R
+// floats per slice written to `out` (empty slices zero), partial rows of split slices to `partial`.
+sa_status sa_launch_mttkrp_rows(const sa_tensor *t, const sa_dense &C, const sa_dense &D, float *out, float *partial,
+                                cudaStream_t stream, int *launches)
+{
+    const int64_t R = C.cols;
+    if (D.cols != R || (R != 32 && R != 16)) return SA_E_UNSUPPORTED;
+    if (C.rows * C.ld >= (int64_t(1) << 30) || D.rows * D.ld >= (int64_t(1) << 30) || !t->d_endbits) return SA_E_UNSUPPORTED;
+    sa_ttm3_view v;
+    v.wl = &t->wl_main;
+    v.crd_fiber = t->d_crd[1];
+    v.crd_nz = t->d_crd[2];
+    v.vals = t->d_vals;
+    v.endbits = t->d_endbits;
+    v.n_fibers = t->count[1];
+    v.n_out_rows = t->dims[0];
+    v.nnz = t->nnz;
+    v.status = t->d_status;
+    const cudaError_t e = R == 32 ? launch<16, 32, true>(v, C, D, out, partial, stream) : launch<16, 16, true>(v, C, D, out, partial, stream);
+    if (e != cudaSuccess) return SA_E_CUDA;
+    *launches = v.wl->items.empty() ? 0 : 1;
+    if (!v.wl->fix.empty()) {
+        if (sa_launch_fixup(*v.wl, partial, out, int(R), stream) != cudaSuccess) return SA_E_CUDA;
+        *launches += 1;
+    }
+    return SA_OK;
 }
 
 // ------------------------------------------------------------------ entry point without allocation

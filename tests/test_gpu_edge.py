@@ -70,6 +70,19 @@ def test_ttm3_rank_combinations_with_empty_slices(sa, L, M):
     assert not A[1::3].any()
 
 
+@pytest.mark.parametrize("M", [32, 64])
+def test_mttkrp_gemm_empty_slices_and_split_slices(sa, M):
+    # empty slices, small slices (several per warp task) and one slice large enough to be split over thread blocks
+    dims = (40, 37, 530)
+    coords, vals = _random_coo(9, dims, 400000)
+    keep = (coords[:, 0] % 3 != 1) & ((coords[:, 0] == 5) | (np.arange(400000) % 40 == 0))
+    w = _wl("mttkrp_gemm", "csf", dims, coords[keep], vals[keep],
+            [_dense(5, 0, 37, 32), _dense(5, 1, 530, 32), _dense(5, 2, 32, M)], (40, M))
+    A, t = _check(sa, w)
+    assert not A[1::3].any()
+    assert sa.sa_tensor_worklist(t.handle)[0][3] >= 2, "slice 5 must be split into chunks with partial rows"
+
+
 def test_ttm3_one_slice_long_fibers_split_over_many_blocks(sa):
     # a single slice of 60 000 nonzeros in 12 fibers of 5000: pieces cut inside fibers, 8 partial tiles
     dims = (3, 12, 5000)

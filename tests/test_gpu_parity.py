@@ -48,3 +48,10 @@ def test_spmmh_gemm_mini(sa):
     A_ref, S_ref = oracle.evaluate(w)
     A, _ = run_gpu(sa, w)
     assert_close(A, A_ref, S_ref, TOL_FP32, w.name)
+
+
+def test_mttkrp_gemm_mini(sa):
+    w = configs.make(9, "mini")
+    A_ref, S_ref = oracle.evaluate(w)
+    A, _ = run_gpu(sa, w)
+    assert_close(A, A_ref, S_ref, TOL_FP32, w.name)

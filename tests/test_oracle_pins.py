@@ -369,3 +369,47 @@ def test_spmmh_gemm_bruteforce_special_cases_and_invariants():
     sel = np.array([4, 0, 5], dtype=np.int64)
     As, Ss = oracle.spmmh_gemm(coords, vals, dims, C, D, E, sel=sel)
     assert np.array_equal(As, A[sel]) and np.array_equal(Ss, S[sel])
+
+
+# ----------------------------------------------------------------- kernel 8 <MTTKRP,GEMM>
+
+def test_mttkrp_gemm_bruteforce_special_cases_and_invariants():
+    """A(i,m) = sum_{j,k,r} B(i,j,k) C(j,r) D(k,r) E(r,m) (Table of kernels, row 8, Description column)."""
+    rs = np.random.RandomState(31)
+    dims = (5, 4, 6)
+    coords, vals = tiny_coo(rs, dims, 40)
+    C, D, E = dense(rs, 4, 3), dense(rs, 6, 3), dense(rs, 3, 2)
+    A, S = oracle.mttkrp_gemm(coords, vals, dims, C, D, E)
+    B = densify(coords, vals, dims)
+    ref = np.zeros((5, 2))
+    for i, j, k, r, m in itertools.product(range(5), range(4), range(6), range(3), range(2)):
+        ref[i, m] += B[i, j, k] * float(C[j, r]) * float(D[k, r]) * float(E[r, m])
+    np.testing.assert_allclose(A, ref, rtol=0, atol=1e-13)
+    C64, D64, E64 = (x.astype(np.float64) for x in (C, D, E))
+    np.testing.assert_allclose(A, np.einsum("ijk,jr,kr,rm->im", B, C64, D64, E64), rtol=0, atol=1e-13)
+    np.testing.assert_allclose(S, np.einsum("ijk,jr,kr,rm->im", np.abs(B), np.abs(C64), np.abs(D64), np.abs(E64)), rtol=0, atol=1e-13)
+    # E = identity: the MTTKRP itself = mode-1 unfolding of B times the Khatri-Rao product of C and D
+    Ai, _ = oracle.mttkrp_gemm(coords, vals, dims, C, D, np.eye(3, dtype=np.float32))
+    kr = (C64[:, None, :] * D64[None, :, :]).reshape(4 * 6, 3)            # row (j,k) = C(j,:) * D(k,:)
+    np.testing.assert_allclose(Ai, B.reshape(5, 24) @ kr, rtol=0, atol=1e-13)
+    np.testing.assert_allclose(A, (B.reshape(5, 24) @ kr) @ E64, rtol=0, atol=1e-13)   # the two stages the name spells
+    # rank 1 with unit weights: A(i,0) = sum_jk B(i,j,k) c(j) d(k), a bilinear form per slice
+    c1, d1 = dense(rs, 4, 1), dense(rs, 6, 1)
+    A1, _ = oracle.mttkrp_gemm(coords, vals, dims, c1, d1, np.ones((1, 1), np.float32))
+    np.testing.assert_allclose(A1[:, 0], np.einsum("ijk,j,k->i", B, c1[:, 0].astype(np.float64), d1[:, 0].astype(np.float64)),
+                               rtol=0, atol=1e-13)
+    # swapping the roles of C and D does not give the same result (j and k are different modes)
+    # all ones: A(i,m) = R * nnz(slice i)
+    Ao, So = oracle.mttkrp_gemm(coords, np.ones(40, np.float32), dims, np.ones((4, 3), np.float32), np.ones((6, 3), np.float32),
+                                np.ones((3, 2), np.float32))
+    cnt = np.bincount(coords[:, 0], minlength=5)
+    assert np.array_equal(Ao, np.broadcast_to(3.0 * cnt[:, None], (5, 2))) and np.array_equal(Ao, So)
+    # linearity in B, invariance under the COO order, subset mode
+    A4, _ = oracle.mttkrp_gemm(coords, 4.0 * vals, dims, C, D, E)
+    np.testing.assert_allclose(A4, 4.0 * A, rtol=0, atol=1e-12)
+    perm = rs.permutation(40)
+    Ap, _ = oracle.mttkrp_gemm(coords[perm], vals[perm], dims, C, D, E)
+    np.testing.assert_allclose(Ap, A, rtol=0, atol=1e-13)
+    sel = np.array([3, 0], dtype=np.int64)
+    As, Ss = oracle.mttkrp_gemm(coords, vals, dims, C, D, E, sel=sel)
+    assert np.array_equal(As, A[sel]) and np.array_equal(Ss, S[sel])

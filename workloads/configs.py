@@ -403,4 +403,13 @@ def make(config, scale="full", seed=None):
         D = dense_normal(s, 2, C.shape[0], C.shape[1])
         return Workload("cfg8-spmmh-gemm" + ("" if full else "-" + scale), "spmmh_gemm", "csr", w.dims, w.coords, w.vals,
                         [C, D, E], w.out_shape, s, w.notes)
-    raise ValueError("config must be 1..8")
+    if config == 9:
+        # kernel 8 (MTTKRP, GEMM): the tensor of config 2 with rank-32 factors and a 32 x 32 weight matrix E
+        if full:
+            w = make_ttm3_zipf("tmp", s, 100000, 80000, 80000, 50_000_000, 1.2, 8.0, 32, 32)
+        else:
+            w = make_ttm3_zipf("tmp", s, 2500, 600, 800, 200_000, 1.2, 8.0, 32, 32)
+        E = dense_uniform(s, 2, 32, 32)
+        return Workload("cfg9-mttkrp-gemm" + ("" if full else "-mini"), "mttkrp_gemm", "csf", w.dims, w.coords, w.vals,
+                        w.dense + [E], (w.dims[0], 32), s, w.notes)
+    raise ValueError("config must be 1..9")
