@@ -115,12 +115,9 @@ spmm_gemm_left_kernel(const sa_item *__restrict__ items, int64_t n_items, const 
 // 32 x M/2.  D stays in shared memory for the whole (persistent) block, already split into its
 // TF32 high and low parts; C streams through a 3-stage cp.async ring in chunks of 32 columns.
 // NPROD = 3: hi*hi + lo*hi + hi*lo (fp32-level accuracy); NPROD = 1: a single TF32 product.
-__device__ __forceinline__ uint32_t g_tf32(float x)
-{
-    uint32_t r;
-    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
-    return r;
-}
+// The upper 19 bits of x: a TF32 number.  x - hi is exact in fp32, so hi.hi + hi.lo + lo.hi misses the product by
+// about 2^-20 relative.  (cvt.rna.tf32 costs about five instructions per value on this target, masking one.)
+__device__ __forceinline__ uint32_t g_tf32(float x) { return __float_as_uint(x) & 0xffffe000u; }
 __device__ __forceinline__ void g_mma(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
 {
     asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
