@@ -129,3 +129,27 @@ def test_cfg7_sddmm_spmm_gemm_full_sampled(sa):
     _compare(out, w, sel, w.name)
     del out, t
     torch.cuda.empty_cache()
+
+
+def test_cfg8_spmmh_gemm_mid_sampled(sa):
+    """Kernel 3 at a quarter of the benchmark size (the full size holds two 4 GB matrices on the host)."""
+    import torch
+    w = configs.make(8, "mid")
+    out, t = _run_full(sa, w)
+    sel = _sample(w, 10_000, 3000)
+    _compare(out, w, sel, w.name)
+    del out, t
+    torch.cuda.empty_cache()
+
+
+def test_cfg9_mttkrp_gemm_full_sampled(sa):
+    import torch
+    w = configs.make(9, "full")
+    out, t = _run_full(sa, w)
+    sel = _sample(w, 3_000_000, 300)                  # includes a slice split over many thread blocks
+    _compare(out, w, sel, w.name)
+    counts = np.bincount(w.coords[:, 0], minlength=w.dims[0])
+    empty = torch.from_numpy(np.nonzero(counts == 0)[0]).cuda()
+    assert not bool(out[empty].any()), "empty slices must be +0"
+    del out, t
+    torch.cuda.empty_cache()
