@@ -9,6 +9,8 @@
 //   the paper's Stage-1 pruning still admits), then the SpMM loop nest of Fig. 1b, A = B.E.
 #include "sa_device.cuh"
 
+constexpr int LEFT_UNROLL = 4;     // gathered rows in flight per warp in the (B.C).D row kernel (8 was slower)
+
 namespace {
 
 #ifndef SA_GEMM_NPROD
@@ -47,7 +49,7 @@ __device__ __forceinline__ void load_D(float *Ds, const float *__restrict__ D, i
 }
 
 template <int L, int M, bool HAD>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 3)
 spmm_gemm_left_kernel(const sa_item *__restrict__ items, int64_t n_items, const int32_t *__restrict__ pos,
                       const int32_t *__restrict__ crd, const float *__restrict__ vals, const float *__restrict__ C,
                       int64_t ldc, const float *__restrict__ H, int64_t ldh, const float *__restrict__ D, int64_t ldd,
@@ -74,7 +76,7 @@ spmm_gemm_left_kernel(const sa_item *__restrict__ items, int64_t n_items, const 
                 int jj = 0;
                 float vv = 0.f;
                 if (lane < n) { jj = crd[base + lane]; vv = vals[base + lane]; }
-#pragma unroll 4
+#pragma unroll LEFT_UNROLL
                 for (int s = 0; s < n; ++s) {
                     const int j = __shfl_sync(SA_FULL_MASK, jj, s);
                     const float v = __shfl_sync(SA_FULL_MASK, vv, s);
