@@ -4,7 +4,7 @@
 //   i < T(r) ;  j' < t(r) ; k': t(r) += B(i,j,k) D(k,r) ,  r: T(r) += t(r) C(j,r) > ,  m,r: A(i,m) += T(r) E(r,m) >
 // The inner pair is the fiber stage of kernel 6 with an element-wise consumer instead of the outer product
 // (sa_ttm3.cu, template flag HAD); the rows T(i,:) pass through the workspace and the dense stage is the
-// TF32x3 GEMM shared with kernels 2 and 4.
+// BF16x3 tensor-core GEMM shared with kernels 2 and 4.
 #include "sa_device.cuh"
 
 sa_status sa_launch_mttkrp_rows(const sa_tensor *t, const sa_dense &C, const sa_dense &D, float *out, float *partial,

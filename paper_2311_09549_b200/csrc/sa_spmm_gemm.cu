@@ -13,9 +13,6 @@ constexpr int LEFT_UNROLL = 4;     // gathered rows in flight per warp in the (B
 
 namespace {
 
-#ifndef SA_GEMM_NPROD
-#define SA_GEMM_NPROD 3
-#endif
 
 // Row (L floats in shared memory) times D (L x M in shared memory); lane owns m = lane + 32*q.
 template <int L, int M>
@@ -115,59 +112,72 @@ spmm_gemm_left_kernel(const sa_item *__restrict__ items, int64_t n_items, const 
 // ---- E = C . D on tensor cores (dense stage of ASSOC_RIGHT) -----------------------------------
 // Thread block: 128 rows of C x all M columns, 8 warps as 4 (rows) x 2 (columns), warp tile
 // 32 x M/2.  D stays in shared memory for the whole (persistent) block, already split into its
-// TF32 high and low parts; C streams through a 3-stage cp.async ring in chunks of 32 columns.
-// NPROD = 3: hi*hi + lo*hi + hi*lo (fp32-level accuracy); NPROD = 1: a single TF32 product.
-// The upper 19 bits of x: a TF32 number.  x - hi is exact in fp32, so hi.hi + hi.lo + lo.hi misses the product by
-// about 2^-20 relative.  (cvt.rna.tf32 costs about five instructions per value on this target, masking one.)
-__device__ __forceinline__ uint32_t g_tf32(float x) { return __float_as_uint(x) & 0xffffe000u; }
-__device__ __forceinline__ void g_mma(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
-{
-    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
+// high and low BF16 parts; C streams through a 3-stage cp.async ring in chunks of 32 columns.
 __device__ __forceinline__ void g_cp_async16(float *dst_smem, const float *src)
 {
     const uint32_t d = static_cast<uint32_t>(__cvta_generic_to_shared(dst_smem));
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(src) : "memory");
 }
 
-template <int L, int M, int NPROD>
-struct gemm_cfg {
+// BF16x3 products: x = b1 + b2 with b1 = bf16(x), b2 = bf16(x - b1) represents x to 2^-18 relative;
+// b1.b1 + b1.b2 + b2.b1 then misses the fp32 product by about 1e-5 relative (inside the 1e-4 tolerance), and one
+// m16n8k16 BF16 MMA does the work of two m16n8k8 TF32 MMAs: three of them cost half the tensor-pipe time of a
+// three-product TF32 scheme, which was what bound this kernel (tensor pipe 56 % busy, DRAM 23 %).  D is kept as
+// packed pairs (D(2p,m), D(2p+1,m)).
+__device__ __forceinline__ uint32_t bf16x2_rn(float lo, float hi)
+{
+    uint32_t d;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
+}
+// (b1, b2) of the pair (x0, x1): h = packed b1 parts, l = packed b2 parts
+__device__ __forceinline__ void bf16_split2(float x0, float x1, uint32_t &h, uint32_t &l)
+{
+    h = bf16x2_rn(x0, x1);
+    l = bf16x2_rn(x0 - __uint_as_float(h << 16), x1 - __uint_as_float(h & 0xffff0000u));
+}
+__device__ __forceinline__ void g_mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+template <int L, int M>
+struct gemm_bf16_cfg {
     static constexpr int BM = 128, KC = 32, NS = 3;
-    static constexpr int CS = KC + 4;                 // row stride of a C chunk (conflict-free A fragments)
-    static constexpr int DS = M + 8;                  // row stride of D (conflict-free B fragments)
+    static constexpr int CS = KC + 8;                 // row stride of a C chunk (conflict-free 64-bit A reads)
+    static constexpr int DS = M + 8;                  // row stride of the packed D pairs (conflict-free B reads)
     static constexpr int NT = M / 16;                 // n8 tiles per warp (warp covers M/2 columns)
-    static constexpr int D_FLOATS = L * DS * (NPROD == 3 ? 2 : 1);
+    static constexpr int D_WORDS = (L / 2) * DS * 2;  // high and low parts
     static constexpr int STAGE = BM * CS;
-    static constexpr size_t SMEM = size_t(D_FLOATS + NS * STAGE) * sizeof(float);
+    static constexpr size_t SMEM = size_t(D_WORDS + NS * STAGE) * sizeof(float);
 };
 
-template <int L, int M, int NPROD>
+template <int L, int M>
 __global__ void __launch_bounds__(256, 1)
-gemm_tf32_kernel(int64_t J, const float *__restrict__ C, int64_t ldc, const float *__restrict__ D, int64_t ldd,
-                 float *__restrict__ Eout)
+gemm_bf16x3_kernel(int64_t J, const float *__restrict__ C, int64_t ldc, const float *__restrict__ D, int64_t ldd,
+                   float *__restrict__ Eout)
 {
-    using G = gemm_cfg<L, M, NPROD>;
+    using G = gemm_bf16_cfg<L, M>;
     extern __shared__ __align__(16) float smem[];
     uint32_t *Dh = reinterpret_cast<uint32_t *>(smem);
-    uint32_t *Dl = Dh + L * G::DS;                     // only with NPROD == 3
-    float *Cs = smem + G::D_FLOATS;
+    uint32_t *Dl = Dh + (L / 2) * G::DS;
+    float *Cs = smem + G::D_WORDS;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int g = lane >> 2, t = lane & 3;
     const int wr = warp >> 1, wc = warp & 1;           // warp tile: rows 32*wr.., columns (M/2)*wc..
-    for (int x = threadIdx.x; x < L * M; x += 256) {
-        const int l = x / M, m = x % M;
-        const float d = __ldg(D + int64_t(l) * ldd + m);
-        const uint32_t hi = g_tf32(d);
-        Dh[l * G::DS + m] = hi;
-        if (NPROD == 3) Dl[l * G::DS + m] = g_tf32(d - __uint_as_float(hi));
+    for (int x = threadIdx.x; x < (L / 2) * M; x += 256) {
+        const int p = x / M, m = x % M;
+        uint32_t h, l;
+        bf16_split2(__ldg(D + int64_t(2 * p) * ldd + m), __ldg(D + int64_t(2 * p + 1) * ldd + m), h, l);
+        Dh[p * G::DS + m] = h;
+        Dl[p * G::DS + m] = l;
     }
     const int64_t n_tiles = (J + G::BM - 1) / G::BM;
     const int64_t my_tiles = blockIdx.x < n_tiles ? (n_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
     constexpr int KCH = L / G::KC;                     // chunks per row tile
     const int64_t n_chunks = my_tiles * KCH;
-    // chunk q of this block: row tile blockIdx.x + (q / KCH) * gridDim.x, columns (q % KCH) * KC ..
     auto issue = [&](int64_t q) {
         if (q < n_chunks) {
             const int64_t row0 = (int64_t(blockIdx.x) + (q / KCH) * gridDim.x) * G::BM;
@@ -200,35 +210,33 @@ gemm_tf32_kernel(int64_t J, const float *__restrict__ C, int64_t ldc, const floa
         __syncthreads();                               // chunk q landed for everyone; chunk q-1 fully consumed
         issue(q + 2);
         const float *cs = Cs + int(q % G::NS) * G::STAGE + (32 * wr) * G::CS;
-        const uint32_t *dh = Dh + (kc * G::KC) * G::DS + (M / 2) * wc;
-        const uint32_t *dl = Dl + (kc * G::KC) * G::DS + (M / 2) * wc;
+        const uint32_t *dh = Dh + (kc * (G::KC / 2)) * G::DS + (M / 2) * wc;
+        const uint32_t *dl = Dl + (kc * (G::KC / 2)) * G::DS + (M / 2) * wc;
 #pragma unroll
-        for (int kt = 0; kt < G::KC / 8; ++kt) {
+        for (int kt = 0; kt < G::KC / 16; ++kt) {
             uint32_t ah[2][4], al[2][4];
 #pragma unroll
             for (int mt = 0; mt < 2; ++mt) {
-                const float *p = cs + (16 * mt + g) * G::CS + 8 * kt + t;
-                const float x0 = p[0], x1 = p[8 * G::CS], x2 = p[4], x3 = p[8 * G::CS + 4];
-                ah[mt][0] = g_tf32(x0); ah[mt][1] = g_tf32(x1); ah[mt][2] = g_tf32(x2); ah[mt][3] = g_tf32(x3);
-                if (NPROD == 3) {
-                    al[mt][0] = g_tf32(x0 - __uint_as_float(ah[mt][0]));
-                    al[mt][1] = g_tf32(x1 - __uint_as_float(ah[mt][1]));
-                    al[mt][2] = g_tf32(x2 - __uint_as_float(ah[mt][2]));
-                    al[mt][3] = g_tf32(x3 - __uint_as_float(ah[mt][3]));
-                }
+                const float *p = cs + (16 * mt + g) * G::CS + 16 * kt + 2 * t;
+                const float2 x0 = *reinterpret_cast<const float2 *>(p);                   // (row g,     k 2t, 2t+1)
+                const float2 x1 = *reinterpret_cast<const float2 *>(p + 8 * G::CS);       // (row g + 8, k 2t, 2t+1)
+                const float2 x2 = *reinterpret_cast<const float2 *>(p + 8);               // (row g,     k 2t+8, 2t+9)
+                const float2 x3 = *reinterpret_cast<const float2 *>(p + 8 * G::CS + 8);   // (row g + 8, k 2t+8, 2t+9)
+                bf16_split2(x0.x, x0.y, ah[mt][0], al[mt][0]);
+                bf16_split2(x1.x, x1.y, ah[mt][1], al[mt][1]);
+                bf16_split2(x2.x, x2.y, ah[mt][2], al[mt][2]);
+                bf16_split2(x3.x, x3.y, ah[mt][3], al[mt][3]);
             }
 #pragma unroll
             for (int nt = 0; nt < G::NT; ++nt) {
-                const int off = (8 * kt + t) * G::DS + 8 * nt + g;
+                const int off = (8 * kt + t) * G::DS + 8 * nt + g;          // pair row (16 kt + 2 t) / 2
                 const uint32_t bh0 = dh[off], bh1 = dh[off + 4 * G::DS];
+                const uint32_t bl0 = dl[off], bl1 = dl[off + 4 * G::DS];
 #pragma unroll
                 for (int mt = 0; mt < 2; ++mt) {
-                    if (NPROD == 3) {
-                        const uint32_t bl0 = dl[off], bl1 = dl[off + 4 * G::DS];
-                        g_mma(acc[mt][nt], al[mt], bh0, bh1);
-                        g_mma(acc[mt][nt], ah[mt], bl0, bl1);
-                    }
-                    g_mma(acc[mt][nt], ah[mt], bh0, bh1);
+                    g_mma_bf16(acc[mt][nt], al[mt], bh0, bh1);
+                    g_mma_bf16(acc[mt][nt], ah[mt], bl0, bl1);
+                    g_mma_bf16(acc[mt][nt], ah[mt], bh0, bh1);
                 }
             }
         }
@@ -328,8 +336,8 @@ sa_status run(const sa_tensor *t, const sa_dense *ops, float *out, void *ws, boo
     const int64_t J = t->dims[1];
     float *E = static_cast<float *>(ws);
     float *partial = reinterpret_cast<float *>(static_cast<char *>(ws) + sa_align256(size_t(J) * M * sizeof(float)));
-    using GC = gemm_cfg<L, M, SA_GEMM_NPROD>;
-    auto gk = gemm_tf32_kernel<L, M, SA_GEMM_NPROD>;
+    using GC = gemm_bf16_cfg<L, M>;
+    auto gk = gemm_bf16x3_kernel<L, M>;
     if (cudaFuncSetAttribute(gk, cudaFuncAttributeMaxDynamicSharedMemorySize, int(GC::SMEM)) != cudaSuccess) return SA_E_CUDA;
     const int64_t gctas = std::min<int64_t>((J + GC::BM - 1) / GC::BM, resident_ctas(reinterpret_cast<const void *>(gk), GC::SMEM));
     gk<<<(unsigned)gctas, 256, GC::SMEM, stream>>>(J, ops[0].ptr, ops[0].ld, ops[1].ptr, ops[1].ld, E);
@@ -377,14 +385,14 @@ sa_status run_hadamard(const sa_tensor *t, const sa_dense *ops, float *out, void
 
 }  // namespace
 
-// out (rows x M) = A (rows x L, leading dimension lda) . B (L x M), TF32x3 on tensor cores; used as the
+// out (rows x M) = A (rows x L, leading dimension lda) . B (L x M), BF16x3 on tensor cores; used as the
 // dense stage of other chains.  L in {32, 64, 128, 256}, M in {32, 64}.
 template <int L, int M>
 static sa_status dense_gemm(int64_t rows, const float *A, int64_t lda, const float *B, int64_t ldb, float *out,
                             cudaStream_t stream)
 {
-    using GC = gemm_cfg<L, M, SA_GEMM_NPROD>;
-    auto gk = gemm_tf32_kernel<L, M, SA_GEMM_NPROD>;
+    using GC = gemm_bf16_cfg<L, M>;
+    auto gk = gemm_bf16x3_kernel<L, M>;
     if (cudaFuncSetAttribute(gk, cudaFuncAttributeMaxDynamicSharedMemorySize, int(GC::SMEM)) != cudaSuccess) return SA_E_CUDA;
     const int64_t ctas = std::min<int64_t>((rows + GC::BM - 1) / GC::BM, resident_ctas(reinterpret_cast<const void *>(gk), GC::SMEM));
     if (ctas > 0) gk<<<(unsigned)ctas, 256, GC::SMEM, stream>>>(rows, A, lda, B, ldb, out);
