@@ -7,7 +7,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsparseauto.so")
-SOURCES = ["sa_api.cu", "sa_build.cu", "sa_ttm3.cu", "sa_ttm4.cu", "sa_sddmm_spmm.cu", "sa_spmm_gemm.cu", "sa_ttmc3.cu", "sa_gather_probe.cu", "sa_mttkrp.cu"]
+SOURCES = ["sa_api.cu", "sa_build.cu", "sa_ttm3.cu", "sa_ttm4.cu", "sa_sddmm_spmm.cu", "sa_spmm_gemm.cu", "sa_ttmc3.cu", "sa_gather_probe.cu", "sa_mttkrp.cu", "sa_dense_tc.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC,-fopenmp,-O3", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 

@@ -153,8 +153,13 @@ sa_status sa_launch_sddmm_spmm_gemm(const sa_tensor *t, const sa_dense *ops, flo
                                     cudaStream_t stream, int *launches);
 size_t sa_ws_sddmm_spmm_gemm(const sa_tensor *t, const sa_dense *ops);
 bool sa_dense_gemm_ok(int64_t L, int64_t M);
+// out (rows x M) = A (rows x L) . B (L x M); `status` is the tensor's device status word (a wait that runs out
+// inside the tcgen05 kernel records SA_E_TIMEOUT there).  L >= 64 runs on tcgen05, L = 32 on mma.sync.
 sa_status sa_launch_dense_gemm(int64_t rows, const float *A, int64_t lda, const float *B, int64_t ldb, int64_t L,
-                               int64_t M, float *out, cudaStream_t stream);
+                               int64_t M, float *out, int32_t *status, cudaStream_t stream);
+bool sa_dense_gemm_tc_ok(int64_t L, int64_t M);
+sa_status sa_launch_dense_gemm_tc(int64_t rows, const float *A, int64_t lda, const float *B, int64_t ldb, int64_t L,
+                                  int64_t M, float *out, int32_t *status, cudaStream_t stream);
 
 // Kernel 8 <MTTKRP,GEMM>
 sa_status sa_launch_mttkrp_gemm(const sa_tensor *t, const sa_dense *ops, float *out, void *ws, size_t ws_bytes,

@@ -28,7 +28,7 @@ sa_status sa_launch_mttkrp_gemm(const sa_tensor *t, const sa_dense *ops, float *
     int n1 = 0;
     sa_status s = sa_launch_mttkrp_rows(t, ops[0], ops[1], T, partial, stream, &n1);
     if (s != SA_OK) return s;
-    s = sa_launch_dense_gemm(I, T, R, ops[2].ptr, ops[2].ld, R, M, out, stream);
+    s = sa_launch_dense_gemm(I, T, R, ops[2].ptr, ops[2].ld, R, M, out, t->d_status, stream);
     if (s != SA_OK) return s;
     *launches = n1 + 1;
     return SA_OK;

@@ -255,7 +255,7 @@ sa_status sa_launch_sddmm_spmm_gemm(const sa_tensor *t, const sa_dense *ops, flo
     int n1 = 0;
     const sa_status s = sa_launch_sddmm_spmm(t, ops, T, static_cast<char *>(ws) + t_bytes, ws_bytes - t_bytes, false, stream, &n1);
     if (s != SA_OK) return s;
-    const sa_status g = sa_launch_dense_gemm(I, T, L, ops[3].ptr, ops[3].ld, L, M, out, stream);
+    const sa_status g = sa_launch_dense_gemm(I, T, L, ops[3].ptr, ops[3].ld, L, M, out, t->d_status, stream);
     if (g != SA_OK) return g;
     *launches = n1 + 1;
     return SA_OK;

@@ -336,12 +336,8 @@ sa_status run(const sa_tensor *t, const sa_dense *ops, float *out, void *ws, boo
     const int64_t J = t->dims[1];
     float *E = static_cast<float *>(ws);
     float *partial = reinterpret_cast<float *>(static_cast<char *>(ws) + sa_align256(size_t(J) * M * sizeof(float)));
-    using GC = gemm_bf16_cfg<L, M>;
-    auto gk = gemm_bf16x3_kernel<L, M>;
-    if (cudaFuncSetAttribute(gk, cudaFuncAttributeMaxDynamicSharedMemorySize, int(GC::SMEM)) != cudaSuccess) return SA_E_CUDA;
-    const int64_t gctas = std::min<int64_t>((J + GC::BM - 1) / GC::BM, resident_ctas(reinterpret_cast<const void *>(gk), GC::SMEM));
-    gk<<<(unsigned)gctas, 256, GC::SMEM, stream>>>(J, ops[0].ptr, ops[0].ld, ops[1].ptr, ops[1].ld, E);
-    if (cudaGetLastError() != cudaSuccess) return SA_E_CUDA;
+    const sa_status gs = sa_launch_dense_gemm(J, ops[0].ptr, ops[0].ld, ops[1].ptr, ops[1].ld, L, M, E, t->d_status, stream);
+    if (gs != SA_OK) return gs;
     *launches += 1;
     const int64_t ctas = (n_items + SA_WARPS_PER_CTA - 1) / SA_WARPS_PER_CTA;
     if (ctas > 0) {
@@ -402,10 +398,11 @@ static sa_status dense_gemm(int64_t rows, const float *A, int64_t lda, const flo
 bool sa_dense_gemm_ok(int64_t L, int64_t M) { return (L == 32 || L == 64 || L == 128 || L == 256) && (M == 32 || M == 64); }
 
 sa_status sa_launch_dense_gemm(int64_t rows, const float *A, int64_t lda, const float *B, int64_t ldb, int64_t L,
-                               int64_t M, float *out, cudaStream_t stream)
+                               int64_t M, float *out, int32_t *status, cudaStream_t stream)
 {
+    if (sa_dense_gemm_tc_ok(L, M)) return sa_launch_dense_gemm_tc(rows, A, lda, B, ldb, L, M, out, status, stream);
 #define SA_CASE(l, m) if (L == l && M == m) return dense_gemm<l, m>(rows, A, lda, B, ldb, out, stream);
-    SA_CASE(32, 32) SA_CASE(32, 64) SA_CASE(64, 32) SA_CASE(64, 64) SA_CASE(128, 32) SA_CASE(128, 64) SA_CASE(256, 32) SA_CASE(256, 64)
+    SA_CASE(32, 32) SA_CASE(32, 64)
 #undef SA_CASE
     return SA_E_UNSUPPORTED;
 }
