@@ -7,15 +7,20 @@
 // and a product is formed as b1.b1 + b1.b2 + b2.b1 (error about 1e-5 relative, inside the 1e-4 bound).
 //
 // One persistent thread block per SM, 128-row tiles, roles by warp:
-//   warps 5..12  cp.async 64-column chunks of C into a private fp32 ring (every thread converts exactly the
-//                bytes it copied itself, so the ring needs no barrier), split them into the two BF16 parts
-//                and write both as K-major 128-byte-swizzled operand tiles;
-//   warp 4       one lane issues tcgen05.mma (M = 128, N = M, K = 16; three per K step) from those tiles and
-//                from D^T, which sits in shared memory (both BF16 parts) for the life of the block; the
-//                accumulator lives in tensor memory, two of them so that a tile's epilogue overlaps the next
-//                tile's products;
-//   warps 0..3   read a finished accumulator with tcgen05.ld (warp w owns TMEM lanes 32w..32w+31 = tile rows)
-//                and store the rows of E.
+//   warps 5..12  load 64-column chunks of C straight into registers (coalesced 128-bit loads, two chunks in
+//                flight per thread while a third is converted), split them into the two BF16 parts and write
+//                both as K-major 128-byte-swizzled operand tiles (four stages);
+//   warp 4       one lane issues tcgen05.mma (M = 128, K = 16) from those tiles and from D^T, which sits in
+//                shared memory for the life of the block with the low parts stacked under the high parts:
+//                b1(C) . [b1(D) | b2(D)] is one product of N = 2M, b2(C) . b1(D) one of N = M onto the first
+//                M columns; the accumulator (2M columns) lives in tensor memory, two of them so that a
+//                tile's epilogue overlaps the next tile's products;
+//   warps 0..3   read a finished accumulator with tcgen05.ld (warp w owns TMEM lanes 32w..32w+31 = tile rows),
+//                add its two halves, transpose through a swizzled shared-memory tile and store E in
+//                512-byte runs.
+// What limits this kernel next to HBM is the shared-memory data pipe (operand writes, tensor-core operand
+// reads, epilogue), which is why C never passes through a shared-memory fp32 stage and why the two products
+// that share b1(C) are merged.
 // Hand-offs are mbarriers; tcgen05.commit signals the completion of the products.  Every wait is bounded by a
 // timer: on expiry the block raises its abort flag, all roles leave their loops, the status word is set to
 // SA_E_TIMEOUT and tensor memory is released as on the normal path.
@@ -27,7 +32,7 @@ namespace {
 
 constexpr int TC_BM = 128;                  // rows per tile = MMA M = TMEM lanes
 constexpr int TC_KC = 64;                   // columns of C per chunk: one 128-byte swizzled BF16 row
-constexpr int TC_NS = 3;                    // fp32 ring stages (two chunks in flight while one is converted)
+constexpr int TC_OPS = 4;                   // operand stages
 constexpr int TC_EPI_WARPS = 4;
 constexpr int TC_MMA_WARP = 4;
 constexpr int TC_CONV_WARPS = 8;
@@ -38,20 +43,20 @@ constexpr uint64_t TC_WAIT_NS = 2000000000ull;   // longest a hand-off may take 
 template <int L, int M>
 struct tc_cfg {
     static constexpr int KCH = L / TC_KC;
-    static constexpr uint32_t D_PART = uint32_t(KCH) * M * 128;        // one BF16 part of D^T (KCH tiles of M x 64)
+    static constexpr uint32_t D_TILE = 2 * M * 128;                    // one chunk of D^T: M rows of b1, then M rows of b2
     static constexpr uint32_t OP_PART = TC_BM * 128;                   // one BF16 part of a chunk of C
-    static constexpr uint32_t RING_STAGE = TC_BM * TC_KC * 4;
-    static constexpr uint32_t OFF_DH = 0, OFF_DL = D_PART, OFF_OP = 2 * D_PART;
-    static constexpr uint32_t OFF_RING = OFF_OP + 4 * OP_PART;         // two operand stages x (high, low)
-    static constexpr uint32_t OFF_BAR = OFF_RING + TC_NS * RING_STAGE;
+    static constexpr uint32_t EPI_WARP = 32 * M * 4;                   // transposition tile of one epilogue warp
+    static constexpr uint32_t OFF_D = 0, OFF_OP = uint32_t(KCH) * D_TILE;
+    static constexpr uint32_t OFF_EPI = OFF_OP + TC_OPS * 2 * OP_PART;
+    static constexpr uint32_t OFF_BAR = OFF_EPI + TC_EPI_WARPS * EPI_WARP;
     static constexpr size_t SMEM = size_t(OFF_BAR) + 128 + 1024;       // barriers + slack to align the base to 1 KB
-    static constexpr uint32_t TMEM_COLS = 2 * M;                       // two fp32 accumulators of M columns
+    static constexpr uint32_t TMEM_COLS = 4 * M;                       // two fp32 accumulators of 2M columns
     static_assert(L % TC_KC == 0 && (M == 32 || M == 64), "unsupported shape");
-    static_assert(D_PART % 1024 == 0, "swizzle atoms must stay 1 KB aligned");
+    static_assert(D_TILE % 1024 == 0, "swizzle atoms must stay 1 KB aligned");
 };
 
 // barrier slots (8 bytes each) behind the ring
-enum { B_FULL = 0, B_EMPTY = 2, B_ACC_FULL = 4, B_ACC_EMPTY = 6, B_DRAIN = 8, B_COUNT = 9 };
+enum { B_FULL = 0, B_EMPTY = TC_OPS, B_ACC_FULL = 2 * TC_OPS, B_ACC_EMPTY = 2 * TC_OPS + 2, B_DRAIN = 2 * TC_OPS + 4, B_COUNT = 2 * TC_OPS + 5 };
 
 __device__ __forceinline__ uint32_t tc_smem_u32(const void *p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
 
@@ -144,9 +149,11 @@ __device__ __forceinline__ void tc_ld16(uint32_t taddr, float (&v)[16])
     for (int x = 0; x < 16; ++x) v[x] = __uint_as_float(r[x]);
 }
 
-__device__ __forceinline__ void tc_cp_async16(uint32_t dst, const float *src)
+__device__ __forceinline__ float4 tc_ldg4(const float *p)
 {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+    float4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p));
+    return v;
 }
 
 // packed BF16 pair, element `lo` in the low half
@@ -183,26 +190,26 @@ gemm_tc_kernel(int64_t J, const float *__restrict__ C, int64_t ldc, const float 
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + G::OFF_BAR + 8 * B_COUNT + 4);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-    // D^T, both BF16 parts, as KCH operand tiles of M rows (n) x 64 columns (k)
+    // D^T as KCH operand tiles of 2M rows x 64 columns (k): rows n < M hold b1(D(k,n)), rows M + n hold b2
     for (int x = threadIdx.x; x < L * M; x += TC_THREADS) {
         const int k = x / M, n = x % M;
         const float v = __ldg(D + int64_t(k) * ldd + n);
         const uint32_t h = tc_bf16x2(v, 0.f) & 0xffffu;
         const uint32_t l = tc_bf16x2(v - __uint_as_float(h << 16), 0.f) & 0xffffu;
-        const uint32_t off = uint32_t(k / TC_KC) * (M * 128) + tc_sw128(n, k % TC_KC);
-        *reinterpret_cast<uint16_t *>(smem + G::OFF_DH + off) = uint16_t(h);
-        *reinterpret_cast<uint16_t *>(smem + G::OFF_DL + off) = uint16_t(l);
+        const uint32_t off = G::OFF_D + uint32_t(k / TC_KC) * G::D_TILE + tc_sw128(n, k % TC_KC);
+        *reinterpret_cast<uint16_t *>(smem + off) = uint16_t(h);
+        *reinterpret_cast<uint16_t *>(smem + off + M * 128) = uint16_t(l);     // row n + M: same swizzle phase
     }
     fence_async_smem();
     if (threadIdx.x == 0) {
-        mbar_init(bars + 8 * (B_FULL + 0), TC_CONV_T);
-        mbar_init(bars + 8 * (B_FULL + 1), TC_CONV_T);
-        mbar_init(bars + 8 * (B_EMPTY + 0), 1);
-        mbar_init(bars + 8 * (B_EMPTY + 1), 1);
-        mbar_init(bars + 8 * (B_ACC_FULL + 0), 1);
-        mbar_init(bars + 8 * (B_ACC_FULL + 1), 1);
-        mbar_init(bars + 8 * (B_ACC_EMPTY + 0), TC_EPI_WARPS * 32);
-        mbar_init(bars + 8 * (B_ACC_EMPTY + 1), TC_EPI_WARPS * 32);
+        for (int x = 0; x < TC_OPS; ++x) {
+            mbar_init(bars + 8 * (B_FULL + x), TC_CONV_T);
+            mbar_init(bars + 8 * (B_EMPTY + x), 1);
+        }
+        for (int x = 0; x < 2; ++x) {
+            mbar_init(bars + 8 * (B_ACC_FULL + x), 1);
+            mbar_init(bars + 8 * (B_ACC_EMPTY + x), TC_EPI_WARPS * 32);
+        }
         mbar_init(bars + 8 * B_DRAIN, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -224,50 +231,62 @@ gemm_tc_kernel(int64_t J, const float *__restrict__ C, int64_t ldc, const float 
     const int64_t n_chunks = my_tiles * G::KCH;
 
     if (warp < TC_EPI_WARPS) {
-        // ---- epilogue: accumulator -> rows of E
+        // ---- epilogue: accumulator halves -> sum -> transposition tile -> rows of E
+        constexpr int RC = M / 4;                                   // 16-byte units per row of E
+        uint8_t *stage = smem + G::OFF_EPI + warp * G::EPI_WARP;
         for (int64_t tl = 0; tl < my_tiles; ++tl) {
             const uint32_t a = uint32_t(tl) & 1u, v = uint32_t(tl >> 1);
             const bool ok = mbar_wait(bars + 8 * (B_ACC_FULL + a), v & 1u, abort_flag);
             if (!__all_sync(SA_FULL_MASK, ok)) break;
             tc_fence_after();
-            const int64_t row = (int64_t(blockIdx.x) + tl * gridDim.x) * TC_BM + 32 * warp + lane;
-            const uint32_t taddr = tmem_base + (uint32_t(32 * warp) << 16) + a * M;
+            const uint32_t taddr = tmem_base + (uint32_t(32 * warp) << 16) + a * (2 * M);
 #pragma unroll
             for (int c = 0; c < M / 16; ++c) {
-                float v16[16];
-                tc_ld16(taddr + 16 * c, v16);
-                if (row < J) {
-                    float4 *dst = reinterpret_cast<float4 *>(Eout + row * M + 16 * c);
+                float p[16], r[16];
+                tc_ld16(taddr + 16 * c, p);
+                tc_ld16(taddr + M + 16 * c, r);
 #pragma unroll
-                    for (int x = 0; x < 4; ++x) dst[x] = make_float4(v16[4 * x], v16[4 * x + 1], v16[4 * x + 2], v16[4 * x + 3]);
-                }
+                for (int x = 0; x < 4; ++x)                         // unit 4c + x of row `lane`, XOR-swizzled by the row
+                    *reinterpret_cast<float4 *>(stage + lane * (M * 4) + (((4 * c + x) ^ (lane & 7)) << 4)) =
+                        make_float4(p[4 * x] + r[4 * x], p[4 * x + 1] + r[4 * x + 1], p[4 * x + 2] + r[4 * x + 2],
+                                    p[4 * x + 3] + r[4 * x + 3]);
             }
             tc_fence_before();
-            mbar_arrive(bars + 8 * (B_ACC_EMPTY + a));
+            mbar_arrive(bars + 8 * (B_ACC_EMPTY + a));               // the accumulator is free again
+            __syncwarp();
+            const int64_t row0 = (int64_t(blockIdx.x) + tl * gridDim.x) * TC_BM + 32 * warp;
+            float4 *dst = reinterpret_cast<float4 *>(Eout + row0 * M);
+#pragma unroll
+            for (int i = 0; i < RC; ++i) {
+                const int idx = i * 32 + lane, r = idx / RC, j = idx % RC;
+                const float4 val = *reinterpret_cast<const float4 *>(stage + r * (M * 4) + ((j ^ (r & 7)) << 4));
+                if (row0 + r < J) dst[idx] = val;
+            }
+            __syncwarp();
         }
     } else if (warp == TC_MMA_WARP) {
         // ---- products: one lane issues, the whole warp follows the hand-offs
-        constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(M >> 3) << 17) | (uint32_t(TC_BM >> 4) << 24);
+        constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(TC_BM >> 4) << 24);   // fp32 += bf16 . bf16, K-major
+        constexpr uint32_t IDESC_2M = IDESC | (uint32_t((2 * M) >> 3) << 17), IDESC_M = IDESC | (uint32_t(M >> 3) << 17);
         for (int64_t q = 0; q < n_chunks; ++q) {
             const int kc = int(q % G::KCH);
             const int64_t tl = q / G::KCH;
             const uint32_t a = uint32_t(tl) & 1u, v = uint32_t(tl >> 1);
-            const uint32_t s = uint32_t(q) & 1u, u = uint32_t(q >> 1);
+            const uint32_t s = uint32_t(q) % TC_OPS, u = uint32_t(q / TC_OPS);
             bool ok = true;
             if (kc == 0) ok = mbar_wait(bars + 8 * (B_ACC_EMPTY + a), (v & 1u) ^ 1u, abort_flag);
             if (ok) ok = mbar_wait(bars + 8 * (B_FULL + s), u & 1u, abort_flag);
             if (!__all_sync(SA_FULL_MASK, ok)) break;
             tc_fence_after();
             if (lane == 0) {
-                const uint32_t d_tmem = tmem_base + a * M;
+                const uint32_t d_tmem = tmem_base + a * (2 * M);
                 const uint32_t a_hi = sbase + G::OFF_OP + s * (2 * G::OP_PART), a_lo = a_hi + G::OP_PART;
-                const uint32_t b_hi = sbase + G::OFF_DH + uint32_t(kc) * (M * 128), b_lo = b_hi + G::D_PART;
+                const uint32_t b = sbase + G::OFF_D + uint32_t(kc) * G::D_TILE;
 #pragma unroll
                 for (int k = 0; k < TC_KC / 16; ++k) {
                     const uint32_t adv = 32u * k;                        // 16 BF16 along K inside the swizzled row
-                    tc_mma(d_tmem, tc_desc(a_lo + adv), tc_desc(b_hi + adv), IDESC, (kc | k) != 0);
-                    tc_mma(d_tmem, tc_desc(a_hi + adv), tc_desc(b_lo + adv), IDESC, 1u);
-                    tc_mma(d_tmem, tc_desc(a_hi + adv), tc_desc(b_hi + adv), IDESC, 1u);
+                    tc_mma(d_tmem, tc_desc(a_hi + adv), tc_desc(b + adv), IDESC_2M, (kc | k) != 0);
+                    tc_mma(d_tmem, tc_desc(a_lo + adv), tc_desc(b + adv), IDESC_M, 1u);
                 }
                 tc_commit(bars + 8 * (B_EMPTY + s));
                 if (kc == G::KCH - 1) tc_commit(bars + 8 * (B_ACC_FULL + a));
@@ -275,46 +294,48 @@ gemm_tc_kernel(int64_t J, const float *__restrict__ C, int64_t ldc, const float 
             __syncwarp();
         }
     } else {
-        // ---- copy and conversion: thread owns float4 column qf of rows r0, r0 + 16, ...
+        // ---- load and conversion: thread owns float4 column qf of rows r0, r0 + 16, ...
         const int t = threadIdx.x - (TC_EPI_WARPS + 1) * 32;
         const uint32_t qf = uint32_t(t) & 15u, r0 = uint32_t(t) >> 4, sw = r0 & 7u;
-        const uint32_t ring = sbase + G::OFF_RING + r0 * 256u + ((qf ^ sw) << 4);
-        const uint32_t op_off = r0 * 128u + (((qf >> 1) ^ sw) << 4) + ((qf & 1u) << 3);
-        auto issue = [&](int64_t q) {
+        const uint32_t op_off = G::OFF_OP + r0 * 128u + (((qf >> 1) ^ sw) << 4) + ((qf & 1u) << 3);
+        constexpr int NR = TC_BM / 16;
+        auto load = [&](float4 (&b)[NR], int64_t q) {
             if (q < n_chunks) {
                 const int64_t row0 = (int64_t(blockIdx.x) + (q / G::KCH) * gridDim.x) * TC_BM + r0;
                 const float *src = C + int(q % G::KCH) * TC_KC + 4 * qf;
-                const uint32_t dst = ring + uint32_t(q % TC_NS) * G::RING_STAGE;
 #pragma unroll
-                for (int i = 0; i < TC_BM / 16; ++i) {
-                    const int64_t row = min(row0 + 16 * i, J - 1);       // rows past the end re-read the last row
-                    tc_cp_async16(dst + uint32_t(i) * (16u * 256u), src + row * ldc);
-                }
+                for (int i = 0; i < NR; ++i) b[i] = tc_ldg4(src + min(row0 + 16 * i, J - 1) * ldc);   // rows past the end re-read the last row
             }
-            asm volatile("cp.async.commit_group;" ::: "memory");
         };
+        auto convert = [&](const float4 (&b)[NR], int64_t q) -> bool {
+            const uint32_t s = uint32_t(q) % TC_OPS, u = uint32_t(q / TC_OPS);
+            if (!mbar_wait(bars + 8 * (B_EMPTY + s), (u & 1u) ^ 1u, abort_flag)) return false;
+            uint8_t *hi = smem + op_off + s * (2 * G::OP_PART), *lo = hi + G::OP_PART;
 #pragma unroll
-        for (int q = 0; q < TC_NS - 1; ++q) issue(q);
-        for (int64_t q = 0; q < n_chunks; ++q) {
-            issue(q + TC_NS - 1);
-            asm volatile("cp.async.wait_group %0;" ::"n"(TC_NS - 1) : "memory");
-            const uint32_t s = uint32_t(q) & 1u, u = uint32_t(q >> 1);
-            if (!mbar_wait(bars + 8 * (B_EMPTY + s), (u & 1u) ^ 1u, abort_flag)) break;
-            const uint8_t *src = smem + (ring - sbase) + uint32_t(q % TC_NS) * G::RING_STAGE;
-            uint8_t *hi = smem + G::OFF_OP + s * (2 * G::OP_PART) + op_off, *lo = hi + G::OP_PART;
-#pragma unroll
-            for (int i = 0; i < TC_BM / 16; ++i) {
-                const float4 x = *reinterpret_cast<const float4 *>(src + i * (16 * 256));
+            for (int i = 0; i < NR; ++i) {
                 uint2 h, l;
-                tc_split2(x.x, x.y, h.x, l.x);
-                tc_split2(x.z, x.w, h.y, l.y);
+                tc_split2(b[i].x, b[i].y, h.x, l.x);
+                tc_split2(b[i].z, b[i].w, h.y, l.y);
                 *reinterpret_cast<uint2 *>(hi + i * (16 * 128)) = h;
                 *reinterpret_cast<uint2 *>(lo + i * (16 * 128)) = l;
             }
             fence_async_smem();
             mbar_arrive(bars + 8 * (B_FULL + s));
+            return true;
+        };
+        float4 b0[NR], b1[NR], b2[NR];
+        load(b0, 0);
+        load(b1, 1);
+        for (int64_t q = 0; q < n_chunks; q += 3) {
+            load(b2, q + 2);
+            if (!convert(b0, q)) break;
+            if (q + 1 >= n_chunks) break;
+            load(b0, q + 3);
+            if (!convert(b1, q + 1)) break;
+            if (q + 2 >= n_chunks) break;
+            load(b1, q + 4);
+            if (!convert(b2, q + 2)) break;
         }
-        asm volatile("cp.async.wait_group 0;" ::: "memory");
     }
 
     tc_fence_before();
