@@ -33,6 +33,7 @@ namespace {
 constexpr int TC_BM = 128;                  // rows per tile = MMA M = TMEM lanes
 constexpr int TC_KC = 64;                   // columns of C per chunk: one 128-byte swizzled BF16 row
 constexpr int TC_OPS = 4;                   // operand stages
+constexpr int TC_PF = 4;                    // chunks requested into L2 ahead of the loads into registers
 constexpr int TC_EPI_WARPS = 4;
 constexpr int TC_MMA_WARP = 4;
 constexpr int TC_CONV_WARPS = 8;
@@ -300,6 +301,11 @@ gemm_tc_kernel(int64_t J, const float *__restrict__ C, int64_t ldc, const float 
         const uint32_t op_off = G::OFF_OP + r0 * 128u + (((qf >> 1) ^ sw) << 4) + ((qf & 1u) << 3);
         constexpr int NR = TC_BM / 16;
         auto load = [&](float4 (&b)[NR], int64_t q) {
+            if (q + TC_PF < n_chunks) {                            // one 128-byte line per thread: HBM latency is paid by L2
+                const int64_t pq = q + TC_PF;
+                const int64_t row = min((int64_t(blockIdx.x) + (pq / G::KCH) * gridDim.x) * TC_BM + (t >> 1), J - 1);
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(C + row * ldc + int(pq % G::KCH) * TC_KC + 32 * (t & 1)));
+            }
             if (q < n_chunks) {
                 const int64_t row0 = (int64_t(blockIdx.x) + (q / G::KCH) * gridDim.x) * TC_BM + r0;
                 const float *src = C + int(q % G::KCH) * TC_KC + 4 * qf;
