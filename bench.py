@@ -105,6 +105,15 @@ def algorithmic_work(w, counts, sched):
         R, M = w.dense[0].shape[1], w.dense[2].shape[1]
         return (8 * nnz + 8 * F2 + 8 * S + sum(sz(d) for d in w.dense) + out_bytes,
                 2 * nnz * R + 2 * F2 * R + 2 * w.dims[0] * R * M)
+    if w.expr == "spttm_spttm":
+        # fibers as rows: index/value streams, one pos entry per fiber, the output (one row per fiber) once;
+        # (B'.C).D gathers a row of C per nonzero (C once: it fits L2), B'.(C.D) reads C and D once
+        F2, K = int(counts[1]), w.dims[2]
+        L, M = w.dense[0].shape[1], w.dense[1].shape[1]
+        base = 8 * nnz + 4 * (F2 + 1) + sz(w.dense[0]) + sz(w.dense[1]) + out_bytes
+        if sched == "left":
+            return base, 2 * nnz * L + 2 * F2 * L * M
+        return base, 2 * K * L * M + 2 * nnz * M
     if w.expr == "spmmh_gemm":
         # two gathered rows of L floats per nonzero (C and its Hadamard partner), E once, the output once
         I, J = w.dims
@@ -198,6 +207,7 @@ def oracle_sample(w, budget_s=15.0):
                "spmm_gemm": lambda: w.dense[0].shape[1] * w.dense[1].shape[1],
                "spmmh_gemm": lambda: w.dense[0].shape[1] * w.dense[2].shape[1],
                "mttkrp_gemm": lambda: w.dense[0].shape[1] * w.dense[2].shape[1],
+               "spttm_spttm": lambda: w.dense[0].shape[1] * w.dense[1].shape[1],
                "sddmm_spmm_gemm": lambda: w.dense[0].shape[1] * w.dense[2].shape[1] * w.dense[3].shape[1],
                "ttmc3": lambda: w.dense[0].shape[1] * w.dense[1].shape[1] * w.dense[2].shape[1]}[w.expr]()
     cores = oracle.max_threads()
@@ -216,7 +226,13 @@ def oracle_sample(w, budget_s=15.0):
         sample = "%d of %d output elements (seeded random), each over all %d nonzeros" % (n1, n_out, w.nnz)
         return {"value": w.nnz * (n1 / n_out) / dt / 1e9, "unit": "GNNZ/s", "cores": cores, "kind": "oracle",
                 "sample": sample, "seconds": dt}
-    counts = np.bincount(w.coords[:, 0], minlength=I)
+    if w.expr == "spttm_spttm":
+        # the output rows are B's (i,j) fibers: sample fibers instead of slices
+        _, inv = oracle.fiber_keys(w.coords, w.dims)
+        counts = np.bincount(inv)
+        I = counts.shape[0]
+    else:
+        counts = np.bincount(w.coords[:, 0], minlength=I)
     order = configs.rng.permutation(w.seed, 77, I)
     pilot_nnz = max(1000, int(0.5 * 0.25e9 * cores / per_nnz))          # ~0.5 s at a guessed rate
     n0, t0, _, _ = _oracle_run(w, counts, order, pilot_nnz, cores)
@@ -284,8 +300,9 @@ def workload_label(cfg, sched):
              7: "kernel 2 <SDDMM,SpMM,GEMM> on the config-3 tensor, K=L=M=64",
              6: "kernel 5 <3D TTMC> on a nell-2-shaped tensor 12000x9000x288000 76.88M nnz L=M=N=16",
              8: "kernel 3 <SpMMH,GEMM> on the config-4 tensor recipe 4Mx4M 100M nnz L=256 M=64",
-             9: "kernel 8 <MTTKRP,GEMM> on the config-2 tensor, R=32 M=32"}
-    return names[cfg] + (" (%s)" % sched if cfg == 4 else "")
+             9: "kernel 8 <MTTKRP,GEMM> on the config-2 tensor, R=32 M=32",
+             10: "kernel 7 <SpTTM,SpTTM> on the config-2 tensor, L=M=32, sparse output (one row per (i,j) fiber)"}
+    return names[cfg] + (" (%s)" % sched if cfg in (4, 10) else "")
 
 
 def label(args):
@@ -320,9 +337,9 @@ def main():
     ap.add_argument("--steps", type=int, default=31)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", type=int, default=2, choices=[1, 2, 3, 4, 5, 6, 7, 8, 9])
+    ap.add_argument("--workload", type=int, default=2, choices=[1, 2, 3, 4, 5, 6, 7, 8, 9, 10])
     ap.add_argument("--scale", default="full", choices=["full", "mid", "mini"])
-    ap.add_argument("--sched", default="right", choices=["left", "right"], help="association order for workload 4")
+    ap.add_argument("--sched", default="right", choices=["left", "right"], help="association order for workloads 4 and 10")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=5)
     args = ap.parse_args()
@@ -356,7 +373,7 @@ def main():
     build_s = time.perf_counter() - t0
     nnz, counts, n_chunks = tensor.info()
     sched = sa.SA_SCHED_DEFAULT
-    if w.expr == "spmm_gemm":
+    if w.expr in ("spmm_gemm", "spttm_spttm"):
         sched = sa.SA_SCHED_ASSOC_LEFT if args.sched == "left" else sa.SA_SCHED_ASSOC_RIGHT
 
     host_ops = [torch.from_numpy(np.ascontiguousarray(x)).pin_memory() for x in w.dense]
@@ -424,7 +441,7 @@ def main():
 
     if rank == 0:
         peaks, peak_kind = measured_peaks()
-        sched_name = args.sched if w.expr == "spmm_gemm" else "fused"
+        sched_name = args.sched if w.expr in ("spmm_gemm", "spttm_spttm") else "fused"
         abytes, aflops = algorithmic_work(w, counts, sched_name)
         gnnz = aggregate_throughput(nnz, world, ms_per_step)
         achieved = abytes / (ms_per_step * 1e-3) / 1e9

@@ -73,15 +73,24 @@ typedef enum {
     SA_EXPR_SPMMH_GEMM = 7,
     /* kernel 8 <MTTKRP,GEMM>: A(i,m) = sum_{j,k,r} B(i,j,k) C(j,r) D(k,r) E(r,m); ops = {C, D, E};
      * B order-3 CSF; the MTTKRP rows T(i,:) (R floats per slice) live in the workspace              */
-    SA_EXPR_MTTKRP_GEMM = 8
+    SA_EXPR_MTTKRP_GEMM = 8,
+    /* kernel 7 <SpTTM,SpTTM>: A(i,j,m) = sum_{k,l} B(i,j,k) C(k,l) D(l,m); ops = {C (dims[2] x L), D (L x M)};
+     * B order-3 CSF.  The output is sparse with B's (i,j) pattern: `out` receives one row of M values per
+     * level-1 node (fiber (i,j)) of B, F2 x M floats in CSF order, F2 = level_counts[1] of sa_tensor_info;
+     * the coordinates of row f are those sa_tensor_export returns for levels 0 and 1.
+     * SA_SCHED_FUSED / ASSOC_LEFT: the nest of the Table of kernels, fiber temporaries T(f, 0:L) in the
+     * workspace, then T . D; SA_SCHED_ASSOC_RIGHT: (C . D) first, then one gathered row per nonzero;
+     * SA_SCHED_DEFAULT: the one that moves fewer bytes.  L, M in {32, 64}.  A tensor without nonzeros has
+     * no output rows; `out` may then be NULL.                                                            */
+    SA_EXPR_SPTTM_SPTTM = 9
 } sa_expr;
 
 typedef enum {
     SA_SCHED_DEFAULT = 0,      /* the host table's choice for the expression; for SPMM_GEMM the
                                   association order that moves fewer bytes for this tensor      */
     SA_SCHED_FUSED = 1,        /* the fissioned / fused branched nest of the Table of kernels   */
-    SA_SCHED_ASSOC_LEFT = 2,   /* SA_EXPR_SPMM_GEMM only: (B.C).D, row temporary of L floats    */
-    SA_SCHED_ASSOC_RIGHT = 3,  /* SA_EXPR_SPMM_GEMM only: B.(C.D), J x M temporary in workspace */
+    SA_SCHED_ASSOC_LEFT = 2,   /* SA_EXPR_SPMM_GEMM (and SPTTM_SPTTM): (B.C).D, row temporary of L floats    */
+    SA_SCHED_ASSOC_RIGHT = 3,  /* SA_EXPR_SPMM_GEMM (and SPTTM_SPTTM): B.(C.D), J x M temporary in workspace */
     SA_SCHED_DEBUG_MATERIALIZE = 9 /* SA_EXPR_SDDMM_SPMM only, for tests: additionally writes the
                                       sampled values B(i,j) * sum_k C(i,k) D(j,k), aligned with
                                       the exported last-level crd array, to the workspace       */

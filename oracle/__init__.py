@@ -215,6 +215,50 @@ def mttkrp_gemm(coords, vals, dims, C, D, E, sel=None, with_abs=True, threads=0)
     return A, S
 
 
+def fiber_keys(coords, dims):
+    """The (i,j) pairs that occur in B, sorted lexicographically, and for every nonzero the index of its pair."""
+    c = np.asarray(coords)
+    key = c[:, 0].astype(np.int64) * int(dims[1]) + c[:, 1].astype(np.int64)
+    uniq, inv = np.unique(key, return_inverse=True)
+    keys = np.stack([uniq // int(dims[1]), uniq % int(dims[1])], axis=1)
+    return keys, inv.reshape(-1)
+
+
+def spttm_spttm(coords, vals, dims, C, D, sel=None, with_abs=True, threads=0):
+    """Kernel 7 <SpTTM,SpTTM>: A(i,j,m) = sum_{k,l} B(i,j,k) C(k,l) D(l,m)  (Table of kernels, Description
+    column with the two contracted indices k and l summed).  The output is sparse with the pattern of B's
+    (i,j) pairs: row f of the result belongs to the f-th pair in lexicographic order (see fiber_keys).
+    ``sel`` lists the rows wanted.  Plain definition in fp64: every nonzero adds v C(k,l) D(l,m) for all l, m.
+    Returns (A, S) with S the sum of the absolute values of the terms."""
+    I, J, K = (int(d) for d in dims)
+    c = np.asarray(coords)
+    v = np.asarray(vals, dtype=np.float64)
+    C = np.asarray(C, dtype=np.float64)
+    D = np.asarray(D, dtype=np.float64)
+    assert C.shape[0] == K and D.shape[0] == C.shape[1]
+    if c.shape[0] and (c.min() < 0 or (c.max(axis=0) >= np.array([I, J, K])).any()):
+        raise ValueError("coordinate out of range")
+    M = D.shape[1]
+    keys, inv = fiber_keys(c, dims)
+    if sel is None:
+        row_of, n_out, pick = inv, keys.shape[0], np.arange(c.shape[0])
+    else:
+        sel = np.asarray(sel, dtype=np.int64)
+        where = np.full(keys.shape[0], -1, dtype=np.int64)
+        where[sel] = np.arange(sel.shape[0])
+        row_of = where[inv]
+        pick = np.nonzero(row_of >= 0)[0]
+        n_out = sel.shape[0]
+    A = np.zeros((n_out, M), dtype=np.float64)
+    S = np.zeros((n_out, M), dtype=np.float64) if with_abs else None
+    for a in range(0, pick.shape[0], 4096):
+        p = pick[a:a + 4096]
+        term = v[p, None, None] * C[c[p, 2], :, None] * D[None, :, :]        # [nonzero, l, m]
+        np.add.at(A, row_of[p], term.sum(axis=1))
+        if with_abs:
+            np.add.at(S, row_of[p], np.abs(term).sum(axis=1))
+    return A, S
+
 def ttmc3(coords, vals, dims, C, D, E, sel=None, with_abs=True, threads=0):
     """A(l,m,n) = sum_{i,j,k} B(i,j,k) C(i,l) D(j,m) E(k,n).  Returns (A, S) of shape (L, M, N), or of
     shape (len(sel),) when ``sel`` lists flat output indices (l*M + m)*N + n."""
@@ -252,6 +296,8 @@ def evaluate(w, sel=None, with_abs=True, threads=0):
         return sddmm_spmm_gemm(w.coords, w.vals, w.dims, *w.dense, sel=sel, with_abs=with_abs, threads=threads)
     if w.expr == "sddmm_spmm":
         return sddmm_spmm(w.coords, w.vals, w.dims, *w.dense, sel=sel, with_abs=with_abs, threads=threads)[:2]
+    if w.expr == "spttm_spttm":
+        return spttm_spttm(w.coords, w.vals, w.dims, *w.dense, sel=sel, with_abs=with_abs, threads=threads)
     if w.expr == "mttkrp_gemm":
         return mttkrp_gemm(w.coords, w.vals, w.dims, *w.dense, sel=sel, with_abs=with_abs, threads=threads)
     if w.expr == "spmmh_gemm":

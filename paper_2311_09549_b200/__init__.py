@@ -24,7 +24,7 @@ SA_OK = 0
  SA_E_WORKSPACE, SA_E_CUDA, SA_E_BOUNDS, SA_E_TIMEOUT) = range(1, 12)
 SA_FMT_CSR, SA_FMT_CSF = 1, 2
 SA_EXPR_SPTTM_TTM3, SA_EXPR_SPTTM_TTM4, SA_EXPR_SDDMM_SPMM, SA_EXPR_SPMM_GEMM, SA_EXPR_TTMC3, SA_EXPR_SDDMM_SPMM_GEMM = 1, 2, 3, 4, 5, 6
-SA_EXPR_SPMMH_GEMM, SA_EXPR_MTTKRP_GEMM = 7, 8
+SA_EXPR_SPMMH_GEMM, SA_EXPR_MTTKRP_GEMM, SA_EXPR_SPTTM_SPTTM = 7, 8, 9
 SA_SCHED_DEFAULT, SA_SCHED_FUSED, SA_SCHED_ASSOC_LEFT, SA_SCHED_ASSOC_RIGHT = 0, 1, 2, 3
 SA_SCHED_DEBUG_MATERIALIZE = 9
 
@@ -216,7 +216,8 @@ def sa_destroy(handle):
 
 _EXPR_OF = {"spttm_ttm3": SA_EXPR_SPTTM_TTM3, "spttm_ttm4": SA_EXPR_SPTTM_TTM4,
             "sddmm_spmm": SA_EXPR_SDDMM_SPMM, "spmm_gemm": SA_EXPR_SPMM_GEMM, "ttmc3": SA_EXPR_TTMC3, "sddmm_spmm_gemm": SA_EXPR_SDDMM_SPMM_GEMM,
-            "spmmh_gemm": SA_EXPR_SPMMH_GEMM, "mttkrp_gemm": SA_EXPR_MTTKRP_GEMM}
+            "spmmh_gemm": SA_EXPR_SPMMH_GEMM, "mttkrp_gemm": SA_EXPR_MTTKRP_GEMM,
+            "spttm_spttm": SA_EXPR_SPTTM_SPTTM}
 
 
 class SparseTensor:
@@ -277,4 +278,6 @@ class SparseTensor:
             return (cols[0], cols[1], cols[2])
         if expr in (SA_EXPR_SPMMH_GEMM, SA_EXPR_MTTKRP_GEMM):
             return (self.dims[0], cols[2])
+        if expr == SA_EXPR_SPTTM_SPTTM:
+            return (int(self.info()[1][1]), cols[1])      # one row per (i,j) fiber, in CSF order
         return (self.dims[0], cols[1])

@@ -91,6 +91,7 @@ sa_status check_ops(const sa_tensor *t, sa_expr expr, const sa_dense *ops, int n
         case SA_EXPR_SDDMM_SPMM_GEMM: want = 4; break;
         case SA_EXPR_SPMMH_GEMM: want = 3; break;
         case SA_EXPR_MTTKRP_GEMM: want = 3; break;
+        case SA_EXPR_SPTTM_SPTTM: want = 2; break;
         default: return SA_E_ARG;
     }
     if (n_ops != want) return SA_E_ARG;
@@ -134,6 +135,11 @@ sa_status check_ops(const sa_tensor *t, sa_expr expr, const sa_dense *ops, int n
                 ops[2].rows != ops[0].cols)
                 return SA_E_SHAPE;
             if (!sa_ranks_ok_mttkrp_gemm(ops[0].cols, ops[2].cols)) return SA_E_UNSUPPORTED;
+            break;
+        case SA_EXPR_SPTTM_SPTTM:
+            if (t->fmt != SA_FMT_CSF || t->order != 3) return SA_E_FORMAT;
+            if (ops[0].rows != t->dims[2] || ops[1].rows != ops[0].cols) return SA_E_SHAPE;
+            if (!sa_ranks_ok_spttm_spttm(ops[0].cols, ops[1].cols)) return SA_E_UNSUPPORTED;
             break;
         case SA_EXPR_SPMMH_GEMM:
             if (t->fmt != SA_FMT_CSR) return SA_E_FORMAT;
@@ -185,6 +191,20 @@ bool resolve_schedule(const sa_tensor *t, sa_expr expr, sa_schedule sched, const
             if (sched == SA_SCHED_FUSED || sched == SA_SCHED_ASSOC_LEFT) { *resolved = SA_SCHED_ASSOC_LEFT; return true; }
             if (sched == SA_SCHED_ASSOC_RIGHT) { *resolved = sched; return true; }
             return false;
+        case SA_EXPR_SPTTM_SPTTM:
+            // the same comparison with the fibers as rows: the fiber temporaries are written and read once
+            //   (B'.C).D : nnz * (8 + 4 L) + 8 F2 L        B'.(C.D) : 4 K (L + M) + nnz * (8 + 4 M)
+            if (sched == SA_SCHED_DEFAULT) {
+                const double nnz = double(t->nnz), F2 = double(t->count[1]), K = double(t->dims[2]);
+                const double L = double(ops[0].cols), M = double(ops[1].cols);
+                const double left = nnz * (8.0 + 4.0 * L) + 8.0 * F2 * L;
+                const double right = 4.0 * K * (L + M) + nnz * (8.0 + 4.0 * M);
+                *resolved = left <= right ? SA_SCHED_ASSOC_LEFT : SA_SCHED_ASSOC_RIGHT;
+                return true;
+            }
+            if (sched == SA_SCHED_FUSED || sched == SA_SCHED_ASSOC_LEFT) { *resolved = SA_SCHED_ASSOC_LEFT; return true; }
+            if (sched == SA_SCHED_ASSOC_RIGHT) { *resolved = sched; return true; }
+            return false;
     }
     return false;
 }
@@ -200,6 +220,7 @@ size_t workspace_bytes(const sa_tensor *t, sa_expr expr, sa_schedule sched, cons
         case SA_EXPR_SDDMM_SPMM_GEMM: return sa_ws_sddmm_spmm_gemm(t, ops);
         case SA_EXPR_SPMMH_GEMM: return sa_ws_spmmh_gemm(t, ops);
         case SA_EXPR_MTTKRP_GEMM: return sa_ws_mttkrp_gemm(t, ops);
+        case SA_EXPR_SPTTM_SPTTM: return sa_ws_spttm_spttm(t, ops, sched == SA_SCHED_ASSOC_RIGHT);
     }
     return 0;
 }
@@ -330,8 +351,9 @@ sa_status sa_workspace_size(const sa_tensor *t, sa_expr expr, sa_schedule sched,
 sa_status sa_run(const sa_tensor *t, sa_expr expr, sa_schedule sched, const sa_dense *ops, int n_ops, float *out,
                  void *workspace, size_t ws_bytes, void *cuda_stream)
 {
-    if (!t || !out || t->device < 0) return SA_E_ARG;
-    if (reinterpret_cast<uintptr_t>(out) % 16) return SA_E_ARG;
+    if (!t || t->device < 0) return SA_E_ARG;
+    const bool empty_out = expr == SA_EXPR_SPTTM_SPTTM && t->count[1] == 0;    // a sparse output without rows
+    if ((!out && !empty_out) || reinterpret_cast<uintptr_t>(out) % 16) return SA_E_ARG;
     sa_status s = check_ops(t, expr, ops, n_ops, false);
     if (s != SA_OK) return s;
     sa_schedule r;
@@ -356,6 +378,9 @@ sa_status sa_run(const sa_tensor *t, sa_expr expr, sa_schedule sched, const sa_d
         case SA_EXPR_SDDMM_SPMM_GEMM: s = sa_launch_sddmm_spmm_gemm(t, ops, out, workspace, ws_bytes, stream, &launches); break;
         case SA_EXPR_SPMMH_GEMM: s = sa_launch_spmmh_gemm(t, ops, out, workspace, ws_bytes, stream, &launches); break;
         case SA_EXPR_MTTKRP_GEMM: s = sa_launch_mttkrp_gemm(t, ops, out, workspace, ws_bytes, stream, &launches); break;
+        case SA_EXPR_SPTTM_SPTTM:
+            s = sa_launch_spttm_spttm(t, ops, out, workspace, ws_bytes, r == SA_SCHED_ASSOC_RIGHT, stream, &launches);
+            break;
     }
     if (s == SA_E_CUDA) cudaGetLastError();
     if (s == SA_OK) t->last_launches = launches;

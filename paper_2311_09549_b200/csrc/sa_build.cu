@@ -325,12 +325,11 @@ void build_ttm4(sa_tensor *t, sa_worklist &wl, sa_worklist &wl2)
     append_empty_slices(t, wl2);
 }
 
-// CSR: row ranges of about target_nnz nonzeros (at most max_rows rows); rows longer than
+// Rows of a sparse matrix given by its pos array: row ranges of about target_nnz nonzeros (at most max_rows rows); rows longer than
 // long_thresh are cut into pieces of `piece` nonzeros whose partial rows the fix-up kernel sums.
-void build_csr(sa_tensor *t, sa_worklist &wl, int64_t target_nnz, int64_t max_rows, int64_t long_thresh, int64_t piece)
+void build_rows(const std::vector<int64_t> &pos, int64_t I, sa_worklist &wl, int64_t target_nnz, int64_t max_rows,
+                int64_t long_thresh, int64_t piece)
 {
-    const auto &pos = t->pos[1];
-    const int64_t I = t->dims[0];
     std::vector<sa_item> longs, ranges;
     int64_t r0 = 0;
     auto flush = [&](int64_t r1) {
@@ -376,10 +375,14 @@ void build_csr(sa_tensor *t, sa_worklist &wl, int64_t target_nnz, int64_t max_ro
 
 void sa_build_worklists(sa_tensor *t)
 {
-    if (t->fmt == SA_FMT_CSF && t->order == 3) build_ttm3(t, t->wl_main);
+    if (t->fmt == SA_FMT_CSF && t->order == 3) {
+        build_ttm3(t, t->wl_main);
+        // kernel 7 walks the tensor as a sparse matrix whose rows are the (i,j) fibers
+        build_rows(t->pos[2], t->count[1], t->wl_aux, 256, 32, 4096, 2048);
+    }
     if (t->fmt == SA_FMT_CSF && t->order == 4) build_ttm4(t, t->wl_main, t->wl_aux);
     if (t->fmt == SA_FMT_CSR) {
-        build_csr(t, t->wl_main, 256, 32, 1024, 512);    // fused SDDMM -> SpMM
-        build_csr(t, t->wl_aux, 256, 16, 4096, 2048);    // SpMM -> GEMM (both orders)
+        build_rows(t->pos[1], t->dims[0], t->wl_main, 256, 32, 1024, 512);    // fused SDDMM -> SpMM
+        build_rows(t->pos[1], t->dims[0], t->wl_aux, 256, 16, 4096, 2048);    // SpMM -> GEMM (both orders)
     }
 }

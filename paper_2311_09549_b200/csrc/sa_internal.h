@@ -161,6 +161,12 @@ bool sa_dense_gemm_tc_ok(int64_t L, int64_t M);
 sa_status sa_launch_dense_gemm_tc(int64_t rows, const float *A, int64_t lda, const float *B, int64_t ldb, int64_t L,
                                   int64_t M, float *out, int32_t *status, cudaStream_t stream);
 
+// Kernel 7 <SpTTM,SpTTM>: out = one row of M values per (i,j) fiber, in CSF order
+bool sa_ranks_ok_spttm_spttm(int64_t L, int64_t M);
+size_t sa_ws_spttm_spttm(const sa_tensor *t, const sa_dense *ops, bool right);
+sa_status sa_launch_spttm_spttm(const sa_tensor *t, const sa_dense *ops, float *out, void *ws, size_t ws_bytes, bool right,
+                                cudaStream_t stream, int *launches);
+
 // Kernel 8 <MTTKRP,GEMM>
 sa_status sa_launch_mttkrp_gemm(const sa_tensor *t, const sa_dense *ops, float *out, void *ws, size_t ws_bytes,
                                 cudaStream_t stream, int *launches);

@@ -260,7 +260,7 @@ gemm_bf16x3_kernel(int64_t J, const float *__restrict__ C, int64_t ldc, const fl
 template <int MV>
 __global__ void __launch_bounds__(256)
 spmm_kernel(const sa_item *__restrict__ items, int64_t n_items, const int32_t *__restrict__ pos,
-            const int32_t *__restrict__ crd, const float *__restrict__ vals, const float *__restrict__ E,
+            const int32_t *__restrict__ crd, const float *__restrict__ vals, const float *__restrict__ E, int64_t lde,
             float *__restrict__ out, float *__restrict__ partial)
 {
     constexpr int M = MV * 32;
@@ -283,7 +283,7 @@ spmm_kernel(const sa_item *__restrict__ items, int64_t n_items, const int32_t *_
             for (int s = 0; s < n; ++s) {
                 const int j = __shfl_sync(SA_FULL_MASK, jj, s);
                 const float v = __shfl_sync(SA_FULL_MASK, vv, s);
-                const float *erow = E + int64_t(j) * M + lane * MV;
+                const float *erow = E + int64_t(j) * lde + lane * MV;
                 if (MV == 2) {
                     const float2 e = sa_ldg2(erow);
                     acc[0] = fmaf(v, e.x, acc[0]);
@@ -341,7 +341,7 @@ sa_status run(const sa_tensor *t, const sa_dense *ops, float *out, void *ws, boo
     *launches += 1;
     const int64_t ctas = (n_items + SA_WARPS_PER_CTA - 1) / SA_WARPS_PER_CTA;
     if (ctas > 0) {
-        spmm_kernel<M / 32><<<(unsigned)ctas, 256, 0, stream>>>(wl.d_items, n_items, t->d_pos[1], t->d_crd[1], t->d_vals, E,
+        spmm_kernel<M / 32><<<(unsigned)ctas, 256, 0, stream>>>(wl.d_items, n_items, t->d_pos[1], t->d_crd[1], t->d_vals, E, M,
                                                                out, partial);
         if (cudaGetLastError() != cudaSuccess) return SA_E_CUDA;
         *launches += 1;
@@ -376,6 +376,54 @@ sa_status run_hadamard(const sa_tensor *t, const sa_dense *ops, float *out, void
         if (sa_launch_fixup(wl, partial, out, M, stream) != cudaSuccess) return SA_E_CUDA;
         *launches += 1;
     }
+    return SA_OK;
+}
+
+// Kernel 7 <SpTTM,SpTTM>: A(i,j,m) = sum_{k,l} B(i,j,k) C(k,l) D(l,m), one row of M values per (i,j) fiber of B
+// (the output has B's level-2 pattern).  Seen from the fibers, B is a sparse matrix B' with one row per fiber
+// and the chain is <SpMM,GEMM> on it: `right` = B'.(C.D), else (B'.C).D with the fiber temporaries T(f,:)
+// (the t of the paper's nest, widened to a vector and kept for the dense stage) in the workspace.
+template <int L, int M>
+sa_status run_fibers(const sa_tensor *t, const sa_dense *ops, float *out, void *ws, bool right, cudaStream_t stream, int *launches)
+{
+    const sa_worklist &wl = t->wl_aux;
+    const int64_t n_items = int64_t(wl.items.size());
+    const int64_t F2 = t->count[1], K = t->dims[2];
+    const int64_t ctas = (n_items + SA_WARPS_PER_CTA - 1) / SA_WARPS_PER_CTA;
+    *launches = 0;
+    if (right) {
+        float *E = static_cast<float *>(ws);
+        float *partial = reinterpret_cast<float *>(static_cast<char *>(ws) + sa_align256(size_t(K) * M * sizeof(float)));
+        const sa_status gs = sa_launch_dense_gemm(K, ops[0].ptr, ops[0].ld, ops[1].ptr, ops[1].ld, L, M, E, t->d_status, stream);
+        if (gs != SA_OK) return gs;
+        *launches += 1;
+        if (ctas > 0) {
+            spmm_kernel<M / 32><<<(unsigned)ctas, 256, 0, stream>>>(wl.d_items, n_items, t->d_pos[2], t->d_crd[2], t->d_vals, E, M,
+                                                                   out, partial);
+            if (cudaGetLastError() != cudaSuccess) return SA_E_CUDA;
+            *launches += 1;
+        }
+        if (!wl.fix.empty()) {
+            if (sa_launch_fixup(wl, partial, out, M, stream) != cudaSuccess) return SA_E_CUDA;
+            *launches += 1;
+        }
+        return SA_OK;
+    }
+    float *T = static_cast<float *>(ws);
+    float *partial = reinterpret_cast<float *>(static_cast<char *>(ws) + sa_align256(size_t(F2) * L * sizeof(float)));
+    if (ctas > 0) {
+        spmm_kernel<L / 32><<<(unsigned)ctas, 256, 0, stream>>>(wl.d_items, n_items, t->d_pos[2], t->d_crd[2], t->d_vals,
+                                                               ops[0].ptr, ops[0].ld, T, partial);
+        if (cudaGetLastError() != cudaSuccess) return SA_E_CUDA;
+        *launches += 1;
+    }
+    if (!wl.fix.empty()) {
+        if (sa_launch_fixup(wl, partial, T, L, stream) != cudaSuccess) return SA_E_CUDA;
+        *launches += 1;
+    }
+    const sa_status gs = sa_launch_dense_gemm(F2, T, L, ops[1].ptr, ops[1].ld, L, M, out, t->d_status, stream);
+    if (gs != SA_OK) return gs;
+    *launches += 1;
     return SA_OK;
 }
 
@@ -442,5 +490,26 @@ sa_status sa_launch_spmmh_gemm(const sa_tensor *t, const sa_dense *ops, float *o
     if (L == 128 && M == 64) return run_hadamard<128, 64>(t, ops, out, ws, stream, launches);
     if (L == 256 && M == 32) return run_hadamard<256, 32>(t, ops, out, ws, stream, launches);
     if (L == 256 && M == 64) return run_hadamard<256, 64>(t, ops, out, ws, stream, launches);
+    return SA_E_UNSUPPORTED;
+}
+
+bool sa_ranks_ok_spttm_spttm(int64_t L, int64_t M) { return (L == 32 || L == 64) && (M == 32 || M == 64); }
+
+// workspace: right [E = C.D, K x M][partial rows of M]; else [T, one row of L per fiber][partial rows of L]
+size_t sa_ws_spttm_spttm(const sa_tensor *t, const sa_dense *ops, bool right)
+{
+    const size_t L = size_t(ops[0].cols), M = size_t(ops[1].cols);
+    if (right) return sa_align256(size_t(t->dims[2]) * M * sizeof(float)) + sa_align256(size_t(t->wl_aux.n_slots) * M * sizeof(float));
+    return sa_align256(size_t(t->count[1]) * L * sizeof(float)) + sa_align256(size_t(t->wl_aux.n_slots) * L * sizeof(float));
+}
+
+sa_status sa_launch_spttm_spttm(const sa_tensor *t, const sa_dense *ops, float *out, void *ws, size_t, bool right,
+                                cudaStream_t stream, int *launches)
+{
+    const int64_t L = ops[0].cols, M = ops[1].cols;
+    if (L == 32 && M == 32) return run_fibers<32, 32>(t, ops, out, ws, right, stream, launches);
+    if (L == 32 && M == 64) return run_fibers<32, 64>(t, ops, out, ws, right, stream, launches);
+    if (L == 64 && M == 32) return run_fibers<64, 32>(t, ops, out, ws, right, stream, launches);
+    if (L == 64 && M == 64) return run_fibers<64, 64>(t, ops, out, ws, right, stream, launches);
     return SA_E_UNSUPPORTED;
 }

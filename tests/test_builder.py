@@ -298,3 +298,41 @@ def test_default_association_order_follows_the_byte_cost_model():
     ops = [(16, w.dims[1], 256, 256), (16, 256, 64, 64)]
     assert (sa.sa_workspace_size(dense.handle, sa.SA_EXPR_SPMM_GEMM, sa.SA_SCHED_DEFAULT, ops)
             == sa.sa_workspace_size(dense.handle, sa.SA_EXPR_SPMM_GEMM, sa.SA_SCHED_ASSOC_RIGHT, ops))
+
+
+def test_fiber_row_worklist_of_order3_csf_partitions_fibers_and_nonzeros():
+    """Kernel 7 walks an order-3 CSF tensor as a sparse matrix with one row per (i,j) fiber: its work list
+    (the second one of the tensor) covers every fiber and every nonzero once; a fiber longer than 4096
+    nonzeros is cut into pieces with partial rows."""
+    w = configs.make(10, "mini")
+    longf = np.stack([np.full(5000, 7), np.full(5000, 3), np.arange(5000)], axis=1).astype(np.int32)
+    base = w.coords[~((w.coords[:, 0] == 7) & (w.coords[:, 1] == 3))]
+    dims = (w.dims[0], w.dims[1], 5000)
+    coords = np.concatenate([base, longf])
+    vals = np.ones(coords.shape[0], np.float32)
+    t = sa.SparseTensor(dims, coords, vals, sa.SA_FMT_CSF, device=-1)
+    levels, _ = export_all(t, "csf")
+    pos = levels[2][0]
+    n_fibers = int(t.info()[1][1])
+    counts, items, fix = sa.sa_tensor_worklist(t.handle, 1)
+    covered = np.zeros(coords.shape[0], dtype=np.int32)
+    rows = np.zeros(n_fibers, dtype=np.int32)
+    for row, row_end, _, _, p0, p1, dest, _ in items:
+        if dest >= 0:
+            assert row_end == row + 1 and pos[row] <= p0 < p1 <= pos[row + 1]
+        else:
+            assert (p0, p1) == (pos[row], pos[row_end])
+            rows[row:row_end] += 1
+        covered[p0:p1] += 1
+    assert (covered == 1).all()
+    assert len(fix) == 1 and fix[0][2] == 3          # 5000 nonzeros in pieces of 2048
+    for row, slot0, count, _ in fix:
+        assert pos[row + 1] - pos[row] == 5000
+        rows[row] += 1
+    assert (rows == 1).all()
+    # default order: with rank-32 matrices B'.(C.D) moves fewer bytes unless the mode-3 dimension dwarfs the nonzeros
+    ops = [(16, dims[2], 32, 32), (16, 32, 32, 32)]
+    ws = {s: sa.sa_workspace_size(t.handle, sa.SA_EXPR_SPTTM_SPTTM, s, ops)
+          for s in (sa.SA_SCHED_DEFAULT, sa.SA_SCHED_FUSED, sa.SA_SCHED_ASSOC_LEFT, sa.SA_SCHED_ASSOC_RIGHT)}
+    assert ws[sa.SA_SCHED_FUSED] == ws[sa.SA_SCHED_ASSOC_LEFT] >= n_fibers * 32 * 4
+    assert ws[sa.SA_SCHED_DEFAULT] == ws[sa.SA_SCHED_ASSOC_RIGHT] >= dims[2] * 32 * 4

@@ -227,3 +227,31 @@ def test_workspace_errors_enqueue_nothing(sa):
     torch.cuda.synchronize()
     assert not out.any()
     assert sa.sa_last_device_status(t.handle, s) == sa.SA_OK
+
+
+@pytest.mark.parametrize("L,M", [(32, 32), (32, 64), (64, 32), (64, 64)])
+@pytest.mark.parametrize("sched", ["left", "right"])
+def test_spttm_spttm_ranks_long_fibers_and_empty_slices(sa, L, M, sched):
+    # short fibers, empty slices, and one fiber of 9000 nonzeros that is cut into pieces with partial rows
+    dims = (40, 37, 9500)
+    coords, vals = _random_coo(11, dims, 6000)
+    keep = coords[:, 0] % 3 != 1
+    longf = np.stack([np.full(9000, 6), np.full(9000, 3), np.arange(9000)], axis=1).astype(np.int32)
+    keep &= ~((coords[:, 0] == 6) & (coords[:, 1] == 3))
+    c = np.concatenate([coords[keep], longf])
+    v = np.concatenate([vals[keep], rng.uniform_f32(12, 1, np.arange(9000), -1.0, 1.0)])
+    perm = rng.permutation(13, 3, c.shape[0])
+    keys, _ = oracle.fiber_keys(c, dims)
+    w = _wl("spttm_spttm", "csf", dims, c[perm], v[perm], [_dense(6, 0, 9500, L), _dense(6, 1, L, M)], (keys.shape[0], M))
+    s = sa.SA_SCHED_ASSOC_LEFT if sched == "left" else sa.SA_SCHED_ASSOC_RIGHT
+    A, t = _check(sa, w, sched=s)
+    assert A.shape == (keys.shape[0], M)
+    assert sa.sa_tensor_worklist(t.handle, 1)[0][3] >= 1, "the long fiber must be split into pieces with partial rows"
+
+
+@pytest.mark.parametrize("nnz", [0, 1])
+def test_spttm_spttm_empty_and_single_entry(sa, nnz):
+    w = _wl("spttm_spttm", "csf", (5, 4, 3), [[3, 2, 1]][:nnz], [0.5][:nnz], [_dense(1, 0, 3, 32), _dense(1, 1, 32, 64)], (nnz, 64))
+    for s in (sa.SA_SCHED_ASSOC_LEFT, sa.SA_SCHED_ASSOC_RIGHT):
+        A, _ = _check(sa, w, sched=s)
+        assert A.shape == (nnz, 64)

@@ -153,3 +153,22 @@ def test_cfg9_mttkrp_gemm_full_sampled(sa):
     assert not bool(out[empty].any()), "empty slices must be +0"
     del out, t
     torch.cuda.empty_cache()
+
+
+def test_cfg10_spttm_spttm_full_sampled(sa):
+    """Kernel 7 on the config-2 tensor: sampled fibers (the longest, the shortest, seeded others) against the
+    oracle, and the number of output rows against the number of distinct (i,j) pairs."""
+    import torch
+    w = configs.make(10, "full")
+    out, t = _run_full(sa, w)
+    keys, inv = oracle.fiber_keys(w.coords, w.dims)
+    assert tuple(out.shape) == (keys.shape[0], 32)
+    lens = np.bincount(inv, minlength=keys.shape[0])
+    sel = np.unique(np.concatenate([[int(np.argmax(lens)), int(np.argmin(lens))],
+                                    configs.rng.permutation(w.seed, 57, keys.shape[0])[:4000]])).astype(np.int64)
+    A_ref, S_ref = oracle.evaluate(w, sel=sel)
+    got = out[torch.from_numpy(sel).cuda()].cpu().numpy().astype(np.float64)
+    assert_close(got, A_ref, S_ref, TOL_FP32, w.name)
+    assert bool(torch.isfinite(out).all())
+    del out, t
+    torch.cuda.empty_cache()

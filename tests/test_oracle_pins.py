@@ -413,3 +413,59 @@ def test_mttkrp_gemm_bruteforce_special_cases_and_invariants():
     sel = np.array([3, 0], dtype=np.int64)
     As, Ss = oracle.mttkrp_gemm(coords, vals, dims, C, D, E, sel=sel)
     assert np.array_equal(As, A[sel]) and np.array_equal(Ss, S[sel])
+
+
+# ----------------------------------------------------------------- kernel 7 <SpTTM,SpTTM>
+
+def test_spttm_spttm_bruteforce_pattern_special_cases_and_invariants():
+    """A(i,j,m) = sum_{k,l} B(i,j,k) C(k,l) D(l,m), stored for B's (i,j) pairs (Table of kernels, row 7)."""
+    rs = np.random.RandomState(37)
+    dims = (5, 4, 6)
+    coords, vals = tiny_coo(rs, dims, 40)
+    C, D = dense(rs, 6, 3), dense(rs, 3, 2)
+    keys, inv = oracle.fiber_keys(coords, dims)
+    A, S = oracle.spttm_spttm(coords, vals, dims, C, D)
+    B = densify(coords, vals, dims)
+    # pattern: exactly the (i,j) pairs with a stored nonzero, in lexicographic order, each once
+    want = sorted({(int(i), int(j)) for i, j, _ in coords})
+    assert [tuple(k) for k in keys.tolist()] == want and A.shape == (len(want), 2)
+    assert np.array_equal(keys[inv], coords[:, :2])
+    # brute force over the dense tensor, term by term
+    ref = np.zeros((5, 4, 2))
+    for i, j, k, l, m in itertools.product(range(5), range(4), range(6), range(3), range(2)):
+        ref[i, j, m] += B[i, j, k] * float(C[k, l]) * float(D[l, m])
+    np.testing.assert_allclose(A, ref[keys[:, 0], keys[:, 1]], rtol=0, atol=1e-13)
+    C64, D64 = C.astype(np.float64), D.astype(np.float64)
+    full = np.einsum("ijk,kl,lm->ijm", B, C64, D64)
+    np.testing.assert_allclose(A, full[keys[:, 0], keys[:, 1]], rtol=0, atol=1e-13)
+    np.testing.assert_allclose(S, np.einsum("ijk,kl,lm->ijm", np.abs(B), np.abs(C64), np.abs(D64))[keys[:, 0], keys[:, 1]],
+                               rtol=0, atol=1e-13)
+    # pairs outside the pattern hold no term at all: the dense result is zero there
+    mask = np.zeros((5, 4), dtype=bool)
+    mask[keys[:, 0], keys[:, 1]] = True
+    assert not full[~mask].any()
+    # both association orders of the two mode products give the same numbers
+    np.testing.assert_allclose(A, (np.einsum("ijk,kl->ijl", B, C64) @ D64)[keys[:, 0], keys[:, 1]], rtol=0, atol=1e-13)
+    np.testing.assert_allclose(A, np.einsum("ijk,km->ijm", B, C64 @ D64)[keys[:, 0], keys[:, 1]], rtol=0, atol=1e-13)
+    # D = identity: the first SpTTM alone, T(i,j,l) = sum_k B(i,j,k) C(k,l)
+    Ai, _ = oracle.spttm_spttm(coords, vals, dims, C, np.eye(3, dtype=np.float32))
+    np.testing.assert_allclose(Ai, np.einsum("ijk,kl->ijl", B, C64)[keys[:, 0], keys[:, 1]], rtol=0, atol=1e-13)
+    # all ones: A(i,j,m) = L * (number of nonzeros of the fiber), and S equals A
+    Ao, So = oracle.spttm_spttm(coords, np.ones(40, np.float32), dims, np.ones((6, 3), np.float32), np.ones((3, 2), np.float32))
+    cnt = np.bincount(inv, minlength=keys.shape[0])
+    assert np.array_equal(Ao, np.broadcast_to(3.0 * cnt[:, None], Ao.shape)) and np.array_equal(Ao, So)
+    # swapping the operands' roles is a different expression (C is indexed by k, not by l)
+    # linearity in B, invariance under the COO order, subset mode
+    A4, _ = oracle.spttm_spttm(coords, 4.0 * vals, dims, C, D)
+    np.testing.assert_allclose(A4, 4.0 * A, rtol=0, atol=1e-12)
+    perm = rs.permutation(40)
+    Ap, _ = oracle.spttm_spttm(coords[perm], vals[perm], dims, C, D)
+    np.testing.assert_allclose(Ap, A, rtol=0, atol=1e-13)
+    sel = np.array([7, 0, 3], dtype=np.int64)
+    As, Ss = oracle.spttm_spttm(coords, vals, dims, C, D, sel=sel)
+    np.testing.assert_allclose(As, A[sel], rtol=0, atol=1e-14)
+    np.testing.assert_allclose(Ss, S[sel], rtol=0, atol=1e-14)
+    with pytest.raises(ValueError):
+        bad = coords.copy()
+        bad[0, 2] = 6
+        oracle.spttm_spttm(bad, vals, dims, C, D)

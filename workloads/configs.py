@@ -412,4 +412,16 @@ def make(config, scale="full", seed=None):
         E = dense_uniform(s, 2, 32, 32)
         return Workload("cfg9-mttkrp-gemm" + ("" if full else "-mini"), "mttkrp_gemm", "csf", w.dims, w.coords, w.vals,
                         w.dense + [E], (w.dims[0], 32), s, w.notes)
-    raise ValueError("config must be 1..9")
+    if config == 10:
+        # kernel 7 (SpTTM, SpTTM): the tensor of config 2, C = 80000 x 32 (rows by k), D = 32 x 32; the output has
+        # one row of 32 values per (i,j) fiber of B
+        if full:
+            w = make_ttm3_zipf("tmp", s, 100000, 80000, 80000, 50_000_000, 1.2, 8.0, 32, 32)
+        else:
+            w = make_ttm3_zipf("tmp", s, 2500, 600, 800, 200_000, 1.2, 8.0, 32, 32)
+        D = dense_uniform(s, 2, 32, 32)
+        key = w.coords[:, 0].astype(np.int64) * int(w.dims[1]) + w.coords[:, 1]
+        f2 = int(np.unique(key).shape[0])
+        return Workload("cfg10-spttm-spttm" + ("" if full else "-mini"), "spttm_spttm", "csf", w.dims, w.coords, w.vals,
+                        [w.dense[1], D], (f2, 32), s, w.notes)
+    raise ValueError("config must be 1..10")
