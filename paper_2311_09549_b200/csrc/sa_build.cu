@@ -378,7 +378,7 @@ void sa_build_worklists(sa_tensor *t)
     if (t->fmt == SA_FMT_CSF && t->order == 3) {
         build_ttm3(t, t->wl_main);
         // kernel 7 walks the tensor as a sparse matrix whose rows are the (i,j) fibers
-        build_rows(t->pos[2], t->count[1], t->wl_aux, 256, 32, 4096, 2048);
+        build_rows(t->pos[2], t->count[1], t->wl_aux, 1024, 4096, 4096, 2048);
     }
     if (t->fmt == SA_FMT_CSF && t->order == 4) build_ttm4(t, t->wl_main, t->wl_aux);
     if (t->fmt == SA_FMT_CSR) {

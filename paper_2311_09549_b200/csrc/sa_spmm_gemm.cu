@@ -299,6 +299,92 @@ spmm_kernel(const sa_item *__restrict__ items, int64_t n_items, const int32_t *_
     }
 }
 
+// The same product over the (i,j) fibers of an order-3 CSF tensor (kernel 7; eight to twelve nonzeros per
+// fiber): M/4 lanes own a row of E as one float4 each, so a warp works on 128/M fibers' streams at once, one
+// nonzero per group and step.  A group takes a contiguous share of the item's fibers and walks their nonzeros
+// as one stream, eight index/value pairs per load (the next eight already requested), eight row gathers in
+// flight; the end-of-fiber bit of a nonzero travels in the sign bit of its index and closes the output row.
+// A piece of a long fiber (dest >= 0) is split over the groups by nonzeros and summed across them at the end.
+template <int M>
+__global__ void __launch_bounds__(256)
+fiber_spmm_kernel(const sa_item *__restrict__ items, int64_t n_items, const int32_t *__restrict__ pos,
+                  const int32_t *__restrict__ crd, const float *__restrict__ vals, const uint32_t *__restrict__ endbits,
+                  const float *__restrict__ E, int64_t lde, float *__restrict__ out, float *__restrict__ partial)
+{
+    constexpr int LPR = M / 4, NG = 32 / LPR;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t idx = int64_t(blockIdx.x) * SA_WARPS_PER_CTA + warp;
+    if (idx >= n_items) return;
+    const sa_item it = items[idx];
+    const int g = lane / LPR, l = lane % LPR;
+    const bool piece = it.dest >= 0;
+    int ga, gb, row = 0;
+    if (piece) {
+        const int64_t len = it.p1 - it.p0;
+        ga = it.p0 + int(len * g / NG);
+        gb = it.p0 + int(len * (g + 1) / NG);
+    } else {
+        const int nr = it.row_end - it.out_row;
+        row = it.out_row + nr * g / NG;
+        ga = __ldg(pos + row);
+        gb = __ldg(pos + it.out_row + nr * (g + 1) / NG);
+    }
+    const int mylen = gb - ga;
+    const int maxlen = __reduce_max_sync(SA_FULL_MASK, mylen);
+    auto fetch = [&](int c, int &x, float &v) {                      // lanes 0..7 of the group: nonzero ga + c + lane
+        const int p = ga + c + (l & 7);
+        x = 0;
+        v = 0.f;
+        if (c + (l & 7) < mylen) {
+            x = __ldg(crd + p);
+            v = __ldg(vals + p);
+            if (!piece) x |= int(((__ldg(endbits + (p >> 5)) >> (p & 31)) & 1u) << 31);
+        }
+    };
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    int xn;
+    float vn;
+    fetch(0, xn, vn);
+    for (int c = 0; c < maxlen; c += 8) {
+        const int x = xn;
+        const float v = vn;
+        fetch(c + 8, xn, vn);
+        int xs[8];
+        float vs[8];
+        float4 e[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {                                 // positions past the group's end: row 0, value 0
+            xs[u] = __shfl_sync(SA_FULL_MASK, x, u, LPR);
+            vs[u] = __shfl_sync(SA_FULL_MASK, v, u, LPR);
+            e[u] = sa_ldg4(E + int64_t(xs[u] & 0x7fffffff) * lde + 4 * l);
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            if (c + u < mylen) {
+                acc.x = fmaf(vs[u], e[u].x, acc.x);
+                acc.y = fmaf(vs[u], e[u].y, acc.y);
+                acc.z = fmaf(vs[u], e[u].z, acc.z);
+                acc.w = fmaf(vs[u], e[u].w, acc.w);
+            }
+            if (xs[u] < 0) {                                          // last nonzero of its fiber
+                *reinterpret_cast<float4 *>(out + int64_t(row) * M + 4 * l) = acc;
+                acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                ++row;
+            }
+        }
+    }
+    if (piece) {
+#pragma unroll
+        for (int off = LPR; off < 32; off <<= 1) {
+            acc.x += __shfl_xor_sync(SA_FULL_MASK, acc.x, off);
+            acc.y += __shfl_xor_sync(SA_FULL_MASK, acc.y, off);
+            acc.z += __shfl_xor_sync(SA_FULL_MASK, acc.z, off);
+            acc.w += __shfl_xor_sync(SA_FULL_MASK, acc.w, off);
+        }
+        if (g == 0) *reinterpret_cast<float4 *>(partial + int64_t(it.dest) * M + 4 * l) = acc;
+    }
+}
+
 int resident_ctas(const void *kernel, size_t smem)
 {
     int dev = 0, sms = 148, per_sm = 1;
@@ -398,8 +484,8 @@ sa_status run_fibers(const sa_tensor *t, const sa_dense *ops, float *out, void *
         if (gs != SA_OK) return gs;
         *launches += 1;
         if (ctas > 0) {
-            spmm_kernel<M / 32><<<(unsigned)ctas, 256, 0, stream>>>(wl.d_items, n_items, t->d_pos[2], t->d_crd[2], t->d_vals, E, M,
-                                                                   out, partial);
+            fiber_spmm_kernel<M><<<(unsigned)ctas, 256, 0, stream>>>(wl.d_items, n_items, t->d_pos[2], t->d_crd[2], t->d_vals,
+                                                                    t->d_endbits, E, M, out, partial);
             if (cudaGetLastError() != cudaSuccess) return SA_E_CUDA;
             *launches += 1;
         }
@@ -412,8 +498,8 @@ sa_status run_fibers(const sa_tensor *t, const sa_dense *ops, float *out, void *
     float *T = static_cast<float *>(ws);
     float *partial = reinterpret_cast<float *>(static_cast<char *>(ws) + sa_align256(size_t(F2) * L * sizeof(float)));
     if (ctas > 0) {
-        spmm_kernel<L / 32><<<(unsigned)ctas, 256, 0, stream>>>(wl.d_items, n_items, t->d_pos[2], t->d_crd[2], t->d_vals,
-                                                               ops[0].ptr, ops[0].ld, T, partial);
+        fiber_spmm_kernel<L><<<(unsigned)ctas, 256, 0, stream>>>(wl.d_items, n_items, t->d_pos[2], t->d_crd[2], t->d_vals,
+                                                                t->d_endbits, ops[0].ptr, ops[0].ld, T, partial);
         if (cudaGetLastError() != cudaSuccess) return SA_E_CUDA;
         *launches += 1;
     }
