@@ -280,6 +280,7 @@ sa_status sa_tensor_create(int order, const int64_t *dims, int64_t nnz, const in
         if (s == SA_OK) s = upload(t, zeros, 4, &t->d_status);
         if (s == SA_OK) s = upload_worklist(t, t->wl_main);
         if (s == SA_OK) s = upload_worklist(t, t->wl_aux);
+        if (s == SA_OK) s = upload_worklist(t, t->wl_sub);
         if (s == SA_OK && cudaDeviceSynchronize() != cudaSuccess) s = SA_E_CUDA;
         if (s == SA_E_CUDA) cudaGetLastError();
     }
@@ -312,8 +313,8 @@ sa_status sa_tensor_export(const sa_tensor *t, int level, int64_t *pos, int32_t 
 
 sa_status sa_tensor_worklist(const sa_tensor *t, int which, int64_t *counts, int32_t *items, int32_t *fix)
 {
-    if (!t || which < 0 || which > 1) return SA_E_ARG;
-    const sa_worklist &wl = which == 0 ? t->wl_main : t->wl_aux;
+    if (!t || which < 0 || which > 2) return SA_E_ARG;
+    const sa_worklist &wl = which == 0 ? t->wl_main : which == 1 ? t->wl_aux : t->wl_sub;
     if (counts) {
         counts[0] = int64_t(wl.items.size());
         counts[1] = wl.n_group_ctas;

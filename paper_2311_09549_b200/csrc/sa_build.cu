@@ -194,14 +194,15 @@ void append_empty_slices(sa_tensor *t, sa_worklist &wl)
 // `n_slices` slices; slice s is output row row_of(s), owns the fibers [pos1[s], pos1[s + 1]) whose nonzeros are
 // [pos2[f], pos2[f + 1]).  (Order 3: the slices of the tensor.  Order 4: the (i,j) subtrees, whose "fibers" are
 // the (i,j,k) fibers; output row = index of the (i,j) fiber.)
-template <typename RowOf>
-void build_ttm3_lists(sa_worklist &wl, int64_t n_slices, RowOf row_of, const std::vector<int64_t> &pos1,
+template <typename RowOf, typename Skip>
+void build_ttm3_lists(sa_worklist &wl, int64_t n_slices, RowOf row_of, Skip skip, const std::vector<int64_t> &pos1,
                       const std::vector<int64_t> &pos2)
 {
     constexpr int64_t SMALL_MAX = 2048, MIN_CHUNK = 8192, MAX_PARTS = 192, MAX_UNITS = 16;
     std::vector<sa_item> small;
     std::vector<group_rec> groups;
     for (int64_t s = 0; s < n_slices; ++s) {
+        if (skip(s)) continue;                    // evaluated by another kernel
         const int64_t fa = pos1[size_t(s)], fb = pos1[size_t(s) + 1];
         const int64_t pa = pos2[size_t(fa)], pb = pos2[size_t(fb)];
         const int64_t n = pb - pa;
@@ -281,19 +282,29 @@ void build_ttm3_lists(sa_worklist &wl, int64_t n_slices, RowOf row_of, const std
 
 void build_ttm3(sa_tensor *t, sa_worklist &wl)
 {
-    build_ttm3_lists(wl, t->count[0], [&](int64_t s) { return t->crd[0][size_t(s)]; }, t->pos[1], t->pos[2]);
+    build_ttm3_lists(wl, t->count[0], [&](int64_t s) { return t->crd[0][size_t(s)]; }, [](int64_t) { return false; }, t->pos[1],
+                     t->pos[2]);
     append_empty_slices(t, wl);
 }
 
 
+// A subtree (i,j) that the subtree kernel of pass 1 can take whole.
+static bool subtree_is_small(const sa_tensor *t, int64_t f2)
+{
+    const auto &pos2 = t->pos[2], &pos3 = t->pos[3];
+    const int64_t fa = pos2[size_t(f2)], fb = pos2[size_t(f2) + 1];
+    return fb - fa <= SA_SUB_MAX_F3 && pos3[size_t(fb)] - pos3[size_t(fa)] <= SA_SUB_MAX_NNZ;
+}
+
 // Order-4 CSF.  The chain is evaluated in two passes (see sa_ttm4.cu).  Pass 1 runs the order-3 kernel with
-// the (i,j) subtrees as slices: `wl` gets the same lists as an order-3 tensor whose slices are the level-1
-// fibers (output row = fiber index).  Pass 2 contracts the per-fiber temporaries of each slice with rows of
+// the large (i,j) subtrees as slices: `wl` gets the same lists as an order-3 tensor whose slices are those
+// level-1 fibers (output row = fiber index); the small subtrees go to the subtree kernel's list.  Pass 2 contracts the per-fiber temporaries of each slice with rows of
 // C: `wl2` holds one item per (piece of a slice, quarter of the 256 temporaries' columns); a slice with more
 // than CHUNK_F fibers is cut into pieces whose partial tiles the fix-up kernel sums.
 void build_ttm4(sa_tensor *t, sa_worklist &wl, sa_worklist &wl2)
 {
-    build_ttm3_lists(wl, t->count[1], [](int64_t f) { return int32_t(f); }, t->pos[2], t->pos[3]);
+    build_ttm3_lists(wl, t->count[1], [](int64_t f) { return int32_t(f); }, [&](int64_t f) { return subtree_is_small(t, f); },
+                     t->pos[2], t->pos[3]);
     constexpr int64_t CHUNK_F = 512;
     const auto &pos1 = t->pos[1];
     std::vector<sa_item> items;
@@ -323,6 +334,43 @@ void build_ttm4(sa_tensor *t, sa_worklist &wl, sa_worklist &wl2)
     wl2.items = std::move(items);
     wl2.n_group_ctas = 0;
     append_empty_slices(t, wl2);
+}
+
+// Order 4, pass 1 on whole (i,j) subtrees: items are ranges of consecutive small subtrees (subtree_is_small) with
+// at most SA_SUB_MAX_F3 level-2 fibers, SA_SUB_MAX_ROWS subtrees and about 1024 nonzeros (f0/f1 = the fibers,
+// p0/p1 = the nonzeros).  No subtree is cut, so there are no partial tiles; the large subtrees are in the main list.
+void build_ttm4_subtrees(sa_tensor *t, sa_worklist &wl)
+{
+    const auto &pos2 = t->pos[2], &pos3 = t->pos[3];
+    const int64_t F2 = t->count[1];
+    constexpr int64_t TARGET_NNZ = 1024;
+    auto nnz_at = [&](int64_t f2) { return pos3[size_t(pos2[size_t(f2)])]; };
+    std::vector<sa_item> items;
+    int64_t r0 = 0;
+    auto flush = [&](int64_t r1) {
+        if (r1 > r0) {
+            sa_item it = empty_item();
+            it.out_row = int32_t(r0); it.row_end = int32_t(r1);
+            it.f0 = int32_t(pos2[size_t(r0)]); it.f1 = int32_t(pos2[size_t(r1)]);
+            it.p0 = int32_t(nnz_at(r0)); it.p1 = int32_t(nnz_at(r1));
+            items.push_back(it);
+        }
+        r0 = r1;
+    };
+    for (int64_t r = 0; r < F2; ++r) {
+        if (!subtree_is_small(t, r)) {
+            flush(r);
+            r0 = r + 1;
+            continue;
+        }
+        if (r > r0 && (pos2[size_t(r) + 1] - pos2[size_t(r0)] > SA_SUB_MAX_F3 || r - r0 >= SA_SUB_MAX_ROWS ||
+                       nnz_at(r + 1) - nnz_at(r0) > TARGET_NNZ))
+            flush(r);
+    }
+    flush(F2);
+    for (const sa_item &it : items) wl.nnz += it.p1 - it.p0;
+    wl.items = std::move(items);
+    wl.n_group_ctas = 0;
 }
 
 // Rows of a sparse matrix given by its pos array: row ranges of about target_nnz nonzeros (at most max_rows rows); rows longer than
@@ -380,7 +428,11 @@ void sa_build_worklists(sa_tensor *t)
         // kernel 7 walks the tensor as a sparse matrix whose rows are the (i,j) fibers
         build_rows(t->pos[2], t->count[1], t->wl_aux, 1024, 4096, 4096, 2048);
     }
-    if (t->fmt == SA_FMT_CSF && t->order == 4) build_ttm4(t, t->wl_main, t->wl_aux);
+    if (t->fmt == SA_FMT_CSF && t->order == 4) {
+        build_ttm4(t, t->wl_main, t->wl_aux);
+        build_ttm4_subtrees(t, t->wl_sub);
+        t->wl_main.nnz = t->nnz - t->wl_sub.nnz;
+    }
     if (t->fmt == SA_FMT_CSR) {
         build_rows(t->pos[1], t->dims[0], t->wl_main, 256, 32, 1024, 512);    // fused SDDMM -> SpMM
         build_rows(t->pos[1], t->dims[0], t->wl_aux, 256, 16, 4096, 2048);    // SpMM -> GEMM (both orders)

@@ -68,6 +68,7 @@ struct sa_worklist {
     std::vector<sa_fix> fix;
     int64_t n_group_ctas = 0;     // leading CTAs whose 8 warps reduce into one tile
     int64_t n_slots = 0;          // partial tiles in the workspace
+    int64_t nnz = 0;              // nonzeros the list covers (set for the order-4 lists of pass 1)
     sa_item *d_items = nullptr;
     sa_fix *d_fix = nullptr;
     // order-3 CSF: warp w evaluates items [task_start[w], task_start[w + 1]); the first
@@ -102,11 +103,19 @@ struct sa_tensor {
     int32_t *d_status = nullptr;              // [4] device status word
 
     sa_worklist wl_main;                      // TTM3 / pass 1 of TTM4 / SDDMM-SpMM
-    sa_worklist wl_aux;                       // CSR: SpMM-GEMM row items; order-4 CSF: pass 2 of TTM4
+    sa_worklist wl_aux;                       // CSR: SpMM-GEMM row items; order-3 CSF: fiber rows (kernel 7); order-4 CSF: pass 2 of TTM4
+    sa_worklist wl_sub;                       // order-4 CSF: ranges of whole (i,j) subtrees for the subtree kernel of pass 1;
+                                              // empty when some subtree exceeds SA_SUB_MAX_F3 fibers or SA_SUB_MAX_NNZ nonzeros
 
     mutable std::atomic<int> last_launches{0};   // the only mutable field: concurrent sa_run calls may write it
     std::vector<void *> dev_blocks;           // everything obtained from the allocator
 };
+
+// Limits of the order-4 subtree kernel: level-2 fibers an item parks in shared memory, rows (subtrees) per item,
+// nonzeros of one subtree.
+constexpr int SA_SUB_MAX_F3 = 128;
+constexpr int SA_SUB_MAX_ROWS = 32;
+constexpr int SA_SUB_MAX_NNZ = 4096;
 
 // ---- host builder (sa_build.cu)
 sa_status sa_build_levels(sa_tensor *t, const int32_t *coords, const float *vals);

@@ -122,6 +122,125 @@ ttm4_slice_kernel(const sa_item *__restrict__ items, int64_t n_items, const int3
     }
 }
 
+// Pass 1 on whole (i,j) subtrees (tensors whose subtrees are all small: the usual case, a subtree holds a few
+// dozen nonzeros).  One warp per item = a range of consecutive subtrees with at most SA_SUB_MAX_F3 level-2 fibers.
+//   Phase A (Q1):  t(f; n) = sum_o B(f; o) E(o,n) for every level-2 fiber f = (i,j,k) of the item.  Four lanes own a
+//     row of E as one float4 each, so the warp's eight lane groups walk separate shares of the item's fibers, one
+//     nonzero per group and step (index/value pairs eight per load and one load ahead, eight row gathers in
+//     flight); the end-of-fiber bit travels in the sign bit of the index and parks t(f; :) in the fiber's own slot
+//     of the warp's shared-memory tile, so the parked rows end up in fiber order without any bookkeeping.
+//   Phase B (Q2):  T2(m,n) += D(k_f, m) t(f; n) over the fibers of each subtree, in order; the 16 x 16 tile is
+//     spread over the warp (lane = two rows m, four columns n), control flow is uniform, and the tile is stored
+//     (1 KB, contiguous) when the subtree's last fiber has been added.
+// Against the order-3 kernel on the same subtrees this drops the per-unit pipeline drains and the padded
+// tensor-core groups: 16.7 M outer products of 256 FMAs are cheap on the ALUs next to 100 M row gathers.
+constexpr int SUB_SMEM = SA_WARPS_PER_CTA * SA_SUB_MAX_F3 * R * int(sizeof(float));   // 64 KB
+
+__global__ void __launch_bounds__(256)
+ttm4_subtree_kernel(const sa_item *__restrict__ items, int64_t n_items, const int32_t *__restrict__ pos2,
+                    const int32_t *__restrict__ pos3, const int32_t *__restrict__ crd_k, const int32_t *__restrict__ crd_o,
+                    const float *__restrict__ vals, const uint32_t *__restrict__ endbits, const float *__restrict__ D,
+                    int64_t ldd, const float *__restrict__ E, int64_t lde, float *__restrict__ T2)
+{
+    extern __shared__ __align__(16) float sub_smem[];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t idx = int64_t(blockIdx.x) * SA_WARPS_PER_CTA + warp;
+    if (idx >= n_items) return;
+    const sa_item it = items[idx];
+    float *pk = sub_smem + warp * (SA_SUB_MAX_F3 * R);
+    const int nf3 = it.f1 - it.f0;
+    {   // ---- phase A
+        const int g = lane >> 2, l = lane & 3;
+        const int fa = it.f0 + nf3 * g / 8, fb = it.f0 + nf3 * (g + 1) / 8;
+        const int ga = __ldg(pos3 + fa), gb = __ldg(pos3 + fb);
+        const int mylen = gb - ga;
+        const int maxlen = __reduce_max_sync(SA_FULL_MASK, mylen);
+        int slot = fa - it.f0;
+        auto fetch1 = [&](int q, int &x, float &v) {
+            x = 0;
+            v = 0.f;
+            if (q < mylen) {
+                const int p = ga + q;
+                x = __ldg(crd_o + p) | int(((__ldg(endbits + (p >> 5)) >> (p & 31)) & 1u) << 31);
+                v = __ldg(vals + p);
+            }
+        };
+        // lane l of the group holds nonzeros c + l and c + 4 + l of the group's stream
+        auto fetch = [&](int c, int (&x)[2], float (&v)[2]) {
+            fetch1(c + l, x[0], v[0]);
+            fetch1(c + 4 + l, x[1], v[1]);
+        };
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        int xn[2];
+        float vn[2];
+        fetch(0, xn, vn);
+        for (int c = 0; c < maxlen; c += 8) {
+            const int x[2] = {xn[0], xn[1]};
+            const float v[2] = {vn[0], vn[1]};
+            fetch(c + 8, xn, vn);
+            int xs[8];
+            float vs[8];
+            float4 e[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                xs[u] = __shfl_sync(SA_FULL_MASK, x[u >> 2], u & 3, 4);
+                vs[u] = __shfl_sync(SA_FULL_MASK, v[u >> 2], u & 3, 4);
+                e[u] = sa_ldg4(E + int64_t(xs[u] & 0x7fffffff) * lde + 4 * l);
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                if (c + u < mylen) {
+                    acc.x = fmaf(vs[u], e[u].x, acc.x);
+                    acc.y = fmaf(vs[u], e[u].y, acc.y);
+                    acc.z = fmaf(vs[u], e[u].z, acc.z);
+                    acc.w = fmaf(vs[u], e[u].w, acc.w);
+                }
+                if (xs[u] < 0) {                                      // last nonzero of fiber it.f0 + slot
+                    *reinterpret_cast<float4 *>(pk + slot * R + 4 * l) = acc;
+                    acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                    ++slot;
+                }
+            }
+        }
+    }
+    __syncwarp();
+    {   // ---- phase B
+        const int mp = lane >> 2, nq = lane & 3;
+        const int nr = it.row_end - it.out_row;
+        const int my_end = lane < nr ? __ldg(pos2 + it.out_row + lane + 1) - it.f0 : 0x7fffffff;   // local end of subtree `lane`
+        int r = 0, fe = __shfl_sync(SA_FULL_MASK, my_end, 0);
+        float4 a0 = make_float4(0.f, 0.f, 0.f, 0.f), a1 = a0;
+        for (int f0 = 0; f0 < nf3; f0 += 4) {
+            float2 d[4];
+            float4 tt[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int k = f0 + u < nf3 ? __ldg(crd_k + it.f0 + f0 + u) : 0;
+                d[u] = sa_ldg2(D + int64_t(k) * ldd + 2 * mp);
+                tt[u] = *reinterpret_cast<const float4 *>(pk + (f0 + u) * R + 4 * nq);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (f0 + u < nf3) {
+                    a0.x = fmaf(d[u].x, tt[u].x, a0.x); a0.y = fmaf(d[u].x, tt[u].y, a0.y);
+                    a0.z = fmaf(d[u].x, tt[u].z, a0.z); a0.w = fmaf(d[u].x, tt[u].w, a0.w);
+                    a1.x = fmaf(d[u].y, tt[u].x, a1.x); a1.y = fmaf(d[u].y, tt[u].y, a1.y);
+                    a1.z = fmaf(d[u].y, tt[u].z, a1.z); a1.w = fmaf(d[u].y, tt[u].w, a1.w);
+                    if (f0 + u + 1 == fe) {                           // the subtree's last fiber
+                        float *dst = T2 + int64_t(it.out_row + r) * T2F + (2 * mp) * R + 4 * nq;
+                        *reinterpret_cast<float4 *>(dst) = a0;
+                        *reinterpret_cast<float4 *>(dst + R) = a1;
+                        a0 = make_float4(0.f, 0.f, 0.f, 0.f);
+                        a1 = a0;
+                        ++r;
+                        fe = __shfl_sync(SA_FULL_MASK, my_end, r & 31);
+                    }
+                }
+            }
+        }
+    }
+}
+
 struct ttm4_plan {
     size_t t2_bytes, p1_bytes, p2_bytes;
 };
@@ -156,7 +275,7 @@ sa_status sa_launch_ttm4(const sa_tensor *t, const sa_dense *ops, float *out, vo
     float *T2 = reinterpret_cast<float *>(base);
     float *part1 = reinterpret_cast<float *>(base + p.t2_bytes);
     float *part2 = reinterpret_cast<float *>(base + p.t2_bytes + p.p1_bytes);
-    // pass 1: kernel 6 on the (i,j) subtrees, factors D (rows by k) and E (rows by o)
+    // the large subtrees: kernel 6 with the (i,j) subtrees as slices, factors D (rows by k) and E (rows by o)
     sa_ttm3_view v;
     v.wl = &t->wl_main;
     v.crd_fiber = t->d_crd[2];
@@ -165,12 +284,27 @@ sa_status sa_launch_ttm4(const sa_tensor *t, const sa_dense *ops, float *out, vo
     v.endbits = t->d_endbits;
     v.n_fibers = t->count[2];
     v.n_out_rows = t->count[1];
-    v.nnz = t->nnz;
+    v.nnz = t->wl_main.nnz;
     v.status = t->d_status;
-    int n1 = 0;
-    const sa_status s = sa_launch_ttm3_view(v, ops[1], ops[2], T2, part1, stream, &n1);
-    if (s != SA_OK) return s;
-    *launches = n1;
+    // pass 1: the small subtrees whole (subtree kernel), the large ones as slices of the order-3 kernel
+    const int64_t n_sub = int64_t(t->wl_sub.items.size());
+    *launches = 0;
+    if (n_sub > 0) {
+        if (cudaFuncSetAttribute(ttm4_subtree_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SUB_SMEM) != cudaSuccess)
+            return SA_E_CUDA;
+        const int64_t ctas = (n_sub + SA_WARPS_PER_CTA - 1) / SA_WARPS_PER_CTA;
+        ttm4_subtree_kernel<<<(unsigned)ctas, 256, SUB_SMEM, stream>>>(t->wl_sub.d_items, n_sub, t->d_pos[2], t->d_pos[3], t->d_crd[2],
+                                                                       t->d_crd[3], t->d_vals, t->d_endbits, ops[1].ptr, ops[1].ld,
+                                                                       ops[2].ptr, ops[2].ld, T2);
+        if (cudaGetLastError() != cudaSuccess) return SA_E_CUDA;
+        *launches += 1;
+    }
+    if (!t->wl_main.items.empty()) {
+        int n1 = 0;
+        const sa_status s = sa_launch_ttm3_view(v, ops[1], ops[2], T2, part1, stream, &n1);
+        if (s != SA_OK) return s;
+        *launches += n1;
+    }
     // pass 2
     const sa_worklist &wl = t->wl_aux;
     const int64_t n_items = int64_t(wl.items.size());

@@ -78,7 +78,17 @@ def test_csf_worklist_partitions_every_nonzero_once(cfg):
     """Main list of a CSF tensor: the units of the order-3 kernel.  For an order-4 tensor its "slices" are the
     (i,j) subtrees (output row = index of the level-1 fiber) and its fibers the (i,j,k) fibers."""
     w = configs.make(cfg, "mini")
-    t = sa.SparseTensor(w.dims, w.coords, w.vals, sa.SA_FMT_CSF, device=-1)
+    coords, vals = w.coords, w.vals
+    if cfg == 5:
+        # two (i,j) subtrees that the subtree kernel does not take (more than 4096 nonzeros), so that the main
+        # list of the order-4 tensor is not empty; all the others are in the third list
+        keep = ~(((coords[:, 0] == 3) & (coords[:, 1] == 5)) | ((coords[:, 0] == 200) & (coords[:, 1] == 7)))
+        k, o = np.divmod(np.arange(4800), 40)
+        extra = [np.stack([np.full(4800, i), np.full(4800, j), k, o], axis=1) for i, j in ((3, 5), (200, 7))]
+        coords = np.concatenate([coords[keep]] + extra).astype(np.int32)
+        vals = np.concatenate([vals[keep], np.ones(9600, np.float32)])
+    nnz_all = coords.shape[0]
+    t = sa.SparseTensor(w.dims, coords, vals, sa.SA_FMT_CSF, device=-1)
     levels, _ = export_all(t, "csf")
     counts, items, fix = sa.sa_tensor_worklist(t.handle)
     n_items, n_groups, n_fix, n_slots = (int(x) for x in counts)
@@ -88,7 +98,12 @@ def test_csf_worklist_partitions_every_nonzero_once(cfg):
         pos1, pos2 = levels[2][0], levels[3][0]
         slice_rows = np.arange(len(pos1) - 1)
     slice_pos = {int(c): n for n, c in enumerate(slice_rows)}
-    covered = np.zeros(w.nnz, dtype=np.int32)
+    covered = np.zeros(nnz_all, dtype=np.int32)
+    if t.order == 4:
+        sub = sa.sa_tensor_worklist(t.handle, 2)[1]
+        assert len(sub) > 0 and n_items > 0
+        for row, row_end, f0, f1, p0, p1, dest, _ in sub:
+            covered[p0:p1] += 1                  # the small subtrees are evaluated from the third list
     slot_owner = {}
     G = 4                                   # warps (tasks) per thread block of the order-3 kernel
     task_start, stream_f0 = sa.sa_tensor_tasks(t.handle)
@@ -130,7 +145,7 @@ def test_csf_worklist_partitions_every_nonzero_once(cfg):
         assert not empties, "every level-1 fiber has nonzeros"
     # nonzero balance: no unit is larger than the small-slice bound / the piece size
     sizes = items[:, 5] - items[:, 4]
-    assert sizes.max() <= max(4096, int(np.ceil(w.nnz / 8)))
+    assert sizes.max() <= max(4096, int(np.ceil(nnz_all / 8)))
     # tasks: a partition of the item list; group tasks hold at most one item and warp 0 of a group has one;
     # small-slice tasks hold at most 16 items and about 2048 nonzeros
     assert task_start[0] == 0 and task_start[-1] == n_items and (np.diff(task_start) >= 0).all()
@@ -336,3 +351,29 @@ def test_fiber_row_worklist_of_order3_csf_partitions_fibers_and_nonzeros():
           for s in (sa.SA_SCHED_DEFAULT, sa.SA_SCHED_FUSED, sa.SA_SCHED_ASSOC_LEFT, sa.SA_SCHED_ASSOC_RIGHT)}
     assert ws[sa.SA_SCHED_FUSED] == ws[sa.SA_SCHED_ASSOC_LEFT] >= n_fibers * 32 * 4
     assert ws[sa.SA_SCHED_DEFAULT] == ws[sa.SA_SCHED_ASSOC_RIGHT] >= dims[2] * 32 * 4
+
+
+def test_order4_subtree_worklist_covers_every_subtree_once_within_its_limits():
+    """Third list of an order-4 tensor: ranges of whole small (i,j) subtrees, at most 128 level-2 fibers and 32
+    subtrees each; a larger subtree is left to the main list."""
+    w = configs.make(5, "mini")
+    t = sa.SparseTensor(w.dims, w.coords, w.vals, sa.SA_FMT_CSF, device=-1)
+    levels, _ = export_all(t, "csf")
+    pos2, pos3 = levels[2][0], levels[3][0]
+    counts, items, fix = sa.sa_tensor_worklist(t.handle, 2)
+    assert counts[0] > 0 and counts[2] == 0 and counts[3] == 0
+    nxt = 0
+    for row, row_end, f0, f1, p0, p1, dest, _ in items:
+        assert row == nxt and row_end > row and dest < 0
+        assert (f0, f1) == (pos2[row], pos2[row_end]) and (p0, p1) == (pos3[f0], pos3[f1])
+        assert f1 - f0 <= 128 and row_end - row <= 32
+        nxt = row_end
+    assert nxt == int(t.info()[1][1])
+    assert sa.sa_tensor_worklist(t.handle, 0)[0][0] == 0, "no large subtree: the main list is empty"
+    # one (i,j) pair with 130 level-2 fibers next to a small one: the large one is in the main list only
+    big = np.stack([np.zeros(130), np.zeros(130), np.arange(130), np.zeros(130)], axis=1).astype(np.int32)
+    both = np.concatenate([big, np.array([[1, 1, 5, 1]], np.int32)])
+    t2 = sa.SparseTensor((2, 2, 130, 2), both, np.ones(131, np.float32), sa.SA_FMT_CSF, device=-1)
+    sub = sa.sa_tensor_worklist(t2.handle, 2)[1]
+    main = sa.sa_tensor_worklist(t2.handle, 0)[1]
+    assert [tuple(x[:2]) for x in sub.tolist()] == [(1, 2)] and set(main[:, 0].tolist()) == {0}

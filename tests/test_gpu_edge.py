@@ -200,6 +200,12 @@ def test_ttm4_ragged_and_split_slices(sa):
     w = configs.make_ttm4_zipf("edge4b", 32, 90, 700, 50, 45, 150_000, 1.4, 5.0, 16, 16, 16)
     A, t = _check(sa, w)
     assert sa.sa_tensor_worklist(t.handle, 1)[0][3] >= 2, "the head slice must be split into several pieces"
+    # both kernels of the first pass in one run: small subtrees (third list) and large ones (main list)
+    for w in (configs.make_ttm4_zipf("edge4c", 33, 90, 40, 160, 110, 150_000, 1.4, 5.0, 16, 16, 16),
+              configs.make_ttm4_zipf("edge4d", 34, 400, 60, 150, 40, 200_000, 1.2, 3.0, 16, 16, 16)):
+        A, t = _check(sa, w)
+        n_main, n_sub = (int(sa.sa_tensor_worklist(t.handle, x)[0][0]) for x in (0, 2))
+        assert n_main > 0 and n_sub > 0, (n_main, n_sub)
 
 
 def test_results_are_reproducible_run_to_run(sa):
