@@ -156,9 +156,9 @@ sa_status sa_tensor_export(const sa_tensor *t, int level, int64_t *pos, int32_t 
  * tensor's list for SA_EXPR_SPMM_GEMM, an order-3 tensor's list of fiber rows for SA_EXPR_SPTTM_SPTTM
  * (rows = level-1 fibers), an order-4 tensor's list for the second pass of SA_EXPR_SPTTM_TTM4;
  * 2 = order-4 tensors: ranges of whole (i,j) subtrees for the first pass, rows [out_row,row_end) =
- * level-1 fibers, [f0,f1) their level-2 fibers (at most 128), [p0,p1) their nonzeros; empty when one
- * subtree alone has more than 128 level-2 fibers or 4096 nonzeros, in which case the first pass uses
- * the main list).  These are the slice / fiber / nonzero partition arrays:
+ * level-1 fibers, [f0,f1) their level-2 fibers (at most 64), [p0,p1) their nonzeros; a subtree with
+ * more than 64 level-2 fibers or 4096 nonzeros is not in this list: the first pass takes it from the
+ * main list, which for an order-4 tensor holds only those).  These are the slice / fiber / nonzero partition arrays:
  *   counts [4]: number of items, number of leading groups that one thread block reduces into a
  *               single tile (8 items each; order-3 tensors: 4 tasks each, see sa_tensor_tasks),
  *               number of fix-up entries, number of partial-tile slots

@@ -337,13 +337,13 @@ void build_ttm4(sa_tensor *t, sa_worklist &wl, sa_worklist &wl2)
 }
 
 // Order 4, pass 1 on whole (i,j) subtrees: items are ranges of consecutive small subtrees (subtree_is_small) with
-// at most SA_SUB_MAX_F3 level-2 fibers, SA_SUB_MAX_ROWS subtrees and about 1024 nonzeros (f0/f1 = the fibers,
+// at most SA_SUB_MAX_F3 level-2 fibers, SA_SUB_MAX_ROWS subtrees and about 512 nonzeros (f0/f1 = the fibers,
 // p0/p1 = the nonzeros).  No subtree is cut, so there are no partial tiles; the large subtrees are in the main list.
 void build_ttm4_subtrees(sa_tensor *t, sa_worklist &wl)
 {
     const auto &pos2 = t->pos[2], &pos3 = t->pos[3];
     const int64_t F2 = t->count[1];
-    constexpr int64_t TARGET_NNZ = 1024;
+    constexpr int64_t TARGET_NNZ = 512;
     auto nnz_at = [&](int64_t f2) { return pos3[size_t(pos2[size_t(f2)])]; };
     std::vector<sa_item> items;
     int64_t r0 = 0;

@@ -113,7 +113,7 @@ struct sa_tensor {
 
 // Limits of the order-4 subtree kernel: level-2 fibers an item parks in shared memory, rows (subtrees) per item,
 // nonzeros of one subtree.
-constexpr int SA_SUB_MAX_F3 = 128;
+constexpr int SA_SUB_MAX_F3 = 64;
 constexpr int SA_SUB_MAX_ROWS = 32;
 constexpr int SA_SUB_MAX_NNZ = 4096;
 

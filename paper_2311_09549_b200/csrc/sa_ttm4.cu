@@ -134,9 +134,9 @@ ttm4_slice_kernel(const sa_item *__restrict__ items, int64_t n_items, const int3
 //     (1 KB, contiguous) when the subtree's last fiber has been added.
 // Against the order-3 kernel on the same subtrees this drops the per-unit pipeline drains and the padded
 // tensor-core groups: 16.7 M outer products of 256 FMAs are cheap on the ALUs next to 100 M row gathers.
-constexpr int SUB_SMEM = SA_WARPS_PER_CTA * SA_SUB_MAX_F3 * R * int(sizeof(float));   // 64 KB
+constexpr int SUB_SMEM = SA_WARPS_PER_CTA * SA_SUB_MAX_F3 * R * int(sizeof(float));   // 32 KB
 
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 4)
 ttm4_subtree_kernel(const sa_item *__restrict__ items, int64_t n_items, const int32_t *__restrict__ pos2,
                     const int32_t *__restrict__ pos3, const int32_t *__restrict__ crd_k, const int32_t *__restrict__ crd_o,
                     const float *__restrict__ vals, const uint32_t *__restrict__ endbits, const float *__restrict__ D,
@@ -149,9 +149,24 @@ ttm4_subtree_kernel(const sa_item *__restrict__ items, int64_t n_items, const in
     const sa_item it = items[idx];
     float *pk = sub_smem + warp * (SA_SUB_MAX_F3 * R);
     const int nf3 = it.f1 - it.f0;
+    // rows of D the item's fibers need in phase B (requested now, used after phase A)
+    static_assert(SA_SUB_MAX_F3 <= 64, "two index registers per lane");
+    const int kk0 = lane < nf3 ? __ldg(crd_k + it.f0 + lane) : 0;
+    const int kk1 = lane + 32 < nf3 ? __ldg(crd_k + it.f0 + 32 + lane) : 0;
     {   // ---- phase A
         const int g = lane >> 2, l = lane & 3;
-        const int fa = it.f0 + nf3 * g / 8, fb = it.f0 + nf3 * (g + 1) / 8;
+        // shares of the eight groups: whole fibers, cut where the nonzero count passes the next eighth of the item
+        // (fiber f belongs to the groups before g when it starts before p0 + g len / 8)
+        const int s0 = lane < nf3 ? __ldg(pos3 + it.f0 + lane) : 0x7fffffff;
+        const int s1 = lane + 32 < nf3 ? __ldg(pos3 + it.f0 + 32 + lane) : 0x7fffffff;
+        int fa = it.f0, fb = it.f1;
+#pragma unroll
+        for (int q = 1; q < 8; ++q) {
+            const int target = it.p0 + int(int64_t(it.p1 - it.p0) * q / 8);
+            const int cnt = __popc(__ballot_sync(SA_FULL_MASK, s0 < target)) + __popc(__ballot_sync(SA_FULL_MASK, s1 < target));
+            if (g == q) fa = it.f0 + cnt;
+            if (g + 1 == q) fb = it.f0 + cnt;
+        }
         const int ga = __ldg(pos3 + fa), gb = __ldg(pos3 + fb);
         const int mylen = gb - ga;
         const int maxlen = __reduce_max_sync(SA_FULL_MASK, mylen);
@@ -210,22 +225,27 @@ ttm4_subtree_kernel(const sa_item *__restrict__ items, int64_t n_items, const in
         const int my_end = lane < nr ? __ldg(pos2 + it.out_row + lane + 1) - it.f0 : 0x7fffffff;   // local end of subtree `lane`
         int r = 0, fe = __shfl_sync(SA_FULL_MASK, my_end, 0);
         float4 a0 = make_float4(0.f, 0.f, 0.f, 0.f), a1 = a0;
-        for (int f0 = 0; f0 < nf3; f0 += 4) {
-            float2 d[4];
-            float4 tt[4];
+        // D(k_f, 2mp..2mp+1) of eight fibers at a time, the next eight requested before the current eight are used
+        auto load_d = [&](int f0, float2 (&d)[8]) {
+            const int ks = f0 < 32 ? kk0 : kk1;
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int k = f0 + u < nf3 ? __ldg(crd_k + it.f0 + f0 + u) : 0;
+            for (int u = 0; u < 8; ++u) {
+                const int k = __shfl_sync(SA_FULL_MASK, ks, (f0 + u) & 31);
                 d[u] = sa_ldg2(D + int64_t(k) * ldd + 2 * mp);
-                tt[u] = *reinterpret_cast<const float4 *>(pk + (f0 + u) * R + 4 * nq);
             }
+        };
+        float2 d[8], dn[8];
+        load_d(0, d);
+        for (int f0 = 0; f0 < nf3; f0 += 8) {
+            if (f0 + 8 < nf3) load_d(f0 + 8, dn);
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
+            for (int u = 0; u < 8; ++u) {
                 if (f0 + u < nf3) {
-                    a0.x = fmaf(d[u].x, tt[u].x, a0.x); a0.y = fmaf(d[u].x, tt[u].y, a0.y);
-                    a0.z = fmaf(d[u].x, tt[u].z, a0.z); a0.w = fmaf(d[u].x, tt[u].w, a0.w);
-                    a1.x = fmaf(d[u].y, tt[u].x, a1.x); a1.y = fmaf(d[u].y, tt[u].y, a1.y);
-                    a1.z = fmaf(d[u].y, tt[u].z, a1.z); a1.w = fmaf(d[u].y, tt[u].w, a1.w);
+                    const float4 tt = *reinterpret_cast<const float4 *>(pk + (f0 + u) * R + 4 * nq);
+                    a0.x = fmaf(d[u].x, tt.x, a0.x); a0.y = fmaf(d[u].x, tt.y, a0.y);
+                    a0.z = fmaf(d[u].x, tt.z, a0.z); a0.w = fmaf(d[u].x, tt.w, a0.w);
+                    a1.x = fmaf(d[u].y, tt.x, a1.x); a1.y = fmaf(d[u].y, tt.y, a1.y);
+                    a1.z = fmaf(d[u].y, tt.z, a1.z); a1.w = fmaf(d[u].y, tt.w, a1.w);
                     if (f0 + u + 1 == fe) {                           // the subtree's last fiber
                         float *dst = T2 + int64_t(it.out_row + r) * T2F + (2 * mp) * R + 4 * nq;
                         *reinterpret_cast<float4 *>(dst) = a0;
@@ -237,6 +257,8 @@ ttm4_subtree_kernel(const sa_item *__restrict__ items, int64_t n_items, const in
                     }
                 }
             }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) d[u] = dn[u];
         }
     }
 }

@@ -354,7 +354,7 @@ def test_fiber_row_worklist_of_order3_csf_partitions_fibers_and_nonzeros():
 
 
 def test_order4_subtree_worklist_covers_every_subtree_once_within_its_limits():
-    """Third list of an order-4 tensor: ranges of whole small (i,j) subtrees, at most 128 level-2 fibers and 32
+    """Third list of an order-4 tensor: ranges of whole small (i,j) subtrees, at most 64 level-2 fibers and 32
     subtrees each; a larger subtree is left to the main list."""
     w = configs.make(5, "mini")
     t = sa.SparseTensor(w.dims, w.coords, w.vals, sa.SA_FMT_CSF, device=-1)
@@ -362,14 +362,19 @@ def test_order4_subtree_worklist_covers_every_subtree_once_within_its_limits():
     pos2, pos3 = levels[2][0], levels[3][0]
     counts, items, fix = sa.sa_tensor_worklist(t.handle, 2)
     assert counts[0] > 0 and counts[2] == 0 and counts[3] == 0
-    nxt = 0
+    n_sub = int(t.info()[1][1])
+    seen = np.zeros(n_sub, dtype=np.int32)
     for row, row_end, f0, f1, p0, p1, dest, _ in items:
-        assert row == nxt and row_end > row and dest < 0
+        assert row_end > row and dest < 0
         assert (f0, f1) == (pos2[row], pos2[row_end]) and (p0, p1) == (pos3[f0], pos3[f1])
-        assert f1 - f0 <= 128 and row_end - row <= 32
-        nxt = row_end
-    assert nxt == int(t.info()[1][1])
-    assert sa.sa_tensor_worklist(t.handle, 0)[0][0] == 0, "no large subtree: the main list is empty"
+        assert f1 - f0 <= 64 and row_end - row <= 32
+        seen[row:row_end] += 1
+    # the others are the large ones, and the main list holds exactly those
+    large = np.nonzero(seen == 0)[0]
+    assert (seen <= 1).all()
+    f3s, nz = np.diff(pos2), pos3[pos2[1:]] - pos3[pos2[:-1]]
+    assert ((f3s[large] > 64) | (nz[large] > 4096)).all() and ((f3s[seen == 1] <= 64) & (nz[seen == 1] <= 4096)).all()
+    assert set(sa.sa_tensor_worklist(t.handle, 0)[1][:, 0].tolist()) == set(large.tolist())
     # one (i,j) pair with 130 level-2 fibers next to a small one: the large one is in the main list only
     big = np.stack([np.zeros(130), np.zeros(130), np.arange(130), np.zeros(130)], axis=1).astype(np.int32)
     both = np.concatenate([big, np.array([[1, 1, 5, 1]], np.int32)])
