@@ -275,6 +275,17 @@ sa_status sa_tensor_create(int order, const int64_t *dims, int64_t nnz, const in
                 bits[size_t(p >> 5)] |= 1u << (p & 31);
             }
             s = upload(t, bits.data(), bits.size(), &t->d_endbits);
+            if (s == SA_OK) {
+                std::vector<int2> pack(size_t(nnz) + 1);
+                for (int64_t p = 0; p < nnz; ++p) {
+                    const uint32_t end = (bits[size_t(p >> 5)] >> (p & 31)) & 1u;
+                    int32_t vb;
+                    std::memcpy(&vb, &t->vals[size_t(p)], sizeof(vb));
+                    pack[size_t(p)] = make_int2(int32_t(uint32_t(t->crd[last][size_t(p)]) | (end << 31)), vb);
+                }
+                pack[size_t(nnz)] = make_int2(0, 0);
+                s = upload(t, pack.data(), pack.size(), &t->d_nzpack);
+            }
         }
         const int32_t zeros[4] = {0, 0, 0, 0};
         if (s == SA_OK) s = upload(t, zeros, 4, &t->d_status);

@@ -100,6 +100,8 @@ struct sa_tensor {
     float *d_vals = nullptr;
     uint32_t *d_endbits = nullptr;            // CSF: bit (p & 31) of word p / 32 is set when nonzero p is the last of
                                               // its last-level fiber ((i,j) for order 3, (i,j,k) for order 4)
+    int2 *d_nzpack = nullptr;                 // CSF: per nonzero (last-level index | end-of-fiber bit << 31, value bits): what the
+                                              // group-per-fiber kernels (kernel 7, order-4 subtree kernel) stream, one 8-byte load
     int32_t *d_status = nullptr;              // [4] device status word
 
     sa_worklist wl_main;                      // TTM3 / pass 1 of TTM4 / SDDMM-SpMM

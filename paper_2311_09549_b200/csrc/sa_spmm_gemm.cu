@@ -303,13 +303,15 @@ spmm_kernel(const sa_item *__restrict__ items, int64_t n_items, const int32_t *_
 // fiber): M/4 lanes own a row of E as one float4 each, so a warp works on 128/M fibers' streams at once, one
 // nonzero per group and step.  A group takes a contiguous share of the item's fibers and walks their nonzeros
 // as one stream, eight index/value pairs per load (the next eight already requested), eight row gathers in
-// flight; the end-of-fiber bit of a nonzero travels in the sign bit of its index and closes the output row.
+// flight; index, end-of-fiber bit (sign bit) and value of a nonzero come as one 8-byte record (half the load
+// wavefronts of separate index, value and bit arrays, and the L1 pipe is what this kernel saturates first); the
+// bit closes the output row.
 // A piece of a long fiber (dest >= 0) is split over the groups by nonzeros and summed across them at the end.
 template <int M>
 __global__ void __launch_bounds__(256)
 fiber_spmm_kernel(const sa_item *__restrict__ items, int64_t n_items, const int32_t *__restrict__ pos,
-                  const int32_t *__restrict__ crd, const float *__restrict__ vals, const uint32_t *__restrict__ endbits,
-                  const float *__restrict__ E, int64_t lde, float *__restrict__ out, float *__restrict__ partial)
+                  const int2 *__restrict__ nz, const float *__restrict__ E, int64_t lde, float *__restrict__ out,
+                  float *__restrict__ partial)
 {
     constexpr int LPR = M / 4, NG = 32 / LPR;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -336,9 +338,9 @@ fiber_spmm_kernel(const sa_item *__restrict__ items, int64_t n_items, const int3
         x = 0;
         v = 0.f;
         if (c + (l & 7) < mylen) {
-            x = __ldg(crd + p);
-            v = __ldg(vals + p);
-            if (!piece) x |= int(((__ldg(endbits + (p >> 5)) >> (p & 31)) & 1u) << 31);
+            const int2 w = __ldg(nz + p);                            // (index | end-of-fiber bit << 31, value bits)
+            x = piece ? (w.x & 0x7fffffff) : w.x;
+            v = __int_as_float(w.y);
         }
     };
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -484,8 +486,7 @@ sa_status run_fibers(const sa_tensor *t, const sa_dense *ops, float *out, void *
         if (gs != SA_OK) return gs;
         *launches += 1;
         if (ctas > 0) {
-            fiber_spmm_kernel<M><<<(unsigned)ctas, 256, 0, stream>>>(wl.d_items, n_items, t->d_pos[2], t->d_crd[2], t->d_vals,
-                                                                    t->d_endbits, E, M, out, partial);
+            fiber_spmm_kernel<M><<<(unsigned)ctas, 256, 0, stream>>>(wl.d_items, n_items, t->d_pos[2], t->d_nzpack, E, M, out, partial);
             if (cudaGetLastError() != cudaSuccess) return SA_E_CUDA;
             *launches += 1;
         }
@@ -498,8 +499,8 @@ sa_status run_fibers(const sa_tensor *t, const sa_dense *ops, float *out, void *
     float *T = static_cast<float *>(ws);
     float *partial = reinterpret_cast<float *>(static_cast<char *>(ws) + sa_align256(size_t(F2) * L * sizeof(float)));
     if (ctas > 0) {
-        fiber_spmm_kernel<L><<<(unsigned)ctas, 256, 0, stream>>>(wl.d_items, n_items, t->d_pos[2], t->d_crd[2], t->d_vals,
-                                                                t->d_endbits, ops[0].ptr, ops[0].ld, T, partial);
+        fiber_spmm_kernel<L><<<(unsigned)ctas, 256, 0, stream>>>(wl.d_items, n_items, t->d_pos[2], t->d_nzpack, ops[0].ptr, ops[0].ld,
+                                                                T, partial);
         if (cudaGetLastError() != cudaSuccess) return SA_E_CUDA;
         *launches += 1;
     }

@@ -138,9 +138,8 @@ constexpr int SUB_SMEM = SA_WARPS_PER_CTA * SA_SUB_MAX_F3 * R * int(sizeof(float
 
 __global__ void __launch_bounds__(256, 4)
 ttm4_subtree_kernel(const sa_item *__restrict__ items, int64_t n_items, const int32_t *__restrict__ pos2,
-                    const int32_t *__restrict__ pos3, const int32_t *__restrict__ crd_k, const int32_t *__restrict__ crd_o,
-                    const float *__restrict__ vals, const uint32_t *__restrict__ endbits, const float *__restrict__ D,
-                    int64_t ldd, const float *__restrict__ E, int64_t lde, float *__restrict__ T2)
+                    const int32_t *__restrict__ pos3, const int32_t *__restrict__ crd_k, const int2 *__restrict__ nz,
+                    const float *__restrict__ D, int64_t ldd, const float *__restrict__ E, int64_t lde, float *__restrict__ T2)
 {
     extern __shared__ __align__(16) float sub_smem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -175,9 +174,9 @@ ttm4_subtree_kernel(const sa_item *__restrict__ items, int64_t n_items, const in
             x = 0;
             v = 0.f;
             if (q < mylen) {
-                const int p = ga + q;
-                x = __ldg(crd_o + p) | int(((__ldg(endbits + (p >> 5)) >> (p & 31)) & 1u) << 31);
-                v = __ldg(vals + p);
+                const int2 w = __ldg(nz + ga + q);                   // (index o | end-of-fiber bit << 31, value bits)
+                x = w.x;
+                v = __int_as_float(w.y);
             }
         };
         // lane l of the group holds nonzeros c + l and c + 4 + l of the group's stream
@@ -316,8 +315,7 @@ sa_status sa_launch_ttm4(const sa_tensor *t, const sa_dense *ops, float *out, vo
             return SA_E_CUDA;
         const int64_t ctas = (n_sub + SA_WARPS_PER_CTA - 1) / SA_WARPS_PER_CTA;
         ttm4_subtree_kernel<<<(unsigned)ctas, 256, SUB_SMEM, stream>>>(t->wl_sub.d_items, n_sub, t->d_pos[2], t->d_pos[3], t->d_crd[2],
-                                                                       t->d_crd[3], t->d_vals, t->d_endbits, ops[1].ptr, ops[1].ld,
-                                                                       ops[2].ptr, ops[2].ld, T2);
+                                                                       t->d_nzpack, ops[1].ptr, ops[1].ld, ops[2].ptr, ops[2].ld, T2);
         if (cudaGetLastError() != cudaSuccess) return SA_E_CUDA;
         *launches += 1;
     }
