@@ -260,7 +260,7 @@ gemm_bf16x3_kernel(int64_t J, const float *__restrict__ C, int64_t ldc, const fl
 template <int MV>
 __global__ void __launch_bounds__(256)
 spmm_kernel(const sa_item *__restrict__ items, int64_t n_items, const int32_t *__restrict__ pos,
-            const int32_t *__restrict__ crd, const float *__restrict__ vals, const float *__restrict__ E, int64_t lde,
+            const int32_t *__restrict__ crd, const float *__restrict__ vals, const float *__restrict__ E,
             float *__restrict__ out, float *__restrict__ partial)
 {
     constexpr int M = MV * 32;
@@ -283,7 +283,7 @@ spmm_kernel(const sa_item *__restrict__ items, int64_t n_items, const int32_t *_
             for (int s = 0; s < n; ++s) {
                 const int j = __shfl_sync(SA_FULL_MASK, jj, s);
                 const float v = __shfl_sync(SA_FULL_MASK, vv, s);
-                const float *erow = E + int64_t(j) * lde + lane * MV;
+                const float *erow = E + int64_t(j) * M + lane * MV;
                 if (MV == 2) {
                     const float2 e = sa_ldg2(erow);
                     acc[0] = fmaf(v, e.x, acc[0]);
@@ -429,7 +429,7 @@ sa_status run(const sa_tensor *t, const sa_dense *ops, float *out, void *ws, boo
     *launches += 1;
     const int64_t ctas = (n_items + SA_WARPS_PER_CTA - 1) / SA_WARPS_PER_CTA;
     if (ctas > 0) {
-        spmm_kernel<M / 32><<<(unsigned)ctas, 256, 0, stream>>>(wl.d_items, n_items, t->d_pos[1], t->d_crd[1], t->d_vals, E, M,
+        spmm_kernel<M / 32><<<(unsigned)ctas, 256, 0, stream>>>(wl.d_items, n_items, t->d_pos[1], t->d_crd[1], t->d_vals, E,
                                                                out, partial);
         if (cudaGetLastError() != cudaSuccess) return SA_E_CUDA;
         *launches += 1;
