@@ -261,3 +261,24 @@ def test_spttm_spttm_empty_and_single_entry(sa, nnz):
     for s in (sa.SA_SCHED_ASSOC_LEFT, sa.SA_SCHED_ASSOC_RIGHT):
         A, _ = _check(sa, w, sched=s)
         assert A.shape == (nnz, 64)
+
+
+@pytest.mark.parametrize("L,M", [(128, 32), (128, 64), (256, 32), (256, 64)])
+def test_dense_stage_ragged_rows_and_padded_leading_dimensions(sa, L, M):
+    """B.(C.D) with a number of columns J that is not a multiple of the dense stage's 128-row tile (the last
+    tile is ragged, several tiles per thread block) and with C and D given as padded views."""
+    import torch
+    I, J = 700, 148 * 128 * 2 + 77
+    coords, vals = _random_coo(21, (I, J), 30_000)
+    C, D = configs.dense_normal(21, 0, J, L), configs.dense_normal(21, 1, L, M)
+    w = _wl("spmm_gemm", "csr", (I, J), coords, vals, [C, D], (I, M))
+    A_ref, S_ref = oracle.evaluate(w)
+    t = sa.SparseTensor(w.dims, w.coords, w.vals, sa.SA_FMT_CSR, device=0)
+    bigC = torch.zeros(J, L + 8, device="cuda")
+    bigD = torch.zeros(L, M + 4, device="cuda")
+    bigC[:, 4:4 + L] = torch.from_numpy(C).cuda()
+    bigD[:, :M] = torch.from_numpy(D).cuda()
+    out, _ = t.run("spmm_gemm", [bigC[:, 4:4 + L], bigD[:, :M]], sched=sa.SA_SCHED_ASSOC_RIGHT)
+    torch.cuda.synchronize()
+    assert sa.sa_last_device_status(t.handle, torch.cuda.current_stream().cuda_stream) == sa.SA_OK
+    assert_close(out.cpu().numpy().astype(np.float64), A_ref, S_ref, TOL_FP32, "dense stage %dx%d" % (L, M))
