@@ -136,6 +136,8 @@ ttm4_slice_kernel(const sa_item *__restrict__ items, int64_t n_items, const int3
 // tensor-core groups: 16.7 M outer products of 256 FMAs are cheap on the ALUs next to 100 M row gathers.
 constexpr int SUB_SMEM = SA_WARPS_PER_CTA * SA_SUB_MAX_F3 * R * int(sizeof(float));   // 32 KB
 
+// CONTIG: both factor matrices are stored without padding (leading dimension 16), so a row offset is a shift.
+template <bool CONTIG>
 __global__ void __launch_bounds__(256, 4)
 ttm4_subtree_kernel(const sa_item *__restrict__ items, int64_t n_items, const int32_t *__restrict__ pos2,
                     const int32_t *__restrict__ pos3, const int32_t *__restrict__ crd_k, const int2 *__restrict__ nz,
@@ -147,6 +149,8 @@ ttm4_subtree_kernel(const sa_item *__restrict__ items, int64_t n_items, const in
     if (idx >= n_items) return;
     const sa_item it = items[idx];
     float *pk = sub_smem + warp * (SA_SUB_MAX_F3 * R);
+    // row offsets in 32-bit arithmetic (the launcher checks rows * ld < 2^31)
+    const uint32_t ld_d = CONTIG ? uint32_t(R) : uint32_t(ldd), ld_e = CONTIG ? uint32_t(R) : uint32_t(lde);
     const int nf3 = it.f1 - it.f0;
     // rows of D the item's fibers need in phase B (requested now, used after phase A)
     static_assert(SA_SUB_MAX_F3 <= 64, "two index registers per lane");
@@ -199,7 +203,7 @@ ttm4_subtree_kernel(const sa_item *__restrict__ items, int64_t n_items, const in
             for (int u = 0; u < 8; ++u) {
                 xs[u] = __shfl_sync(SA_FULL_MASK, x[u >> 2], u & 3, 4);
                 vs[u] = __shfl_sync(SA_FULL_MASK, v[u >> 2], u & 3, 4);
-                e[u] = sa_ldg4(E + int64_t(xs[u] & 0x7fffffff) * lde + 4 * l);
+                e[u] = sa_ldg4(E + (uint32_t(xs[u] & 0x7fffffff) * ld_e + 4u * l));
             }
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
@@ -230,7 +234,7 @@ ttm4_subtree_kernel(const sa_item *__restrict__ items, int64_t n_items, const in
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
                 const int k = __shfl_sync(SA_FULL_MASK, ks, (f0 + u) & 31);
-                d[u] = sa_ldg2(D + int64_t(k) * ldd + 2 * mp);
+                d[u] = sa_ldg2(D + (uint32_t(k) * ld_d + 2u * mp));
             }
         };
         float2 d[8], dn[8];
@@ -311,10 +315,12 @@ sa_status sa_launch_ttm4(const sa_tensor *t, const sa_dense *ops, float *out, vo
     const int64_t n_sub = int64_t(t->wl_sub.items.size());
     *launches = 0;
     if (n_sub > 0) {
-        if (cudaFuncSetAttribute(ttm4_subtree_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SUB_SMEM) != cudaSuccess)
-            return SA_E_CUDA;
+        if (ops[1].rows * ops[1].ld >= (int64_t(1) << 31) || ops[2].rows * ops[2].ld >= (int64_t(1) << 31)) return SA_E_UNSUPPORTED;
+        const bool contig = ops[1].ld == R && ops[2].ld == R;
+        auto kern = contig ? ttm4_subtree_kernel<true> : ttm4_subtree_kernel<false>;
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SUB_SMEM) != cudaSuccess) return SA_E_CUDA;
         const int64_t ctas = (n_sub + SA_WARPS_PER_CTA - 1) / SA_WARPS_PER_CTA;
-        ttm4_subtree_kernel<<<(unsigned)ctas, 256, SUB_SMEM, stream>>>(t->wl_sub.d_items, n_sub, t->d_pos[2], t->d_pos[3], t->d_crd[2],
+        kern<<<(unsigned)ctas, 256, SUB_SMEM, stream>>>(t->wl_sub.d_items, n_sub, t->d_pos[2], t->d_pos[3], t->d_crd[2],
                                                                        t->d_nzpack, ops[1].ptr, ops[1].ld, ops[2].ptr, ops[2].ld, T2);
         if (cudaGetLastError() != cudaSuccess) return SA_E_CUDA;
         *launches += 1;

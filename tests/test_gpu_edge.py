@@ -282,3 +282,22 @@ def test_dense_stage_ragged_rows_and_padded_leading_dimensions(sa, L, M):
     torch.cuda.synchronize()
     assert sa.sa_last_device_status(t.handle, torch.cuda.current_stream().cuda_stream) == sa.SA_OK
     assert_close(out.cpu().numpy().astype(np.float64), A_ref, S_ref, TOL_FP32, "dense stage %dx%d" % (L, M))
+
+
+def test_ttm4_padded_factor_matrices(sa):
+    """Order-4 chain with the factor matrices given as padded views (leading dimension 20): the subtree kernel's
+    general-stride variant and the order-3 kernel's row addressing."""
+    import torch
+    w = configs.make_ttm4_zipf("edge4e", 35, 300, 60, 150, 40, 120_000, 1.2, 3.0, 16, 16, 16)
+    A_ref, S_ref = oracle.evaluate(w)
+    t = sa.SparseTensor(w.dims, w.coords, w.vals, sa.SA_FMT_CSF, device=0)
+    views = []
+    for x in w.dense:
+        b = torch.zeros(x.shape[0], 20, device="cuda")
+        b[:, :16] = torch.from_numpy(x).cuda()
+        views.append(b[:, :16])
+    out, _ = t.run(w.expr, views)
+    torch.cuda.synchronize()
+    assert sa.sa_last_device_status(t.handle, torch.cuda.current_stream().cuda_stream) == sa.SA_OK
+    assert_close(out.cpu().numpy().astype(np.float64), A_ref, S_ref, TOL_FP32, "ttm4 padded ld")
+    assert int(sa.sa_tensor_worklist(t.handle, 2)[0][0]) > 0
