@@ -41,8 +41,8 @@ NCU_TRAFFIC = {
         "dram_bytes": 851268608, "profile": "profiles/ttm3_kernel_cfg2.md"},
     5: {"kernel": "ttm4_subtree_kernel (pass 1 of the order-4 chain on the small subtrees, 51 % of the step)",
         "source": "paper_2311_09549_b200/csrc/sa_ttm4.cu",
-        "sha256": "b1bf316f3d5dafd74ae7ad0e438f6fc9d6f5bb819f0ff5c8d796e1044123469a",
-        "dram_bytes": 2218000000, "profile": "profiles/ttm4_kernel_cfg5.md"},
+        "sha256": "0cf1a9b53532ebf95fe9cccc071d824a69c9d457ac76a6d37f6355f062eef7c9",
+        "dram_bytes": 2217051392, "profile": "profiles/ttm4_kernel_cfg5.md"},
     10: {"kernel": "fiber_spmm_kernel<32> (99 % of the step)", "source": "paper_2311_09549_b200/csrc/sa_spmm_gemm.cu",
          "sha256": "408ed3d1f40077ca8fcb6e4ebeb2dc9b8ca08986b342d17b370a87df4d7b251e",
          "dram_bytes": 955500000, "profile": "profiles/fiber_spmm_kernel_w10.md"},
