@@ -210,7 +210,13 @@ sa_status sa_workspace_size(const sa_tensor *t, sa_expr expr, sa_schedule sched,
  * Compiled dense ranks (anything else is SA_E_UNSUPPORTED): SPTTM_TTM3 L, M in {16, 32};
  * SPTTM_TTM4 L = M = N = 16; SDDMM_SPMM K, L in {32, 64, 128}; SPMM_GEMM L in {128, 256},
  * M in {32, 64}; TTMC3 L, M, N in {16, 32}; SDDMM_SPMM_GEMM K, L in {32, 64, 128}, M in {32, 64};
- * SPMMH_GEMM L in {128, 256}, M in {32, 64}; MTTKRP_GEMM R = 32, M in {32, 64}.
+ * SPMMH_GEMM L in {128, 256}, M in {32, 64}; MTTKRP_GEMM R = 32, M in {32, 64};
+ * SPTTM_SPTTM L, M in {32, 64} (out: level_counts[1] x M, see sa_expr).
+ * Arithmetic: fp32 throughout; stages on tensor cores split every fp32 operand into two parts and
+ * add three partial products (TF32 parts in the per-slice contractions, BF16 parts in the dense GEMM
+ * stage), so every output element stays within 1e-4 of the sum of the absolute values of its terms.
+ * The dense GEMM stage (SPMM_GEMM as B.(C.D), SDDMM_SPMM_GEMM) waits on on-chip hand-offs with a
+ * 2-second limit; if one runs out the kernel returns and sa_last_device_status reports SA_E_TIMEOUT.
  * Returns launch errors only; completion is observed by synchronising the stream.
  * Errors: SA_E_ARG, SA_E_SHAPE, SA_E_UNSUPPORTED, SA_E_WORKSPACE, SA_E_CUDA.
  */
