@@ -292,6 +292,10 @@ sa_status sa_tensor_create(int order, const int64_t *dims, int64_t nnz, const in
         if (s == SA_OK) s = upload_worklist(t, t->wl_main);
         if (s == SA_OK) s = upload_worklist(t, t->wl_aux);
         if (s == SA_OK) s = upload_worklist(t, t->wl_sub);
+        if (s == SA_OK && fmt == SA_FMT_CSF && order == 4) {
+            s = upload(t, t->f4_supers.data(), t->f4_supers.size(), &t->d_f4_supers);
+            if (s == SA_OK) s = upload(t, t->f4_pieces.data(), t->f4_pieces.size(), &t->d_f4_pieces);
+        }
         if (s == SA_OK && cudaDeviceSynchronize() != cudaSuccess) s = SA_E_CUDA;
         if (s == SA_E_CUDA) cudaGetLastError();
     }
@@ -324,7 +328,20 @@ sa_status sa_tensor_export(const sa_tensor *t, int level, int64_t *pos, int32_t 
 
 sa_status sa_tensor_worklist(const sa_tensor *t, int which, int64_t *counts, int32_t *items, int32_t *fix)
 {
-    if (!t || which < 0 || which > 2) return SA_E_ARG;
+    if (!t || which < 0 || which > 3) return SA_E_ARG;
+    if (which == 3) {
+        // order-4 CSF: the pieces (8 integers each, returned as items) and super-items (4 integers each, returned
+        // as fix-up entries) of the fused kernel
+        if (counts) {
+            counts[0] = int64_t(t->f4_pieces.size() / 8);
+            counts[1] = t->f4_n_large;
+            counts[2] = int64_t(t->f4_supers.size() / 4);
+            counts[3] = 0;
+        }
+        if (items) std::memcpy(items, t->f4_pieces.data(), t->f4_pieces.size() * sizeof(int32_t));
+        if (fix) std::memcpy(fix, t->f4_supers.data(), t->f4_supers.size() * sizeof(int32_t));
+        return SA_OK;
+    }
     const sa_worklist &wl = which == 0 ? t->wl_main : which == 1 ? t->wl_aux : t->wl_sub;
     if (counts) {
         counts[0] = int64_t(wl.items.size());

@@ -288,89 +288,116 @@ void build_ttm3(sa_tensor *t, sa_worklist &wl)
 }
 
 
-// A subtree (i,j) that the subtree kernel of pass 1 can take whole.
-static bool subtree_is_small(const sa_tensor *t, int64_t f2)
+// Order-4 CSF (see sa_ttm4.cu).  The chain runs as one fused kernel over *pieces*: contiguous ranges of (i,j)
+// subtrees holding about PIECE_NNZ nonzeros, one thread block each.  A piece is a run of *super-items* (at most
+// SA_F4_POOL subtrees: what the block's pool of 16 x 16 temporaries holds), a super-item a run of *items* that
+// the block's warps take one at a time:
+//   kind 0: consecutive subtrees with at most SA_F4_ROWS level-2 fibers in all (one batch of parked fiber rows),
+//           or one subtree with more fibers (evaluated in several batches);   f0/f1 = fibers, p0/p1 = nonzeros
+//   kind 1: up to 8 consecutive *large* subtrees (more than SA_SUB_MAX_NNZ nonzeros), whose temporaries the
+//           order-3 kernel has written beforehand; f0 = index of the first one among the large subtrees.
+// Nothing is cut at a slice boundary: the block follows the slices through pos[1] while it consumes the
+// temporaries.  A slice that lies in several pieces gets one partial tile per piece (consecutive slots) and a
+// fix-up entry.  `wl` (main list): the order-3 lists over the large subtrees, output row = index among them.
+static bool subtree_is_large(const sa_tensor *t, int64_t f2)
 {
     const auto &pos2 = t->pos[2], &pos3 = t->pos[3];
-    const int64_t fa = pos2[size_t(f2)], fb = pos2[size_t(f2) + 1];
-    return fb - fa <= SA_SUB_MAX_F3 && pos3[size_t(fb)] - pos3[size_t(fa)] <= SA_SUB_MAX_NNZ;
+    return pos3[size_t(pos2[size_t(f2) + 1])] - pos3[size_t(pos2[size_t(f2)])] > SA_SUB_MAX_NNZ;
 }
 
-// Order-4 CSF.  The chain is evaluated in two passes (see sa_ttm4.cu).  Pass 1 runs the order-3 kernel with
-// the large (i,j) subtrees as slices: `wl` gets the same lists as an order-3 tensor whose slices are those
-// level-1 fibers (output row = fiber index); the small subtrees go to the subtree kernel's list.  Pass 2 contracts the per-fiber temporaries of each slice with rows of
-// C: `wl2` holds one item per (piece of a slice, quarter of the 256 temporaries' columns); a slice with more
-// than CHUNK_F fibers is cut into pieces whose partial tiles the fix-up kernel sums.
-void build_ttm4(sa_tensor *t, sa_worklist &wl, sa_worklist &wl2)
+void build_ttm4(sa_tensor *t, sa_worklist &wl, sa_worklist &wl_items, sa_worklist &wl_fix)
 {
-    build_ttm3_lists(wl, t->count[1], [](int64_t f) { return int32_t(f); }, [&](int64_t f) { return subtree_is_small(t, f); },
-                     t->pos[2], t->pos[3]);
-    constexpr int64_t CHUNK_F = 512;
-    const auto &pos1 = t->pos[1];
-    std::vector<sa_item> items;
-    for (int64_t s = 0; s < t->count[0]; ++s) {
-        const int64_t fa = pos1[size_t(s)], fb = pos1[size_t(s) + 1];
-        const int32_t row = t->crd[0][size_t(s)];
-        const int64_t nc = (fb - fa + CHUNK_F - 1) / CHUNK_F;
-        int32_t slot0 = -1;
-        if (nc > 1) {
-            slot0 = int32_t(wl2.n_slots);
-            wl2.fix.push_back(sa_fix{row, slot0, int32_t(nc), 0});
-            wl2.n_slots += nc;
-        }
-        for (int64_t c = 0; c < nc; ++c)
-            for (int qc = 0; qc < 4; ++qc) {
-                sa_item it = empty_item();
-                it.out_row = row; it.row_end = row + 1;
-                it.f0 = int32_t(fa + c * CHUNK_F); it.f1 = int32_t(std::min(fb, fa + (c + 1) * CHUNK_F));
-                it.p0 = it.f0; it.p1 = it.f1;          // size key: fibers
-                it.dest = nc > 1 ? slot0 + int32_t(c) : -1;
-                it.pad = qc;
-                items.push_back(it);
-            }
-    }
-    // largest first: the tail of the launch is then made of the cheapest items
-    std::stable_sort(items.begin(), items.end(), [](const sa_item &a, const sa_item &b) { return (a.f1 - a.f0) > (b.f1 - b.f0); });
-    wl2.items = std::move(items);
-    wl2.n_group_ctas = 0;
-    append_empty_slices(t, wl2);
-}
+    const auto &pos1 = t->pos[1], &pos2 = t->pos[2], &pos3 = t->pos[3];
+    const int64_t F2 = t->count[1], S = t->count[0];
+    std::vector<int32_t> large_ord(size_t(F2), -1);
+    int32_t n_large = 0;
+    for (int64_t r = 0; r < F2; ++r)
+        if (subtree_is_large(t, r)) large_ord[size_t(r)] = n_large++;
+    t->f4_n_large = n_large;
+    build_ttm3_lists(wl, F2, [&](int64_t r) { return large_ord[size_t(r)]; }, [&](int64_t r) { return large_ord[size_t(r)] < 0; },
+                     pos2, pos3);
+    wl.nnz = 0;
+    for (const sa_item &it : wl.items) wl.nnz += it.p1 - it.p0;
 
-// Order 4, pass 1 on whole (i,j) subtrees: items are ranges of consecutive small subtrees (subtree_is_small) with
-// at most SA_SUB_MAX_F3 level-2 fibers, SA_SUB_MAX_ROWS subtrees and about 512 nonzeros (f0/f1 = the fibers,
-// p0/p1 = the nonzeros).  No subtree is cut, so there are no partial tiles; the large subtrees are in the main list.
-void build_ttm4_subtrees(sa_tensor *t, sa_worklist &wl)
-{
-    const auto &pos2 = t->pos[2], &pos3 = t->pos[3];
-    const int64_t F2 = t->count[1];
-    constexpr int64_t TARGET_NNZ = 512;
-    auto nnz_at = [&](int64_t f2) { return pos3[size_t(pos2[size_t(f2)])]; };
-    std::vector<sa_item> items;
-    int64_t r0 = 0;
-    auto flush = [&](int64_t r1) {
-        if (r1 > r0) {
+    constexpr int64_t PIECE_NNZ = 16384, LARGE_WEIGHT = 64;
+    auto nnz_at = [&](int64_t r) { return pos3[size_t(pos2[size_t(r)])]; };
+    std::vector<sa_item> &items = wl_items.items;
+    std::vector<int32_t> &supers = t->f4_supers, &pieces = t->f4_pieces;
+    // state of the open item / super-item / piece
+    int64_t it_r0 = 0, sup_item0 = 0, sup_r0 = 0, piece_sup0 = 0, piece_r0 = 0, piece_w = 0;
+    int it_kind = -1;
+    auto close_item = [&](int64_t r) {
+        if (it_kind >= 0 && r > it_r0) {
             sa_item it = empty_item();
-            it.out_row = int32_t(r0); it.row_end = int32_t(r1);
-            it.f0 = int32_t(pos2[size_t(r0)]); it.f1 = int32_t(pos2[size_t(r1)]);
-            it.p0 = int32_t(nnz_at(r0)); it.p1 = int32_t(nnz_at(r1));
+            it.out_row = int32_t(it_r0); it.row_end = int32_t(r); it.pad = it_kind;
+            if (it_kind == 0) {
+                it.f0 = int32_t(pos2[size_t(it_r0)]); it.f1 = int32_t(pos2[size_t(r)]);
+                it.p0 = int32_t(nnz_at(it_r0)); it.p1 = int32_t(nnz_at(r));
+            } else {
+                it.f0 = large_ord[size_t(it_r0)]; it.f1 = it.f0 + int32_t(r - it_r0);
+            }
             items.push_back(it);
         }
-        r0 = r1;
+        it_kind = -1;
+        it_r0 = r;
+    };
+    auto close_super = [&](int64_t r) {
+        close_item(r);
+        if (int64_t(items.size()) > sup_item0) {
+            supers.push_back(int32_t(sup_item0)); supers.push_back(int32_t(items.size()));
+            supers.push_back(int32_t(sup_r0)); supers.push_back(int32_t(r));
+        }
+        sup_item0 = int64_t(items.size());
+        sup_r0 = r;
+    };
+    // slice that holds subtree r (r < F2)
+    auto slice_of = [&](int64_t r) { return int64_t(std::upper_bound(pos1.begin(), pos1.end(), r) - pos1.begin()) - 1; };
+    auto close_piece = [&](int64_t r) {
+        close_super(r);
+        if (int64_t(supers.size() / 4) > piece_sup0) {
+            const int64_t sa = slice_of(piece_r0), sb = slice_of(r - 1);
+            pieces.push_back(int32_t(piece_sup0)); pieces.push_back(int32_t(supers.size() / 4));
+            pieces.push_back(int32_t(sa)); pieces.push_back(int32_t(sb));
+            pieces.push_back(-1); pieces.push_back(-1);       // destinations of the first / last slice: set below
+            pieces.push_back(int32_t(piece_r0)); pieces.push_back(int32_t(r));
+        }
+        piece_sup0 = int64_t(supers.size() / 4);
+        piece_r0 = r;
+        piece_w = 0;
     };
     for (int64_t r = 0; r < F2; ++r) {
-        if (!subtree_is_small(t, r)) {
-            flush(r);
-            r0 = r + 1;
-            continue;
+        const bool large = large_ord[size_t(r)] >= 0;
+        if (piece_w >= PIECE_NNZ) close_piece(r);
+        if (r - sup_r0 >= SA_F4_POOL) close_super(r);
+        if (it_kind >= 0) {
+            const bool full = large ? (it_kind != 1 || r - it_r0 >= 8)
+                                    : (it_kind != 0 || r - it_r0 >= 32 || pos2[size_t(r) + 1] - pos2[size_t(it_r0)] > SA_F4_ROWS);
+            if (full) close_item(r);
         }
-        if (r > r0 && (pos2[size_t(r) + 1] - pos2[size_t(r0)] > SA_SUB_MAX_F3 || r - r0 >= SA_SUB_MAX_ROWS ||
-                       nnz_at(r + 1) - nnz_at(r0) > TARGET_NNZ))
-            flush(r);
+        if (it_kind < 0) { it_kind = large ? 1 : 0; it_r0 = r; }
+        piece_w += large ? LARGE_WEIGHT : nnz_at(r + 1) - nnz_at(r);
     }
-    flush(F2);
-    for (const sa_item &it : items) wl.nnz += it.p1 - it.p0;
-    wl.items = std::move(items);
-    wl.n_group_ctas = 0;
+    close_piece(F2);
+    wl_items.n_group_ctas = 0;
+    // partial tiles: a slice that lies in more than one piece gets one slot per piece
+    std::vector<int32_t> slice_slots(size_t(S), 0), slice_slot0(size_t(S), -1);
+    const size_t n_pieces = pieces.size() / 8;
+    for (size_t p = 0; p < n_pieces; ++p)
+        for (int64_t s = pieces[8 * p + 2]; s <= pieces[8 * p + 3]; ++s) slice_slots[size_t(s)]++;
+    for (int64_t s = 0; s < S; ++s)
+        if (slice_slots[size_t(s)] > 1) {
+            slice_slot0[size_t(s)] = int32_t(wl_fix.n_slots);
+            wl_fix.fix.push_back(sa_fix{t->crd[0][size_t(s)], int32_t(wl_fix.n_slots), slice_slots[size_t(s)], 0});
+            wl_fix.n_slots += slice_slots[size_t(s)];
+        }
+    std::vector<int32_t> next_slot(slice_slot0);
+    for (size_t p = 0; p < n_pieces; ++p) {
+        const int64_t sa = pieces[8 * p + 2], sb = pieces[8 * p + 3];
+        if (slice_slot0[size_t(sa)] >= 0) pieces[8 * p + 4] = next_slot[size_t(sa)]++;
+        if (sb != sa) { if (slice_slot0[size_t(sb)] >= 0) pieces[8 * p + 5] = next_slot[size_t(sb)]++; }
+        else pieces[8 * p + 5] = pieces[8 * p + 4];
+    }
+    append_empty_slices(t, wl_fix);
 }
 
 // Rows of a sparse matrix given by its pos array: row ranges of about target_nnz nonzeros (at most max_rows rows); rows longer than
@@ -429,9 +456,7 @@ void sa_build_worklists(sa_tensor *t)
         build_rows(t->pos[2], t->count[1], t->wl_aux, 1024, 4096, 4096, 2048);
     }
     if (t->fmt == SA_FMT_CSF && t->order == 4) {
-        build_ttm4(t, t->wl_main, t->wl_aux);
-        build_ttm4_subtrees(t, t->wl_sub);
-        t->wl_main.nnz = t->nnz - t->wl_sub.nnz;
+        build_ttm4(t, t->wl_main, t->wl_sub, t->wl_aux);
     }
     if (t->fmt == SA_FMT_CSR) {
         build_rows(t->pos[1], t->dims[0], t->wl_main, 256, 32, 1024, 512);    // fused SDDMM -> SpMM

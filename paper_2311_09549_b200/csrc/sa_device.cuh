@@ -17,6 +17,52 @@ __device__ __forceinline__ void sa_st_cs(float *p, float v) { __stcs(p, v); }
 __device__ __forceinline__ void sa_st_cs4(float *p, float4 v) { __stcs(reinterpret_cast<float4 *>(p), v); }
 __device__ __forceinline__ void sa_st_cs2(float *p, float2 v) { __stcs(reinterpret_cast<float2 *>(p), v); }
 
+// Self-checking build (-DSA_DEBUG_BOUNDS): every index that comes out of the tensor's arrays is checked before it
+// is turned into an address; the first violation is recorded in the tensor's status word (check number, offending
+// value, thread; read back by sa_last_device_status / sa_device_status_words) and the caller redirects the access to
+// a valid element.  Nothing traps.  In the normal build SA_CHK is the constant true.
+#ifdef SA_DEBUG_BOUNDS
+__device__ __forceinline__ bool sa_dbg_ok(int32_t *status, bool ok, int code, int64_t value)
+{
+    if (!ok && atomicCAS(status, 0, int(SA_E_BOUNDS)) == 0) {
+        status[1] = code;
+        status[2] = int32_t(value);
+        status[3] = int32_t(blockIdx.x * blockDim.x + threadIdx.x);
+    }
+    return ok;
+}
+#define SA_CHK(status, cond, code, value) sa_dbg_ok(status, cond, code, int64_t(value))
+#else
+#define SA_CHK(status, cond, code, value) true
+#endif
+
+// ---- PTX helpers shared by the kernels
+
+// x = hi + lo with hi the upper 19 bits of x (a TF32 number) and lo = x - hi (exact in fp32), itself cut to
+// TF32.  hi.hi + hi.lo + lo.hi then misses the true product by about 2^-20 relative.  (cvt.rna.tf32 costs
+// several instructions per value on this target; plain masking is one.)
+__device__ __forceinline__ void split_tf32(float x, uint32_t &hi, uint32_t &lo)
+{
+    hi = __float_as_uint(x) & 0xffffe000u;
+    lo = __float_as_uint(x - __uint_as_float(hi)) & 0xffffe000u;
+}
+
+__device__ __forceinline__ void mma_m16n8k8_tf32(float (&c)[4], const uint32_t (&a)[4], const uint32_t (&b)[2])
+{
+    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
+}
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+__device__ __forceinline__ void cp_async16_raw(uint32_t dst_smem, const void *src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst_smem), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
 // Sum `count` partial tiles into out rows (count == 0: zero fill).  Tile size in floats is a
 // power of two >= 16.  Block = 256 threads = W float4 columns x P phases over the partials;
 // grid = (entries, tile_f4 / W).  Fixed summation order: deterministic.

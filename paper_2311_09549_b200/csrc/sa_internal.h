@@ -104,19 +104,25 @@ struct sa_tensor {
                                               // group-per-fiber kernels (kernel 7, order-4 subtree kernel) stream, one 8-byte load
     int32_t *d_status = nullptr;              // [4] device status word
 
-    sa_worklist wl_main;                      // TTM3 / pass 1 of TTM4 / SDDMM-SpMM
-    sa_worklist wl_aux;                       // CSR: SpMM-GEMM row items; order-3 CSF: fiber rows (kernel 7); order-4 CSF: pass 2 of TTM4
-    sa_worklist wl_sub;                       // order-4 CSF: ranges of whole (i,j) subtrees for the subtree kernel of pass 1;
-                                              // empty when some subtree exceeds SA_SUB_MAX_F3 fibers or SA_SUB_MAX_NNZ nonzeros
+    sa_worklist wl_main;                      // TTM3 / SDDMM-SpMM; order-4 CSF: the order-3 lists over the large (i,j) subtrees
+    sa_worklist wl_aux;                       // CSR: SpMM-GEMM row items; order-3 CSF: fiber rows (kernel 7); order-4 CSF: partial
+                                              // slice tiles and fix-up entries of the fused kernel
+    sa_worklist wl_sub;                       // order-4 CSF: items of the fused kernel (runs of (i,j) subtrees)
+    // order-4 CSF: super-items (item0, item1, r0, r1) and pieces (sup0, sup1, first slice, last slice, destination of
+    // the first slice, of the last slice, r0, r1) of the fused kernel, see build_ttm4; subtrees above SA_SUB_MAX_NNZ
+    std::vector<int32_t> f4_supers, f4_pieces;
+    int32_t *d_f4_supers = nullptr, *d_f4_pieces = nullptr;
+    int32_t f4_n_large = 0;
 
     mutable std::atomic<int> last_launches{0};   // the only mutable field: concurrent sa_run calls may write it
     std::vector<void *> dev_blocks;           // everything obtained from the allocator
 };
 
-// Limits of the order-4 subtree kernel: level-2 fibers an item parks in shared memory, rows (subtrees) per item,
-// nonzeros of one subtree.
-constexpr int SA_SUB_MAX_F3 = 64;
-constexpr int SA_SUB_MAX_ROWS = 32;
+// Limits of the fused order-4 kernel: level-2 fiber rows a warp parks per batch, temporaries in a thread block's
+// pool (= subtrees per super-item), nonzeros of a subtree the kernel evaluates itself (larger ones go through the
+// order-3 kernel first).
+constexpr int SA_F4_ROWS = 32;
+constexpr int SA_F4_POOL = 64;
 constexpr int SA_SUB_MAX_NNZ = 4096;
 
 // ---- host builder (sa_build.cu)
@@ -131,7 +137,9 @@ struct sa_ttm3_view {
     const int32_t *crd_nz;        // per nonzero: row of the second factor
     const float *vals;
     const uint32_t *endbits;      // bit p set: nonzero p is the last of its fiber
-    int64_t n_fibers, n_out_rows, nnz;
+    int64_t n_fibers, n_out_rows;
+    int64_t nnz;                  // nonzeros the lists cover (chooses the register budget)
+    int64_t nnz_total;            // length of the index / value arrays (bounds of the self-checking build)
     int32_t *status;              // the tensor's device status word
 };
 sa_status sa_launch_ttm3_view(const sa_ttm3_view &v, const sa_dense &first, const sa_dense &second, float *out,

@@ -20,49 +20,12 @@
 
 namespace {
 
-// x = hi + lo with hi the upper 19 bits of x (a TF32 number) and lo = x - hi (exact in fp32), itself cut to
-// TF32.  hi.hi + hi.lo + lo.hi then misses the true product by about 2^-20 relative.  (cvt.rna.tf32 costs
-// several instructions per value on this target; plain masking is one.)
-__device__ __forceinline__ void split_tf32(float x, uint32_t &hi, uint32_t &lo)
-{
-    hi = __float_as_uint(x) & 0xffffe000u;
-    lo = __float_as_uint(x - __uint_as_float(hi)) & 0xffffe000u;
-}
-
-__device__ __forceinline__ void mma_m16n8k8_tf32(float (&c)[4], const uint32_t (&a)[4], const uint32_t (&b)[2])
-{
-    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
-}
-
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
-
-
-// Debug build (-DSA_DEBUG_BOUNDS): every index that comes out of the tensor's arrays is checked before it
-// is turned into an address; the first violation is recorded in the tensor's status word (read back by
-// sa_last_device_status) and the access is redirected to element 0.  Nothing traps.
+// Limits for the checks of the self-checking build (SA_CHK, sa_device.cuh).
 struct dbg_limits {
     int32_t *status;
     uint32_t c_rows, d_rows, n_fibers, n_slices_dim;
     int64_t nnz;
 };
-#ifdef SA_DEBUG_BOUNDS
-__device__ __forceinline__ bool dbg_ok(const dbg_limits &lim, bool ok, int code, int64_t value)
-{
-    if (!ok && atomicCAS(lim.status, 0, int(SA_E_BOUNDS)) == 0) {
-        lim.status[1] = code;
-        lim.status[2] = int32_t(value);
-        lim.status[3] = int32_t(blockIdx.x * blockDim.x + threadIdx.x);
-    }
-    return ok;
-}
-#define SA_CHK(lim, cond, code, value) dbg_ok(lim, cond, code, int64_t(value))
-#else
-#define SA_CHK(lim, cond, code, value) true
-#endif
 
 
 template <int L, int M>
@@ -88,11 +51,6 @@ struct cfg {
     static_assert(L * RS * 4 <= WARP_BYTES, "the CTA reduction reuses a warp's region for its tile");
 };
 
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
-__device__ __forceinline__ void cp_async16_raw(uint32_t dst_smem, const void *src)
-{
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst_smem), "l"(src) : "memory");
-}
 __device__ __forceinline__ void cp_async4_raw(uint32_t dst_smem, const void *src)
 {
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst_smem), "l"(src) : "memory");
@@ -100,13 +58,13 @@ __device__ __forceinline__ void cp_async4_raw(uint32_t dst_smem, const void *src
 __device__ __forceinline__ uint32_t lds32(uint32_t a)
 {
     uint32_t v;
-    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a));
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a) : "memory");
     return v;
 }
 __device__ __forceinline__ uint4 lds128(uint32_t a)
 {
     uint4 v;
-    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a) : "memory");
     return v;
 }
 __device__ __forceinline__ void sts32(uint32_t a, uint32_t v) { asm volatile("st.shared.u32 [%0], %1;" ::"r"(a), "r"(v) : "memory"); }
@@ -155,8 +113,8 @@ __device__ __forceinline__ void ttm3_flush(float (&acc)[cfg<L, M>::MT][cfg<L, M>
     {
         const bool va = t < n, vb = t + 4 < n;
         uint32_t oa = va ? __float_as_uint(ra[M]) : 0u, ob = vb ? __float_as_uint(rb[M]) : 0u;
-        if (!SA_CHK(lim, oa < lim.c_rows * ldc, 1, oa)) oa = 0u;
-        if (!SA_CHK(lim, ob < lim.c_rows * ldc, 2, ob)) ob = 0u;
+        if (!SA_CHK(lim.status, oa < lim.c_rows * ldc, 1, oa)) oa = 0u;
+        if (!SA_CHK(lim.status, ob < lim.c_rows * ldc, 2, ob)) ob = 0u;
         const float *ca = C + oa + g;
         const float *cb = C + ob + g;
 #pragma unroll
@@ -289,7 +247,7 @@ __device__ __forceinline__ void ttm3_warp_task(const sa_unit3 *__restrict__ unit
     auto fetch_round = [&](int slot) {
         if (fu < nu) {
             const int pg = fs.base + 8 * fr;
-            if (pg < fs.hi && pg + 8 > fs.lo && SA_CHK(lim, pg >= 0 && pg + 8 <= lim.nnz + 8, 3, pg)) {
+            if (pg < fs.hi && pg + 8 > fs.lo && SA_CHK(lim.status, pg >= 0 && pg + 8 <= lim.nnz + 8, 3, pg)) {
                 const uint32_t dst = s_kv + slot * (K::NS * K::SLOT);
                 if (c < 4) cp_async16_raw(dst + 16 * c, (c < 2 ? reinterpret_cast<const char *>(crd_k) : reinterpret_cast<const char *>(vals)) + 4 * int64_t(pg) + 16 * (c & 1));
                 else if (c == 4) cp_async4_raw(dst + 64, endbits + (pg >> 5));
@@ -314,7 +272,7 @@ __device__ __forceinline__ void ttm3_warp_task(const sa_unit3 *__restrict__ unit
     unit_head cnext = load_head(nu > 1 ? 1 : 0);        // the unit the consumer turns to next
     int fnext_q = load_sf(nu > 1 ? 1 : 0);              // and the fiber its stream q starts in
     int fq = load_sf(0);                                // next fiber this stream parks
-    if (!SA_CHK(lim, uint32_t(fq) <= lim.n_fibers, 4, fq)) fq = 0;
+    if (!SA_CHK(lim.status, uint32_t(fq) <= lim.n_fibers, 4, fq)) fq = 0;
     int jreg = __ldg(crd_j + fq + c);                   // C rows of the next eight fibers of the stream, one per lane
     const char *dlane = reinterpret_cast<const char *>(D + c * VEC);
     const uint32_t row_bytes = ldd * 4u;
@@ -325,7 +283,7 @@ __device__ __forceinline__ void ttm3_warp_task(const sa_unit3 *__restrict__ unit
         const uint4 ka = lds128(s_kv), kb = lds128(s_kv + 16);
         const uint32_t k8[8] = {ka.x, ka.y, ka.z, ka.w, kb.x, kb.y, kb.z, kb.w};
 #pragma unroll
-        for (int s = 0; s < 8; ++s) buf[s].load(dlane + uint64_t(SA_CHK(lim, k8[s] < lim.d_rows, 5, k8[s]) ? k8[s] : 0u) * row_bytes);
+        for (int s = 0; s < 8; ++s) buf[s].load(dlane + uint64_t(SA_CHK(lim.status, k8[s] < lim.d_rows, 5, k8[s]) ? k8[s] : 0u) * row_bytes);
     }
     float T[VEC];
 #pragma unroll
@@ -339,7 +297,7 @@ __device__ __forceinline__ void ttm3_warp_task(const sa_unit3 *__restrict__ unit
 #pragma unroll 1
       for (cr = 0; cr < rounds; ++cr) {
 #ifdef SA_DEBUG_BOUNDS
-        if (!SA_CHK(lim, ++dbg_rounds <= (1 << 16), 9, cs.rounds)) return;    // a task has at most ~300 rounds
+        if (!SA_CHK(lim.status, ++dbg_rounds <= (1 << 16), 9, cs.rounds)) return;    // a task has at most ~300 rounds
 #endif
         fetch_round(sc == 0 ? DEPTH - 1 : sc - 1);
         cp_async_wait<DEPTH - 2>();
@@ -378,7 +336,7 @@ __device__ __forceinline__ void ttm3_warp_task(const sa_unit3 *__restrict__ unit
         fq += cnt;
         const bool last = cr + 1 == rounds;
         if (last && cu + 1 < nu) fq = fnext_q;
-        if (!SA_CHK(lim, uint32_t(fq) <= lim.n_fibers, 6, fq)) fq = 0;
+        if (!SA_CHK(lim.status, uint32_t(fq) <= lim.n_fibers, 6, fq)) fq = 0;
         const int jnext = __ldg(crd_j + fq + c);
         // Eight steps: consume the row requested one round ago, then request the row of the same step of
         // the next round into the same registers.  MASKED: some stream of the warp is at a ragged end of
@@ -398,7 +356,7 @@ __device__ __forceinline__ void ttm3_warp_task(const sa_unit3 *__restrict__ unit
 #pragma unroll
                         for (int x = 0; x < VEC; ++x) T[x] = fmaf(v4[s4], buf[s].x[x], T[x]);
                     }
-                    buf[s].load(dlane + uint64_t(SA_CHK(lim, k4[s4] < lim.d_rows, 7, k4[s4]) ? k4[s4] : 0u) * row_bytes);
+                    buf[s].load(dlane + uint64_t(SA_CHK(lim.status, k4[s4] < lim.d_rows, 7, k4[s4]) ? k4[s4] : 0u) * row_bytes);
                     if (e8 & (1u << s)) {
                         rowvec<VEC> tv;
 #pragma unroll
@@ -450,10 +408,10 @@ __device__ __forceinline__ void ttm3_warp_task(const sa_unit3 *__restrict__ unit
         if (!keep) {
             if (HAD) {
                 if (M == 16) hacc += __shfl_xor_sync(SA_FULL_MASK, hacc, 16);
-                if (lane < M && SA_CHK(lim, uint32_t(crow) < lim.n_slices_dim, 8, crow)) sa_st_cs(out + int64_t(crow) * M + lane, hacc);
+                if (lane < M && SA_CHK(lim.status, uint32_t(crow) < lim.n_slices_dim, 8, crow)) sa_st_cs(out + int64_t(crow) * M + lane, hacc);
                 hacc = 0.f;
             } else {
-                if (SA_CHK(lim, uint32_t(crow) < lim.n_slices_dim, 8, crow)) store_tile<L, M>(acc, out + int64_t(crow) * (L * M), lane);
+                if (SA_CHK(lim.status, uint32_t(crow) < lim.n_slices_dim, 8, crow)) store_tile<L, M>(acc, out + int64_t(crow) * (L * M), lane);
                 zero_tile<L, M>(acc);
             }
         }
@@ -461,7 +419,7 @@ __device__ __forceinline__ void ttm3_warp_task(const sa_unit3 *__restrict__ unit
         if (cu < nu) {
             cs = stream_of(cnext.p0, cnext.p1, q);
             crow = cnext.row;
-            SA_CHK(lim, cs.rounds >= 1, 10, cu);
+            SA_CHK(lim.status, cs.rounds >= 1, 10, cu);
             if (cu + 1 < nu) {
                 cnext = load_head(cu + 1);
                 fnext_q = load_sf(cu + 1);
@@ -558,7 +516,7 @@ cudaError_t launch(const sa_ttm3_view &v, const sa_dense &first, const sa_dense 
     lim.status = v.status;
     lim.c_rows = uint32_t(first.rows); lim.d_rows = uint32_t(second.rows);
     lim.n_fibers = uint32_t(v.n_fibers); lim.n_slices_dim = uint32_t(v.n_out_rows);
-    lim.nnz = v.nnz;
+    lim.nnz = v.nnz_total;
     kern<<<(unsigned)ctas, 32 * SA_TTM3_WARPS, smem, stream>>>(wl.d_units3, wl.d_task_start, n_tasks, int(wl.n_group_ctas), v.crd_fiber,
                                                               v.crd_nz, v.vals, v.endbits, first.ptr, uint32_t(first.ld), second.ptr,
                                                               uint32_t(second.ld), out, partial, lim);
@@ -609,6 +567,7 @@ sa_status sa_launch_ttm3(const sa_tensor *t, const sa_dense *ops, float *out, vo
     v.n_fibers = t->count[1];
     v.n_out_rows = t->dims[0];
     v.nnz = t->nnz;
+    v.nnz_total = t->nnz;
     v.status = t->d_status;
     return sa_launch_ttm3_view(v, ops[0], ops[1], out, static_cast<float *>(ws), stream, launches);
 }
@@ -630,6 +589,7 @@ sa_status sa_launch_mttkrp_rows(const sa_tensor *t, const sa_dense &C, const sa_
     v.n_fibers = t->count[1];
     v.n_out_rows = t->dims[0];
     v.nnz = t->nnz;
+    v.nnz_total = t->nnz;
     v.status = t->d_status;
     const cudaError_t e = R == 32 ? launch<16, 32, true>(v, C, D, out, partial, stream) : launch<16, 16, true>(v, C, D, out, partial, stream);
     if (e != cudaSuccess) return SA_E_CUDA;

@@ -76,12 +76,13 @@ def test_levels_match_independent_construction(cfg):
 @pytest.mark.parametrize("cfg", [1, 2, 5])
 def test_csf_worklist_partitions_every_nonzero_once(cfg):
     """Main list of a CSF tensor: the units of the order-3 kernel.  For an order-4 tensor its "slices" are the
-    (i,j) subtrees (output row = index of the level-1 fiber) and its fibers the (i,j,k) fibers."""
+    large (i,j) subtrees (more than 4096 nonzeros; output row = index among the large ones) and its fibers the
+    (i,j,k) fibers; the other subtrees are covered by the items of the fused kernel."""
     w = configs.make(cfg, "mini")
     coords, vals = w.coords, w.vals
     if cfg == 5:
-        # two (i,j) subtrees that the subtree kernel does not take (more than 4096 nonzeros), so that the main
-        # list of the order-4 tensor is not empty; all the others are in the third list
+        # two (i,j) subtrees that the fused kernel does not evaluate itself (more than 4096 nonzeros), so that the
+        # main list of the order-4 tensor is not empty; all the others are in the third list
         keep = ~(((coords[:, 0] == 3) & (coords[:, 1] == 5)) | ((coords[:, 0] == 200) & (coords[:, 1] == 7)))
         k, o = np.divmod(np.arange(4800), 40)
         extra = [np.stack([np.full(4800, i), np.full(4800, j), k, o], axis=1) for i, j in ((3, 5), (200, 7))]
@@ -94,16 +95,21 @@ def test_csf_worklist_partitions_every_nonzero_once(cfg):
     n_items, n_groups, n_fix, n_slots = (int(x) for x in counts)
     if t.order == 3:
         slice_rows, pos1, pos2 = levels[0][1], levels[1][0], levels[2][0]
+        slice_pos = {int(c): n for n, c in enumerate(slice_rows)}
     else:
         pos1, pos2 = levels[2][0], levels[3][0]
-        slice_rows = np.arange(len(pos1) - 1)
-    slice_pos = {int(c): n for n, c in enumerate(slice_rows)}
+        nz_sub = pos2[pos1[1:]] - pos2[pos1[:-1]]
+        large = np.nonzero(nz_sub > 4096)[0]
+        assert len(large) == 2
+        slice_rows = np.arange(len(large))
+        slice_pos = {n: int(r) for n, r in enumerate(large)}      # output row = index among the large subtrees
     covered = np.zeros(nnz_all, dtype=np.int32)
     if t.order == 4:
         sub = sa.sa_tensor_worklist(t.handle, 2)[1]
         assert len(sub) > 0 and n_items > 0
-        for row, row_end, f0, f1, p0, p1, dest, _ in sub:
-            covered[p0:p1] += 1                  # the small subtrees are evaluated from the third list
+        for row, row_end, f0, f1, p0, p1, dest, kind in sub:
+            if kind == 0:
+                covered[p0:p1] += 1              # the other subtrees are evaluated from the third list
     slot_owner = {}
     G = 4                                   # warps (tasks) per thread block of the order-3 kernel
     task_start, stream_f0 = sa.sa_tensor_tasks(t.handle)
@@ -142,7 +148,7 @@ def test_csf_worklist_partitions_every_nonzero_once(cfg):
     if t.order == 3:
         assert empties == set(range(w.dims[0])) - set(int(c) for c in slice_rows)
     else:
-        assert not empties, "every level-1 fiber has nonzeros"
+        assert not empties, "every large subtree has nonzeros"
     # nonzero balance: no unit is larger than the small-slice bound / the piece size
     sizes = items[:, 5] - items[:, 4]
     assert sizes.max() <= max(4096, int(np.ceil(nnz_all / 8)))
@@ -167,36 +173,104 @@ def test_csf_worklist_partitions_every_nonzero_once(cfg):
                 assert f == f0
 
 
-def test_order4_second_pass_worklist_covers_every_fiber_quarter_once():
-    """Second list of an order-4 tensor: (piece of a slice) x (quarter of the temporaries' columns)."""
-    w = configs.make(5, "mini")
-    t = sa.SparseTensor(w.dims, w.coords, w.vals, sa.SA_FMT_CSF, device=-1)
+def _order4_lists(t):
     levels, _ = export_all(t, "csf")
-    crd0, pos1 = levels[0][1], levels[1][0]
-    counts, items, fix = sa.sa_tensor_worklist(t.handle, 1)
-    slice_pos = {int(c): n for n, c in enumerate(crd0)}
-    covered = np.zeros((len(levels[1][1]), 4), dtype=np.int32)
-    pieces = {}
-    for row, row_end, f0, f1, _, _, dest, quarter in items:
-        s = slice_pos[int(row)]
-        assert pos1[s] <= f0 < f1 <= pos1[s + 1] and f1 - f0 <= 512 and 0 <= quarter < 4
-        covered[f0:f1, quarter] += 1
-        if dest >= 0:
-            pieces.setdefault(int(row), set()).add(int(dest))
+    items = sa.sa_tensor_worklist(t.handle, 2)[1]
+    counts3, pieces, supers = sa.sa_tensor_worklist(t.handle, 3)
+    counts1, _, fix = sa.sa_tensor_worklist(t.handle, 1)
+    return levels, items, pieces, supers, fix, int(counts3[1]), int(counts1[3])
+
+
+def check_order4_fused_lists(t, dims0):
+    """Items, super-items and pieces of the fused order-4 kernel: every (i,j) subtree belongs to exactly one item,
+    the items of a super-item and the super-items of a piece are consecutive and fit the pool, and every slice
+    has exactly one destination per piece it lies in."""
+    levels, items, pieces, supers, fix, n_large, n_slots = _order4_lists(t)
+    crd0, pos1, pos2, pos3 = levels[0][1], levels[1][0], levels[2][0], levels[3][0]
+    F2 = len(pos1) and int(pos1[-1])
+    nz_sub = pos3[pos2[1:]] - pos3[pos2[:-1]]
+    is_large = nz_sub > 4096
+    assert n_large == int(is_large.sum())
+    large_ord = np.cumsum(is_large) - 1
+    seen = np.zeros(F2, dtype=np.int32)
+    for r0, r1, f0, f1, p0, p1, dest, kind in items:
+        assert r0 < r1 <= F2 and r1 - r0 <= 32
+        seen[r0:r1] += 1
+        if kind == 0:
+            assert not is_large[r0:r1].any()
+            assert (f0, f1) == (pos2[r0], pos2[r1]) and (p0, p1) == (pos3[f0], pos3[f1])
+            assert f1 - f0 <= 32 or r1 - r0 == 1, "more than one batch of fibers only for a single subtree"
         else:
-            assert (f0, f1) == (pos1[s], pos1[s + 1])
-    assert (covered == 1).all()
-    assert (np.diff(items[:, 3] - items[:, 2]) <= 0).all(), "largest items first"
+            assert kind == 1 and is_large[r0:r1].all() and r1 - r0 <= 8
+            assert f0 == large_ord[r0] and f1 - f0 == r1 - r0
+    assert (seen == 1).all()
+    # super-items: consecutive items, consecutive subtrees, at most 64 subtrees
+    nxt_item, nxt_r = 0, 0
+    for i0, i1, r0, r1 in supers:
+        assert i0 == nxt_item and i1 > i0 and r0 == nxt_r and 0 < r1 - r0 <= 64
+        assert items[i0][0] == r0 and items[i1 - 1][1] == r1
+        assert all(items[k][1] == items[k + 1][0] for k in range(i0, i1 - 1))
+        nxt_item, nxt_r = i1, r1
+    assert nxt_item == len(items) and nxt_r == F2
+    # pieces: consecutive super-items; slices and destinations
+    slot_user = {}
+    nxt_sup = 0
+    dests = {}
+    for sup0, sup1, sa_, sb_, d_first, d_last, r0, r1 in pieces:
+        assert sup0 == nxt_sup and sup1 > sup0 and supers[sup0][2] == r0 and supers[sup1 - 1][3] == r1
+        nxt_sup = sup1
+        assert pos1[sa_] <= r0 < pos1[sa_ + 1] and pos1[sb_] < r1 <= pos1[sb_ + 1] and sa_ <= sb_
+        for s_ in range(sa_, sb_ + 1):
+            whole = r0 <= pos1[s_] and pos1[s_ + 1] <= r1
+            d = d_first if s_ == sa_ else d_last if s_ == sb_ else -1
+            if whole:
+                assert d == -1, "a slice inside one piece goes straight to the output"
+            else:
+                assert d >= 0 and d not in slot_user
+                slot_user[d] = s_
+            dests.setdefault(s_, []).append(d)
+        if sa_ == sb_:
+            assert d_first == d_last
+    assert nxt_sup == len(supers)
+    used = np.zeros(n_slots, dtype=np.int32)
     empties = set()
-    used = np.zeros(int(counts[3]), dtype=np.int32)
     for row, slot0, count, _ in fix:
         if count == 0:
             empties.add(int(row))
             continue
-        assert pieces[int(row)] == set(range(slot0, slot0 + count))
+        s_ = int(np.nonzero(crd0 == row)[0][0])
+        assert dests[s_] == list(range(slot0, slot0 + count)), "one partial tile per piece, in piece order"
         used[slot0:slot0 + count] += 1
-    assert (used == 1).all()
-    assert empties == set(range(w.dims[0])) - set(int(c) for c in crd0)
+    assert (used == 1).all() and set(slot_user) == set(range(n_slots))
+    assert empties == set(range(dims0)) - set(int(c) for c in crd0)
+    return items, pieces, supers
+
+
+def test_order4_fused_worklists_cover_every_subtree_once():
+    w = configs.make(5, "mini")
+    t = sa.SparseTensor(w.dims, w.coords, w.vals, sa.SA_FMT_CSF, device=-1)
+    items, pieces, supers = check_order4_fused_lists(t, w.dims[0])
+    assert len(pieces) > 4, "the mini tensor spans several pieces"
+    # a tensor with one slice: every piece is inside it and leaves a partial tile
+    keep = w.coords[:, 0] == w.coords[0, 0]
+    one = np.ascontiguousarray(w.coords[keep])
+    t1 = sa.SparseTensor(w.dims, one, w.vals[keep], sa.SA_FMT_CSF, device=-1)
+    check_order4_fused_lists(t1, w.dims[0])
+
+
+def test_order4_large_and_many_fiber_subtrees():
+    """A subtree above 4096 nonzeros is left to the order-3 lists (item of kind 1); one with 130 fibers but few
+    nonzeros is a single item of kind 0 that the kernel evaluates in batches."""
+    k, o = np.divmod(np.arange(4800), 40)
+    big = np.stack([np.zeros(4800), np.zeros(4800), k, o], axis=1).astype(np.int32)
+    many = np.stack([np.ones(130), np.ones(130), np.arange(130), np.zeros(130)], axis=1).astype(np.int32)
+    both = np.concatenate([big, many, np.array([[1, 2, 5, 1]], np.int32)])
+    t2 = sa.SparseTensor((2, 3, 130, 40), both, np.ones(len(both), np.float32), sa.SA_FMT_CSF, device=-1)
+    items, pieces, supers = check_order4_fused_lists(t2, 2)
+    kinds = {(int(x[0]), int(x[1])): int(x[7]) for x in items}
+    assert kinds == {(0, 1): 1, (1, 2): 0, (2, 3): 0}
+    main = sa.sa_tensor_worklist(t2.handle, 0)[1]
+    assert set(main[:, 0].tolist()) == {0} and (main[:, 5] - main[:, 4]).sum() == 4800
 
 
 @pytest.mark.parametrize("cfg,which", [(3, 0), (4, 1), (4, 0)])
@@ -351,34 +425,3 @@ def test_fiber_row_worklist_of_order3_csf_partitions_fibers_and_nonzeros():
           for s in (sa.SA_SCHED_DEFAULT, sa.SA_SCHED_FUSED, sa.SA_SCHED_ASSOC_LEFT, sa.SA_SCHED_ASSOC_RIGHT)}
     assert ws[sa.SA_SCHED_FUSED] == ws[sa.SA_SCHED_ASSOC_LEFT] >= n_fibers * 32 * 4
     assert ws[sa.SA_SCHED_DEFAULT] == ws[sa.SA_SCHED_ASSOC_RIGHT] >= dims[2] * 32 * 4
-
-
-def test_order4_subtree_worklist_covers_every_subtree_once_within_its_limits():
-    """Third list of an order-4 tensor: ranges of whole small (i,j) subtrees, at most 64 level-2 fibers and 32
-    subtrees each; a larger subtree is left to the main list."""
-    w = configs.make(5, "mini")
-    t = sa.SparseTensor(w.dims, w.coords, w.vals, sa.SA_FMT_CSF, device=-1)
-    levels, _ = export_all(t, "csf")
-    pos2, pos3 = levels[2][0], levels[3][0]
-    counts, items, fix = sa.sa_tensor_worklist(t.handle, 2)
-    assert counts[0] > 0 and counts[2] == 0 and counts[3] == 0
-    n_sub = int(t.info()[1][1])
-    seen = np.zeros(n_sub, dtype=np.int32)
-    for row, row_end, f0, f1, p0, p1, dest, _ in items:
-        assert row_end > row and dest < 0
-        assert (f0, f1) == (pos2[row], pos2[row_end]) and (p0, p1) == (pos3[f0], pos3[f1])
-        assert f1 - f0 <= 64 and row_end - row <= 32
-        seen[row:row_end] += 1
-    # the others are the large ones, and the main list holds exactly those
-    large = np.nonzero(seen == 0)[0]
-    assert (seen <= 1).all()
-    f3s, nz = np.diff(pos2), pos3[pos2[1:]] - pos3[pos2[:-1]]
-    assert ((f3s[large] > 64) | (nz[large] > 4096)).all() and ((f3s[seen == 1] <= 64) & (nz[seen == 1] <= 4096)).all()
-    assert set(sa.sa_tensor_worklist(t.handle, 0)[1][:, 0].tolist()) == set(large.tolist())
-    # one (i,j) pair with 130 level-2 fibers next to a small one: the large one is in the main list only
-    big = np.stack([np.zeros(130), np.zeros(130), np.arange(130), np.zeros(130)], axis=1).astype(np.int32)
-    both = np.concatenate([big, np.array([[1, 1, 5, 1]], np.int32)])
-    t2 = sa.SparseTensor((2, 2, 130, 2), both, np.ones(131, np.float32), sa.SA_FMT_CSF, device=-1)
-    sub = sa.sa_tensor_worklist(t2.handle, 2)[1]
-    main = sa.sa_tensor_worklist(t2.handle, 0)[1]
-    assert [tuple(x[:2]) for x in sub.tolist()] == [(1, 2)] and set(main[:, 0].tolist()) == {0}

@@ -191,21 +191,25 @@ def test_spmm_gemm_rank_combinations_and_long_rows(sa, L, M):
 
 
 def test_ttm4_ragged_and_split_slices(sa):
-    # few level-1 fibers per slice: the head slice's (i,j) subtrees exceed one thread block's chunk, so the
-    # first pass writes partial temporaries that the fix-up kernel sums
+    # few level-1 fibers per slice: the head slice's (i,j) subtrees are above the size the fused kernel evaluates
+    # itself, so the order-3 kernel writes their temporaries first (some split over several thread blocks, with
+    # partial temporaries that the fix-up kernel sums) and items of kind 1 copy them into the pool
     w = configs.make_ttm4_zipf("edge4", 31, 90, 6, 130, 110, 150_000, 1.4, 5.0, 16, 16, 16)
     A, t = _check(sa, w)
     assert sa.sa_tensor_worklist(t.handle, 0)[0][3] >= 2, "a large (i,j) subtree must be split over several thread blocks"
-    # many level-1 fibers per slice: the second pass cuts the head slices into pieces of 512 fibers
+    kinds = sa.sa_tensor_worklist(t.handle, 2)[1][:, 7]
+    assert (kinds == 1).any() and (kinds == 0).any()
+    # many level-1 fibers per slice: the head slices span several pieces and leave partial slice tiles
     w = configs.make_ttm4_zipf("edge4b", 32, 90, 700, 50, 45, 150_000, 1.4, 5.0, 16, 16, 16)
     A, t = _check(sa, w)
     assert sa.sa_tensor_worklist(t.handle, 1)[0][3] >= 2, "the head slice must be split into several pieces"
-    # both kernels of the first pass in one run: small subtrees (third list) and large ones (main list)
+    # subtrees with more level-2 fibers than one batch holds next to small ones
     for w in (configs.make_ttm4_zipf("edge4c", 33, 90, 40, 160, 110, 150_000, 1.4, 5.0, 16, 16, 16),
               configs.make_ttm4_zipf("edge4d", 34, 400, 60, 150, 40, 200_000, 1.2, 3.0, 16, 16, 16)):
         A, t = _check(sa, w)
-        n_main, n_sub = (int(sa.sa_tensor_worklist(t.handle, x)[0][0]) for x in (0, 2))
-        assert n_main > 0 and n_sub > 0, (n_main, n_sub)
+        items = sa.sa_tensor_worklist(t.handle, 2)[1]
+        nf = items[:, 3] - items[:, 2]
+        assert ((items[:, 7] == 0) & (nf > 32)).any() and ((items[:, 7] == 0) & (nf <= 32) & (items[:, 1] - items[:, 0] > 1)).any()
 
 
 def test_results_are_reproducible_run_to_run(sa):
@@ -285,8 +289,8 @@ def test_dense_stage_ragged_rows_and_padded_leading_dimensions(sa, L, M):
 
 
 def test_ttm4_padded_factor_matrices(sa):
-    """Order-4 chain with the factor matrices given as padded views (leading dimension 20): the subtree kernel's
-    general-stride variant and the order-3 kernel's row addressing."""
+    """Order-4 chain with the factor matrices given as padded views (leading dimension 20): the fused kernel's
+    general-stride variant."""
     import torch
     w = configs.make_ttm4_zipf("edge4e", 35, 300, 60, 150, 40, 120_000, 1.2, 3.0, 16, 16, 16)
     A_ref, S_ref = oracle.evaluate(w)

@@ -350,7 +350,7 @@ def make_spmm_gemm(name, seed, I, J, nnz, L, M):
 # --------------------------------------------------------------------------- presets
 
 def make(config, scale="full", seed=None):
-    """Build workload ``config`` (1..5) at ``scale`` 'full' or 'mini' ('mid' exists for config 4 only)."""
+    """Build workload ``config`` (1..5) at ``scale`` 'full' or 'mini' ('mid', a quarter-size profiling case, exists for configs 2, 4, 5 and 8)."""
     config = int(config)
     s = BASE_SEED + config if seed is None else int(seed)
     full = scale == "full"
@@ -359,6 +359,8 @@ def make(config, scale="full", seed=None):
     if config == 2:
         if full:
             return make_ttm3_zipf("cfg2-ttm3-zipf", s, 100000, 80000, 80000, 50_000_000, 1.2, 8.0, 32, 32)
+        if scale == "mid":      # a quarter of the slices and nonzeros, same factor tables (profiling case)
+            return make_ttm3_zipf("cfg2-ttm3-zipf-mid", s, 25000, 80000, 80000, 12_500_000, 1.2, 8.0, 32, 32)
         return make_ttm3_zipf("cfg2-ttm3-zipf-mini", s, 3000, 700, 900, 250_000, 1.2, 8.0, 32, 32)
     if config == 3:
         if full:
@@ -373,6 +375,9 @@ def make(config, scale="full", seed=None):
     if config == 5:
         if full:
             return make_ttm4_zipf("cfg5-ttm4-zipf", s, 50_000, 20_000, 20_000, 20_000, 100_000_000,
+                                  1.2, 6.0, 16, 16, 16)
+        if scale == "mid":      # a quarter of the slices and nonzeros, same factor tables (profiling case)
+            return make_ttm4_zipf("cfg5-ttm4-zipf-mid", s, 12_500, 20_000, 20_000, 20_000, 25_000_000,
                                   1.2, 6.0, 16, 16, 16)
         return make_ttm4_zipf("cfg5-ttm4-zipf-mini", s, 600, 150, 120, 130, 200_000, 1.2, 6.0, 16, 16, 16)
     if config == 6:
