@@ -49,9 +49,9 @@ NCU_TRAFFIC = {
 }
 
 
-def ncu_traffic(workload):
+def ncu_traffic(workload, sched=None):
     import hashlib
-    e = NCU_TRAFFIC.get(workload)
+    e = NCU_TRAFFIC.get((workload, sched)) or NCU_TRAFFIC.get(workload)
     if e is None:
         return None, None
     try:
@@ -309,7 +309,7 @@ def workload_label(cfg, sched):
 
 
 def label(args):
-    return workload_label(args.workload, args.sched) + ("" if args.scale == "full" else " [%s-scale stand-in]" % args.scale)
+    return workload_label(args.workload or 2, args.sched) + ("" if args.scale == "full" else " [%s-scale stand-in]" % args.scale)
 
 
 def run_reference(args, w, rank, world):
@@ -334,19 +334,142 @@ def run_reference(args, w, rank, world):
     print(json.dumps(line), flush=True)
 
 
+def measure(sa, torch, dist, w, sched_name, steps, warmup, e2e_steps, dev, rank, world, sample_clocks=True,
+            gather_probe=False, scale="full", workload_id=None):
+    """Time ``steps`` steps of workload ``w`` (after ``warmup`` untimed ones) with CUDA events on the launching
+    stream, then the same call end to end from / to pinned host memory.  Returns the record of one
+    (config, schedule) pair (rank 0; other ranks return None after taking part in the barriers)."""
+    fmt = sa.SA_FMT_CSR if w.fmt == "csr" else sa.SA_FMT_CSF
+    t0 = time.perf_counter()
+    tensor = sa.SparseTensor(w.dims, w.coords, w.vals, fmt, device=dev.index)
+    build_s = time.perf_counter() - t0
+    nnz, counts, n_chunks = tensor.info()
+    sched = {"left": sa.SA_SCHED_ASSOC_LEFT, "right": sa.SA_SCHED_ASSOC_RIGHT, "default": sa.SA_SCHED_DEFAULT,
+             "fused": sa.SA_SCHED_DEFAULT}[sched_name]
+    host_ops = [torch.from_numpy(np.ascontiguousarray(x)).pin_memory() for x in w.dense]
+    ops = [x.to(dev, non_blocking=False) for x in host_ops]
+    out = torch.empty(w.out_shape, dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream(dev)
+
+    def step():
+        tensor.run(w.expr, ops, out=out, sched=sched, stream=stream)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    for _ in range(warmup):
+        step()
+    launches_per_step = sa.sa_last_launch_count(tensor.handle)
+    barrier()
+    sampler = ClockSampler(dev.index)
+    if rank == 0 and sample_clocks:
+        sampler.start()
+        time.sleep(0.3)
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    barrier()
+    evs[0].record(stream)
+    for k in range(steps):
+        step()
+        evs[k + 1].record(stream)
+    barrier()
+    total_ms = evs[0].elapsed_time(evs[-1])
+    per_step = [evs[k].elapsed_time(evs[k + 1]) for k in range(steps)]
+    clocks = None
+    if rank == 0 and sample_clocks:
+        # keep the GPU busy a little longer so that the clock sampler sees the loaded state
+        t_end = time.perf_counter() + 1.0
+        while time.perf_counter() < t_end:
+            for _ in range(20):
+                step()
+            torch.cuda.synchronize(dev)
+        clocks = sampler.stop()
+
+    # end to end: dense operands from pinned host memory, result back to pinned host memory
+    host_out = torch.empty(w.out_shape, dtype=torch.float32).pin_memory()
+    e2e_steps = max(1, min(e2e_steps, steps))
+
+    def e2e_step():
+        dops = [x.to(dev, non_blocking=True) for x in host_ops]
+        tensor.run(w.expr, dops, out=out, sched=sched, stream=stream)
+        host_out.copy_(out, non_blocking=True)
+
+    e2e_step()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record(stream)
+    barrier()
+    e2e_ms = e0.elapsed_time(e1) / e2e_steps
+    total_ms, e2e_ms = reduce_max_over_ranks([total_ms, e2e_ms], dev, world)
+    ms_per_step = total_ms / steps
+    rec = None
+    if rank == 0:
+        peaks, peak_kind = measured_peaks()
+        # the schedule that ran: the library's choice when the default was asked for
+        ran = sched_name
+        if sched_name == "default" and w.expr in ("spmm_gemm", "spttm_spttm"):
+            ops_desc = [(x.data_ptr(), x.shape[0], x.shape[1], x.stride(0)) for x in ops]
+            ws = {k: sa.sa_workspace_size(tensor.handle, sa._EXPR_OF[w.expr], v, ops_desc)
+                  for k, v in (("default", sa.SA_SCHED_DEFAULT), ("left", sa.SA_SCHED_ASSOC_LEFT), ("right", sa.SA_SCHED_ASSOC_RIGHT))}
+            ran = "left" if ws["default"] == ws["left"] and ws["left"] != ws["right"] else "right"
+        abytes, aflops = algorithmic_work(w, counts, ran if w.expr in ("spmm_gemm", "spttm_spttm") else "fused")
+        achieved = abytes / (ms_per_step * 1e-3) / 1e9
+        traffic, traffic_kernel = ncu_traffic(workload_id, ran) if scale == "full" else (None, None)
+        rec = {
+            "workload": workload_label(workload_id, sched_name) + ("" if scale == "full" else " [%s-scale stand-in]" % scale),
+            "schedule": sched_name if sched_name == ran else "%s (ran %s)" % (sched_name, ran),
+            "value": aggregate_throughput(nnz, world, ms_per_step), "unit": "GNNZ/s", "ms_per_step": ms_per_step,
+            "steps": steps, "warmup": warmup, "step_ms_median": statistics.median(per_step),
+            "step_ms_stdev": statistics.pstdev(per_step), "nnz": nnz, "level_counts": [int(c) for c in counts],
+            "work_items": int(n_chunks), "build_s": round(build_s, 3),
+            "l2": "inputs + output exceed L2 (126 MB); no flush" if abytes > 200e6 else "smaller than L2; launch-bound",
+            "gflops": aflops / (ms_per_step * 1e-3) / 1e9,
+            "hbm_gbs_algorithmic": achieved, "hbm_frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS,
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": achieved / peaks["hbm_gbs"], "traffic": traffic, "peak_kind": "of " + peak_kind,
+                         "kernel": "whole step (main kernel(s) + fix-up, fix-up <= 4 % by the ncu launch lists)",
+                         "traffic_kernel": traffic_kernel, "algorithmic_bytes_per_launch": abytes},
+            "e2e": {"value": aggregate_throughput(nnz, world, e2e_ms), "unit": "GNNZ/s",
+                    "h2d_bytes_per_step": sum(int(x.numel()) * 4 for x in host_ops),
+                    "d2h_bytes_per_step": int(host_out.numel()) * 4, "ms_per_step": e2e_ms},
+            "gpu_launches": launches_per_step * steps, "clocks": clocks,
+        }
+        if gather_probe and scale == "full":
+            gather = l2_gather_ceiling(sa, torch, w, ops, dev, stream)
+            if gather is not None:
+                rec["l2_gather_ceiling"] = gather
+    tensor.close()
+    del ops, out, host_ops, host_out
+    torch.cuda.empty_cache()
+    return rec
+
+
+# (config, schedule) pairs of the default run besides the headline config 2
+PER_CONFIG = [(1, "fused"), (3, "fused"), (4, "left"), (4, "right"), (4, "default"), (5, "fused")]
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=31)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", type=int, default=2, choices=[1, 2, 3, 4, 5, 6, 7, 8, 9, 10])
+    ap.add_argument("--workload", type=int, default=None, choices=[1, 2, 3, 4, 5, 6, 7, 8, 9, 10],
+                    help="one workload only; without it: config 2 as the headline plus a per_config list of all five configs")
     ap.add_argument("--scale", default="full", choices=["full", "mid", "mini"])
-    ap.add_argument("--sched", default="right", choices=["left", "right"], help="association order for workloads 4 and 10")
+    ap.add_argument("--sched", default="right", choices=["left", "right", "default"], help="association order for workloads 4 and 10")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-per-config", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=5)
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    all_configs = args.workload is None and not args.no_per_config and args.scale == "full" and args.impl == "ours"
+    if args.workload is None:
+        args.workload = 2
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -368,116 +491,60 @@ def main():
     dev = torch.device("cuda", local_rank)
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
+    all_configs = all_configs and world == 1
+
+    # the other configs' inputs are generated on host threads while the GPU runs (numpy releases the GIL)
+    pending = {}
+    pool = None
+    if all_configs:
+        from concurrent.futures import ThreadPoolExecutor
+        pool = ThreadPoolExecutor(max_workers=2)
+        for cfg in sorted({c for c, _ in PER_CONFIG}, key=lambda c: (c != 5, c != 4, c)):
+            pending[cfg] = pool.submit(configs.make, cfg, "full")
 
     w = configs.make(args.workload, args.scale)
-    fmt = sa.SA_FMT_CSR if w.fmt == "csr" else sa.SA_FMT_CSF
-    t0 = time.perf_counter()
-    tensor = sa.SparseTensor(w.dims, w.coords, w.vals, fmt, device=local_rank)
-    build_s = time.perf_counter() - t0
-    nnz, counts, n_chunks = tensor.info()
-    sched = sa.SA_SCHED_DEFAULT
-    if w.expr in ("spmm_gemm", "spttm_spttm"):
-        sched = sa.SA_SCHED_ASSOC_LEFT if args.sched == "left" else sa.SA_SCHED_ASSOC_RIGHT
-
-    host_ops = [torch.from_numpy(np.ascontiguousarray(x)).pin_memory() for x in w.dense]
-    ops = [x.to(dev, non_blocking=False) for x in host_ops]
-    out = torch.empty(w.out_shape, dtype=torch.float32, device=dev)
-    stream = torch.cuda.current_stream(dev)
-
-    def step():
-        tensor.run(w.expr, ops, out=out, sched=sched, stream=stream)
-
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize(dev)
-
-    for _ in range(args.warmup):
-        step()
-    launches_per_step = sa.sa_last_launch_count(tensor.handle)
-    barrier()
-    sampler = ClockSampler(local_rank)
+    sched_name = args.sched if w.expr in ("spmm_gemm", "spttm_spttm") else "fused"
+    rec = measure(sa, torch, dist, w, sched_name, args.steps, args.warmup, args.e2e_steps, dev, rank, world,
+                  gather_probe=True, scale=args.scale, workload_id=args.workload)
     if rank == 0:
-        sampler.start()
-        time.sleep(0.3)
-    evs = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
-    barrier()
-    evs[0].record(stream)
-    for k in range(args.steps):
-        step()
-        evs[k + 1].record(stream)
-    barrier()
-    total_ms = evs[0].elapsed_time(evs[-1])
-    per_step = [evs[k].elapsed_time(evs[k + 1]) for k in range(args.steps)]
-    # keep the GPU busy a little longer so that the clock sampler sees the loaded state
-    if rank == 0:
-        t_end = time.perf_counter() + 1.0
-        while time.perf_counter() < t_end:
-            for _ in range(20):
-                step()
-            torch.cuda.synchronize(dev)
-        clocks = sampler.stop()
-    else:
-        clocks = None
-
-    # end to end: dense operands from pinned host memory, result back to pinned host memory
-    host_out = torch.empty(w.out_shape, dtype=torch.float32).pin_memory()
-    e2e_steps = max(1, min(args.e2e_steps, args.steps))
-
-    def e2e_step():
-        dops = [x.to(dev, non_blocking=True) for x in host_ops]
-        tensor.run(w.expr, dops, out=out, sched=sched, stream=stream)
-        host_out.copy_(out, non_blocking=True)
-
-    e2e_step()
-    barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for _ in range(e2e_steps):
-        e2e_step()
-    e1.record(stream)
-    barrier()
-    e2e_ms = e0.elapsed_time(e1) / e2e_steps
-
-    total_ms, e2e_ms = reduce_max_over_ranks([total_ms, e2e_ms], dev, world)
-    ms_per_step = total_ms / args.steps
-
-    if rank == 0:
-        peaks, peak_kind = measured_peaks()
-        sched_name = args.sched if w.expr in ("spmm_gemm", "spttm_spttm") else "fused"
-        abytes, aflops = algorithmic_work(w, counts, sched_name)
-        gnnz = aggregate_throughput(nnz, world, ms_per_step)
-        achieved = abytes / (ms_per_step * 1e-3) / 1e9
-        h2d = sum(int(x.numel()) * 4 for x in host_ops)
-        d2h = int(host_out.numel()) * 4
-        traffic, traffic_kernel = ncu_traffic(args.workload) if args.scale == "full" else (None, None)
         line = {
-            "metric": METRIC, "value": gnnz, "unit": "GNNZ/s", "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "metric": METRIC, "value": rec["value"], "unit": "GNNZ/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": rec["ms_per_step"], "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": label(args), "scale": args.scale, "nnz": nnz,
-                       "level_counts": [int(c) for c in counts], "work_items": int(n_chunks),
-                       "l2": "inputs + output exceed L2 (126 MB); no flush" if abytes > 200e6 else "smaller than L2; launch-bound",
-                       "parallelism": "replicas x%d" % world, "build_s": round(build_s, 3),
-                       "step_ms_median": statistics.median(per_step), "step_ms_stdev": statistics.pstdev(per_step)},
-            "gflops": aflops / (ms_per_step * 1e-3) / 1e9,
-            "hbm_gbs_algorithmic": achieved, "hbm_frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS,
-            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                         "frac": achieved / peaks["hbm_gbs"], "traffic": traffic, "peak_kind": "of " + peak_kind,
-                         "kernel": "whole step (main kernel(s) + fix-up, fix-up <= 2 % by the ncu launch list)",
-                         "traffic_kernel": traffic_kernel, "algorithmic_bytes_per_launch": abytes},
-            "e2e": {"value": aggregate_throughput(nnz, world, e2e_ms), "unit": "GNNZ/s", "h2d_bytes_per_step": h2d,
-                    "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
-            "gpu_launches": launches_per_step * args.steps,
-            "clocks": clocks,
+            "config": {"workload": rec["workload"], "scale": args.scale, "nnz": rec["nnz"],
+                       "level_counts": rec["level_counts"], "work_items": rec["work_items"], "l2": rec["l2"],
+                       "parallelism": "replicas x%d" % world, "build_s": rec["build_s"],
+                       "step_ms_median": rec["step_ms_median"], "step_ms_stdev": rec["step_ms_stdev"]},
+            "gflops": rec["gflops"], "hbm_gbs_algorithmic": rec["hbm_gbs_algorithmic"],
+            "hbm_frac_of_nominal_8000": rec["hbm_frac_of_nominal_8000"], "roofline": rec["roofline"],
+            "e2e": rec["e2e"], "gpu_launches": rec["gpu_launches"], "clocks": rec["clocks"],
         }
-        gather = l2_gather_ceiling(sa, torch, w, ops, dev, stream) if args.scale == "full" else None
-        if gather is not None:
-            line["l2_gather_ceiling"] = gather
+        if "l2_gather_ceiling" in rec:
+            line["l2_gather_ceiling"] = rec["l2_gather_ceiling"]
+        kept = {args.workload: w}
+        records = [dict(rec, config=args.workload)]
+        if all_configs:
+            steps_pc = min(args.steps, 10)
+            for cfg, sname in PER_CONFIG:
+                if cfg not in kept:
+                    kept[cfg] = pending[cfg].result()
+                r = measure(sa, torch, dist, kept[cfg], sname, steps_pc, args.warmup, min(args.e2e_steps, 2), dev, rank, world,
+                            scale="full", workload_id=cfg)
+                records.append(dict(r, config=cfg))
+            pool.shutdown()
         if not args.no_cpu_baseline and world == 1:
-            cb = oracle_sample(w)
-            cb.pop("seconds")
-            line["cpu_baseline"] = cb
+            budget = 15.0 if not all_configs else 6.0
+            done = {}
+            for r in records:
+                cfg = r["config"]
+                if cfg not in done:
+                    cb = oracle_sample(kept[cfg], budget_s=budget)
+                    cb.pop("seconds")
+                    done[cfg] = cb
+                r["cpu_baseline"] = done[cfg]
+            line["cpu_baseline"] = done[args.workload]
+        if all_configs:
+            line["per_config"] = records
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()

@@ -11,7 +11,8 @@ import os
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libsparseauto.so")
+# SPARSEAUTO_LIB selects another build of the same library (the self-checking one, libsparseauto_checked.so)
+LIB_PATH = os.environ.get("SPARSEAUTO_LIB") or os.path.join(_HERE, "libsparseauto.so")
 
 if not os.path.exists(LIB_PATH):
     raise ImportError("libsparseauto.so is missing: run `python paper_2311_09549_b200/build.py` "

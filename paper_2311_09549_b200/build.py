@@ -7,30 +7,42 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsparseauto.so")
+LIB_CHECKED = os.path.join(HERE, "libsparseauto_checked.so")
 SOURCES = ["sa_api.cu", "sa_build.cu", "sa_ttm3.cu", "sa_ttm4.cu", "sa_sddmm_spmm.cu", "sa_spmm_gemm.cu", "sa_ttmc3.cu", "sa_gather_probe.cu", "sa_mttkrp.cu", "sa_dense_tc.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC,-fopenmp,-O3", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 
 
-def _stale():
-    if not os.path.exists(LIB):
+def _stale(lib=LIB):
+    if not os.path.exists(lib):
         return True
-    t = os.path.getmtime(LIB)
-    deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)] + [os.path.join(ROOT, "include", "sparseauto.h")]
+    t = os.path.getmtime(lib)
+    deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)] + [os.path.join(ROOT, "include", "sparseauto.h"), __file__]
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force=False, verbose=False):
-    """SA_NVCC_EXTRA (environment) adds flags, e.g. -DSA_DEBUG_BOUNDS for the self-checking kernels."""
-    extra = os.environ.get("SA_NVCC_EXTRA", "").split()
-    if not force and not extra and not _stale():
-        return LIB
+def build(force=False, verbose=False, flags=(), lib=LIB):
+    """Compile the sources into ``lib``.  ``flags`` (and SA_NVCC_EXTRA in the environment) add nvcc flags."""
+    extra = list(flags) + os.environ.get("SA_NVCC_EXTRA", "").split()
+    if not force and not os.environ.get("SA_NVCC_EXTRA") and not _stale(lib):
+        return lib
+    return _compile(extra, verbose, lib, os.path.splitext(os.path.basename(lib))[0])
+
+
+def build_checked(force=False):
+    """The self-checking build (-DSA_DEBUG_BOUNDS): every index taken from the tensor's arrays is checked on the
+    device before it becomes an address.  Loaded instead of the normal library when the environment variable
+    SPARSEAUTO_LIB names it."""
+    return build(force=force, flags=["-DSA_DEBUG_BOUNDS"], lib=LIB_CHECKED)
+
+
+def _compile(extra, verbose, LIB, tag):
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     objs = []
     procs = []
-    os.makedirs(os.path.join(HERE, "_build"), exist_ok=True)
+    os.makedirs(os.path.join(HERE, "_build", tag), exist_ok=True)
     for src in SOURCES:
-        obj = os.path.join(HERE, "_build", src.replace(".cu", ".o"))
+        obj = os.path.join(HERE, "_build", tag, src.replace(".cu", ".o"))
         cmd = [nvcc] + NVCC_FLAGS + extra + (["-Xptxas", "-v"] if verbose else []) + ["-c", os.path.join(CSRC, src), "-o", obj]
         procs.append((src, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
         objs.append(obj)
@@ -49,4 +61,8 @@ def build(force=False, verbose=False):
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    if "--checked" in sys.argv:
+        print(build_checked(force="--force" in sys.argv))
+    else:
+        out = [a.split("=", 1)[1] for a in sys.argv if a.startswith("--out=")]
+        print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, lib=os.path.abspath(out[0]) if out else LIB))

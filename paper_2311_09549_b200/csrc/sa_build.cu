@@ -292,8 +292,8 @@ void build_ttm3(sa_tensor *t, sa_worklist &wl)
 // subtrees holding about PIECE_NNZ nonzeros, one thread block each.  A piece is a run of *super-items* (at most
 // SA_F4_POOL subtrees: what the block's pool of 16 x 16 temporaries holds), a super-item a run of *items* that
 // the block's warps take one at a time:
-//   kind 0: consecutive subtrees with at most SA_F4_ROWS level-2 fibers in all (one batch of parked fiber rows),
-//           or one subtree with more fibers (evaluated in several batches);   f0/f1 = fibers, p0/p1 = nonzeros
+//   kind 0: at most 32 consecutive subtrees, about an eighth of the super-item's nonzeros (the kernel evaluates
+//           their level-2 fibers in batches of at most SA_F4_ROWS);   f0/f1 = fibers, p0/p1 = nonzeros
 //   kind 1: up to 8 consecutive *large* subtrees (more than SA_SUB_MAX_NNZ nonzeros), whose temporaries the
 //           order-3 kernel has written beforehand; f0 = index of the first one among the large subtrees.
 // Nothing is cut at a slice boundary: the block follows the slices through pos[1] while it consumes the
@@ -323,61 +323,56 @@ void build_ttm4(sa_tensor *t, sa_worklist &wl, sa_worklist &wl_items, sa_worklis
     auto nnz_at = [&](int64_t r) { return pos3[size_t(pos2[size_t(r)])]; };
     std::vector<sa_item> &items = wl_items.items;
     std::vector<int32_t> &supers = t->f4_supers, &pieces = t->f4_pieces;
-    // state of the open item / super-item / piece
-    int64_t it_r0 = 0, sup_item0 = 0, sup_r0 = 0, piece_sup0 = 0, piece_r0 = 0, piece_w = 0;
-    int it_kind = -1;
-    auto close_item = [&](int64_t r) {
-        if (it_kind >= 0 && r > it_r0) {
-            sa_item it = empty_item();
-            it.out_row = int32_t(it_r0); it.row_end = int32_t(r); it.pad = it_kind;
-            if (it_kind == 0) {
-                it.f0 = int32_t(pos2[size_t(it_r0)]); it.f1 = int32_t(pos2[size_t(r)]);
-                it.p0 = int32_t(nnz_at(it_r0)); it.p1 = int32_t(nnz_at(r));
-            } else {
-                it.f0 = large_ord[size_t(it_r0)]; it.f1 = it.f0 + int32_t(r - it_r0);
-            }
-            items.push_back(it);
+    auto push_item = [&](int64_t r0, int64_t r1, int kind) {
+        sa_item it = empty_item();
+        it.out_row = int32_t(r0); it.row_end = int32_t(r1); it.pad = kind;
+        if (kind == 0) {
+            it.f0 = int32_t(pos2[size_t(r0)]); it.f1 = int32_t(pos2[size_t(r1)]);
+            it.p0 = int32_t(nnz_at(r0)); it.p1 = int32_t(nnz_at(r1));
+        } else {
+            it.f0 = large_ord[size_t(r0)]; it.f1 = it.f0 + int32_t(r1 - r0);
         }
-        it_kind = -1;
-        it_r0 = r;
+        items.push_back(it);
     };
-    auto close_super = [&](int64_t r) {
-        close_item(r);
-        if (int64_t(items.size()) > sup_item0) {
-            supers.push_back(int32_t(sup_item0)); supers.push_back(int32_t(items.size()));
-            supers.push_back(int32_t(sup_r0)); supers.push_back(int32_t(r));
+    // One super-item = the subtrees [r0, r1), r1 - r0 <= SA_F4_POOL.  Its small subtrees are cut into at most eight
+    // nonzero-balanced runs (one per warp of the block); a run also ends at a large subtree and after 32 subtrees.
+    auto push_super = [&](int64_t r0, int64_t r1) {
+        int64_t small_nnz = 0;
+        for (int64_t r = r0; r < r1; ++r)
+            if (large_ord[size_t(r)] < 0) small_nnz += nnz_at(r + 1) - nnz_at(r);
+        const int64_t target = (small_nnz + 7) / 8;
+        const int32_t item0 = int32_t(items.size());
+        int64_t run0 = r0, run_nnz = 0;
+        int run_kind = -1;
+        for (int64_t r = r0; r < r1; ++r) {
+            const int kind = large_ord[size_t(r)] >= 0 ? 1 : 0;
+            const bool full = run_kind >= 0 && (kind != run_kind || (kind == 1 ? r - run0 >= 8 : (run_nnz >= target || r - run0 >= 32)));
+            if (full) { push_item(run0, r, run_kind); run_kind = -1; }
+            if (run_kind < 0) { run_kind = kind; run0 = r; run_nnz = 0; }
+            if (kind == 0) run_nnz += nnz_at(r + 1) - nnz_at(r);
         }
-        sup_item0 = int64_t(items.size());
-        sup_r0 = r;
+        if (run_kind >= 0) push_item(run0, r1, run_kind);
+        supers.push_back(item0); supers.push_back(int32_t(items.size()));
+        supers.push_back(int32_t(r0)); supers.push_back(int32_t(r1));
     };
     // slice that holds subtree r (r < F2)
     auto slice_of = [&](int64_t r) { return int64_t(std::upper_bound(pos1.begin(), pos1.end(), r) - pos1.begin()) - 1; };
-    auto close_piece = [&](int64_t r) {
-        close_super(r);
-        if (int64_t(supers.size() / 4) > piece_sup0) {
-            const int64_t sa = slice_of(piece_r0), sb = slice_of(r - 1);
-            pieces.push_back(int32_t(piece_sup0)); pieces.push_back(int32_t(supers.size() / 4));
-            pieces.push_back(int32_t(sa)); pieces.push_back(int32_t(sb));
-            pieces.push_back(-1); pieces.push_back(-1);       // destinations of the first / last slice: set below
-            pieces.push_back(int32_t(piece_r0)); pieces.push_back(int32_t(r));
-        }
-        piece_sup0 = int64_t(supers.size() / 4);
-        piece_r0 = r;
-        piece_w = 0;
+    auto push_piece = [&](int64_t r0, int64_t r1) {
+        const int32_t sup0 = int32_t(supers.size() / 4);
+        for (int64_t r = r0; r < r1; r += SA_F4_POOL) push_super(r, std::min<int64_t>(r1, r + SA_F4_POOL));
+        pieces.push_back(sup0); pieces.push_back(int32_t(supers.size() / 4));
+        pieces.push_back(int32_t(slice_of(r0))); pieces.push_back(int32_t(slice_of(r1 - 1)));
+        pieces.push_back(-1); pieces.push_back(-1);       // destinations of the first / last slice: set below
+        pieces.push_back(int32_t(r0)); pieces.push_back(int32_t(r1));
     };
-    for (int64_t r = 0; r < F2; ++r) {
-        const bool large = large_ord[size_t(r)] >= 0;
-        if (piece_w >= PIECE_NNZ) close_piece(r);
-        if (r - sup_r0 >= SA_F4_POOL) close_super(r);
-        if (it_kind >= 0) {
-            const bool full = large ? (it_kind != 1 || r - it_r0 >= 8)
-                                    : (it_kind != 0 || r - it_r0 >= 32 || pos2[size_t(r) + 1] - pos2[size_t(it_r0)] > SA_F4_ROWS);
-            if (full) close_item(r);
+    {
+        int64_t piece_r0 = 0, piece_w = 0;
+        for (int64_t r = 0; r < F2; ++r) {
+            if (piece_w >= PIECE_NNZ) { push_piece(piece_r0, r); piece_r0 = r; piece_w = 0; }
+            piece_w += large_ord[size_t(r)] >= 0 ? LARGE_WEIGHT : nnz_at(r + 1) - nnz_at(r);
         }
-        if (it_kind < 0) { it_kind = large ? 1 : 0; it_r0 = r; }
-        piece_w += large ? LARGE_WEIGHT : nnz_at(r + 1) - nnz_at(r);
+        if (F2 > piece_r0) push_piece(piece_r0, F2);
     }
-    close_piece(F2);
     wl_items.n_group_ctas = 0;
     // partial tiles: a slice that lies in more than one piece gets one slot per piece
     std::vector<int32_t> slice_slots(size_t(S), 0), slice_slot0(size_t(S), -1);

@@ -121,8 +121,18 @@ struct sa_tensor {
 // Limits of the fused order-4 kernel: level-2 fiber rows a warp parks per batch, temporaries in a thread block's
 // pool (= subtrees per super-item), nonzeros of a subtree the kernel evaluates itself (larger ones go through the
 // order-3 kernel first).
-constexpr int SA_F4_ROWS = 32;
-constexpr int SA_F4_POOL = 64;
+#ifndef SA_F4_ROWS_N
+#define SA_F4_ROWS_N 32
+#endif
+#ifndef SA_F4_POOL_N
+#define SA_F4_POOL_N 64
+#endif
+#ifndef SA_F4_CTAS_N
+#define SA_F4_CTAS_N 2
+#endif
+constexpr int SA_F4_ROWS = SA_F4_ROWS_N;
+constexpr int SA_F4_POOL = SA_F4_POOL_N;
+constexpr int SA_F4_CTAS = SA_F4_CTAS_N;      // thread blocks per SM the fused kernel's register budget is set for
 constexpr int SA_SUB_MAX_NNZ = 4096;
 
 // ---- host builder (sa_build.cu)

@@ -39,7 +39,7 @@ constexpr int R = 16;                  // L = M = N = 16
 constexpr int TILE4 = R * R * R;       // floats per output slice
 constexpr int T2F = R * R;             // floats per temporary
 constexpr int F4_WARPS = 8;
-constexpr int F4_RS = 40;              // floats per parked fiber row: t(f; 0..15) | D(k_f, 0..15) | pad; rows 8 banks apart
+constexpr int F4_RS = 32;              // floats per parked fiber row: t(f; 0..15) | D(k_f, 0..15), rotated by 8 (row & 3) floats
 constexpr int F4_TS = T2F + 8;         // floats per pooled temporary: consecutive temporaries 8 banks apart
 constexpr int F4_CS = 24;              // floats per staged row of C
 constexpr int F4_PARK = SA_F4_ROWS * F4_RS;
@@ -55,27 +55,36 @@ struct f4_limits {
 // neither the accumulator-fragment stores of stage B nor the operand-fragment loads of the consumer collide.
 __device__ __forceinline__ int f4_pos(int m, int n) { return m * R + (n ^ (((m >> 1) & 1) << 3)); }
 
-// Stage A on the fibers [fb0, fb0 + nf) (nf <= 32): rows 0 .. nf - 1 of pk get t(f; :).  s3 = pos3[fb0 + lane]
-// (INT_MAX past the batch), pe = pos3[fb0 + nf].
-__device__ __forceinline__ void f4_stage_a(float *pk, int nf, int s3, int pe, const int2 *__restrict__ nz,
+// Where float `pos` (0..15: t(f; pos), 16..31: D(k_f, pos - 16)) of parked row r lives: every row is rotated by a
+// quarter more than the one before, so that the operand-fragment loads of stage B (four consecutive rows x eight
+// consecutive floats) fall into 32 different banks without padding.
+__device__ __forceinline__ int f4_rowpos(int r, int pos) { return r * F4_RS + ((pos + 8 * (r & 3)) & 31); }
+
+// Stage A on a batch of nf <= SA_F4_ROWS fibers: row r of pk gets t(f_r; :).  s3 = pos3[first fiber + lane] (INT_MAX
+// past the batch), pe = pos3[one past the last fiber].  A lane group keeps ONE running sum over its whole share and
+// parks it at every end-of-fiber bit (no reset: a predicated store and a pointer bump per step); the rows are
+// turned into per-fiber sums afterwards by subtracting the previous row inside each group's share.
+__device__ __forceinline__ void f4_stage_a(float *pk, uint32_t pk_s, int nf, int s3, int pe, const int2 *__restrict__ nz,
                                            const float *__restrict__ E, uint32_t ld_e, int lane, const f4_limits &lim)
 {
     const int g = lane >> 2, l = lane & 3;
     const int pb0 = __shfl_sync(SA_FULL_MASK, s3, 0);
     // shares of the eight groups: whole fibers, cut where the nonzero count passes the next eighth of the batch
     int fa = 0, fb = nf;
+    uint32_t first = 1u;                                      // bit r: row r is the first of some group's share
 #pragma unroll
     for (int q = 1; q < 8; ++q) {
         const int target = pb0 + int(int64_t(pe - pb0) * q / 8);
         const int cnt = __popc(__ballot_sync(SA_FULL_MASK, s3 < target));
         if (g == q) fa = cnt;
         if (g + 1 == q) fb = cnt;
+        first |= 1u << (cnt & 31);
     }
     const int sa = __shfl_sync(SA_FULL_MASK, s3, fa & 31), sb = __shfl_sync(SA_FULL_MASK, s3, fb & 31);
     const int ga = fa < nf ? sa : pe, gb = fb < nf ? sb : pe;
     const int mylen = gb - ga;
     const int maxlen = __reduce_max_sync(SA_FULL_MASK, mylen);
-    int slot = fa;
+    int slot = fa;                                            // row the group parks next
     auto fetch1 = [&](int q, int &x, float &v) {
         x = 0;
         v = 0.f;
@@ -117,12 +126,33 @@ __device__ __forceinline__ void f4_stage_a(float *pk, int nf, int s3, int pe, co
                 acc.z = fmaf(vs[u], e[u].z, acc.z);
                 acc.w = fmaf(vs[u], e[u].w, acc.w);
             }
-            if (xs[u] < 0) {                                      // last nonzero of fiber fb0 + slot
-                if (SA_CHK(lim.status, slot >= 0 && slot < nf, 23, slot)) *reinterpret_cast<float4 *>(pk + slot * F4_RS + 4 * l) = acc;
-                acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (xs[u] < 0) {                                      // last nonzero of a fiber: park the running sum
+                if (!SA_CHK(lim.status, slot < nf, 23, slot)) slot = 0;
+                *reinterpret_cast<float4 *>(pk + f4_rowpos(slot, 4 * l)) = acc;
                 ++slot;
             }
         }
+    }
+    __syncwarp();
+    // running sums -> per-fiber sums: row r -= row r - 1 unless r opens a group's share (eight rows per pass, lane =
+    // (row, float4 of the row); everything is read before anything is written)
+    float4 cur[SA_F4_ROWS / 8], prev[SA_F4_ROWS / 8];
+#pragma unroll
+    for (int i = 0; i < SA_F4_ROWS / 8; ++i) {
+        const int row = g + 8 * i;
+        cur[i] = prev[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (row < nf) {
+            cur[i] = *reinterpret_cast<const float4 *>(pk + f4_rowpos(row, 4 * l));
+            if (!((first >> row) & 1u)) prev[i] = *reinterpret_cast<const float4 *>(pk + f4_rowpos(row - 1, 4 * l));
+        }
+    }
+    __syncwarp();
+#pragma unroll
+    for (int i = 0; i < SA_F4_ROWS / 8; ++i) {
+        const int row = g + 8 * i;
+        if (row < nf)
+            *reinterpret_cast<float4 *>(pk + f4_rowpos(row, 4 * l)) =
+                make_float4(cur[i].x - prev[i].x, cur[i].y - prev[i].y, cur[i].z - prev[i].z, cur[i].w - prev[i].w);
     }
 }
 
@@ -136,7 +166,6 @@ __device__ __forceinline__ void f4_small_item(const sa_item &it, float *pk, floa
     const int g = lane >> 2, t = lane & 3;
     const int nsub = it.row_end - it.out_row;
     const int my_end = lane < nsub ? __ldg(pos2 + it.out_row + lane + 1) : 0x7fffffff;   // fiber at which subtree `lane` ends
-    int cur = 0, cur_end = __shfl_sync(SA_FULL_MASK, my_end, 0);
     float tacc[2][4];
 #pragma unroll
     for (int nt = 0; nt < 2; ++nt)
@@ -145,22 +174,34 @@ __device__ __forceinline__ void f4_small_item(const sa_item &it, float *pk, floa
     const int nft = it.f1 - it.f0;
     const int nbat = (nft + SA_F4_ROWS - 1) / SA_F4_ROWS, bsz = (nft + nbat - 1) / nbat;
     const uint32_t pk_s = smem_u32(pk);
-    for (int fb0 = it.f0; fb0 < it.f1; fb0 += bsz) {
+    // per-batch arrays: start of every fiber, its row of D, end of the last fiber -- read one batch ahead
+    struct meta { int s3, kk, pe; };
+    auto load_meta = [&](int fb0) {
+        meta m;
         const int nf = min(bsz, it.f1 - fb0);
         const bool mine = lane < nf && SA_CHK(lim.status, fb0 + lane >= 0 && fb0 + lane < lim.n_fibers, 24, fb0 + lane);
-        const int s3 = mine ? __ldg(pos3 + fb0 + lane) : 0x7fffffff;
-        int kk = mine ? __ldg(crd_k + fb0 + lane) : 0;
+        m.s3 = mine ? __ldg(pos3 + fb0 + lane) : 0x7fffffff;
+        m.kk = mine ? __ldg(crd_k + fb0 + lane) : 0;
+        m.pe = __ldg(pos3 + fb0 + nf);
+        return m;
+    };
+    meta cm = load_meta(it.f0);
+    int cur = 0, cur_end = __shfl_sync(SA_FULL_MASK, my_end, 0);
+    for (int fb0 = it.f0; fb0 < it.f1; fb0 += bsz) {
+        const int nf = min(bsz, it.f1 - fb0);
+        const meta m = cm;
+        if (fb0 + bsz < it.f1) cm = load_meta(fb0 + bsz);
+        int kk = m.kk;
         if (!SA_CHK(lim.status, uint32_t(kk) < lim.d_rows, 25, kk)) kk = 0;
-        const int pe = __ldg(pos3 + fb0 + nf);
         // rows of D the batch's fibers need in stage B: fetched while stage A runs
 #pragma unroll
         for (int i = 0; i < SA_F4_ROWS / 8; ++i) {
             const int row = g + 8 * i;
             const int k = __shfl_sync(SA_FULL_MASK, kk, row);
-            if (row < nf) cp_async16_raw(pk_s + uint32_t(row * F4_RS + R + 4 * t) * 4u, D + (uint32_t(k) * ld_d + 4u * t));
+            if (row < nf) cp_async16_raw(pk_s + uint32_t(f4_rowpos(row, R + 4 * t)) * 4u, D + (uint32_t(k) * ld_d + 4u * t));
         }
         cp_async_commit();
-        f4_stage_a(pk, nf, s3, pe, nz, E, ld_e, lane, lim);
+        f4_stage_a(pk, pk_s, nf, m.s3, m.pe, nz, E, ld_e, lane, lim);
         cp_async_wait<0>();
         __syncwarp();
         // ---- stage B: the batch's fibers, subtree by subtree, eight per product
@@ -170,19 +211,20 @@ __device__ __forceinline__ void f4_small_item(const sa_item &it, float *pk, floa
             const int e = max(f, min(cur_end, fb1));
             for (int g8 = f; g8 < e; g8 += 8) {
                 const bool va = g8 + t < e, vb = g8 + t + 4 < e;
-                const float *ra = pk + min(g8 - fb0 + t, SA_F4_ROWS - 1) * F4_RS;
-                const float *rb = pk + min(g8 - fb0 + t + 4, SA_F4_ROWS - 1) * F4_RS;
+                const int qa = min(g8 - fb0 + t, SA_F4_ROWS - 1), qb = min(g8 - fb0 + t + 4, SA_F4_ROWS - 1);
+                const float *ra = pk + qa * F4_RS, *rb = pk + qb * F4_RS;
+                const int oa = 8 * (qa & 3), ob = 8 * (qb & 3);          // rotation of the two rows
                 // A operand: D(k_f, m), m = g and g + 8, fibers t and t + 4;  B operand: t(f; n), n = 8 nt + g
                 uint32_t ah[4], al[4];
-                split_tf32(va ? ra[R + g] : 0.f, ah[0], al[0]);
-                split_tf32(va ? ra[R + g + 8] : 0.f, ah[1], al[1]);
-                split_tf32(vb ? rb[R + g] : 0.f, ah[2], al[2]);
-                split_tf32(vb ? rb[R + g + 8] : 0.f, ah[3], al[3]);
+                split_tf32(va ? ra[(R + g + oa) & 31] : 0.f, ah[0], al[0]);
+                split_tf32(va ? ra[(R + g + 8 + oa) & 31] : 0.f, ah[1], al[1]);
+                split_tf32(vb ? rb[(R + g + ob) & 31] : 0.f, ah[2], al[2]);
+                split_tf32(vb ? rb[(R + g + 8 + ob) & 31] : 0.f, ah[3], al[3]);
 #pragma unroll
                 for (int nt = 0; nt < 2; ++nt) {
                     uint32_t bh[2], bl[2];
-                    split_tf32(va ? ra[8 * nt + g] : 0.f, bh[0], bl[0]);
-                    split_tf32(vb ? rb[8 * nt + g] : 0.f, bh[1], bl[1]);
+                    split_tf32(va ? ra[(8 * nt + g + oa) & 31] : 0.f, bh[0], bl[0]);
+                    split_tf32(vb ? rb[(8 * nt + g + ob) & 31] : 0.f, bh[1], bl[1]);
                     mma_m16n8k8_tf32(tacc[nt], al, bh);
                     mma_m16n8k8_tf32(tacc[nt], ah, bl);
                     mma_m16n8k8_tf32(tacc[nt], ah, bh);
@@ -271,7 +313,7 @@ __device__ __forceinline__ void f4_store(const float (&acc)[4][4], float *dst, b
 
 // CONTIG: D and E are stored without padding (leading dimension 16), so a row offset is a shift.
 template <bool CONTIG>
-__global__ void __launch_bounds__(32 * F4_WARPS, 2)
+__global__ void __launch_bounds__(32 * F4_WARPS, SA_F4_CTAS)
 ttm4_fused_kernel(const int4 *__restrict__ pieces, const int4 *__restrict__ supers, const sa_item *__restrict__ items,
                   const int32_t *__restrict__ pos1, const int32_t *__restrict__ crd0, const int32_t *__restrict__ crd_j,
                   const int32_t *__restrict__ pos2, const int32_t *__restrict__ pos3, const int32_t *__restrict__ crd_k,

@@ -199,17 +199,18 @@ def check_order4_fused_lists(t, dims0):
         if kind == 0:
             assert not is_large[r0:r1].any()
             assert (f0, f1) == (pos2[r0], pos2[r1]) and (p0, p1) == (pos3[f0], pos3[f1])
-            assert f1 - f0 <= 32 or r1 - r0 == 1, "more than one batch of fibers only for a single subtree"
         else:
             assert kind == 1 and is_large[r0:r1].all() and r1 - r0 <= 8
             assert f0 == large_ord[r0] and f1 - f0 == r1 - r0
     assert (seen == 1).all()
-    # super-items: consecutive items, consecutive subtrees, at most 64 subtrees
+    # super-items: consecutive items, consecutive subtrees, at most 64 subtrees, at most 8 runs of small subtrees
     nxt_item, nxt_r = 0, 0
     for i0, i1, r0, r1 in supers:
         assert i0 == nxt_item and i1 > i0 and r0 == nxt_r and 0 < r1 - r0 <= 64
         assert items[i0][0] == r0 and items[i1 - 1][1] == r1
         assert all(items[k][1] == items[k + 1][0] for k in range(i0, i1 - 1))
+        n_large_runs = sum(1 for k in range(i0, i1) if items[k][7] == 1)
+        assert sum(1 for k in range(i0, i1) if items[k][7] == 0) <= 8 + n_large_runs
         nxt_item, nxt_r = i1, r1
     assert nxt_item == len(items) and nxt_r == F2
     # pieces: consecutive super-items; slices and destinations
@@ -260,7 +261,7 @@ def test_order4_fused_worklists_cover_every_subtree_once():
 
 def test_order4_large_and_many_fiber_subtrees():
     """A subtree above 4096 nonzeros is left to the order-3 lists (item of kind 1); one with 130 fibers but few
-    nonzeros is a single item of kind 0 that the kernel evaluates in batches."""
+    nonzeros is part of an item of kind 0 that the kernel evaluates in batches."""
     k, o = np.divmod(np.arange(4800), 40)
     big = np.stack([np.zeros(4800), np.zeros(4800), k, o], axis=1).astype(np.int32)
     many = np.stack([np.ones(130), np.ones(130), np.arange(130), np.zeros(130)], axis=1).astype(np.int32)

@@ -53,12 +53,29 @@ def _compare(out, w, sel, what):
     return assert_close(got, A_ref, S_ref, TOL_FP32, what)
 
 
+def _compare_head_slice(out, w, what, parts=16):
+    """The slice with the most nonzeros, which the sample above leaves out because the oracle evaluates a slice on
+    one thread: its nonzeros are dealt to ``parts`` pseudo-slices (the contraction is linear in B, and so is the sum
+    of absolute terms), the oracle evaluates those in parallel, and the sums are compared with the GPU's slice."""
+    counts = np.bincount(w.coords[:, 0], minlength=w.dims[0])
+    top = int(np.argmax(counts))
+    rows = np.nonzero(w.coords[:, 0] == top)[0]
+    coords = np.ascontiguousarray(w.coords[rows])
+    coords[:, 0] = np.arange(rows.shape[0]) % parts
+    sub = configs.Workload(w.name + "-head", w.expr, w.fmt, (parts,) + tuple(w.dims[1:]), coords,
+                           np.ascontiguousarray(w.vals[rows]), w.dense, (parts,) + tuple(w.out_shape[1:]), w.seed)
+    A_parts, S_parts = oracle.evaluate(sub)
+    got = out[top].cpu().numpy().astype(np.float64)
+    return assert_close(got, A_parts.sum(axis=0), S_parts.sum(axis=0), TOL_FP32, what + " head slice %d (%d nonzeros)" % (top, rows.shape[0]))
+
+
 def test_cfg2_full_sampled(sa):
     import torch
     w = configs.make(2, "full")
     out, t = _run_full(sa, w)
     sel = _sample(w, 3_000_000, 300)                  # includes a slice split over ~50 thread blocks
     _compare(out, w, sel, w.name)
+    _compare_head_slice(out, w, w.name)               # 19.6 % of B in one slice
     # whole-output properties that hold at any size: finite, and slices scale with B
     assert bool(torch.isfinite(out).all())
     del out, t
@@ -101,6 +118,7 @@ def test_cfg5_full_sampled(sa):
     out, t = _run_full(sa, w)
     sel = _sample(w, 600_000, 150)                    # includes a slice split over several thread blocks
     _compare(out, w, sel, w.name)
+    _compare_head_slice(out, w, w.name)               # 19.9 % of B in one slice
     del out, t
     torch.cuda.empty_cache()
 

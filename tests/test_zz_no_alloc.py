@@ -1,4 +1,4 @@
-"""The allocation-free entry point (sa_run_ttm3_static_scratch) against the regular sa_run.
+"""The allocation-free entry point (sa_run_ttm3_static_scratch) against the oracle and the regular sa_run.
 
 It exists for callers that cannot get device memory at call time (fixed memory plans, plug-ins
 whose host owns allocation, loops that must not touch cudaMalloc) and therefore cannot pass a
@@ -24,10 +24,16 @@ def _run_both(sa, torch, w):
     torch.cuda.synchronize()
     stream = torch.cuda.current_stream().cuda_stream
 
-    def static_call(_keep=ops_t):     # the operand tensors must outlive the raw pointers in `ops`
+    def static_call(check_memory=False, _keep=ops_t):     # the operand tensors must outlive the raw pointers in `ops`
         out = torch.full(w.out_shape, float("nan"), dtype=torch.float32, device="cuda")
+        torch.cuda.synchronize()
+        before = (torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated(), torch.cuda.memory_reserved())
         sa.sa_run_ttm3_static_scratch(t.handle, ops, out.data_ptr(), stream)
         torch.cuda.synchronize()
+        after = (torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated(), torch.cuda.memory_reserved())
+        if check_memory:
+            # neither the driver's free memory nor torch's allocator moved: the call obtained no device memory
+            assert after == before, (before, after)
         return out.cpu().numpy().astype(np.float64)
 
     return t, ref.cpu().numpy().astype(np.float64), static_call
@@ -40,16 +46,18 @@ def test_static_scratch_matches_sa_run_on_two_calls_in_a_row():
     w = configs.make(2, "mini")                       # has slices split over several thread blocks
     t, ref, static_call = _run_both(sa, torch, w)
     assert sa.sa_tensor_worklist(t.handle)[0][3] > 0, "the case must really use partial-tile slots"
-    _, S = oracle.evaluate(w)
-    first = static_call()
-    assert_close(first, ref, S, TOL_FP32, "static scratch, first call")
+    A_ref, S = oracle.evaluate(w)
+    first = static_call()                             # the first call on a device also looks up the scratch's address
+    assert_close(first, A_ref, S, TOL_FP32, "static scratch against the oracle, first call")
+    assert_close(first, ref, S, TOL_FP32, "static scratch against sa_run, first call")
     # another tensor overwrites the shared scratch in between
     w5 = configs.make_ttm3_zipf("other", 99, 400, 300, 300, 120_000, 1.2, 8.0, 32, 32)
     t5, ref5, static_call5 = _run_both(sa, torch, w5)
-    _, S5 = oracle.evaluate(w5)
-    assert_close(static_call5(), ref5, S5, TOL_FP32, "static scratch, other tensor")
-    second = static_call()
-    assert_close(second, ref, S, TOL_FP32, "static scratch, second call")
+    A5, S5 = oracle.evaluate(w5)
+    assert_close(static_call5(check_memory=True), A5, S5, TOL_FP32, "static scratch against the oracle, other tensor")
+    second = static_call(check_memory=True)
+    assert_close(second, A_ref, S, TOL_FP32, "static scratch against the oracle, second call")
+    assert_close(second, ref, S, TOL_FP32, "static scratch against sa_run, second call")
     assert np.array_equal(first, second)
 
 
