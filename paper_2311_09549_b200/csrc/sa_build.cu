@@ -334,13 +334,13 @@ void build_ttm4(sa_tensor *t, sa_worklist &wl, sa_worklist &wl_items, sa_worklis
         }
         items.push_back(it);
     };
-    // One super-item = the subtrees [r0, r1), r1 - r0 <= SA_F4_POOL.  Its small subtrees are cut into at most eight
+    // One super-item = the subtrees [r0, r1), r1 - r0 <= SA_F4_POOL.  Its small subtrees are cut into at most SA_F4_WARPS
     // nonzero-balanced runs (one per warp of the block); a run also ends at a large subtree and after 32 subtrees.
     auto push_super = [&](int64_t r0, int64_t r1) {
         int64_t small_nnz = 0;
         for (int64_t r = r0; r < r1; ++r)
             if (large_ord[size_t(r)] < 0) small_nnz += nnz_at(r + 1) - nnz_at(r);
-        const int64_t target = (small_nnz + 7) / 8;
+        const int64_t target = (small_nnz + SA_F4_WARPS - 1) / SA_F4_WARPS;
         const int32_t item0 = int32_t(items.size());
         int64_t run0 = r0, run_nnz = 0;
         int run_kind = -1;

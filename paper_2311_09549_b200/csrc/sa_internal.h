@@ -127,11 +127,15 @@ struct sa_tensor {
 #ifndef SA_F4_POOL_N
 #define SA_F4_POOL_N 64
 #endif
+#ifndef SA_F4_WARPS_N
+#define SA_F4_WARPS_N 8
+#endif
 #ifndef SA_F4_CTAS_N
 #define SA_F4_CTAS_N 2
 #endif
 constexpr int SA_F4_ROWS = SA_F4_ROWS_N;
 constexpr int SA_F4_POOL = SA_F4_POOL_N;
+constexpr int SA_F4_WARPS = SA_F4_WARPS_N;    // warps per thread block of the fused kernel
 constexpr int SA_F4_CTAS = SA_F4_CTAS_N;      // thread blocks per SM the fused kernel's register budget is set for
 constexpr int SA_SUB_MAX_NNZ = 4096;
 

@@ -38,7 +38,8 @@ namespace {
 constexpr int R = 16;                  // L = M = N = 16
 constexpr int TILE4 = R * R * R;       // floats per output slice
 constexpr int T2F = R * R;             // floats per temporary
-constexpr int F4_WARPS = 8;
+constexpr int F4_WARPS = SA_F4_WARPS;   // warps that produce; the first F4_CWARPS of them also consume
+constexpr int F4_CWARPS = 8;           // 256 columns (m,n) / 32 per warp
 constexpr int F4_RS = 32;              // floats per parked fiber row: t(f; 0..15) | D(k_f, 0..15), rotated by 8 (row & 3) floats
 constexpr int F4_TS = T2F + 8;         // floats per pooled temporary: consecutive temporaries 8 banks apart
 constexpr int F4_CS = 24;              // floats per staged row of C
@@ -379,13 +380,13 @@ ttm4_fused_kernel(const int4 *__restrict__ pieces, const int4 *__restrict__ supe
                 SA_CHK(lim.status, false, 29, r);
                 break;
             }
-            f4_consume(acc, pool + (r - S.z) * F4_TS, cs + (r - S.z) * F4_CS, n, warp, lane);
+            if (warp < F4_CWARPS) f4_consume(acc, pool + (r - S.z) * F4_TS, cs + (r - S.z) * F4_CS, n, warp, lane);
             r += n;
             if (r == bound) {
                 // slice s is complete (as far as this piece holds it)
                 const bool part = s == pa.z && pb.x >= 0;
                 const uint32_t row = uint32_t(__ldg(crd0 + s));
-                if (part ? SA_CHK(lim.status, pb.x < lim.n_slots, 30, pb.x) : SA_CHK(lim.status, row < lim.n_slices, 31, row))
+                if (warp < F4_CWARPS && (part ? SA_CHK(lim.status, pb.x < lim.n_slots, 30, pb.x) : SA_CHK(lim.status, row < lim.n_slices, 31, row)))
                     f4_store(acc, part ? partial + int64_t(pb.x) * TILE4 : out + int64_t(row) * TILE4, !part, warp, lane);
 #pragma unroll
                 for (int nt = 0; nt < 4; ++nt)
@@ -398,7 +399,7 @@ ttm4_fused_kernel(const int4 *__restrict__ pieces, const int4 *__restrict__ supe
         __syncthreads();
     }
     // the piece ends inside slice s: what it holds of that slice is a partial tile
-    if (s <= pa.w && SA_CHK(lim.status, pb.y >= 0 && pb.y < lim.n_slots, 32, pb.y))
+    if (warp < F4_CWARPS && s <= pa.w && SA_CHK(lim.status, pb.y >= 0 && pb.y < lim.n_slots, 32, pb.y))
         f4_store(acc, partial + int64_t(pb.y) * TILE4, false, warp, lane);
 }
 
