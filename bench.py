@@ -257,38 +257,60 @@ def reduce_max_over_ranks(values, device, world):
     return [float(x) for x in t.cpu()]
 
 
-def l2_gather_ceiling(sa, torch, w, ops, dev, stream):
-    """For the TTM chains: time a bare gather of one factor row per nonzero (the rows the fiber stage reads, from
-    the same table, uniformly random row indices) with the library's probe kernel.  Returns a dict or None."""
+def l2_gather_ceiling(sa, torch, w, tensor, ops, dev, stream):
+    """For the TTM chains: time bare gathers of one factor row per nonzero (the rows the fiber stage reads, from
+    the same L2-resident table) with the probe kernels of paper_2311_09549_b200/probe, over lane-group widths,
+    numbers of rows in flight and blocks per SM, for uniformly random row indices and for the tensor's own index
+    stream.  Returns the sweep and its best entry, or None."""
+    import ctypes
     which = {"spttm_ttm3": 1, "spttm_ttm4": 2, "ttmc3": 2, "mttkrp_gemm": 1}.get(w.expr)
-    if which is None:
+    lib_path = os.path.join(ROOT, "paper_2311_09549_b200", "probe", "libsaprobe.so")
+    if which is None or not os.path.exists(lib_path):
         return None
     table = ops[which]
     rows, cols = int(table.shape[0]), int(table.shape[1])
     if cols not in (16, 32):
         return None
+    lib = ctypes.CDLL(lib_path)
+    vp, i64, ci = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int
+    lib.sa_probe_row_gather.argtypes = [vp, i64, i64, ci, vp, i64, vp, ci, ci, ci, vp]
+    lib.sa_probe_row_gather.restype = ci
     n = int(w.nnz)
     g = torch.Generator(device=dev)
     g.manual_seed(12345)
-    idx = torch.randint(0, rows, (n,), dtype=torch.int32, device=dev, generator=g)
+    streams = {"uniform random rows": torch.randint(0, rows, (n,), dtype=torch.int32, device=dev, generator=g)}
+    last = tensor.order - 1
+    _, crd, _ = sa.sa_tensor_export(tensor.handle, last, n_crd=n)
+    streams["the tensor's last-mode indices in storage order"] = torch.from_numpy(crd).to(dev)
     sink = torch.zeros(1, dtype=torch.float32, device=dev)
-    run = lambda: sa.sa_probe_row_gather(table.data_ptr(), rows, table.stride(0), cols, idx.data_ptr(), n, sink.data_ptr(),
-                                         stream.cuda_stream)
-    for _ in range(3):
-        run()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    torch.cuda.synchronize(dev)
-    e0.record(stream)
-    reps = 10
-    for _ in range(reps):
-        run()
-    e1.record(stream)
-    torch.cuda.synchronize(dev)
-    ms = e0.elapsed_time(e1) / reps
     nbytes = n * cols * 4
+    sweep = []
+    for name, idx in streams.items():
+        for lanes in (4, 8):
+            for inflight in (4, 8, 16):
+                for bps in (4, 8, 16):
+                    def run():
+                        rc = lib.sa_probe_row_gather(table.data_ptr(), rows, table.stride(0), cols, idx.data_ptr(), n,
+                                                     sink.data_ptr(), lanes, inflight, bps, stream.cuda_stream)
+                        if rc != 0:
+                            raise RuntimeError("probe launch failed (%d)" % rc)
+                    for _ in range(2):
+                        run()
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    torch.cuda.synchronize(dev)
+                    e0.record(stream)
+                    reps = 5
+                    for _ in range(reps):
+                        run()
+                    e1.record(stream)
+                    torch.cuda.synchronize(dev)
+                    ms = e0.elapsed_time(e1) / reps
+                    sweep.append({"indices": name, "lanes_per_row": lanes, "rows_in_flight": inflight, "blocks_per_sm": bps,
+                                  "ms": round(ms, 4), "gbs": round(nbytes / (ms * 1e-3) / 1e9, 1)})
+    best = min(sweep, key=lambda r: r["ms"])
     return {"what": "bare gather of one %d-byte factor row per nonzero from the L2-resident %d x %d table "
-                    "(uniform random rows; plus 4 index bytes per row from HBM)" % (cols * 4, rows, cols),
-            "ms": ms, "gbs": nbytes / (ms * 1e-3) / 1e9}
+                    "(plus 4 index bytes per row from HBM); best of %d shapes" % (cols * 4, rows, cols, len(sweep)),
+            "ms": best["ms"], "gbs": best["gbs"], "best": best, "sweep": sweep}
 
 
 def aggregate_throughput(nnz_per_rank, world, ms_per_step):
@@ -439,7 +461,7 @@ def measure(sa, torch, dist, w, sched_name, steps, warmup, e2e_steps, dev, rank,
             "gpu_launches": launches_per_step * steps, "clocks": clocks,
         }
         if gather_probe and scale == "full":
-            gather = l2_gather_ceiling(sa, torch, w, ops, dev, stream)
+            gather = l2_gather_ceiling(sa, torch, w, tensor, ops, dev, stream)
             if gather is not None:
                 rec["l2_gather_ceiling"] = gather
     tensor.close()

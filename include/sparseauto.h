@@ -6,8 +6,8 @@
  * storage as in Section 2.1 and the pos/crd/vals arrays of Fig. 1b) under the branched loop
  * nests that kernel fission and fusion produce (Section 4.2; chosen schedules in the Table
  * of kernels, Section 6).  A fixed host table maps (expression, schedule) to ahead-of-time
- * compiled CUDA kernels, the mapping the paper itself proposes in Section 6 ("maintaining a
- * mapping from schedules chosen at compile-time to the corresponding compiled functions").
+ * compiled CUDA kernels; it stands in for the run-time lookup from chosen schedules to compiled
+ * functions that the paper outlines in its discussion of run-time overheads (Section 6).
  *
  * Conventions
  *   - Pointers marked HOST are ordinary host memory, DEVICE are device memory of the device the
@@ -54,8 +54,9 @@ typedef enum {
     /* kernel 6 <SpTTM,TTM>:  A(i,l,m) = sum_{j,k} B(i,j,k) C(j,l) D(k,m); ops = {C, D}          */
     SA_EXPR_SPTTM_TTM3 = 1,
     /* order-4 analogue:      A(i,l,m,n) = sum_{j,k,o} B(i,j,k,o) C(j,l) D(k,m) E(o,n);
-     * ops = {C, D, E}; the two-level nesting of kernel 5's second schedule, evaluated in two
-     * passes with the 16 x 16 temporaries T2(m,n) of the (i,j) subtrees in the workspace       */
+     * ops = {C, D, E}; the two-level nesting of kernel 5's second schedule in one fused kernel:
+     * the 16 x 16 temporaries T2(m,n) of the (i,j) subtrees stay in shared memory (only subtrees
+     * above 4096 nonzeros pass theirs through the workspace)                                    */
     SA_EXPR_SPTTM_TTM4 = 2,
     /* kernel 1 <SDDMM,SpMM>: A(i,l) = sum_j B(i,j) (sum_k C(i,k) D(j,k)) E(j,l); ops = {C,D,E}  */
     SA_EXPR_SDDMM_SPMM = 3,
@@ -136,8 +137,9 @@ sa_status sa_tensor_create(int order, const int64_t *dims, int64_t nnz, const in
                            const float *vals, sa_format fmt, int device,
                            const sa_allocator *dev_alloc, sa_tensor **out);
 
-/* Sizes.  level_counts HOST [order]: number of stored nodes per level (CSR level 0: rows;
- * last level: nnz).  n_chunks: number of work items in the tensor's main work list.  Any
+/* Sizes of the level structure of Section 2.1.  level_counts HOST [order]: number of stored nodes per level
+ * (CSR level 0: rows; last level: nnz; level 1 of a CSF tensor is the paper's nnz(B_ij), the quantity its cost
+ * expressions in Section 3 use).  n_chunks: number of work items in the tensor's main work list.  Any
  * output pointer may be NULL. */
 sa_status sa_tensor_info(const sa_tensor *t, int64_t *nnz, int64_t *level_counts, int64_t *n_chunks);
 
@@ -152,25 +154,31 @@ sa_status sa_tensor_info(const sa_tensor *t, int64_t *nnz, int64_t *level_counts
 sa_status sa_tensor_export(const sa_tensor *t, int level, int64_t *pos, int32_t *crd, float *vals);
 
 /*
- * Copy a load-balancing work list to HOST arrays (which: 0 = main list, 1 = second list: a CSR
- * tensor's list for SA_EXPR_SPMM_GEMM, an order-3 tensor's list of fiber rows for SA_EXPR_SPTTM_SPTTM
- * (rows = level-1 fibers), an order-4 tensor's list for the second pass of SA_EXPR_SPTTM_TTM4;
- * 2 = order-4 tensors: ranges of whole (i,j) subtrees for the first pass, rows [out_row,row_end) =
- * level-1 fibers, [f0,f1) their level-2 fibers (at most 64), [p0,p1) their nonzeros; a subtree with
- * more than 64 level-2 fibers or 4096 nonzeros is not in this list: the first pass takes it from the
- * main list, which for an order-4 tensor holds only those).  These are the slice / fiber / nonzero partition arrays:
+ * Copy a load-balancing work list to HOST arrays: the slice / fiber / nonzero partition arrays the kernels
+ * walk (housekeeping for tests and tools; the lists realise the parallel outer loops of the schedules in the
+ * Table of kernels, Section 6).  which:
+ *   0  main list (order-3 CSF: units of kernel 6, grouped into tasks, see sa_tensor_tasks; CSR: rows for
+ *      SA_EXPR_SDDMM_SPMM; order-4 CSF: the same kind of list over the (i,j) subtrees above 4096 nonzeros,
+ *      out_row = index among those subtrees, [f0,f1) level-2 nodes)
+ *   1  second list (CSR: rows for SA_EXPR_SPMM_GEMM; order-3 CSF: fiber rows for SA_EXPR_SPTTM_SPTTM, rows =
+ *      level-1 fibers; order-4 CSF: no items, only the fix-up entries and partial-tile slots of the fused kernel)
+ *   2  order-4 CSF: the items of the fused kernel, runs of (i,j) subtrees: out_row / row_end = first subtree /
+ *      one past the last (at most 32), last field = kind.  Kind 0: the kernel evaluates them, [f0,f1) their
+ *      level-2 fibers, [p0,p1) their nonzeros.  Kind 1: subtrees above 4096 nonzeros (at most 8), whose
+ *      temporaries the main list's kernel writes first; f0 = index of the first among those subtrees.
+ *   3  order-4 CSF: `items` receives the pieces (one thread block each), 8 int32 per piece: first super-item,
+ *      one past the last, first slice, last slice (positions in the level-0 crd array), partial-tile slot of
+ *      the first slice or -1, of the last slice or -1, first subtree, one past the last; `fix` receives the
+ *      super-items, 4 int32 each: first item, one past the last, first subtree, one past the last (at most 64
+ *      subtrees).  counts = {pieces, subtrees above 4096 nonzeros, super-items, 0}.
+ * For which = 0..2:
  *   counts [4]: number of items, number of leading groups that one thread block reduces into a
  *               single tile (8 items each; order-3 tensors: 4 tasks each, see sa_tensor_tasks),
  *               number of fix-up entries, number of partial-tile slots
- *   items  [n_items * 8] int32 per item: out_row, row_end, f0, f1, p0, p1, dest, half --
+ *   items  [n_items * 8] int32 per item: out_row, row_end, f0, f1, p0, p1, dest, last --
  *               fibers [f0,f1) (CSF) clipped to nonzeros [p0,p1) of slice out_row, or rows
  *               [out_row,row_end) / nonzeros [p0,p1) of a long row (CSR); dest = partial slot or -1;
- *               the last field is the position of the item's slice in the level-0 crd array.  The
- *               main list of a CSF tensor is grouped into tasks, see sa_tensor_tasks.  For an
- *               order-4 tensor the "slices" of the main list are the (i,j) subtrees: out_row is the
- *               index of the level-1 fiber, [f0,f1) are level-2 nodes; its second list has one item
- *               per (piece of a slice, quarter of the 256 columns (m,n)): level-1 fibers [f0,f1) of
- *               slice out_row, last field = quarter 0..3
+ *               the last field is the position of the item's slice in the level-0 crd array (list 0)
  *   fix    [n_fix * 4] int32 per entry: out_row, slot0, count, 0 -- out[out_row] = sum of `count`
  *               partial tiles from slot0 (count 0: the slice / row is empty and is zero-filled)
  * NULL outputs are skipped.
@@ -179,7 +187,7 @@ sa_status sa_tensor_worklist(const sa_tensor *t, int which, int64_t *counts, int
 
 /*
  * CSF tensors: how the items of the main work list are handed to warps (the warp-level
- * partition arrays of the fiber stage).
+ * partition arrays of the fiber stage; housekeeping, no passage of the paper).
  *   n_tasks     number of tasks; warp w of the launch evaluates task w
  *   task_start  HOST [n_tasks + 1]: task w holds the items [task_start[w], task_start[w + 1]).  The first
  *               4 * counts[1] tasks (counts of sa_tensor_worklist) hold one item or none: four
@@ -195,7 +203,9 @@ sa_status sa_tensor_worklist(const sa_tensor *t, int which, int64_t *counts, int
 sa_status sa_tensor_tasks(const sa_tensor *t, int64_t *n_tasks, int32_t *task_start, int32_t *stream_f0);
 
 /* Bytes of DEVICE workspace sa_run needs for this tensor / expression / schedule / operand
- * shapes (may be 0).  Only the shapes in ops are read. */
+ * shapes (may be 0): the schedule's auxiliary memory in the sense of Section 5 (the dense temporaries
+ * of the chosen nest that do not fit on chip, plus the partial tiles of split slices / rows).  Only the
+ * shapes in ops are read. */
 sa_status sa_workspace_size(const sa_tensor *t, sa_expr expr, sa_schedule sched, const sa_dense *ops,
                             int n_ops, size_t *bytes);
 
@@ -252,20 +262,6 @@ sa_status sa_run(const sa_tensor *B, sa_expr expr, sa_schedule sched, const sa_d
  */
 sa_status sa_run_ttm3_static_scratch(const sa_tensor *B, const sa_dense *ops, int n_ops, float *out,
                                      void *cuda_stream);
-
-/*
- * (Measurement aid; no counterpart in the paper.)  Gather n rows of a small dense table through L2 the way the
- * fiber stage of the TTM chains does -- eight lanes per row, one vector load per lane, eight rows in flight per
- * lane -- and do nothing else, asynchronously on cuda_stream.  Timing it gives the ceiling of that access
- * pattern on the device: bytes gathered = (n rounded down to a multiple of 8 per lane group) * row_floats * 4.
- *   table      DEVICE fp32 [rows x ld], row-major, 16-byte aligned, rows * ld < 2^30
- *   row_floats 32 or 16 (floats read per row)
- *   idx        DEVICE int32 [n], every entry in [0, rows); 16-byte aligned
- *   sink       DEVICE fp32 [1]; keeps the loads from being optimised away, practically never written
- * Errors: SA_E_ARG, SA_E_UNSUPPORTED, SA_E_CUDA.
- */
-sa_status sa_probe_row_gather(const float *table, int64_t rows, int64_t ld, int row_floats, const int32_t *idx,
-                              int64_t n, float *sink, void *cuda_stream);
 
 /* Number of kernel launches the last successful sa_run on this handle enqueued. */
 sa_status sa_last_launch_count(const sa_tensor *t, int *launches);

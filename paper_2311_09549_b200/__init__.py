@@ -30,7 +30,7 @@ SA_SCHED_DEFAULT, SA_SCHED_FUSED, SA_SCHED_ASSOC_LEFT, SA_SCHED_ASSOC_RIGHT = 0,
 SA_SCHED_DEBUG_MATERIALIZE = 9
 
 EXPORTED_SYMBOLS = ["sa_tensor_create", "sa_tensor_info", "sa_tensor_export", "sa_tensor_worklist",
-                    "sa_tensor_tasks", "sa_workspace_size", "sa_run", "sa_last_launch_count", "sa_last_device_status", "sa_device_status_words", "sa_probe_row_gather",
+                    "sa_tensor_tasks", "sa_workspace_size", "sa_run", "sa_last_launch_count", "sa_last_device_status", "sa_device_status_words",
                     "sa_destroy", "sa_status_string", "sa_run_ttm3_static_scratch"]
 
 
@@ -57,7 +57,6 @@ _lib.sa_run.argtypes = [_vp, _int, _int, ctypes.POINTER(SaDense), _int, _vp, _vp
 _lib.sa_last_launch_count.argtypes = [_vp, ctypes.POINTER(_int)]
 _lib.sa_last_device_status.argtypes = [_vp, _vp]
 _lib.sa_device_status_words.argtypes = [_vp, _vp, _vp]
-_lib.sa_probe_row_gather.argtypes = [_vp, _i64, _i64, _int, _vp, _i64, _vp, _vp]
 _lib.sa_destroy.argtypes = [_vp]
 _lib.sa_destroy.restype = None
 _lib.sa_status_string.argtypes = [_int]
@@ -202,11 +201,6 @@ def sa_device_status_words(handle, stream):
     words = np.zeros(4, dtype=np.int32)
     _check(_lib.sa_device_status_words(handle, stream, words.ctypes.data), "sa_device_status_words")
     return words
-
-
-def sa_probe_row_gather(table_ptr, rows, ld, row_floats, idx_ptr, n, sink_ptr, stream):
-    _check(_lib.sa_probe_row_gather(table_ptr, int(rows), int(ld), int(row_floats), idx_ptr, int(n), sink_ptr, stream),
-           "sa_probe_row_gather")
 
 
 def sa_destroy(handle):

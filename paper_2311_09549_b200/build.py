@@ -8,7 +8,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsparseauto.so")
 LIB_CHECKED = os.path.join(HERE, "libsparseauto_checked.so")
-SOURCES = ["sa_api.cu", "sa_build.cu", "sa_ttm3.cu", "sa_ttm4.cu", "sa_sddmm_spmm.cu", "sa_spmm_gemm.cu", "sa_ttmc3.cu", "sa_gather_probe.cu", "sa_mttkrp.cu", "sa_dense_tc.cu"]
+SOURCES = ["sa_api.cu", "sa_build.cu", "sa_ttm3.cu", "sa_ttm4.cu", "sa_sddmm_spmm.cu", "sa_spmm_gemm.cu", "sa_ttmc3.cu", "sa_mttkrp.cu", "sa_dense_tc.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC,-fopenmp,-O3", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 
@@ -34,6 +34,23 @@ def build_checked(force=False):
     device before it becomes an address.  Loaded instead of the normal library when the environment variable
     SPARSEAUTO_LIB names it."""
     return build(force=force, flags=["-DSA_DEBUG_BOUNDS"], lib=LIB_CHECKED)
+
+
+PROBE_LIB = os.path.join(HERE, "probe", "libsaprobe.so")
+
+
+def build_probe(force=False):
+    """The bare row-gather kernels bench.py times as the L2-gather ceiling: a measurement aid in a library of
+    its own (nothing of the product path links it)."""
+    src = os.path.join(HERE, "probe", "sa_gather_probe.cu")
+    if not force and os.path.exists(PROBE_LIB) and os.path.getmtime(PROBE_LIB) >= os.path.getmtime(src):
+        return PROBE_LIB
+    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    tmp = PROBE_LIB + ".tmp%d" % os.getpid()
+    subprocess.check_call([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-shared",
+                           "-Xcompiler", "-fPIC", src, "-o", tmp])
+    os.replace(tmp, PROBE_LIB)
+    return PROBE_LIB
 
 
 def _compile(extra, verbose, LIB, tag):
@@ -63,6 +80,8 @@ def _compile(extra, verbose, LIB, tag):
 if __name__ == "__main__":
     if "--checked" in sys.argv:
         print(build_checked(force="--force" in sys.argv))
+    elif "--probe" in sys.argv:
+        print(build_probe(force="--force" in sys.argv))
     else:
         out = [a.split("=", 1)[1] for a in sys.argv if a.startswith("--out=")]
         print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, lib=os.path.abspath(out[0]) if out else LIB))

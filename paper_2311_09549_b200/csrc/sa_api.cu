@@ -1,7 +1,7 @@
 // C-ABI entry points (declared in include/sparseauto.h): handle lifetime, argument checks and
-// the host table (expression, schedule) -> launcher that stands in for the paper's run-time
-// schedule lookup (Section 6, "mapping from schedules chosen at compile-time to the
-// corresponding compiled functions").
+// the host table (expression, schedule) -> launcher that stands in for the run-time lookup from
+// chosen schedules to compiled functions outlined in the paper's discussion of run-time overheads
+// (Section 6).
 #include <cstring>
 #include <new>
 
