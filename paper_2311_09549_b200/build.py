@@ -8,6 +8,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsparseauto.so")
 LIB_CHECKED = os.path.join(HERE, "libsparseauto_checked.so")
+LIB_WAITTEST = os.path.join(HERE, "libsparseauto_waittest.so")
 SOURCES = ["sa_api.cu", "sa_build.cu", "sa_ttm3.cu", "sa_ttm4.cu", "sa_sddmm_spmm.cu", "sa_spmm_gemm.cu", "sa_ttmc3.cu", "sa_mttkrp.cu", "sa_dense_tc.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC,-fopenmp,-O3", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
@@ -34,6 +35,12 @@ def build_checked(force=False):
     device before it becomes an address.  Loaded instead of the normal library when the environment variable
     SPARSEAUTO_LIB names it."""
     return build(force=force, flags=["-DSA_DEBUG_BOUNDS"], lib=LIB_CHECKED)
+
+
+def build_waittest(force=False):
+    """Test library for the bounded device-side waits of the dense stage: hand-offs give up after 2 ms instead of
+    2 s, and a hook (status word 3) makes one arrival stay away so that the time-out path runs."""
+    return build(force=force, flags=["-DSA_TEST_HOOKS", "-DSA_TC_WAIT_NS=2000000ull"], lib=LIB_WAITTEST)
 
 
 PROBE_LIB = os.path.join(HERE, "probe", "libsaprobe.so")
@@ -80,6 +87,8 @@ def _compile(extra, verbose, LIB, tag):
 if __name__ == "__main__":
     if "--checked" in sys.argv:
         print(build_checked(force="--force" in sys.argv))
+    elif "--waittest" in sys.argv:
+        print(build_waittest(force="--force" in sys.argv))
     elif "--probe" in sys.argv:
         print(build_probe(force="--force" in sys.argv))
     else:

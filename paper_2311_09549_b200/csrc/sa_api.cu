@@ -257,15 +257,18 @@ sa_status sa_tensor_create(int order, const int64_t *dims, int64_t nnz, const in
     if (s == SA_OK) {
         try { sa_build_worklists(t); } catch (...) { s = SA_E_ALLOC; }
     }
-    if (s == SA_OK && device >= 0) {
+    if (s == SA_OK && device >= 0) try {
         device_guard g(device);
         if (!g.ok) s = SA_E_CUDA;
+        // An order-4 tensor without subtrees for the order-3 kernel is read through the packed nonzero records
+        // alone: its separate last-level index, value and end-of-fiber arrays stay on the host.
+        const bool packed_only = fmt == SA_FMT_CSF && order == 4 && t->wl_main.items.empty();
         for (int l = 0; l < order && s == SA_OK; ++l) {
             if (fmt == SA_FMT_CSR && l == 0) continue;   // dense level: nothing stored
             s = upload_pos32(t, t->pos[l], &t->d_pos[l]);
-            if (s == SA_OK) s = upload(t, t->crd[l].data(), t->crd[l].size(), &t->d_crd[l]);
+            if (s == SA_OK && !(packed_only && l == order - 1)) s = upload(t, t->crd[l].data(), t->crd[l].size(), &t->d_crd[l]);
         }
-        if (s == SA_OK) s = upload(t, t->vals.data(), t->vals.size(), &t->d_vals);
+        if (s == SA_OK && !packed_only) s = upload(t, t->vals.data(), t->vals.size(), &t->d_vals);
         if (s == SA_OK && fmt == SA_FMT_CSF) {
             // one bit per nonzero: set on the last nonzero of every last-level fiber
             const int last = order - 1;
@@ -274,7 +277,7 @@ sa_status sa_tensor_create(int order, const int64_t *dims, int64_t nnz, const in
                 const int64_t p = t->pos[last][size_t(f) + 1] - 1;
                 bits[size_t(p >> 5)] |= 1u << (p & 31);
             }
-            s = upload(t, bits.data(), bits.size(), &t->d_endbits);
+            if (!packed_only) s = upload(t, bits.data(), bits.size(), &t->d_endbits);
             if (s == SA_OK) {
                 std::vector<int2> pack(size_t(nnz) + 1);
                 for (int64_t p = 0; p < nnz; ++p) {
@@ -298,7 +301,7 @@ sa_status sa_tensor_create(int order, const int64_t *dims, int64_t nnz, const in
         }
         if (s == SA_OK && cudaDeviceSynchronize() != cudaSuccess) s = SA_E_CUDA;
         if (s == SA_E_CUDA) cudaGetLastError();
-    }
+    } catch (...) { s = SA_E_ALLOC; }      // a host vector of the upload section could not be allocated
     if (s != SA_OK) { sa_destroy(t); return s; }
     *out = t;
     return SA_OK;
@@ -456,6 +459,23 @@ sa_status sa_last_device_status(const sa_tensor *t, void *cuda_stream)
     }
     return SA_OK;
 }
+
+#ifdef SA_TEST_HOOKS
+// Test library only (not declared in sparseauto.h): write one of the four device status words.
+sa_status sa_test_set_status_word(const sa_tensor *t, int index, int32_t value, void *cuda_stream)
+{
+    if (!t || t->device < 0 || index < 0 || index > 3) return SA_E_ARG;
+    device_guard g(t->device);
+    if (!g.ok) return SA_E_CUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaMemcpyAsync(t->d_status + index, &value, sizeof(value), cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+        cudaStreamSynchronize(stream) != cudaSuccess) {
+        cudaGetLastError();
+        return SA_E_CUDA;
+    }
+    return SA_OK;
+}
+#endif
 
 void sa_destroy(sa_tensor *t)
 {

@@ -39,7 +39,15 @@ constexpr int TC_MMA_WARP = 4;
 constexpr int TC_CONV_WARPS = 8;
 constexpr int TC_CONV_T = TC_CONV_WARPS * 32;
 constexpr int TC_THREADS = (TC_EPI_WARPS + 1 + TC_CONV_WARPS) * 32;
-constexpr uint64_t TC_WAIT_NS = 2000000000ull;   // longest a hand-off may take before the block gives up
+#ifndef SA_TC_WAIT_NS
+#define SA_TC_WAIT_NS 2000000000ull
+#endif
+constexpr uint64_t TC_WAIT_NS = SA_TC_WAIT_NS;   // longest a hand-off may take before the block gives up (the test
+                                                  // library that exercises the time-out path is built with 2 ms)
+// Library built with -DSA_TEST_HOOKS only: when word 3 of the status words holds this value at launch, one
+// conversion thread of every block withholds its first arrival, so that the first operand hand-off never
+// completes and the bounded waits have to run out (tests/test_gpu_bounded_wait.py).
+constexpr int TC_TEST_WITHHOLD = 0x7e57;
 
 template <int L, int M>
 struct tc_cfg {
@@ -313,6 +321,9 @@ gemm_tc_kernel(int64_t J, const float *__restrict__ C, int64_t ldc, const float 
                 for (int i = 0; i < NR; ++i) b[i] = tc_ldg4(src + min(row0 + 16 * i, J - 1) * ldc);   // rows past the end re-read the last row
             }
         };
+#ifdef SA_TEST_HOOKS
+        const bool withhold = t == 0 && status != nullptr && status[3] == TC_TEST_WITHHOLD;
+#endif
         auto convert = [&](const float4 (&b)[NR], int64_t q) -> bool {
             const uint32_t s = uint32_t(q) % TC_OPS, u = uint32_t(q / TC_OPS);
             if (!mbar_wait(bars + 8 * (B_EMPTY + s), (u & 1u) ^ 1u, abort_flag)) return false;
@@ -326,6 +337,9 @@ gemm_tc_kernel(int64_t J, const float *__restrict__ C, int64_t ldc, const float 
                 *reinterpret_cast<uint2 *>(lo + i * (16 * 128)) = l;
             }
             fence_async_smem();
+#ifdef SA_TEST_HOOKS
+            if (withhold && q == 0) return true;
+#endif
             mbar_arrive(bars + 8 * (B_FULL + s));
             return true;
         };

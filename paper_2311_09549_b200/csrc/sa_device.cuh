@@ -36,6 +36,25 @@ __device__ __forceinline__ bool sa_dbg_ok(int32_t *status, bool ok, int code, in
 #define SA_CHK(status, cond, code, value) true
 #endif
 
+// What the checks of the row / fiber kernels compare against: rows of the gathered dense operand(s), output rows,
+// partial slots, nonzeros (items come from the work lists, indices from crd).
+struct sa_limits {
+    int32_t *status;
+    uint32_t gather_rows, out_rows;
+    int32_t n_slots, nnz;
+};
+
+static inline sa_limits sa_make_limits(const sa_tensor *t, int64_t gather_rows, int64_t out_rows, int64_t n_slots)
+{
+    sa_limits lim;
+    lim.status = t->d_status;
+    lim.gather_rows = uint32_t(gather_rows);
+    lim.out_rows = uint32_t(out_rows);
+    lim.n_slots = int32_t(n_slots);
+    lim.nnz = int32_t(t->nnz);
+    return lim;
+}
+
 // ---- PTX helpers shared by the kernels
 
 // x = hi + lo with hi the upper 19 bits of x (a TF32 number) and lo = x - hi (exact in fp32), itself cut to

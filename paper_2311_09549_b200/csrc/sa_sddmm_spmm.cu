@@ -30,7 +30,7 @@ __global__ void __launch_bounds__(256, 2)
 sddmm_spmm_kernel(const sa_item *__restrict__ items, int64_t n_items, const int32_t *__restrict__ pos,
                   const int32_t *__restrict__ crd, const float *__restrict__ vals, const float *__restrict__ C,
                   uint32_t ldc, const float *__restrict__ D, uint32_t ldd, const float *__restrict__ E, uint32_t lde,
-                  float *__restrict__ out, float *__restrict__ partial, float *__restrict__ sampled)
+                  float *__restrict__ out, float *__restrict__ partial, float *__restrict__ sampled, const sa_limits lim)
 {
     using G = sd_cfg<K, L>;
     extern __shared__ __align__(16) float smem[];
@@ -49,7 +49,8 @@ sddmm_spmm_kernel(const sa_item *__restrict__ items, int64_t n_items, const int3
         const int p = 32 * b + lane;
         j = 0;
         v = 0.f;
-        if (p < total) { j = crd[P0 + p]; v = vals[P0 + p]; }
+        if (p < total && SA_CHK(lim.status, P0 + p >= 0 && P0 + p < lim.nnz, 41, P0 + p)) { j = crd[P0 + p]; v = vals[P0 + p]; }
+        if (!SA_CHK(lim.status, uint32_t(j) < lim.gather_rows, 42, j)) j = 0;
     };
     int cb = 0;                                       // batch the consumer is in
     // per-lane constants of the gather: copy q of a stage moves 16-byte piece x = 32 q + lane, i.e. piece
@@ -107,6 +108,7 @@ sddmm_spmm_kernel(const sa_item *__restrict__ items, int64_t n_items, const int3
 
     const bool piece = it.dest >= 0;
     for (int r = it.out_row; r < it.row_end; ++r) {
+        if (!SA_CHK(lim.status, uint32_t(r) < lim.out_rows && (!piece || it.dest < lim.n_slots), 43, r)) continue;
         const int a = piece ? 0 : pos[r] - P0;
         const int b = piece ? total : pos[r + 1] - P0;
         float acc[G::EV];
@@ -185,7 +187,8 @@ cudaError_t launch(const sa_tensor *t, const sa_dense *ops, float *out, float *p
         return cudaGetLastError();
     kern<<<(unsigned)ctas, 256, smem, stream>>>(wl.d_items, n_items, t->d_pos[1], t->d_crd[1], t->d_vals, ops[0].ptr,
                                                uint32_t(ops[0].ld), ops[1].ptr, uint32_t(ops[1].ld), ops[2].ptr,
-                                               uint32_t(ops[2].ld), out, partial, sampled);
+                                               uint32_t(ops[2].ld), out, partial, sampled,
+                                               sa_make_limits(t, t->dims[1], t->dims[0], wl.n_slots));
     return cudaGetLastError();
 }
 

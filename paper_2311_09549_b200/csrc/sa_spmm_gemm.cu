@@ -50,7 +50,7 @@ __global__ void __launch_bounds__(256, 3)
 spmm_gemm_left_kernel(const sa_item *__restrict__ items, int64_t n_items, const int32_t *__restrict__ pos,
                       const int32_t *__restrict__ crd, const float *__restrict__ vals, const float *__restrict__ C,
                       int64_t ldc, const float *__restrict__ H, int64_t ldh, const float *__restrict__ D, int64_t ldd,
-                      float *__restrict__ out, float *__restrict__ partial)
+                      float *__restrict__ out, float *__restrict__ partial, const sa_limits lim)
 {
     constexpr int LV4 = L / 128, MV = M / 32;
     extern __shared__ __align__(16) float smem[];
@@ -63,8 +63,10 @@ spmm_gemm_left_kernel(const sa_item *__restrict__ items, int64_t n_items, const 
          idx += int64_t(gridDim.x) * SA_WARPS_PER_CTA) {
         const sa_item it = items[idx];
         for (int r = it.out_row; r < it.row_end; ++r) {
+            if (!SA_CHK(lim.status, uint32_t(r) < lim.out_rows && it.dest < lim.n_slots, 51, r)) continue;
             const int a = it.dest >= 0 ? it.p0 : pos[r];
             const int b = it.dest >= 0 ? it.p1 : pos[r + 1];
+            if (!SA_CHK(lim.status, a >= 0 && a <= b && b <= lim.nnz, 52, b)) continue;
             float4 t[LV4];
 #pragma unroll
             for (int q = 0; q < LV4; ++q) t[q] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -73,6 +75,7 @@ spmm_gemm_left_kernel(const sa_item *__restrict__ items, int64_t n_items, const 
                 int jj = 0;
                 float vv = 0.f;
                 if (lane < n) { jj = crd[base + lane]; vv = vals[base + lane]; }
+                if (!SA_CHK(lim.status, uint32_t(jj) < lim.gather_rows, 53, jj)) jj = 0;
 #pragma unroll LEFT_UNROLL
                 for (int s = 0; s < n; ++s) {
                     const int j = __shfl_sync(SA_FULL_MASK, jj, s);
@@ -261,7 +264,7 @@ template <int MV>
 __global__ void __launch_bounds__(256)
 spmm_kernel(const sa_item *__restrict__ items, int64_t n_items, const int32_t *__restrict__ pos,
             const int32_t *__restrict__ crd, const float *__restrict__ vals, const float *__restrict__ E,
-            float *__restrict__ out, float *__restrict__ partial)
+            float *__restrict__ out, float *__restrict__ partial, const sa_limits lim)
 {
     constexpr int M = MV * 32;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -269,8 +272,10 @@ spmm_kernel(const sa_item *__restrict__ items, int64_t n_items, const int32_t *_
     if (idx >= n_items) return;
     const sa_item it = items[idx];
     for (int r = it.out_row; r < it.row_end; ++r) {
+        if (!SA_CHK(lim.status, uint32_t(r) < lim.out_rows && it.dest < lim.n_slots, 54, r)) continue;
         const int a = it.dest >= 0 ? it.p0 : pos[r];
         const int b = it.dest >= 0 ? it.p1 : pos[r + 1];
+        if (!SA_CHK(lim.status, a >= 0 && a <= b && b <= lim.nnz, 55, b)) continue;
         float acc[MV];
 #pragma unroll
         for (int q = 0; q < MV; ++q) acc[q] = 0.f;
@@ -279,6 +284,7 @@ spmm_kernel(const sa_item *__restrict__ items, int64_t n_items, const int32_t *_
             int jj = 0;
             float vv = 0.f;
             if (lane < n) { jj = crd[base + lane]; vv = vals[base + lane]; }
+            if (!SA_CHK(lim.status, uint32_t(jj) < lim.gather_rows, 56, jj)) jj = 0;
 #pragma unroll 8
             for (int s = 0; s < n; ++s) {
                 const int j = __shfl_sync(SA_FULL_MASK, jj, s);
@@ -311,7 +317,7 @@ template <int M>
 __global__ void __launch_bounds__(256)
 fiber_spmm_kernel(const sa_item *__restrict__ items, int64_t n_items, const int32_t *__restrict__ pos,
                   const int2 *__restrict__ nz, const float *__restrict__ E, int64_t lde, float *__restrict__ out,
-                  float *__restrict__ partial)
+                  float *__restrict__ partial, const sa_limits lim)
 {
     constexpr int LPR = M / 4, NG = 32 / LPR;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -337,7 +343,7 @@ fiber_spmm_kernel(const sa_item *__restrict__ items, int64_t n_items, const int3
         const int p = ga + c + (l & 7);
         x = 0;
         v = 0.f;
-        if (c + (l & 7) < mylen) {
+        if (c + (l & 7) < mylen && SA_CHK(lim.status, p >= 0 && p < lim.nnz, 61, p)) {
             const int2 w = __ldg(nz + p);                            // (index | end-of-fiber bit << 31, value bits)
             x = piece ? (w.x & 0x7fffffff) : w.x;
             v = __int_as_float(w.y);
@@ -358,7 +364,9 @@ fiber_spmm_kernel(const sa_item *__restrict__ items, int64_t n_items, const int3
         for (int u = 0; u < 8; ++u) {                                 // positions past the group's end: row 0, value 0
             xs[u] = __shfl_sync(SA_FULL_MASK, x, u, LPR);
             vs[u] = __shfl_sync(SA_FULL_MASK, v, u, LPR);
-            e[u] = sa_ldg4(E + int64_t(xs[u] & 0x7fffffff) * lde + 4 * l);
+            uint32_t k = uint32_t(xs[u]) & 0x7fffffffu;
+            if (!SA_CHK(lim.status, k < lim.gather_rows, 62, k)) k = 0u;
+            e[u] = sa_ldg4(E + int64_t(k) * lde + 4 * l);
         }
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
@@ -369,7 +377,7 @@ fiber_spmm_kernel(const sa_item *__restrict__ items, int64_t n_items, const int3
                 acc.w = fmaf(vs[u], e[u].w, acc.w);
             }
             if (xs[u] < 0) {                                          // last nonzero of its fiber
-                *reinterpret_cast<float4 *>(out + int64_t(row) * M + 4 * l) = acc;
+                if (SA_CHK(lim.status, uint32_t(row) < lim.out_rows, 63, row)) *reinterpret_cast<float4 *>(out + int64_t(row) * M + 4 * l) = acc;
                 acc = make_float4(0.f, 0.f, 0.f, 0.f);
                 ++row;
             }
@@ -383,7 +391,7 @@ fiber_spmm_kernel(const sa_item *__restrict__ items, int64_t n_items, const int3
             acc.z += __shfl_xor_sync(SA_FULL_MASK, acc.z, off);
             acc.w += __shfl_xor_sync(SA_FULL_MASK, acc.w, off);
         }
-        if (g == 0) *reinterpret_cast<float4 *>(partial + int64_t(it.dest) * M + 4 * l) = acc;
+        if (g == 0 && SA_CHK(lim.status, it.dest < lim.n_slots, 64, it.dest)) *reinterpret_cast<float4 *>(partial + int64_t(it.dest) * M + 4 * l) = acc;
     }
 }
 
@@ -411,7 +419,8 @@ sa_status run(const sa_tensor *t, const sa_dense *ops, float *out, void *ws, boo
         const int64_t ctas = std::min<int64_t>(want, resident_ctas(reinterpret_cast<const void *>(kern), smem));
         if (ctas > 0) {
             kern<<<(unsigned)ctas, 256, smem, stream>>>(wl.d_items, n_items, t->d_pos[1], t->d_crd[1], t->d_vals, ops[0].ptr,
-                                                       ops[0].ld, ops[0].ptr, ops[0].ld, ops[1].ptr, ops[1].ld, out, partial);
+                                                       ops[0].ld, ops[0].ptr, ops[0].ld, ops[1].ptr, ops[1].ld, out, partial,
+                                                       sa_make_limits(t, t->dims[1], t->dims[0], wl.n_slots));
             if (cudaGetLastError() != cudaSuccess) return SA_E_CUDA;
             *launches += 1;
         }
@@ -430,7 +439,7 @@ sa_status run(const sa_tensor *t, const sa_dense *ops, float *out, void *ws, boo
     const int64_t ctas = (n_items + SA_WARPS_PER_CTA - 1) / SA_WARPS_PER_CTA;
     if (ctas > 0) {
         spmm_kernel<M / 32><<<(unsigned)ctas, 256, 0, stream>>>(wl.d_items, n_items, t->d_pos[1], t->d_crd[1], t->d_vals, E,
-                                                               out, partial);
+                                                               out, partial, sa_make_limits(t, J, t->dims[0], wl.n_slots));
         if (cudaGetLastError() != cudaSuccess) return SA_E_CUDA;
         *launches += 1;
     }
@@ -456,7 +465,8 @@ sa_status run_hadamard(const sa_tensor *t, const sa_dense *ops, float *out, void
     const int64_t ctas = std::min<int64_t>(want, resident_ctas(reinterpret_cast<const void *>(kern), smem));
     if (ctas > 0) {
         kern<<<(unsigned)ctas, 256, smem, stream>>>(wl.d_items, n_items, t->d_pos[1], t->d_crd[1], t->d_vals, ops[0].ptr,
-                                                   ops[0].ld, ops[1].ptr, ops[1].ld, ops[2].ptr, ops[2].ld, out, partial);
+                                                   ops[0].ld, ops[1].ptr, ops[1].ld, ops[2].ptr, ops[2].ld, out, partial,
+                                                   sa_make_limits(t, t->dims[1], t->dims[0], wl.n_slots));
         if (cudaGetLastError() != cudaSuccess) return SA_E_CUDA;
         *launches += 1;
     }
@@ -486,7 +496,8 @@ sa_status run_fibers(const sa_tensor *t, const sa_dense *ops, float *out, void *
         if (gs != SA_OK) return gs;
         *launches += 1;
         if (ctas > 0) {
-            fiber_spmm_kernel<M><<<(unsigned)ctas, 256, 0, stream>>>(wl.d_items, n_items, t->d_pos[2], t->d_nzpack, E, M, out, partial);
+            fiber_spmm_kernel<M><<<(unsigned)ctas, 256, 0, stream>>>(wl.d_items, n_items, t->d_pos[2], t->d_nzpack, E, M, out, partial,
+                                                                     sa_make_limits(t, K, F2, wl.n_slots));
             if (cudaGetLastError() != cudaSuccess) return SA_E_CUDA;
             *launches += 1;
         }
@@ -500,7 +511,7 @@ sa_status run_fibers(const sa_tensor *t, const sa_dense *ops, float *out, void *
     float *partial = reinterpret_cast<float *>(static_cast<char *>(ws) + sa_align256(size_t(F2) * L * sizeof(float)));
     if (ctas > 0) {
         fiber_spmm_kernel<L><<<(unsigned)ctas, 256, 0, stream>>>(wl.d_items, n_items, t->d_pos[2], t->d_nzpack, ops[0].ptr, ops[0].ld,
-                                                                T, partial);
+                                                                T, partial, sa_make_limits(t, K, F2, wl.n_slots));
         if (cudaGetLastError() != cudaSuccess) return SA_E_CUDA;
         *launches += 1;
     }

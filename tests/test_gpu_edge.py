@@ -6,7 +6,7 @@ import pytest
 
 import oracle
 from workloads import configs, rng
-from util import TOL_FP32, assert_close, run_gpu
+from util import TOL_FP32, assert_close, fmt_of, run_gpu
 
 pytestmark = pytest.mark.gpu
 
@@ -305,3 +305,51 @@ def test_ttm4_padded_factor_matrices(sa):
     assert sa.sa_last_device_status(t.handle, torch.cuda.current_stream().cuda_stream) == sa.SA_OK
     assert_close(out.cpu().numpy().astype(np.float64), A_ref, S_ref, TOL_FP32, "ttm4 padded ld")
     assert int(sa.sa_tensor_worklist(t.handle, 2)[0][0]) > 0
+
+
+def test_allocator_failure_at_every_upload_is_reported_and_leaks_nothing(sa):
+    """The device allocator returns NULL at the k-th request, for every k up to the number of requests a tensor
+    makes: create answers SA_E_ALLOC, hands out no handle, and every block it had obtained is released."""
+    import ctypes
+    import torch
+    base = sa.TorchAllocator(0)
+
+    class Failing:
+        def __init__(self, fail_at):
+            self.calls, self.fail_at, self.live = 0, fail_at, set()
+            self._a = sa._ALLOC_FN(self.alloc)
+            self._r = sa._RELEASE_FN(self.release)
+            self.struct = sa.SaAllocator(self._a, self._r, None)
+
+        def alloc(self, nbytes, ctx):
+            self.calls += 1
+            if self.calls - 1 == self.fail_at:
+                return None
+            p = base._do_alloc(nbytes, ctx)
+            self.live.add(p)
+            return p
+
+        def release(self, ptr, ctx):
+            self.live.discard(ptr)
+            base._do_release(ptr, ctx)
+
+    for cfg in (1, 3, 5):
+        w = configs.make(cfg, "mini")
+        fmt = fmt_of(sa, w)
+        k = 0
+        while True:
+            a = Failing(k)
+            try:
+                h = sa.sa_tensor_create(len(w.dims), w.dims, len(w.vals), w.coords, w.vals, fmt, 0, a.struct)
+            except sa.SaError as e:
+                assert e.status == sa.SA_E_ALLOC, (cfg, k, e)
+                assert a.calls == k + 1 and not a.live, "blocks obtained before the failure must be released"
+                k += 1
+                continue
+            assert a.calls <= k, "with no failing request the tensor is created"
+            assert len(a.live) == a.calls
+            sa.sa_destroy(h)
+            assert not a.live
+            break
+        assert k >= 8, "the loop really walked through the uploads"
+    torch.cuda.synchronize()
