@@ -87,8 +87,9 @@ typedef enum {
 } sa_expr;
 
 typedef enum {
-    SA_SCHED_DEFAULT = 0,      /* the host table's choice for the expression; for SPMM_GEMM the
-                                  association order that moves fewer bytes for this tensor      */
+    SA_SCHED_DEFAULT = 0,      /* the host table's choice for the expression; where two schedules exist
+                                  (SPMM_GEMM, SPTTM_SPTTM) the one that moves fewer bytes for this
+                                  tensor among those within the auxiliary-memory cap, see sa_schedule_cost */
     SA_SCHED_FUSED = 1,        /* the fissioned / fused branched nest of the Table of kernels   */
     SA_SCHED_ASSOC_LEFT = 2,   /* SA_EXPR_SPMM_GEMM (and SPTTM_SPTTM): (B.C).D, row temporary of L floats    */
     SA_SCHED_ASSOC_RIGHT = 3,  /* SA_EXPR_SPMM_GEMM (and SPTTM_SPTTM): B.(C.D), J x M temporary in workspace */
@@ -208,6 +209,41 @@ sa_status sa_tensor_tasks(const sa_tensor *t, int64_t *n_tasks, int32_t *task_st
  * shapes in ops are read. */
 sa_status sa_workspace_size(const sa_tensor *t, sa_expr expr, sa_schedule sched, const sa_dense *ops,
                             int n_ops, size_t *bytes);
+
+/*
+ * What a schedule costs for this tensor and these operand shapes: the quantities the paper's run-time Stage 4
+ * (Section 5.2) compares -- a time term and the auxiliary memory -- with concrete sizes plugged in.
+ *   iterations      iteration complexity of the branched loop nest that runs, i.e. its total number of loop
+ *                   iterations in the sense of Section 3 (the caption formulas of the figure with the five
+ *                   schedules of kernel 5 are of this kind); sparse loops count stored nodes of their level
+ *   moved_bytes     bytes the schedule's kernels load and store: streams of B once, the output once, dense
+ *                   operands that are read in order once, gathered rows once per use (a row served by the
+ *                   last-level cache still occupies the load path), temporaries in the workspace written and
+ *                   read.  This is the time term the default schedule is chosen by (the chains are bound by
+ *                   memory traffic here, not by loop iterations).
+ *   temp_elements   dense temporaries that pass values from producer to consumer nests, in elements: the
+ *                   paper's auxiliary memory (Section 4.2; table of auxiliary memory requirements, Section 6),
+ *                   whether they live in registers, shared memory or the workspace
+ *   workspace_bytes what sa_workspace_size returns for the schedule
+ *   resolved        the schedule that runs (differs from `sched` for SA_SCHED_DEFAULT)
+ * Only the shapes in ops are read.  Errors: SA_E_ARG, SA_E_FORMAT, SA_E_SHAPE, SA_E_UNSUPPORTED.
+ */
+typedef struct {
+    double iterations, moved_bytes, temp_elements;
+    size_t workspace_bytes;
+    int resolved;
+} sa_cost;
+sa_status sa_schedule_cost(const sa_tensor *t, sa_expr expr, sa_schedule sched, const sa_dense *ops, int n_ops,
+                           sa_cost *cost);
+
+/*
+ * Cap, in bytes, on the workspace a schedule picked by SA_SCHED_DEFAULT may need (the user-given upper bound on
+ * auxiliary memory that Section 5.2 mentions for its memory pruning; the paper's own Stage 4 uses half of the
+ * last-level cache).  Among the expression's schedules whose workspace fits, the default takes the one with the
+ * smallest moved_bytes; if none fits, the one with the smallest workspace.  Explicitly named schedules are not
+ * affected.  Default: no cap.  Set it before sizing workspaces; not synchronised with concurrent sa_run calls.
+ */
+sa_status sa_tensor_set_aux_limit(sa_tensor *t, size_t bytes);
 
 /*
  * Evaluate the chain: out = expr(B, ops...), asynchronously on cuda_stream.

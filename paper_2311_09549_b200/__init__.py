@@ -30,7 +30,7 @@ SA_SCHED_DEFAULT, SA_SCHED_FUSED, SA_SCHED_ASSOC_LEFT, SA_SCHED_ASSOC_RIGHT = 0,
 SA_SCHED_DEBUG_MATERIALIZE = 9
 
 EXPORTED_SYMBOLS = ["sa_tensor_create", "sa_tensor_info", "sa_tensor_export", "sa_tensor_worklist",
-                    "sa_tensor_tasks", "sa_workspace_size", "sa_run", "sa_last_launch_count", "sa_last_device_status", "sa_device_status_words",
+                    "sa_tensor_tasks", "sa_workspace_size", "sa_schedule_cost", "sa_tensor_set_aux_limit", "sa_run", "sa_last_launch_count", "sa_last_device_status", "sa_device_status_words",
                     "sa_destroy", "sa_status_string", "sa_run_ttm3_static_scratch"]
 
 
@@ -53,6 +53,13 @@ _lib.sa_tensor_export.argtypes = [_vp, _int, _vp, _vp, _vp]
 _lib.sa_tensor_worklist.argtypes = [_vp, _int, _vp, _vp, _vp]
 _lib.sa_tensor_tasks.argtypes = [_vp, ctypes.POINTER(_i64), _vp, _vp]
 _lib.sa_workspace_size.argtypes = [_vp, _int, _int, ctypes.POINTER(SaDense), _int, ctypes.POINTER(ctypes.c_size_t)]
+class SaCost(ctypes.Structure):
+    _fields_ = [("iterations", ctypes.c_double), ("moved_bytes", ctypes.c_double), ("temp_elements", ctypes.c_double),
+                ("workspace_bytes", ctypes.c_size_t), ("resolved", ctypes.c_int)]
+
+
+_lib.sa_schedule_cost.argtypes = [_vp, _int, _int, ctypes.POINTER(SaDense), _int, ctypes.POINTER(SaCost)]
+_lib.sa_tensor_set_aux_limit.argtypes = [_vp, ctypes.c_size_t]
 _lib.sa_run.argtypes = [_vp, _int, _int, ctypes.POINTER(SaDense), _int, _vp, _vp, ctypes.c_size_t, _vp]
 _lib.sa_last_launch_count.argtypes = [_vp, ctypes.POINTER(_int)]
 _lib.sa_last_device_status.argtypes = [_vp, _vp]
@@ -171,6 +178,18 @@ def sa_workspace_size(handle, expr, sched, ops):
     _check(_lib.sa_workspace_size(handle, int(expr), int(sched), _dense_array(ops), len(ops), ctypes.byref(n)),
            "sa_workspace_size")
     return n.value
+
+
+def sa_schedule_cost(handle, expr, sched, ops):
+    """ops: list of (ptr, rows, cols, ld); only the shapes are read.  Returns a dict of the sa_cost fields."""
+    c = SaCost()
+    _check(_lib.sa_schedule_cost(handle, int(expr), int(sched), _dense_array(ops), len(ops), ctypes.byref(c)), "sa_schedule_cost")
+    return {"iterations": c.iterations, "moved_bytes": c.moved_bytes, "temp_elements": c.temp_elements,
+            "workspace_bytes": int(c.workspace_bytes), "resolved": int(c.resolved)}
+
+
+def sa_tensor_set_aux_limit(handle, nbytes):
+    _check(_lib.sa_tensor_set_aux_limit(handle, int(nbytes)), "sa_tensor_set_aux_limit")
 
 
 def sa_run(handle, expr, sched, ops, out_ptr, workspace_ptr, workspace_bytes, stream):

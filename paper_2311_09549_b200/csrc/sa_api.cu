@@ -157,14 +157,115 @@ sa_status check_ops(const sa_tensor *t, sa_expr expr, const sa_dense *ops, int n
     return SA_OK;
 }
 
-// Host table: which concrete schedule runs for (expr, sched).  Returns false if the pair is
-// not in the table.  For SA_EXPR_SPMM_GEMM the default is chosen per tensor, in the spirit of the
-// paper's run-time Stage 4 (Section 5: the schedules that survive compile-time pruning are
-// compared with the concrete sizes plugged into their cost expressions): both association orders
-// are bound by memory traffic here, so the cost is the bytes each one must move,
-//   (B.C).D : nnz * (8 + 4 L)                     one row of C per nonzero
-//   B.(C.D) : 4 J (L + M) + nnz * (8 + 4 M)       C read and E = C.D written once, one row of E per nonzero
-// and the cheaper one runs (its J x M temporary comes out of the caller's workspace).
+size_t workspace_bytes(const sa_tensor *t, sa_expr expr, sa_schedule sched, const sa_dense *ops);
+
+// Bytes loaded for `uses` row reads of a dense table with `cols` columns: one row per use, whether the row comes
+// from HBM or from the last-level cache (a gathered row occupies the load path either way; with the table
+// counted once when it fits the cache, the model preferred (B.C).D on cache-resident C where B.(C.D) measured
+// 1.2 to 1.8 times faster).
+double table_bytes(const sa_tensor *, double, double cols, double uses) { return 4.0 * cols * uses; }
+
+// Cost of one concrete schedule (not DEFAULT): see sa_schedule_cost in sparseauto.h.
+void schedule_cost(const sa_tensor *t, sa_expr expr, sa_schedule sched, const sa_dense *ops, sa_cost *c)
+{
+    const double nnz = double(t->nnz), I = double(t->dims[0]);
+    const double F2 = t->fmt == SA_FMT_CSF ? double(t->count[1]) : 0.0, F3 = t->order == 4 ? double(t->count[2]) : 0.0;
+    const double S = t->fmt == SA_FMT_CSF ? double(t->count[0]) : I;
+    double it = 0, by = 0, tmp = 0;
+    switch (expr) {
+        case SA_EXPR_SPTTM_TTM3: {      // i, j' < t(m); k': t += B D , l: A += t C >
+            const double L = ops[0].cols, M = ops[1].cols;
+            it = nnz * M + F2 * L * M;
+            tmp = M;
+            by = 8 * nnz + 8 * F2 + 8 * S + table_bytes(t, ops[0].rows, L, F2) + table_bytes(t, ops[1].rows, M, nnz) + 4 * I * L * M;
+            break;
+        }
+        case SA_EXPR_SPTTM_TTM4: {      // i, j' < T2(m,n); k' < t(n); o': .. , m: .. > , l: .. >
+            const double L = ops[0].cols, M = ops[1].cols, N = ops[2].cols;
+            it = nnz * N + F3 * M * N + F2 * L * M * N;
+            tmp = N + M * N;
+            by = 8 * nnz + 8 * F3 + 8 * F2 + 8 * S + table_bytes(t, ops[0].rows, L, F2) + table_bytes(t, ops[1].rows, M, F3) +
+                 table_bytes(t, ops[2].rows, N, nnz) + 4 * I * L * M * N;
+            break;
+        }
+        case SA_EXPR_SDDMM_SPMM: {      // i, j' < t; k: t += B C D , l: A += t E >
+            const double K = ops[0].cols, L = ops[2].cols;
+            it = nnz * (K + L);
+            tmp = 1;
+            by = 8 * nnz + 4 * (I + 1) + 4 * I * K + table_bytes(t, ops[1].rows, K, nnz) + table_bytes(t, ops[2].rows, L, nnz) + 4 * I * L;
+            break;
+        }
+        case SA_EXPR_SDDMM_SPMM_GEMM: { // i < T(l); j' < t; k: .. , l: T += t E > , m,l: A += T F >
+            const double K = ops[0].cols, L = ops[2].cols, M = ops[3].cols;
+            it = nnz * (K + L) + I * L * M;
+            tmp = 1 + L;
+            by = 8 * nnz + 4 * (I + 1) + 4 * I * K + table_bytes(t, ops[1].rows, K, nnz) + table_bytes(t, ops[2].rows, L, nnz) +
+                 8 * I * L + 4 * L * M + 4 * I * M;
+            break;
+        }
+        case SA_EXPR_SPMMH_GEMM: {      // i < T(l); j', l: T += B C D , m,l: A += T E >
+            const double L = ops[0].cols, M = ops[2].cols;
+            it = nnz * L + I * L * M;
+            tmp = L;
+            by = 8 * nnz + 4 * (I + 1) + table_bytes(t, ops[0].rows, L, nnz) + table_bytes(t, ops[1].rows, L, nnz) + 4 * L * M + 4 * I * M;
+            break;
+        }
+        case SA_EXPR_SPMM_GEMM: {
+            const double J = double(t->dims[1]), L = ops[0].cols, M = ops[1].cols;
+            if (sched == SA_SCHED_ASSOC_RIGHT) {   // < E(j,m); j,l,m: E += C D , i,j',m: A += B E >
+                it = J * L * M + nnz * M;
+                tmp = J * M;
+                by = 4 * J * (L + M) + 4 * L * M + 8 * nnz + 4 * (I + 1) + table_bytes(t, J, M, nnz) + 4 * I * M;
+            } else {                               // i < T(l); j',l: T += B C , m,l: A += T D >
+                it = nnz * L + I * L * M;
+                tmp = L;
+                by = 8 * nnz + 4 * (I + 1) + table_bytes(t, J, L, nnz) + 4 * L * M + 4 * I * M;
+            }
+            break;
+        }
+        case SA_EXPR_SPTTM_SPTTM: {
+            const double K = double(t->dims[2]), L = ops[0].cols, M = ops[1].cols;
+            if (sched == SA_SCHED_ASSOC_RIGHT) {   // < E(k,m); k,l,m: E += C D , (i,j'),k',m: A += B E >
+                it = K * L * M + nnz * M;
+                tmp = K * M;
+                by = 4 * K * (L + M) + 4 * L * M + 8 * nnz + 4 * (F2 + 1) + table_bytes(t, K, M, nnz) + 4 * F2 * M;
+            } else {                               // (i,j') < T(l); k',l: T += B C , m,l: A += T D >, T kept for the dense stage
+                it = nnz * L + F2 * L * M;
+                tmp = F2 * L;
+                by = 8 * nnz + 4 * (F2 + 1) + table_bytes(t, K, L, nnz) + 8 * F2 * L + 4 * L * M + 4 * F2 * M;
+            }
+            break;
+        }
+        case SA_EXPR_TTMC3: {           // i < T(m,n); j' < t(n); k': .. , m: .. > > fissioned from l: A += T C
+            const double L = ops[0].cols, M = ops[1].cols, N = ops[2].cols;
+            it = nnz * N + F2 * M * N + I * L * M * N;
+            tmp = N + I * M * N;
+            by = 8 * nnz + 8 * F2 + 8 * S + table_bytes(t, ops[1].rows, M, F2) + table_bytes(t, ops[2].rows, N, nnz) + 8 * I * M * N +
+                 4 * I * L + 4 * L * M * N;
+            break;
+        }
+        case SA_EXPR_MTTKRP_GEMM: {     // i < T(r); j' < t(r); k': t += B D , r: T += t C > , m,r: A += T E >
+            const double R = ops[0].cols, M = ops[2].cols;
+            it = nnz * R + F2 * R + I * R * M;
+            tmp = R + I * R;
+            by = 8 * nnz + 8 * F2 + 8 * S + table_bytes(t, ops[0].rows, R, F2) + table_bytes(t, ops[1].rows, R, nnz) + 8 * I * R +
+                 4 * R * M + 4 * I * M;
+            break;
+        }
+    }
+    c->iterations = it;
+    c->moved_bytes = by;
+    c->temp_elements = tmp;
+    c->workspace_bytes = workspace_bytes(t, expr, sched, ops);
+    c->resolved = int(sched);
+}
+
+// Host table: which concrete schedule runs for (expr, sched).  Returns false if the pair is not in the table.
+// Where an expression has two schedules the default is chosen per tensor, in the spirit of the paper's run-time
+// Stage 4 (Section 5.2: the schedules that survive compile-time pruning are compared with the concrete sizes
+// plugged into their cost expressions, and one whose auxiliary memory is too large is passed over): among the
+// candidates whose workspace is within the tensor's auxiliary-memory cap the one that moves fewer bytes runs;
+// when none fits, the one with the smaller workspace.
 bool resolve_schedule(const sa_tensor *t, sa_expr expr, sa_schedule sched, const sa_dense *ops, sa_schedule *resolved)
 {
     switch (expr) {
@@ -181,25 +282,18 @@ bool resolve_schedule(const sa_tensor *t, sa_expr expr, sa_schedule sched, const
             if (sched == SA_SCHED_DEBUG_MATERIALIZE) { *resolved = sched; return true; }
             return false;
         case SA_EXPR_SPMM_GEMM:
-            if (sched == SA_SCHED_DEFAULT) {
-                const double nnz = double(t->nnz), J = double(t->dims[1]), L = double(ops[0].cols), M = double(ops[1].cols);
-                const double left = nnz * (8.0 + 4.0 * L);
-                const double right = 4.0 * J * (L + M) + nnz * (8.0 + 4.0 * M);
-                *resolved = left <= right ? SA_SCHED_ASSOC_LEFT : SA_SCHED_ASSOC_RIGHT;
-                return true;
-            }
-            if (sched == SA_SCHED_FUSED || sched == SA_SCHED_ASSOC_LEFT) { *resolved = SA_SCHED_ASSOC_LEFT; return true; }
-            if (sched == SA_SCHED_ASSOC_RIGHT) { *resolved = sched; return true; }
-            return false;
         case SA_EXPR_SPTTM_SPTTM:
-            // the same comparison with the fibers as rows: the fiber temporaries are written and read once
-            //   (B'.C).D : nnz * (8 + 4 L) + 8 F2 L        B'.(C.D) : 4 K (L + M) + nnz * (8 + 4 M)
             if (sched == SA_SCHED_DEFAULT) {
-                const double nnz = double(t->nnz), F2 = double(t->count[1]), K = double(t->dims[2]);
-                const double L = double(ops[0].cols), M = double(ops[1].cols);
-                const double left = nnz * (8.0 + 4.0 * L) + 8.0 * F2 * L;
-                const double right = 4.0 * K * (L + M) + nnz * (8.0 + 4.0 * M);
-                *resolved = left <= right ? SA_SCHED_ASSOC_LEFT : SA_SCHED_ASSOC_RIGHT;
+                sa_cost left, right;
+                schedule_cost(t, expr, SA_SCHED_ASSOC_LEFT, ops, &left);
+                schedule_cost(t, expr, SA_SCHED_ASSOC_RIGHT, ops, &right);
+                const uint64_t cap = t->aux_limit.load();
+                const bool lf = left.workspace_bytes <= cap, rf = right.workspace_bytes <= cap;
+                bool take_left;
+                if (lf != rf) take_left = lf;
+                else if (!lf) take_left = left.workspace_bytes <= right.workspace_bytes;
+                else take_left = left.moved_bytes <= right.moved_bytes;
+                *resolved = take_left ? SA_SCHED_ASSOC_LEFT : SA_SCHED_ASSOC_RIGHT;
                 return true;
             }
             if (sched == SA_SCHED_FUSED || sched == SA_SCHED_ASSOC_LEFT) { *resolved = SA_SCHED_ASSOC_LEFT; return true; }
@@ -377,6 +471,24 @@ sa_status sa_workspace_size(const sa_tensor *t, sa_expr expr, sa_schedule sched,
     sa_schedule r;
     if (!resolve_schedule(t, expr, sched, ops, &r)) return SA_E_UNSUPPORTED;
     *bytes = workspace_bytes(t, expr, r, ops);
+    return SA_OK;
+}
+
+sa_status sa_schedule_cost(const sa_tensor *t, sa_expr expr, sa_schedule sched, const sa_dense *ops, int n_ops, sa_cost *cost)
+{
+    if (!t || !cost) return SA_E_ARG;
+    sa_status s = check_ops(t, expr, ops, n_ops, true);
+    if (s != SA_OK) return s;
+    sa_schedule r;
+    if (!resolve_schedule(t, expr, sched, ops, &r)) return SA_E_UNSUPPORTED;
+    schedule_cost(t, expr, r, ops, cost);
+    return SA_OK;
+}
+
+sa_status sa_tensor_set_aux_limit(sa_tensor *t, size_t bytes)
+{
+    if (!t) return SA_E_ARG;
+    t->aux_limit = uint64_t(bytes);
     return SA_OK;
 }
 

@@ -114,7 +114,8 @@ struct sa_tensor {
     int32_t *d_f4_supers = nullptr, *d_f4_pieces = nullptr;
     int32_t f4_n_large = 0;
 
-    mutable std::atomic<int> last_launches{0};   // the only mutable field: concurrent sa_run calls may write it
+    mutable std::atomic<int> last_launches{0};   // concurrent sa_run calls may write it
+    std::atomic<uint64_t> aux_limit{~uint64_t(0)};   // caller's cap on a default schedule's workspace (sa_tensor_set_aux_limit)
     std::vector<void *> dev_blocks;           // everything obtained from the allocator
 };
 

@@ -371,25 +371,6 @@ def test_library_exports_every_declared_symbol():
         assert hasattr(lib, name), name
 
 
-def test_default_association_order_follows_the_byte_cost_model():
-    # few nonzeros, many columns: B.(C.D) would compute C.D for 50 000 rows that are hardly used
-    rs = np.random.RandomState(3)
-    J = 50_000
-    coords = np.stack([rs.randint(0, 100, 500), rs.choice(J, 500, replace=False)], axis=1).astype(np.int32)
-    sparse = sa.SparseTensor((100, J), coords, np.ones(500, np.float32), sa.SA_FMT_CSR, device=-1)
-    ops = [(16, J, 256, 256), (16, 256, 64, 64)]
-    ws = {s: sa.sa_workspace_size(sparse.handle, sa.SA_EXPR_SPMM_GEMM, s, ops)
-          for s in (sa.SA_SCHED_DEFAULT, sa.SA_SCHED_ASSOC_LEFT, sa.SA_SCHED_ASSOC_RIGHT)}
-    assert ws[sa.SA_SCHED_ASSOC_RIGHT] >= J * 64 * 4 > ws[sa.SA_SCHED_ASSOC_LEFT]
-    assert ws[sa.SA_SCHED_DEFAULT] == ws[sa.SA_SCHED_ASSOC_LEFT]
-    # many nonzeros per column: gathering 1 KB rows of C per nonzero costs more than forming E = C.D once
-    w = configs.make(4, "mini")
-    dense = sa.SparseTensor(w.dims, w.coords, w.vals, sa.SA_FMT_CSR, device=-1)
-    ops = [(16, w.dims[1], 256, 256), (16, 256, 64, 64)]
-    assert (sa.sa_workspace_size(dense.handle, sa.SA_EXPR_SPMM_GEMM, sa.SA_SCHED_DEFAULT, ops)
-            == sa.sa_workspace_size(dense.handle, sa.SA_EXPR_SPMM_GEMM, sa.SA_SCHED_ASSOC_RIGHT, ops))
-
-
 def test_fiber_row_worklist_of_order3_csf_partitions_fibers_and_nonzeros():
     """Kernel 7 walks an order-3 CSF tensor as a sparse matrix with one row per (i,j) fiber: its work list
     (the second one of the tensor) covers every fiber and every nonzero once; a fiber longer than 4096

@@ -353,3 +353,40 @@ def test_allocator_failure_at_every_upload_is_reported_and_leaks_nothing(sa):
             break
         assert k >= 8, "the loop really walked through the uploads"
     torch.cuda.synchronize()
+
+
+def test_default_order_of_spmm_gemm_picks_the_faster_one_on_both_sides(sa):
+    """The run-time choice between (B.C).D and B.(C.D) on two tensors where it goes opposite ways, checked against
+    device timings: with few nonzeros on a huge C, forming C.D reads 2 GB that (B.C).D never touches; with many
+    nonzeros per column, one gathered 1 KB row per nonzero is the larger cost."""
+    import torch
+
+    def both(I, J, nnz, seed):
+        w = configs.make_spmm_gemm("order-%d" % J, seed, I, J, nnz, 256, 64)
+        t = sa.SparseTensor(w.dims, w.coords, w.vals, sa.SA_FMT_CSR, device=0)
+        ops = [torch.from_numpy(x).cuda() for x in w.dense]
+        desc = [(x.data_ptr(), x.shape[0], x.shape[1], x.stride(0)) for x in ops]
+        chosen = sa.sa_schedule_cost(t.handle, sa.SA_EXPR_SPMM_GEMM, sa.SA_SCHED_DEFAULT, desc)["resolved"]
+        ms = {}
+        for s in (sa.SA_SCHED_ASSOC_LEFT, sa.SA_SCHED_ASSOC_RIGHT):
+            out, _ = t.run(w.expr, ops, sched=s)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(10):
+                t.run(w.expr, ops, out=out, sched=s)
+            e1.record()
+            torch.cuda.synchronize()
+            ms[s] = e0.elapsed_time(e1) / 10
+        # the default really runs the chosen order (same launches, same result)
+        a, _ = t.run(w.expr, ops, sched=sa.SA_SCHED_DEFAULT)
+        b, _ = t.run(w.expr, ops, sched=chosen)
+        torch.cuda.synchronize()
+        assert torch.equal(a, b)
+        t.close()
+        return chosen, ms
+
+    chosen, ms = both(5_000, 2_000_000, 200_000, 61)
+    assert chosen == sa.SA_SCHED_ASSOC_LEFT and ms[sa.SA_SCHED_ASSOC_LEFT] < ms[sa.SA_SCHED_ASSOC_RIGHT], ms
+    chosen, ms = both(20_000, 400_000, 1_500_000, 62)
+    assert chosen == sa.SA_SCHED_ASSOC_RIGHT and ms[sa.SA_SCHED_ASSOC_RIGHT] < ms[sa.SA_SCHED_ASSOC_LEFT], ms
