@@ -82,10 +82,12 @@ def algorithmic_work(w, counts, sched):
         L, M = w.dense[0].shape[1], w.dense[1].shape[1]
         return 8 * nnz + 8 * F2 + 8 * S + sz(w.dense[0]) + sz(w.dense[1]) + out_bytes, 2 * nnz * M + 2 * F2 * L * M
     if w.expr == "ttmc3":
-        # the slice temporaries T(i,m,n) are an artefact of the fissioned i loop and are not counted
+        # fused over i: nothing but the streams, the factors and the output; fissioned: the slice temporaries
+        # T(i,m,n) are written and read once
         S, F2 = int(counts[0]), int(counts[1])
         L, M, N = (d.shape[1] for d in w.dense)
-        return (8 * nnz + 8 * F2 + 8 * S + sum(sz(d) for d in w.dense) + out_bytes,
+        temp = 8 * w.dims[0] * M * N if sched == "fissioned" else 0
+        return (8 * nnz + 8 * F2 + 8 * S + sum(sz(d) for d in w.dense) + out_bytes + temp,
                 2 * nnz * N + 2 * F2 * M * N + 2 * w.dims[0] * L * M * N)
     if w.expr == "spttm_ttm4":
         S, F2, F3 = int(counts[0]), int(counts[1]), int(counts[2])
@@ -326,8 +328,9 @@ def workload_label(cfg, sched):
              6: "kernel 5 <3D TTMC> on a nell-2-shaped tensor 12000x9000x288000 76.88M nnz L=M=N=16",
              8: "kernel 3 <SpMMH,GEMM> on the config-4 tensor recipe 4Mx4M 100M nnz L=256 M=64",
              9: "kernel 8 <MTTKRP,GEMM> on the config-2 tensor, R=32 M=32",
-             10: "kernel 7 <SpTTM,SpTTM> on the config-2 tensor, L=M=32, sparse output (one row per (i,j) fiber)"}
-    return names[cfg] + (" (%s)" % sched if cfg in (4, 10) else "")
+             10: "kernel 7 <SpTTM,SpTTM> on the config-2 tensor, L=M=32, sparse output (one row per (i,j) fiber)",
+             11: "kernel 5 <3D TTMC> on a flickr-3d-shaped tensor 320000x2820000x1600000 112.89M nnz L=M=N=16"}
+    return names[cfg] + (" (%s)" % sched if cfg in (4, 10) or (cfg in (6, 11) and sched == "fissioned") else "")
 
 
 def label(args):
@@ -367,7 +370,7 @@ def measure(sa, torch, dist, w, sched_name, steps, warmup, e2e_steps, dev, rank,
     build_s = time.perf_counter() - t0
     nnz, counts, n_chunks = tensor.info()
     sched = {"left": sa.SA_SCHED_ASSOC_LEFT, "right": sa.SA_SCHED_ASSOC_RIGHT, "default": sa.SA_SCHED_DEFAULT,
-             "fused": sa.SA_SCHED_DEFAULT}[sched_name]
+             "fused": sa.SA_SCHED_DEFAULT, "fissioned": sa.SA_SCHED_FISSIONED}[sched_name]
     host_ops = [torch.from_numpy(np.ascontiguousarray(x)).pin_memory() for x in w.dense]
     ops = [x.to(dev, non_blocking=False) for x in host_ops]
     out = torch.empty(w.out_shape, dtype=torch.float32, device=dev)
@@ -438,7 +441,7 @@ def measure(sa, torch, dist, w, sched_name, steps, warmup, e2e_steps, dev, rank,
             ws = {k: sa.sa_workspace_size(tensor.handle, sa._EXPR_OF[w.expr], v, ops_desc)
                   for k, v in (("default", sa.SA_SCHED_DEFAULT), ("left", sa.SA_SCHED_ASSOC_LEFT), ("right", sa.SA_SCHED_ASSOC_RIGHT))}
             ran = "left" if ws["default"] == ws["left"] and ws["left"] != ws["right"] else "right"
-        abytes, aflops = algorithmic_work(w, counts, ran if w.expr in ("spmm_gemm", "spttm_spttm") else "fused")
+        abytes, aflops = algorithmic_work(w, counts, ran if w.expr in ("spmm_gemm", "spttm_spttm", "ttmc3") else "fused")
         achieved = abytes / (ms_per_step * 1e-3) / 1e9
         traffic, traffic_kernel = ncu_traffic(workload_id, ran) if scale == "full" else (None, None)
         rec = {
@@ -480,10 +483,11 @@ def main():
     ap.add_argument("--steps", type=int, default=31)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", type=int, default=None, choices=[1, 2, 3, 4, 5, 6, 7, 8, 9, 10],
+    ap.add_argument("--workload", type=int, default=None, choices=[1, 2, 3, 4, 5, 6, 7, 8, 9, 10, 11],
                     help="one workload only; without it: config 2 as the headline plus a per_config list of all five configs")
     ap.add_argument("--scale", default="full", choices=["full", "mid", "mini"])
-    ap.add_argument("--sched", default="right", choices=["left", "right", "default"], help="association order for workloads 4 and 10")
+    ap.add_argument("--sched", default="right", choices=["left", "right", "default", "fissioned"],
+                    help="association order for workloads 4 and 10; 'fissioned' selects the second schedule of workload 6")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-per-config", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=5)
@@ -526,6 +530,8 @@ def main():
 
     w = configs.make(args.workload, args.scale)
     sched_name = args.sched if w.expr in ("spmm_gemm", "spttm_spttm") else "fused"
+    if w.expr == "ttmc3" and args.sched == "fissioned":
+        sched_name = "fissioned"
     rec = measure(sa, torch, dist, w, sched_name, args.steps, args.warmup, args.e2e_steps, dev, rank, world,
                   gather_probe=True, scale=args.scale, workload_id=args.workload)
     if rank == 0:

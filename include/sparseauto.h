@@ -63,7 +63,10 @@ typedef enum {
     /* kernel 4 <SpMM,GEMM>:  A(i,m) = sum_{j,l} B(i,j) C(j,l) D(l,m); ops = {C, D}             */
     SA_EXPR_SPMM_GEMM = 4,
     /* kernel 5 <3D TTMC>:    A(l,m,n) = sum_{i,j,k} B(i,j,k) C(i,l) D(j,m) E(k,n); ops = {C, D, E};
-     * B order-3 CSF; the slice temporaries T(i,m,n) live in the workspace                      */
+     * B order-3 CSF.  SA_SCHED_FUSED (L M N <= 8192): the slice temporaries T(i; m,n) stay on chip,
+     * every thread block accumulates into its own L x M x N tile; SA_SCHED_FISSIONED: they pass
+     * through the workspace (faster on this device: more resident warps); SA_SCHED_DEFAULT: fissioned
+     * unless its workspace is above the auxiliary-memory cap and the fused one's is not          */
     SA_EXPR_TTMC3 = 5,
     /* kernel 2 <SDDMM,SpMM,GEMM>: A(i,m) = sum_{j,k,l} B(i,j) C(i,k) D(j,k) E(j,l) F(l,m);
      * ops = {C, D, E, F}; B CSR; two-level schedule with the row temporary T(l) in the workspace */
@@ -93,6 +96,9 @@ typedef enum {
     SA_SCHED_FUSED = 1,        /* the fissioned / fused branched nest of the Table of kernels   */
     SA_SCHED_ASSOC_LEFT = 2,   /* SA_EXPR_SPMM_GEMM (and SPTTM_SPTTM): (B.C).D, row temporary of L floats    */
     SA_SCHED_ASSOC_RIGHT = 3,  /* SA_EXPR_SPMM_GEMM (and SPTTM_SPTTM): B.(C.D), J x M temporary in workspace */
+    SA_SCHED_FISSIONED = 4,    /* SA_EXPR_TTMC3: the loop over i fissioned from the l loop, the slice temporaries
+                                  T(i,m,n) in the workspace; bitwise reproducible (SA_SCHED_FUSED is not: its
+                                  block accumulators take shared-memory atomic adds)              */
     SA_SCHED_DEBUG_MATERIALIZE = 9 /* SA_EXPR_SDDMM_SPMM only, for tests: additionally writes the
                                       sampled values B(i,j) * sum_k C(i,k) D(j,k), aligned with
                                       the exported last-level crd array, to the workspace       */

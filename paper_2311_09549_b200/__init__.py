@@ -26,7 +26,7 @@ SA_OK = 0
 SA_FMT_CSR, SA_FMT_CSF = 1, 2
 SA_EXPR_SPTTM_TTM3, SA_EXPR_SPTTM_TTM4, SA_EXPR_SDDMM_SPMM, SA_EXPR_SPMM_GEMM, SA_EXPR_TTMC3, SA_EXPR_SDDMM_SPMM_GEMM = 1, 2, 3, 4, 5, 6
 SA_EXPR_SPMMH_GEMM, SA_EXPR_MTTKRP_GEMM, SA_EXPR_SPTTM_SPTTM = 7, 8, 9
-SA_SCHED_DEFAULT, SA_SCHED_FUSED, SA_SCHED_ASSOC_LEFT, SA_SCHED_ASSOC_RIGHT = 0, 1, 2, 3
+SA_SCHED_DEFAULT, SA_SCHED_FUSED, SA_SCHED_ASSOC_LEFT, SA_SCHED_ASSOC_RIGHT, SA_SCHED_FISSIONED = 0, 1, 2, 3, 4
 SA_SCHED_DEBUG_MATERIALIZE = 9
 
 EXPORTED_SYMBOLS = ["sa_tensor_create", "sa_tensor_info", "sa_tensor_export", "sa_tensor_worklist",

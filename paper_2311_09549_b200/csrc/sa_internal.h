@@ -178,9 +178,14 @@ sa_status sa_launch_spmmh_gemm(const sa_tensor *t, const sa_dense *ops, float *o
                                cudaStream_t stream, int *launches);
 size_t sa_ws_spmmh_gemm(const sa_tensor *t, const sa_dense *ops);
 
-sa_status sa_launch_ttmc3(const sa_tensor *t, const sa_dense *ops, float *out, void *ws, size_t ws_bytes,
+sa_status sa_launch_ttmc3(const sa_tensor *t, const sa_dense *ops, float *out, void *ws, size_t ws_bytes, bool fissioned,
                           cudaStream_t stream, int *launches);
-size_t sa_ws_ttmc3(const sa_tensor *t, const sa_dense *ops);
+size_t sa_ws_ttmc3(const sa_tensor *t, const sa_dense *ops, bool fissioned);
+// Kernel 5 with the loop over i kept fused (sa_ttm3.cu): available while the block accumulator fits shared memory
+bool sa_ttmc3_fused_ok(int64_t L3, int64_t M, int64_t N);
+size_t sa_ws_ttmc3_fused(int64_t L3, int64_t M, int64_t N);
+sa_status sa_launch_ttmc3_fused_stage(const sa_tensor *t, const sa_dense &C3, const sa_dense &D, const sa_dense &E, float *partials,
+                                      cudaStream_t stream, int *n_blocks);
 
 // Kernel 2 <SDDMM,SpMM,GEMM>: the fused SDDMM->SpMM kernel into a row temporary, then the dense stage.
 sa_status sa_launch_sddmm_spmm_gemm(const sa_tensor *t, const sa_dense *ops, float *out, void *ws, size_t ws_bytes,

@@ -14,6 +14,7 @@
 // A(i,:,:) += Cg^T (L x 8) . T (8 x M) with m16n8k8 TF32 MMAs, each operand split into a high and a low
 // TF32 part (three products), which keeps fp32-level accuracy.  The order-3 intermediate T(i,j,m) is
 // never stored.
+#include <algorithm>
 #include <type_traits>
 
 #include "sa_device.cuh"
@@ -209,14 +210,46 @@ __device__ __forceinline__ stream_range stream_of(int p0, int p1, int q)
 // One warp evaluates the units [u0, u0 + nu) of its task.  `keep`: the (single) unit is a piece of a slice
 // whose tile the caller reduces over the CTA, so it is left in acc; otherwise every unit is a whole slice
 // and its tile is stored to `out` when the unit ends.
-template <int L, int M, bool HAD>
+// What kernel 5 adds at the end of a unit (TTMC = true): the slice temporary T(i; m,n) in `acc` is not stored but
+// contracted with C(i,:) into the block's accumulator of the whole output, accs[l][m][n] += C(i,l) T(i; m,n).
+struct ttmc_sink {
+    const float *C3;        // C of kernel 5 (rows by i)
+    uint32_t ldc3;
+    int L3;                 // its columns
+    float *accs;            // shared memory, L3 x L x M floats
+};
+
+// Several warps of a block add to the same accumulator at unrelated times: shared-memory atomic adds.
+template <int L, int M>
+__device__ __forceinline__ void ttmc_accumulate(const float (&acc)[cfg<L, M>::MT][cfg<L, M>::NT][4], const ttmc_sink &sk, int row, int lane)
+{
+    using K = cfg<L, M>;
+    const int g = lane >> 2, t = lane & 3;
+    const float *crow = sk.C3 + uint32_t(row) * sk.ldc3;
+    for (int l = 0; l < sk.L3; ++l) {
+        const float c = __ldg(crow + l);
+        float *base = sk.accs + l * (L * M) + g * M + 2 * t;
+#pragma unroll
+        for (int mt = 0; mt < K::MT; ++mt)
+#pragma unroll
+            for (int nt = 0; nt < K::NT; ++nt) {
+                float *p = base + (16 * mt) * M + 8 * nt;
+                atomicAdd(p, c * acc[mt][nt][0]);
+                atomicAdd(p + 1, c * acc[mt][nt][1]);
+                atomicAdd(p + 8 * M, c * acc[mt][nt][2]);
+                atomicAdd(p + 8 * M + 1, c * acc[mt][nt][3]);
+            }
+    }
+}
+
+template <int L, int M, bool HAD, bool TTMC = false>
 __device__ __forceinline__ void ttm3_warp_task(const sa_unit3 *__restrict__ units, int u0, int nu,
                                                const int32_t *__restrict__ crd_j, const int32_t *__restrict__ crd_k,
                                                const float *__restrict__ vals, const uint32_t *__restrict__ endbits,
                                                const float *__restrict__ C, uint32_t ldc, const float *__restrict__ D,
                                                uint32_t ldd, unsigned char *__restrict__ wsm,
                                                float (&acc)[cfg<L, M>::MT][cfg<L, M>::NT][4], float &hacc, const bool keep,
-                                               float *__restrict__ out, const dbg_limits &lim)
+                                               float *__restrict__ out, const dbg_limits &lim, const ttmc_sink *sink = nullptr)
 {
     using K = cfg<L, M>;
     constexpr int VEC = K::VEC, DEPTH = K::DEPTH;
@@ -410,6 +443,9 @@ __device__ __forceinline__ void ttm3_warp_task(const sa_unit3 *__restrict__ unit
                 if (M == 16) hacc += __shfl_xor_sync(SA_FULL_MASK, hacc, 16);
                 if (lane < M && SA_CHK(lim.status, uint32_t(crow) < lim.n_slices_dim, 8, crow)) sa_st_cs(out + int64_t(crow) * M + lane, hacc);
                 hacc = 0.f;
+            } else if (TTMC) {
+                if (SA_CHK(lim.status, uint32_t(crow) < lim.n_slices_dim, 8, crow)) ttmc_accumulate<L, M>(acc, *sink, crow, lane);
+                zero_tile<L, M>(acc);
             } else {
                 if (SA_CHK(lim.status, uint32_t(crow) < lim.n_slices_dim, 8, crow)) store_tile<L, M>(acc, out + int64_t(crow) * (L * M), lane);
                 zero_tile<L, M>(acc);
@@ -499,6 +535,85 @@ ttm3_kernel(const sa_unit3 *__restrict__ units, const int32_t *__restrict__ task
     }
 }
 
+// Kernel 5 with the loop over i kept fused (second schedule of the 3-D TTMC row of the Table of kernels, the slice
+// temporary never leaving the chip): the slice stage of kernel 6 with (D, E) as factors, whose finished temporaries
+// T(i; m,n) are contracted with C(i,:) into an L3 x L x M accumulator in the block's shared memory.  Blocks are
+// persistent (block b takes the block-tasks b, b + grid, ...: chunks of large slices first, then tasks of small
+// slices) and write their accumulators to `partials` (grid x L3 x L x M), which a second kernel adds in block order.
+// Nothing is needed for split slices: the contraction is linear, every chunk adds its share.
+template <int L, int M, int NCTA>
+__global__ void __launch_bounds__(32 * SA_TTM3_WARPS, NCTA)
+ttmc3_fused_kernel(const sa_unit3 *__restrict__ units, const int32_t *__restrict__ task_start, int64_t n_tasks, int n_group_ctas,
+                   const int32_t *__restrict__ crd_j, const int32_t *__restrict__ crd_k, const float *__restrict__ vals,
+                   const uint32_t *__restrict__ endbits, const float *__restrict__ C, uint32_t ldc,
+                   const float *__restrict__ D, uint32_t ldd, const float *__restrict__ C3, uint32_t ldc3, int L3,
+                   float *__restrict__ partials, const dbg_limits lim)
+{
+    using K = cfg<L, M>;
+    constexpr int TILE = L * M;
+    extern __shared__ __align__(16) unsigned char smem[];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int g = lane >> 2, t = lane & 3;
+    unsigned char *wsm = smem + warp * K::WARP_BYTES;
+    float *accs = reinterpret_cast<float *>(smem + SA_TTM3_WARPS * K::WARP_BYTES);
+    const int n_acc = L3 * TILE;
+    for (int x = threadIdx.x; x < n_acc; x += 32 * SA_TTM3_WARPS) accs[x] = 0.f;
+    __syncthreads();
+    ttmc_sink sink;
+    sink.C3 = C3; sink.ldc3 = ldc3; sink.L3 = L3; sink.accs = accs;
+    const int64_t n_block_tasks = (n_tasks + SA_TTM3_WARPS - 1) / SA_TTM3_WARPS;
+    for (int64_t bt = blockIdx.x; bt < n_block_tasks; bt += gridDim.x) {
+        const int64_t task = bt * SA_TTM3_WARPS + warp;
+        const bool group = bt < n_group_ctas;          // the same for all warps of the block
+        float acc[K::MT][K::NT][4];
+        float hacc = 0.f;
+        zero_tile<L, M>(acc);
+        int u0 = 0, u1 = 0;
+        if (task < n_tasks) { u0 = task_start[task]; u1 = task_start[task + 1]; }
+        if (u1 > u0)
+            ttm3_warp_task<L, M, false, true>(units, u0, u1 - u0, crd_j, crd_k, vals, endbits, C, ldc, D, ldd, wsm, acc, hacc, group,
+                                              nullptr, lim, &sink);
+        if (!group) continue;              // whole small slices: added to the accumulator when their units ended
+        // the block's warps hold partial temporaries of the same slice: sum them, then one rank-1 update
+        __syncthreads();                   // every warp is done with its shared-memory region
+        float *wt = reinterpret_cast<float *>(wsm);
+#pragma unroll
+        for (int mt = 0; mt < K::MT; ++mt)
+#pragma unroll
+            for (int nt = 0; nt < K::NT; ++nt) {
+                const int l = 16 * mt + g, mm = 8 * nt + 2 * t;
+                *reinterpret_cast<float2 *>(wt + l * K::RS + mm) = make_float2(acc[mt][nt][0], acc[mt][nt][1]);
+                *reinterpret_cast<float2 *>(wt + (l + 8) * K::RS + mm) = make_float2(acc[mt][nt][2], acc[mt][nt][3]);
+            }
+        __syncthreads();
+        const int row = units[task_start[bt * SA_TTM3_WARPS]].out_row;       // warp 0 always has a unit
+        const float *all = reinterpret_cast<const float *>(smem);
+        if (SA_CHK(lim.status, uint32_t(row) < lim.n_slices_dim, 8, row)) {
+            const float *crow = C3 + uint32_t(row) * ldc3;
+            for (int x = threadIdx.x * 4; x < TILE; x += 32 * SA_TTM3_WARPS * 4) {
+                const int off = (x / M) * K::RS + (x % M);
+                float4 s = *reinterpret_cast<const float4 *>(all + off);
+#pragma unroll
+                for (int w = 1; w < SA_TTM3_WARPS; ++w) {
+                    const float4 v = *reinterpret_cast<const float4 *>(all + w * (K::WARP_BYTES / 4) + off);
+                    s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+                }
+                for (int l = 0; l < L3; ++l) {          // no other warp touches the accumulator during a chunk
+                    const float c = __ldg(crow + l);
+                    float4 *a = reinterpret_cast<float4 *>(accs + l * TILE + x);
+                    float4 o = *a;
+                    o.x = fmaf(c, s.x, o.x); o.y = fmaf(c, s.y, o.y); o.z = fmaf(c, s.z, o.z); o.w = fmaf(c, s.w, o.w);
+                    *a = o;
+                }
+            }
+        }
+        __syncthreads();                   // the next block-task reuses the warps' regions
+    }
+    __syncthreads();
+    float *dst = partials + int64_t(blockIdx.x) * n_acc;
+    for (int x = threadIdx.x; x < n_acc; x += 32 * SA_TTM3_WARPS) dst[x] = accs[x];
+}
+
 template <int L, int M, bool HAD>
 cudaError_t launch(const sa_ttm3_view &v, const sa_dense &first, const sa_dense &second, float *out, float *partial,
                    cudaStream_t stream)
@@ -570,6 +685,67 @@ sa_status sa_launch_ttm3(const sa_tensor *t, const sa_dense *ops, float *out, vo
     v.nnz_total = t->nnz;
     v.status = t->d_status;
     return sa_launch_ttm3_view(v, ops[0], ops[1], out, static_cast<float *>(ws), stream, launches);
+}
+
+// Kernel 5, fused over i: grid size and shared memory of ttmc3_fused_kernel for temporaries of M x N and L3 columns of C.
+template <int L, int M>
+static bool ttmc3_fused_shape(int L3, int *grid, size_t *smem_bytes)
+{
+    const size_t smem = size_t(SA_TTM3_WARPS) * cfg<L, M>::WARP_BYTES + size_t(L3) * L * M * sizeof(float);
+    auto kern = ttmc3_fused_kernel<L, M, 4>;
+    int dev = 0, sms = 148, per_sm = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess ||
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, 32 * SA_TTM3_WARPS, smem) != cudaSuccess || per_sm < 1) {
+        cudaGetLastError();
+        return false;
+    }
+    *grid = sms * per_sm;
+    *smem_bytes = smem;
+    return true;
+}
+
+// Accumulator elements the fused schedule of kernel 5 keeps per block; beyond this only the fissioned schedule runs.
+constexpr int64_t SA_TTMC3_FUSED_MAX = 8192;
+// Upper bound on the blocks of the fused schedule (sizes the workspace without asking the device).
+constexpr int SA_TTMC3_MAX_BLOCKS = 148 * 6 * 2;
+
+bool sa_ttmc3_fused_ok(int64_t L3, int64_t M, int64_t N) { return L3 * M * N <= SA_TTMC3_FUSED_MAX; }
+size_t sa_ws_ttmc3_fused(int64_t L3, int64_t M, int64_t N) { return sa_align256(size_t(SA_TTMC3_MAX_BLOCKS) * size_t(L3 * M * N) * sizeof(float)); }
+
+// Launches ttmc3_fused_kernel; *n_blocks receives the number of partial accumulators written to `partials`.
+sa_status sa_launch_ttmc3_fused_stage(const sa_tensor *t, const sa_dense &C3, const sa_dense &D, const sa_dense &E, float *partials,
+                                      cudaStream_t stream, int *n_blocks)
+{
+    const int64_t M = D.cols, N = E.cols;
+    if (D.rows * D.ld >= (int64_t(1) << 30) || E.rows * E.ld >= (int64_t(1) << 30) || C3.rows * C3.ld >= (int64_t(1) << 30)) return SA_E_UNSUPPORTED;
+    if (!t->d_endbits || !sa_ttmc3_fused_ok(C3.cols, M, N)) return SA_E_UNSUPPORTED;
+    const sa_worklist &wl = t->wl_main;
+    const int64_t n_tasks = int64_t(wl.task_start.size()) - 1;
+    const int64_t n_block_tasks = (n_tasks + SA_TTM3_WARPS - 1) / SA_TTM3_WARPS;
+    *n_blocks = 0;
+    if (n_block_tasks <= 0) return SA_OK;
+    dbg_limits lim;
+    lim.status = t->d_status;
+    lim.c_rows = uint32_t(D.rows); lim.d_rows = uint32_t(E.rows);
+    lim.n_fibers = uint32_t(t->count[1]); lim.n_slices_dim = uint32_t(t->dims[0]);
+    lim.nnz = t->nnz;
+    int grid = 0;
+    size_t smem = 0;
+#define SA_TTMC_CASE(m, n)                                                                                                        \
+    if (M == m && N == n) {                                                                                                       \
+        if (!ttmc3_fused_shape<m, n>(int(C3.cols), &grid, &smem)) return SA_E_CUDA;                                               \
+        grid = int(std::min<int64_t>(std::min<int64_t>(grid, SA_TTMC3_MAX_BLOCKS), n_block_tasks));                               \
+        ttmc3_fused_kernel<m, n, 4><<<unsigned(grid), 32 * SA_TTM3_WARPS, smem, stream>>>(                                        \
+            wl.d_units3, wl.d_task_start, n_tasks, int(wl.n_group_ctas), t->d_crd[1], t->d_crd[2], t->d_vals, t->d_endbits, D.ptr, \
+            uint32_t(D.ld), E.ptr, uint32_t(E.ld), C3.ptr, uint32_t(C3.ld), int(C3.cols), partials, lim);                         \
+        if (cudaGetLastError() != cudaSuccess) return SA_E_CUDA;                                                                  \
+        *n_blocks = grid;                                                                                                         \
+        return SA_OK;                                                                                                             \
+    }
+    SA_TTMC_CASE(16, 16) SA_TTMC_CASE(16, 32) SA_TTMC_CASE(32, 16)
+#undef SA_TTMC_CASE
+    return SA_E_UNSUPPORTED;
 }
 
 // Kernel 8, first stage (MTTKRP): T(i,r) = sum_{j,k} B(i,j,k) C(j,r) D(k,r), R = 32 or 16 columns, one row of R

@@ -2,11 +2,19 @@
 // the paper, Sections 1 and 3; chosen schedules in the Table of kernels, Section 6).  Evaluated as
 //   T(i,m,n) = sum_j D(j,m) ( sum_k B(i,j,k) E(k,n) )        per slice, the branched nest of kernel 6
 //   A(l,m,n) = sum_i C(i,l) T(i,m,n)                         contraction over the slices
-// i.e. the inner two levels are the paper's second schedule for this kernel (scalar-per-lane t, then
-// the temporary over m), while the loop over i is fissioned from the l loop: the slice temporaries
-// T(i,:,:) (I x M x N floats, in the workspace) are written by the slice kernel and reduced over i
-// by a small dense kernel, instead of every slice updating the shared L x M x N output.  The second
-// stage is deterministic: fixed chunks of slices, partial sums added in chunk order.
+// in two schedules:
+//   SA_SCHED_FUSED      the paper's second schedule for this kernel with its temporaries widened to
+//     vectors: i < T(m,n) ; j' < t(n) ; k': t += B E , m: T += t D > , l: A += T C >.  The slice
+//     temporary stays on chip; every thread block keeps its own L x M x N accumulator in shared
+//     memory (sa_ttm3.cu, ttmc3_fused_kernel) and the blocks' accumulators are added in block order.
+//     Additions inside a block are shared-memory atomics: their order, and with it the last bits of
+//     the result, may differ from run to run.
+//   SA_SCHED_FISSIONED  the loop over i is fissioned from the l loop: the slice temporaries T(i,:,:)
+//     (I x M x N floats, in the workspace) are written by the slice kernel of kernel 6 and reduced
+//     over i by a small dense kernel (fixed chunks of slices, partial sums added in chunk order:
+//     bitwise reproducible).  A temporary of three dimensions is what Stage 1 of the paper's
+//     auto-scheduler prunes; it is kept as the reproducible alternative and for rank combinations
+//     whose accumulator does not fit shared memory.
 #include <algorithm>
 
 #include "sa_device.cuh"
@@ -77,20 +85,34 @@ ttmc3_plan plan(const sa_tensor *t, const sa_dense *ops)
 
 bool sa_ranks_ok_ttmc3(int64_t L, int64_t M, int64_t N) { return (L == 16 || L == 32) && sa_ranks_ok_ttm3(M, N); }
 
-// workspace: [T: I x M x N][partial tiles of the slice kernel][P: chunks x L x M x N]
-size_t sa_ws_ttmc3(const sa_tensor *t, const sa_dense *ops)
+// workspace, fissioned: [T: I x M x N][partial tiles of the slice kernel][P: chunks x L x M x N]
+//            fused:     [accumulators of the blocks: blocks x L x M x N]
+size_t sa_ws_ttmc3(const sa_tensor *t, const sa_dense *ops, bool fissioned)
 {
+    if (!fissioned) return sa_ws_ttmc3_fused(ops[0].cols, ops[1].cols, ops[2].cols);
     const ttmc3_plan p = plan(t, ops);
     return p.t_bytes + p.ttm3_bytes + p.p_bytes;
 }
 
-sa_status sa_launch_ttmc3(const sa_tensor *t, const sa_dense *ops, float *out, void *ws, size_t, cudaStream_t stream,
-                          int *launches)
+sa_status sa_launch_ttmc3(const sa_tensor *t, const sa_dense *ops, float *out, void *ws, size_t, bool fissioned,
+                          cudaStream_t stream, int *launches)
 {
-    const ttmc3_plan p = plan(t, ops);
     const int64_t I = t->dims[0], L = ops[0].cols;
     const int cols = int(ops[1].cols * ops[2].cols);
     if (ops[0].rows * ops[0].ld >= (int64_t(1) << 30)) return SA_E_UNSUPPORTED;
+    if (!fissioned) {
+        float *partials = static_cast<float *>(ws);
+        int n_blocks = 0;
+        const sa_status s = sa_launch_ttmc3_fused_stage(t, ops[0], ops[1], ops[2], partials, stream, &n_blocks);
+        if (s != SA_OK) return s;
+        const int64_t n_out = L * cols;
+        // n_blocks == 0 (a tensor without nonzeros): the sum over no accumulators writes zeros
+        ttmc3_final_kernel<<<(unsigned)((n_out + 255) / 256), 256, 0, stream>>>(n_blocks, n_out, partials, out);
+        if (cudaGetLastError() != cudaSuccess) return SA_E_CUDA;
+        *launches = (n_blocks > 0 ? 1 : 0) + 1;
+        return SA_OK;
+    }
+    const ttmc3_plan p = plan(t, ops);
     char *base = static_cast<char *>(ws);
     float *T = reinterpret_cast<float *>(base);
     void *ws3 = base + p.t_bytes;

@@ -152,3 +152,24 @@ def test_default_schedule_takes_fewer_bytes_within_the_auxiliary_memory_cap():
     assert sa.sa_schedule_cost(dense.handle, E4, sa.SA_SCHED_ASSOC_RIGHT, ops)["resolved"] == sa.SA_SCHED_ASSOC_RIGHT
     sa.sa_tensor_set_aux_limit(dense.handle, 2**62)
     assert sa.sa_schedule_cost(dense.handle, E4, sa.SA_SCHED_DEFAULT, ops)["resolved"] == sa.SA_SCHED_ASSOC_RIGHT
+
+
+def test_kernel5_default_is_fissioned_until_its_temporaries_exceed_the_cap():
+    """Kernel 5: the fissioned schedule (slice temporaries I x M x N in the workspace) is the default; when the
+    caller caps auxiliary memory below that, the schedule with the temporaries on chip runs instead (Stage 4's
+    memory condition, Section 5.2; Stage 1 of the paper prunes temporaries of three dimensions altogether)."""
+    rs = np.random.RandomState(9)
+    I = 200_000
+    coords = np.unique(np.stack([rs.randint(0, I, 5000), rs.randint(0, 50, 5000), rs.randint(0, 60, 5000)], axis=1), axis=0).astype(np.int32)
+    t = sa.SparseTensor((I, 50, 60), coords, np.ones(len(coords), np.float32), sa.SA_FMT_CSF, device=-1)
+    ops = [(16, I, 16, 16), (16, 50, 16, 16), (16, 60, 16, 16)]
+    E5 = sa.SA_EXPR_TTMC3
+    fis = sa.sa_schedule_cost(t.handle, E5, sa.SA_SCHED_FISSIONED, ops)
+    fus = sa.sa_schedule_cost(t.handle, E5, sa.SA_SCHED_FUSED, ops)
+    assert fis["workspace_bytes"] >= I * 256 * 4 > fus["workspace_bytes"]
+    assert fis["temp_elements"] == 16 + I * 256 and fus["temp_elements"] == 16 + 256
+    assert fis["iterations"] == fus["iterations"] and fis["moved_bytes"] == fus["moved_bytes"] + 8 * I * 256
+    assert sa.sa_schedule_cost(t.handle, E5, sa.SA_SCHED_DEFAULT, ops)["resolved"] == sa.SA_SCHED_FISSIONED
+    sa.sa_tensor_set_aux_limit(t.handle, 100 << 20)
+    assert sa.sa_schedule_cost(t.handle, E5, sa.SA_SCHED_DEFAULT, ops)["resolved"] == sa.SA_SCHED_FUSED
+    assert sa.sa_workspace_size(t.handle, E5, sa.SA_SCHED_DEFAULT, ops) == fus["workspace_bytes"]

@@ -26,6 +26,37 @@ def test_ttm_chains_mini(sa, cfg):
     assert_close(A, A_ref, S_ref, TOL_FP32, w.name)
 
 
+@pytest.mark.parametrize("ranks", [(16, 16, 16), (32, 16, 16), (16, 32, 16), (16, 16, 32), (32, 32, 16)])
+def test_ttmc3_both_schedules(sa, ranks):
+    """Kernel 5 with the loop over i fused (block accumulators in shared memory) and fissioned (slice temporaries in
+    the workspace); the fused one exists while L M N <= 8192.  The tensor has slices split over several thread
+    blocks, whose chunks the fused schedule adds without a fix-up pass."""
+    L, M, N = ranks
+    w = configs.make_ttmc3_zipf("ttmc3-%d-%d-%d" % ranks, 77, 300, 200, 250, 60_000, 1.2, 8.0, L, M, N)
+    A_ref, S_ref = oracle.evaluate(w)
+    A, t = run_gpu(sa, w, sched=sa.SA_SCHED_FISSIONED)
+    assert_close(A, A_ref, S_ref, TOL_FP32, w.name + "/fissioned")
+    A2, _ = run_gpu(sa, w, sched=sa.SA_SCHED_FISSIONED, tensor=t)
+    assert np.array_equal(A, A2), "the fissioned schedule is bitwise reproducible"
+    ops = [(16, d.shape[0], d.shape[1], d.shape[1]) for d in w.dense]
+    if L * M * N <= 8192:
+        A, _ = run_gpu(sa, w, sched=sa.SA_SCHED_FUSED, tensor=t)
+        assert_close(A, A_ref, S_ref, TOL_FP32, w.name + "/fused")
+        c = sa.sa_schedule_cost(t.handle, sa.SA_EXPR_TTMC3, sa.SA_SCHED_FUSED, ops)
+        assert c["resolved"] == sa.SA_SCHED_FUSED and c["temp_elements"] == N + M * N
+        # the default is the fissioned schedule until its I x M x N temporary is above the caller's cap
+        assert sa.sa_schedule_cost(t.handle, sa.SA_EXPR_TTMC3, sa.SA_SCHED_DEFAULT, ops)["resolved"] == sa.SA_SCHED_FISSIONED
+        sa.sa_tensor_set_aux_limit(t.handle, 300 * M * N * 4 - 1)
+        assert sa.sa_schedule_cost(t.handle, sa.SA_EXPR_TTMC3, sa.SA_SCHED_DEFAULT, ops)["resolved"] == sa.SA_SCHED_FISSIONED, \
+            "neither fits: stay with the default"
+        sa.sa_tensor_set_aux_limit(t.handle, 2**62)
+    else:
+        with pytest.raises(sa.SaError) as e:
+            sa.sa_workspace_size(t.handle, sa.SA_EXPR_TTMC3, sa.SA_SCHED_FUSED, ops)
+        assert e.value.status == sa.SA_E_UNSUPPORTED
+        assert sa.sa_schedule_cost(t.handle, sa.SA_EXPR_TTMC3, sa.SA_SCHED_DEFAULT, ops)["resolved"] == sa.SA_SCHED_FISSIONED
+
+
 @pytest.mark.parametrize("cfg", [3, 7])
 def test_sddmm_spmm_mini(sa, cfg):
     w = configs.make(cfg, "mini")

@@ -385,6 +385,12 @@ def make(config, scale="full", seed=None):
         if full:
             return make_ttmc3_zipf("cfg6-ttmc3-nell2-shaped", s, 12_000, 9_000, 288_000, 76_880_000, 1.2, 8.0, 16, 16, 16)
         return make_ttmc3_zipf("cfg6-ttmc3-mini", s, 300, 200, 250, 60_000, 1.2, 8.0, 16, 16, 16)
+    if config == 11:
+        # kernel 5 on a tensor with the shape and size the paper quotes for flickr-3d: many more slices than
+        # nell-2, so the slice temporaries of the fissioned schedule (I x M x N floats) weigh as much as B itself
+        if full:
+            return make_ttmc3_zipf("cfg11-ttmc3-flickr-shaped", s, 320_000, 2_820_000, 1_600_000, 112_890_000, 1.2, 8.0, 16, 16, 16)
+        return make_ttmc3_zipf("cfg11-ttmc3-mini", s, 3000, 2000, 1500, 60_000, 1.2, 8.0, 16, 16, 16)
     if config == 7:
         # kernel 2 (SDDMM, SpMM, GEMM) on the tensor of config 3 with a 64 x 64 weight matrix F
         if full:
@@ -429,4 +435,4 @@ def make(config, scale="full", seed=None):
         f2 = int(np.unique(key).shape[0])
         return Workload("cfg10-spttm-spttm" + ("" if full else "-mini"), "spttm_spttm", "csf", w.dims, w.coords, w.vals,
                         [w.dense[1], D], (f2, 32), s, w.notes)
-    raise ValueError("config must be 1..10")
+    raise ValueError("config must be 1..11")
