@@ -54,9 +54,12 @@ typedef enum {
     /* kernel 6 <SpTTM,TTM>:  A(i,l,m) = sum_{j,k} B(i,j,k) C(j,l) D(k,m); ops = {C, D}          */
     SA_EXPR_SPTTM_TTM3 = 1,
     /* order-4 analogue:      A(i,l,m,n) = sum_{j,k,o} B(i,j,k,o) C(j,l) D(k,m) E(o,n);
-     * ops = {C, D, E}; the two-level nesting of kernel 5's second schedule in one fused kernel:
-     * the 16 x 16 temporaries T2(m,n) of the (i,j) subtrees stay in shared memory (only subtrees
-     * above 4096 nonzeros pass theirs through the workspace)                                    */
+     * ops = {C, D, E}; the two-level nesting of kernel 5's second schedule.  SA_SCHED_FUSED: one
+     * kernel, the 16 x 16 temporaries T2(m,n) of the (i,j) subtrees stay in shared memory (only
+     * subtrees above 4096 nonzeros pass theirs through the workspace).  SA_SCHED_FISSIONED: two
+     * passes with all temporaries in the workspace (1 KB per subtree), faster on this device while
+     * memory allows.  SA_SCHED_DEFAULT: fissioned unless its workspace is above the auxiliary-memory
+     * cap and the fused one's is not                                                             */
     SA_EXPR_SPTTM_TTM4 = 2,
     /* kernel 1 <SDDMM,SpMM>: A(i,l) = sum_j B(i,j) (sum_k C(i,k) D(j,k)) E(j,l); ops = {C,D,E}  */
     SA_EXPR_SDDMM_SPMM = 3,
@@ -96,9 +99,11 @@ typedef enum {
     SA_SCHED_FUSED = 1,        /* the fissioned / fused branched nest of the Table of kernels   */
     SA_SCHED_ASSOC_LEFT = 2,   /* SA_EXPR_SPMM_GEMM (and SPTTM_SPTTM): (B.C).D, row temporary of L floats    */
     SA_SCHED_ASSOC_RIGHT = 3,  /* SA_EXPR_SPMM_GEMM (and SPTTM_SPTTM): B.(C.D), J x M temporary in workspace */
-    SA_SCHED_FISSIONED = 4,    /* SA_EXPR_TTMC3: the loop over i fissioned from the l loop, the slice temporaries
-                                  T(i,m,n) in the workspace; bitwise reproducible (SA_SCHED_FUSED is not: its
-                                  block accumulators take shared-memory atomic adds)              */
+    SA_SCHED_FISSIONED = 4,    /* one more level of kernel fission: the temporaries of the outermost producer /
+                                  consumer pair pass through the workspace.  SA_EXPR_TTMC3: T(i,m,n) per slice
+                                  (bitwise reproducible, which SA_SCHED_FUSED is not there: its block
+                                  accumulators take shared-memory atomic adds); SA_EXPR_SPTTM_TTM4: T2(m,n) per
+                                  (i,j) subtree                                                    */
     SA_SCHED_DEBUG_MATERIALIZE = 9 /* SA_EXPR_SDDMM_SPMM only, for tests: additionally writes the
                                       sampled values B(i,j) * sum_k C(i,k) D(j,k), aligned with
                                       the exported last-level crd array, to the workspace       */
@@ -178,7 +183,12 @@ sa_status sa_tensor_export(const sa_tensor *t, int level, int64_t *pos, int32_t 
  *      the first slice or -1, of the last slice or -1, first subtree, one past the last; `fix` receives the
  *      super-items, 4 int32 each: first item, one past the last, first subtree, one past the last (at most 64
  *      subtrees).  counts = {pieces, subtrees above 4096 nonzeros, super-items, 0}.
- * For which = 0..2:
+ *   4, 5, 6  order-4 CSF, the lists of SA_SCHED_FISSIONED: 4 = like list 0 over the (i,j) subtrees with more than 64
+ *      level-2 fibers or 4096 nonzeros (out_row = index of the level-1 fiber); 5 = second pass, one item per (piece
+ *      of at most 512 level-1 fibers [f0,f1) of slice out_row, quarter of the 256 columns (m,n) in the last field),
+ *      with the fix-up entries of slices cut into pieces; 6 = first pass on whole small subtrees: rows
+ *      [out_row,row_end) = level-1 fibers, [f0,f1) their level-2 fibers (at most 64), [p0,p1) their nonzeros
+ * For which = 0..2 and 4..6:
  *   counts [4]: number of items, number of leading groups that one thread block reduces into a
  *               single tile (8 items each; order-3 tensors: 4 tasks each, see sa_tensor_tasks),
  *               number of fix-up entries, number of partial-tile slots

@@ -9,7 +9,7 @@ CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsparseauto.so")
 LIB_CHECKED = os.path.join(HERE, "libsparseauto_checked.so")
 LIB_WAITTEST = os.path.join(HERE, "libsparseauto_waittest.so")
-SOURCES = ["sa_api.cu", "sa_build.cu", "sa_ttm3.cu", "sa_ttm4.cu", "sa_sddmm_spmm.cu", "sa_spmm_gemm.cu", "sa_ttmc3.cu", "sa_mttkrp.cu", "sa_dense_tc.cu"]
+SOURCES = ["sa_api.cu", "sa_build.cu", "sa_ttm3.cu", "sa_ttm4.cu", "sa_ttm4_fis.cu", "sa_sddmm_spmm.cu", "sa_spmm_gemm.cu", "sa_ttmc3.cu", "sa_mttkrp.cu", "sa_dense_tc.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC,-fopenmp,-O3", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 

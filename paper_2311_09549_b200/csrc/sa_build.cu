@@ -288,6 +288,91 @@ void build_ttm3(sa_tensor *t, sa_worklist &wl)
 }
 
 
+// A subtree (i,j) that the subtree kernel of pass 1 can take whole.
+static bool subtree_is_small(const sa_tensor *t, int64_t f2)
+{
+    const auto &pos2 = t->pos[2], &pos3 = t->pos[3];
+    const int64_t fa = pos2[size_t(f2)], fb = pos2[size_t(f2) + 1];
+    return fb - fa <= SA_SUB_MAX_F3 && pos3[size_t(fb)] - pos3[size_t(fa)] <= SA_SUB_MAX_NNZ;
+}
+
+// Order-4 CSF, schedule SA_SCHED_FISSIONED: the chain is evaluated in two passes (see sa_ttm4_fis.cu).  Pass 1 runs the order-3 kernel with
+// the large (i,j) subtrees as slices: `wl` gets the same lists as an order-3 tensor whose slices are those
+// level-1 fibers (output row = fiber index); the small subtrees go to the subtree kernel's list.  Pass 2 contracts the per-fiber temporaries of each slice with rows of
+// C: `wl2` holds one item per (piece of a slice, quarter of the 256 temporaries' columns); a slice with more
+// than CHUNK_F fibers is cut into pieces whose partial tiles the fix-up kernel sums.
+void build_ttm4_fissioned(sa_tensor *t, sa_worklist &wl, sa_worklist &wl2)
+{
+    build_ttm3_lists(wl, t->count[1], [](int64_t f) { return int32_t(f); }, [&](int64_t f) { return subtree_is_small(t, f); },
+                     t->pos[2], t->pos[3]);
+    constexpr int64_t CHUNK_F = 512;
+    const auto &pos1 = t->pos[1];
+    std::vector<sa_item> items;
+    for (int64_t s = 0; s < t->count[0]; ++s) {
+        const int64_t fa = pos1[size_t(s)], fb = pos1[size_t(s) + 1];
+        const int32_t row = t->crd[0][size_t(s)];
+        const int64_t nc = (fb - fa + CHUNK_F - 1) / CHUNK_F;
+        int32_t slot0 = -1;
+        if (nc > 1) {
+            slot0 = int32_t(wl2.n_slots);
+            wl2.fix.push_back(sa_fix{row, slot0, int32_t(nc), 0});
+            wl2.n_slots += nc;
+        }
+        for (int64_t c = 0; c < nc; ++c)
+            for (int qc = 0; qc < 4; ++qc) {
+                sa_item it = empty_item();
+                it.out_row = row; it.row_end = row + 1;
+                it.f0 = int32_t(fa + c * CHUNK_F); it.f1 = int32_t(std::min(fb, fa + (c + 1) * CHUNK_F));
+                it.p0 = it.f0; it.p1 = it.f1;          // size key: fibers
+                it.dest = nc > 1 ? slot0 + int32_t(c) : -1;
+                it.pad = qc;
+                items.push_back(it);
+            }
+    }
+    // largest first: the tail of the launch is then made of the cheapest items
+    std::stable_sort(items.begin(), items.end(), [](const sa_item &a, const sa_item &b) { return (a.f1 - a.f0) > (b.f1 - b.f0); });
+    wl2.items = std::move(items);
+    wl2.n_group_ctas = 0;
+    append_empty_slices(t, wl2);
+}
+
+// Order 4, pass 1 on whole (i,j) subtrees: items are ranges of consecutive small subtrees (subtree_is_small) with
+// at most SA_SUB_MAX_F3 level-2 fibers, SA_SUB_MAX_ROWS subtrees and about 512 nonzeros (f0/f1 = the fibers,
+// p0/p1 = the nonzeros).  No subtree is cut, so there are no partial tiles; the large subtrees are in the main list.
+void build_ttm4_subtrees(sa_tensor *t, sa_worklist &wl)
+{
+    const auto &pos2 = t->pos[2], &pos3 = t->pos[3];
+    const int64_t F2 = t->count[1];
+    constexpr int64_t TARGET_NNZ = 512;
+    auto nnz_at = [&](int64_t f2) { return pos3[size_t(pos2[size_t(f2)])]; };
+    std::vector<sa_item> items;
+    int64_t r0 = 0;
+    auto flush = [&](int64_t r1) {
+        if (r1 > r0) {
+            sa_item it = empty_item();
+            it.out_row = int32_t(r0); it.row_end = int32_t(r1);
+            it.f0 = int32_t(pos2[size_t(r0)]); it.f1 = int32_t(pos2[size_t(r1)]);
+            it.p0 = int32_t(nnz_at(r0)); it.p1 = int32_t(nnz_at(r1));
+            items.push_back(it);
+        }
+        r0 = r1;
+    };
+    for (int64_t r = 0; r < F2; ++r) {
+        if (!subtree_is_small(t, r)) {
+            flush(r);
+            r0 = r + 1;
+            continue;
+        }
+        if (r > r0 && (pos2[size_t(r) + 1] - pos2[size_t(r0)] > SA_SUB_MAX_F3 || r - r0 >= SA_SUB_MAX_ROWS ||
+                       nnz_at(r + 1) - nnz_at(r0) > TARGET_NNZ))
+            flush(r);
+    }
+    flush(F2);
+    for (const sa_item &it : items) wl.nnz += it.p1 - it.p0;
+    wl.items = std::move(items);
+    wl.n_group_ctas = 0;
+}
+
 // Order-4 CSF (see sa_ttm4.cu).  The chain runs as one fused kernel over *pieces*: contiguous ranges of (i,j)
 // subtrees holding about PIECE_NNZ nonzeros, one thread block each.  A piece is a run of *super-items* (at most
 // SA_F4_POOL subtrees: what the block's pool of 16 x 16 temporaries holds), a super-item a run of *items* that
@@ -452,6 +537,9 @@ void sa_build_worklists(sa_tensor *t)
     }
     if (t->fmt == SA_FMT_CSF && t->order == 4) {
         build_ttm4(t, t->wl_main, t->wl_sub, t->wl_aux);
+        build_ttm4_fissioned(t, t->wl4_main, t->wl4_aux);
+        build_ttm4_subtrees(t, t->wl4_sub);
+        t->wl4_main.nnz = t->nnz - t->wl4_sub.nnz;
     }
     if (t->fmt == SA_FMT_CSR) {
         build_rows(t->pos[1], t->dims[0], t->wl_main, 256, 32, 1024, 512);    // fused SDDMM -> SpMM

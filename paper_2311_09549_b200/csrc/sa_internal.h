@@ -108,6 +108,10 @@ struct sa_tensor {
     sa_worklist wl_aux;                       // CSR: SpMM-GEMM row items; order-3 CSF: fiber rows (kernel 7); order-4 CSF: partial
                                               // slice tiles and fix-up entries of the fused kernel
     sa_worklist wl_sub;                       // order-4 CSF: items of the fused kernel (runs of (i,j) subtrees)
+    // order-4 CSF, schedule SA_SCHED_FISSIONED (sa_ttm4_fis.cu): order-3 lists over the (i,j) subtrees the subtree kernel
+    // does not take, pass-2 items (piece of a slice x quarter of the columns) with their fix-up entries, and ranges of
+    // whole small subtrees for the subtree kernel
+    sa_worklist wl4_main, wl4_aux, wl4_sub;
     // order-4 CSF: super-items (item0, item1, r0, r1) and pieces (sup0, sup1, first slice, last slice, destination of
     // the first slice, of the last slice, r0, r1) of the fused kernel, see build_ttm4; subtrees above SA_SUB_MAX_NNZ
     std::vector<int32_t> f4_supers, f4_pieces;
@@ -139,6 +143,10 @@ constexpr int SA_F4_POOL = SA_F4_POOL_N;
 constexpr int SA_F4_WARPS = SA_F4_WARPS_N;    // warps per thread block of the fused kernel
 constexpr int SA_F4_CTAS = SA_F4_CTAS_N;      // thread blocks per SM the fused kernel's register budget is set for
 constexpr int SA_SUB_MAX_NNZ = 4096;
+// Limits of the subtree kernel of the fissioned order-4 schedule: level-2 fibers an item parks in shared memory and
+// rows (subtrees) per item.
+constexpr int SA_SUB_MAX_F3 = 64;
+constexpr int SA_SUB_MAX_ROWS = 32;
 
 // ---- host builder (sa_build.cu)
 sa_status sa_build_levels(sa_tensor *t, const int32_t *coords, const float *vals);
@@ -167,6 +175,9 @@ size_t sa_ws_ttm3(const sa_tensor *t, const sa_dense *ops);
 sa_status sa_launch_ttm4(const sa_tensor *t, const sa_dense *ops, float *out, void *ws, size_t ws_bytes,
                          cudaStream_t stream, int *launches);
 size_t sa_ws_ttm4(const sa_tensor *t, const sa_dense *ops);
+sa_status sa_launch_ttm4_fissioned(const sa_tensor *t, const sa_dense *ops, float *out, void *ws, size_t ws_bytes,
+                                   cudaStream_t stream, int *launches);
+size_t sa_ws_ttm4_fissioned(const sa_tensor *t, const sa_dense *ops);
 sa_status sa_launch_sddmm_spmm(const sa_tensor *t, const sa_dense *ops, float *out, void *ws, size_t ws_bytes,
                                bool materialize, cudaStream_t stream, int *launches);
 size_t sa_ws_sddmm_spmm(const sa_tensor *t, const sa_dense *ops, bool materialize);

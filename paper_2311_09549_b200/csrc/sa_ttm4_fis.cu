@@ -1,0 +1,367 @@
+// Order-4 chain A(i,l,m,n) = sum_{j,k,o} B(i,j,k,o) C(j,l) D(k,m) E(o,n), schedule SA_SCHED_FISSIONED: the two-level
+// nest of sa_ttm4.cu with its outer producer/consumer pair fissioned at the j' loop,
+//   pass 1:  T2(f; m,n) = sum_{k,o} B(f; k,o) D(k,m) E(o,n)   for every level-1 fiber f = (i,j)   -> workspace
+//   pass 2:  A(i, l, (m,n)) = sum_{f in slice i} C(j_f, l) T2(f; (m,n))                              per slice
+// The temporaries T2 (1 KB per (i,j) subtree) are written and read once through HBM: about three times the bytes
+// of the fused schedule, and a workspace that grows with the tensor.  In exchange pass 1 needs neither a pool of
+// temporaries nor the slice accumulators in registers, keeps twice as many warps per SM resident, and the two
+// passes together are faster on the benchmark tensor; the default schedule takes it while the workspace fits the
+// caller's cap (sa_tensor_set_aux_limit).
+// Pass 1 is kernel 6 on the (i,j) subtrees: the small ones (at most 64 level-2 fibers and 4096 nonzeros) by the
+// subtree kernel below, the others by the order-3 kernel (sa_ttm3.cu) with the level-1 fibers as slices, D and E as
+// factors.  Pass 2 contracts, per slice, the temporaries with the rows C(j,:) on tensor cores.
+#include <algorithm>
+
+#include "sa_device.cuh"
+
+namespace {
+
+constexpr int R = 16;                  // L = M = N = 16
+constexpr int TILE4 = R * R * R;       // floats per output slice
+constexpr int T2F = R * R;             // floats per temporary
+constexpr int QC = 64;                 // temporary columns per item (a quarter)
+constexpr int NT4 = QC / 8;            // n8 tiles per item
+
+// Limits for the checks of the self-checking build (SA_CHK, sa_device.cuh).
+struct fis_limits {
+    int32_t *status;
+    uint32_t c_rows, d_rows, e_rows, n_slices;
+    int32_t n_subtrees, n_fibers, n_slots, nnz;
+};
+
+// Values one group of eight fibers contributes to a lane's MMA fragments: C(j,:) entries for the A operand
+// (fibers t and t + 4 of the group, columns g and g + 8) and T2 entries for the B operand (same two
+// fibers, column 8 nt + g of the item's quarter).  Fibers past the end of the item read as zero.
+struct group_vals {
+    float c[4];
+    float b[NT4][2];
+};
+
+__device__ __forceinline__ void load_group(group_vals &v, int f, int f1, int lane, const int32_t *__restrict__ crd_j,
+                                           const float *__restrict__ C, uint32_t ldc, const float *__restrict__ t2q,
+                                           const fis_limits &lim)
+{
+    const int g = lane >> 2, t = lane & 3;
+    const int fa = f + t, fb = f + t + 4;
+    const bool va = fa < f1, vb = fb < f1;
+    uint32_t ja = uint32_t(va ? __ldg(crd_j + fa) : 0), jb = uint32_t(vb ? __ldg(crd_j + fb) : 0);
+    if (!SA_CHK(lim.status, ja < lim.c_rows, 71, ja)) ja = 0u;
+    if (!SA_CHK(lim.status, jb < lim.c_rows, 71, jb)) jb = 0u;
+    const float *ca = C + ja * ldc + g;
+    const float *cb = C + jb * ldc + g;
+    v.c[0] = va ? __ldg(ca) : 0.f;
+    v.c[1] = va ? __ldg(ca + 8) : 0.f;
+    v.c[2] = vb ? __ldg(cb) : 0.f;
+    v.c[3] = vb ? __ldg(cb + 8) : 0.f;
+    const float *ra = t2q + int64_t(va ? fa : f) * T2F + g;
+    const float *rb = t2q + int64_t(vb ? fb : f) * T2F + g;
+#pragma unroll
+    for (int nt = 0; nt < NT4; ++nt) {
+        const float xa = __ldcs(ra + 8 * nt), xb = __ldcs(rb + 8 * nt);       // read once: streaming
+        v.b[nt][0] = va ? xa : 0.f;
+        v.b[nt][1] = vb ? xb : 0.f;
+    }
+}
+
+// Pass 2.  One warp per item (fibers [f0, f1) of one slice, quarter `pad` of the temporaries' columns);
+// warps take items in a grid-wide stride, largest items first.
+__global__ void __launch_bounds__(256, 2)
+ttm4_slice_kernel(const sa_item *__restrict__ items, int64_t n_items, const int32_t *__restrict__ crd_j,
+                  const float *__restrict__ T2, const float *__restrict__ C, uint32_t ldc, float *__restrict__ out,
+                  float *__restrict__ partial, const fis_limits lim)
+{
+    const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+    const int64_t stride = int64_t(gridDim.x) * SA_WARPS_PER_CTA;
+    for (int64_t n = int64_t(blockIdx.x) * SA_WARPS_PER_CTA + (threadIdx.x >> 5); n < n_items; n += stride) {
+        const int4 ia = __ldg(reinterpret_cast<const int4 *>(items + n));          // out_row, row_end, f0, f1
+        const int4 ib = __ldg(reinterpret_cast<const int4 *>(items + n) + 1);      // p0, p1, dest, quarter
+        const int f0 = ia.z, f1 = ia.w, qc = ib.w;
+        if (!SA_CHK(lim.status, f0 >= 0 && f0 <= f1 && f1 <= lim.n_subtrees && uint32_t(qc) < 4u && uint32_t(ia.x) < lim.n_slices &&
+                                    ib.z < lim.n_slots, 72, n))
+            continue;
+        const float *t2q = T2 + qc * QC;
+        float acc[NT4][4];
+#pragma unroll
+        for (int nt = 0; nt < NT4; ++nt)
+#pragma unroll
+            for (int x = 0; x < 4; ++x) acc[nt][x] = 0.f;
+        group_vals cur, nxt;
+        load_group(cur, f0, f1, lane, crd_j, C, ldc, t2q, lim);
+        nxt = cur;
+#pragma unroll 1
+        for (int f = f0; f < f1; f += 8) {
+            if (f + 8 < f1) load_group(nxt, f + 8, f1, lane, crd_j, C, ldc, t2q, lim);   // in flight during the products below
+            uint32_t ah[4], al[4];
+#pragma unroll
+            for (int x = 0; x < 4; ++x) split_tf32(cur.c[x], ah[x], al[x]);
+#pragma unroll
+            for (int nt = 0; nt < NT4; ++nt) {
+                uint32_t bh[2], bl[2];
+                split_tf32(cur.b[nt][0], bh[0], bl[0]);
+                split_tf32(cur.b[nt][1], bh[1], bl[1]);
+                mma_m16n8k8_tf32(acc[nt], al, bh);
+                mma_m16n8k8_tf32(acc[nt], ah, bl);
+                mma_m16n8k8_tf32(acc[nt], ah, bh);
+            }
+            cur = nxt;
+        }
+        // element (l, column 64 qc + 8 nt + 2 t (+1)) of the slice tile, l = g and g + 8
+        float *dst = (ib.z >= 0 ? partial + int64_t(ib.z) * TILE4 : out + int64_t(ia.x) * TILE4) + qc * QC + 2 * t;
+#pragma unroll
+        for (int nt = 0; nt < NT4; ++nt) {
+            const float2 lo = make_float2(acc[nt][0], acc[nt][1]), hi = make_float2(acc[nt][2], acc[nt][3]);
+            if (ib.z >= 0) {
+                *reinterpret_cast<float2 *>(dst + g * T2F + 8 * nt) = lo;
+                *reinterpret_cast<float2 *>(dst + (g + 8) * T2F + 8 * nt) = hi;
+            } else {
+                sa_st_cs2(dst + g * T2F + 8 * nt, lo);
+                sa_st_cs2(dst + (g + 8) * T2F + 8 * nt, hi);
+            }
+        }
+    }
+}
+
+// Pass 1 on whole (i,j) subtrees (tensors whose subtrees are all small: the usual case, a subtree holds a few
+// dozen nonzeros).  One warp per item = a range of consecutive subtrees with at most SA_SUB_MAX_F3 level-2 fibers.
+//   Phase A (Q1):  t(f; n) = sum_o B(f; o) E(o,n) for every level-2 fiber f = (i,j,k) of the item.  Four lanes own a
+//     row of E as one float4 each, so the warp's eight lane groups walk separate shares of the item's fibers, one
+//     nonzero per group and step (index/value pairs eight per load and one load ahead, eight row gathers in
+//     flight); the end-of-fiber bit travels in the sign bit of the index and parks t(f; :) in the fiber's own slot
+//     of the warp's shared-memory tile, so the parked rows end up in fiber order without any bookkeeping.
+//   Phase B (Q2):  T2(m,n) += D(k_f, m) t(f; n) over the fibers of each subtree, in order; the 16 x 16 tile is
+//     spread over the warp (lane = two rows m, four columns n), control flow is uniform, and the tile is stored
+//     (1 KB, contiguous) when the subtree's last fiber has been added.
+// Against the order-3 kernel on the same subtrees this drops the per-unit pipeline drains and the padded
+// tensor-core groups: 16.7 M outer products of 256 FMAs are cheap on the ALUs next to 100 M row gathers.
+constexpr int SUB_SMEM = SA_WARPS_PER_CTA * SA_SUB_MAX_F3 * R * int(sizeof(float));   // 32 KB
+
+// CONTIG: both factor matrices are stored without padding (leading dimension 16), so a row offset is a shift.
+template <bool CONTIG>
+__global__ void __launch_bounds__(256, 4)
+ttm4_subtree_kernel(const sa_item *__restrict__ items, int64_t n_items, const int32_t *__restrict__ pos2,
+                    const int32_t *__restrict__ pos3, const int32_t *__restrict__ crd_k, const int2 *__restrict__ nz,
+                    const float *__restrict__ D, int64_t ldd, const float *__restrict__ E, int64_t lde, float *__restrict__ T2,
+                    const fis_limits lim)
+{
+    extern __shared__ __align__(16) float sub_smem[];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t idx = int64_t(blockIdx.x) * SA_WARPS_PER_CTA + warp;
+    if (idx >= n_items) return;
+    const sa_item it = items[idx];
+    if (!SA_CHK(lim.status, it.f0 >= 0 && it.f1 - it.f0 <= SA_SUB_MAX_F3 && it.f1 <= lim.n_fibers && it.out_row >= 0 &&
+                                it.row_end - it.out_row <= SA_SUB_MAX_ROWS && it.row_end <= lim.n_subtrees && it.p0 >= 0 && it.p1 <= lim.nnz,
+                73, idx))
+        return;
+    float *pk = sub_smem + warp * (SA_SUB_MAX_F3 * R);
+    // row offsets in 32-bit arithmetic (the launcher checks rows * ld < 2^31)
+    const uint32_t ld_d = CONTIG ? uint32_t(R) : uint32_t(ldd), ld_e = CONTIG ? uint32_t(R) : uint32_t(lde);
+    const int nf3 = it.f1 - it.f0;
+    // rows of D the item's fibers need in phase B (requested now, used after phase A)
+    static_assert(SA_SUB_MAX_F3 <= 64, "two index registers per lane");
+    int kk0 = lane < nf3 ? __ldg(crd_k + it.f0 + lane) : 0;
+    int kk1 = lane + 32 < nf3 ? __ldg(crd_k + it.f0 + 32 + lane) : 0;
+    if (!SA_CHK(lim.status, uint32_t(kk0) < lim.d_rows && uint32_t(kk1) < lim.d_rows, 74, kk0)) kk0 = kk1 = 0;
+    {   // ---- phase A
+        const int g = lane >> 2, l = lane & 3;
+        // shares of the eight groups: whole fibers, cut where the nonzero count passes the next eighth of the item
+        // (fiber f belongs to the groups before g when it starts before p0 + g len / 8)
+        const int s0 = lane < nf3 ? __ldg(pos3 + it.f0 + lane) : 0x7fffffff;
+        const int s1 = lane + 32 < nf3 ? __ldg(pos3 + it.f0 + 32 + lane) : 0x7fffffff;
+        int fa = it.f0, fb = it.f1;
+#pragma unroll
+        for (int q = 1; q < 8; ++q) {
+            const int target = it.p0 + int(int64_t(it.p1 - it.p0) * q / 8);
+            const int cnt = __popc(__ballot_sync(SA_FULL_MASK, s0 < target)) + __popc(__ballot_sync(SA_FULL_MASK, s1 < target));
+            if (g == q) fa = it.f0 + cnt;
+            if (g + 1 == q) fb = it.f0 + cnt;
+        }
+        const int ga = __ldg(pos3 + fa), gb = __ldg(pos3 + fb);
+        const int mylen = gb - ga;
+        const int maxlen = __reduce_max_sync(SA_FULL_MASK, mylen);
+        int slot = fa - it.f0;
+        auto fetch1 = [&](int q, int &x, float &v) {
+            x = 0;
+            v = 0.f;
+            if (q < mylen && SA_CHK(lim.status, ga + q >= 0 && ga + q < lim.nnz, 75, ga + q)) {
+                const int2 w = __ldg(nz + ga + q);                   // (index o | end-of-fiber bit << 31, value bits)
+                x = w.x;
+                v = __int_as_float(w.y);
+            }
+        };
+        // lane l of the group holds nonzeros c + l and c + 4 + l of the group's stream
+        auto fetch = [&](int c, int (&x)[2], float (&v)[2]) {
+            fetch1(c + l, x[0], v[0]);
+            fetch1(c + 4 + l, x[1], v[1]);
+        };
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        int xn[2];
+        float vn[2];
+        fetch(0, xn, vn);
+        for (int c = 0; c < maxlen; c += 8) {
+            const int x[2] = {xn[0], xn[1]};
+            const float v[2] = {vn[0], vn[1]};
+            fetch(c + 8, xn, vn);
+            int xs[8];
+            float vs[8];
+            float4 e[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                xs[u] = __shfl_sync(SA_FULL_MASK, x[u >> 2], u & 3, 4);
+                vs[u] = __shfl_sync(SA_FULL_MASK, v[u >> 2], u & 3, 4);
+                uint32_t o = uint32_t(xs[u]) & 0x7fffffffu;
+                if (!SA_CHK(lim.status, o < lim.e_rows, 76, o)) o = 0u;
+                e[u] = sa_ldg4(E + (o * ld_e + 4u * l));
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                if (c + u < mylen) {
+                    acc.x = fmaf(vs[u], e[u].x, acc.x);
+                    acc.y = fmaf(vs[u], e[u].y, acc.y);
+                    acc.z = fmaf(vs[u], e[u].z, acc.z);
+                    acc.w = fmaf(vs[u], e[u].w, acc.w);
+                }
+                if (xs[u] < 0) {                                      // last nonzero of fiber it.f0 + slot
+                    if (SA_CHK(lim.status, slot >= 0 && slot < nf3, 77, slot)) *reinterpret_cast<float4 *>(pk + slot * R + 4 * l) = acc;
+                    acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                    ++slot;
+                }
+            }
+        }
+    }
+    __syncwarp();
+    {   // ---- phase B
+        const int mp = lane >> 2, nq = lane & 3;
+        const int nr = it.row_end - it.out_row;
+        const int my_end = lane < nr ? __ldg(pos2 + it.out_row + lane + 1) - it.f0 : 0x7fffffff;   // local end of subtree `lane`
+        int r = 0, fe = __shfl_sync(SA_FULL_MASK, my_end, 0);
+        float4 a0 = make_float4(0.f, 0.f, 0.f, 0.f), a1 = a0;
+        // D(k_f, 2mp..2mp+1) of eight fibers at a time, the next eight requested before the current eight are used
+        auto load_d = [&](int f0, float2 (&d)[8]) {
+            const int ks = f0 < 32 ? kk0 : kk1;
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int k = __shfl_sync(SA_FULL_MASK, ks, (f0 + u) & 31);
+                d[u] = sa_ldg2(D + (uint32_t(k) * ld_d + 2u * mp));
+            }
+        };
+        float2 d[8], dn[8];
+        load_d(0, d);
+        for (int f0 = 0; f0 < nf3; f0 += 8) {
+            if (f0 + 8 < nf3) load_d(f0 + 8, dn);
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                if (f0 + u < nf3) {
+                    const float4 tt = *reinterpret_cast<const float4 *>(pk + (f0 + u) * R + 4 * nq);
+                    a0.x = fmaf(d[u].x, tt.x, a0.x); a0.y = fmaf(d[u].x, tt.y, a0.y);
+                    a0.z = fmaf(d[u].x, tt.z, a0.z); a0.w = fmaf(d[u].x, tt.w, a0.w);
+                    a1.x = fmaf(d[u].y, tt.x, a1.x); a1.y = fmaf(d[u].y, tt.y, a1.y);
+                    a1.z = fmaf(d[u].y, tt.z, a1.z); a1.w = fmaf(d[u].y, tt.w, a1.w);
+                    if (f0 + u + 1 == fe) {                           // the subtree's last fiber
+                        float *dst = T2 + int64_t(it.out_row + r) * T2F + (2 * mp) * R + 4 * nq;
+                        *reinterpret_cast<float4 *>(dst) = a0;
+                        *reinterpret_cast<float4 *>(dst + R) = a1;
+                        a0 = make_float4(0.f, 0.f, 0.f, 0.f);
+                        a1 = a0;
+                        ++r;
+                        fe = __shfl_sync(SA_FULL_MASK, my_end, r & 31);
+                    }
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) d[u] = dn[u];
+        }
+    }
+}
+
+struct ttm4_plan {
+    size_t t2_bytes, p1_bytes, p2_bytes;
+};
+
+ttm4_plan plan(const sa_tensor *t)
+{
+    ttm4_plan p;
+    p.t2_bytes = sa_align256(size_t(t->count[1]) * T2F * sizeof(float));
+    p.p1_bytes = sa_align256(size_t(t->wl4_main.n_slots) * T2F * sizeof(float));
+    p.p2_bytes = sa_align256(size_t(t->wl4_aux.n_slots) * TILE4 * sizeof(float));
+    return p;
+}
+
+}  // namespace
+
+// workspace: [T2: one 16 x 16 temporary per level-1 fiber][partial temporaries of pass 1][partial tiles of pass 2]
+size_t sa_ws_ttm4_fissioned(const sa_tensor *t, const sa_dense *)
+{
+    const ttm4_plan p = plan(t);
+    return p.t2_bytes + p.p1_bytes + p.p2_bytes;
+}
+
+sa_status sa_launch_ttm4_fissioned(const sa_tensor *t, const sa_dense *ops, float *out, void *ws, size_t, cudaStream_t stream,
+                         int *launches)
+{
+    const ttm4_plan p = plan(t);
+    *launches = 0;
+    for (int i = 0; i < 3; ++i)                     // every range check comes before the first launch
+        if (ops[i].rows * ops[i].ld >= (int64_t(1) << 30)) return SA_E_UNSUPPORTED;   // 32-bit element offsets of factor rows
+    char *base = static_cast<char *>(ws);
+    float *T2 = reinterpret_cast<float *>(base);
+    float *part1 = reinterpret_cast<float *>(base + p.t2_bytes);
+    float *part2 = reinterpret_cast<float *>(base + p.t2_bytes + p.p1_bytes);
+    // the large subtrees: kernel 6 with the (i,j) subtrees as slices, factors D (rows by k) and E (rows by o)
+    sa_ttm3_view v;
+    v.wl = &t->wl4_main;
+    v.crd_fiber = t->d_crd[2];
+    v.crd_nz = t->d_crd[3];
+    v.vals = t->d_vals;
+    v.endbits = t->d_endbits;
+    v.n_fibers = t->count[2];
+    v.n_out_rows = t->count[1];
+    v.nnz = t->wl4_main.nnz;
+    v.nnz_total = t->nnz;
+    v.status = t->d_status;
+    fis_limits lim;
+    lim.status = t->d_status;
+    lim.c_rows = uint32_t(ops[0].rows); lim.d_rows = uint32_t(ops[1].rows); lim.e_rows = uint32_t(ops[2].rows);
+    lim.n_slices = uint32_t(t->dims[0]);
+    lim.n_subtrees = int32_t(t->count[1]); lim.n_fibers = int32_t(t->count[2]);
+    lim.n_slots = int32_t(t->wl4_aux.n_slots); lim.nnz = int32_t(t->nnz);
+    // pass 1: the small subtrees whole (subtree kernel), the large ones as slices of the order-3 kernel
+    const int64_t n_sub = int64_t(t->wl4_sub.items.size());
+    *launches = 0;
+    if (n_sub > 0) {
+        const bool contig = ops[1].ld == R && ops[2].ld == R;
+        auto kern = contig ? ttm4_subtree_kernel<true> : ttm4_subtree_kernel<false>;
+        static bool attr_set[2] = {false, false};
+        if (!attr_set[contig]) {
+            if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SUB_SMEM) != cudaSuccess) return SA_E_CUDA;
+            attr_set[contig] = true;
+        }
+        const int64_t ctas = (n_sub + SA_WARPS_PER_CTA - 1) / SA_WARPS_PER_CTA;
+        kern<<<(unsigned)ctas, 256, SUB_SMEM, stream>>>(t->wl4_sub.d_items, n_sub, t->d_pos[2], t->d_pos[3], t->d_crd[2],
+                                                                       t->d_nzpack, ops[1].ptr, ops[1].ld, ops[2].ptr, ops[2].ld, T2, lim);
+        if (cudaGetLastError() != cudaSuccess) return SA_E_CUDA;
+        *launches += 1;
+    }
+    if (!t->wl4_main.items.empty()) {
+        int n1 = 0;
+        const sa_status s = sa_launch_ttm3_view(v, ops[1], ops[2], T2, part1, stream, &n1);
+        if (s != SA_OK) return s;
+        *launches += n1;
+    }
+    // pass 2
+    const sa_worklist &wl = t->wl4_aux;
+    const int64_t n_items = int64_t(wl.items.size());
+    if (n_items > 0) {
+        int dev = 0, sms = 148;
+        if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        const int64_t ctas = std::min<int64_t>((n_items + SA_WARPS_PER_CTA - 1) / SA_WARPS_PER_CTA, int64_t(sms) * 2);
+        ttm4_slice_kernel<<<(unsigned)ctas, 256, 0, stream>>>(wl.d_items, n_items, t->d_crd[1], T2, ops[0].ptr, uint32_t(ops[0].ld),
+                                                            out, part2, lim);
+        if (cudaGetLastError() != cudaSuccess) return SA_E_CUDA;
+        *launches += 1;
+    }
+    if (!wl.fix.empty()) {
+        if (sa_launch_fixup(wl, part2, out, TILE4, stream) != cudaSuccess) return SA_E_CUDA;
+        *launches += 1;
+    }
+    return SA_OK;
+}

@@ -407,3 +407,66 @@ def test_fiber_row_worklist_of_order3_csf_partitions_fibers_and_nonzeros():
           for s in (sa.SA_SCHED_DEFAULT, sa.SA_SCHED_FUSED, sa.SA_SCHED_ASSOC_LEFT, sa.SA_SCHED_ASSOC_RIGHT)}
     assert ws[sa.SA_SCHED_FUSED] == ws[sa.SA_SCHED_ASSOC_LEFT] >= n_fibers * 32 * 4
     assert ws[sa.SA_SCHED_DEFAULT] == ws[sa.SA_SCHED_ASSOC_RIGHT] >= dims[2] * 32 * 4
+
+
+def test_order4_fissioned_second_pass_worklist_covers_every_fiber_quarter_once():
+    """Fissioned schedule of the order-4 chain, list 5: (piece of a slice) x (quarter of the temporaries' columns)."""
+    w = configs.make(5, "mini")
+    t = sa.SparseTensor(w.dims, w.coords, w.vals, sa.SA_FMT_CSF, device=-1)
+    levels, _ = export_all(t, "csf")
+    crd0, pos1 = levels[0][1], levels[1][0]
+    counts, items, fix = sa.sa_tensor_worklist(t.handle, 5)
+    slice_pos = {int(c): n for n, c in enumerate(crd0)}
+    covered = np.zeros((len(levels[1][1]), 4), dtype=np.int32)
+    pieces = {}
+    for row, row_end, f0, f1, _, _, dest, quarter in items:
+        s = slice_pos[int(row)]
+        assert pos1[s] <= f0 < f1 <= pos1[s + 1] and f1 - f0 <= 512 and 0 <= quarter < 4
+        covered[f0:f1, quarter] += 1
+        if dest >= 0:
+            pieces.setdefault(int(row), set()).add(int(dest))
+        else:
+            assert (f0, f1) == (pos1[s], pos1[s + 1])
+    assert (covered == 1).all()
+    assert (np.diff(items[:, 3] - items[:, 2]) <= 0).all(), "largest items first"
+    empties = set()
+    used = np.zeros(int(counts[3]), dtype=np.int32)
+    for row, slot0, count, _ in fix:
+        if count == 0:
+            empties.add(int(row))
+            continue
+        assert pieces[int(row)] == set(range(slot0, slot0 + count))
+        used[slot0:slot0 + count] += 1
+    assert (used == 1).all()
+    assert empties == set(range(w.dims[0])) - set(int(c) for c in crd0)
+
+
+def test_order4_fissioned_subtree_worklist_covers_every_subtree_once_within_its_limits():
+    """Fissioned schedule of the order-4 chain, list 6: ranges of whole small (i,j) subtrees, at most 64 level-2 fibers and 32
+    subtrees each; a larger subtree is left to list 4 (the order-3 lists over those subtrees)."""
+    w = configs.make(5, "mini")
+    t = sa.SparseTensor(w.dims, w.coords, w.vals, sa.SA_FMT_CSF, device=-1)
+    levels, _ = export_all(t, "csf")
+    pos2, pos3 = levels[2][0], levels[3][0]
+    counts, items, fix = sa.sa_tensor_worklist(t.handle, 6)
+    assert counts[0] > 0 and counts[2] == 0 and counts[3] == 0
+    n_sub = int(t.info()[1][1])
+    seen = np.zeros(n_sub, dtype=np.int32)
+    for row, row_end, f0, f1, p0, p1, dest, _ in items:
+        assert row_end > row and dest < 0
+        assert (f0, f1) == (pos2[row], pos2[row_end]) and (p0, p1) == (pos3[f0], pos3[f1])
+        assert f1 - f0 <= 64 and row_end - row <= 32
+        seen[row:row_end] += 1
+    # the others are the large ones, and the main list holds exactly those
+    large = np.nonzero(seen == 0)[0]
+    assert (seen <= 1).all()
+    f3s, nz = np.diff(pos2), pos3[pos2[1:]] - pos3[pos2[:-1]]
+    assert ((f3s[large] > 64) | (nz[large] > 4096)).all() and ((f3s[seen == 1] <= 64) & (nz[seen == 1] <= 4096)).all()
+    assert set(sa.sa_tensor_worklist(t.handle, 4)[1][:, 0].tolist()) == set(large.tolist())
+    # one (i,j) pair with 130 level-2 fibers next to a small one: the large one is in the main list only
+    big = np.stack([np.zeros(130), np.zeros(130), np.arange(130), np.zeros(130)], axis=1).astype(np.int32)
+    both = np.concatenate([big, np.array([[1, 1, 5, 1]], np.int32)])
+    t2 = sa.SparseTensor((2, 2, 130, 2), both, np.ones(131, np.float32), sa.SA_FMT_CSF, device=-1)
+    sub = sa.sa_tensor_worklist(t2.handle, 6)[1]
+    main = sa.sa_tensor_worklist(t2.handle, 4)[1]
+    assert [tuple(x[:2]) for x in sub.tolist()] == [(1, 2)] and set(main[:, 0].tolist()) == {0}

@@ -45,11 +45,15 @@ for cfg in range(1, 11):
     if w.expr in ("spmm_gemm", "spttm_spttm"):
         check(w, sa.SA_SCHED_ASSOC_LEFT)
         check(w, sa.SA_SCHED_ASSOC_RIGHT)
+    elif w.expr in ("spttm_ttm4", "ttmc3"):
+        check(w, sa.SA_SCHED_FUSED)
+        check(w, sa.SA_SCHED_FISSIONED)
     else:
         check(w)
 # edge tensors: large (i,j) subtrees and split slices of the order-4 chain, long fibers of the order-3 chain
-check(configs.make_ttm4_zipf("edge4", 31, 90, 6, 130, 110, 150_000, 1.4, 5.0, 16, 16, 16))
-check(configs.make_ttm4_zipf("edge4b", 32, 90, 700, 50, 45, 150_000, 1.4, 5.0, 16, 16, 16))
+for s4 in (sa.SA_SCHED_FUSED, sa.SA_SCHED_FISSIONED):
+    check(configs.make_ttm4_zipf("edge4", 31, 90, 6, 130, 110, 150_000, 1.4, 5.0, 16, 16, 16), s4)
+    check(configs.make_ttm4_zipf("edge4b", 32, 90, 700, 50, 45, 150_000, 1.4, 5.0, 16, 16, 16), s4)
 check(configs.make_ttm3_zipf("edge3", 41, 50, 40, 3000, 120_000, 1.4, 300.0, 32, 16))
 check(configs.make_ttm3_zipf("edge3b", 42, 700, 300, 40, 60_000, 1.0, 2.0, 16, 32))
 print("CHECKED-OK")

@@ -195,21 +195,41 @@ def test_ttm4_ragged_and_split_slices(sa):
     # itself, so the order-3 kernel writes their temporaries first (some split over several thread blocks, with
     # partial temporaries that the fix-up kernel sums) and items of kind 1 copy them into the pool
     w = configs.make_ttm4_zipf("edge4", 31, 90, 6, 130, 110, 150_000, 1.4, 5.0, 16, 16, 16)
-    A, t = _check(sa, w)
+    A, t = _check(sa, w, sched=sa.SA_SCHED_FUSED)
     assert sa.sa_tensor_worklist(t.handle, 0)[0][3] >= 2, "a large (i,j) subtree must be split over several thread blocks"
     kinds = sa.sa_tensor_worklist(t.handle, 2)[1][:, 7]
     assert (kinds == 1).any() and (kinds == 0).any()
     # many level-1 fibers per slice: the head slices span several pieces and leave partial slice tiles
     w = configs.make_ttm4_zipf("edge4b", 32, 90, 700, 50, 45, 150_000, 1.4, 5.0, 16, 16, 16)
-    A, t = _check(sa, w)
+    A, t = _check(sa, w, sched=sa.SA_SCHED_FUSED)
     assert sa.sa_tensor_worklist(t.handle, 1)[0][3] >= 2, "the head slice must be split into several pieces"
     # subtrees with more level-2 fibers than one batch holds next to small ones
     for w in (configs.make_ttm4_zipf("edge4c", 33, 90, 40, 160, 110, 150_000, 1.4, 5.0, 16, 16, 16),
               configs.make_ttm4_zipf("edge4d", 34, 400, 60, 150, 40, 200_000, 1.2, 3.0, 16, 16, 16)):
-        A, t = _check(sa, w)
+        A, t = _check(sa, w, sched=sa.SA_SCHED_FUSED)
         items = sa.sa_tensor_worklist(t.handle, 2)[1]
         nf = items[:, 3] - items[:, 2]
         assert ((items[:, 7] == 0) & (nf > 32)).any() and ((items[:, 7] == 0) & (nf <= 32) & (items[:, 1] - items[:, 0] > 1)).any()
+
+
+def test_ttm4_fissioned_ragged_and_split_slices(sa):
+    """The same tensors through the two-pass schedule (temporaries of all (i,j) subtrees in the workspace)."""
+    F = sa.SA_SCHED_FISSIONED
+    # few level-1 fibers per slice: the head slice's (i,j) subtrees exceed one thread block's chunk, so the
+    # first pass writes partial temporaries that the fix-up kernel sums
+    w = configs.make_ttm4_zipf("edge4", 31, 90, 6, 130, 110, 150_000, 1.4, 5.0, 16, 16, 16)
+    A, t = _check(sa, w, sched=F)
+    assert sa.sa_tensor_worklist(t.handle, 4)[0][3] >= 2, "a large (i,j) subtree must be split over several thread blocks"
+    # many level-1 fibers per slice: the second pass cuts the head slices into pieces of 512 fibers
+    w = configs.make_ttm4_zipf("edge4b", 32, 90, 700, 50, 45, 150_000, 1.4, 5.0, 16, 16, 16)
+    A, t = _check(sa, w, sched=F)
+    assert sa.sa_tensor_worklist(t.handle, 5)[0][3] >= 2, "the head slice must be split into several pieces"
+    # both kernels of the first pass in one run: small subtrees (list 6) and large ones (list 4)
+    for w in (configs.make_ttm4_zipf("edge4c", 33, 90, 40, 160, 110, 150_000, 1.4, 5.0, 16, 16, 16),
+              configs.make_ttm4_zipf("edge4d", 34, 400, 60, 150, 40, 200_000, 1.2, 3.0, 16, 16, 16)):
+        A, t = _check(sa, w, sched=F)
+        n_main, n_sub = (int(sa.sa_tensor_worklist(t.handle, x)[0][0]) for x in (4, 6))
+        assert n_main > 0 and n_sub > 0, (n_main, n_sub)
 
 
 def test_results_are_reproducible_run_to_run(sa):
@@ -290,7 +310,7 @@ def test_dense_stage_ragged_rows_and_padded_leading_dimensions(sa, L, M):
 
 def test_ttm4_padded_factor_matrices(sa):
     """Order-4 chain with the factor matrices given as padded views (leading dimension 20): the fused kernel's
-    general-stride variant."""
+    general-stride variant, and the subtree kernel's of the two-pass schedule."""
     import torch
     w = configs.make_ttm4_zipf("edge4e", 35, 300, 60, 150, 40, 120_000, 1.2, 3.0, 16, 16, 16)
     A_ref, S_ref = oracle.evaluate(w)
@@ -300,11 +320,12 @@ def test_ttm4_padded_factor_matrices(sa):
         b = torch.zeros(x.shape[0], 20, device="cuda")
         b[:, :16] = torch.from_numpy(x).cuda()
         views.append(b[:, :16])
-    out, _ = t.run(w.expr, views)
-    torch.cuda.synchronize()
-    assert sa.sa_last_device_status(t.handle, torch.cuda.current_stream().cuda_stream) == sa.SA_OK
-    assert_close(out.cpu().numpy().astype(np.float64), A_ref, S_ref, TOL_FP32, "ttm4 padded ld")
-    assert int(sa.sa_tensor_worklist(t.handle, 2)[0][0]) > 0
+    for sched in (sa.SA_SCHED_FUSED, sa.SA_SCHED_FISSIONED):
+        out, _ = t.run(w.expr, views, sched=sched)
+        torch.cuda.synchronize()
+        assert sa.sa_last_device_status(t.handle, torch.cuda.current_stream().cuda_stream) == sa.SA_OK
+        assert_close(out.cpu().numpy().astype(np.float64), A_ref, S_ref, TOL_FP32, "ttm4 padded ld, schedule %d" % sched)
+    assert int(sa.sa_tensor_worklist(t.handle, 2)[0][0]) > 0 and int(sa.sa_tensor_worklist(t.handle, 6)[0][0]) > 0
 
 
 def test_allocator_failure_at_every_upload_is_reported_and_leaks_nothing(sa):

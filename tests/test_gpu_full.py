@@ -112,13 +112,19 @@ def test_cfg4_full_sampled(sa, cfg4, sched):
     torch.cuda.empty_cache()
 
 
-def test_cfg5_full_sampled(sa):
+@pytest.fixture(scope="module")
+def cfg5():
+    return configs.make(5, "full")
+
+
+@pytest.mark.parametrize("sched", ["fused", "fissioned"])
+def test_cfg5_full_sampled(sa, cfg5, sched):
     import torch
-    w = configs.make(5, "full")
-    out, t = _run_full(sa, w)
+    w = cfg5
+    out, t = _run_full(sa, w, sched=sa.SA_SCHED_FUSED if sched == "fused" else sa.SA_SCHED_FISSIONED)
     sel = _sample(w, 600_000, 150)                    # includes a slice split over several thread blocks
-    _compare(out, w, sel, w.name)
-    _compare_head_slice(out, w, w.name)               # 19.9 % of B in one slice
+    _compare(out, w, sel, w.name + "/" + sched)
+    _compare_head_slice(out, w, w.name + "/" + sched)  # 19.9 % of B in one slice
     del out, t
     torch.cuda.empty_cache()
 

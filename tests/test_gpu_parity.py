@@ -26,6 +26,29 @@ def test_ttm_chains_mini(sa, cfg):
     assert_close(A, A_ref, S_ref, TOL_FP32, w.name)
 
 
+@pytest.mark.parametrize("sched", ["fused", "fissioned", "default"])
+def test_ttm4_mini_every_schedule(sa, sched):
+    """Order-4 chain: temporaries on chip (fused), through the workspace (fissioned), and the default, which is the
+    fissioned schedule until a cap on auxiliary memory rules it out."""
+    w = configs.make(5, "mini")
+    A_ref, S_ref = oracle.evaluate(w)
+    s = {"fused": sa.SA_SCHED_FUSED, "fissioned": sa.SA_SCHED_FISSIONED, "default": sa.SA_SCHED_DEFAULT}[sched]
+    A, t = run_gpu(sa, w, sched=s)
+    assert_close(A, A_ref, S_ref, TOL_FP32, w.name + "/" + sched)
+    ops = [(16, d.shape[0], d.shape[1], d.shape[1]) for d in w.dense]
+    E4 = sa.SA_EXPR_SPTTM_TTM4
+    fus, fis = (sa.sa_schedule_cost(t.handle, E4, x, ops) for x in (sa.SA_SCHED_FUSED, sa.SA_SCHED_FISSIONED))
+    n_sub = int(t.info()[1][1])
+    assert fis["workspace_bytes"] >= n_sub * 1024 > fus["workspace_bytes"]
+    assert fis["moved_bytes"] == fus["moved_bytes"] + 8 * n_sub * 256 and fis["iterations"] == fus["iterations"]
+    assert sa.sa_schedule_cost(t.handle, E4, sa.SA_SCHED_DEFAULT, ops)["resolved"] == sa.SA_SCHED_FISSIONED
+    if sched == "default":
+        sa.sa_tensor_set_aux_limit(t.handle, n_sub * 1024 - 1)
+        assert sa.sa_schedule_cost(t.handle, E4, sa.SA_SCHED_DEFAULT, ops)["resolved"] == sa.SA_SCHED_FUSED
+        A2, _ = run_gpu(sa, w, sched=s, tensor=t)          # now the fused kernel runs
+        assert_close(A2, A_ref, S_ref, TOL_FP32, w.name + "/default under a cap")
+
+
 @pytest.mark.parametrize("ranks", [(16, 16, 16), (32, 16, 16), (16, 32, 16), (16, 16, 32), (32, 32, 16)])
 def test_ttmc3_both_schedules(sa, ranks):
     """Kernel 5 with the loop over i fused (block accumulators in shared memory) and fissioned (slice temporaries in
