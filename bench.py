@@ -82,14 +82,15 @@ def algorithmic_work(w, counts, sched):
         L, M = w.dense[0].shape[1], w.dense[1].shape[1]
         return 8 * nnz + 8 * F2 + 8 * S + sz(w.dense[0]) + sz(w.dense[1]) + out_bytes, 2 * nnz * M + 2 * F2 * L * M
     if w.expr == "ttmc3":
-        # fused over i: nothing but the streams, the factors and the output; fissioned: the slice temporaries
-        # T(i,m,n) are written and read once
+        # the streams, the factors and the output (the slice temporaries T(i,m,n) of the fissioned schedule are
+        # traffic, not algorithmic bytes: 8 I M N more)
         S, F2 = int(counts[0]), int(counts[1])
         L, M, N = (d.shape[1] for d in w.dense)
-        temp = 8 * w.dims[0] * M * N if sched == "fissioned" else 0
-        return (8 * nnz + 8 * F2 + 8 * S + sum(sz(d) for d in w.dense) + out_bytes + temp,
+        return (8 * nnz + 8 * F2 + 8 * S + sum(sz(d) for d in w.dense) + out_bytes,
                 2 * nnz * N + 2 * F2 * M * N + 2 * w.dims[0] * L * M * N)
     if w.expr == "spttm_ttm4":
+        # what the method must move: the same for both schedules (the temporaries that the fissioned schedule sends
+        # through the workspace are traffic, not algorithmic bytes)
         S, F2, F3 = int(counts[0]), int(counts[1]), int(counts[2])
         L, M, N = (d.shape[1] for d in w.dense)
         b = 8 * nnz + 8 * F3 + 8 * F2 + 8 * S + sum(sz(d) for d in w.dense) + out_bytes
@@ -330,11 +331,13 @@ def workload_label(cfg, sched):
              9: "kernel 8 <MTTKRP,GEMM> on the config-2 tensor, R=32 M=32",
              10: "kernel 7 <SpTTM,SpTTM> on the config-2 tensor, L=M=32, sparse output (one row per (i,j) fiber)",
              11: "kernel 5 <3D TTMC> on a flickr-3d-shaped tensor 320000x2820000x1600000 112.89M nnz L=M=N=16"}
-    return names[cfg] + (" (%s)" % sched if cfg in (4, 10) or (cfg in (6, 11) and sched == "fissioned") else "")
+    return names[cfg] + (" (%s)" % sched if cfg in (4, 5, 6, 10, 11) else "")
 
 
 def label(args):
-    return workload_label(args.workload or 2, args.sched) + ("" if args.scale == "full" else " [%s-scale stand-in]" % args.scale)
+    cfg = args.workload or 2
+    sched = args.sched or ("right" if cfg in (4, 10) else "default")
+    return workload_label(cfg, sched) + ("" if args.scale == "full" else " [%s-scale stand-in]" % args.scale)
 
 
 def run_reference(args, w, rank, world):
@@ -369,8 +372,9 @@ def measure(sa, torch, dist, w, sched_name, steps, warmup, e2e_steps, dev, rank,
     tensor = sa.SparseTensor(w.dims, w.coords, w.vals, fmt, device=dev.index)
     build_s = time.perf_counter() - t0
     nnz, counts, n_chunks = tensor.info()
+    two_schedules = w.expr in ("spttm_ttm4", "ttmc3")          # fused / fissioned
     sched = {"left": sa.SA_SCHED_ASSOC_LEFT, "right": sa.SA_SCHED_ASSOC_RIGHT, "default": sa.SA_SCHED_DEFAULT,
-             "fused": sa.SA_SCHED_DEFAULT, "fissioned": sa.SA_SCHED_FISSIONED}[sched_name]
+             "fused": sa.SA_SCHED_FUSED if two_schedules else sa.SA_SCHED_DEFAULT, "fissioned": sa.SA_SCHED_FISSIONED}[sched_name]
     host_ops = [torch.from_numpy(np.ascontiguousarray(x)).pin_memory() for x in w.dense]
     ops = [x.to(dev, non_blocking=False) for x in host_ops]
     out = torch.empty(w.out_shape, dtype=torch.float32, device=dev)
@@ -436,12 +440,12 @@ def measure(sa, torch, dist, w, sched_name, steps, warmup, e2e_steps, dev, rank,
         peaks, peak_kind = measured_peaks()
         # the schedule that ran: the library's choice when the default was asked for
         ran = sched_name
-        if sched_name == "default" and w.expr in ("spmm_gemm", "spttm_spttm"):
+        if sched_name == "default":
             ops_desc = [(x.data_ptr(), x.shape[0], x.shape[1], x.stride(0)) for x in ops]
-            ws = {k: sa.sa_workspace_size(tensor.handle, sa._EXPR_OF[w.expr], v, ops_desc)
-                  for k, v in (("default", sa.SA_SCHED_DEFAULT), ("left", sa.SA_SCHED_ASSOC_LEFT), ("right", sa.SA_SCHED_ASSOC_RIGHT))}
-            ran = "left" if ws["default"] == ws["left"] and ws["left"] != ws["right"] else "right"
-        abytes, aflops = algorithmic_work(w, counts, ran if w.expr in ("spmm_gemm", "spttm_spttm", "ttmc3") else "fused")
+            resolved = sa.sa_schedule_cost(tensor.handle, sa._EXPR_OF[w.expr], sa.SA_SCHED_DEFAULT, ops_desc)["resolved"]
+            ran = {sa.SA_SCHED_FUSED: "fused", sa.SA_SCHED_ASSOC_LEFT: "left", sa.SA_SCHED_ASSOC_RIGHT: "right",
+                   sa.SA_SCHED_FISSIONED: "fissioned"}[resolved]
+        abytes, aflops = algorithmic_work(w, counts, ran)
         achieved = abytes / (ms_per_step * 1e-3) / 1e9
         traffic, traffic_kernel = ncu_traffic(workload_id, ran) if scale == "full" else (None, None)
         rec = {
@@ -474,7 +478,7 @@ def measure(sa, torch, dist, w, sched_name, steps, warmup, e2e_steps, dev, rank,
 
 
 # (config, schedule) pairs of the default run besides the headline config 2
-PER_CONFIG = [(1, "fused"), (3, "fused"), (4, "left"), (4, "right"), (4, "default"), (5, "fused")]
+PER_CONFIG = [(1, "fused"), (3, "fused"), (4, "left"), (4, "right"), (4, "default"), (5, "fused"), (5, "fissioned"), (5, "default")]
 
 
 def main():
@@ -486,8 +490,9 @@ def main():
     ap.add_argument("--workload", type=int, default=None, choices=[1, 2, 3, 4, 5, 6, 7, 8, 9, 10, 11],
                     help="one workload only; without it: config 2 as the headline plus a per_config list of all five configs")
     ap.add_argument("--scale", default="full", choices=["full", "mid", "mini"])
-    ap.add_argument("--sched", default="right", choices=["left", "right", "default", "fissioned"],
-                    help="association order for workloads 4 and 10; 'fissioned' selects the second schedule of workload 6")
+    ap.add_argument("--sched", default=None, choices=["left", "right", "fused", "fissioned", "default"],
+                    help="schedule: left / right (association order, workloads 4 and 10), fused / fissioned (workloads 5, 6, 11), "
+                         "default (the library's choice; also the default here, except workloads 4 and 10: right)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-per-config", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=5)
@@ -529,9 +534,12 @@ def main():
             pending[cfg] = pool.submit(configs.make, cfg, "full")
 
     w = configs.make(args.workload, args.scale)
-    sched_name = args.sched if w.expr in ("spmm_gemm", "spttm_spttm") else "fused"
-    if w.expr == "ttmc3" and args.sched == "fissioned":
-        sched_name = "fissioned"
+    if w.expr in ("spmm_gemm", "spttm_spttm"):
+        sched_name = args.sched if args.sched in ("left", "right", "default") else "right"
+    elif w.expr in ("spttm_ttm4", "ttmc3"):
+        sched_name = args.sched if args.sched in ("fused", "fissioned", "default") else "default"
+    else:
+        sched_name = "fused"
     rec = measure(sa, torch, dist, w, sched_name, args.steps, args.warmup, args.e2e_steps, dev, rank, world,
                   gather_probe=True, scale=args.scale, workload_id=args.workload)
     if rank == 0:

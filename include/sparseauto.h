@@ -185,7 +185,8 @@ sa_status sa_tensor_export(const sa_tensor *t, int level, int64_t *pos, int32_t 
  *      subtrees).  counts = {pieces, subtrees above 4096 nonzeros, super-items, 0}.
  *   4, 5, 6  order-4 CSF, the lists of SA_SCHED_FISSIONED: 4 = like list 0 over the (i,j) subtrees with more than 64
  *      level-2 fibers or 4096 nonzeros (out_row = index of the level-1 fiber); 5 = second pass, one item per (piece
- *      of at most 512 level-1 fibers [f0,f1) of slice out_row, quarter of the 256 columns (m,n) in the last field),
+ *      of at most 512 level-1 fibers [f0,f1) of slice out_row, quarter of the 256 columns (m,n) in the last field;
+ *      a piece of at most eight fibers is a single item with 4 there: all quarters),
  *      with the fix-up entries of slices cut into pieces; 6 = first pass on whole small subtrees: rows
  *      [out_row,row_end) = level-1 fibers, [f0,f1) their level-2 fibers (at most 64), [p0,p1) their nonzeros
  * For which = 0..2 and 4..6:

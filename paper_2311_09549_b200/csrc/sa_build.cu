@@ -318,16 +318,20 @@ void build_ttm4_fissioned(sa_tensor *t, sa_worklist &wl, sa_worklist &wl2)
             wl2.fix.push_back(sa_fix{row, slot0, int32_t(nc), 0});
             wl2.n_slots += nc;
         }
-        for (int64_t c = 0; c < nc; ++c)
-            for (int qc = 0; qc < 4; ++qc) {
+        for (int64_t c = 0; c < nc; ++c) {
+            const int64_t f0 = fa + c * CHUNK_F, f1 = std::min(fb, fa + (c + 1) * CHUNK_F);
+            // a piece of at most eight fibers (one tensor-core group) is one item that takes the four quarters in turn
+            const int nq = f1 - f0 <= 8 ? 1 : 4;
+            for (int qc = 0; qc < nq; ++qc) {
                 sa_item it = empty_item();
                 it.out_row = row; it.row_end = row + 1;
-                it.f0 = int32_t(fa + c * CHUNK_F); it.f1 = int32_t(std::min(fb, fa + (c + 1) * CHUNK_F));
+                it.f0 = int32_t(f0); it.f1 = int32_t(f1);
                 it.p0 = it.f0; it.p1 = it.f1;          // size key: fibers
                 it.dest = nc > 1 ? slot0 + int32_t(c) : -1;
-                it.pad = qc;
+                it.pad = nq == 1 ? 4 : qc;
                 items.push_back(it);
             }
+        }
     }
     // largest first: the tail of the launch is then made of the cheapest items
     std::stable_sort(items.begin(), items.end(), [](const sa_item &a, const sa_item &b) { return (a.f1 - a.f0) > (b.f1 - b.f0); });

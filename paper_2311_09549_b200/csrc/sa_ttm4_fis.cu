@@ -75,10 +75,15 @@ ttm4_slice_kernel(const sa_item *__restrict__ items, int64_t n_items, const int3
     for (int64_t n = int64_t(blockIdx.x) * SA_WARPS_PER_CTA + (threadIdx.x >> 5); n < n_items; n += stride) {
         const int4 ia = __ldg(reinterpret_cast<const int4 *>(items + n));          // out_row, row_end, f0, f1
         const int4 ib = __ldg(reinterpret_cast<const int4 *>(items + n) + 1);      // p0, p1, dest, quarter
-        const int f0 = ia.z, f1 = ia.w, qc = ib.w;
-        if (!SA_CHK(lim.status, f0 >= 0 && f0 <= f1 && f1 <= lim.n_subtrees && uint32_t(qc) < 4u && uint32_t(ia.x) < lim.n_slices &&
+        const int f0 = ia.z, f1 = ia.w;
+        if (!SA_CHK(lim.status, f0 >= 0 && f0 <= f1 && f1 <= lim.n_subtrees && uint32_t(ib.w) <= 4u && uint32_t(ia.x) < lim.n_slices &&
                                     ib.z < lim.n_slots, 72, n))
             continue;
+        // quarter 4 = all four quarters, one after the other (pieces of at most eight fibers: one record, one set of
+        // C values and one latency chain instead of four)
+        const int q_first = ib.w == 4 ? 0 : ib.w, q_last = ib.w == 4 ? 3 : ib.w;
+#pragma unroll 1
+        for (int qc = q_first; qc <= q_last; ++qc) {
         const float *t2q = T2 + qc * QC;
         float acc[NT4][4];
 #pragma unroll
@@ -117,6 +122,7 @@ ttm4_slice_kernel(const sa_item *__restrict__ items, int64_t n_items, const int3
                 sa_st_cs2(dst + g * T2F + 8 * nt, lo);
                 sa_st_cs2(dst + (g + 8) * T2F + 8 * nt, hi);
             }
+        }
         }
     }
 }

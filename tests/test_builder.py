@@ -421,8 +421,13 @@ def test_order4_fissioned_second_pass_worklist_covers_every_fiber_quarter_once()
     pieces = {}
     for row, row_end, f0, f1, _, _, dest, quarter in items:
         s = slice_pos[int(row)]
-        assert pos1[s] <= f0 < f1 <= pos1[s + 1] and f1 - f0 <= 512 and 0 <= quarter < 4
-        covered[f0:f1, quarter] += 1
+        assert pos1[s] <= f0 < f1 <= pos1[s + 1] and f1 - f0 <= 512 and 0 <= quarter <= 4
+        if quarter == 4:
+            assert f1 - f0 <= 8, "only a piece of one tensor-core group takes all four quarters in one item"
+            covered[f0:f1, :] += 1
+        else:
+            assert f1 - f0 > 8
+            covered[f0:f1, quarter] += 1
         if dest >= 0:
             pieces.setdefault(int(row), set()).add(int(dest))
         else:
