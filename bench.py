@@ -33,16 +33,29 @@ FALLBACK_HBM_GBS = 6650.0
 
 
 # DRAM bytes (read + write) of one launch of the dominant kernel, from the ncu captures summarised under
-# profiles/.  A figure is reported only while the kernel's source file still has the hash it had when the
-# counters were taken; otherwise `traffic` is null.
+# profiles/ (keyed by workload, or by (workload, schedule that ran)).  A figure is reported only while the kernel's
+# source file still has the hash it had when the counters were taken; otherwise `traffic` is null.  Workloads 4 and 5
+# are captured at a quarter of their size (--scale mid) and scaled by the nonzeros, see the profiles.
 NCU_TRAFFIC = {
-    2: {"kernel": "ttm3_kernel<32,32>", "source": "paper_2311_09549_b200/csrc/sa_ttm3.cu",
-        "sha256": "339c0c9c7e9ba6ecce502229659dadc513dea0778eb8559c09c4a9ad12aec82b",
-        "dram_bytes": 851268608, "profile": "profiles/ttm3_kernel_cfg2.md"},
-    5: {"kernel": "ttm4_subtree_kernel (pass 1 of the order-4 chain on the small subtrees, 51 % of the step)",
-        "source": "paper_2311_09549_b200/csrc/sa_ttm4.cu",
-        "sha256": "0cf1a9b53532ebf95fe9cccc071d824a69c9d457ac76a6d37f6355f062eef7c9",
-        "dram_bytes": 2217051392, "profile": "profiles/ttm4_kernel_cfg5.md"},
+    2: {"kernel": "ttm3_kernel<32,32> (98.5 % of the step)", "source": "paper_2311_09549_b200/csrc/sa_ttm3.cu",
+        "sha256": "af4a25219f07837e9092aca54ff9ea55ba69cb5e7ed164513575012bddb546ec",
+        "dram_bytes": 848247808, "profile": "profiles/ttm3_kernel_cfg2.md"},
+    3: {"kernel": "sddmm_spmm_kernel<64,64> (99.6 % of the step)", "source": "paper_2311_09549_b200/csrc/sa_sddmm_spmm.cu",
+        "sha256": "7c9971e0e72e49dfbb4404b68def327568372ea956767048b5d3d830810b8ead",
+        "dram_bytes": 13186066944, "profile": "profiles/sddmm_spmm_kernel_cfg3.md"},
+    (4, "left"): {"kernel": "spmm_gemm_left_kernel<256,64> (the whole step; counters of the quarter-size case x 4)",
+                  "source": "paper_2311_09549_b200/csrc/sa_spmm_gemm.cu", "sha256": "a7d3ddb4c4f3e2c41bc5f803c06e42250d24443649e1f4c918744c74fbb8b39f",
+                  "dram_bytes": 4 * 24086787584, "profile": "profiles/spmm_gemm_kernels_cfg4.md"},
+    (4, "right"): {"kernel": "spmm_kernel<2> (85 % of the step; counters of the quarter-size case x 4)",
+                   "source": "paper_2311_09549_b200/csrc/sa_spmm_gemm.cu", "sha256": "a7d3ddb4c4f3e2c41bc5f803c06e42250d24443649e1f4c918744c74fbb8b39f",
+                   "dram_bytes": 4 * 4974276864, "profile": "profiles/spmm_gemm_kernels_cfg4.md"},
+    (5, "fused"): {"kernel": "ttm4_fused_kernel (94 % of the step; counters of the quarter-size case x 4)",
+                   "source": "paper_2311_09549_b200/csrc/sa_ttm4.cu", "sha256": "97022d6fa719293c229dc5e2d93ca15ae4c4ac958aa96d03b58b1b36d5fc2da3",
+                   "dram_bytes": 4 * 424575488, "profile": "profiles/ttm4_kernels_cfg5.md"},
+    (5, "fissioned"): {"kernel": "ttm4_subtree_kernel (pass 1 on the small subtrees, 51 % of the step; counters of the "
+                                 "quarter-size case x 4)",
+                       "source": "paper_2311_09549_b200/csrc/sa_ttm4_fis.cu", "sha256": "6cd1680b60cc8a1c0240b7d13638a8dcca5f99c35a48a9b7a50a9aed7424ebd7",
+                       "dram_bytes": 4 * 670214912, "profile": "profiles/ttm4_kernels_cfg5.md"},
     10: {"kernel": "fiber_spmm_kernel<32> (99 % of the step)", "source": "paper_2311_09549_b200/csrc/sa_spmm_gemm.cu",
          "sha256": "408ed3d1f40077ca8fcb6e4ebeb2dc9b8ca08986b342d17b370a87df4d7b251e",
          "dram_bytes": 955500000, "profile": "profiles/fiber_spmm_kernel_w10.md"},
