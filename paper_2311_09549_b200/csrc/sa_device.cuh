@@ -55,6 +55,20 @@ static inline sa_limits sa_make_limits(const sa_tensor *t, int64_t gather_rows, 
     return lim;
 }
 
+// Opt a kernel into `bytes` of dynamic shared memory once per device instead of once per launch (the attribute is
+// per device; `done` is the caller's flag array, one entry per device ordinal).
+constexpr int SA_MAX_DEVICE_FLAGS = 64;
+template <typename Kernel>
+static inline bool sa_set_smem_once(Kernel kernel, int bytes, bool (&done)[SA_MAX_DEVICE_FLAGS])
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return false;
+    if (dev >= 0 && dev < SA_MAX_DEVICE_FLAGS && done[dev]) return true;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) return false;
+    if (dev >= 0 && dev < SA_MAX_DEVICE_FLAGS) done[dev] = true;
+    return true;
+}
+
 // ---- PTX helpers shared by the kernels
 
 // x = hi + lo with hi the upper 19 bits of x (a TF32 number) and lo = x - hi (exact in fp32), itself cut to

@@ -38,9 +38,10 @@ struct sa_fix {
 
 // Order-3 CSF only: what the kernel reads per item (a piece of one slice, "unit").  The warp's 32 lanes
 // form SA_STREAMS groups of 8 lanes; each group streams one contiguous part of [p0, p1) whose start is a
-// multiple of 8 nonzeros (see sa_unit3_streams); sf[q] is the level-1 fiber that holds the first
+// multiple of SA_ROUND nonzeros (see sa_unit3_streams); sf[q] is the level-1 fiber that holds the first
 // nonzero of part q.
 constexpr int SA_STREAMS = 4;
+constexpr int SA_ROUND = 16;         // nonzeros a stream takes per round of the order-3 kernel
 struct sa_unit3 {
     int32_t out_row;
     int32_t dest;
@@ -50,14 +51,14 @@ struct sa_unit3 {
 static_assert(sizeof(sa_unit3) == 32, "sa_unit3 is read as two 16-byte pieces");
 
 // Nonzero ranges of the SA_STREAMS parts of a unit [p0, p1): part q = [lo[q], hi[q]) (empty if lo >= hi);
-// every part starts at base8 + q * slen with base8 = p0 rounded down to a multiple of 8 and slen a
-// multiple of 8, clipped to [p0, p1).  The same arithmetic runs in the kernel.
+// every part starts at base + q * slen with base = p0 rounded down to a multiple of SA_ROUND and slen a
+// multiple of SA_ROUND, clipped to [p0, p1).  The same arithmetic runs in the kernel.
 static inline void sa_unit3_streams(int64_t p0, int64_t p1, int64_t *lo, int64_t *hi)
 {
-    const int64_t base8 = p0 & ~int64_t(7), span = p1 - base8;
-    const int64_t slen = ((span + SA_STREAMS - 1) / SA_STREAMS + 7) & ~int64_t(7);
+    const int64_t base = p0 & ~int64_t(SA_ROUND - 1), span = p1 - base;
+    const int64_t slen = ((span + SA_STREAMS - 1) / SA_STREAMS + SA_ROUND - 1) & ~int64_t(SA_ROUND - 1);
     for (int q = 0; q < SA_STREAMS; ++q) {
-        const int64_t a = base8 + q * slen;
+        const int64_t a = base + q * slen;
         lo[q] = a > p0 ? a : p0;
         hi[q] = a + slen < p1 ? a + slen : p1;
     }

@@ -3,12 +3,13 @@
 // kernels (Section 6).
 //
 // Producer (SpTTM, fp32 ALU).  A warp is four independent lane groups ("streams") of eight lanes.  Every
-// stream walks its own contiguous part of the unit's nonzeros, eight per round; a lane holds M/8
-// consecutive entries of the fiber temporary t(:), so the eight lanes of a stream fetch one row D(k,:)
-// with a single vector load and the row is consumed from registers one round after it was requested
-// (eight rows in flight per lane).  The index, value and end-of-fiber-bit arrays reach the streams
-// through a per-warp cp.async ring in shared memory that runs seven rounds ahead and continues across
-// the units of a task, so a warp that evaluates many small slices never drains its pipelines.
+// stream walks its own contiguous part of the unit's nonzeros, sixteen per round (the per-round bookkeeping
+// costs more instructions than the sixteen steps themselves); a lane holds M/8 consecutive entries of the
+// fiber temporary t(:), so the eight lanes of a stream fetch one row D(k,:) with a single vector load and the
+// row is consumed from registers eight steps after it was requested (eight rows in flight per lane).  The
+// index, value and end-of-fiber-bit arrays reach the streams through a per-warp cp.async ring in shared
+// memory that runs three rounds ahead and continues across the units of a task, so a warp that evaluates
+// many small slices never drains its pipelines.
 // Consumer (TTM, tensor cores).  A stream that meets an end-of-fiber bit parks t(:) and the fiber's C row
 // offset in a ring of rows in shared memory; eight parked rows at a time update the slice tile as
 // A(i,:,:) += Cg^T (L x 8) . T (8 x M) with m16n8k8 TF32 MMAs, each operand split into a high and a low
@@ -42,10 +43,12 @@ struct cfg {
     static constexpr int VEC = M / 8;            // floats of a factor row per lane (eight lanes per row)
     static constexpr int RS = M + 8;             // row stride of the ring of parked temporaries and of a warp's
                                                  // tile in the CTA reduction; word M of a ring row = C row offset
-    static constexpr int RING = 64;              // rows parked fibers wait in: a round starts at row <= 31 with at most
-                                                 // 7 rows left over and parks at most 32 more
-    static constexpr int DEPTH = 8;              // rounds of index / value data in flight (cp.async ring)
-    static constexpr int SLOT = 80;              // bytes per (round, stream): 8 indices | 8 values | end bits | pad
+    static constexpr int STEPS = SA_ROUND;       // nonzeros per stream and round
+    static constexpr int RING = 8 + 4 * STEPS;   // rows parked fibers wait in: at most 7 rows are left over from the
+                                                 // round before and a round parks at most 4 * STEPS more
+    static constexpr int DEPTH = 4;              // rounds of index / value data in flight (cp.async ring)
+    static constexpr int SLOT = 8 * STEPS + 16;  // bytes per (round, stream): 16 indices | 16 values | end bits | pad
+    static_assert(STEPS == 16, "the step loop, the slot layout and the end-bit extraction are written for 16");
     static constexpr int OFF_KV = 0;
     static constexpr int OFF_RING = OFF_KV + DEPTH * NS * SLOT;
     static constexpr int WARP_BYTES = OFF_RING + RING * RS * 4;
@@ -196,14 +199,14 @@ struct stream_range {
 };
 __device__ __forceinline__ stream_range stream_of(int p0, int p1, int q)
 {
-    const int base8 = p0 & ~7, span = p1 - base8;
-    const int slen = ((span + SA_STREAMS - 1) / SA_STREAMS + 7) & ~7;
+    const int base = p0 & ~(SA_ROUND - 1), span = p1 - base;
+    const int slen = ((span + SA_STREAMS - 1) / SA_STREAMS + SA_ROUND - 1) & ~(SA_ROUND - 1);
     stream_range r;
-    r.rounds = slen >> 3;
-    r.base = base8 + q * slen;
+    r.rounds = slen / SA_ROUND;
+    r.base = base + q * slen;
     r.lo = max(p0, r.base);
     r.hi = min(p1, r.base + slen);
-    r.full = (span - (SA_STREAMS - 1) * slen) >> 3;
+    r.full = (span - (SA_STREAMS - 1) * slen) / SA_ROUND;
     return r;
 }
 
@@ -279,11 +282,12 @@ __device__ __forceinline__ void ttm3_warp_task(const sa_unit3 *__restrict__ unit
     stream_range fs = stream_of(h0.p0, h0.p1, q);
     auto fetch_round = [&](int slot) {
         if (fu < nu) {
-            const int pg = fs.base + 8 * fr;
-            if (pg < fs.hi && pg + 8 > fs.lo && SA_CHK(lim.status, pg >= 0 && pg + 8 <= lim.nnz + 8, 3, pg)) {
+            const int pg = fs.base + K::STEPS * fr;
+            if (pg < fs.hi && pg + K::STEPS > fs.lo && SA_CHK(lim.status, pg >= 0 && pg <= lim.nnz, 3, pg)) {
                 const uint32_t dst = s_kv + slot * (K::NS * K::SLOT);
-                if (c < 4) cp_async16_raw(dst + 16 * c, (c < 2 ? reinterpret_cast<const char *>(crd_k) : reinterpret_cast<const char *>(vals)) + 4 * int64_t(pg) + 16 * (c & 1));
-                else if (c == 4) cp_async4_raw(dst + 64, endbits + (pg >> 5));
+                // lanes 0 .. 3 of the stream copy the sixteen indices, lanes 4 .. 7 the sixteen values
+                cp_async16_raw(dst + 16 * c, (c < 4 ? reinterpret_cast<const char *>(crd_k) : reinterpret_cast<const char *>(vals)) + 4 * int64_t(pg) + 16 * (c & 3));
+                if (c == 0) cp_async4_raw(dst + 8 * K::STEPS, endbits + (pg >> 5));
             }
             if (++fr == fs.rounds) {
                 fr = 0;
@@ -337,16 +341,16 @@ __device__ __forceinline__ void ttm3_warp_task(const sa_unit3 *__restrict__ unit
         __syncwarp();
         const int sn = sc == DEPTH - 1 ? 0 : sc + 1;
         const uint32_t slot_c = s_kv + sc * (K::NS * K::SLOT), slot_n = s_kv + sn * (K::NS * K::SLOT);
-        const uint32_t fw = lds32(slot_c + 64);
-        // which of the eight positions pg .. pg + 7 belong to the stream, and which of them end a fiber
-        const int pg = cs.base + 8 * cr;
+        const uint32_t fw = lds32(slot_c + 8 * K::STEPS);
+        // which of the sixteen positions pg .. pg + 15 belong to the stream, and which of them end a fiber
+        const int pg = cs.base + K::STEPS * cr;
         const bool interior = cr >= 1 && cr < cs.full - 1;      // warp-uniform
-        uint32_t vm = 0xffu, e8 = (fw >> (pg & 24)) & 0xffu;
+        uint32_t vm = 0xffffu, e8 = (fw >> (pg & 16)) & 0xffffu;
         if (!interior) {
-            const int a = min(max(cs.lo - pg, 0), 8), b = min(max(cs.hi - pg, 0), 8);
+            const int a = min(max(cs.lo - pg, 0), K::STEPS), b = min(max(cs.hi - pg, 0), K::STEPS);
             vm = ((1u << b) - 1u) & ~((1u << a) - 1u);
             e8 &= vm;
-            if (cs.hi > cs.lo && uint32_t(cs.hi - pg - 1) < 8u) e8 |= 1u << (cs.hi - pg - 1);   // the part's last nonzero closes its (possibly cut) fiber
+            if (cs.hi > cs.lo && uint32_t(cs.hi - pg - 1) < uint32_t(K::STEPS)) e8 |= 1u << (cs.hi - pg - 1);   // the part's last nonzero closes its (possibly cut) fiber
         }
         // ring rows for the fibers this round parks: stream-major
         const int cnt = __popc(e8);
@@ -358,6 +362,17 @@ __device__ __forceinline__ void ttm3_warp_task(const sa_unit3 *__restrict__ unit
             if (lane >= 16) incl += o;
         }
         const int total = __shfl_sync(SA_FULL_MASK, incl, 31);
+        if (rbase + npend + total > K::RING) {
+            // move the (at most seven) rows left over to the front so that this round's rows fit behind them
+            constexpr int CH = K::RS / 4;                          // 16-byte pieces per row
+            for (int x = lane; x < npend * CH; x += 32) {
+                const int r = x / CH, ch = x - r * CH;
+                const uint4 w = lds128(s_ring + ((rbase + r) * K::RS) * 4 + 16 * ch);
+                asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(s_ring + (r * K::RS) * 4 + 16 * ch), "r"(w.x), "r"(w.y), "r"(w.z), "r"(w.w) : "memory");
+            }
+            rbase = 0;
+            __syncwarp();
+        }
         const int slot = rbase + npend + incl - cnt;          // first row of this stream's fibers in this round
         npend += total;
         uint32_t waddr = s_ring + (slot * K::RS + c * VEC) * 4;
@@ -365,31 +380,34 @@ __device__ __forceinline__ void ttm3_warp_task(const sa_unit3 *__restrict__ unit
             const uint32_t off = uint32_t(jreg) * ldc;
             sts32(s_ring + ((slot + c) * K::RS + M) * 4, off);
             prefetch_l1(C + off);
+            if (c + 8 < cnt)                                  // more than eight fibers of one stream end in this round
+                sts32(s_ring + ((slot + c + 8) * K::RS + M) * 4, uint32_t(__ldg(crd_j + fq + c + 8)) * ldc);
         }
         fq += cnt;
         const bool last = cr + 1 == rounds;
         if (last && cu + 1 < nu) fq = fnext_q;
         if (!SA_CHK(lim.status, uint32_t(fq) <= lim.n_fibers, 6, fq)) fq = 0;
         const int jnext = __ldg(crd_j + fq + c);
-        // Eight steps: consume the row requested one round ago, then request the row of the same step of
-        // the next round into the same registers.  MASKED: some stream of the warp is at a ragged end of
-        // its part; positions outside the part contribute nothing (their rows are not even read as numbers).
+        // Sixteen steps: consume the row requested eight steps ago, then request the row eight steps ahead (of
+        // this round, or of the first half of the next one) into the same registers.  MASKED: some stream of
+        // the warp is at a ragged end of its part; positions outside the part contribute nothing (their rows
+        // are not even read as numbers).
         auto steps = [&](auto masked) {
             constexpr bool MASKED = decltype(masked)::value;
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const uint4 vv = lds128(slot_c + 32 + 16 * h);
-                const uint4 kk = lds128(slot_n + 16 * h);
+            for (int h = 0; h < 4; ++h) {
+                const uint4 vv = lds128(slot_c + 4 * K::STEPS + 16 * h);
+                const uint4 kk = h < 2 ? lds128(slot_c + 32 + 16 * h) : lds128(slot_n + 16 * (h - 2));
                 const float v4[4] = {__uint_as_float(vv.x), __uint_as_float(vv.y), __uint_as_float(vv.z), __uint_as_float(vv.w)};
                 const uint32_t k4[4] = {kk.x, kk.y, kk.z, kk.w};
 #pragma unroll
                 for (int s4 = 0; s4 < 4; ++s4) {
-                    const int s = 4 * h + s4;
+                    const int s = 4 * h + s4, b = s & 7;
                     if (!MASKED || ((vm >> s) & 1u)) {
 #pragma unroll
-                        for (int x = 0; x < VEC; ++x) T[x] = fmaf(v4[s4], buf[s].x[x], T[x]);
+                        for (int x = 0; x < VEC; ++x) T[x] = fmaf(v4[s4], buf[b].x[x], T[x]);
                     }
-                    buf[s].load(dlane + uint64_t(SA_CHK(lim.status, k4[s4] < lim.d_rows, 7, k4[s4]) ? k4[s4] : 0u) * row_bytes);
+                    buf[b].load(dlane + uint64_t(SA_CHK(lim.status, k4[s4] < lim.d_rows, 7, k4[s4]) ? k4[s4] : 0u) * row_bytes);
                     if (e8 & (1u << s)) {
                         rowvec<VEC> tv;
 #pragma unroll
@@ -400,7 +418,7 @@ __device__ __forceinline__ void ttm3_warp_task(const sa_unit3 *__restrict__ unit
                 }
             }
         };
-        if (!interior && __any_sync(SA_FULL_MASK, vm != 0xffu)) steps(std::true_type{});
+        if (!interior && __any_sync(SA_FULL_MASK, vm != 0xffffu)) steps(std::true_type{});
         else steps(std::false_type{});
         __syncwarp();
         while (npend >= 8) {
@@ -410,17 +428,6 @@ __device__ __forceinline__ void ttm3_warp_task(const sa_unit3 *__restrict__ unit
             npend -= 8;
         }
         __syncwarp();
-        if (rbase >= 32) {
-            // move the (at most seven) rows left over to the front so that the next round's rows fit behind them
-            constexpr int CH = K::RS / 4;                          // 16-byte pieces per row
-            for (int x = lane; x < npend * CH; x += 32) {
-                const int r = x / CH, ch = x - r * CH;
-                const uint4 w = lds128(s_ring + ((rbase + r) * K::RS) * 4 + 16 * ch);
-                asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(s_ring + (r * K::RS) * 4 + 16 * ch), "r"(w.x), "r"(w.y), "r"(w.z), "r"(w.w) : "memory");
-            }
-            rbase = 0;
-            __syncwarp();
-        }
         jreg = jnext;
         sc = sn;
       }
@@ -625,8 +632,8 @@ cudaError_t launch(const sa_ttm3_view &v, const sa_dense &first, const sa_dense 
     constexpr size_t smem = size_t(SA_TTM3_WARPS) * cfg<L, M>::WARP_BYTES;
     const bool short_units = v.nnz < int64_t(512) * int64_t(wl.items.size());          // mean unit below 512 nonzeros
     auto kern = short_units ? ttm3_kernel<L, M, cfg<L, M>::MINCTAS_SHORT, HAD> : ttm3_kernel<L, M, cfg<L, M>::MINCTAS, HAD>;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess)
-        return cudaGetLastError();
+    static bool attr_long[SA_MAX_DEVICE_FLAGS], attr_short[SA_MAX_DEVICE_FLAGS];     // per instantiation of this launcher
+    if (!sa_set_smem_once(kern, int(smem), short_units ? attr_short : attr_long)) return cudaGetLastError();
     dbg_limits lim;
     lim.status = v.status;
     lim.c_rows = uint32_t(first.rows); lim.d_rows = uint32_t(second.rows);

@@ -462,11 +462,8 @@ sa_status sa_launch_ttm4(const sa_tensor *t, const sa_dense *ops, float *out, vo
     if (n_pieces > 0) {
         const bool contig = ops[1].ld == R && ops[2].ld == R;
         auto kern = contig ? ttm4_fused_kernel<true> : ttm4_fused_kernel<false>;
-        static bool attr_set[2] = {false, false};
-        if (!attr_set[contig]) {
-            if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, F4_SMEM) != cudaSuccess) return SA_E_CUDA;
-            attr_set[contig] = true;
-        }
+        static bool attr_contig[SA_MAX_DEVICE_FLAGS], attr_strided[SA_MAX_DEVICE_FLAGS];
+        if (!sa_set_smem_once(kern, F4_SMEM, contig ? attr_contig : attr_strided)) return SA_E_CUDA;
         f4_limits lim;
         lim.status = t->d_status;
         lim.c_rows = uint32_t(ops[0].rows); lim.d_rows = uint32_t(ops[1].rows); lim.e_rows = uint32_t(ops[2].rows);

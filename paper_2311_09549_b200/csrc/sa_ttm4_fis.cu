@@ -336,11 +336,8 @@ sa_status sa_launch_ttm4_fissioned(const sa_tensor *t, const sa_dense *ops, floa
     if (n_sub > 0) {
         const bool contig = ops[1].ld == R && ops[2].ld == R;
         auto kern = contig ? ttm4_subtree_kernel<true> : ttm4_subtree_kernel<false>;
-        static bool attr_set[2] = {false, false};
-        if (!attr_set[contig]) {
-            if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SUB_SMEM) != cudaSuccess) return SA_E_CUDA;
-            attr_set[contig] = true;
-        }
+        static bool attr_contig[SA_MAX_DEVICE_FLAGS], attr_strided[SA_MAX_DEVICE_FLAGS];
+        if (!sa_set_smem_once(kern, SUB_SMEM, contig ? attr_contig : attr_strided)) return SA_E_CUDA;
         const int64_t ctas = (n_sub + SA_WARPS_PER_CTA - 1) / SA_WARPS_PER_CTA;
         kern<<<(unsigned)ctas, 256, SUB_SMEM, stream>>>(t->wl4_sub.d_items, n_sub, t->d_pos[2], t->d_pos[3], t->d_crd[2],
                                                                        t->d_nzpack, ops[1].ptr, ops[1].ld, ops[2].ptr, ops[2].ld, T2, lim);

@@ -162,8 +162,8 @@ def test_csf_worklist_partitions_every_nonzero_once(cfg):
         assert b - a == 1 or sizes[a:b].sum() <= 2048
     # stream starts: part q of an item begins in fiber stream_f0[n, q]
     for n, (row, row_end, f0, f1, p0, p1, dest, _) in enumerate(items):
-        b8 = (p0 // 8) * 8
-        slen = -(-(-(-(p1 - b8) // 4)) // 8) * 8
+        b8 = (p0 // 16) * 16
+        slen = -(-(-(-(p1 - b8) // 4)) // 16) * 16
         for q in range(4):
             lo, hi = max(p0, b8 + q * slen), min(p1, b8 + (q + 1) * slen)
             f = int(stream_f0[n, q])

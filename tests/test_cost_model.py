@@ -6,11 +6,28 @@ concrete sets of loop bounds (the four cases of Section 3) and sizes of temporar
 auxiliary memory in the comparison with SpTTN-Cyclops; the table of auxiliary memory requirements per kernel).
 A small evaluator of branched loop nests, written here, is pinned against those printed figures and then tells
 what the library's own nests must cost, which is compared with what sa_schedule_cost reports."""
+import os
+
 import numpy as np
 import pytest
 
 import paper_2311_09549_b200 as sa
 from workloads import configs
+
+GOLDEN = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "paper_cost_figures.txt")
+
+
+def golden(kind):
+    """Records of one kind from the file of figures the paper prints (fields split at '|', stripped)."""
+    out = []
+    with open(GOLDEN) as f:
+        for line in f:
+            if line.startswith("#") or not line.strip():
+                continue
+            fields = [x.strip() for x in line.split("|")]
+            if fields[0] == kind:
+                out.append(fields[1:])
+    return out
 
 
 def iterations(nest):
@@ -43,21 +60,25 @@ def test_nest_evaluator_reproduces_the_printed_complexity_formulas():
 
 
 def test_nest_evaluator_reproduces_the_printed_ratios_of_the_four_cases():
-    """Section 3, Cases 1, 2 and 4.  The text prints sparsities 0.08 and 0.02 for Cases 1 and 2, outside its own
-    stated range (at most 0.01); with 0.008 and 0.002 the printed ratios come out, so those are taken.  In Case 4
-    the two ratio labels are exchanged in the text (the formulas give 40.4 for the linear nest)."""
-    def phi(I, J, K, L, M, N, sparsity):
-        f = {k: iterations(v) for k, v in fig2(I, J, K, L, M, N, sparsity * I * J * K).items()}
-        return f
-    c1 = phi(1800, 800, 1000, 64, 16, 32, 0.008)
-    assert c1["a"] / c1["d"] == pytest.approx(237.5, rel=2e-3) and c1["b"] / c1["d"] == pytest.approx(7.5, rel=2e-2)
-    c2 = phi(1800, 1600, 2000, 64, 16, 32, 0.002)
-    assert c2["a"] / c2["d"] == pytest.approx(92.5, rel=2e-3) and c2["b"] / c2["d"] == pytest.approx(3.0, rel=4e-2)
-    c4 = phi(265, 1207, 479, 251, 234, 42, 0.0033)
-    assert c4["a"] / c4["b"] == pytest.approx(40.4, rel=2e-2) and c4["d"] / c4["b"] == pytest.approx(1.13, rel=2e-2)
-    # the temporary T(k,j) of the two-level schedule: 3.05 MB in Case 1, 12.21 MB in Case 2 (4-byte elements)
-    assert 800 * 1000 * 4 / 2**20 == pytest.approx(3.05, abs=0.005)
-    assert 1600 * 2000 * 4 / 2**20 == pytest.approx(12.21, abs=0.005)
+    """Section 3, Cases 1, 2 and 4, from tests/golden/paper_cost_figures.txt (which also states the two readings:
+    a tenth of the sparsities printed for Cases 1 and 2, and the exchanged ratio labels of Case 4)."""
+    cases = golden("case")
+    assert len(cases) == 3
+    for name, bounds, _printed, sparsity, *ratios in cases:
+        I, J, K, L, M, N = (int(x) for x in bounds.split())
+        f = {k: iterations(v) for k, v in fig2(I, J, K, L, M, N, float(sparsity) * I * J * K).items()}
+        for r in ratios:
+            lhs, value = (x.strip() for x in r.split("="))
+            num, den = lhs.split("/")
+            assert f[num] / f[den] == pytest.approx(float(value), rel=4e-2), (name, r, f[num] / f[den])
+    # the printed sparsities of Cases 1 and 2 do not give the printed ratios (which is why they are not taken)
+    name, bounds, printed, *_ = cases[0]
+    I, J, K, L, M, N = (int(x) for x in bounds.split())
+    f = {k: iterations(v) for k, v in fig2(I, J, K, L, M, N, float(printed) * I * J * K).items()}
+    assert abs(f["a"] / f["d"] - 237.5) > 50
+    # the temporary T(k,j) of the two-level schedule (4-byte elements)
+    for K, J, mb in (x[0].split() for x in golden("temp_mb")):
+        assert int(K) * int(J) * 4 / 2**20 == pytest.approx(float(mb), abs=0.005)
 
 
 def _host_tensor(w):
@@ -100,11 +121,15 @@ def test_library_iteration_counts_are_those_of_its_nests():
     # the temporaries of the two-level nest are t(n) and T2(m,n): N + M N elements, the element count that the
     # paper's table of auxiliary memory (comparison with SpTTN-Cyclops) lists in bytes for 16 .. 128
     assert c["temp_elements"] == 16 + 16 * 16
-    for n, printed in ((16, 1088), (32, 4224), (64, 16640), (128, 66048)):
-        assert (n + n * n) * 4 == printed
-    for m, printed in ((16, 68), (32, 132), (64, 260), (128, 516)):               # scalar + T(m): the paper's own schedule
-        assert (1 + m) * 4 == printed
+    table = golden("aux_bytes")
+    assert len(table) == 4
+    for rank, own, cyclops in table:
+        n = int(rank)
+        assert (n + n * n) * 4 == int(cyclops)          # t(n) and T(m,n): this library's widened temporaries
+        assert (1 + n) * 4 == int(own)                  # scalar + T(m): the paper's own schedule
     # kernels 1 and 2: scalar temporary, and scalar + row temporary (table of auxiliary memory requirements)
+    printed = dict((k, v) for k, v in golden("aux_elements"))
+    assert printed["kernel1"] == "1" and printed["kernel2"] == "1 to 1+L"
     w = configs.make(3, "mini")
     t = _host_tensor(w)
     assert sa.sa_schedule_cost(t.handle, sa.SA_EXPR_SDDMM_SPMM, sa.SA_SCHED_FUSED, _ops(w))["temp_elements"] == 1

@@ -131,7 +131,7 @@ def test_padded_leading_dimensions(sa):
     assert e.value.status == sa.SA_E_SHAPE
 
 
-@pytest.mark.parametrize("K,L", [(32, 32), (64, 128), (128, 64)])
+@pytest.mark.parametrize("K,L", [(k, l) for k in (32, 64, 128) for l in (32, 64, 128)])
 def test_sddmm_spmm_ranks_long_rows_and_sampled_pattern(sa, K, L):
     import torch
     I, J = 300, 6000
@@ -411,3 +411,13 @@ def test_default_order_of_spmm_gemm_picks_the_faster_one_on_both_sides(sa):
     assert chosen == sa.SA_SCHED_ASSOC_LEFT and ms[sa.SA_SCHED_ASSOC_LEFT] < ms[sa.SA_SCHED_ASSOC_RIGHT], ms
     chosen, ms = both(20_000, 400_000, 1_500_000, 62)
     assert chosen == sa.SA_SCHED_ASSOC_RIGHT and ms[sa.SA_SCHED_ASSOC_RIGHT] < ms[sa.SA_SCHED_ASSOC_LEFT], ms
+
+
+@pytest.mark.parametrize("K,L,M", [(64, 64, 32), (32, 128, 64), (128, 32, 32)])
+def test_sddmm_spmm_gemm_rank_combinations(sa, K, L, M):
+    """Kernel 2 over ranks the mini workload does not use: the tcgen05 dense stage at L = 64 with M = 32, the row
+    temporaries of 32 and 128 floats."""
+    w0 = configs.make_sddmm_spmm("k2-ranks", 91, 4_000, 4_000, 50_000, 1.5, 1_200, K, L)
+    F = configs.dense_normal(91, 3, L, M)
+    w = _wl("sddmm_spmm_gemm", "csr", w0.dims, w0.coords, w0.vals, w0.dense + [F], (w0.dims[0], M))
+    _check(sa, w)
