@@ -37,9 +37,9 @@ FALLBACK_HBM_GBS = 6650.0
 # source file still has the hash it had when the counters were taken; otherwise `traffic` is null.  Workloads 4 and 5
 # are captured at a quarter of their size (--scale mid) and scaled by the nonzeros, see the profiles.
 NCU_TRAFFIC = {
-    2: {"kernel": "ttm3_kernel<32,32> (98.5 % of the step)", "source": "paper_2311_09549_b200/csrc/sa_ttm3.cu",
-        "sha256": "af4a25219f07837e9092aca54ff9ea55ba69cb5e7ed164513575012bddb546ec",
-        "dram_bytes": 848247808, "profile": "profiles/ttm3_kernel_cfg2.md"},
+    2: {"kernel": "ttm3_kernel<32,32> (98.4 % of the step)", "source": "paper_2311_09549_b200/csrc/sa_ttm3.cu",
+        "sha256": "ad4a961ff060c1a94169e3e9d2ed35d4fa41685769def36ea8d9744050c7ac0e",
+        "dram_bytes": 853379328, "profile": "profiles/ttm3_kernel_cfg2.md"},
     3: {"kernel": "sddmm_spmm_kernel<64,64> (99.6 % of the step)", "source": "paper_2311_09549_b200/csrc/sa_sddmm_spmm.cu",
         "sha256": "7c9971e0e72e49dfbb4404b68def327568372ea956767048b5d3d830810b8ead",
         "dram_bytes": 13186066944, "profile": "profiles/sddmm_spmm_kernel_cfg3.md"},
@@ -50,15 +50,15 @@ NCU_TRAFFIC = {
                    "source": "paper_2311_09549_b200/csrc/sa_spmm_gemm.cu", "sha256": "a7d3ddb4c4f3e2c41bc5f803c06e42250d24443649e1f4c918744c74fbb8b39f",
                    "dram_bytes": 4 * 4974276864, "profile": "profiles/spmm_gemm_kernels_cfg4.md"},
     (5, "fused"): {"kernel": "ttm4_fused_kernel (94 % of the step; counters of the quarter-size case x 4)",
-                   "source": "paper_2311_09549_b200/csrc/sa_ttm4.cu", "sha256": "97022d6fa719293c229dc5e2d93ca15ae4c4ac958aa96d03b58b1b36d5fc2da3",
-                   "dram_bytes": 4 * 424575488, "profile": "profiles/ttm4_kernels_cfg5.md"},
+                   "source": "paper_2311_09549_b200/csrc/sa_ttm4.cu", "sha256": "77b9b58137c8e565f84a5ffd8762e5448c910f5befc50c3838442ae6007d0823",
+                   "dram_bytes": 4 * 424084480, "profile": "profiles/ttm4_kernels_cfg5.md"},
     (5, "fissioned"): {"kernel": "ttm4_subtree_kernel (pass 1 on the small subtrees, 51 % of the step; counters of the "
                                  "quarter-size case x 4)",
-                       "source": "paper_2311_09549_b200/csrc/sa_ttm4_fis.cu", "sha256": "6cd1680b60cc8a1c0240b7d13638a8dcca5f99c35a48a9b7a50a9aed7424ebd7",
-                       "dram_bytes": 4 * 670214912, "profile": "profiles/ttm4_kernels_cfg5.md"},
+                       "source": "paper_2311_09549_b200/csrc/sa_ttm4_fis.cu", "sha256": "330c537c47ea8e58b5e16d2de6016edd8084712e73f0124a737a8869b77cba4f",
+                       "dram_bytes": 4 * 671109120, "profile": "profiles/ttm4_kernels_cfg5.md"},
     10: {"kernel": "fiber_spmm_kernel<32> (99 % of the step)", "source": "paper_2311_09549_b200/csrc/sa_spmm_gemm.cu",
-         "sha256": "408ed3d1f40077ca8fcb6e4ebeb2dc9b8ca08986b342d17b370a87df4d7b251e",
-         "dram_bytes": 955500000, "profile": "profiles/fiber_spmm_kernel_w10.md"},
+         "sha256": "a7d3ddb4c4f3e2c41bc5f803c06e42250d24443649e1f4c918744c74fbb8b39f",
+         "dram_bytes": 955089920, "profile": "profiles/fiber_spmm_kernel_w10.md"},
 }
 
 
@@ -324,9 +324,40 @@ def l2_gather_ceiling(sa, torch, w, tensor, ops, dev, stream):
                     sweep.append({"indices": name, "lanes_per_row": lanes, "rows_in_flight": inflight, "blocks_per_sm": bps,
                                   "ms": round(ms, 4), "gbs": round(nbytes / (ms * 1e-3) / 1e9, 1)})
     best = min(sweep, key=lambda r: r["ms"])
+    # the same rows through the copy engine (cp.async.bulk.tensor tile::gather4 into shared memory, read back from there)
+    lib.sa_probe_tma_gather.argtypes = [vp, i64, i64, ci, vp, i64, vp, ci, ci, vp, vp]
+    lib.sa_probe_tma_gather.restype = ci
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    sink2 = torch.zeros(2, dtype=torch.float32, device=dev)
+    idx = streams["the tensor's last-mode indices in storage order"]
+    tma = []
+    for stages in (1, 2, 4):
+        for bps in (2, 4, 8):
+            def run():
+                rc = lib.sa_probe_tma_gather(table.data_ptr(), rows, table.stride(0), cols, idx.data_ptr(), n, sink2.data_ptr(),
+                                             stages, bps, status.data_ptr(), stream.cuda_stream)
+                if rc != 0:
+                    raise RuntimeError("copy-engine probe launch failed (%d)" % rc)
+            run()
+            torch.cuda.synchronize(dev)
+            if int(status[0]) != 0:
+                raise RuntimeError("copy-engine probe gave up waiting for its rows (status %d)" % int(status[0]))
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            reps = 3
+            for _ in range(reps):
+                run()
+            e1.record(stream)
+            torch.cuda.synchronize(dev)
+            ms = e0.elapsed_time(e1) / reps
+            tma.append({"groups_of_16_rows_in_flight_per_warp": stages, "blocks_of_4_warps_per_sm": bps, "ms": round(ms, 4),
+                        "gbs": round(nbytes / (ms * 1e-3) / 1e9, 1)})
     return {"what": "bare gather of one %d-byte factor row per nonzero from the L2-resident %d x %d table "
                     "(plus 4 index bytes per row from HBM); best of %d shapes" % (cols * 4, rows, cols, len(sweep)),
-            "ms": best["ms"], "gbs": best["gbs"], "best": best, "sweep": sweep}
+            "ms": best["ms"], "gbs": best["gbs"], "best": best, "sweep": sweep,
+            "copy_engine_gather4": {"what": "the same rows fetched four per instruction by the copy engine into shared memory and "
+                                            "read back from there (the tensor's own indices)",
+                                    "ms": min(r["ms"] for r in tma), "sweep": tma}}
 
 
 def aggregate_throughput(nnz_per_rank, world, ms_per_step):
