@@ -70,3 +70,17 @@ def test_checked_build_runs_clean_and_agrees_with_the_oracle():
                PYTHONPATH=os.pathsep.join([ROOT, os.path.join(ROOT, "tests"), os.environ.get("PYTHONPATH", "")]))
     r = subprocess.run([sys.executable, "-c", CHILD], env=env, cwd=ROOT, capture_output=True, text=True, timeout=900)
     assert r.returncode == 0 and "CHECKED-OK" in r.stdout, r.stdout[-2000:] + "\n" + r.stderr[-4000:]
+
+
+def test_random_sweep_under_the_checked_build():
+    """The randomised shapes of test_gpu_random.py once more with every device-side index check compiled in (its
+    helper asserts that the status word stays SA_OK after each run)."""
+    import importlib.util
+    spec = importlib.util.spec_from_file_location("_sa_build", os.path.join(ROOT, "paper_2311_09549_b200", "build.py"))
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    lib = mod.build_checked()
+    env = dict(os.environ, SPARSEAUTO_LIB=lib)
+    r = subprocess.run([sys.executable, "-m", "pytest", os.path.join(ROOT, "tests", "test_gpu_random.py"), "-x", "-q", "-m", "gpu",
+                        "-p", "no:cacheprovider"], env=env, cwd=ROOT, capture_output=True, text=True, timeout=900)
+    assert r.returncode == 0 and " passed" in r.stdout, r.stdout[-3000:] + "\n" + r.stderr[-2000:]
