@@ -79,7 +79,7 @@ def _compile(extra, verbose, LIB, tag):
     if failed:
         raise RuntimeError("nvcc failed")
     tmp = LIB + ".tmp%d" % os.getpid()
-    subprocess.check_call([nvcc, "-shared", "-o", tmp] + objs + ["-Xcompiler", "-fopenmp", "-lgomp"])
+    subprocess.check_call([nvcc, "-Wno-deprecated-gpu-targets", "-shared", "-o", tmp] + objs + ["-Xcompiler", "-fopenmp", "-lgomp"])
     os.replace(tmp, LIB)
     return LIB
 

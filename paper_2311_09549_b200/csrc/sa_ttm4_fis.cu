@@ -29,102 +29,184 @@ struct fis_limits {
     int32_t n_subtrees, n_fibers, n_slots, nnz;
 };
 
-// Values one group of eight fibers contributes to a lane's MMA fragments: C(j,:) entries for the A operand
-// (fibers t and t + 4 of the group, columns g and g + 8) and T2 entries for the B operand (same two
-// fibers, column 8 nt + g of the item's quarter).  Fibers past the end of the item read as zero.
-struct group_vals {
-    float c[4];
-    float b[NT4][2];
+// Pass 2.  One warp per item (fibers [f0, f1) of one slice, quarter `pad` of the temporaries' columns; `pad` = 4:
+// all four quarters, one after the other, for pieces of at most eight fibers); warps take items in a grid-wide
+// stride, largest items first.  Seen from a warp, its items are one sequence of groups (item, quarter, eight fibers).
+// The temporaries of a group (8 rows of 64 floats) are copied to shared memory with cp.async three groups ahead of
+// their use, across quarter and item boundaries, so that the stream of 1 KB tiles out of HBM never stops at the many
+// short items; the C values of a group (a few gathered words out of L2) are loaded one group ahead into registers.
+constexpr int SL_DEPTH = 4;                        // stages of the shared-memory ring (groups in flight + 1)
+constexpr int SL_RS = QC + 8;                      // row stride in floats: rows t and t + 1 land 8 banks apart
+constexpr int SL_STAGE = 8 * SL_RS;                // floats per stage
+constexpr int SL_SMEM = SA_WARPS_PER_CTA * SL_DEPTH * SL_STAGE * int(sizeof(float));   // 72 KB
+
+// Position in a warp's sequence of groups.
+struct sl_cursor {
+    int64_t n;              // item
+    int row, dest;          // its output slice and partial slot (< 0: none)
+    int f0, f1, f;          // its fibers, and the first fiber of the current group
+    int qc, q_last;         // current and last quarter
+    bool live;
 };
 
-__device__ __forceinline__ void load_group(group_vals &v, int f, int f1, int lane, const int32_t *__restrict__ crd_j,
-                                           const float *__restrict__ C, uint32_t ldc, const float *__restrict__ t2q,
-                                           const fis_limits &lim)
+__device__ __forceinline__ void sl_load_item(sl_cursor &c, const sa_item *__restrict__ items, int64_t n_items, int64_t stride,
+                                             const fis_limits &lim)
 {
-    const int g = lane >> 2, t = lane & 3;
-    const int fa = f + t, fb = f + t + 4;
-    const bool va = fa < f1, vb = fb < f1;
-    uint32_t ja = uint32_t(va ? __ldg(crd_j + fa) : 0), jb = uint32_t(vb ? __ldg(crd_j + fb) : 0);
-    if (!SA_CHK(lim.status, ja < lim.c_rows, 71, ja)) ja = 0u;
-    if (!SA_CHK(lim.status, jb < lim.c_rows, 71, jb)) jb = 0u;
-    const float *ca = C + ja * ldc + g;
-    const float *cb = C + jb * ldc + g;
-    v.c[0] = va ? __ldg(ca) : 0.f;
-    v.c[1] = va ? __ldg(ca + 8) : 0.f;
-    v.c[2] = vb ? __ldg(cb) : 0.f;
-    v.c[3] = vb ? __ldg(cb + 8) : 0.f;
-    const float *ra = t2q + int64_t(va ? fa : f) * T2F + g;
-    const float *rb = t2q + int64_t(vb ? fb : f) * T2F + g;
-#pragma unroll
-    for (int nt = 0; nt < NT4; ++nt) {
-        const float xa = __ldcs(ra + 8 * nt), xb = __ldcs(rb + 8 * nt);       // read once: streaming
-        v.b[nt][0] = va ? xa : 0.f;
-        v.b[nt][1] = vb ? xb : 0.f;
+    for (;;) {
+        c.live = c.n < n_items;
+        if (!c.live) return;
+        const int4 ia = __ldg(reinterpret_cast<const int4 *>(items + c.n));          // out_row, row_end, f0, f1
+        const int4 ib = __ldg(reinterpret_cast<const int4 *>(items + c.n) + 1);      // p0, p1, dest, quarter
+        if (SA_CHK(lim.status, ia.z >= 0 && ia.z <= ia.w && ia.w <= lim.n_subtrees && uint32_t(ib.w) <= 4u && uint32_t(ia.x) < lim.n_slices &&
+                                   ib.z < lim.n_slots, 72, c.n)) {
+            c.row = ia.x; c.dest = ib.z;
+            c.f0 = c.f = ia.z; c.f1 = ia.w;
+            c.qc = ib.w == 4 ? 0 : ib.w;
+            c.q_last = ib.w == 4 ? 3 : ib.w;
+            return;
+        }
+        c.n += stride;          // a record that fails its check is skipped
     }
 }
 
-// Pass 2.  One warp per item (fibers [f0, f1) of one slice, quarter `pad` of the temporaries' columns);
-// warps take items in a grid-wide stride, largest items first.
+// To the next group: eight fibers on, else the next quarter of the item, else the next item of the warp.
+__device__ __forceinline__ void sl_advance(sl_cursor &c, const sa_item *__restrict__ items, int64_t n_items, int64_t stride,
+                                           const fis_limits &lim)
+{
+    c.f += 8;
+    if (c.f < c.f1) return;
+    c.f = c.f0;
+    if (++c.qc <= c.q_last) return;
+    c.n += stride;
+    sl_load_item(c, items, n_items, stride, lim);
+}
+
+// The C entries of a group for a lane's A fragments: fibers t and t + 4 of the group, columns g and g + 8; fibers
+// past the end of the item read as zero.  Two dependent gathers (the fiber's j, then C(j,:)), taken in two steps one
+// group apart so that neither latency lies between two groups' products.
+__device__ __forceinline__ void sl_load_j(uint32_t (&j)[2], const sl_cursor &cur, int lane, const int32_t *__restrict__ crd_j,
+                                          const fis_limits &lim)
+{
+    const int t = lane & 3;
+    const int fa = cur.f + t, fb = cur.f + t + 4;
+    const bool va = cur.live && fa < cur.f1, vb = cur.live && fb < cur.f1;
+    j[0] = uint32_t(va ? __ldg(crd_j + fa) : 0);
+    j[1] = uint32_t(vb ? __ldg(crd_j + fb) : 0);
+    if (!SA_CHK(lim.status, j[0] < lim.c_rows, 71, j[0])) j[0] = 0u;
+    if (!SA_CHK(lim.status, j[1] < lim.c_rows, 71, j[1])) j[1] = 0u;
+}
+__device__ __forceinline__ void sl_load_c(float (&c)[4], const uint32_t (&j)[2], const sl_cursor &cur, int lane,
+                                          const float *__restrict__ C, uint32_t ldc)
+{
+    const int g = lane >> 2, t = lane & 3;
+    const bool va = cur.live && cur.f + t < cur.f1, vb = cur.live && cur.f + t + 4 < cur.f1;
+    const float *ca = C + j[0] * ldc + g;
+    const float *cb = C + j[1] * ldc + g;
+    c[0] = va ? __ldg(ca) : 0.f;
+    c[1] = va ? __ldg(ca + 8) : 0.f;
+    c[2] = vb ? __ldg(cb) : 0.f;
+    c[3] = vb ? __ldg(cb + 8) : 0.f;
+}
+
+// Copies of the group's eight quarter rows into a stage: 128 pieces of 16 bytes, four per lane; rows past the end of
+// the item are filled with zeros (their C entries are zero too, but what the stage held before need not be finite).
+__device__ __forceinline__ void sl_issue(const sl_cursor &cur, uint32_t stage, int lane, const float *__restrict__ T2)
+{
+    if (cur.live) {
+        const int piece = lane & 15;
+        const float *src = T2 + int64_t(cur.f) * T2F + cur.qc * QC + 4 * piece;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int r = (lane >> 4) + 2 * i;
+            const uint32_t dst = stage + uint32_t(r * SL_RS + 4 * piece) * 4u;
+            if (cur.f + r < cur.f1) cp_async16_raw(dst, src + int64_t(r) * T2F);
+            else asm volatile("st.shared.v4.f32 [%0], {%1,%1,%1,%1};" ::"r"(dst), "f"(0.f) : "memory");
+        }
+    }
+    cp_async_commit();
+}
+
 __global__ void __launch_bounds__(256, 2)
 ttm4_slice_kernel(const sa_item *__restrict__ items, int64_t n_items, const int32_t *__restrict__ crd_j,
                   const float *__restrict__ T2, const float *__restrict__ C, uint32_t ldc, float *__restrict__ out,
                   float *__restrict__ partial, const fis_limits lim)
 {
-    const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+    extern __shared__ __align__(16) float sl_smem[];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane >> 2, t = lane & 3;
     const int64_t stride = int64_t(gridDim.x) * SA_WARPS_PER_CTA;
-    for (int64_t n = int64_t(blockIdx.x) * SA_WARPS_PER_CTA + (threadIdx.x >> 5); n < n_items; n += stride) {
-        const int4 ia = __ldg(reinterpret_cast<const int4 *>(items + n));          // out_row, row_end, f0, f1
-        const int4 ib = __ldg(reinterpret_cast<const int4 *>(items + n) + 1);      // p0, p1, dest, quarter
-        const int f0 = ia.z, f1 = ia.w;
-        if (!SA_CHK(lim.status, f0 >= 0 && f0 <= f1 && f1 <= lim.n_subtrees && uint32_t(ib.w) <= 4u && uint32_t(ia.x) < lim.n_slices &&
-                                    ib.z < lim.n_slots, 72, n))
-            continue;
-        // quarter 4 = all four quarters, one after the other (pieces of at most eight fibers: one record, one set of
-        // C values and one latency chain instead of four)
-        const int q_first = ib.w == 4 ? 0 : ib.w, q_last = ib.w == 4 ? 3 : ib.w;
-#pragma unroll 1
-        for (int qc = q_first; qc <= q_last; ++qc) {
-        const float *t2q = T2 + qc * QC;
-        float acc[NT4][4];
+    const uint32_t ring = smem_u32(sl_smem) + uint32_t(warp) * uint32_t(SL_DEPTH * SL_STAGE * 4);
+    sl_cursor prod, cons, next, next2;               // groups i + 3, i, i + 1, i + 2
+    prod.n = int64_t(blockIdx.x) * SA_WARPS_PER_CTA + warp;
+    sl_load_item(prod, items, n_items, stride, lim);
+    cons = next = prod;
+    if (!cons.live) return;
+    // the first SL_DEPTH - 1 groups go out before anything is consumed
 #pragma unroll
-        for (int nt = 0; nt < NT4; ++nt)
+    for (int s = 0; s < SL_DEPTH - 1; ++s) {
+        sl_issue(prod, ring + uint32_t(s * SL_STAGE * 4), lane, T2);
+        if (prod.live) sl_advance(prod, items, n_items, stride, lim);
+    }
+    float cc[4], cn[4];
+    uint32_t jc[2], jn[2], jn2[2];
+    sl_load_j(jc, cons, lane, crd_j, lim);
+    sl_advance(next, items, n_items, stride, lim);
+    sl_load_j(jn, next, lane, crd_j, lim);
+    sl_load_c(cc, jc, cons, lane, C, ldc);
+    next2 = next;
+    if (next2.live) sl_advance(next2, items, n_items, stride, lim);
+    float acc[NT4][4];
 #pragma unroll
-            for (int x = 0; x < 4; ++x) acc[nt][x] = 0.f;
-        group_vals cur, nxt;
-        load_group(cur, f0, f1, lane, crd_j, C, ldc, t2q, lim);
-        nxt = cur;
-#pragma unroll 1
-        for (int f = f0; f < f1; f += 8) {
-            if (f + 8 < f1) load_group(nxt, f + 8, f1, lane, crd_j, C, ldc, t2q, lim);   // in flight during the products below
-            uint32_t ah[4], al[4];
+    for (int nt = 0; nt < NT4; ++nt)
 #pragma unroll
-            for (int x = 0; x < 4; ++x) split_tf32(cur.c[x], ah[x], al[x]);
+        for (int x = 0; x < 4; ++x) acc[nt][x] = 0.f;
+    int sc = 0;                                       // stage of the group being consumed
+    while (cons.live) {
+        __syncwarp();                                 // every lane is done with the stage that is filled next
+        sl_issue(prod, ring + uint32_t((sc == 0 ? SL_DEPTH - 1 : sc - 1) * SL_STAGE * 4), lane, T2);
+        if (prod.live) sl_advance(prod, items, n_items, stride, lim);
+        sl_load_j(jn2, next2, lane, crd_j, lim);                  // both in flight during the products below
+        sl_load_c(cn, jn, next, lane, C, ldc);
+        cp_async_wait<SL_DEPTH - 1>();
+        __syncwarp();
+        const float *st = sl_smem + (warp * SL_DEPTH + sc) * SL_STAGE;
+        uint32_t ah[4], al[4];
 #pragma unroll
-            for (int nt = 0; nt < NT4; ++nt) {
-                uint32_t bh[2], bl[2];
-                split_tf32(cur.b[nt][0], bh[0], bl[0]);
-                split_tf32(cur.b[nt][1], bh[1], bl[1]);
-                mma_m16n8k8_tf32(acc[nt], al, bh);
-                mma_m16n8k8_tf32(acc[nt], ah, bl);
-                mma_m16n8k8_tf32(acc[nt], ah, bh);
-            }
-            cur = nxt;
-        }
-        // element (l, column 64 qc + 8 nt + 2 t (+1)) of the slice tile, l = g and g + 8
-        float *dst = (ib.z >= 0 ? partial + int64_t(ib.z) * TILE4 : out + int64_t(ia.x) * TILE4) + qc * QC + 2 * t;
+        for (int x = 0; x < 4; ++x) split_tf32(cc[x], ah[x], al[x]);
 #pragma unroll
         for (int nt = 0; nt < NT4; ++nt) {
-            const float2 lo = make_float2(acc[nt][0], acc[nt][1]), hi = make_float2(acc[nt][2], acc[nt][3]);
-            if (ib.z >= 0) {
-                *reinterpret_cast<float2 *>(dst + g * T2F + 8 * nt) = lo;
-                *reinterpret_cast<float2 *>(dst + (g + 8) * T2F + 8 * nt) = hi;
-            } else {
-                sa_st_cs2(dst + g * T2F + 8 * nt, lo);
-                sa_st_cs2(dst + (g + 8) * T2F + 8 * nt, hi);
+            uint32_t bh[2], bl[2];
+            split_tf32(st[t * SL_RS + 8 * nt + g], bh[0], bl[0]);
+            split_tf32(st[(t + 4) * SL_RS + 8 * nt + g], bh[1], bl[1]);
+            mma_m16n8k8_tf32(acc[nt], al, bh);
+            mma_m16n8k8_tf32(acc[nt], ah, bl);
+            mma_m16n8k8_tf32(acc[nt], ah, bh);
+        }
+        if (cons.f + 8 >= cons.f1) {
+            // the quarter's last group: element (l, column 64 qc + 8 nt + 2 t (+1)) of the slice tile, l = g and g + 8
+            float *dst = (cons.dest >= 0 ? partial + int64_t(cons.dest) * TILE4 : out + int64_t(cons.row) * TILE4) + cons.qc * QC + 2 * t;
+#pragma unroll
+            for (int nt = 0; nt < NT4; ++nt) {
+                const float2 lo = make_float2(acc[nt][0], acc[nt][1]), hi = make_float2(acc[nt][2], acc[nt][3]);
+                if (cons.dest >= 0) {
+                    *reinterpret_cast<float2 *>(dst + g * T2F + 8 * nt) = lo;
+                    *reinterpret_cast<float2 *>(dst + (g + 8) * T2F + 8 * nt) = hi;
+                } else {
+                    sa_st_cs2(dst + g * T2F + 8 * nt, lo);
+                    sa_st_cs2(dst + (g + 8) * T2F + 8 * nt, hi);
+                }
+#pragma unroll
+                for (int x = 0; x < 4; ++x) acc[nt][x] = 0.f;
             }
         }
-        }
+        cons = next;
+        next = next2;
+        if (next2.live) sl_advance(next2, items, n_items, stride, lim);
+#pragma unroll
+        for (int x = 0; x < 4; ++x) cc[x] = cn[x];
+        jn[0] = jn2[0]; jn[1] = jn2[1];
+        sc = sc == SL_DEPTH - 1 ? 0 : sc + 1;
     }
+    cp_async_wait<0>();
 }
 
 // Pass 1 on whole (i,j) subtrees (tensors whose subtrees are all small: the usual case, a subtree holds a few
@@ -357,8 +439,10 @@ sa_status sa_launch_ttm4_fissioned(const sa_tensor *t, const sa_dense *ops, floa
         int dev = 0, sms = 148;
         if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
         const int64_t ctas = std::min<int64_t>((n_items + SA_WARPS_PER_CTA - 1) / SA_WARPS_PER_CTA, int64_t(sms) * 2);
-        ttm4_slice_kernel<<<(unsigned)ctas, 256, 0, stream>>>(wl.d_items, n_items, t->d_crd[1], T2, ops[0].ptr, uint32_t(ops[0].ld),
-                                                            out, part2, lim);
+        static bool attr_slice[SA_MAX_DEVICE_FLAGS];
+        if (!sa_set_smem_once(ttm4_slice_kernel, SL_SMEM, attr_slice)) return SA_E_CUDA;
+        ttm4_slice_kernel<<<(unsigned)ctas, 256, SL_SMEM, stream>>>(wl.d_items, n_items, t->d_crd[1], T2, ops[0].ptr, uint32_t(ops[0].ld),
+                                                                  out, part2, lim);
         if (cudaGetLastError() != cudaSuccess) return SA_E_CUDA;
         *launches += 1;
     }
