@@ -165,20 +165,29 @@ __device__ __forceinline__ void had_flush(float &hacc, const float *__restrict__
     }
 }
 
-// Store a slice tile held as MMA accumulator fragments (streaming stores: the output is written once).
+// Store a slice tile held as MMA accumulator fragments (streaming stores: the output is written once).  The
+// fragments go through the warp's ring of parked rows (empty at the end of a unit), so that every store instruction
+// writes 512 contiguous bytes of the tile instead of eight 32-byte pieces of eight rows.
 template <int L, int M>
-__device__ __forceinline__ void store_tile(const float (&acc)[cfg<L, M>::MT][cfg<L, M>::NT][4], float *__restrict__ dst, int lane)
+__device__ __forceinline__ void store_tile(const float (&acc)[cfg<L, M>::MT][cfg<L, M>::NT][4], float *__restrict__ dst, int lane,
+                                           float *__restrict__ ring)
 {
     using K = cfg<L, M>;
+    static_assert(L * K::RS <= K::RING * K::RS, "the tile fits the ring");
     const int g = lane >> 2, t = lane & 3;
 #pragma unroll
     for (int mt = 0; mt < K::MT; ++mt)
 #pragma unroll
         for (int nt = 0; nt < K::NT; ++nt) {
             const int l = 16 * mt + g, mm = 8 * nt + 2 * t;
-            sa_st_cs2(dst + l * M + mm, make_float2(acc[mt][nt][0], acc[mt][nt][1]));
-            sa_st_cs2(dst + (l + 8) * M + mm, make_float2(acc[mt][nt][2], acc[mt][nt][3]));
+            *reinterpret_cast<float2 *>(ring + l * K::RS + mm) = make_float2(acc[mt][nt][0], acc[mt][nt][1]);
+            *reinterpret_cast<float2 *>(ring + (l + 8) * K::RS + mm) = make_float2(acc[mt][nt][2], acc[mt][nt][3]);
         }
+    __syncwarp();
+#pragma unroll
+    for (int x = 4 * lane; x < L * M; x += 128)
+        sa_st_cs4(dst + x, *reinterpret_cast<const float4 *>(ring + (x / M) * K::RS + (x % M)));
+    __syncwarp();
 }
 
 template <int L, int M>
@@ -454,7 +463,7 @@ __device__ __forceinline__ void ttm3_warp_task(const sa_unit3 *__restrict__ unit
                 if (SA_CHK(lim.status, uint32_t(crow) < lim.n_slices_dim, 8, crow)) ttmc_accumulate<L, M>(acc, *sink, crow, lane);
                 zero_tile<L, M>(acc);
             } else {
-                if (SA_CHK(lim.status, uint32_t(crow) < lim.n_slices_dim, 8, crow)) store_tile<L, M>(acc, out + int64_t(crow) * (L * M), lane);
+                if (SA_CHK(lim.status, uint32_t(crow) < lim.n_slices_dim, 8, crow)) store_tile<L, M>(acc, out + int64_t(crow) * (L * M), lane, ring);
                 zero_tile<L, M>(acc);
             }
         }
