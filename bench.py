@@ -360,6 +360,45 @@ def l2_gather_ceiling(sa, torch, w, tensor, ops, dev, stream):
                                     "ms": min(r["ms"] for r in tma), "sweep": tma}}
 
 
+def nest_sample(w, target_nnz=4_000_000, seed=7):
+    """Time the paper's scheduled loop nest of the chain on the host cores (oracle/nests.c: fp64, OpenMP over i), on
+    seeded random output slices / rows holding about target_nnz nonzeros.  The sort into compressed storage is not
+    timed (the GPU figure excludes the build as well).  Returns None for chains without a nest there."""
+    import collections
+    from oracle import nests
+    import oracle
+    if w.expr not in ("spttm_ttm3", "spttm_ttm4", "ttmc3", "sddmm_spmm", "spmm_gemm"):
+        return None
+    I = int(w.dims[0])
+    i = w.coords[:, 0]
+    counts = np.bincount(i, minlength=I)
+    rs = np.random.RandomState(seed)
+    cand = rs.permutation(I)
+    cand = cand[counts[cand] <= max(1, target_nnz // 4)]           # one slice must not dominate the sample
+    csum = np.cumsum(counts[cand])
+    n_sel = min(int(np.searchsorted(csum, target_nnz, side="left")) + 1, cand.shape[0])
+    sel = np.sort(cand[:n_sel])
+    remap = np.full(I, -1, dtype=np.int64)
+    remap[sel] = np.arange(n_sel)
+    keep = remap[i] >= 0
+    coords = w.coords[keep].copy()
+    coords[:, 0] = remap[coords[:, 0]]
+    dense = list(w.dense)
+    if w.expr in ("sddmm_spmm", "ttmc3"):
+        dense[0] = np.ascontiguousarray(dense[0][sel])             # the operand indexed by i
+    Sub = collections.namedtuple("Sub", "expr dims coords vals dense")
+    sub = Sub(w.expr, (n_sel,) + tuple(int(d) for d in w.dims[1:]), coords, w.vals[keep], dense)
+    run = nests.prepare(sub, order="left")      # (B.C).D: its cost follows the sampled rows (C.D would be formed for all J)
+    run()
+    t0 = time.perf_counter()
+    run()
+    dt = time.perf_counter() - t0
+    nnz_sel = int(keep.sum())
+    return {"value": nnz_sel / dt / 1e9, "unit": "GNNZ/s", "cores": oracle.max_threads(), "kind": "paper's scheduled nest (fp64)",
+            "sample": "%d of %d output slices/rows (seeded random among those with <= %d nonzeros), %d of %d nonzeros"
+                      % (n_sel, I, max(1, target_nnz // 4), nnz_sel, int(w.nnz))}
+
+
 def aggregate_throughput(nnz_per_rank, world, ms_per_step):
     """Whole-job GNNZ/s of ``world`` independent replicas that all finish within ms_per_step."""
     return world * nnz_per_rank / (ms_per_step * 1e-3) / 1e9
@@ -623,6 +662,9 @@ def main():
                     done[cfg] = cb
                 r["cpu_baseline"] = done[cfg]
             line["cpu_baseline"] = done[args.workload]
+            nest = nest_sample(kept[args.workload])
+            if nest is not None:
+                line["cpu_scheduled_nest"] = nest
         if all_configs:
             line["per_config"] = records
         print(json.dumps(line), flush=True)

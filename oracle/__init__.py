@@ -4,6 +4,9 @@ TEST INFRASTRUCTURE ONLY.  The oracle evaluates each contraction chain as its un
 Einsum definition over COO input with fp64 accumulation (Table of kernels, Section 6 of
 the paper); the product code never imports this package.  ``liboracle.so`` is compiled
 from ``oracle.c`` by :func:`build` (plain ``gcc -O2 -fopenmp``).
+
+``oracle.nests`` (``nests.c``) holds a second CPU evaluation, the paper's scheduled loop nests over compressed
+storage; the tests hold the two against each other and bench.py times both.
 """
 import ctypes
 import os
