@@ -272,3 +272,166 @@ int nest_ttmc3(int64_t S, const int32_t *slice_i, const int64_t *pos1, const int
     free(copies);
     return bad ? -1 : 0;
 }
+
+/* Kernel 2 <SDDMM,SpMM,GEMM>, two-level nest of the Table of kernels:
+ *   i < T(l) ; j' < t ; k: t += B(i,j) C(i,k) D(j,k) , l: T(l) += t E(j,l) > , l,m: A(i,m) += T(l) F(l,m) >.
+ * A (I x M) must be zero on entry. */
+int nest_sddmm_spmm_gemm(int64_t I, const int64_t *pos1, const int32_t *crd1, const float *vals, int64_t K, int64_t L, int64_t M,
+                         const float *C, const float *D, const float *E, const float *F, double *A, int threads)
+{
+    set_threads(threads);
+    int bad = 0;
+    #pragma omp parallel
+    {
+        double *T = (double *)malloc(sizeof(double) * (size_t)L);
+        if (!T) {
+            #pragma omp atomic write
+            bad = 1;
+        }
+        #pragma omp barrier
+        if (!bad) {
+            #pragma omp for schedule(dynamic, 64)
+            for (int64_t i = 0; i < I; ++i) {
+                const float *Ci = C + i * K;
+                for (int64_t l = 0; l < L; ++l) T[l] = 0.0;
+                for (int64_t p = pos1[i]; p < pos1[i + 1]; ++p) {                  /* j' */
+                    const int64_t j = crd1[p];
+                    const double b = (double)vals[p];
+                    const float *Dj = D + j * K, *Ej = E + j * L;
+                    double t = 0.0;
+                    for (int64_t k = 0; k < K; ++k) t += b * (double)Ci[k] * (double)Dj[k];
+                    for (int64_t l = 0; l < L; ++l) T[l] += t * (double)Ej[l];
+                }
+                double *Ai = A + i * M;
+                for (int64_t l = 0; l < L; ++l) {
+                    const double tl = T[l];
+                    const float *Fl = F + l * M;
+                    for (int64_t m = 0; m < M; ++m) Ai[m] += tl * (double)Fl[m];
+                }
+            }
+        }
+        free(T);
+    }
+    return bad ? -1 : 0;
+}
+
+/* Kernel 3 <SpMMH,GEMM>, nest  i < T(l) ; j',l: T(l) += B(i,j) C(j,l) D(j,l) , l,m: A(i,m) += T(l) E(l,m) >.
+ * A (I x M) must be zero on entry. */
+int nest_spmmh_gemm(int64_t I, const int64_t *pos1, const int32_t *crd1, const float *vals, int64_t L, int64_t M,
+                    const float *C, const float *D, const float *E, double *A, int threads)
+{
+    set_threads(threads);
+    int bad = 0;
+    #pragma omp parallel
+    {
+        double *T = (double *)malloc(sizeof(double) * (size_t)L);
+        if (!T) {
+            #pragma omp atomic write
+            bad = 1;
+        }
+        #pragma omp barrier
+        if (!bad) {
+            #pragma omp for schedule(dynamic, 64)
+            for (int64_t i = 0; i < I; ++i) {
+                for (int64_t l = 0; l < L; ++l) T[l] = 0.0;
+                for (int64_t p = pos1[i]; p < pos1[i + 1]; ++p) {                  /* j' */
+                    const int64_t j = crd1[p];
+                    const double b = (double)vals[p];
+                    const float *Cj = C + j * L, *Dj = D + j * L;
+                    for (int64_t l = 0; l < L; ++l) T[l] += b * (double)Cj[l] * (double)Dj[l];
+                }
+                double *Ai = A + i * M;
+                for (int64_t l = 0; l < L; ++l) {
+                    const double tl = T[l];
+                    const float *El = E + l * M;
+                    for (int64_t m = 0; m < M; ++m) Ai[m] += tl * (double)El[m];
+                }
+            }
+        }
+        free(T);
+    }
+    return bad ? -1 : 0;
+}
+
+/* Kernel 8 <MTTKRP,GEMM>, nest
+ *   i < T(r) ; j' < t(r) ; k',r: t(r) += B(i,j,k) D(k,r) , r: T(r) += t(r) C(j,r) > , r,m: A(i,m) += T(r) E(r,m) >.
+ * A (I x M) must be zero on entry. */
+int nest_mttkrp_gemm(int64_t S, const int32_t *slice_i, const int64_t *pos1, const int32_t *crd1, const int64_t *pos2,
+                     const int32_t *crd2, const float *vals, int64_t R, int64_t M, const float *C, const float *D,
+                     const float *E, double *A, int threads)
+{
+    set_threads(threads);
+    int bad = 0;
+    #pragma omp parallel
+    {
+        double *t = (double *)malloc(sizeof(double) * (size_t)(2 * R));
+        double *T = t ? t + R : NULL;
+        if (!t) {
+            #pragma omp atomic write
+            bad = 1;
+        }
+        #pragma omp barrier
+        if (!bad) {
+            #pragma omp for schedule(dynamic, 4)
+            for (int64_t s = 0; s < S; ++s) {
+                for (int64_t r = 0; r < R; ++r) T[r] = 0.0;
+                for (int64_t f = pos1[s]; f < pos1[s + 1]; ++f) {                  /* j' */
+                    const float *Cj = C + (int64_t)crd1[f] * R;
+                    for (int64_t r = 0; r < R; ++r) t[r] = 0.0;
+                    for (int64_t p = pos2[f]; p < pos2[f + 1]; ++p) {              /* k' */
+                        const double b = (double)vals[p];
+                        const float *Dk = D + (int64_t)crd2[p] * R;
+                        for (int64_t r = 0; r < R; ++r) t[r] += b * (double)Dk[r];
+                    }
+                    for (int64_t r = 0; r < R; ++r) T[r] += t[r] * (double)Cj[r];
+                }
+                double *Ai = A + (int64_t)slice_i[s] * M;
+                for (int64_t r = 0; r < R; ++r) {
+                    const double tr = T[r];
+                    const float *Er = E + r * M;
+                    for (int64_t m = 0; m < M; ++m) Ai[m] += tr * (double)Er[m];
+                }
+            }
+        }
+        free(t);
+    }
+    return bad ? -1 : 0;
+}
+
+/* Kernel 7 <SpTTM,SpTTM>, nest  i, j' < T(l) ; k',l: T(l) += B(i,j,k) C(k,l) , l,m: A(f,m) += T(l) D(l,m) >  with one
+ * output row per level-1 fiber f = (i,j), in storage order (the output keeps B's (i,j) pattern).
+ * A (F x M) must be zero on entry. */
+int nest_spttm_spttm(int64_t F, const int64_t *pos2, const int32_t *crd2, const float *vals, int64_t L, int64_t M,
+                     const float *C, const float *D, double *A, int threads)
+{
+    set_threads(threads);
+    int bad = 0;
+    #pragma omp parallel
+    {
+        double *T = (double *)malloc(sizeof(double) * (size_t)L);
+        if (!T) {
+            #pragma omp atomic write
+            bad = 1;
+        }
+        #pragma omp barrier
+        if (!bad) {
+            #pragma omp for schedule(dynamic, 64)
+            for (int64_t f = 0; f < F; ++f) {                                      /* i, j' */
+                for (int64_t l = 0; l < L; ++l) T[l] = 0.0;
+                for (int64_t p = pos2[f]; p < pos2[f + 1]; ++p) {                  /* k' */
+                    const double b = (double)vals[p];
+                    const float *Ck = C + (int64_t)crd2[p] * L;
+                    for (int64_t l = 0; l < L; ++l) T[l] += b * (double)Ck[l];
+                }
+                double *Af = A + f * M;
+                for (int64_t l = 0; l < L; ++l) {
+                    const double tl = T[l];
+                    const float *Dl = D + l * M;
+                    for (int64_t m = 0; m < M; ++m) Af[m] += tl * (double)Dl[m];
+                }
+            }
+        }
+        free(T);
+    }
+    return bad ? -1 : 0;
+}

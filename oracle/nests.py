@@ -157,18 +157,79 @@ def spmm_gemm(pos, crd, vals, C, D, order="left", threads=0):
     return A
 
 
+def sddmm_spmm_gemm(pos, crd, vals, C, D, E, F, threads=0):
+    C, Cp = _arr(C, np.float32)
+    D, Dp = _arr(D, np.float32)
+    E, Ep = _arr(E, np.float32)
+    F, Fp = _arr(F, np.float32)
+    I, K, L, M = C.shape[0], C.shape[1], E.shape[1], F.shape[1]
+    A = np.zeros((I, M), dtype=np.float64)
+    keep = [_arr(pos, np.int64), _arr(crd, np.int32), _arr(vals, np.float32)]
+    _check(_load().nest_sddmm_spmm_gemm(_i64(I), *[k[1] for k in keep], _i64(K), _i64(L), _i64(M), Cp, Dp, Ep, Fp,
+                                        A.ctypes.data_as(_p), ctypes.c_int(threads)))
+    return A
+
+
+def spmmh_gemm(pos, crd, vals, C, D, E, threads=0):
+    C, Cp = _arr(C, np.float32)
+    D, Dp = _arr(D, np.float32)
+    E, Ep = _arr(E, np.float32)
+    I, L, M = pos.shape[0] - 1, C.shape[1], E.shape[1]
+    A = np.zeros((I, M), dtype=np.float64)
+    keep = [_arr(pos, np.int64), _arr(crd, np.int32), _arr(vals, np.float32)]
+    _check(_load().nest_spmmh_gemm(_i64(I), *[k[1] for k in keep], _i64(L), _i64(M), Cp, Dp, Ep, A.ctypes.data_as(_p),
+                                   ctypes.c_int(threads)))
+    return A
+
+
+def mttkrp_gemm(levels, vals, I, C, D, E, threads=0):
+    (_, s_i), (pos1, crd1), (pos2, crd2) = levels
+    C, Cp = _arr(C, np.float32)
+    D, Dp = _arr(D, np.float32)
+    E, Ep = _arr(E, np.float32)
+    R, M = C.shape[1], E.shape[1]
+    A = np.zeros((I, M), dtype=np.float64)
+    keep = [_arr(s_i, np.int32), _arr(pos1, np.int64), _arr(crd1, np.int32), _arr(pos2, np.int64), _arr(crd2, np.int32),
+            _arr(vals, np.float32)]
+    _check(_load().nest_mttkrp_gemm(_i64(keep[0][0].shape[0]), *[k[1] for k in keep], _i64(R), _i64(M), Cp, Dp, Ep,
+                                    A.ctypes.data_as(_p), ctypes.c_int(threads)))
+    return A
+
+
+def spttm_spttm(levels, vals, C, D, threads=0):
+    """One output row per (i,j) fiber, in lexicographic order of the pairs."""
+    (_, _s), (_pos1, crd1), (pos2, crd2) = levels
+    C, Cp = _arr(C, np.float32)
+    D, Dp = _arr(D, np.float32)
+    L, M = C.shape[1], D.shape[1]
+    F = crd1.shape[0]
+    A = np.zeros((F, M), dtype=np.float64)
+    keep = [_arr(pos2, np.int64), _arr(crd2, np.int32), _arr(vals, np.float32)]
+    _check(_load().nest_spttm_spttm(_i64(F), *[k[1] for k in keep], _i64(L), _i64(M), Cp, Dp, A.ctypes.data_as(_p),
+                                    ctypes.c_int(threads)))
+    return A
+
+
 def prepare(w, order="left", threads=0):
     """Builds the compressed storage of the workload's sparse operand and returns a function that runs the chain's
     nest on it (so that a caller can time the nest without the sort)."""
-    if w.expr in ("spttm_ttm3", "spttm_ttm4", "ttmc3"):
+    if w.expr in ("spttm_ttm3", "spttm_ttm4", "ttmc3", "mttkrp_gemm", "spttm_spttm"):
         levels, v = csf_from_coo(w.coords, w.vals)
+        if w.expr == "mttkrp_gemm":
+            return lambda: mttkrp_gemm(levels, v, int(w.dims[0]), *w.dense, threads=threads)
+        if w.expr == "spttm_spttm":
+            return lambda: spttm_spttm(levels, v, *w.dense, threads=threads)
         if w.expr == "spttm_ttm3":
             return lambda: spttm_ttm3(levels, v, int(w.dims[0]), *w.dense, threads=threads)
         if w.expr == "spttm_ttm4":
             return lambda: spttm_ttm4(levels, v, int(w.dims[0]), *w.dense, threads=threads)
         return lambda: ttmc3(levels, v, *w.dense, threads=threads)
-    if w.expr in ("sddmm_spmm", "spmm_gemm"):
+    if w.expr in ("sddmm_spmm", "spmm_gemm", "sddmm_spmm_gemm", "spmmh_gemm"):
         pos, crd, v = csr_from_coo(w.coords, w.vals, int(w.dims[0]))
+        if w.expr == "sddmm_spmm_gemm":
+            return lambda: sddmm_spmm_gemm(pos, crd, v, *w.dense, threads=threads)
+        if w.expr == "spmmh_gemm":
+            return lambda: spmmh_gemm(pos, crd, v, *w.dense, threads=threads)
         if w.expr == "sddmm_spmm":
             return lambda: sddmm_spmm(pos, crd, v, *w.dense, threads=threads)
         return lambda: spmm_gemm(pos, crd, v, *w.dense, order=order, threads=threads)

@@ -20,7 +20,7 @@ def _close(A, A_ref, S, what):
     assert (np.abs(A - A_ref) <= 1e-12 * S).all(), what
 
 
-@pytest.mark.parametrize("cfg", [1, 2, 3, 4, 5, 6])
+@pytest.mark.parametrize("cfg", [1, 2, 3, 4, 5, 6, 7, 8, 9, 10])
 def test_nests_agree_with_the_definition_on_the_mini_configurations(cfg):
     w = configs.make(cfg, "mini")
     A_ref, S = oracle.evaluate(w)
