@@ -216,12 +216,15 @@ ttm4_slice_kernel(const sa_item *__restrict__ items, int64_t n_items, const int3
 //     nonzero per group and step (index/value pairs eight per load and one load ahead, eight row gathers in
 //     flight); the end-of-fiber bit travels in the sign bit of the index and parks t(f; :) in the fiber's own slot
 //     of the warp's shared-memory tile, so the parked rows end up in fiber order without any bookkeeping.
-//   Phase B (Q2):  T2(m,n) += D(k_f, m) t(f; n) over the fibers of each subtree, in order; the 16 x 16 tile is
-//     spread over the warp (lane = two rows m, four columns n), control flow is uniform, and the tile is stored
-//     (1 KB, contiguous) when the subtree's last fiber has been added.
-// Against the order-3 kernel on the same subtrees this drops the per-unit pipeline drains and the padded
-// tensor-core groups: 16.7 M outer products of 256 FMAs are cheap on the ALUs next to 100 M row gathers.
-constexpr int SUB_SMEM = SA_WARPS_PER_CTA * SA_SUB_MAX_F3 * R * int(sizeof(float));   // 32 KB
+//   Phase B (Q2):  T2(m,n) += D(k_f, m) t(f; n) over the fibers of each subtree, eight fibers at a time as
+//     T2 += Dg^T (16 x 8) . t (8 x 16) on tensor cores (m16n8k8 TF32, both operands split into a high and a low part,
+//     three products): a lane loads four values of D and four of the parked rows per group, where one fiber per step
+//     on the ALUs cost it six values per fiber, and the load/store pipe is what bounds this kernel.  Fibers past
+//     the end of a subtree enter as zero rows.  The 1 KB tile is stored when the subtree's last group is in.
+// Against the order-3 kernel on the same subtrees this drops the per-unit pipeline drains, the cross-stream
+// bookkeeping of parked rows and the slice-wide accumulator tile.
+constexpr int SUB_RS = R + 8;          // floats per parked row: t(16), the fiber's k, pad; rows t and t + 1 land 8 banks apart
+constexpr int SUB_SMEM = SA_WARPS_PER_CTA * SA_SUB_MAX_F3 * SUB_RS * int(sizeof(float));   // 48 KB
 
 // CONTIG: both factor matrices are stored without padding (leading dimension 16), so a row offset is a shift.
 template <bool CONTIG>
@@ -240,15 +243,18 @@ ttm4_subtree_kernel(const sa_item *__restrict__ items, int64_t n_items, const in
                                 it.row_end - it.out_row <= SA_SUB_MAX_ROWS && it.row_end <= lim.n_subtrees && it.p0 >= 0 && it.p1 <= lim.nnz,
                 73, idx))
         return;
-    float *pk = sub_smem + warp * (SA_SUB_MAX_F3 * R);
+    float *pk = sub_smem + warp * (SA_SUB_MAX_F3 * SUB_RS);
     // row offsets in 32-bit arithmetic (the launcher checks rows * ld < 2^31)
     const uint32_t ld_d = CONTIG ? uint32_t(R) : uint32_t(ldd), ld_e = CONTIG ? uint32_t(R) : uint32_t(lde);
     const int nf3 = it.f1 - it.f0;
-    // rows of D the item's fibers need in phase B (requested now, used after phase A)
+    // the k of the item's fibers (requested now; their D row offsets are parked beside the rows of t)
     static_assert(SA_SUB_MAX_F3 <= 64, "two index registers per lane");
     int kk0 = lane < nf3 ? __ldg(crd_k + it.f0 + lane) : 0;
     int kk1 = lane + 32 < nf3 ? __ldg(crd_k + it.f0 + 32 + lane) : 0;
     if (!SA_CHK(lim.status, uint32_t(kk0) < lim.d_rows && uint32_t(kk1) < lim.d_rows, 74, kk0)) kk0 = kk1 = 0;
+    // word 16 of a fiber's parked row: the element offset of its row of D
+    pk[lane * SUB_RS + R] = __uint_as_float(uint32_t(kk0) * ld_d);
+    pk[(lane + 32) * SUB_RS + R] = __uint_as_float(uint32_t(kk1) * ld_d);
     {   // ---- phase A
         const int g = lane >> 2, l = lane & 3;
         // shares of the eight groups: whole fibers, cut where the nonzero count passes the next eighth of the item
@@ -309,7 +315,7 @@ ttm4_subtree_kernel(const sa_item *__restrict__ items, int64_t n_items, const in
                     acc.w = fmaf(vs[u], e[u].w, acc.w);
                 }
                 if (xs[u] < 0) {                                      // last nonzero of fiber it.f0 + slot
-                    if (SA_CHK(lim.status, slot >= 0 && slot < nf3, 77, slot)) *reinterpret_cast<float4 *>(pk + slot * R + 4 * l) = acc;
+                    if (SA_CHK(lim.status, slot >= 0 && slot < nf3, 77, slot)) *reinterpret_cast<float4 *>(pk + slot * SUB_RS + 4 * l) = acc;
                     acc = make_float4(0.f, 0.f, 0.f, 0.f);
                     ++slot;
                 }
@@ -317,46 +323,51 @@ ttm4_subtree_kernel(const sa_item *__restrict__ items, int64_t n_items, const in
         }
     }
     __syncwarp();
-    {   // ---- phase B
-        const int mp = lane >> 2, nq = lane & 3;
+    {   // ---- phase B: per subtree, eight fibers at a time, T2 += D(k_f, :)^T (16 x 8) . t (8 x 16) on tensor cores
+        const int g = lane >> 2, t = lane & 3;
         const int nr = it.row_end - it.out_row;
         const int my_end = lane < nr ? __ldg(pos2 + it.out_row + lane + 1) - it.f0 : 0x7fffffff;   // local end of subtree `lane`
-        int r = 0, fe = __shfl_sync(SA_FULL_MASK, my_end, 0);
-        float4 a0 = make_float4(0.f, 0.f, 0.f, 0.f), a1 = a0;
-        // D(k_f, 2mp..2mp+1) of eight fibers at a time, the next eight requested before the current eight are used
-        auto load_d = [&](int f0, float2 (&d)[8]) {
-            const int ks = f0 < 32 ? kk0 : kk1;
+        int fbeg = 0;
+        for (int r = 0; r < nr; ++r) {
+            const int fend = min(__shfl_sync(SA_FULL_MASK, my_end, r), nf3);
+            float acc[2][4];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                const int k = __shfl_sync(SA_FULL_MASK, ks, (f0 + u) & 31);
-                d[u] = sa_ldg2(D + (uint32_t(k) * ld_d + 2u * mp));
-            }
-        };
-        float2 d[8], dn[8];
-        load_d(0, d);
-        for (int f0 = 0; f0 < nf3; f0 += 8) {
-            if (f0 + 8 < nf3) load_d(f0 + 8, dn);
+            for (int nt = 0; nt < 2; ++nt)
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                if (f0 + u < nf3) {
-                    const float4 tt = *reinterpret_cast<const float4 *>(pk + (f0 + u) * R + 4 * nq);
-                    a0.x = fmaf(d[u].x, tt.x, a0.x); a0.y = fmaf(d[u].x, tt.y, a0.y);
-                    a0.z = fmaf(d[u].x, tt.z, a0.z); a0.w = fmaf(d[u].x, tt.w, a0.w);
-                    a1.x = fmaf(d[u].y, tt.x, a1.x); a1.y = fmaf(d[u].y, tt.y, a1.y);
-                    a1.z = fmaf(d[u].y, tt.z, a1.z); a1.w = fmaf(d[u].y, tt.w, a1.w);
-                    if (f0 + u + 1 == fe) {                           // the subtree's last fiber
-                        float *dst = T2 + int64_t(it.out_row + r) * T2F + (2 * mp) * R + 4 * nq;
-                        *reinterpret_cast<float4 *>(dst) = a0;
-                        *reinterpret_cast<float4 *>(dst + R) = a1;
-                        a0 = make_float4(0.f, 0.f, 0.f, 0.f);
-                        a1 = a0;
-                        ++r;
-                        fe = __shfl_sync(SA_FULL_MASK, my_end, r & 31);
-                    }
+                for (int x = 0; x < 4; ++x) acc[nt][x] = 0.f;
+            for (int fg = fbeg; fg < fend; fg += 8) {
+                // fibers fg + t and fg + t + 4 of the group; past the subtree's end they count as zero rows
+                const bool va = fg + t < fend, vb = fg + t + 4 < fend;
+                const float *ra = pk + (va ? fg + t : fbeg) * SUB_RS;
+                const float *rb = pk + (vb ? fg + t + 4 : fbeg) * SUB_RS;
+                const float *da = D + __float_as_uint(ra[R]) + g;
+                const float *db = D + __float_as_uint(rb[R]) + g;
+                float av[4];
+                av[0] = va ? __ldg(da) : 0.f;
+                av[1] = va ? __ldg(da + 8) : 0.f;
+                av[2] = vb ? __ldg(db) : 0.f;
+                av[3] = vb ? __ldg(db + 8) : 0.f;
+                uint32_t ah[4], al[4];
+#pragma unroll
+                for (int x = 0; x < 4; ++x) split_tf32(av[x], ah[x], al[x]);
+#pragma unroll
+                for (int nt = 0; nt < 2; ++nt) {
+                    uint32_t bh[2], bl[2];
+                    split_tf32(va ? ra[8 * nt + g] : 0.f, bh[0], bl[0]);
+                    split_tf32(vb ? rb[8 * nt + g] : 0.f, bh[1], bl[1]);
+                    mma_m16n8k8_tf32(acc[nt], al, bh);
+                    mma_m16n8k8_tf32(acc[nt], ah, bl);
+                    mma_m16n8k8_tf32(acc[nt], ah, bh);
                 }
             }
+            // element (m, n) of the subtree's temporary: m = g and g + 8, n = 8 nt + 2 t (+ 1)
+            float *dst = T2 + int64_t(it.out_row + r) * T2F + 2 * t;
 #pragma unroll
-            for (int u = 0; u < 8; ++u) d[u] = dn[u];
+            for (int nt = 0; nt < 2; ++nt) {
+                *reinterpret_cast<float2 *>(dst + g * R + 8 * nt) = make_float2(acc[nt][0], acc[nt][1]);
+                *reinterpret_cast<float2 *>(dst + (g + 8) * R + 8 * nt) = make_float2(acc[nt][2], acc[nt][3]);
+            }
+            fbeg = fend;
         }
     }
 }
