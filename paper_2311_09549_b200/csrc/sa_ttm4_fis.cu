@@ -212,7 +212,7 @@ ttm4_slice_kernel(const sa_item *__restrict__ items, int64_t n_items, const int3
 // Pass 1 on whole (i,j) subtrees (tensors whose subtrees are all small: the usual case, a subtree holds a few
 // dozen nonzeros).  One warp per item = a range of consecutive subtrees with at most SA_SUB_MAX_F3 level-2 fibers.
 //   Phase A (Q1):  t(f; n) = sum_o B(f; o) E(o,n) for every level-2 fiber f = (i,j,k) of the item.  Four lanes own a
-//     row of E as one float4 each, so the warp's eight lane groups walk separate shares of the item's fibers, one
+//     row of E as one float4 each, so the warp's eight lane groups walk equal shares of the item's nonzeros, one
 //     nonzero per group and step (index/value pairs eight per load and one load ahead, eight row gathers in
 //     flight); the end-of-fiber bit travels in the sign bit of the index and parks t(f; :) in the fiber's own slot
 //     of the warp's shared-memory tile, so the parked rows end up in fiber order without any bookkeeping.
@@ -257,22 +257,22 @@ ttm4_subtree_kernel(const sa_item *__restrict__ items, int64_t n_items, const in
     pk[(lane + 32) * SUB_RS + R] = __uint_as_float(uint32_t(kk1) * ld_d);
     {   // ---- phase A
         const int g = lane >> 2, l = lane & 3;
-        // shares of the eight groups: whole fibers, cut where the nonzero count passes the next eighth of the item
-        // (fiber f belongs to the groups before g when it starts before p0 + g len / 8)
+        // shares of the eight groups: equal counts of nonzeros, whatever the fiber boundaries (whole-fiber shares left
+        // the longest group 1.6 times the mean, and every group runs as many steps as the longest).  A fiber cut by
+        // a share boundary gets its parts added together after the loop.
         const int s0 = lane < nf3 ? __ldg(pos3 + it.f0 + lane) : 0x7fffffff;
         const int s1 = lane + 32 < nf3 ? __ldg(pos3 + it.f0 + 32 + lane) : 0x7fffffff;
-        int fa = it.f0, fb = it.f1;
-#pragma unroll
-        for (int q = 1; q < 8; ++q) {
-            const int target = it.p0 + int(int64_t(it.p1 - it.p0) * q / 8);
-            const int cnt = __popc(__ballot_sync(SA_FULL_MASK, s0 < target)) + __popc(__ballot_sync(SA_FULL_MASK, s1 < target));
-            if (g == q) fa = it.f0 + cnt;
-            if (g + 1 == q) fb = it.f0 + cnt;
-        }
-        const int ga = __ldg(pos3 + fa), gb = __ldg(pos3 + fb);
+        const int share = (it.p1 - it.p0 + 7) >> 3;
+        const int ga = min(it.p0 + g * share, it.p1), gb = min(ga + share, it.p1);
         const int mylen = gb - ga;
-        const int maxlen = __reduce_max_sync(SA_FULL_MASK, mylen);
-        int slot = fa - it.f0;
+        const int maxlen = share;
+        int slot = 0;                                   // the fiber that holds nonzero ga: the last one starting at or before it
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const int target = min(it.p0 + q * share, it.p1);
+            const int cnt = __popc(__ballot_sync(SA_FULL_MASK, s0 <= target)) + __popc(__ballot_sync(SA_FULL_MASK, s1 <= target));
+            if (g == q) slot = cnt - 1;
+        }
         auto fetch1 = [&](int q, int &x, float &v) {
             x = 0;
             v = 0.f;
@@ -295,31 +295,44 @@ ttm4_subtree_kernel(const sa_item *__restrict__ items, int64_t n_items, const in
             const int x[2] = {xn[0], xn[1]};
             const float v[2] = {vn[0], vn[1]};
             fetch(c + 8, xn, vn);
-            int xs[8];
-            float vs[8];
-            float4 e[8];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                xs[u] = __shfl_sync(SA_FULL_MASK, x[u >> 2], u & 3, 4);
-                vs[u] = __shfl_sync(SA_FULL_MASK, v[u >> 2], u & 3, 4);
-                uint32_t o = uint32_t(xs[u]) & 0x7fffffffu;
-                if (!SA_CHK(lim.status, o < lim.e_rows, 76, o)) o = 0u;
-                e[u] = sa_ldg4(E + (o * ld_e + 4u * l));
-            }
+            for (int h = 0; h < 2; ++h) {               // two batches of four row gathers
+                int xs[4];
+                float vs[4];
+                float4 e[4];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                if (c + u < mylen) {
-                    acc.x = fmaf(vs[u], e[u].x, acc.x);
-                    acc.y = fmaf(vs[u], e[u].y, acc.y);
-                    acc.z = fmaf(vs[u], e[u].z, acc.z);
-                    acc.w = fmaf(vs[u], e[u].w, acc.w);
+                for (int u = 0; u < 4; ++u) {
+                    xs[u] = __shfl_sync(SA_FULL_MASK, x[h], u, 4);
+                    vs[u] = __shfl_sync(SA_FULL_MASK, v[h], u, 4);
+                    uint32_t o = uint32_t(xs[u]) & 0x7fffffffu;
+                    if (!SA_CHK(lim.status, o < lim.e_rows, 76, o)) o = 0u;
+                    e[u] = sa_ldg4(E + (o * ld_e + 4u * l));
                 }
-                if (xs[u] < 0) {                                      // last nonzero of fiber it.f0 + slot
-                    if (SA_CHK(lim.status, slot >= 0 && slot < nf3, 77, slot)) *reinterpret_cast<float4 *>(pk + slot * SUB_RS + 4 * l) = acc;
-                    acc = make_float4(0.f, 0.f, 0.f, 0.f);
-                    ++slot;
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    if (c + 4 * h + u < mylen) {
+                        acc.x = fmaf(vs[u], e[u].x, acc.x);
+                        acc.y = fmaf(vs[u], e[u].y, acc.y);
+                        acc.z = fmaf(vs[u], e[u].z, acc.z);
+                        acc.w = fmaf(vs[u], e[u].w, acc.w);
+                    }
+                    if (xs[u] < 0) {                                  // last nonzero of fiber it.f0 + slot
+                        if (SA_CHK(lim.status, slot >= 0 && slot < nf3, 77, slot)) *reinterpret_cast<float4 *>(pk + slot * SUB_RS + 4 * l) = acc;
+                        acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                        ++slot;
+                    }
                 }
             }
+        }
+        // the open part of a cut fiber is added to the fiber's row once every group has stored the rows it closed
+        __syncwarp();
+        // (a sum left open is what the accumulator holds; after a fiber's last nonzero it is zero and nothing is added)
+        if ((acc.x != 0.f || acc.y != 0.f || acc.z != 0.f || acc.w != 0.f) && SA_CHK(lim.status, slot >= 0 && slot < nf3, 77, slot)) {
+            float *row = pk + slot * SUB_RS + 4 * l;
+            atomicAdd(row, acc.x);
+            atomicAdd(row + 1, acc.y);
+            atomicAdd(row + 2, acc.z);
+            atomicAdd(row + 3, acc.w);
         }
     }
     __syncwarp();
