@@ -52,10 +52,10 @@ NCU_TRAFFIC = {
     (5, "fused"): {"kernel": "ttm4_fused_kernel (94 % of the step; counters of the quarter-size case x 4)",
                    "source": "paper_2311_09549_b200/csrc/sa_ttm4.cu", "sha256": "77b9b58137c8e565f84a5ffd8762e5448c910f5befc50c3838442ae6007d0823",
                    "dram_bytes": 4 * 424084480, "profile": "profiles/ttm4_kernels_cfg5.md"},
-    (5, "fissioned"): {"kernel": "ttm4_subtree_kernel (pass 1 on the small subtrees, 53 % of the step; counters of the "
+    (5, "fissioned"): {"kernel": "ttm4_subtree_kernel (pass 1 on the small subtrees, 51 % of the step; counters of the "
                                  "quarter-size case x 4)",
-                       "source": "paper_2311_09549_b200/csrc/sa_ttm4_fis.cu", "sha256": "d2e6abec2db097615441195314bfa89659946dee35f3ba45c511bdec9c0f17bf",
-                       "dram_bytes": 4 * 662830848, "profile": "profiles/ttm4_kernels_cfg5.md"},
+                       "source": "paper_2311_09549_b200/csrc/sa_ttm4_fis.cu", "sha256": "be9575594a14a3633f6a12fba75381f08305534e694d350516c738ba12c2d61b",
+                       "dram_bytes": 4 * 663252480, "profile": "profiles/ttm4_kernels_cfg5.md"},
     10: {"kernel": "fiber_spmm_kernel<32> (99 % of the step)", "source": "paper_2311_09549_b200/csrc/sa_spmm_gemm.cu",
          "sha256": "a7d3ddb4c4f3e2c41bc5f803c06e42250d24443649e1f4c918744c74fbb8b39f",
          "dram_bytes": 955089920, "profile": "profiles/fiber_spmm_kernel_w10.md"},
