@@ -486,8 +486,10 @@ void build_ttm4(sa_tensor *t, sa_worklist &wl, sa_worklist &wl_items, sa_worklis
 
 // Rows of a sparse matrix given by its pos array: row ranges of about target_nnz nonzeros (at most max_rows rows); rows longer than
 // long_thresh are cut into pieces of `piece` nonzeros whose partial rows the fix-up kernel sums.
+// quarter_rows: a range item also records the rows that hold its nonzeros p0 + q ceil((p1 - p0) / 4), q = 1, 2, 3
+// (fields f0, f1, pad), for kernels whose lane groups take equal counts of nonzeros rather than of rows.
 void build_rows(const std::vector<int64_t> &pos, int64_t I, sa_worklist &wl, int64_t target_nnz, int64_t max_rows,
-                int64_t long_thresh, int64_t piece)
+                int64_t long_thresh, int64_t piece, bool quarter_rows = false)
 {
     std::vector<sa_item> longs, ranges;
     int64_t r0 = 0;
@@ -496,6 +498,17 @@ void build_rows(const std::vector<int64_t> &pos, int64_t I, sa_worklist &wl, int
             sa_item it = empty_item();
             it.out_row = int32_t(r0); it.row_end = int32_t(r1);
             it.p0 = int32_t(pos[size_t(r0)]); it.p1 = int32_t(pos[size_t(r1)]);
+            if (quarter_rows) {
+                const int64_t share = (int64_t(it.p1) - it.p0 + 3) / 4;
+                int32_t rows[3];
+                for (int q = 1; q < 4; ++q) {
+                    const int64_t at = std::min<int64_t>(int64_t(it.p0) + q * share, it.p1);
+                    // the last row starting at or before `at`, inside the item
+                    int64_t r = (std::upper_bound(pos.begin() + r0, pos.begin() + r1 + 1, at) - pos.begin()) - 1;
+                    rows[q - 1] = int32_t(std::min<int64_t>(std::max<int64_t>(r, r0), r1 - 1));
+                }
+                it.f0 = rows[0]; it.f1 = rows[1]; it.pad = rows[2];
+            }
             ranges.push_back(it);
         }
         r0 = r1;
@@ -537,7 +550,7 @@ void sa_build_worklists(sa_tensor *t)
     if (t->fmt == SA_FMT_CSF && t->order == 3) {
         build_ttm3(t, t->wl_main);
         // kernel 7 walks the tensor as a sparse matrix whose rows are the (i,j) fibers
-        build_rows(t->pos[2], t->count[1], t->wl_aux, 1024, 4096, 4096, 2048);
+        build_rows(t->pos[2], t->count[1], t->wl_aux, 1024, 4096, 4096, 2048, true);
     }
     if (t->fmt == SA_FMT_CSF && t->order == 4) {
         build_ttm4(t, t->wl_main, t->wl_sub, t->wl_aux);

@@ -312,7 +312,8 @@ spmm_kernel(const sa_item *__restrict__ items, int64_t n_items, const int32_t *_
 // flight; index, end-of-fiber bit (sign bit) and value of a nonzero come as one 8-byte record (half the load
 // wavefronts of separate index, value and bit arrays, and the L1 pipe is what this kernel saturates first); the
 // bit closes the output row.
-// A piece of a long fiber (dest >= 0) is split over the groups by nonzeros and summed across them at the end.
+// A piece of a long fiber (dest >= 0) is split over the groups by nonzeros and summed across them at the end; a range
+// of whole fibers is split by nonzeros as well, and the parts of a fiber cut between two groups are added in order.
 template <int M>
 __global__ void __launch_bounds__(256)
 fiber_spmm_kernel(const sa_item *__restrict__ items, int64_t n_items, const int32_t *__restrict__ pos,
@@ -332,13 +333,18 @@ fiber_spmm_kernel(const sa_item *__restrict__ items, int64_t n_items, const int3
         ga = it.p0 + int(len * g / NG);
         gb = it.p0 + int(len * (g + 1) / NG);
     } else {
-        const int nr = it.row_end - it.out_row;
-        row = it.out_row + nr * g / NG;
-        ga = __ldg(pos + row);
-        gb = __ldg(pos + it.out_row + nr * (g + 1) / NG);
+        // equal counts of nonzeros per group, whatever the row boundaries: quarters of the item (the work list names
+        // the row each quarter starts in), two of them per group when there are two groups.  With equal counts of
+        // rows the longest group had 1.2 times the mean length, and a range of one long row was all one group's.
+        static_assert(NG == 4 || NG == 2, "quarter rows of the work list");
+        const int quarter = (it.p1 - it.p0 + 3) >> 2, share = quarter * (4 / NG), first = g * (4 / NG);
+        ga = min(it.p0 + g * share, it.p1);
+        gb = min(ga + share, it.p1);
+        row = first == 0 ? it.out_row : first == 1 ? it.f0 : first == 2 ? it.f1 : it.pad;
     }
     const int mylen = gb - ga;
     const int maxlen = __reduce_max_sync(SA_FULL_MASK, mylen);
+    bool open = false;                      // the group's last nonzero did not end its row
     auto fetch = [&](int c, int &x, float &v) {                      // lanes 0..7 of the group: nonzero ga + c + lane
         const int p = ga + c + (l & 7);
         x = 0;
@@ -376,10 +382,25 @@ fiber_spmm_kernel(const sa_item *__restrict__ items, int64_t n_items, const int3
                 acc.z = fmaf(vs[u], e[u].z, acc.z);
                 acc.w = fmaf(vs[u], e[u].w, acc.w);
             }
+            if (c + u < mylen) open = xs[u] >= 0;
             if (xs[u] < 0) {                                          // last nonzero of its fiber
                 if (SA_CHK(lim.status, uint32_t(row) < lim.out_rows, 63, row)) *reinterpret_cast<float4 *>(out + int64_t(row) * M + 4 * l) = acc;
                 acc = make_float4(0.f, 0.f, 0.f, 0.f);
                 ++row;
+            }
+        }
+    }
+    if (!piece) {
+        // A row cut by a share boundary was stored by the group that met its end; the groups before it add their
+        // parts now, one group after the other (a long row may have several), so that the sum has a fixed order.
+#pragma unroll
+        for (int s = 0; s < NG - 1; ++s) {
+            __syncwarp();
+            if (g == s && open && SA_CHK(lim.status, uint32_t(row) < lim.out_rows, 63, row)) {
+                float4 *dst = reinterpret_cast<float4 *>(out + int64_t(row) * M + 4 * l);
+                float4 o = __ldcg(dst);
+                o.x += acc.x; o.y += acc.y; o.z += acc.z; o.w += acc.w;
+                *dst = o;
             }
         }
     }

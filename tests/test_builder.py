@@ -388,12 +388,18 @@ def test_fiber_row_worklist_of_order3_csf_partitions_fibers_and_nonzeros():
     counts, items, fix = sa.sa_tensor_worklist(t.handle, 1)
     covered = np.zeros(coords.shape[0], dtype=np.int32)
     rows = np.zeros(n_fibers, dtype=np.int32)
-    for row, row_end, _, _, p0, p1, dest, _ in items:
+    for row, row_end, q1, q2, p0, p1, dest, q3 in items:
         if dest >= 0:
             assert row_end == row + 1 and pos[row] <= p0 < p1 <= pos[row + 1]
         else:
             assert (p0, p1) == (pos[row], pos[row_end])
             rows[row:row_end] += 1
+            # the rows in which the item's quarters (equal counts of nonzeros) start
+            share = -(-(p1 - p0) // 4)
+            for q, got in ((1, q1), (2, q2), (3, q3)):
+                at = min(p0 + q * share, p1)
+                want = min(int(np.searchsorted(pos, at, side="right")) - 1, row_end - 1)
+                assert got == want and row <= got < row_end, (row, row_end, q, got, want)
         covered[p0:p1] += 1
     assert (covered == 1).all()
     assert len(fix) == 1 and fix[0][2] == 3          # 5000 nonzeros in pieces of 2048
